@@ -1,0 +1,378 @@
+"""CPU oracle for the Bi-Mask per-layer sparse training step.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain restatement of the
+method that the CUDA path is checked against.  Only the test-suite, the smoke
+check and the benchmark's CPU-baseline leg may import it; the product path
+never does.  It shares no code with the CUDA path and imports nothing from the
+package.
+
+Notation follows the paper: W is I x J (output rows x input dim), B is the
+forward N:M mask (N:M along each row, Eq. 2 / Eq. 4), B-bar the backward mask
+(N:M along each column of the row-permuted matrix, Eq. 7 / Eq. 11), `perm` the
+row permutation vector of Eq. 10 (gather: Wp[k, :] = W[perm[k], :], 0-based).
+
+All arrays are numpy.  Floating-point products are done in float64.  Integer
+results (mask bits, packed indices, counts, the chosen permutation) are exact.
+
+Readings of points the paper leaves open (listed again in the design notes):
+  * blocks are the aligned, disjoint index ranges [g*M, (g+1)*M), 0-based;
+  * "Top(., N)" of Eq. 4 / Eq. 11 is applied as a rank: an element is kept when
+    fewer than N elements of its block beat it, where an element q beats m if
+    its magnitude is larger, or equal with q < m.  With distinct magnitudes
+    this is Eq. 4 / Eq. 11 verbatim; with ties it keeps exactly N (Eq. 2);
+  * magnitudes are compared on the fp32 weights through the integer key
+    bits(w) & 0x7fffffff (monotone in |w|, -0 == +0);
+  * in the backward mask only positions with a forward bit of 1 are ranked, so
+    B-bar is always a subset of B[perm] (the paper's second rationale for
+    Eq. 9), also when a kept weight is exactly zero;
+  * an "eligible" column block (the quantity the permutation search counts,
+    Alg. 1) has at most N forward-mask bits among its M rows;
+  * ties between candidate permutations go to the lowest candidate index;
+  * the weight gradient is the dense straight-through one, dW = dY^T X.
+
+Parity unpinned: the pseudo-random candidate generator (`candidates`).  The
+paper only says the K candidates are random; the generator below is this
+build's contract (its mixing function is pinned to the published SplitMix64
+test vector, the rest by permutation validity and a uniformity test).
+"""
+from __future__ import annotations
+
+import numpy as np
+
+MASK64 = (1 << 64) - 1
+
+
+# --------------------------------------------------------------------------
+# helpers: magnitude key, bf16 rounding
+# --------------------------------------------------------------------------
+def magnitude_key(W: np.ndarray) -> np.ndarray:
+    """Integer magnitude of fp32 values: the bit pattern with the sign cleared."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    return (W.view(np.uint32) & np.uint32(0x7FFFFFFF)).astype(np.int64)
+
+
+def bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round fp32 to bfloat16 (round to nearest, ties to even); returns uint16 bit patterns.
+
+    NaN becomes a quiet NaN with the sign kept; infinities are kept."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    u = x.view(np.uint32).astype(np.uint64)
+    rounded = (u + np.uint64(0x7FFF) + ((u >> np.uint64(16)) & np.uint64(1))) >> np.uint64(16)
+    is_nan = (u & np.uint64(0x7FFFFFFF)) > np.uint64(0x7F800000)
+    nan_bits = (u >> np.uint64(16)) | np.uint64(0x0040)
+    return np.where(is_nan, nan_bits, rounded).astype(np.uint16)
+
+
+def bf16_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Exact value of bfloat16 bit patterns, as float64."""
+    b = np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)
+    return b.view(np.float32).astype(np.float64)
+
+
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """fp32 -> bf16 -> float64 (the value the tensor core sees)."""
+    return bf16_to_f64(bf16_bits(x))
+
+
+# --------------------------------------------------------------------------
+# Eq. 4: forward mask
+# --------------------------------------------------------------------------
+def _rank_keep(key: np.ndarray, valid: np.ndarray, N: int) -> np.ndarray:
+    """key, valid: (..., M).  Keep element m iff it is valid and fewer than N valid
+    elements of its block beat it (larger key, or equal key at a lower position)."""
+    M = key.shape[-1]
+    keep = np.zeros(key.shape, dtype=bool)
+    for m in range(M):
+        beaten_by = np.zeros(key.shape[:-1], dtype=np.int64)
+        for q in range(M):
+            if q == m:
+                continue
+            if q < m:
+                beats = key[..., q] >= key[..., m]
+            else:
+                beats = key[..., q] > key[..., m]
+            beaten_by += (beats & valid[..., q]).astype(np.int64)
+        keep[..., m] = valid[..., m] & (beaten_by < N)
+    return keep
+
+
+def forward_mask(W: np.ndarray, N: int, M: int) -> np.ndarray:
+    """Eq. 4 (constraint Eq. 2): B[i, gM:(g+1)M] keeps the N largest |W| of the block.
+
+    Returns a bool array I x J with exactly N ones in every aligned row block."""
+    I, J = W.shape
+    assert J % M == 0 and 1 <= N <= M
+    key = magnitude_key(W).reshape(I, J // M, M)
+    keep = _rank_keep(key, np.ones_like(key, dtype=bool), N)
+    return keep.reshape(I, J)
+
+
+# --------------------------------------------------------------------------
+# Alg. 1 (permutation step): candidates, eligible-block count, pick
+# --------------------------------------------------------------------------
+def _mix64(z: int) -> int:
+    z &= MASK64
+    z ^= z >> 30
+    z = (z * 0xBF58476D1CE4E5B9) & MASK64
+    z ^= z >> 27
+    z = (z * 0x94D049BB133111EB) & MASK64
+    z ^= z >> 31
+    return z
+
+
+def _mix64_np(z: np.ndarray) -> np.ndarray:
+    z = z.astype(np.uint64)
+    z ^= z >> np.uint64(30)
+    z *= np.uint64(0xBF58476D1CE4E5B9)
+    z ^= z >> np.uint64(27)
+    z *= np.uint64(0x94D049BB133111EB)
+    z ^= z >> np.uint64(31)
+    return z
+
+
+def candidates(seed: int, P: int, I: int) -> np.ndarray:
+    """P pseudo-random permutations of {0..I-1} ("randomly generate K permutations", Alg. 1).
+
+    Candidate c sorts the rows by a hashed key: row i gets
+        h = mix64(mix64(seed + 0x9E3779B97F4A7C15 * (c + 1)) ^ i)
+    and the sort key (h with its low 24 bits replaced by i), so keys are distinct
+    and the result does not depend on the sorting algorithm.  Requires I < 2**24."""
+    assert 0 < I < (1 << 24) and P >= 1
+    out = np.empty((P, I), dtype=np.int32)
+    rows = np.arange(I, dtype=np.uint64)
+    with np.errstate(over="ignore"):
+        for c in range(P):
+            stream = _mix64((seed + 0x9E3779B97F4A7C15 * (c + 1)) & MASK64)
+            h = _mix64_np(np.uint64(stream) ^ rows)
+            v = (h & ~np.uint64(0xFFFFFF)) | rows
+            v.sort()
+            out[c] = (v & np.uint64(0xFFFFFF)).astype(np.int32)
+    return out
+
+
+def eligible_blocks(B: np.ndarray, perm: np.ndarray, N: int, M: int) -> int:
+    """Number of (row block k, column l) pairs of B[perm, :] that already satisfy N:M,
+    i.e. hold at most N ones among rows kM..kM+M-1 (the paper's "eligible N:M blocks")."""
+    I, J = B.shape
+    assert I % M == 0
+    Bp = B[np.asarray(perm, dtype=np.int64), :]
+    pop = Bp.reshape(I // M, M, J).sum(axis=1)
+    return int((pop <= N).sum())
+
+
+def perm_search(B: np.ndarray, cands: np.ndarray, N: int, M: int):
+    """Alg. 1, permutation step: score every candidate, pick the one with the most
+    eligible blocks (lowest index on ties).  Returns (best_idx, best_perm, counts)."""
+    counts = np.array([eligible_blocks(B, c, N, M) for c in cands], dtype=np.int64)
+    best = int(np.argmax(counts))          # argmax returns the first maximum
+    return best, np.array(cands[best], dtype=np.int32), counts
+
+
+# --------------------------------------------------------------------------
+# Eq. 11 (Eq. 9 when perm is the identity): backward mask
+# --------------------------------------------------------------------------
+def backward_mask(W: np.ndarray, B: np.ndarray, perm: np.ndarray, N: int, M: int) -> np.ndarray:
+    """Eq. 11: on the row-permuted masked weights (B*W)[perm, :], every aligned block of M
+    rows of every column keeps its N largest magnitudes among the entries whose forward
+    bit is set.  Returns B-bar (bool, I x J) in PERMUTED row order (row k <-> W row perm[k])."""
+    I, J = W.shape
+    assert I % M == 0 and 1 <= N <= M
+    p = np.asarray(perm, dtype=np.int64)
+    key = magnitude_key(W)[p, :].reshape(I // M, M, J).transpose(0, 2, 1)   # (blocks, J, M)
+    valid = B[p, :].reshape(I // M, M, J).transpose(0, 2, 1)
+    keep = _rank_keep(key, valid, N)
+    return keep.transpose(0, 2, 1).reshape(I, J)
+
+
+def unpermute_rows(Bbar_p: np.ndarray, perm: np.ndarray) -> np.ndarray:
+    """M_b[perm[k], :] = B-bar[k, :]  (backward mask in the original row order)."""
+    out = np.zeros_like(Bbar_p)
+    out[np.asarray(perm, dtype=np.int64), :] = Bbar_p
+    return out
+
+
+# --------------------------------------------------------------------------
+# 2:4 operand format (not in the paper; defined by this build's interface)
+# --------------------------------------------------------------------------
+def pack_bits(mask: np.ndarray) -> np.ndarray:
+    """bool R x C (C % 32 == 0) -> uint32 R x C/32, bit (c % 32) of word c // 32."""
+    R, C = mask.shape
+    assert C % 32 == 0
+    m = mask.reshape(R, C // 32, 32).astype(np.uint64)
+    weights = (np.uint64(1) << np.arange(32, dtype=np.uint64))
+    return (m * weights).sum(axis=2).astype(np.uint32)
+
+
+def unpack_bits(words: np.ndarray, C: int) -> np.ndarray:
+    R = words.shape[0]
+    w = words.astype(np.uint64)[:, :, None] >> np.arange(32, dtype=np.uint64)
+    return (w & np.uint64(1)).astype(bool).reshape(R, -1)[:, :C]
+
+
+def pack_2to4(A: np.ndarray, keep: np.ndarray):
+    """Compress a matrix whose kept entries number at most 2 per aligned group of 4 along
+    the rows into the 2:4 tensor-core operand: two bf16 values and one 4-bit index code
+    per group.
+
+    A: fp32 R x C, keep: bool R x C.  Returns (vals uint16 R x C/2, meta uint32 R x C/32).
+    Per group: S = kept positions ascending.  Fewer than 2 kept: pad with the lowest
+    positions not in S and sort.  Code = idx0 | idx1 << 2; slot s holds bf16(A[idx_s]) if
+    idx_s is kept, else +0.  Code g of a row sits in bits [4 (g % 8), +4) of word g // 8."""
+    R, C = A.shape
+    assert C % 32 == 0
+    G = C // 4
+    keep4 = keep.reshape(R, G, 4)
+    assert int(keep4.sum(axis=2).max(initial=0)) <= 2
+    abits = bf16_bits(A).reshape(R, G, 4)
+    vals = np.zeros((R, G, 2), dtype=np.uint16)
+    code = np.zeros((R, G), dtype=np.uint32)
+    for r in range(R):
+        for g in range(G):
+            S = [m for m in range(4) if keep4[r, g, m]]
+            idx = list(S)
+            m = 0
+            while len(idx) < 2:
+                if m not in idx:
+                    idx.append(m)
+                m += 1
+            idx.sort()
+            code[r, g] = idx[0] | (idx[1] << 2)
+            for s in range(2):
+                vals[r, g, s] = abits[r, g, idx[s]] if idx[s] in S else 0
+    shifts = (4 * (np.arange(G) % 8)).astype(np.uint32)
+    meta = (code << shifts).reshape(R, G // 8, 8).sum(axis=2).astype(np.uint32)
+    return vals.reshape(R, C // 2), meta
+
+
+def pack_2to4_fast(A: np.ndarray, keep: np.ndarray):
+    """Same result as pack_2to4, vectorised over groups (used at sizes where the
+    per-group Python loop would take minutes).  Checked against pack_2to4 in the tests."""
+    R, C = A.shape
+    assert C % 32 == 0
+    G = C // 4
+    keep4 = keep.reshape(R, G, 4)
+    cnt = keep4.sum(axis=2)
+    assert int(cnt.max(initial=0)) <= 2
+    abits = bf16_bits(A).reshape(R, G, 4)
+    pos = np.arange(4)
+    # first and last kept position of each group
+    first = np.where(keep4, pos, 9).min(axis=2)
+    last = np.where(keep4, pos, -1).max(axis=2)
+    idx0 = np.zeros((R, G), dtype=np.int64)
+    idx1 = np.ones((R, G), dtype=np.int64)
+    two = cnt == 2
+    idx0[two] = first[two]
+    idx1[two] = last[two]
+    one = cnt == 1
+    p = first[one]
+    idx0[one] = 0
+    idx1[one] = np.where(p <= 1, 1, p)
+    code = (idx0 | (idx1 << 2)).astype(np.uint32)
+    take0 = np.take_along_axis(abits, idx0[..., None], axis=2)[..., 0]
+    take1 = np.take_along_axis(abits, idx1[..., None], axis=2)[..., 0]
+    kept0 = np.take_along_axis(keep4, idx0[..., None], axis=2)[..., 0]
+    kept1 = np.take_along_axis(keep4, idx1[..., None], axis=2)[..., 0]
+    vals = np.stack([np.where(kept0, take0, 0), np.where(kept1, take1, 0)], axis=2).astype(np.uint16)
+    shifts = (4 * (np.arange(G) % 8)).astype(np.uint32)
+    meta = (code << shifts).reshape(R, G // 8, 8).sum(axis=2).astype(np.uint32)
+    return vals.reshape(R, C // 2), meta
+
+
+def unpack_2to4(vals: np.ndarray, meta: np.ndarray) -> np.ndarray:
+    """Expand a packed 2:4 operand back to a dense float64 R x C matrix."""
+    R, half = vals.shape
+    G = half // 2
+    v = bf16_to_f64(vals).reshape(R, G, 2)
+    out = np.zeros((R, G, 4), dtype=np.float64)
+    for r in range(R):
+        for g in range(G):
+            c = (int(meta[r, g // 8]) >> (4 * (g % 8))) & 0xF
+            # a slot holding +0 adds nothing, so a padded slot never disturbs a kept one
+            out[r, g, c & 3] += v[r, g, 0]
+            out[r, g, (c >> 2) & 3] += v[r, g, 1]
+    return out.reshape(R, 4 * G)
+
+
+def forward_operand(W: np.ndarray, B: np.ndarray):
+    """Packed forward operand A_f = B*W (I x J, 2:4 along J): (maskbits, vals, meta)."""
+    vals, meta = pack_2to4_fast(W, B)
+    return pack_bits(B), vals, meta
+
+
+def backward_operand(W: np.ndarray, Bbar_p: np.ndarray, perm: np.ndarray):
+    """Packed backward operand A' = (B-bar * W[perm, :])^T  (J x I, 2:4 along the permuted
+    rows of W, which is the reduction dim of Eq. 10): (maskbits of B-bar, vals, meta)."""
+    Wp = np.ascontiguousarray(W[np.asarray(perm, dtype=np.int64), :], dtype=np.float32)
+    vals, meta = pack_2to4_fast(np.ascontiguousarray(Wp.T), np.ascontiguousarray(Bbar_p.T))
+    return pack_bits(Bbar_p), vals, meta
+
+
+# --------------------------------------------------------------------------
+# Eq. 3, Eq. 8 / Eq. 10, STE weight gradient
+# --------------------------------------------------------------------------
+def spmm_fwd(X_bits: np.ndarray, W: np.ndarray, B: np.ndarray) -> np.ndarray:
+    """Eq. 3 in the row-major activation layout: Y[t, i] = sum_j X[t, j] (B*W)[i, j],
+    on bf16-rounded W and bf16 X, accumulated in float64."""
+    Wf = bf16_round(W) * B
+    return bf16_to_f64(X_bits) @ Wf.T
+
+
+def spmm_dgrad(dY_bits: np.ndarray, W: np.ndarray, Mb: np.ndarray) -> np.ndarray:
+    """Eq. 8: dX[t, j] = sum_i dY[t, i] (M_b*W)[i, j], with M_b the backward mask in the
+    original row order (the unpermuted form, which Eq. 10 says equals the permuted one)."""
+    Wb = bf16_round(W) * Mb
+    return bf16_to_f64(dY_bits) @ Wb
+
+
+def spmm_dgrad_permuted(dY_bits: np.ndarray, W: np.ndarray, Bbar_p: np.ndarray, perm: np.ndarray) -> np.ndarray:
+    """Eq. 10 as printed: (B-bar * W[perm, :])^T applied to dY[:, perm]."""
+    p = np.asarray(perm, dtype=np.int64)
+    Wp = bf16_round(W)[p, :] * Bbar_p
+    return bf16_to_f64(dY_bits)[:, p] @ Wp
+
+
+def dense_dgrad(dY_bits: np.ndarray, W: np.ndarray, B: np.ndarray) -> np.ndarray:
+    """Eq. 5: the exact input gradient through the forward mask (what Bi-Mask approximates)."""
+    return bf16_to_f64(dY_bits) @ (bf16_round(W) * B)
+
+
+def wgrad(dY_bits: np.ndarray, X_bits: np.ndarray) -> np.ndarray:
+    """Straight-through weight gradient: dW[i, j] = sum_t dY[t, i] X[t, j] (dense, unmasked)."""
+    return bf16_to_f64(dY_bits).T @ bf16_to_f64(X_bits)
+
+
+# --------------------------------------------------------------------------
+# Alg. 1 body for one layer
+# --------------------------------------------------------------------------
+def layer_step(W, X_bits, dY_bits, N, M, P, seed, do_search=True, perm=None, cands=None,
+               with_gemms=True):
+    """One iteration of Alg. 1 for one layer, minus the optimizer update.
+
+    Returns a dict with B, the packed forward operand, the candidates' counts, the chosen
+    permutation, B-bar (permuted order), M_b, the packed backward operand and, when
+    with_gemms, Y, dX and dW (float64)."""
+    I, J = W.shape
+    out = {}
+    B = forward_mask(W, N, M)
+    out["B"] = B
+    packable = (M == 4 and N <= 2)      # only such masks fit the 2:4 operand format
+    if packable:
+        out["maskbits_f"], out["vals_f"], out["meta_f"] = forward_operand(W, B)
+    if do_search:
+        if cands is None:
+            cands = candidates(seed, P, I)
+        best, perm, counts = perm_search(B, cands, N, M)
+        out["best_idx"], out["counts"] = best, counts
+    else:
+        perm = np.arange(I, dtype=np.int32) if perm is None else np.asarray(perm, dtype=np.int32)
+    out["perm"] = perm
+    Bbar_p = backward_mask(W, B, perm, N, M)
+    out["Bbar_p"] = Bbar_p
+    out["M_b"] = unpermute_rows(Bbar_p, perm)
+    if packable:
+        out["maskbits_b"], out["vals_b"], out["meta_b"] = backward_operand(W, Bbar_p, perm)
+    if with_gemms:
+        out["Y"] = spmm_fwd(X_bits, W, B)
+        out["dX"] = spmm_dgrad(dY_bits, W, out["M_b"])
+        out["dW"] = wgrad(dY_bits, X_bits)
+    return out

@@ -1,0 +1,358 @@
+"""Pins for the CPU oracle: everything here checks oracle/ against something other than
+itself -- hand-worked examples (tests/golden), brute force written a different way,
+closed forms, invariants the paper states, and special cases that reduce to library
+routines.  No GPU needed."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+from hypothesis import given, settings, strategies as st
+
+from oracle import bimask_oracle as O
+from paper_2302_06058_b200 import inputs
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ---------------------------------------------------------------- golden readers
+def _read_blocks():
+    rows = []
+    with open(os.path.join(GOLDEN, "handworked_blocks.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            n, w, kept, code, slots = [p.strip() for p in line.split("|")]
+            rows.append((int(n), [float(x) for x in w.split()], [int(x) for x in kept.split()],
+                         int(code, 16), [float(x) for x in slots.split()]))
+    return rows
+
+
+def _read_example():
+    sections = {}
+    cur = None
+    with open(os.path.join(GOLDEN, "example_8x8.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            if line.startswith("["):
+                cur = line
+                sections[cur] = []
+            else:
+                sections[cur].append(line)
+    W = np.array([[float(x) for x in r.split()] for r in sections["[W]"]], dtype=np.float32)
+    B = np.array([[int(x) for x in r.split()] for r in sections["[B]"]], dtype=bool)
+    perms = []
+    for r in sections["[perm count nnz(B-bar)]"]:
+        p, c, n = [q.strip() for q in r.split("|")]
+        perms.append(([int(x) for x in p.split()], int(c), int(n)))
+    return W, B, perms
+
+
+# ---------------------------------------------------------------- independent brute force
+def brute_forward_mask(W, N, M):
+    """Top-N per block by sorting (-|w|, index): a different formulation of Eq. 4."""
+    I, J = W.shape
+    B = np.zeros((I, J), dtype=bool)
+    for i in range(I):
+        for g in range(J // M):
+            blk = [(-abs(float(W[i, g * M + m])), m) for m in range(M)]
+            for _, m in sorted(blk)[:N]:
+                B[i, g * M + m] = True
+    return B
+
+
+def brute_backward_mask(W, B, perm, N, M):
+    """Eq. 11 by sorting, on (B*W)[perm, :] restricted to forward survivors."""
+    I, J = W.shape
+    out = np.zeros((I, J), dtype=bool)
+    for l in range(J):
+        for k in range(I // M):
+            blk = [(-abs(float(W[perm[k * M + m], l])), m) for m in range(M) if B[perm[k * M + m], l]]
+            for _, m in sorted(blk)[:N]:
+                out[k * M + m, l] = True
+    return out
+
+
+def brute_count(B, perm, N, M):
+    I, J = B.shape
+    total = 0
+    for k in range(I // M):
+        for l in range(J):
+            s = 0
+            for m in range(M):
+                s += 1 if B[perm[k * M + m], l] else 0
+            total += 1 if s <= N else 0
+    return total
+
+
+# ---------------------------------------------------------------- hand-worked examples
+@pytest.mark.parametrize("row", _read_blocks())
+def test_handworked_block(row):
+    n, w, kept, code, slots = row
+    # a full 32-wide row so that the packed format applies; the block under test is group 0,
+    # the other groups are copies (every group packs independently)
+    W = np.tile(np.array(w, dtype=np.float32), 8)[None, :]
+    B = O.forward_mask(W, n, 4)
+    assert list(np.nonzero(B[0, :4])[0]) == kept
+    vals, meta = O.pack_2to4(W, B)
+    assert (int(meta[0, 0]) & 0xF) == code
+    assert int(meta[0, 0]) == sum(code << (4 * g) for g in range(8))
+    got = O.bf16_to_f64(vals[0, :2])
+    assert list(got) == slots
+
+
+def test_two_blocks_share_a_byte():
+    W = np.tile(np.array([9, -1, 4, -6, 2, 7, -3, 5], dtype=np.float32), 4)[None, :]
+    B = O.forward_mask(W, 2, 4)
+    _, meta = O.pack_2to4(W, B)
+    assert (int(meta[0, 0]) & 0xFF) == 0xDC          # block 0 in the low nibble
+    bits = O.pack_bits(B)
+    assert (int(bits[0, 0]) & 0xFF) == 0b10101001    # bit j of the word = column j
+
+
+def test_example_8x8_mask_and_counts():
+    W, B, perms = _read_example()
+    assert np.array_equal(O.forward_mask(W, 2, 4), B)
+    for p, count, nnz in perms:
+        assert O.eligible_blocks(B, np.array(p), 2, 4) == count
+        Bbar = O.backward_mask(W, B, np.array(p), 2, 4)
+        assert int(Bbar.sum()) == nnz
+        assert np.array_equal(Bbar, brute_backward_mask(W, B, p, 2, 4))
+
+
+def test_example_8x8_all_permutations():
+    """All 8! row orders: the oracle's count equals a plain triple loop, and the search over
+    all of them returns the first maximiser."""
+    W, B, _ = _read_example()
+    allp = np.array(list(itertools.permutations(range(8))), dtype=np.int32)
+    ref = np.array([brute_count(B, p, 2, 4) for p in allp])
+    best, best_perm, counts = O.perm_search(B, allp, 2, 4)
+    assert np.array_equal(counts, ref)
+    assert counts.max() == 16 and counts.min() == 8
+    assert best == int(np.nonzero(ref == 16)[0][0])
+    assert np.array_equal(best_perm, allp[best])
+    # the count depends only on which rows share a block: 8!/(4!4!2) = 35 splits, each hit 1152 times
+    hist = {int(v): int((ref == v).sum()) for v in np.unique(ref)}
+    assert all(n % 1152 == 0 for n in hist.values())
+    assert sum(hist.values()) == math.factorial(8)
+
+
+# ---------------------------------------------------------------- brute force on random inputs
+@pytest.mark.parametrize("N,M", [(2, 4), (1, 4), (3, 4), (4, 4), (2, 8), (4, 8), (1, 16)])
+def test_masks_match_sort_based_definition(N, M):
+    rng = np.random.default_rng(5)
+    I, J = 2 * M * 2, 32 * max(1, M // 4)
+    # few distinct magnitudes => many ties, plus exact zeros and negative zero
+    W = rng.integers(-3, 4, size=(I, J)).astype(np.float32)
+    W[0, :4] = [-0.0, 0.0, 0.0, -0.0]
+    B = O.forward_mask(W, N, M)
+    assert np.array_equal(B, brute_forward_mask(W, N, M))
+    perm = rng.permutation(I)
+    Bbar = O.backward_mask(W, B, perm, N, M)
+    assert np.array_equal(Bbar, brute_backward_mask(W, B, perm, N, M))
+    assert O.eligible_blocks(B, perm, N, M) == brute_count(B, perm, N, M)
+
+
+def test_literal_eq4_agrees_when_magnitudes_distinct():
+    """Eq. 4 verbatim (zero iff |w| < N-th largest of the block) on tie-free weights."""
+    rng = np.random.default_rng(11)
+    W = rng.standard_normal((16, 64)).astype(np.float32)
+    for N, M in [(2, 4), (1, 4), (2, 8)]:
+        blocks = np.abs(W).reshape(16, 64 // M, M)
+        nth = np.sort(blocks, axis=2)[:, :, M - N][:, :, None]
+        literal = (blocks >= nth).reshape(16, 64)
+        assert np.array_equal(O.forward_mask(W, N, M), literal)
+
+
+def test_literal_eq9_agrees_when_magnitudes_distinct():
+    rng = np.random.default_rng(12)
+    W = rng.standard_normal((16, 32)).astype(np.float32)
+    B = O.forward_mask(W, 2, 4)
+    masked = np.abs(W) * B
+    blocks = masked.reshape(4, 4, 32)                       # (block, m, column)
+    nth = np.sort(blocks, axis=1)[:, 2, :][:, None, :]      # 2nd largest of 4
+    literal = np.where(blocks < nth, False, B.reshape(4, 4, 32)).reshape(16, 32)
+    got = O.backward_mask(W, B, np.arange(16), 2, 4)
+    assert np.array_equal(got, literal)
+
+
+# ---------------------------------------------------------------- invariants
+@settings(max_examples=40, deadline=None)
+@given(st.integers(0, 2**31 - 1), st.sampled_from([(2, 4), (1, 4), (2, 8), (1, 8)]),
+       st.integers(1, 3), st.integers(1, 2))
+def test_invariants(seed, nm, ib, jb):
+    N, M = nm
+    I, J = 8 * ib * (M // 4), 32 * jb
+    rng = np.random.default_rng(seed)
+    W = rng.standard_normal((I, J)).astype(np.float32)
+    W[rng.random((I, J)) < 0.1] = 0.0
+    B = O.forward_mask(W, N, M)
+    assert (B.reshape(I, J // M, M).sum(axis=2) == N).all()                 # Eq. 2, exactly N
+    perm = rng.permutation(I).astype(np.int32)
+    Bbar = O.backward_mask(W, B, perm, N, M)
+    Bp = B[perm]
+    assert not (Bbar & ~Bp).any()                                            # B = 0 => B-bar = 0
+    pop_f = Bp.reshape(I // M, M, J).sum(axis=1)
+    pop_b = Bbar.reshape(I // M, M, J).sum(axis=1)
+    assert (pop_b <= N).all()                                                # Eq. 7
+    assert np.array_equal(pop_b, np.minimum(pop_f, N))
+    same = (Bbar.reshape(I // M, M, J) == Bp.reshape(I // M, M, J)).all(axis=1)
+    assert np.array_equal(same, pop_f <= N)          # eligible block <=> B-bar block == B block
+    assert O.eligible_blocks(B, perm, N, M) == int(same.sum())
+    Mb = O.unpermute_rows(Bbar, perm)
+    assert np.array_equal(Mb[perm], Bbar)
+    if M == 4:
+        vals, meta = O.pack_2to4(W, B)
+        vf, mf = O.pack_2to4_fast(W, B)
+        assert np.array_equal(vals, vf) and np.array_equal(meta, mf)
+        codes = (meta[:, :, None] >> (4 * np.arange(8, dtype=np.uint32))) & 0xF
+        assert np.isin(codes, [0x4, 0x8, 0xC, 0x9, 0xD, 0xE]).all()
+        assert np.array_equal(O.unpack_2to4(vals, meta), O.bf16_round(W) * B)
+        assert np.array_equal(O.unpack_bits(O.pack_bits(B), J), B)
+        if I % 32 == 0:
+            _, vb, mb = O.backward_operand(W, Bbar, perm)
+            vb2, mb2 = O.pack_2to4(np.ascontiguousarray(W[perm].T), np.ascontiguousarray(Bbar.T))
+            assert np.array_equal(vb, vb2) and np.array_equal(mb, mb2)
+            assert np.array_equal(O.unpack_2to4(vb, mb), (O.bf16_round(W)[perm] * Bbar).T)
+
+
+# ---------------------------------------------------------------- closed forms
+@pytest.mark.parametrize("N,M,elig,ratio", [(2, 4, 11 / 16, 13 / 16), (1, 4, 189 / 256, 175 / 256)])
+def test_closed_form_eligible_fraction(N, M, elig, ratio):
+    """For i.i.d. continuous weights the forward bits of one column over distinct rows are
+    i.i.d. Bernoulli(N/M): P(eligible) = P(Bin(M, N/M) <= N), E nnz(B-bar)/nnz(B) =
+    E min(Bin, N) / N."""
+    binom = [math.comb(M, k) * (N / M) ** k * (1 - N / M) ** (M - k) for k in range(M + 1)]
+    assert abs(sum(binom[:N + 1]) - elig) < 1e-12
+    assert abs(sum(min(k, N) * binom[k] for k in range(M + 1)) / N - ratio) < 1e-12
+    W = inputs.make_weight(512, 1024, 7)
+    B = O.forward_mask(W, N, M)
+    perm = np.random.default_rng(3).permutation(512)
+    nblocks = (512 // M) * 1024
+    frac = O.eligible_blocks(B, perm, N, M) / nblocks
+    sigma = math.sqrt(elig * (1 - elig) / nblocks)
+    assert abs(frac - elig) < 6 * sigma
+    Bbar = O.backward_mask(W, B, perm, N, M)
+    assert abs(Bbar.sum() / B.sum() - ratio) < 5e-3
+
+
+# ---------------------------------------------------------------- special cases -> library routines
+def test_n_equals_m_reduces_to_plain_matmul():
+    W, X, dY = inputs.make_layer(1, 0, T=48)
+    out = O.layer_step(W, X, dY, 4, 4, 2, 1)
+    assert out["B"].all() and out["Bbar_p"].all()
+    Wt = torch.from_numpy(W).to(torch.bfloat16).to(torch.float64)
+    Xt = torch.from_numpy(X.view(np.int16)).view(torch.bfloat16).to(torch.float64)
+    dYt = torch.from_numpy(dY.view(np.int16)).view(torch.bfloat16).to(torch.float64)
+    assert np.allclose(out["Y"], (Xt @ Wt.T).numpy(), rtol=1e-12, atol=1e-12)
+    assert np.allclose(out["dX"], (dYt @ Wt).numpy(), rtol=1e-12, atol=1e-12)
+    assert np.allclose(out["dW"], (dYt.T @ Xt).numpy(), rtol=1e-12, atol=1e-12)
+
+
+def test_masked_products_against_torch():
+    W, X, dY = inputs.make_layer(1, 0, T=40)
+    out = O.layer_step(W, X, dY, 2, 4, 8, 43)
+    Wt = torch.from_numpy(W).to(torch.bfloat16).to(torch.float64)
+    Xt = torch.from_numpy(X.view(np.int16)).view(torch.bfloat16).to(torch.float64)
+    dYt = torch.from_numpy(dY.view(np.int16)).view(torch.bfloat16).to(torch.float64)
+    Bf = torch.from_numpy(brute_forward_mask(W, 2, 4)).to(torch.float64)
+    assert np.allclose(out["Y"], (Xt @ (Wt * Bf).T).numpy(), rtol=1e-12, atol=1e-12)
+    Mb = torch.from_numpy(out["M_b"]).to(torch.float64)
+    assert np.allclose(out["dX"], (dYt @ (Wt * Mb)).numpy(), rtol=1e-12, atol=1e-12)
+    assert np.allclose(out["dW"], (dYt.T @ Xt).numpy(), rtol=1e-12, atol=1e-12)
+    # transposition check: Y is T x I, dX is T x J, dW is I x J
+    assert out["Y"].shape == (40, 256) and out["dX"].shape == (40, 256) and out["dW"].shape == (256, 256)
+
+
+def test_permuted_form_equals_unpermuted_form():
+    """Eq. 10: permuting W's rows and dY's columns together leaves the product unchanged."""
+    W, X, dY = inputs.make_layer(1, 0, T=32)
+    B = O.forward_mask(W, 2, 4)
+    perm = O.candidates(9, 1, 256)[0]
+    Bbar = O.backward_mask(W, B, perm, 2, 4)
+    a = O.spmm_dgrad(dY, W, O.unpermute_rows(Bbar, perm))
+    b = O.spmm_dgrad_permuted(dY, W, Bbar, perm)
+    assert np.allclose(a, b, rtol=1e-12, atol=1e-12)
+
+
+def test_planted_transposable_mask_gives_exact_gradient():
+    """If every column block of B[perm] is already N:M, B-bar = B[perm], every block is
+    eligible and Eq. 10 equals the exact gradient of Eq. 5."""
+    for N in (2, 1):
+        W, Q = inputs.planted_transposable(64, 96, N, 4, 21)
+        B = O.forward_mask(W, N, 4)
+        rng = np.random.default_rng(0)
+        cands = np.stack([rng.permutation(64) for _ in range(5)] + [Q] +
+                         [rng.permutation(64) for _ in range(3)]).astype(np.int32)
+        best, perm, counts = O.perm_search(B, cands, N, 4)
+        assert best == 5 and counts[5] == (64 // 4) * 96 and (counts[:5] < counts[5]).all()
+        Bbar = O.backward_mask(W, B, perm, N, 4)
+        assert np.array_equal(Bbar, B[perm])
+        dY = inputs.make_activation(24, 64, 3)
+        exact = O.dense_dgrad(dY, W, B)
+        approx = O.spmm_dgrad(dY, W, O.unpermute_rows(Bbar, perm))
+        assert np.allclose(exact, approx, rtol=1e-12, atol=1e-12)
+
+
+# ---------------------------------------------------------------- bf16 rounding, generator
+def test_bf16_rounding_matches_torch():
+    rng = np.random.default_rng(1)
+    x = np.concatenate([rng.standard_normal(100000).astype(np.float32),
+                        np.array([0.0, -0.0, 1.0, 1.00390625, 1.01171875, np.inf, -np.inf,
+                                  3.3895314e38, 1e-40, -1e-40, 65504.0], dtype=np.float32),
+                        # exact ties: mantissa ends in 0x8000
+                        (np.arange(0x3F800000, 0x3F800000 + 64 * 0x8000, 0x8000, dtype=np.uint32)).view(np.float32)])
+    ref = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(O.bf16_bits(x), ref)
+    assert np.array_equal(O.bf16_to_f64(ref), torch.from_numpy(x).to(torch.bfloat16).to(torch.float64).numpy())
+    nan = O.bf16_bits(np.array([np.nan], dtype=np.float32))
+    assert (int(nan[0]) & 0x7F80) == 0x7F80 and (int(nan[0]) & 0x7F) != 0
+
+
+def test_mixer_matches_splitmix64_test_vector():
+    """mix64(seed + golden gamma) is SplitMix64's output function; its published outputs for
+    seed 0 are e220a8397b1dcdaf, 6e789e6aa1b965f4, 06c45d188009454f."""
+    g = 0x9E3779B97F4A7C15
+    got = [O._mix64((k * g) & O.MASK64) for k in (1, 2, 3)]
+    assert got == [0xE220A8397B1DCDAF, 0x6E789E6AA1B965F4, 0x06C45D188009454F]
+    z = np.array([(k * g) & O.MASK64 for k in (1, 2, 3)], dtype=np.uint64)
+    with np.errstate(over="ignore"):
+        assert [int(v) for v in O._mix64_np(z)] == got
+
+
+def test_candidates_are_permutations_and_uniform():
+    c = O.candidates(42, 16, 1000)
+    assert c.shape == (16, 1000) and c.dtype == np.int32
+    for row in c:
+        assert np.array_equal(np.sort(row), np.arange(1000))
+    assert len({tuple(r) for r in c}) == 16
+    assert np.array_equal(O.candidates(42, 16, 1000)[3], c[3])          # deterministic
+    assert not np.array_equal(O.candidates(43, 1, 1000)[0], c[0])       # seed matters
+    # position x value chi-square on many small permutations (49 degrees of freedom)
+    n = 20000
+    small = O.candidates(7, n, 8)
+    table = np.zeros((8, 8))
+    for pos in range(8):
+        table[pos] = np.bincount(small[:, pos], minlength=8)
+    chi2 = ((table - n / 8) ** 2 / (n / 8)).sum()
+    assert chi2 < 49 + 6 * math.sqrt(2 * 49)
+    # independent restatement of the key construction for one candidate, in Python integers
+    seed, cidx, I = 42, 2, 50
+    stream = O._mix64((seed + 0x9E3779B97F4A7C15 * (cidx + 1)) & O.MASK64)
+    keys = sorted(((O._mix64(stream ^ i) & ~0xFFFFFF) | i) for i in range(I))
+    assert [k & 0xFFFFFF for k in keys] == list(O.candidates(seed, 3, I)[2])
+
+
+def test_layer_step_identity_when_not_searching():
+    W, X, dY = inputs.make_layer(1, 0, T=8)
+    out = O.layer_step(W, X, dY, 2, 4, 8, 43, do_search=False)
+    assert np.array_equal(out["perm"], np.arange(256))
+    out2 = O.layer_step(W, X, dY, 2, 4, 8, 43, do_search=True)
+    assert out2["counts"].shape == (8,)
+    assert out2["counts"][out2["best_idx"]] == out2["counts"].max()
+    assert np.array_equal(out2["perm"], O.candidates(43, 8, 256)[out2["best_idx"]])
