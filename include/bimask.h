@@ -1,0 +1,159 @@
+/*
+ * bimask.h -- C ABI of the Bi-Mask per-layer sparse training step on one B200 (sm_100a).
+ *
+ * The step follows "Bi-directional Masks for Efficient N:M Sparse Training" (Alg. 1):
+ * forward N:M mask (Eq. 4), sparse forward product (Eq. 3), row-permutation search
+ * (Alg. 1, "pick the permutation with the most eligible N:M blocks"), backward mask on the
+ * permuted weights (Eq. 11), sparse input-gradient product (Eq. 10) and the dense
+ * straight-through weight gradient (Sec. 3.1).
+ *
+ * Conventions for every call unless stated otherwise
+ *   - All matrices are row-major and dense.  W is I x J fp32 (output rows x input dim),
+ *     X is T x J bf16, dY is T x I bf16 (bf16 is passed as uint16_t bit patterns).
+ *   - Every pointer is a DEVICE pointer owned by the caller, 16-byte aligned.  The library
+ *     allocates nothing, frees nothing and never synchronises: work is enqueued on `stream`
+ *     (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - Outputs are fully overwritten, inputs are never modified.
+ *   - Return value: BIMASK_OK or a negative bimask_status.  On a negative return caused by
+ *     argument validation nothing was launched.  bimask_last_error() gives a text for the
+ *     calling thread's last failure.
+ *   - Shapes: I % 32 == 0, J % 32 == 0, M == 4, 1 <= N <= 2 (1:4 is stored in the 2:4
+ *     container with the spare slot holding +0).
+ *   - `perm[k]` is the source row of permuted row k (gather: Wp[k,:] = W[perm[k],:]), 0-based.
+ *   - Device-side trouble (a bounded wait that ran out) is reported by writing a non-zero
+ *     code into *status_word (a device int the caller reads when it chooses to sync);
+ *     kernels never trap.
+ *
+ * Packed 2:4 operand ("vals" + "meta", not defined by the paper; it is the tensor core's
+ * compressed format written row by row):
+ *   per aligned group g of 4 consecutive elements of a row: S = kept positions ascending.
+ *   |S| = 2: (idx0, idx1) = S.  |S| < 2: pad with the lowest positions not in S, sort.
+ *   vals[row][2g + s] = bf16_rne(value at idx_s) if idx_s in S else +0.
+ *   code = idx0 | idx1 << 2, stored in bits [4 (g % 8), +4) of meta[row][g / 8].
+ *   maskbits[row][c / 32] bit (c % 32) = mask at column c.
+ *   "hw_meta" is an opaque re-ordering of meta for the tensor core; size from
+ *   bimask_hw_meta_bytes(rows, K).
+ */
+#ifndef BIMASK_H
+#define BIMASK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  BIMASK_OK = 0,
+  BIMASK_EINVAL = -1,       /* null / misaligned pointer, bad shape, N or P out of range, workspace too small */
+  BIMASK_EUNSUPPORTED = -2, /* N:M that does not fit the 2:4 container, M != 4, size beyond a kernel limit */
+  BIMASK_ECUDA = -3,        /* a CUDA call failed; see bimask_last_error() */
+  BIMASK_ETIMEOUT = -4      /* value written to *status_word when a device-side bounded wait ran out */
+} bimask_status;
+
+/* Text of the calling thread's last error ("" if none).  Host memory owned by the library. */
+const char* bimask_last_error(void);
+
+/* Bytes of the opaque tensor-core metadata buffer for a packed operand with `rows` rows and
+ * reduction length K (K = J for the forward operand, K = I for the backward one). */
+size_t bimask_hw_meta_bytes(int rows, int K);
+
+/* Bytes of scratch (`ws`) large enough for every call below on a layer of this size. */
+size_t bimask_workspace_bytes(int T, int I, int J, int P);
+
+/* Eq. 4 + packing.  Forward mask: in every row, every aligned block of M along J keeps its N
+ * largest |W| (ties: lowest index), compared on the fp32 values.
+ *   W          in   I x J fp32
+ *   maskbits_f out  I x J/32 u32
+ *   vals_f     out  I x J/2 bf16,  meta_f out I x J/32 u32,  hw_meta_f out (opaque) */
+int bimask_fwd_mask(const float* W, int I, int J, int N, int M,
+                    uint32_t* maskbits_f, uint16_t* vals_f, uint32_t* meta_f, void* hw_meta_f,
+                    void* stream);
+
+/* Alg. 1, permutation step.  counts[c] = number of (row block k, column l) whose M rows
+ * cand_c[kM .. kM+M-1] hold at most N forward-mask bits in column l ("eligible N:M blocks");
+ * best_idx = lowest c with the largest count; best_perm = cand_best.
+ *   cands_or_null  in   P x I i32 explicit candidates (each a permutation of 0..I-1), or NULL:
+ *                       then candidate c is generated from `seed` by sorting the rows by the
+ *                       key  mix64(mix64(seed + 0x9E3779B97F4A7C15 (c+1)) ^ i)  (low 24 bits
+ *                       replaced by i; mix64 = SplitMix64's output function).  Generated
+ *                       candidates need I <= 16384 (BIMASK_EUNSUPPORTED beyond).
+ *   This call alone accepts any I % 4 == 0 (the packed operands need I % 32 == 0).
+ *   best_perm out I i32, best_idx out 1 i32, counts out P i64
+ *   ws: scratch of at least bimask_workspace_bytes(...) bytes (holds the generated candidates). */
+int bimask_perm_search(const uint32_t* maskbits_f, int I, int J, int N, int M, int P, uint64_t seed,
+                       const int32_t* cands_or_null,
+                       int32_t* best_perm, int32_t* best_idx, int64_t* counts,
+                       void* ws, size_t ws_bytes, void* stream);
+
+/* Eq. 11 + transposed packing.  Backward mask on the permuted rows: in every column l, every
+ * aligned block of M permuted rows keeps, among the entries with forward bit 1, the N largest
+ * |W| (ties: lowest permuted row).  B-bar is a subset of B[perm].
+ *   maskbits_b out I x J/32 u32, row k = B-bar of W row perm[k]
+ *   vals_b out J x I/2 bf16, meta_b out J x I/32 u32: the operand (B-bar * W[perm,:])^T, 2:4
+ *   along the permuted row index (the reduction dim of Eq. 10); hw_meta_b opaque. */
+int bimask_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* perm,
+                    int I, int J, int N, int M,
+                    uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_b,
+                    void* stream);
+
+/* Eq. 3: Y[t, i] = sum_j X[t, j] (B * W)[i, j].  bf16 operands, fp32 accumulation, Y T x I bf16
+ * (round to nearest even).  vals_f / hw_meta_f as written by bimask_fwd_mask. */
+int bimask_spmm_fwd(const uint16_t* X, const uint16_t* vals_f, const void* hw_meta_f,
+                    int T, int I, int J, uint16_t* Y, int32_t* status_word, void* stream);
+
+/* Eq. 10: dX = (B-bar * W[perm,:])^T applied to dY[:, perm]; dX T x J bf16.
+ *   ws: scratch (holds the column-permuted copy of dY, T x I bf16). */
+int bimask_spmm_dgrad(const uint16_t* dY, const int32_t* perm, const uint16_t* vals_b,
+                      const void* hw_meta_b, int T, int I, int J, uint16_t* dX,
+                      void* ws, size_t ws_bytes, int32_t* status_word, void* stream);
+
+/* Straight-through weight gradient (Sec. 3.1): dW[i, j] = sum_t dY[t, i] X[t, j], dense,
+ * unmasked, fp32 I x J. */
+int bimask_wgrad(const uint16_t* dY, const uint16_t* X, int T, int I, int J, float* dW,
+                 void* ws, size_t ws_bytes, int32_t* status_word, void* stream);
+
+/* One iteration of Alg. 1 for one layer (without the optimizer update): fwd mask + pack,
+ * [search if do_search], bwd mask + pack, then the three products, all on `stream`. */
+typedef struct {
+  int T, I, J, N, M, P;
+  uint64_t seed;
+  int do_search;              /* 0: use perm as given; 1: search and overwrite perm */
+  const float* W;             /* I x J */
+  const uint16_t* X;          /* T x J bf16 */
+  const uint16_t* dY;         /* T x I bf16 */
+  const int32_t* cands;       /* P x I or NULL (generate from seed) */
+  int32_t* perm;              /* I, in/out */
+  int32_t* best_idx;          /* 1 */
+  int64_t* counts;            /* P */
+  uint32_t* maskbits_f; uint16_t* vals_f; uint32_t* meta_f; void* hw_meta_f;
+  uint32_t* maskbits_b; uint16_t* vals_b; uint32_t* meta_b; void* hw_meta_b;
+  uint16_t* Y;                /* T x I bf16 */
+  uint16_t* dX;               /* T x J bf16 */
+  float* dW;                  /* I x J fp32 */
+  void* ws; size_t ws_bytes;
+  int32_t* status_word;
+  void* stream;
+} bimask_layer_args;
+
+int bimask_layer_step(const bimask_layer_args* args);
+
+/* The same step for a caller whose data lives in HOST memory (pinned memory recommended):
+ * copies W, X, dY (and perm when do_search == 0) to the device buffers named in `dev`,
+ * runs bimask_layer_step there, copies Y, dX, dW, perm, best_idx, counts and the status word
+ * back into the host buffers named in `host`, and synchronises `dev->stream` before it
+ * returns.  Pointer fields of `host` that are NULL are skipped (not copied).  `dev` must be
+ * fully populated; its sizes/flags are used, those of `host` are ignored. */
+int bimask_layer_step_host(const bimask_layer_args* dev, const bimask_layer_args* host,
+                           int32_t* host_status_word);
+
+/* Debug helper, not on the hot path: sets *ok (device int) to 1 iff each of the P rows of
+ * cands is a permutation of 0..I-1.  ws: at least P * I bytes of scratch. */
+int bimask_check_perms(const int32_t* cands, int P, int I, int32_t* ok, void* ws, size_t ws_bytes,
+                       void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BIMASK_H */

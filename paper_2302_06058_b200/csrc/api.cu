@@ -1,0 +1,243 @@
+// C ABI of the library: argument validation, workspace carving and the order of launches.
+// No kernel code lives here.
+#include "common.cuh"
+#include <string.h>
+
+namespace bimask {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+}
+
+int cuda_fail(cudaError_t e, const char* what) {
+  set_error("%s failed: %s", what, cudaGetErrorString(e));
+  return BIMASK_ECUDA;
+}
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+static int check_shape(int I, int J, int N, int M) {
+  BIMASK_REQUIRE(M == 4, BIMASK_EUNSUPPORTED, "M = %d: only M = 4 is implemented", M);
+  BIMASK_REQUIRE(I > 0 && J > 0 && I % 32 == 0 && J % 32 == 0, BIMASK_EINVAL,
+                 "I = %d, J = %d: both must be positive multiples of 32", I, J);
+  BIMASK_REQUIRE(N >= 1 && N <= M, BIMASK_EINVAL, "N = %d out of range 1..%d", N, M);
+  BIMASK_REQUIRE(N <= 2, BIMASK_EUNSUPPORTED, "N:M = %d:%d does not fit the 2:4 container", N, M);
+  return BIMASK_OK;
+}
+
+struct WsPlan {
+  size_t cands_off, cands_bytes;
+  size_t dyp_off, dyp_bytes;
+  size_t part_off, part_bytes;
+  size_t total;
+};
+
+static WsPlan plan_ws(int T, int I, int J, int P) {
+  WsPlan w;
+  size_t off = 0;
+  w.cands_off = off; w.cands_bytes = align_up((size_t)(P > 0 ? P : 0) * I * sizeof(int32_t), 256); off += w.cands_bytes;
+  w.dyp_off = off; w.dyp_bytes = align_up((size_t)(T > 0 ? T : 0) * I * 2, 256); off += w.dyp_bytes;
+  int nt = 0, splits = 1, per = 0;
+  if (T > 0) wgrad_plan(T, I, J, &nt, &splits, &per);
+  w.part_off = off; w.part_bytes = splits > 1 ? align_up((size_t)splits * I * J * sizeof(float), 256) : 0; off += w.part_bytes;
+  w.total = off > 256 ? off : 256;
+  return w;
+}
+
+}  // namespace bimask
+
+using namespace bimask;
+
+extern "C" {
+
+const char* bimask_last_error(void) { return g_err; }
+
+size_t bimask_hw_meta_bytes(int rows, int K) {
+  if (rows <= 0 || K <= 0) return 0;
+  return (size_t)((rows + 127) / 128) * ((K + 127) / 128) * 2048;
+}
+
+size_t bimask_workspace_bytes(int T, int I, int J, int P) {
+  if (I <= 0 || J <= 0) return 0;
+  return plan_ws(T, I, J, P).total;
+}
+
+int bimask_fwd_mask(const float* W, int I, int J, int N, int M, uint32_t* maskbits_f, uint16_t* vals_f,
+                    uint32_t* meta_f, void* hw_meta_f, void* stream) {
+  int rc = check_shape(I, J, N, M);
+  if (rc != BIMASK_OK) return rc;
+  BIMASK_REQUIRE(W && maskbits_f && vals_f && meta_f && hw_meta_f, BIMASK_EINVAL, "bimask_fwd_mask: null pointer");
+  BIMASK_REQUIRE(aligned16(W) && aligned16(maskbits_f) && aligned16(vals_f) && aligned16(meta_f) && aligned16(hw_meta_f),
+                 BIMASK_EINVAL, "bimask_fwd_mask: pointers must be 16-byte aligned");
+  cudaStream_t s = (cudaStream_t)stream;
+  if ((rc = launch_fwd_mask(W, I, J, N, maskbits_f, vals_f, meta_f, s)) != BIMASK_OK) return rc;
+  return launch_hw_meta(meta_f, I, J, hw_meta_f, s);
+}
+
+int bimask_perm_search(const uint32_t* maskbits_f, int I, int J, int N, int M, int P, uint64_t seed,
+                       const int32_t* cands_or_null, int32_t* best_perm, int32_t* best_idx, int64_t* counts,
+                       void* ws, size_t ws_bytes, void* stream) {
+  BIMASK_REQUIRE(M == 4, BIMASK_EUNSUPPORTED, "M = %d: only M = 4 is implemented", M);
+  BIMASK_REQUIRE(I > 0 && J > 0 && I % 4 == 0 && J % 32 == 0, BIMASK_EINVAL,
+                 "I = %d, J = %d: I must be a positive multiple of 4, J of 32", I, J);
+  BIMASK_REQUIRE(N >= 1 && N <= M, BIMASK_EINVAL, "N = %d out of range 1..%d", N, M);
+  BIMASK_REQUIRE(P >= 1 && P <= 65535, BIMASK_EINVAL, "P = %d out of range 1..65535", P);
+  BIMASK_REQUIRE(maskbits_f && best_perm && best_idx && counts, BIMASK_EINVAL, "bimask_perm_search: null pointer");
+  BIMASK_REQUIRE(aligned16(maskbits_f) && aligned16(best_perm) && (!cands_or_null || aligned16(cands_or_null)) &&
+                     ((uintptr_t)counts % 8 == 0) && ((uintptr_t)best_idx % 4 == 0),
+                 BIMASK_EINVAL, "bimask_perm_search: misaligned pointer");
+  cudaStream_t s = (cudaStream_t)stream;
+  const int32_t* cands = cands_or_null;
+  int rc;
+  if (!cands) {
+    BIMASK_REQUIRE(I <= 16384, BIMASK_EUNSUPPORTED, "generated candidates need I <= 16384 (I = %d)", I);
+    const WsPlan w = plan_ws(0, I, J, P);
+    BIMASK_REQUIRE(ws && aligned16(ws) && ws_bytes >= w.cands_off + w.cands_bytes, BIMASK_EINVAL,
+                   "bimask_perm_search: workspace too small (%zu bytes, need %zu)", ws_bytes, w.cands_off + w.cands_bytes);
+    int32_t* gen = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(ws) + w.cands_off);
+    if ((rc = launch_gen_candidates(seed, P, I, gen, s)) != BIMASK_OK) return rc;
+    cands = gen;
+  }
+  if ((rc = launch_score(maskbits_f, cands, I, J, N, P, counts, s)) != BIMASK_OK) return rc;
+  return launch_pick(counts, cands, P, I, best_idx, best_perm, s);
+}
+
+int bimask_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J, int N, int M,
+                    uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_b, void* stream) {
+  int rc = check_shape(I, J, N, M);
+  if (rc != BIMASK_OK) return rc;
+  BIMASK_REQUIRE(W && maskbits_f && perm && maskbits_b && vals_b && meta_b && hw_meta_b, BIMASK_EINVAL,
+                 "bimask_bwd_mask: null pointer");
+  BIMASK_REQUIRE(aligned16(W) && aligned16(maskbits_f) && aligned16(perm) && aligned16(maskbits_b) &&
+                     aligned16(vals_b) && aligned16(meta_b) && aligned16(hw_meta_b),
+                 BIMASK_EINVAL, "bimask_bwd_mask: pointers must be 16-byte aligned");
+  cudaStream_t s = (cudaStream_t)stream;
+  if ((rc = launch_bwd_mask(W, maskbits_f, perm, I, J, N, maskbits_b, vals_b, meta_b, s)) != BIMASK_OK) return rc;
+  return launch_hw_meta(meta_b, J, I, hw_meta_b, s);
+}
+
+static int check_gemm(int T, int I, int J) {
+  BIMASK_REQUIRE(T > 0 && I > 0 && J > 0 && I % 32 == 0 && J % 32 == 0, BIMASK_EINVAL,
+                 "T = %d, I = %d, J = %d: T positive, I and J positive multiples of 32", T, I, J);
+  return BIMASK_OK;
+}
+
+int bimask_spmm_fwd(const uint16_t* X, const uint16_t* vals_f, const void* hw_meta_f, int T, int I, int J,
+                    uint16_t* Y, int32_t* status_word, void* stream) {
+  int rc = check_gemm(T, I, J);
+  if (rc != BIMASK_OK) return rc;
+  BIMASK_REQUIRE(X && vals_f && hw_meta_f && Y && status_word, BIMASK_EINVAL, "bimask_spmm_fwd: null pointer");
+  BIMASK_REQUIRE(aligned16(X) && aligned16(vals_f) && aligned16(hw_meta_f) && aligned16(Y), BIMASK_EINVAL,
+                 "bimask_spmm_fwd: pointers must be 16-byte aligned");
+  return launch_spmm(vals_f, hw_meta_f, X, I, T, J, Y, status_word, (cudaStream_t)stream);
+}
+
+int bimask_spmm_dgrad(const uint16_t* dY, const int32_t* perm, const uint16_t* vals_b, const void* hw_meta_b,
+                      int T, int I, int J, uint16_t* dX, void* ws, size_t ws_bytes, int32_t* status_word,
+                      void* stream) {
+  int rc = check_gemm(T, I, J);
+  if (rc != BIMASK_OK) return rc;
+  BIMASK_REQUIRE(dY && perm && vals_b && hw_meta_b && dX && status_word && ws, BIMASK_EINVAL,
+                 "bimask_spmm_dgrad: null pointer");
+  BIMASK_REQUIRE(aligned16(dY) && aligned16(perm) && aligned16(vals_b) && aligned16(hw_meta_b) && aligned16(dX) &&
+                     aligned16(ws),
+                 BIMASK_EINVAL, "bimask_spmm_dgrad: pointers must be 16-byte aligned");
+  BIMASK_REQUIRE((size_t)I * 2 <= 200 * 1024, BIMASK_EUNSUPPORTED, "I = %d too large for the column permute pass", I);
+  const WsPlan w = plan_ws(T, I, J, 0);
+  BIMASK_REQUIRE(ws_bytes >= w.dyp_off + w.dyp_bytes, BIMASK_EINVAL,
+                 "bimask_spmm_dgrad: workspace too small (%zu bytes, need %zu)", ws_bytes, w.dyp_off + w.dyp_bytes);
+  uint16_t* dYp = reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(ws) + w.dyp_off);
+  cudaStream_t s = (cudaStream_t)stream;
+  if ((rc = launch_permute_cols(dY, perm, T, I, dYp, s)) != BIMASK_OK) return rc;
+  return launch_spmm(vals_b, hw_meta_b, dYp, J, T, I, dX, status_word, s);
+}
+
+int bimask_wgrad(const uint16_t* dY, const uint16_t* X, int T, int I, int J, float* dW, void* ws, size_t ws_bytes,
+                 int32_t* status_word, void* stream) {
+  int rc = check_gemm(T, I, J);
+  if (rc != BIMASK_OK) return rc;
+  BIMASK_REQUIRE(dY && X && dW && status_word, BIMASK_EINVAL, "bimask_wgrad: null pointer");
+  BIMASK_REQUIRE(aligned16(dY) && aligned16(X) && aligned16(dW) && (!ws || aligned16(ws)), BIMASK_EINVAL,
+                 "bimask_wgrad: pointers must be 16-byte aligned");
+  const WsPlan w = plan_ws(T, I, J, 0);
+  float* partials = nullptr;
+  if (w.part_bytes) {
+    BIMASK_REQUIRE(ws && ws_bytes >= w.part_off + w.part_bytes, BIMASK_EINVAL,
+                   "bimask_wgrad: workspace too small (%zu bytes, need %zu)", ws_bytes, w.part_off + w.part_bytes);
+    partials = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(ws) + w.part_off);
+  }
+  return launch_wgrad_impl(dY, X, T, I, J, dW, partials, status_word, (cudaStream_t)stream);
+}
+
+int bimask_layer_step(const bimask_layer_args* a) {
+  BIMASK_REQUIRE(a != nullptr, BIMASK_EINVAL, "bimask_layer_step: null argument block");
+  int rc = check_shape(a->I, a->J, a->N, a->M);
+  if (rc != BIMASK_OK) return rc;
+  if ((rc = check_gemm(a->T, a->I, a->J)) != BIMASK_OK) return rc;
+  BIMASK_REQUIRE(a->perm && a->ws && a->status_word, BIMASK_EINVAL, "bimask_layer_step: null pointer");
+  const size_t need = plan_ws(a->T, a->I, a->J, a->do_search ? a->P : 0).total;
+  BIMASK_REQUIRE(a->ws_bytes >= need, BIMASK_EINVAL, "bimask_layer_step: workspace too small (%zu bytes, need %zu)",
+                 a->ws_bytes, need);
+  // scratch is reused in stream order: the candidates are consumed by the pick before the
+  // permuted copy of dY is written over them; the split-K partials sit behind that copy
+  if ((rc = bimask_fwd_mask(a->W, a->I, a->J, a->N, a->M, a->maskbits_f, a->vals_f, a->meta_f, a->hw_meta_f, a->stream)))
+    return rc;
+  if ((rc = bimask_spmm_fwd(a->X, a->vals_f, a->hw_meta_f, a->T, a->I, a->J, a->Y, a->status_word, a->stream))) return rc;
+  if (a->do_search) {
+    if ((rc = bimask_perm_search(a->maskbits_f, a->I, a->J, a->N, a->M, a->P, a->seed, a->cands, a->perm, a->best_idx,
+                                 a->counts, a->ws, a->ws_bytes, a->stream)))
+      return rc;
+  }
+  if ((rc = bimask_bwd_mask(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->M, a->maskbits_b, a->vals_b, a->meta_b,
+                            a->hw_meta_b, a->stream)))
+    return rc;
+  if ((rc = bimask_spmm_dgrad(a->dY, a->perm, a->vals_b, a->hw_meta_b, a->T, a->I, a->J, a->dX, a->ws, a->ws_bytes,
+                              a->status_word, a->stream)))
+    return rc;
+  return bimask_wgrad(a->dY, a->X, a->T, a->I, a->J, a->dW, a->ws, a->ws_bytes, a->status_word, a->stream);
+}
+
+int bimask_layer_step_host(const bimask_layer_args* d, const bimask_layer_args* h, int32_t* host_status_word) {
+  BIMASK_REQUIRE(d && h, BIMASK_EINVAL, "bimask_layer_step_host: null argument block");
+  cudaStream_t s = (cudaStream_t)d->stream;
+  const size_t IJ = (size_t)d->I * d->J, TJ = (size_t)d->T * d->J, TI = (size_t)d->T * d->I;
+  BIMASK_REQUIRE(h->W && h->X && h->dY, BIMASK_EINVAL, "bimask_layer_step_host: host W, X and dY are required");
+  BIMASK_CUDA_OK(cudaMemcpyAsync(const_cast<float*>(d->W), h->W, IJ * 4, cudaMemcpyHostToDevice, s));
+  BIMASK_CUDA_OK(cudaMemcpyAsync(const_cast<uint16_t*>(d->X), h->X, TJ * 2, cudaMemcpyHostToDevice, s));
+  BIMASK_CUDA_OK(cudaMemcpyAsync(const_cast<uint16_t*>(d->dY), h->dY, TI * 2, cudaMemcpyHostToDevice, s));
+  if (!d->do_search && h->perm)
+    BIMASK_CUDA_OK(cudaMemcpyAsync(d->perm, h->perm, (size_t)d->I * 4, cudaMemcpyHostToDevice, s));
+  if (d->do_search && d->cands && h->cands)
+    BIMASK_CUDA_OK(cudaMemcpyAsync(const_cast<int32_t*>(d->cands), h->cands, (size_t)d->P * d->I * 4,
+                                   cudaMemcpyHostToDevice, s));
+  BIMASK_CUDA_OK(cudaMemsetAsync(d->status_word, 0, sizeof(int32_t), s));
+  int rc = bimask_layer_step(d);
+  if (rc != BIMASK_OK) return rc;
+  if (h->Y) BIMASK_CUDA_OK(cudaMemcpyAsync(h->Y, d->Y, TI * 2, cudaMemcpyDeviceToHost, s));
+  if (h->dX) BIMASK_CUDA_OK(cudaMemcpyAsync(h->dX, d->dX, TJ * 2, cudaMemcpyDeviceToHost, s));
+  if (h->dW) BIMASK_CUDA_OK(cudaMemcpyAsync(h->dW, d->dW, IJ * 4, cudaMemcpyDeviceToHost, s));
+  if (h->perm) BIMASK_CUDA_OK(cudaMemcpyAsync(h->perm, d->perm, (size_t)d->I * 4, cudaMemcpyDeviceToHost, s));
+  if (d->do_search && h->best_idx)
+    BIMASK_CUDA_OK(cudaMemcpyAsync(h->best_idx, d->best_idx, 4, cudaMemcpyDeviceToHost, s));
+  if (d->do_search && h->counts)
+    BIMASK_CUDA_OK(cudaMemcpyAsync(h->counts, d->counts, (size_t)d->P * 8, cudaMemcpyDeviceToHost, s));
+  if (h->maskbits_f) BIMASK_CUDA_OK(cudaMemcpyAsync(h->maskbits_f, d->maskbits_f, IJ / 8, cudaMemcpyDeviceToHost, s));
+  if (h->maskbits_b) BIMASK_CUDA_OK(cudaMemcpyAsync(h->maskbits_b, d->maskbits_b, IJ / 8, cudaMemcpyDeviceToHost, s));
+  if (host_status_word)
+    BIMASK_CUDA_OK(cudaMemcpyAsync(host_status_word, d->status_word, 4, cudaMemcpyDeviceToHost, s));
+  BIMASK_CUDA_OK(cudaStreamSynchronize(s));
+  return BIMASK_OK;
+}
+
+int bimask_check_perms(const int32_t* cands, int P, int I, int32_t* ok, void* ws, size_t ws_bytes, void* stream) {
+  BIMASK_REQUIRE(cands && ok && ws && P >= 1 && I >= 1, BIMASK_EINVAL, "bimask_check_perms: bad argument");
+  BIMASK_REQUIRE(ws_bytes >= (size_t)P * I, BIMASK_EINVAL, "bimask_check_perms: workspace too small");
+  return launch_check_perms(cands, P, I, ok, reinterpret_cast<uint8_t*>(ws), (cudaStream_t)stream);
+}
+
+}  // extern "C"

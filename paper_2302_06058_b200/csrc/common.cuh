@@ -1,0 +1,50 @@
+// Shared host-side plumbing of the library: status codes, the per-thread error text and
+// launch checking.  Device code in the other files includes this for the small bit helpers.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <stdarg.h>
+#include "../../include/bimask.h"
+
+namespace bimask {
+
+void set_error(const char* fmt, ...);       // defined in api.cu
+int cuda_fail(cudaError_t e, const char* what);
+
+#define BIMASK_CUDA_OK(call)                                   \
+  do {                                                         \
+    cudaError_t e__ = (call);                                  \
+    if (e__ != cudaSuccess) return ::bimask::cuda_fail(e__, #call); \
+  } while (0)
+
+#define BIMASK_REQUIRE(cond, code, ...)        \
+  do {                                         \
+    if (!(cond)) {                             \
+      ::bimask::set_error(__VA_ARGS__);        \
+      return (code);                           \
+    }                                          \
+  } while (0)
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Launchers implemented in the .cu files (all enqueue on `s`, none synchronise).
+int launch_fwd_mask(const float* W, int I, int J, int N, uint32_t* maskbits, uint16_t* vals,
+                    uint32_t* meta, cudaStream_t s);
+int launch_hw_meta(const uint32_t* meta, int rows, int K, void* hw_meta, cudaStream_t s);
+int launch_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
+                    int N, uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, cudaStream_t s);
+int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStream_t s);
+int launch_score(const uint32_t* maskbits_f, const int32_t* cands, int I, int J, int N, int P,
+                 int64_t* counts, cudaStream_t s);
+int launch_pick(const int64_t* counts, const int32_t* cands, int P, int I, int32_t* best_idx,
+                int32_t* best_perm, cudaStream_t s);
+int launch_check_perms(const int32_t* cands, int P, int I, int32_t* ok, uint8_t* seen, cudaStream_t s);
+int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, uint16_t* dYp, cudaStream_t s);
+int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim, int Kdim,
+                uint16_t* out, int32_t* status_word, cudaStream_t s);
+void wgrad_plan(int T, int I, int J, int* n_tile, int* splits, int* k_tiles_per_split);
+int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J, float* dW, float* partials,
+                      int32_t* status_word, cudaStream_t s);
+
+}  // namespace bimask

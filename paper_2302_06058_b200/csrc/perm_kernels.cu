@@ -1,0 +1,218 @@
+// Row-permutation search of Alg. 1: candidate generation, eligible-block counting and the pick.
+//
+// Counting works on the forward mask BITS (I x J/32 words, 1/32 of the weight bytes, resident in
+// L2): a block of M = 4 permuted rows is tested for 32 columns at a time with a handful of
+// AND/OR operations on the four row words and a popcount.
+#include "common.cuh"
+
+namespace bimask {
+
+namespace {
+
+__device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
+  z ^= z >> 30;
+  z *= 0xBF58476D1CE4E5B9ull;
+  z ^= z >> 27;
+  z *= 0x94D049BB133111EBull;
+  z ^= z >> 31;
+  return z;
+}
+
+// ---------------------------------------------------------------------------------------
+// Candidate generation: one CTA per candidate sorts the I hashed keys in shared memory
+// (bitonic network on the next power of two, padding keys = all ones sort to the end).
+// ---------------------------------------------------------------------------------------
+constexpr int GEN_THREADS = 1024;
+
+__global__ void __launch_bounds__(GEN_THREADS)
+gen_candidates_kernel(unsigned long long seed, int I, int n_pow2, int32_t* __restrict__ cands) {
+  extern __shared__ unsigned long long keys[];
+  const int c = blockIdx.x;
+  const unsigned long long stream = mix64(seed + 0x9E3779B97F4A7C15ull * (unsigned long long)(c + 1));
+  for (int i = threadIdx.x; i < n_pow2; i += GEN_THREADS) {
+    unsigned long long v = ~0ull;
+    if (i < I) v = (mix64(stream ^ (unsigned long long)i) & ~0xFFFFFFull) | (unsigned long long)i;
+    keys[i] = v;
+  }
+  __syncthreads();
+  for (int k = 2; k <= n_pow2; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int t = threadIdx.x; t < (n_pow2 >> 1); t += GEN_THREADS) {
+        const int lo = ((t & ~(j - 1)) << 1) | (t & (j - 1));   // element with bit j clear
+        const int hi = lo | j;
+        const bool up = (lo & k) == 0;
+        const unsigned long long a = keys[lo], b = keys[hi];
+        if ((a > b) == up) { keys[lo] = b; keys[hi] = a; }
+      }
+      __syncthreads();
+    }
+  }
+  for (int i = threadIdx.x; i < I; i += GEN_THREADS)
+    cands[(long long)c * I + i] = (int32_t)(keys[i] & 0xFFFFFFull);
+}
+
+// ---------------------------------------------------------------------------------------
+// Eligible-block count.  grid = (row-block chunks, P).  A warp takes one row block of a
+// candidate at a time: the four row indices are one 16-byte load, each lane then reads its
+// slice of the four mask rows (128-bit loads when J % 128 == 0) and counts columns whose
+// four bits hold at most N ones.  One 64-bit atomic per CTA.
+// ---------------------------------------------------------------------------------------
+constexpr int SCORE_THREADS = 256;
+constexpr int SCORE_KB_PER_CTA = 64;
+
+template <int N>
+__device__ __forceinline__ uint32_t ineligible(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  if (N == 1) return (a & b) | (c & d) | ((a | b) & (c | d));     // two or more set
+  if (N == 2) return (a & b & (c | d)) | (c & d & (a | b));       // three or more set
+  if (N == 3) return a & b & c & d;
+  return 0u;
+}
+
+template <int N>
+__global__ void __launch_bounds__(SCORE_THREADS)
+score_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cands, int I, int jwords,
+             unsigned long long* __restrict__ counts) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int c = blockIdx.y;
+  const int nkb = I >> 2;
+  const int kb0 = blockIdx.x * SCORE_KB_PER_CTA;
+  const int kb1 = min(nkb, kb0 + SCORE_KB_PER_CTA);
+  const int4* cand4 = reinterpret_cast<const int4*>(cands + (long long)c * I);
+  uint32_t cnt = 0;
+  if ((jwords & 3) == 0) {
+    const int jq = jwords >> 2;
+    for (int k = kb0 + warp; k < kb1; k += SCORE_THREADS / 32) {
+      const int4 r = __ldg(cand4 + k);
+      const uint4* r0 = reinterpret_cast<const uint4*>(bits + (long long)r.x * jwords);
+      const uint4* r1 = reinterpret_cast<const uint4*>(bits + (long long)r.y * jwords);
+      const uint4* r2 = reinterpret_cast<const uint4*>(bits + (long long)r.z * jwords);
+      const uint4* r3 = reinterpret_cast<const uint4*>(bits + (long long)r.w * jwords);
+      for (int q = lane; q < jq; q += 32) {
+        const uint4 a = __ldg(r0 + q), b = __ldg(r1 + q), cc = __ldg(r2 + q), d = __ldg(r3 + q);
+        cnt += __popc(~ineligible<N>(a.x, b.x, cc.x, d.x)) + __popc(~ineligible<N>(a.y, b.y, cc.y, d.y)) +
+               __popc(~ineligible<N>(a.z, b.z, cc.z, d.z)) + __popc(~ineligible<N>(a.w, b.w, cc.w, d.w));
+      }
+    }
+  } else {
+    for (int k = kb0 + warp; k < kb1; k += SCORE_THREADS / 32) {
+      const int4 r = __ldg(cand4 + k);
+      const uint32_t* r0 = bits + (long long)r.x * jwords;
+      const uint32_t* r1 = bits + (long long)r.y * jwords;
+      const uint32_t* r2 = bits + (long long)r.z * jwords;
+      const uint32_t* r3 = bits + (long long)r.w * jwords;
+      for (int q = lane; q < jwords; q += 32)
+        cnt += __popc(~ineligible<N>(__ldg(r0 + q), __ldg(r1 + q), __ldg(r2 + q), __ldg(r3 + q)));
+    }
+  }
+  cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+  __shared__ uint32_t part[SCORE_THREADS / 32];
+  if (lane == 0) part[warp] = cnt;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long s = 0;
+#pragma unroll
+    for (int w = 0; w < SCORE_THREADS / 32; ++w) s += part[w];
+    atomicAdd(counts + c, s);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Pick: arg-max of counts with ties to the lowest candidate index, then copy that candidate.
+// ---------------------------------------------------------------------------------------
+constexpr int PICK_THREADS = 256;
+
+__global__ void __launch_bounds__(PICK_THREADS)
+pick_kernel(const long long* __restrict__ counts, const int32_t* __restrict__ cands, int P, int I,
+            int32_t* __restrict__ best_idx, int32_t* __restrict__ best_perm) {
+  __shared__ long long s_cnt[PICK_THREADS];
+  __shared__ int s_idx[PICK_THREADS];
+  long long bc = -1;
+  int bi = 0x7FFFFFFF;
+  for (int c = threadIdx.x; c < P; c += PICK_THREADS) {
+    const long long v = counts[c];
+    if (v > bc) { bc = v; bi = c; }      // ascending c per thread: first maximum is kept
+  }
+  s_cnt[threadIdx.x] = bc;
+  s_idx[threadIdx.x] = bi;
+  __syncthreads();
+  for (int s = PICK_THREADS / 2; s > 0; s >>= 1) {
+    if (threadIdx.x < s) {
+      const long long oc = s_cnt[threadIdx.x + s];
+      const int oi = s_idx[threadIdx.x + s];
+      if (oc > s_cnt[threadIdx.x] || (oc == s_cnt[threadIdx.x] && oi < s_idx[threadIdx.x])) {
+        s_cnt[threadIdx.x] = oc;
+        s_idx[threadIdx.x] = oi;
+      }
+    }
+    __syncthreads();
+  }
+  const int best = s_idx[0];
+  if (threadIdx.x == 0) *best_idx = best;
+  for (int i = threadIdx.x; i < I; i += PICK_THREADS) best_perm[i] = cands[(long long)best * I + i];
+}
+
+// Debug: every row of cands is a permutation of 0..I-1.
+__global__ void check_perms_kernel(const int32_t* __restrict__ cands, int P, int I,
+                                   uint8_t* __restrict__ seen, int32_t* __restrict__ ok) {
+  const int c = blockIdx.x;
+  for (int i = threadIdx.x; i < I; i += blockDim.x) {
+    const int v = cands[(long long)c * I + i];
+    if (v < 0 || v >= I) { atomicExch(ok, 0); continue; }
+    seen[(long long)c * I + v] = 1;
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < I; i += blockDim.x)
+    if (!seen[(long long)c * I + i]) atomicExch(ok, 0);
+}
+
+__global__ void set_int_kernel(int32_t* p, int32_t v) { *p = v; }
+
+}  // namespace
+
+int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStream_t s) {
+  int n = 2;
+  while (n < I) n <<= 1;
+  const size_t smem = (size_t)n * sizeof(unsigned long long);
+  static bool attr_done = false;     // same value every time; a race only repeats the call
+  if (!attr_done) {
+    BIMASK_CUDA_OK(cudaFuncSetAttribute(gen_candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        16384 * (int)sizeof(unsigned long long)));
+    attr_done = true;
+  }
+  gen_candidates_kernel<<<P, GEN_THREADS, smem, s>>>((unsigned long long)seed, I, n, cands);
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
+int launch_score(const uint32_t* maskbits_f, const int32_t* cands, int I, int J, int N, int P,
+                 int64_t* counts, cudaStream_t s) {
+  BIMASK_CUDA_OK(cudaMemsetAsync(counts, 0, (size_t)P * sizeof(int64_t), s));
+  dim3 grid((I / 4 + SCORE_KB_PER_CTA - 1) / SCORE_KB_PER_CTA, P);
+  unsigned long long* cnt = reinterpret_cast<unsigned long long*>(counts);
+  switch (N) {
+    case 1: score_kernel<1><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt); break;
+    case 2: score_kernel<2><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt); break;
+    case 3: score_kernel<3><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt); break;
+    default: score_kernel<4><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt); break;
+  }
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
+int launch_pick(const int64_t* counts, const int32_t* cands, int P, int I, int32_t* best_idx,
+                int32_t* best_perm, cudaStream_t s) {
+  pick_kernel<<<1, PICK_THREADS, 0, s>>>(reinterpret_cast<const long long*>(counts), cands, P, I,
+                                         best_idx, best_perm);
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
+int launch_check_perms(const int32_t* cands, int P, int I, int32_t* ok, uint8_t* seen, cudaStream_t s) {
+  BIMASK_CUDA_OK(cudaMemsetAsync(seen, 0, (size_t)P * I, s));
+  set_int_kernel<<<1, 1, 0, s>>>(ok, 1);
+  check_perms_kernel<<<P, 256, 0, s>>>(cands, P, I, seen, ok);
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
+}  // namespace bimask

@@ -1,0 +1,218 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Integer outputs (mask bits, packed values and codes, counts, the chosen
+permutation) must match bit for bit; products within max |y - ref| / max(|ref|, rms(ref)) <= 2e-2
+(bf16 inputs, fp32 accumulation, bf16 outputs for Y and dX)."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2302_06058_b200 as bm
+from oracle import bimask_oracle as O
+from paper_2302_06058_b200 import inputs
+from tests.gpu_util import bits_dev, dev, rel_err, run_fwd_mask, run_layer_step, u16, u32
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+
+
+def special_weights(I, J, seed):
+    """Normal weights with planted ties, zeros, negative zeros, denormals, inf and NaN."""
+    rng = np.random.default_rng(seed)
+    W = rng.standard_normal((I, J)).astype(np.float32)
+    W[rng.random((I, J)) < 0.15] = 0.0
+    W[rng.random((I, J)) < 0.05] = -0.0
+    t = rng.random((I, J)) < 0.2
+    W[t] = np.round(W[t] * 2) / 2                       # many equal magnitudes
+    W[0, :8] = [np.inf, -np.inf, 1.0, np.nan, 1e-41, -1e-41, 3.0, -3.0]
+    return W
+
+
+@pytest.mark.parametrize("I,J,N", [(256, 256, 2), (32, 32, 2), (64, 576, 2), (96, 160, 1), (512, 4608, 1),
+                                   (1152, 384, 2), (2048, 1056, 2)])
+def test_fwd_mask_bit_exact(I, J, N):
+    W = special_weights(I, J, I + J + N) if I < 1000 else inputs.make_weight(I, J, 5)
+    _, b = run_fwd_mask(W, N)
+    B = O.forward_mask(W, N, 4)
+    bits, vals, meta = O.forward_operand(W, B)
+    assert np.array_equal(u32(b["maskbits_f"]), bits)
+    assert np.array_equal(u32(b["meta_f"]), meta)
+    assert np.array_equal(u16(b["vals_f"]), vals)
+
+
+@pytest.mark.parametrize("I,J,N", [(256, 256, 2), (32, 32, 1), (64, 576, 2), (96, 160, 1), (512, 1184, 2),
+                                   (1152, 384, 2)])
+def test_bwd_mask_bit_exact(I, J, N):
+    W = special_weights(I, J, 3 * I + J + N)
+    Wd, b = run_fwd_mask(W, N)
+    perm = np.random.default_rng(I).permutation(I).astype(np.int32)
+    pd = dev(perm)
+    bm.bimask_bwd_mask(Wd, b["maskbits_f"], pd, I, J, N, 4, b["maskbits_b"], b["vals_b"], b["meta_b"], b["hw_meta_b"])
+    torch.cuda.synchronize()
+    B = O.forward_mask(W, N, 4)
+    Bbar = O.backward_mask(W, B, perm, N, 4)
+    bits, vals, meta = O.backward_operand(W, Bbar, perm)
+    assert np.array_equal(u32(b["maskbits_b"]), bits)
+    assert np.array_equal(u32(b["meta_b"]), meta)
+    assert np.array_equal(u16(b["vals_b"]), vals)
+
+
+@pytest.mark.parametrize("I,J,N,P", [(256, 256, 2, 8), (64, 576, 2, 32), (512, 4608, 1, 64), (1152, 384, 2, 32),
+                                     (100, 96, 2, 5), (16384, 64, 2, 3)])
+def test_perm_search_generated(I, J, N, P):
+    W = inputs.make_weight(I, J, I + P)
+    B = O.forward_mask(W, N, 4)
+    bits = dev(O.pack_bits(B).view(np.int32))
+    ws_bytes = bm.bimask_workspace_bytes(1, I, J, P)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    best_perm = torch.empty(I, dtype=torch.int32, device="cuda")
+    best_idx = torch.empty(1, dtype=torch.int32, device="cuda")
+    counts = torch.empty(P, dtype=torch.int64, device="cuda")
+    seed = 42 + I
+    bm.bimask_perm_search(bits, I, J, N, 4, P, seed, None, best_perm, best_idx, counts, ws, ws_bytes)
+    torch.cuda.synchronize()
+    cands = O.candidates(seed, P, I)
+    best, perm, cnt = O.perm_search(B, cands, N, 4)
+    got_cands = ws[: P * I * 4].view(torch.int32).view(P, I).cpu().numpy()
+    assert np.array_equal(got_cands, cands)
+    assert np.array_equal(counts.cpu().numpy(), cnt)
+    assert int(best_idx.item()) == best
+    assert np.array_equal(best_perm.cpu().numpy(), perm)
+    ok = torch.zeros(1, dtype=torch.int32, device="cuda")
+    scratch = torch.empty(P * I, dtype=torch.uint8, device="cuda")
+    bm.bimask_check_perms(ws[: P * I * 4].view(torch.int32), P, I, ok, scratch, P * I)
+    assert int(ok.item()) == 1
+
+
+def test_perm_search_all_permutations_of_8_rows():
+    """All 8! explicit candidates on the hand-worked 8 x 8 example (tiled to 32 columns, so every
+    count is four times the 8 x 8 one): counts and the first maximiser must match."""
+    from tests.test_oracle_pins import _read_example, brute_count
+    W8, B8, _ = _read_example()
+    B = np.tile(B8, (1, 4))
+    allp = np.array(list(itertools.permutations(range(8))), dtype=np.int32)
+    P = allp.shape[0]
+    bits = dev(O.pack_bits(B).view(np.int32))
+    best_perm = torch.empty(8, dtype=torch.int32, device="cuda")
+    best_idx = torch.empty(1, dtype=torch.int32, device="cuda")
+    counts = torch.empty(P, dtype=torch.int64, device="cuda")
+    bm.bimask_perm_search(bits, 8, 32, 2, 4, P, 0, dev(allp), best_perm, best_idx, counts, None, 0)
+    torch.cuda.synchronize()
+    ref8 = np.array([brute_count(B8, p, 2, 4) for p in allp])
+    got = counts.cpu().numpy()
+    assert np.array_equal(got, 4 * ref8)
+    first = int(np.nonzero(ref8 == 16)[0][0])
+    assert int(best_idx.item()) == first
+    assert np.array_equal(best_perm.cpu().numpy(), allp[first])
+    best, perm, cnt = O.perm_search(B, allp, 2, 4)
+    assert best == first and np.array_equal(cnt, got)
+
+
+def test_planted_permutation_wins():
+    I, J, N = 256, 512, 2
+    W, Q = inputs.planted_transposable(I, J, N, 4, 77)
+    rng = np.random.default_rng(1)
+    cands = np.stack([rng.permutation(I) for _ in range(6)] + [Q] + [rng.permutation(I) for _ in range(4)]).astype(np.int32)
+    X = inputs.make_activation(64, J, 1)
+    dY = inputs.make_activation(64, I, 2)
+    b = run_layer_step(W, X, dY, N, 4, cands.shape[0], 0, do_search=True, cands=cands)
+    assert int(b["best_idx"].item()) == 6
+    assert int(b["counts"][6].item()) == (I // 4) * J
+    assert np.array_equal(b["perm"].cpu().numpy(), Q)
+    B = O.forward_mask(W, N, 4)
+    assert np.array_equal(u32(b["maskbits_b"]), O.pack_bits(B[Q]))        # B-bar == B[perm]
+    exact = O.dense_dgrad(dY, W, B)                                         # Eq. 5
+    got = b["dX"].float().cpu().numpy()
+    assert rel_err(got, exact) <= TOL
+
+
+GEMM_SHAPES = [  # (I, J, T, N)
+    (256, 256, 128, 2),      # config 1
+    (128, 128, 128, 2),      # exactly one tile
+    (64, 576, 300, 2),       # rows < tile, ragged reduction (576 = 4.5 x 128), ragged tokens
+    (384, 384, 129, 1),      # 1:4 in the 2:4 container, T = tile + 1
+    (160, 96, 1, 2),         # a single token
+    (512, 1184, 1568, 2),    # several tiles each way with ragged tails
+]
+
+
+@pytest.mark.parametrize("I,J,T,N", GEMM_SHAPES)
+def test_layer_step_parity(I, J, T, N):
+    W = inputs.make_weight(I, J, 11 * I + J)
+    X = inputs.make_activation(T, J, 5 * I + T)
+    dY = inputs.make_activation(T, I, 7 * J + T)
+    P, seed = 6, 1234 + I
+    b = run_layer_step(W, X, dY, N, 4, P, seed, do_search=True)
+    ref = O.layer_step(W, X, dY, N, 4, P, seed, do_search=True)
+    assert int(b["status_word"].item()) == 0
+    assert np.array_equal(u32(b["maskbits_f"]), ref["maskbits_f"])
+    assert np.array_equal(u32(b["meta_f"]), ref["meta_f"])
+    assert np.array_equal(u16(b["vals_f"]), ref["vals_f"])
+    assert np.array_equal(b["counts"].cpu().numpy(), ref["counts"])
+    assert int(b["best_idx"].item()) == ref["best_idx"]
+    assert np.array_equal(b["perm"].cpu().numpy(), ref["perm"])
+    assert np.array_equal(u32(b["maskbits_b"]), ref["maskbits_b"])
+    assert np.array_equal(u32(b["meta_b"]), ref["meta_b"])
+    assert np.array_equal(u16(b["vals_b"]), ref["vals_b"])
+    assert rel_err(b["Y"].float().cpu().numpy(), ref["Y"]) <= TOL
+    assert rel_err(b["dX"].float().cpu().numpy(), ref["dX"]) <= TOL
+    assert rel_err(b["dW"].cpu().numpy(), ref["dW"]) <= TOL
+
+
+def test_metadata_round_trip_through_the_tensor_core():
+    """Multiply the packed forward operand by an identity activation: the product must be the
+    masked, bf16-rounded weight itself, exactly (pins the opaque metadata order)."""
+    I = J = T = 256
+    W = inputs.make_weight(I, J, 99)
+    Wd, b = run_fwd_mask(W, 2)
+    X = torch.eye(J, dtype=torch.bfloat16, device="cuda")
+    Y = torch.empty(T, I, dtype=torch.bfloat16, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    bm.bimask_spmm_fwd(X, b["vals_f"], b["hw_meta_f"], T, I, J, Y, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    B = O.forward_mask(W, 2, 4)
+    expect = (O.bf16_round(W) * B).T                  # Y[t, i] = (B*W)[i, t]
+    assert np.array_equal(Y.float().cpu().numpy().astype(np.float64), expect)
+
+
+def test_do_search_zero_uses_given_perm():
+    I, J, T = 128, 160, 70
+    W = inputs.make_weight(I, J, 3)
+    X = inputs.make_activation(T, J, 4)
+    dY = inputs.make_activation(T, I, 5)
+    perm = np.random.default_rng(9).permutation(I).astype(np.int32)
+    b = run_layer_step(W, X, dY, 2, 4, 1, 0, do_search=False, perm=perm)
+    ref = O.layer_step(W, X, dY, 2, 4, 1, 0, do_search=False, perm=perm)
+    assert np.array_equal(b["perm"].cpu().numpy(), perm)
+    assert np.array_equal(u32(b["maskbits_b"]), ref["maskbits_b"])
+    assert rel_err(b["dX"].float().cpu().numpy(), ref["dX"]) <= TOL
+
+
+def test_error_paths_launch_nothing():
+    W = torch.zeros(64, 64, device="cuda")
+    b = bm.alloc_layer_buffers(8, 64, 64, 2)
+    with pytest.raises(bm.BimaskError) as e:
+        bm.bimask_fwd_mask(W, 64, 48, 2, 4, b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"])
+    assert e.value.code == bm.binding.BIMASK_EINVAL
+    with pytest.raises(bm.BimaskError) as e:
+        bm.bimask_fwd_mask(W, 64, 64, 2, 8, b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"])
+    assert e.value.code == bm.binding.BIMASK_EUNSUPPORTED
+    with pytest.raises(bm.BimaskError) as e:
+        bm.bimask_fwd_mask(W, 64, 64, 3, 4, b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"])
+    assert e.value.code == bm.binding.BIMASK_EUNSUPPORTED
+    with pytest.raises(bm.BimaskError) as e:
+        bm.bimask_fwd_mask(None, 64, 64, 2, 4, b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"])
+    assert e.value.code == bm.binding.BIMASK_EINVAL
+    with pytest.raises(bm.BimaskError) as e:     # misaligned pointer
+        bm.bimask_fwd_mask(W.data_ptr() + 4, 64, 64, 2, 4, b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"])
+    assert e.value.code == bm.binding.BIMASK_EINVAL
+    with pytest.raises(bm.BimaskError) as e:     # P = 0
+        bm.bimask_perm_search(b["maskbits_f"], 64, 64, 2, 4, 0, 1, None, b["perm"], b["best_idx"], b["counts"], b["ws"], 1 << 20)
+    assert e.value.code == bm.binding.BIMASK_EINVAL
+    with pytest.raises(bm.BimaskError) as e:     # workspace too small
+        bm.bimask_perm_search(b["maskbits_f"], 64, 64, 2, 4, 2, 1, None, b["perm"], b["best_idx"], b["counts"], b["ws"], 16)
+    assert e.value.code == bm.binding.BIMASK_EINVAL
+    assert "workspace" in bm.bimask_last_error()
+    torch.cuda.synchronize()
