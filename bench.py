@@ -1,0 +1,397 @@
+#!/usr/bin/env python
+"""Benchmark of the Bi-Mask layer step (mask + permutation search + three GEMMs).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+A "step" is one pass of the whole hot path (Alg. 1 body without the optimizer: forward mask and
+pack, permutation search, backward mask and pack, sparse forward, sparse input gradient, dense
+weight gradient) over every layer of the configuration; the metric is layer-steps per second.
+One JSON line is printed by rank 0.  With N > 1 (torchrun) every rank runs an independent replica
+(the step has no exchange between GPUs), and the value is the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "bimask_layer_steps_per_sec"
+UNIT = "layer-steps/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+# --------------------------------------------------------------------------------------------
+# CPU oracle arm (reference / cpu_baseline)
+# --------------------------------------------------------------------------------------------
+def oracle_sample_time(cfg_id: int, rows: int = 1024, tokens: int = 256, cands: int = 4):
+    """Times the CPU oracle, as it stands, on a bounded sample of every layer of the config
+    (the first `rows` rows of W with the full input dim, `tokens` tokens, `cands` candidates) and
+    scales each part by its own work ratio to the full layer.  Returns (seconds for a full pass
+    over all layers [extrapolated], seconds actually spent, description)."""
+    from oracle import bimask_oracle as O
+    from paper_2302_06058_b200 import inputs
+    cfg = inputs.CONFIGS[cfg_id]
+    total_full = 0.0
+    spent = 0.0
+    for li, L in enumerate(cfg.layers):
+        Is, Ts, Ps = min(rows, L.I), min(tokens, L.T), min(cands, cfg.P)
+        W = inputs.make_weight(Is, L.J, 1000 * cfg_id + 10 * li, cfg.init)
+        X = inputs.make_activation(Ts, L.J, 1000 * cfg_id + 10 * li + 1)
+        dY = inputs.make_activation(Ts, Is, 1000 * cfg_id + 10 * li + 2)
+        t0 = time.perf_counter()
+        B = O.forward_mask(W, cfg.N, cfg.M)
+        O.forward_operand(W, B)
+        t1 = time.perf_counter()
+        cand = O.candidates(inputs.perm_seed(cfg_id), Ps, Is)
+        _, perm, _ = O.perm_search(B, cand, cfg.N, cfg.M)
+        t2 = time.perf_counter()
+        Bbar = O.backward_mask(W, B, perm, cfg.N, cfg.M)
+        Mb = O.unpermute_rows(Bbar, perm)
+        O.backward_operand(W, Bbar, perm)
+        t3 = time.perf_counter()
+        O.spmm_fwd(X, W, B)
+        O.spmm_dgrad(dY, W, Mb)
+        O.wgrad(dY, X)
+        t4 = time.perf_counter()
+        r_mask = (L.I * L.J) / (Is * L.J)
+        r_search = (cfg.P * L.I * L.J) / (Ps * Is * L.J)
+        r_gemm = (L.T * L.I * L.J) / (Ts * Is * L.J)
+        total_full += ((t1 - t0) + (t3 - t2)) * r_mask + (t2 - t1) * r_search + (t4 - t3) * r_gemm
+        spent += t4 - t0
+    desc = (f"config {cfg_id}: per layer the first {rows} rows of W (full input dim), {tokens} tokens, "
+            f"{cands} candidates; masks, search and GEMMs timed separately and each scaled by its work "
+            f"ratio to the full layer (extrapolated)")
+    return total_full, spent, desc
+
+
+def cpu_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+        return int(n)
+    except Exception:
+        return len(os.sched_getaffinity(0))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2302_06058_b200 import inputs
+    cfg = inputs.CONFIGS[args.config]
+    for _ in range(args.warmup):
+        oracle_sample_time(args.config, rows=128, tokens=32, cands=1)
+    per_pass = []
+    t_begin = time.perf_counter()
+    for _ in range(args.steps):
+        full, _, desc = oracle_sample_time(args.config, rows=args.ref_rows, tokens=args.ref_tokens, cands=2)
+        per_pass.append(full)
+    wall = time.perf_counter() - t_begin
+    sec = float(np.mean(per_pass))
+    value = len(cfg.layers) / sec
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"config {args.config} ({cfg.name})", "layers": [[L.I, L.J, L.T] for L in cfg.layers],
+                   "N": cfg.N, "M": cfg.M, "P": cfg.P},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0, "wall_s": wall,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------
+# clocks sampler
+# --------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.gpu_id = gpu_id
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            with open(self.path) as f:
+                for line in f:
+                    p = [x.strip() for x in line.split(",")]
+                    if len(p) < 8:
+                        continue
+                    try:
+                        sm.append(float(p[0]))
+                        mx.append(float(p[1]))
+                    except ValueError:
+                        continue
+                    for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[4:8]):
+                        if v.lower().startswith("active"):
+                            reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# --------------------------------------------------------------------------------------------
+# GPU arm
+# --------------------------------------------------------------------------------------------
+def algorithmic_work(L, P):
+    """Algorithmic bytes / flops per launch of each timed call for one layer (see the design notes)."""
+    I, J, T = L.I, L.J, L.T
+    IJ = I * J
+    return {
+        "fwd_mask": {"bound": "hbm", "bytes": 4 * IJ + IJ + IJ / 8 + IJ / 8 + 2 * IJ / 8},
+        "perm_search": {"bound": "hbm", "bytes": 4 * IJ},      # time relative to one pass over W
+        "bwd_mask": {"bound": "hbm", "bytes": 4 * IJ + IJ / 8 + 4 * I + IJ + IJ / 8 + IJ / 8 + 2 * IJ / 8},
+        "spmm_fwd": {"bound": "tensor", "flops": 2.0 * T * IJ, "bytes": 2 * T * J + 1.125 * IJ + 2 * T * I},
+        "spmm_dgrad": {"bound": "tensor", "flops": 2.0 * T * IJ, "bytes": 2 * T * I + 1.125 * IJ + 2 * T * J + 4 * T * I},
+        "wgrad": {"bound": "tensor", "flops": 2.0 * T * IJ, "bytes": 2 * T * I + 2 * T * J + 4 * IJ},
+    }
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2302_06058_b200 as bm
+    from paper_2302_06058_b200 import inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    cfg = inputs.CONFIGS[args.config]
+    seed = inputs.perm_seed(args.config)
+    peaks = load_peaks()
+    stream = torch.cuda.current_stream()
+
+    layers = []
+    host = []
+    for li, L in enumerate(cfg.layers):
+        W, X, dY = inputs.make_layer(args.config, li)
+        b = bm.alloc_layer_buffers(L.T, L.I, L.J, cfg.P)
+        hW = torch.from_numpy(W).pin_memory()
+        hX = torch.from_numpy(X.view(np.int16)).view(torch.bfloat16).pin_memory()
+        hdY = torch.from_numpy(dY.view(np.int16)).view(torch.bfloat16).pin_memory()
+        b["W"], b["X"], b["dY"] = hW.cuda(), hX.cuda(), hdY.cuda()
+        largs = bm.make_layer_args(L.T, L.I, L.J, cfg.N, cfg.M, cfg.P, seed, True, b)
+        layers.append((L, b, largs))
+        host.append({"W": hW, "X": hX, "dY": hdY})
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def one_step():
+        for _, _, largs in layers:
+            bm.bimask_layer_step(largs)
+
+    # ---- warm-up, then the timed region: K steps through bimask_layer_step ----
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    barrier()
+    gpu_uuid = str(local)
+    try:
+        gpu_uuid = "GPU-" + str(torch.cuda.get_device_properties(local).uuid)
+    except Exception:
+        pass
+    sampler = ClockSampler(gpu_uuid)
+    sampler.start()
+    launches0 = bm.bimask_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        one_step()
+    ev1.record(stream)
+    barrier()
+    step_ms_total = ev0.elapsed_time(ev1)
+    launches = bm.bimask_launch_count() - launches0
+
+    # ---- per-call breakdown over the same K steps (CUDA events between the C-ABI calls) ----
+    names = ["fwd_mask", "spmm_fwd", "perm_search", "bwd_mask", "spmm_dgrad", "wgrad"]
+    acc = {li: {n: 0.0 for n in names} for li in range(len(layers))}
+    for _ in range(args.steps):
+        for li, (L, b, _) in enumerate(layers):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(7)]
+            wsb = b["ws"].numel()
+            ev[0].record(stream)
+            bm.bimask_fwd_mask(b["W"], L.I, L.J, cfg.N, cfg.M, b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"])
+            ev[1].record(stream)
+            bm.bimask_spmm_fwd(b["X"], b["vals_f"], b["hw_meta_f"], L.T, L.I, L.J, b["Y"], b["status_word"])
+            ev[2].record(stream)
+            bm.bimask_perm_search(b["maskbits_f"], L.I, L.J, cfg.N, cfg.M, cfg.P, seed, None, b["perm"], b["best_idx"],
+                                  b["counts"], b["ws"], wsb)
+            ev[3].record(stream)
+            bm.bimask_bwd_mask(b["W"], b["maskbits_f"], b["perm"], L.I, L.J, cfg.N, cfg.M, b["maskbits_b"], b["vals_b"],
+                               b["meta_b"], b["hw_meta_b"])
+            ev[4].record(stream)
+            bm.bimask_spmm_dgrad(b["dY"], b["perm"], b["vals_b"], b["hw_meta_b"], L.T, L.I, L.J, b["dX"], b["ws"], wsb,
+                                 b["status_word"])
+            ev[5].record(stream)
+            bm.bimask_wgrad(b["dY"], b["X"], L.T, L.I, L.J, b["dW"], b["ws"], wsb, b["status_word"])
+            ev[6].record(stream)
+            torch.cuda.synchronize()
+            for k, n in enumerate(names):
+                acc[li][n] += ev[k].elapsed_time(ev[k + 1])
+    clocks = sampler.stop()
+    status = [int(b["status_word"].item()) for _, b, _ in layers]
+    if any(status):
+        raise RuntimeError(f"device status words non-zero: {status}")
+
+    # ---- roofline of every call, and of the dominant one ----
+    sparse_peak = 2.0 * peaks["bf16_tflops_sustained"]
+    dense_peak = peaks["bf16_tflops_sustained"]
+    kernels = []
+    for li, (L, b, _) in enumerate(layers):
+        work = algorithmic_work(L, cfg.P)
+        for n in names:
+            ms = acc[li][n] / args.steps
+            w = work[n]
+            entry = {"layer": li, "call": n, "ms": ms}
+            if w["bound"] == "hbm":
+                entry.update(bound="hbm", achieved=w["bytes"] / (ms * 1e-3) / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
+            else:
+                pk = dense_peak if n == "wgrad" else sparse_peak
+                entry.update(bound="tensor", achieved=w["flops"] / (ms * 1e-3) / 1e12, peak=pk, unit="TFLOP/s")
+            entry["frac"] = entry["achieved"] / entry["peak"]
+            kernels.append(entry)
+    dom = max(kernels, key=lambda e: e["ms"])
+    roofline = {"bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"], "unit": dom["unit"],
+                "frac": dom["frac"], "traffic": None, "kernel": f"layer {dom['layer']} {dom['call']}",
+                "peak_source": peaks["source"] + (" (sustained bf16; x2 for the 2:4 sparse products)"
+                                                   if dom["bound"] == "tensor" else " (copy bandwidth)")}
+
+    # ---- end to end through the host-buffer entry point ----
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    host_args = []
+    h2d = d2h = 0
+    for (L, b, largs), hb in zip(layers, host):
+        ho = {"W": hb["W"], "X": hb["X"], "dY": hb["dY"],
+              "Y": torch.empty(L.T, L.I, dtype=torch.bfloat16).pin_memory(),
+              "dX": torch.empty(L.T, L.J, dtype=torch.bfloat16).pin_memory(),
+              "dW": torch.empty(L.I, L.J, dtype=torch.float32).pin_memory(),
+              "perm": torch.empty(L.I, dtype=torch.int32).pin_memory(),
+              "best_idx": torch.empty(1, dtype=torch.int32).pin_memory(),
+              "counts": torch.empty(cfg.P, dtype=torch.int64).pin_memory()}
+        hst = torch.zeros(1, dtype=torch.int32).pin_memory()
+        host_args.append((bm.make_layer_args(L.T, L.I, L.J, cfg.N, cfg.M, cfg.P, seed, True, ho), ho, hst))
+        h2d += sum(hb[k].numel() * hb[k].element_size() for k in ("W", "X", "dY"))
+        d2h += sum(ho[k].numel() * ho[k].element_size() for k in ("Y", "dX", "dW", "perm", "best_idx", "counts")) + 4
+    for (L, b, largs), (ha, _, hst) in zip(layers, host_args):      # one untimed pass
+        bm.bimask_layer_step_host(largs, ha, hst)
+    barrier()
+    t0 = time.perf_counter()
+    ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ee0.record(stream)
+    for _ in range(e2e_steps):
+        for (L, b, largs), (ha, _, hst) in zip(layers, host_args):
+            bm.bimask_layer_step_host(largs, ha, hst)
+    ee1.record(stream)
+    barrier()
+    e2e_ms = max(ee0.elapsed_time(ee1), (time.perf_counter() - t0) * 1e3)
+
+    # ---- max over ranks ----
+    t = torch.tensor([step_ms_total, e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    step_ms_total, e2e_ms = float(t[0]), float(t[1])
+    nl = len(layers)
+    value = world * nl * args.steps / (step_ms_total * 1e-3)
+    e2e_value = world * nl * e2e_steps / (e2e_ms * 1e-3)
+
+    if rank == 0:
+        cpu_full, cpu_spent, desc = oracle_sample_time(args.config, rows=args.ref_rows, tokens=args.ref_tokens, cands=2)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": step_ms_total / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"config {args.config} ({cfg.name})",
+                       "layers": [[L.I, L.J, L.T] for L in cfg.layers], "N": cfg.N, "M": cfg.M, "P": cfg.P,
+                       "search_every_step": True, "parallelism": f"replicas x{world}",
+                       "l2": "inputs larger than L2 (W alone is %.0f MB per layer)" % (cfg.layers[0].I * cfg.layers[0].J * 4 / 1e6)
+                       if cfg.layers[0].I * cfg.layers[0].J * 4 > 126e6 else "inputs smaller than L2: warm-cache numbers"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps, "api": "bimask_layer_step_host (pinned host buffers)"},
+            "gpu_launches": int(launches),
+            "roofline": roofline,
+            "kernels": kernels,
+            "cpu_baseline": {"value": nl / cpu_full, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                             "sample": desc, "cpu_seconds_spent": cpu_spent},
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=5, help="workload: 1..5 (default 5, the largest)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--ref-rows", type=int, default=1024)
+    ap.add_argument("--ref-tokens", type=int, default=256)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

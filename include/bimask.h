@@ -55,6 +55,9 @@ typedef enum {
 /* Text of the calling thread's last error ("" if none).  Host memory owned by the library. */
 const char* bimask_last_error(void);
 
+/* Number of kernels this library has launched in this process so far (all threads). */
+uint64_t bimask_launch_count(void);
+
 /* Bytes of the opaque tensor-core metadata buffer for a packed operand with `rows` rows and
  * reduction length K (K = J for the forward operand, K = I for the backward one). */
 size_t bimask_hw_meta_bytes(int rows, int K);

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libbimask.so")
 
 BIMASK_OK, BIMASK_EINVAL, BIMASK_EUNSUPPORTED, BIMASK_ECUDA, BIMASK_ETIMEOUT = 0, -1, -2, -3, -4
 
-EXPORTS = ("bimask_last_error", "bimask_hw_meta_bytes", "bimask_workspace_bytes", "bimask_fwd_mask",
+EXPORTS = ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "bimask_workspace_bytes", "bimask_fwd_mask",
            "bimask_perm_search", "bimask_bwd_mask", "bimask_spmm_fwd", "bimask_spmm_dgrad", "bimask_wgrad",
            "bimask_layer_step", "bimask_layer_step_host", "bimask_check_perms")
 
@@ -50,6 +50,7 @@ def lib() -> ctypes.CDLL:
                                "(there is no fallback path)")
         L = ctypes.CDLL(LIB_PATH)
         L.bimask_last_error.restype = c_char_p
+        L.bimask_launch_count.restype = c_uint64
         L.bimask_hw_meta_bytes.restype = c_size_t
         L.bimask_hw_meta_bytes.argtypes = [c_int, c_int]
         L.bimask_workspace_bytes.restype = c_size_t
@@ -67,7 +68,7 @@ def lib() -> ctypes.CDLL:
         L.bimask_layer_step_host.argtypes = [POINTER(LayerArgs), POINTER(LayerArgs), c_void_p]
         L.bimask_check_perms.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_size_t, c_void_p]
         for name in EXPORTS:
-            if name not in ("bimask_last_error", "bimask_hw_meta_bytes", "bimask_workspace_bytes"):
+            if name not in ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "bimask_workspace_bytes"):
                 getattr(L, name).restype = c_int
         _lib = L
     return _lib
@@ -102,6 +103,10 @@ def _check(rc: int) -> int:
 
 def bimask_last_error() -> str:
     return lib().bimask_last_error().decode()
+
+
+def bimask_launch_count() -> int:
+    return int(lib().bimask_launch_count())
 
 
 def bimask_hw_meta_bytes(rows: int, K: int) -> int:

@@ -2,10 +2,14 @@
 // No kernel code lives here.
 #include "common.cuh"
 #include <string.h>
+#include <atomic>
 
 namespace bimask {
 
 static thread_local char g_err[512] = "";
+static std::atomic<unsigned long long> g_launches{0};
+
+void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 
 void set_error(const char* fmt, ...) {
   va_list ap;
@@ -56,6 +60,8 @@ using namespace bimask;
 extern "C" {
 
 const char* bimask_last_error(void) { return g_err; }
+
+uint64_t bimask_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 size_t bimask_hw_meta_bytes(int rows, int K) {
   if (rows <= 0 || K <= 0) return 0;

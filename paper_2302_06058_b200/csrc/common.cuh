@@ -10,6 +10,7 @@
 namespace bimask {
 
 void set_error(const char* fmt, ...);       // defined in api.cu
+void count_launch(int n = 1);               // defined in api.cu: kernel launches made so far
 int cuda_fail(cudaError_t e, const char* what);
 
 #define BIMASK_CUDA_OK(call)                                   \

@@ -305,6 +305,7 @@ int run_sparse(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, i
   p.status_word = status_word;
   dim3 grid((Mdim + 127) / 128, (Ndim + N_TILE - 1) / N_TILE, 1);
   kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p);
+  count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }
@@ -326,6 +327,7 @@ int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, u
   }
   int grid = T < 148 * 8 ? T : 148 * 8;
   permute_cols_kernel<<<grid, PERMUTE_THREADS, smem, s>>>(dY, perm, T, I, dYp);
+  count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }
@@ -366,6 +368,7 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
   p.status_word = status_word;
   dim3 grid((I + 127) / 128, (J + nt - 1) / nt, splits);
   kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p);
+  count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   if (splits > 1) {
     const long long n4 = (long long)I * J / 4;
@@ -373,6 +376,7 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
     if (blocks > 148 * 8) blocks = 148 * 8;
     splitk_reduce_kernel<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(partials), splits, n4,
                                                          reinterpret_cast<float4*>(dW));
+  count_launch();
     BIMASK_CUDA_OK(cudaGetLastError());
   }
   return BIMASK_OK;

@@ -233,6 +233,7 @@ int launch_fwd_mask(const float* W, int I, int J, int N, uint32_t* maskbits, uin
   if (ctas < 1) ctas = 1;
   fwd_mask_pack_kernel<<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
       reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint32_t*>(vals), meta);
+  count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }
@@ -242,6 +243,7 @@ int launch_hw_meta(const uint32_t* meta, int rows, int K, void* hw_meta, cudaStr
   const long long total = (long long)tiles_m * tiles_k * 512;
   hw_meta_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(meta, rows, K / 32, tiles_k, total,
                                                                  reinterpret_cast<uint32_t*>(hw_meta));
+  count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }
@@ -251,6 +253,7 @@ int launch_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* p
   dim3 grid((J + BWD_COLS - 1) / BWD_COLS, (I / 4 + BWD_KB - 1) / BWD_KB);
   bwd_mask_pack_kernel<<<grid, BWD_THREADS, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b,
                                                     reinterpret_cast<uint32_t*>(vals_b), meta_b);
+  count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }

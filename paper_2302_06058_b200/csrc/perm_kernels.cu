@@ -180,6 +180,7 @@ int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStrea
     attr_done = true;
   }
   gen_candidates_kernel<<<P, GEN_THREADS, smem, s>>>((unsigned long long)seed, I, n, cands);
+  count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }
@@ -195,6 +196,7 @@ int launch_score(const uint32_t* maskbits_f, const int32_t* cands, int I, int J,
     case 3: score_kernel<3><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt); break;
     default: score_kernel<4><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt); break;
   }
+  count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }
@@ -203,6 +205,7 @@ int launch_pick(const int64_t* counts, const int32_t* cands, int P, int I, int32
                 int32_t* best_perm, cudaStream_t s) {
   pick_kernel<<<1, PICK_THREADS, 0, s>>>(reinterpret_cast<const long long*>(counts), cands, P, I,
                                          best_idx, best_perm);
+  count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }
@@ -210,7 +213,9 @@ int launch_pick(const int64_t* counts, const int32_t* cands, int P, int I, int32
 int launch_check_perms(const int32_t* cands, int P, int I, int32_t* ok, uint8_t* seen, cudaStream_t s) {
   BIMASK_CUDA_OK(cudaMemsetAsync(seen, 0, (size_t)P * I, s));
   set_int_kernel<<<1, 1, 0, s>>>(ok, 1);
+  count_launch();
   check_perms_kernel<<<P, 256, 0, s>>>(cands, P, I, seen, ok);
+  count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }
