@@ -217,6 +217,8 @@ def run_gpu(args):
     layers = []
     host = []
     for li, L in enumerate(cfg.layers):
+        if args.profile and li != args.layer:
+            continue
         W, X, dY = inputs.make_layer(args.config, li)
         b = bm.alloc_layer_buffers(L.T, L.I, L.J, cfg.P)
         hW = torch.from_numpy(W).pin_memory()
@@ -232,6 +234,25 @@ def run_gpu(args):
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
+
+    if args.profile:
+        # one layer, the individual C-ABI calls in step order: the command line used under ncu
+        L, b, largs = layers[0]
+        wsb = b["ws"].numel()
+        for _ in range(args.warmup + args.steps):
+            bm.bimask_fwd_mask(b["W"], L.I, L.J, cfg.N, cfg.M, b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"])
+            bm.bimask_spmm_fwd(b["X"], b["vals_f"], b["hw_meta_f"], L.T, L.I, L.J, b["Y"], b["status_word"])
+            bm.bimask_perm_search(b["maskbits_f"], L.I, L.J, cfg.N, cfg.M, cfg.P, seed, None, b["perm"], b["best_idx"],
+                                  b["counts"], b["ws"], wsb)
+            bm.bimask_bwd_mask(b["W"], b["maskbits_f"], b["perm"], L.I, L.J, cfg.N, cfg.M, b["maskbits_b"], b["vals_b"],
+                               b["meta_b"], b["hw_meta_b"])
+            bm.bimask_spmm_dgrad(b["dY"], b["perm"], b["vals_b"], b["hw_meta_b"], L.T, L.I, L.J, b["dX"], b["ws"], wsb,
+                                 b["status_word"])
+            bm.bimask_wgrad(b["dY"], b["X"], L.T, L.I, L.J, b["dW"], b["ws"], wsb, b["status_word"])
+            torch.cuda.synchronize()
+        print(json.dumps({"profile": True, "config": args.config, "layer": args.layer,
+                          "status": int(b["status_word"].item())}), flush=True)
+        return
 
     def one_step():
         for _, _, largs in layers:
@@ -384,6 +405,8 @@ def main():
     ap.add_argument("--config", type=int, default=5, help="workload: 1..5 (default 5, the largest)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--profile", action="store_true", help="run only the C-ABI calls of one layer (for ncu)")
+    ap.add_argument("--layer", type=int, default=0)
     ap.add_argument("--ref-rows", type=int, default=1024)
     ap.add_argument("--ref-tokens", type=int, default=256)
     args = ap.parse_args()

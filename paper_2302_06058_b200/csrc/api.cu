@@ -153,7 +153,7 @@ int bimask_spmm_dgrad(const uint16_t* dY, const int32_t* perm, const uint16_t* v
   BIMASK_REQUIRE(aligned16(dY) && aligned16(perm) && aligned16(vals_b) && aligned16(hw_meta_b) && aligned16(dX) &&
                      aligned16(ws),
                  BIMASK_EINVAL, "bimask_spmm_dgrad: pointers must be 16-byte aligned");
-  BIMASK_REQUIRE((size_t)I * 2 <= 200 * 1024, BIMASK_EUNSUPPORTED, "I = %d too large for the column permute pass", I);
+  BIMASK_REQUIRE((size_t)I * 8 <= 200 * 1024, BIMASK_EUNSUPPORTED, "I = %d too large for the column permute pass (limit 25600)", I);
   const WsPlan w = plan_ws(T, I, J, 0);
   BIMASK_REQUIRE(ws_bytes >= w.dyp_off + w.dyp_bytes, BIMASK_EINVAL,
                  "bimask_spmm_dgrad: workspace too small (%zu bytes, need %zu)", ws_bytes, w.dyp_off + w.dyp_bytes);

@@ -42,9 +42,25 @@ struct GemmParams {
   int tiles_k_meta;         // number of 128-wide k tiles in the metadata image
   int Mdim, Ndim, Kdim;     // D is Mdim x Ndim, reduction length Kdim (logical)
   int k_tiles_per_split;    // dense split-K: k tiles handled by one blockIdx.z
+  int tiles_m, tiles_n;     // output tiles (CTA pairs along M for the pair kernel)
+  int raster_group;         // tiles walked along M before advancing along N
   void* out;                // sparse: bf16 [Ndim][Mdim];  dense: fp32 [split][Mdim][Ndim]
   int32_t* status_word;
 };
+
+
+// Tile order.  A linear id walks `group` tiles along M before it advances along N, so that the
+// CTAs resident at one time cover a near-square patch of the output and both operands are
+// re-used out of L2 instead of being streamed from HBM once per wave.
+__device__ __forceinline__ void raster(int id, int tiles_m, int tiles_n, int group, int& tm, int& tn) {
+  const int per_group = group * tiles_n;
+  const int g = id / per_group;
+  const int first = g * group;
+  const int gsize = min(group, tiles_m - first);
+  const int in = id - g * per_group;
+  tm = first + in % gsize;
+  tn = in / gsize;
+}
 
 template <bool SPARSE, int N_TILE, int STAGES>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
@@ -63,8 +79,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ C
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * C::M_TILE;
-  const int n0 = blockIdx.y * N_TILE;
+  int tile_m, tile_n;
+  raster((int)blockIdx.x, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
+  const int m0 = tile_m * C::M_TILE;
+  const int n0 = tile_n * N_TILE;
   const int k_tiles_total = (p.Kdim + C::K_TILE - 1) / C::K_TILE;
   const int kt_begin = blockIdx.z * p.k_tiles_per_split;
   const int kt_end = min(k_tiles_total, kt_begin + p.k_tiles_per_split);
@@ -107,7 +125,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ C
           ptx::tma_load_2d(b_s, &tmapB, kt * 128, n0, full_bar(s));                     // k 0..63
           ptx::tma_load_2d(b_s + N_TILE * 128, &tmapB, kt * 128 + 64, n0, full_bar(s)); // k 64..127
           ptx::bulk_load(b_s + C::B_BYTES,
-                         p.hw_meta + ((size_t)blockIdx.x * p.tiles_k_meta + kt) * 2048, 2048, full_bar(s));
+                         p.hw_meta + ((size_t)tile_m * p.tiles_k_meta + kt) * 2048, 2048, full_bar(s));
         } else {
 #pragma unroll
           for (int b = 0; b < 2; ++b) ptx::tma_load_2d(a_s + b * 8192, &tmapA, m0 + 64 * b, kt * 64, full_bar(s));
@@ -198,34 +216,370 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ C
   }
 }
 
+
 // ------------------------------------------------------------------------------------------
-// dY[:, perm]: a streaming pass, one CTA per token row chunk; the row is read coalesced into
-// shared memory and written back permuted with 16-byte stores.
+// 2:4 product on CTA pairs.  Two CTAs of a cluster share one 256 x 256 output tile: each loads
+// its own 128 rows of the compressed operand (and their metadata) and half of the 256 rows of
+// the dense operand; the pair's leader issues tcgen05.mma.sp.cta_group::2, which reads both
+// CTAs' shared memory and writes 128 accumulator rows into each CTA's tensor memory.  Per MMA
+// a CTA streams 12 KB of shared memory instead of 20 KB, which is what lets the sparse tensor
+// pipe run above the dense rate.  TMA loads carry no multicast; completion of both CTAs' loads
+// is counted on the leader's mbarrier, and tcgen05.commit releases a stage in both CTAs.
 // ------------------------------------------------------------------------------------------
-constexpr int PERMUTE_THREADS = 256;
+template <int STAGES>
+struct PairCfg {
+  static constexpr int A_BYTES = 16384;                 // 128 rows x 64 compressed bf16
+  static constexpr int B_BYTES = 32768;                 // 128 rows x 128 bf16 (two 64-wide boxes)
+  static constexpr int E_BYTES = 2048;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
+  static constexpr int TMEM_COLS = 512;                 // 256 accumulator columns + 4 metadata columns
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+};
+
+template <int STAGES>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+spmm_pair_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
+                 const __grid_constant__ CUtensorMap tmapE, const GemmParams p) {
+  using C = PairCfg<STAGES>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = ptx::smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - raw);
+  const uint32_t bar_base = base + STAGES * C::STAGE_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  const uint32_t tmem_full_bar = bar_base + 8u * (2 * STAGES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * C::STAGE_BYTES + 8 * (2 * STAGES + 1));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = ptx::cluster_ctarank();          // 0 = leader of the pair
+  int tile_m, tile_n;
+  raster((int)(blockIdx.x >> 1), p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
+  const int mt128 = 2 * tile_m + (int)rank;              // this CTA's 128 rows of the 256-row tile
+  const int m0 = mt128 * 128;
+  const int n0 = tile_n * 256;
+  const int num_kt = (p.Kdim + 127) / 128;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    ptx::mbar_init(tmem_full_bar, 1);
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmapA);
+    ptx::prefetch_tmap(&tmapB);
+    ptx::prefetch_tmap(&tmapE);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
+    ptx::tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync();                                   // both CTAs' barriers are initialised
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_meta = tmem_base + 256;
+
+  if (warp == 0) {
+    if (ptx::elect_one()) {
+      for (int it = 0; it < num_kt; ++it) {
+        const int s = it % STAGES;
+        const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+        if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
+        const uint32_t a_s = base + s * C::STAGE_BYTES;
+        const uint32_t b_s = a_s + C::A_BYTES;
+        const uint32_t e_s = b_s + C::B_BYTES;
+        const uint32_t bar = ptx::mapa(full_bar(s), 0);  // the leader counts both CTAs' bytes
+        if (rank == 0) ptx::mbar_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
+        ptx::tma_load_2d_pair(a_s, &tmapA, it * 64, m0, bar);
+        ptx::tma_load_2d_pair(b_s, &tmapB, it * 128, n0 + 128 * (int)rank, bar);
+        ptx::tma_load_2d_pair(b_s + 16384, &tmapB, it * 128 + 64, n0 + 128 * (int)rank, bar);
+        ptx::tma_load_2d_pair(e_s, &tmapE, 0, 2 * (mt128 * p.tiles_k_meta + it), bar);
+      }
+    }
+  } else if (warp == 1) {
+    if (rank == 0 && ptx::elect_one()) {
+      constexpr uint32_t idesc = ptx::idesc_bf16(256, 256, false, false, true);
+      bool ok = true;
+      for (int it = 0; it < num_kt; ++it) {
+        const int s = it % STAGES;
+        const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+        if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; ok = false; break; }
+        ptx::tc_fence_after();
+        const uint32_t a_s = base + s * C::STAGE_BYTES;
+        const uint32_t b_s = a_s + C::A_BYTES;
+        ptx::tmem_cp_128x128b_pair(tmem_meta, ptx::smem_desc(b_s + C::B_BYTES, 0, 128, 0));
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+          const uint64_t ad = ptx::smem_desc(a_s + kb * 32, 16, 1024, 2);
+          const uint64_t bd = ptx::smem_desc(b_s + (kb >> 1) * 16384 + (kb & 1) * 64, 16, 1024, 2);
+          ptx::mma_sparse_pair(tmem_base, ad, bd, tmem_meta + (kb & ~1), idesc | (uint32_t)(kb & 1), (it | kb) != 0);
+        }
+        ptx::tc_commit_pair(empty_bar(s), 3);
+      }
+      if (ok) ptx::tc_commit_pair(tmem_full_bar, 3);
+    }
+  } else {
+    const int q = warp & 3;
+    bool ok = ptx::mbar_wait_bounded(tmem_full_bar, 0, abort_flag, WAIT_BUDGET);
+    if (!ok) *abort_flag = 1;
+    ptx::tc_fence_after();
+    const int m = m0 + 32 * q + lane;
+    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
+    if (ok) {
+#pragma unroll 1
+      for (int c = 0; c < 8; ++c) {
+        uint32_t r[32];
+        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + 32 * c, r);
+        ptx::tmem_ld_wait();
+        const int nb = n0 + 32 * c;
+        if (m < p.Mdim) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (nb + j < p.Ndim) out[(size_t)(nb + j) * p.Mdim + m] = __float2bfloat16_rn(__uint_as_float(r[j]));
+        }
+      }
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status_word, (int32_t)BIMASK_ETIMEOUT);
+  ptx::cluster_sync();                                   // the peer no longer reads this CTA's memory
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
+  }
+}
+
+
+// ------------------------------------------------------------------------------------------
+// Persistent form of the CTA-pair 2:4 product: one pair per two SMs walks the output tiles in
+// raster order.  The TMA producer runs ahead across tile boundaries, so the next tile's operands
+// are already in flight while the four epilogue warps drain the accumulator: tensor memory ->
+// registers -> bf16 -> a transposed staging tile in shared memory (tensor memory is handed back
+// to the MMA thread at that point) -> one TMA store per tile, which also clips ragged edges.
+// ------------------------------------------------------------------------------------------
+template <int STAGES>
+struct PairPCfg {
+  static constexpr int A_BYTES = 16384, B_BYTES = 32768, E_BYTES = 2048;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
+  static constexpr int STAGING_BYTES = 4 * 2 * 2048;   // per epilogue warp: two [32 tokens][32 rows] bf16 buffers
+  static constexpr int TMEM_COLS = 512;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 + 256;
+};
+
+template <int STAGES>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
+                            const __grid_constant__ CUtensorMap tmapE, const __grid_constant__ CUtensorMap tmapOut,
+                            const GemmParams p) {
+  using C = PairPCfg<STAGES>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = ptx::smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - raw);
+  const uint32_t staging = base + STAGES * C::STAGE_BYTES;
+  uint8_t* staging_ptr = base_ptr + STAGES * C::STAGE_BYTES;
+  const uint32_t bar_base = staging + C::STAGING_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  const uint32_t tmem_full_bar = bar_base + 8u * (2 * STAGES);
+  const uint32_t tmem_empty_bar = bar_base + 8u * (2 * STAGES + 1);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(staging_ptr + C::STAGING_BYTES + 8 * (2 * STAGES + 2));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = ptx::cluster_ctarank();
+  const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+  const int num_tiles = p.tiles_m * p.tiles_n;
+  const int num_kt = (p.Kdim + 127) / 128;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    ptx::mbar_init(tmem_full_bar, 1);
+    ptx::mbar_init(tmem_empty_bar, 8);                   // four epilogue warps in each CTA of the pair
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmapA);
+    ptx::prefetch_tmap(&tmapB);
+    ptx::prefetch_tmap(&tmapE);
+    ptx::prefetch_tmap(&tmapOut);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
+    ptx::tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_meta = tmem_base + 256;
+
+  if (warp == 0) {
+    if (ptx::elect_one()) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+        int tile_m, tile_n;
+        raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
+        const int mt128 = 2 * tile_m + (int)rank;
+        const int m0 = mt128 * 128, nrow = tile_n * 256 + 128 * (int)rank;
+        for (int kt = 0; kt < num_kt; ++kt, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; ok = false; break; }
+          const uint32_t a_s = base + s * C::STAGE_BYTES;
+          const uint32_t b_s = a_s + C::A_BYTES;
+          const uint32_t bar = ptx::mapa(full_bar(s), 0);
+          if (rank == 0) ptx::mbar_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
+          ptx::tma_load_2d_pair(a_s, &tmapA, kt * 64, m0, bar);
+          ptx::tma_load_2d_pair(b_s, &tmapB, kt * 128, nrow, bar);
+          ptx::tma_load_2d_pair(b_s + 16384, &tmapB, kt * 128 + 64, nrow, bar);
+          ptx::tma_load_2d_pair(b_s + C::B_BYTES, &tmapE, 0, 2 * (mt128 * p.tiles_k_meta + kt), bar);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (rank == 0 && ptx::elect_one()) {
+      constexpr uint32_t idesc = ptx::idesc_bf16(256, 256, false, false, true);
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++tcount) {
+        // the accumulator must have been drained by both CTAs' epilogues
+        if (!ptx::mbar_wait_bounded(tmem_empty_bar, (tcount & 1u) ^ 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
+        ptx::tc_fence_after();
+        for (int kt = 0; kt < num_kt; ++kt, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t a_s = base + s * C::STAGE_BYTES;
+          const uint32_t b_s = a_s + C::A_BYTES;
+          ptx::tmem_cp_128x128b_pair(tmem_meta, ptx::smem_desc(b_s + C::B_BYTES, 0, 128, 0));
+#pragma unroll
+          for (int kb = 0; kb < 4; ++kb) {
+            const uint64_t ad = ptx::smem_desc(a_s + kb * 32, 16, 1024, 2);
+            const uint64_t bd = ptx::smem_desc(b_s + (kb >> 1) * 16384 + (kb & 1) * 64, 16, 1024, 2);
+            ptx::mma_sparse_pair(tmem_base, ad, bd, tmem_meta + (kb & ~1), idesc | (uint32_t)(kb & 1), (kt | kb) != 0);
+          }
+          ptx::tc_commit_pair(empty_bar(s), 3);
+        }
+        if (ok) ptx::tc_commit_pair(tmem_full_bar, 3);
+      }
+    }
+  } else {
+    // Each epilogue warp owns 32 accumulator rows (its TMEM lane quadrant) and a private pair of
+    // 2 KB staging buffers: 32 columns at a time go tensor memory -> registers -> bf16 ->
+    // staging[token][row] -> one TMA store of a 32 x 32 box (clipped at ragged edges).  Warps
+    // never wait for each other; a buffer is reused once the store issued two chunks earlier
+    // has finished reading it.
+    const int q = warp & 3;
+    const uint32_t leader_empty = ptx::mapa(tmem_empty_bar, 0);
+    const uint32_t stg_base = staging + q * 4096;
+    uint16_t* stg_ptr = reinterpret_cast<uint16_t*>(staging_ptr + q * 4096);
+    uint32_t tcount = 0, chunk = 0;
+    for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++tcount) {
+      int tile_m, tile_n;
+      raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
+      const int m0 = (2 * tile_m + (int)rank) * 128 + 32 * q, n0 = tile_n * 256;
+      if (!ptx::mbar_wait_bounded(tmem_full_bar, tcount & 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
+      ptx::tc_fence_after();
+#pragma unroll 1
+      for (int c = 0; c < 8; ++c, ++chunk) {
+        uint32_t r[32];
+        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + 32 * c, r);
+        ptx::tmem_ld_wait();
+        if (c == 7) {
+          // accumulator drained: hand tensor memory back to the MMA thread of the pair's leader
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive_cluster(leader_empty);
+        }
+        uint16_t* buf = stg_ptr + (chunk & 1u) * 1024;
+        if (lane == 0) ptx::tma_store_wait_read1();        // the store that last used this buffer is done
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) {
+          const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+          const uint32_t u = *reinterpret_cast<const uint32_t*>(&v);
+          buf[j * 32 + lane] = (uint16_t)(u & 0xFFFFu);
+          buf[(j + 1) * 32 + lane] = (uint16_t)(u >> 16);
+        }
+        ptx::fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) {
+          if (m0 < p.Mdim && n0 + 32 * c < p.Ndim)
+            ptx::tma_store_2d(&tmapOut, m0, n0 + 32 * c, stg_base + (chunk & 1u) * 2048);
+          ptx::tma_store_commit();
+        }
+      }
+    }
+    if (lane == 0) ptx::tma_store_wait_all();
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status_word, (int32_t)BIMASK_ETIMEOUT);
+  ptx::cluster_sync();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// dY[:, perm]: a streaming pass.  A CTA takes four token rows at a time: it reads them coalesced
+// and stores them column-interleaved in shared memory (one 8-byte word = the four rows' values of
+// one column), so that the gather costs one 8-byte shared load per permuted column for all four
+// rows; every thread then assembles eight consecutive permuted columns per row and writes them
+// with one 16-byte store.
+// ------------------------------------------------------------------------------------------
+constexpr int PERMUTE_THREADS = 1024;
 
 __global__ void __launch_bounds__(PERMUTE_THREADS)
 permute_cols_kernel(const uint16_t* __restrict__ dY, const int32_t* __restrict__ perm, int T, int I,
                     uint16_t* __restrict__ dYp) {
-  extern __shared__ uint16_t row_s[];
-  for (int t = blockIdx.x; t < T; t += gridDim.x) {
-    const uint4* src = reinterpret_cast<const uint4*>(dY + (size_t)t * I);
-    uint4* row4 = reinterpret_cast<uint4*>(row_s);
-    for (int i = threadIdx.x; i < (I >> 3); i += PERMUTE_THREADS) row4[i] = __ldg(src + i);
-    __syncthreads();
-    uint4* dst = reinterpret_cast<uint4*>(dYp + (size_t)t * I);
-    for (int i = threadIdx.x; i < (I >> 3); i += PERMUTE_THREADS) {
-      const int4 pa = __ldg(reinterpret_cast<const int4*>(perm) + 2 * i);
-      const int4 pb = __ldg(reinterpret_cast<const int4*>(perm) + 2 * i + 1);
-      const int idx[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
-      uint32_t v[4];
+  extern __shared__ uint4 tile4[];                       // tile4[c] = columns 2c and 2c+1, four rows each
+  const uint2* tile = reinterpret_cast<const uint2*>(tile4);
+  const int half = I >> 1;
+  for (int t0 = blockIdx.x * 4; t0 < T; t0 += gridDim.x * 4) {
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(dY) + (size_t)t0 * half;
+    for (int c = threadIdx.x; c < half; c += PERMUTE_THREADS) {
+      uint32_t r[4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const uint32_t lo = row_s[min(max(idx[2 * e], 0), I - 1)];
-        const uint32_t hi = row_s[min(max(idx[2 * e + 1], 0), I - 1)];
-        v[e] = lo | (hi << 16);
-      }
-      dst[i] = make_uint4(v[0], v[1], v[2], v[3]);
+      for (int j = 0; j < 4; ++j) r[j] = (t0 + j < T) ? __ldg(src + (size_t)j * half + c) : 0u;
+      tile4[c] = make_uint4(__byte_perm(r[0], r[1], 0x5410), __byte_perm(r[2], r[3], 0x5410),
+                            __byte_perm(r[0], r[1], 0x7632), __byte_perm(r[2], r[3], 0x7632));
+    }
+    __syncthreads();
+    for (int k8 = threadIdx.x; k8 < (I >> 3); k8 += PERMUTE_THREADS) {
+      const int4 pa = __ldg(reinterpret_cast<const int4*>(perm) + 2 * k8);
+      const int4 pb = __ldg(reinterpret_cast<const int4*>(perm) + 2 * k8 + 1);
+      const int idx[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
+      uint2 v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = tile[min(max(idx[e], 0), I - 1)];
+      uint4 o[4];
+      o[0] = make_uint4(__byte_perm(v[0].x, v[1].x, 0x5410), __byte_perm(v[2].x, v[3].x, 0x5410),
+                        __byte_perm(v[4].x, v[5].x, 0x5410), __byte_perm(v[6].x, v[7].x, 0x5410));
+      o[1] = make_uint4(__byte_perm(v[0].x, v[1].x, 0x7632), __byte_perm(v[2].x, v[3].x, 0x7632),
+                        __byte_perm(v[4].x, v[5].x, 0x7632), __byte_perm(v[6].x, v[7].x, 0x7632));
+      o[2] = make_uint4(__byte_perm(v[0].y, v[1].y, 0x5410), __byte_perm(v[2].y, v[3].y, 0x5410),
+                        __byte_perm(v[4].y, v[5].y, 0x5410), __byte_perm(v[6].y, v[7].y, 0x5410));
+      o[3] = make_uint4(__byte_perm(v[0].y, v[1].y, 0x7632), __byte_perm(v[2].y, v[3].y, 0x7632),
+                        __byte_perm(v[4].y, v[5].y, 0x7632), __byte_perm(v[6].y, v[7].y, 0x7632));
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (t0 + j < T) reinterpret_cast<uint4*>(dYp + (size_t)(t0 + j) * I)[k8] = o[j];
     }
     __syncthreads();
   }
@@ -303,8 +657,106 @@ int run_sparse(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, i
   p.k_tiles_per_split = (Kdim + 127) / 128;
   p.out = out;
   p.status_word = status_word;
-  dim3 grid((Mdim + 127) / 128, (Ndim + N_TILE - 1) / N_TILE, 1);
+  p.tiles_m = (Mdim + 127) / 128;
+  p.tiles_n = (Ndim + N_TILE - 1) / N_TILE;
+  p.raster_group = 16;
+  dim3 grid(p.tiles_m * p.tiles_n, 1, 1);
   kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p);
+  count_launch();
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
+
+// The metadata image as a 2-D tensor of u32: 256 words per row, two rows per 2048-byte block.
+int make_tmap_meta(CUtensorMap* m, const void* ptr, uint64_t blocks) {
+  EncodeTiledFn fn = get_encode_fn();
+  BIMASK_REQUIRE(fn != nullptr, BIMASK_ECUDA, "cuTensorMapEncodeTiled entry point not available");
+  cuuint64_t dims[2] = {256, blocks * 2};
+  cuuint64_t strides[1] = {1024};
+  cuuint32_t box[2] = {256, 2};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  BIMASK_REQUIRE(r == CUDA_SUCCESS, BIMASK_ECUDA, "cuTensorMapEncodeTiled (metadata) failed with CUresult %d", (int)r);
+  return BIMASK_OK;
+}
+
+int run_sparse_pair(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim, int Kdim,
+                    uint16_t* out, int32_t* status_word, cudaStream_t s) {
+  constexpr int STAGES = 4;
+  using C = PairCfg<STAGES>;
+  CUtensorMap ta, tb, te;
+  int rc;
+  const int tiles_m = (Mdim + 127) / 128, tiles_k = (Kdim + 127) / 128;
+  if ((rc = make_tmap(&ta, vals, (uint64_t)Kdim / 2, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, 128)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_meta(&te, hw_meta, (uint64_t)tiles_m * tiles_k)) != BIMASK_OK) return rc;
+  auto kern = spmm_pair_kernel<STAGES>;
+  if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
+  GemmParams p;
+  p.hw_meta = reinterpret_cast<const uint8_t*>(hw_meta);
+  p.tiles_k_meta = tiles_k;
+  p.Mdim = Mdim; p.Ndim = Ndim; p.Kdim = Kdim;
+  p.k_tiles_per_split = tiles_k;
+  p.out = out;
+  p.status_word = status_word;
+  p.tiles_m = (tiles_m + 1) / 2;
+  p.tiles_n = (Ndim + 255) / 256;
+  p.raster_group = 8;
+  dim3 grid(2 * p.tiles_m * p.tiles_n, 1, 1);
+  kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, p);
+  count_launch();
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
+
+// bf16 tensor map for TMA stores of 32 x 32 boxes into [rows][inner], no swizzle.
+int make_tmap_out(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  BIMASK_REQUIRE(fn != nullptr, BIMASK_ECUDA, "cuTensorMapEncodeTiled entry point not available");
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {inner * 2};
+  cuuint32_t box[2] = {32, 32};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  BIMASK_REQUIRE(r == CUDA_SUCCESS, BIMASK_ECUDA, "cuTensorMapEncodeTiled (output) failed with CUresult %d", (int)r);
+  return BIMASK_OK;
+}
+
+int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim,
+                               int Kdim, uint16_t* out, int32_t* status_word, cudaStream_t s) {
+  constexpr int STAGES = 4;
+  using C = PairPCfg<STAGES>;
+  CUtensorMap ta, tb, te, to;
+  int rc;
+  const int tiles_m = (Mdim + 127) / 128, tiles_k = (Kdim + 127) / 128;
+  if ((rc = make_tmap(&ta, vals, (uint64_t)Kdim / 2, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, 128)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_meta(&te, hw_meta, (uint64_t)tiles_m * tiles_k)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_out(&to, out, (uint64_t)Mdim, (uint64_t)Ndim)) != BIMASK_OK) return rc;
+  auto kern = spmm_pair_persistent_kernel<STAGES>;
+  if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
+  GemmParams p;
+  p.hw_meta = reinterpret_cast<const uint8_t*>(hw_meta);
+  p.tiles_k_meta = tiles_k;
+  p.Mdim = Mdim; p.Ndim = Ndim; p.Kdim = Kdim;
+  p.k_tiles_per_split = tiles_k;
+  p.out = out;
+  p.status_word = status_word;
+  p.tiles_m = (tiles_m + 1) / 2;
+  p.tiles_n = (Ndim + 255) / 256;
+  p.raster_group = 8;
+  const int total = p.tiles_m * p.tiles_n;
+  int sms = 148;
+  int dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int clusters = total < sms / 2 ? total : sms / 2;
+  kern<<<2 * clusters, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, to, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -314,18 +766,21 @@ int run_sparse(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, i
 
 int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim, int Kdim,
                 uint16_t* out, int32_t* status_word, cudaStream_t s) {
+  if (Ndim > 128 && Mdim > 128) return run_sparse_pair_persistent(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   if (Ndim > 128) return run_sparse<256, 2>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   return run_sparse<128, 4>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
 }
 
 int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, uint16_t* dYp, cudaStream_t s) {
-  const size_t smem = (size_t)I * 2;
+  const size_t smem = (size_t)I * 8;
   static bool attr_done = false;
   if (!attr_done) {
     BIMASK_CUDA_OK(cudaFuncSetAttribute(permute_cols_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     attr_done = true;
   }
-  int grid = T < 148 * 8 ? T : 148 * 8;
+  const int groups = (T + 3) / 4;
+  const int per_sm = smem <= 100 * 1024 ? 2 : 1;
+  int grid = groups < 148 * per_sm ? groups : 148 * per_sm;
   permute_cols_kernel<<<grid, PERMUTE_THREADS, smem, s>>>(dY, perm, T, I, dYp);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
@@ -366,7 +821,10 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
   p.k_tiles_per_split = per;
   p.out = splits > 1 ? partials : dW;
   p.status_word = status_word;
-  dim3 grid((I + 127) / 128, (J + nt - 1) / nt, splits);
+  p.tiles_m = (I + 127) / 128;
+  p.tiles_n = (J + nt - 1) / nt;
+  p.raster_group = 16;
+  dim3 grid(p.tiles_m * p.tiles_n, 1, splits);
   kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());

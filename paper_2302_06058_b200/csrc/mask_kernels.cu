@@ -20,92 +20,128 @@ __device__ __forceinline__ uint32_t to_bf16(float w) {
   return (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;
 }
 
-// Rank selection inside one block of four: element m is kept when it is a candidate
-// (bit m of `valid`) and fewer than N candidates beat it; q beats m when key_q > key_m, or
-// key_q == key_m with q < m.  Returns the 4-bit keep mask.
-__device__ __forceinline__ uint32_t keep4(uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3,
-                                          uint32_t valid, int N) {
+// Selection inside one block of four, table driven.  The six pairwise magnitude comparisons
+// (b_qm = key_q >= key_m for q < m) and the four candidate bits index a table whose entry holds
+// everything the block needs:
+//   bits [0,4)   keep mask: element m is kept when it is a candidate and fewer than N candidates
+//                beat it; q beats m when key_q > key_m, or key_q == key_m with q < m
+//   bits [4,8)   index code idx0 | idx1 << 2 of the 2:4 container (pad rule for < 2 kept)
+//   bit 8 / 9    slot 0 / slot 1 holds a kept element (else the slot is +0)
+//   bits [16,32) byte-permute selector that picks the two slots out of the four bf16 values
+// The table (64 entries for "all candidates", 1024 with candidate bits) is rebuilt in shared
+// memory by every CTA from the rule itself.
+__device__ __forceinline__ uint32_t lut_entry(uint32_t cmp, uint32_t valid, int N) {
+  const uint32_t b01 = (cmp >> 5) & 1u, b02 = (cmp >> 4) & 1u, b03 = (cmp >> 3) & 1u;
+  const uint32_t b12 = (cmp >> 2) & 1u, b13 = (cmp >> 1) & 1u, b23 = cmp & 1u;
   const uint32_t v0 = valid & 1u, v1 = (valid >> 1) & 1u, v2 = (valid >> 2) & 1u, v3 = (valid >> 3) & 1u;
-  // b_qm = 1 when the lower-index element q beats the higher-index element m (ties -> q)
-  const uint32_t b01 = k0 >= k1, b02 = k0 >= k2, b03 = k0 >= k3;
-  const uint32_t b12 = k1 >= k2, b13 = k1 >= k3, b23 = k2 >= k3;
   const uint32_t r0 = (v1 & (b01 ^ 1u)) + (v2 & (b02 ^ 1u)) + (v3 & (b03 ^ 1u));
   const uint32_t r1 = (v0 & b01) + (v2 & (b12 ^ 1u)) + (v3 & (b13 ^ 1u));
   const uint32_t r2 = (v0 & b02) + (v1 & b12) + (v3 & (b23 ^ 1u));
   const uint32_t r3 = (v0 & b03) + (v1 & b13) + (v2 & b23);
   const uint32_t n = (uint32_t)N;
-  return (v0 & (r0 < n)) | ((v1 & (r1 < n)) << 1) | ((v2 & (r2 < n)) << 2) | ((v3 & (r3 < n)) << 3);
-}
-
-// 2:4 container for a block with at most two kept elements: index code and the two bf16 slots.
-__device__ __forceinline__ void pack4(uint32_t kb, float w0, float w1, float w2, float w3,
-                                      uint32_t& code, uint32_t& vals) {
+  const uint32_t kb = (v0 & (r0 < n)) | ((v1 & (r1 < n)) << 1) | ((v2 & (r2 < n)) << 2) | ((v3 & (r3 < n)) << 3);
   const int pop = __popc(kb);
-  const uint32_t lo = (uint32_t)(__ffs(kb) - 1);          // lowest kept (unused if pop == 0)
-  uint32_t idx0, idx1;
+  uint32_t idx0 = 0u, idx1 = 1u;
   if (pop >= 2) {
-    idx0 = lo;
+    idx0 = (uint32_t)(__ffs(kb) - 1);
     idx1 = 31u - (uint32_t)__clz(kb);
   } else if (pop == 1) {
-    idx0 = 0u;
+    const uint32_t lo = (uint32_t)(__ffs(kb) - 1);
     idx1 = lo < 1u ? 1u : lo;
-  } else {
-    idx0 = 0u;
-    idx1 = 1u;
   }
-  const float s0 = idx0 == 0 ? w0 : idx0 == 1 ? w1 : idx0 == 2 ? w2 : w3;
-  const float s1 = idx1 == 0 ? w0 : idx1 == 1 ? w1 : idx1 == 2 ? w2 : w3;
-  const uint32_t a = ((kb >> idx0) & 1u) ? to_bf16(s0) : 0u;
-  const uint32_t b = ((kb >> idx1) & 1u) ? to_bf16(s1) : 0u;
-  code = idx0 | (idx1 << 2);
-  vals = a | (b << 16);
+  const uint32_t sel = (2u * idx0) | ((2u * idx0 + 1u) << 4) | ((2u * idx1) << 8) | ((2u * idx1 + 1u) << 12);
+  return kb | (idx0 << 4) | (idx1 << 6) | (((kb >> idx0) & 1u) << 8) | (((kb >> idx1) & 1u) << 9) | (sel << 16);
+}
+
+// Six comparison bits of a block, b01 first (bit 5) ... b23 last (bit 0).  Keys are < 2^31, so
+// key_m - key_q - 1 is negative exactly when key_q >= key_m; a funnel shift moves each sign bit in.
+__device__ __forceinline__ uint32_t cmp6(uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3) {
+  uint32_t c = 0;
+  c = __funnelshift_l(k1 - k0 - 1u, c, 1);
+  c = __funnelshift_l(k2 - k0 - 1u, c, 1);
+  c = __funnelshift_l(k3 - k0 - 1u, c, 1);
+  c = __funnelshift_l(k2 - k1 - 1u, c, 1);
+  c = __funnelshift_l(k3 - k1 - 1u, c, 1);
+  c = __funnelshift_l(k3 - k2 - 1u, c, 1);
+  return c;
+}
+
+// {hi, lo} -> packed bf16x2, round to nearest even (NaN comes out as 0x7fff: see slots()).
+__device__ __forceinline__ uint32_t cvt_bf16x2(float hi, float lo) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+
+// The two bf16 slots of a block from its table entry.  Fast path: two packed conversions and
+// one byte permute; a block that holds a NaN takes the exact integer conversion instead so that
+// the NaN payload rule (quiet bit set, sign and top payload bits kept) holds bit for bit.
+template <bool BOTH_KEPT>
+__device__ __forceinline__ uint32_t slots(uint32_t e, float w0, float w1, float w2, float w3,
+                                          uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3) {
+  if (max(max(k0, k1), max(k2, k3)) > 0x7F800000u) {
+    const uint32_t idx0 = (e >> 4) & 3u, idx1 = (e >> 6) & 3u;
+    const float s0 = idx0 == 0 ? w0 : idx0 == 1 ? w1 : w2;      // idx0 is never 3
+    const float s1 = idx1 == 1 ? w1 : idx1 == 2 ? w2 : w3;      // idx1 is never 0
+    const uint32_t a = (e & 0x100u) ? to_bf16(s0) : 0u;
+    const uint32_t b = (e & 0x200u) ? to_bf16(s1) : 0u;
+    return a | (b << 16);
+  }
+  uint32_t v = __byte_perm(cvt_bf16x2(w1, w0), cvt_bf16x2(w3, w2), e >> 16);
+  if (!BOTH_KEPT) v &= (((e >> 8) & 1u) * 0xFFFFu) | (((e >> 9) & 1u) * 0xFFFF0000u);
+  return v;
 }
 
 // ---------------------------------------------------------------------------------------
 // Forward mask + pack.  W is treated as a flat stream of 4-element blocks (J % 32 == 0, so
-// blocks, 32-column words and rows all nest).  A warp owns chunks of 256 blocks: 8 coalesced
-// float4 loads per lane are issued up front, then each lane's 4 mask bits / index nibble are
-// OR-reduced over 8-lane groups into words and routed so that lane w stores word w of the
-// chunk (one coalesced 128-byte store each for maskbits and meta).
+// blocks, 32-column words and rows all nest).  A warp owns chunks of 256 blocks: eight
+// coalesced float4 loads per lane go through an XOR-swizzled shared-memory stage so that each
+// lane then owns EIGHT CONSECUTIVE blocks (one 32-column word): it builds the mask word and
+// the code word locally, and stores its 32 bytes of values, with no cross-lane traffic.
 // ---------------------------------------------------------------------------------------
 constexpr int FWD_THREADS = 256;
 
+template <bool N_IS_2>
 __global__ void __launch_bounds__(FWD_THREADS)
 fwd_mask_pack_kernel(const float4* __restrict__ W4, long long nblk, int N,
-                     uint32_t* __restrict__ maskbits, uint32_t* __restrict__ vals,
+                     uint32_t* __restrict__ maskbits, uint4* __restrict__ vals4,
                      uint32_t* __restrict__ meta) {
-  const int lane = threadIdx.x & 31;
-  const long long warp = ((long long)blockIdx.x * FWD_THREADS + threadIdx.x) >> 5;
-  const long long nwarps = ((long long)gridDim.x * FWD_THREADS) >> 5;
+  __shared__ uint32_t lut[64];
+  __shared__ float4 stage[FWD_THREADS / 32][256];
+  if (threadIdx.x < 64) lut[threadIdx.x] = lut_entry(threadIdx.x, 0xFu, N);
+  __syncthreads();
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const long long warp = (long long)blockIdx.x * (FWD_THREADS / 32) + wib;
+  const long long nwarps = (long long)gridDim.x * (FWD_THREADS / 32);
   const long long nchunks = (nblk + 255) >> 8;
-  const uint32_t gmask = 0xFFu << (lane & 24);
-  const int sh = 4 * (lane & 7);
+  float4* st = stage[wib];
   for (long long ch = warp; ch < nchunks; ch += nwarps) {
-    const long long base = ch << 8;
-    float4 w[8];
+    const float4* src = W4 + (ch << 8);
+    const int left = (int)min((long long)256, nblk - (ch << 8));      // multiple of 8
 #pragma unroll
     for (int it = 0; it < 8; ++it) {
-      const long long b = base + it * 32 + lane;
-      w[it] = b < nblk ? __ldg(W4 + b) : make_float4(0.f, 0.f, 0.f, 0.f);
+      const int b = it * 32 + lane;
+      const float4 w = b < left ? __ldg(src + b) : make_float4(0.f, 0.f, 0.f, 0.f);
+      st[b ^ ((b >> 3) & 7)] = w;
     }
-    uint32_t my_bits = 0, my_meta = 0;
+    __syncwarp();
+    uint32_t bits = 0, codes = 0, v[8];
 #pragma unroll
-    for (int it = 0; it < 8; ++it) {
-      const long long b = base + it * 32 + lane;
-      const uint32_t kb = keep4(mag_key(w[it].x), mag_key(w[it].y), mag_key(w[it].z), mag_key(w[it].w), 0xFu, N);
-      uint32_t code, v;
-      pack4(kb, w[it].x, w[it].y, w[it].z, w[it].w, code, v);
-      if (b < nblk) vals[b] = v;
-      const uint32_t wb = __reduce_or_sync(gmask, kb << sh);
-      const uint32_t wm = __reduce_or_sync(gmask, code << sh);
-      const uint32_t rb = __shfl_sync(0xFFFFFFFFu, wb, (lane & 3) * 8);
-      const uint32_t rm = __shfl_sync(0xFFFFFFFFu, wm, (lane & 3) * 8);
-      if ((lane >> 2) == it) { my_bits = rb; my_meta = rm; }
+    for (int j = 0; j < 8; ++j) {
+      const float4 w = st[lane * 8 + (j ^ (lane & 7))];
+      const uint32_t k0 = mag_key(w.x), k1 = mag_key(w.y), k2 = mag_key(w.z), k3 = mag_key(w.w);
+      const uint32_t e = lut[cmp6(k0, k1, k2, k3)];
+      v[j] = slots<N_IS_2>(e, w.x, w.y, w.z, w.w, k0, k1, k2, k3);
+      bits |= (e & 15u) << (4 * j);
+      codes |= ((e >> 4) & 15u) << (4 * j);
     }
-    const long long word = (base >> 3) + lane;
-    if (word < (nblk >> 3)) {
-      maskbits[word] = my_bits;
-      meta[word] = my_meta;
+    __syncwarp();
+    if (lane * 8 < left) {
+      const long long word = (ch << 5) + lane;
+      maskbits[word] = bits;
+      meta[word] = codes;
+      vals4[2 * word] = make_uint4(v[0], v[1], v[2], v[3]);
+      vals4[2 * word + 1] = make_uint4(v[4], v[5], v[6], v[7]);
     }
   }
 }
@@ -139,86 +175,91 @@ __global__ void hw_meta_kernel(const uint32_t* __restrict__ meta, int rows, int 
 }
 
 // ---------------------------------------------------------------------------------------
-// Backward mask + transposed pack.  A CTA owns 128 columns x 64 row-blocks (256 permuted
-// rows).  Warp w handles row-blocks w, w+8, ...: for a row-block it gathers the four source
-// rows perm[4k..4k+3]; lane handles columns lane + 32 q (q < 4) so every load is a coalesced
-// 128-byte segment and a ballot over the warp yields a complete mask word.  The (value pair,
-// index code) of block (k, l) belongs to row l of the transposed operand, so it is staged in
-// shared memory ([l][k], padded) and written out with k contiguous.
+// Backward mask + transposed pack.  A CTA owns 128 columns x 64 row-blocks (256 permuted rows);
+// warp w walks the eight consecutive row-blocks 8w .. 8w+7.  For a row-block it gathers the four
+// source rows perm[4k..4k+3] with one coalesced 128-bit load per row (lane = four columns) and
+// selects per column through the table.  The operand it feeds is transposed (row = column l of
+// W, k contiguous), so each lane keeps the eight consecutive k results of its four columns in
+// registers and writes them as full 32-byte sectors -- no shared-memory transpose.  Mask words
+// (32 columns of one permuted row) are assembled with 4x4 bit transposes and an 8-lane OR.
 // ---------------------------------------------------------------------------------------
 constexpr int BWD_COLS = 128;
 constexpr int BWD_KB = 64;
 constexpr int BWD_THREADS = 256;
-constexpr int BWD_VSTRIDE = BWD_KB + 1;   // u32 words per staged row (odd => conflict-free)
-constexpr int BWD_CSTRIDE = BWD_KB + 4;   // bytes per staged code row (17 words, odd)
+
+// bit c of each of the four nibbles of x (bits c, c+4, c+8, c+12) gathered into a nibble
+__device__ __forceinline__ uint32_t gather4(uint32_t x, int c) {
+  return ((((x >> c) & 0x1111u) * 0x1248u) >> 12) & 15u;
+}
 
 __global__ void __launch_bounds__(BWD_THREADS)
 bwd_mask_pack_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,
                      const int32_t* __restrict__ perm, int I, int J, int N,
                      uint32_t* __restrict__ maskbits_b, uint32_t* __restrict__ vals_b,
                      uint32_t* __restrict__ meta_b) {
-  __shared__ uint32_t vals_s[BWD_COLS * BWD_VSTRIDE];
-  __shared__ uint8_t code_s[BWD_COLS * BWD_CSTRIDE];
+  __shared__ uint32_t lut[1024];
+  for (int e = threadIdx.x; e < 1024; e += BWD_THREADS) lut[e] = lut_entry(e & 63u, e >> 6, N);
+  __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int col0 = blockIdx.x * BWD_COLS;
-  const int kb0 = blockIdx.y * BWD_KB;
-  const int nkb = I >> 2;
+  // row-block tiles vary fastest over the grid: CTAs resident together write neighbouring
+  // pieces of the same operand rows, which L2 merges into long bursts
+  const int col0 = blockIdx.y * BWD_COLS;
   const int jwords = J >> 5;
-  const int kb_here = min(BWD_KB, nkb - kb0);
-  const int cols_here = min(BWD_COLS, J - col0);          // multiple of 32
-  const int nq = cols_here >> 5;
-
-  for (int kk = warp; kk < kb_here; kk += BWD_THREADS / 32) {
-    const int k = kb0 + kk;
+  const int kfirst = blockIdx.x * BWD_KB + 8 * warp;      // this warp's eight row-blocks
+  if (kfirst >= (I >> 2)) return;                         // I % 32 == 0: all eight or none
+  const int col = col0 + 4 * lane;                        // this lane's four columns
+  const bool active = col < J;
+  const int fword = (col0 >> 5) + (lane >> 3);            // mask word holding those columns
+  const int fshift = 4 * (lane & 7);
+  const uint32_t gmask = 0xFFu << (lane & 24);
+  uint32_t vacc[4][8];
+  uint32_t cacc[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int k = kfirst + j;
     const int4 p4 = __ldg(reinterpret_cast<const int4*>(perm) + k);
-    const int src[4] = {p4.x, p4.y, p4.z, p4.w};
-    float w[4][4];
-    uint32_t fb[4][4];
+    const int src[4] = {min(max(p4.x, 0), I - 1), min(max(p4.y, 0), I - 1), min(max(p4.z, 0), I - 1),
+                        min(max(p4.w, 0), I - 1)};
+    float4 w[4];
+    uint32_t fn = 0;
 #pragma unroll
-    for (int m = 0; m < 4; ++m)
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        if (q < nq) {
-          w[m][q] = __ldg(W + (long long)src[m] * J + col0 + 32 * q + lane);
-          fb[m][q] = __ldg(maskbits_f + (long long)src[m] * jwords + (col0 >> 5) + q);
-        } else {
-          w[m][q] = 0.f;
-          fb[m][q] = 0u;
-        }
-      }
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      if (q >= nq) break;
-      const uint32_t valid = ((fb[0][q] >> lane) & 1u) | (((fb[1][q] >> lane) & 1u) << 1) |
-                             (((fb[2][q] >> lane) & 1u) << 2) | (((fb[3][q] >> lane) & 1u) << 3);
-      const uint32_t kb = keep4(mag_key(w[0][q]), mag_key(w[1][q]), mag_key(w[2][q]), mag_key(w[3][q]), valid, N);
-      uint32_t code, v;
-      pack4(kb, w[0][q], w[1][q], w[2][q], w[3][q], code, v);
-      const int l = 32 * q + lane;
-      vals_s[l * BWD_VSTRIDE + kk] = v;
-      code_s[l * BWD_CSTRIDE + kk] = (uint8_t)code;
-#pragma unroll
-      for (int m = 0; m < 4; ++m) {
-        const uint32_t word = __ballot_sync(0xFFFFFFFFu, (kb >> m) & 1u);
-        if (lane == m) maskbits_b[(long long)(4 * k + m) * jwords + (col0 >> 5) + q] = word;
+    for (int m = 0; m < 4; ++m) {
+      if (active) {
+        w[m] = __ldg(reinterpret_cast<const float4*>(W + (size_t)src[m] * J + col));
+        fn |= ((__ldg(maskbits_f + (size_t)src[m] * jwords + fword) >> fshift) & 15u) << (4 * m);
+      } else {
+        w[m] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
-  }
-  __syncthreads();
-  // transposed operand: row l = column of W, k contiguous
-  const long long vrow = (long long)(I >> 1) >> 1;     // u32 (bf16 pairs) per row of vals_b = I/4
-  for (int l = warp; l < cols_here; l += BWD_THREADS / 32) {
-    for (int kk = lane; kk < kb_here; kk += 32)
-      vals_b[(long long)(col0 + l) * vrow + kb0 + kk] = vals_s[l * BWD_VSTRIDE + kk];
-  }
-  const int mwords_here = kb_here >> 3;                // I % 32 == 0 => whole words
-  const int mrow = I >> 5;
-  for (int e = threadIdx.x; e < cols_here * mwords_here; e += BWD_THREADS) {
-    const int l = e / mwords_here, wd = e % mwords_here;
-    uint32_t word = 0;
+    uint32_t kept = 0;                                    // nibble c = keep mask of column c
 #pragma unroll
-    for (int g = 0; g < 8; ++g) word |= (uint32_t)code_s[l * BWD_CSTRIDE + 8 * wd + g] << (4 * g);
-    meta_b[(long long)(col0 + l) * mrow + (kb0 >> 3) + wd] = word;
+    for (int c = 0; c < 4; ++c) {
+      const float w0 = c == 0 ? w[0].x : c == 1 ? w[0].y : c == 2 ? w[0].z : w[0].w;
+      const float w1 = c == 0 ? w[1].x : c == 1 ? w[1].y : c == 2 ? w[1].z : w[1].w;
+      const float w2 = c == 0 ? w[2].x : c == 1 ? w[2].y : c == 2 ? w[2].z : w[2].w;
+      const float w3 = c == 0 ? w[3].x : c == 1 ? w[3].y : c == 2 ? w[3].z : w[3].w;
+      const uint32_t k0 = mag_key(w0), k1 = mag_key(w1), k2 = mag_key(w2), k3 = mag_key(w3);
+      const uint32_t e = lut[(gather4(fn, c) << 6) | cmp6(k0, k1, k2, k3)];
+      vacc[c][j] = slots<false>(e, w0, w1, w2, w3, k0, k1, k2, k3);
+      cacc[c] |= ((e >> 4) & 15u) << (4 * j);
+      kept |= (e & 15u) << (4 * c);
+    }
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+      const uint32_t word = __reduce_or_sync(gmask, gather4(kept, m) << fshift);
+      if (active && (lane & 7) == 0) maskbits_b[(size_t)(4 * k + m) * jwords + fword] = word;
+    }
+  }
+  if (active) {
+    const size_t vrow = (size_t)I >> 2;                   // u32 (bf16 pairs) per row of vals_b
+    const size_t mrow = (size_t)I >> 5;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      uint4* dst = reinterpret_cast<uint4*>(vals_b + (size_t)(col + c) * vrow + kfirst);
+      dst[0] = make_uint4(vacc[c][0], vacc[c][1], vacc[c][2], vacc[c][3]);
+      dst[1] = make_uint4(vacc[c][4], vacc[c][5], vacc[c][6], vacc[c][7]);
+      meta_b[(size_t)(col + c) * mrow + (kfirst >> 3)] = cacc[c];
+    }
   }
 }
 
@@ -231,8 +272,12 @@ int launch_fwd_mask(const float* W, int I, int J, int N, uint32_t* maskbits, uin
   long long ctas = (nchunks + 7) / 8;
   if (ctas > 148 * 8) ctas = 148 * 8;
   if (ctas < 1) ctas = 1;
-  fwd_mask_pack_kernel<<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
-      reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint32_t*>(vals), meta);
+  if (N == 2)
+    fwd_mask_pack_kernel<true><<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
+        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta);
+  else
+    fwd_mask_pack_kernel<false><<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
+        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -250,7 +295,7 @@ int launch_hw_meta(const uint32_t* meta, int rows, int K, void* hw_meta, cudaStr
 
 int launch_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                     int N, uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, cudaStream_t s) {
-  dim3 grid((J + BWD_COLS - 1) / BWD_COLS, (I / 4 + BWD_KB - 1) / BWD_KB);
+  dim3 grid((I / 4 + BWD_KB - 1) / BWD_KB, (J + BWD_COLS - 1) / BWD_COLS);
   bwd_mask_pack_kernel<<<grid, BWD_THREADS, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b,
                                                     reinterpret_cast<uint32_t*>(vals_b), meta_b);
   count_launch();

@@ -81,21 +81,37 @@ score_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cand
   uint32_t cnt = 0;
   if ((jwords & 3) == 0) {
     const int jq = jwords >> 2;
-    for (int k = kb0 + warp; k < kb1; k += SCORE_THREADS / 32) {
-      const int4 r = __ldg(cand4 + k);
+    // two row blocks per trip: eight independent 128-bit loads in flight per lane
+    for (int k = kb0 + warp; k < kb1; k += 2 * (SCORE_THREADS / 32)) {
+      const int k2 = k + SCORE_THREADS / 32;
+      const bool two = k2 < kb1;
+      int4 r = __ldg(cand4 + k);
+      int4 t = __ldg(cand4 + (two ? k2 : k));
+      r.x = min(max(r.x, 0), I - 1); r.y = min(max(r.y, 0), I - 1); r.z = min(max(r.z, 0), I - 1); r.w = min(max(r.w, 0), I - 1);
+      t.x = min(max(t.x, 0), I - 1); t.y = min(max(t.y, 0), I - 1); t.z = min(max(t.z, 0), I - 1); t.w = min(max(t.w, 0), I - 1);
       const uint4* r0 = reinterpret_cast<const uint4*>(bits + (long long)r.x * jwords);
       const uint4* r1 = reinterpret_cast<const uint4*>(bits + (long long)r.y * jwords);
       const uint4* r2 = reinterpret_cast<const uint4*>(bits + (long long)r.z * jwords);
       const uint4* r3 = reinterpret_cast<const uint4*>(bits + (long long)r.w * jwords);
+      const uint4* t0 = reinterpret_cast<const uint4*>(bits + (long long)t.x * jwords);
+      const uint4* t1 = reinterpret_cast<const uint4*>(bits + (long long)t.y * jwords);
+      const uint4* t2 = reinterpret_cast<const uint4*>(bits + (long long)t.z * jwords);
+      const uint4* t3 = reinterpret_cast<const uint4*>(bits + (long long)t.w * jwords);
+      uint32_t c1 = 0, c2 = 0;
       for (int q = lane; q < jq; q += 32) {
         const uint4 a = __ldg(r0 + q), b = __ldg(r1 + q), cc = __ldg(r2 + q), d = __ldg(r3 + q);
-        cnt += __popc(~ineligible<N>(a.x, b.x, cc.x, d.x)) + __popc(~ineligible<N>(a.y, b.y, cc.y, d.y)) +
-               __popc(~ineligible<N>(a.z, b.z, cc.z, d.z)) + __popc(~ineligible<N>(a.w, b.w, cc.w, d.w));
+        const uint4 e = __ldg(t0 + q), f = __ldg(t1 + q), g = __ldg(t2 + q), h = __ldg(t3 + q);
+        c1 += __popc(~ineligible<N>(a.x, b.x, cc.x, d.x)) + __popc(~ineligible<N>(a.y, b.y, cc.y, d.y)) +
+              __popc(~ineligible<N>(a.z, b.z, cc.z, d.z)) + __popc(~ineligible<N>(a.w, b.w, cc.w, d.w));
+        c2 += __popc(~ineligible<N>(e.x, f.x, g.x, h.x)) + __popc(~ineligible<N>(e.y, f.y, g.y, h.y)) +
+              __popc(~ineligible<N>(e.z, f.z, g.z, h.z)) + __popc(~ineligible<N>(e.w, f.w, g.w, h.w));
       }
+      cnt += c1 + (two ? c2 : 0u);
     }
   } else {
     for (int k = kb0 + warp; k < kb1; k += SCORE_THREADS / 32) {
-      const int4 r = __ldg(cand4 + k);
+      int4 r = __ldg(cand4 + k);
+      r.x = min(max(r.x, 0), I - 1); r.y = min(max(r.y, 0), I - 1); r.z = min(max(r.z, 0), I - 1); r.w = min(max(r.w, 0), I - 1);
       const uint32_t* r0 = bits + (long long)r.x * jwords;
       const uint32_t* r1 = bits + (long long)r.y * jwords;
       const uint32_t* r2 = bits + (long long)r.z * jwords;
