@@ -536,6 +536,179 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
   }
 }
 
+
+// ------------------------------------------------------------------------------------------
+// Dense weight gradient on CTA pairs, persistent.  D[i, j] = sum_t dY[t, i] X[t, j]: both
+// operands are read MN-major straight from the row-major activations (no transpose pass).  A
+// pair owns a 256 x 256 tile; each CTA loads its 128 rows of dY^T and 128 of the 256 columns of
+// X per stage (32 KB), the leader issues tcgen05.mma.cta_group::2, and the 512 tensor-memory
+// columns hold TWO accumulators, so the epilogue of one tile (tensor memory -> registers ->
+// 128-byte runs of fp32 in global memory) overlaps the main loop of the next.
+// Work items are (tile, k-split) pairs; with more than one split the partial sums go to scratch.
+// ------------------------------------------------------------------------------------------
+template <int STAGES>
+struct WgradCfg {
+  static constexpr int A_BYTES = 16384, B_BYTES = 16384;     // 128 x 64 bf16 each, as two 64-wide boxes
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int TMEM_COLS = 512;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+};
+
+template <int STAGES>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
+                  const GemmParams p, int splits) {
+  using C = WgradCfg<STAGES>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = ptx::smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - raw);
+  const uint32_t bar_base = base + STAGES * C::STAGE_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tmem_full_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
+  auto tmem_empty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * C::STAGE_BYTES + 8 * (2 * STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = ptx::cluster_ctarank();
+  const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+  const int num_tiles = p.tiles_m * p.tiles_n;
+  const int num_items = num_tiles * splits;
+  const int k_tiles_total = (p.Kdim + 63) / 64;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(tmem_full_bar(b), 1);
+      ptx::mbar_init(tmem_empty_bar(b), 8);
+    }
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmapA);
+    ptx::prefetch_tmap(&tmapB);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
+    ptx::tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // item -> (tile, split) -> coordinates; identical in every role
+  auto item_coords = [&](int item, int& m0, int& n0, int& kt0, int& nkt, int& split) {
+    const int tile = item % num_tiles;
+    split = item / num_tiles;
+    int tile_m, tile_n;
+    raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
+    m0 = (2 * tile_m + (int)rank) * 128;
+    n0 = tile_n * 256;
+    kt0 = split * p.k_tiles_per_split;
+    nkt = min(k_tiles_total, kt0 + p.k_tiles_per_split) - kt0;
+  };
+
+  if (warp == 0) {
+    if (ptx::elect_one()) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int item = cluster_id; item < num_items && ok; item += num_clusters) {
+        int m0, n0, kt0, nkt, split;
+        item_coords(item, m0, n0, kt0, nkt, split);
+        for (int kt = kt0; kt < kt0 + nkt; ++kt, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; ok = false; break; }
+          const uint32_t a_s = base + s * C::STAGE_BYTES;
+          const uint32_t b_s = a_s + C::A_BYTES;
+          const uint32_t bar = ptx::mapa(full_bar(s), 0);
+          if (rank == 0) ptx::mbar_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
+          ptx::tma_load_2d_pair(a_s, &tmapA, m0, kt * 64, bar);
+          ptx::tma_load_2d_pair(a_s + 8192, &tmapA, m0 + 64, kt * 64, bar);
+          ptx::tma_load_2d_pair(b_s, &tmapB, n0 + 128 * (int)rank, kt * 64, bar);
+          ptx::tma_load_2d_pair(b_s + 8192, &tmapB, n0 + 128 * (int)rank + 64, kt * 64, bar);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (rank == 0 && ptx::elect_one()) {
+      constexpr uint32_t idesc = ptx::idesc_bf16(256, 256, true, true, false);
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int item = cluster_id; item < num_items && ok; item += num_clusters, ++tcount) {
+        int m0, n0, kt0, nkt, split;
+        item_coords(item, m0, n0, kt0, nkt, split);
+        const uint32_t buf = tcount & 1u;
+        if (!ptx::mbar_wait_bounded(tmem_empty_bar(buf), ((tcount >> 1) & 1u) ^ 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
+        ptx::tc_fence_after();
+        const uint32_t acc = tmem_base + 256u * buf;
+        for (int k = 0; k < nkt; ++k, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t a_s = base + s * C::STAGE_BYTES;
+          const uint32_t b_s = a_s + C::A_BYTES;
+#pragma unroll
+          for (int kb = 0; kb < 4; ++kb) {
+            const uint64_t ad = ptx::smem_desc(a_s + kb * 2048, 8192, 1024, 2);
+            const uint64_t bd = ptx::smem_desc(b_s + kb * 2048, 8192, 1024, 2);
+            ptx::mma_dense_pair(acc, ad, bd, idesc, (k | kb) != 0);
+          }
+          ptx::tc_commit_pair(empty_bar(s), 3);
+        }
+        if (ok) ptx::tc_commit_pair(tmem_full_bar(buf), 3);
+      }
+    }
+  } else {
+    const int q = warp & 3;
+    uint32_t tcount = 0;
+    for (int item = cluster_id; item < num_items; item += num_clusters, ++tcount) {
+      int m0, n0, kt0, nkt, split;
+      item_coords(item, m0, n0, kt0, nkt, split);
+      const uint32_t buf = tcount & 1u;
+      if (!ptx::mbar_wait_bounded(tmem_full_bar(buf), (tcount >> 1) & 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
+      ptx::tc_fence_after();
+      const int m = m0 + 32 * q + lane;
+      float* out = reinterpret_cast<float*>(p.out) + (size_t)split * p.Mdim * p.Ndim;
+#pragma unroll 1
+      for (int c = 0; c < 8; ++c) {
+        uint32_t r[32];
+        ptx::tmem_ld_32x32(tmem_base + 256u * buf + ((uint32_t)(32 * q) << 16) + 32 * c, r);
+        ptx::tmem_ld_wait();
+        if (c == 7) {                                      // accumulator drained: release it
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa(tmem_empty_bar(buf), 0));
+        }
+        const int nb = n0 + 32 * c;
+        if (m < p.Mdim && nb < p.Ndim) {                  // Ndim % 32 == 0: a chunk is all in or all out
+          float4* dst = reinterpret_cast<float4*>(out + (size_t)m * p.Ndim + nb);
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                 __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+        }
+      }
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status_word, (int32_t)BIMASK_ETIMEOUT);
+  ptx::cluster_sync();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
+  }
+}
+
 // ------------------------------------------------------------------------------------------
 // dY[:, perm]: a streaming pass.  A CTA takes four token rows at a time: it reads them coalesced
 // and stores them column-interleaved in shared memory (one 8-byte word = the four rows' values of
@@ -790,11 +963,11 @@ int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, u
 // Split-K plan of the dense product, shared by the launcher and the workspace-size query.
 void wgrad_plan(int T, int I, int J, int* n_tile, int* splits, int* k_tiles_per_split) {
   const int nt = 256;
-  const int tiles = ((I + 127) / 128) * ((J + nt - 1) / nt);
+  const int tiles = (((I + 127) / 128 + 1) / 2) * ((J + nt - 1) / nt);     // 256 x 256 pair tiles
   const int k_tiles = (T + 63) / 64;
   int sp = 1;
-  if (tiles < 148) {
-    sp = (2 * 148 + tiles - 1) / tiles;
+  if (tiles < 74) {
+    sp = (2 * 74 + tiles - 1) / tiles;
     const int max_by_k = k_tiles / 8 > 0 ? k_tiles / 8 : 1;        // at least 8 k tiles per split
     if (sp > max_by_k) sp = max_by_k;
     if (sp > 64) sp = 64;
@@ -808,12 +981,13 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
                       int32_t* status_word, cudaStream_t s) {
   int nt, splits, per;
   wgrad_plan(T, I, J, &nt, &splits, &per);
-  using C = Cfg<false, 256, 4>;
+  constexpr int STAGES = 4;
+  using C = WgradCfg<STAGES>;
   CUtensorMap ta, tb;
   int rc;
   if ((rc = make_tmap(&ta, dY, (uint64_t)I, (uint64_t)T, 64)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, X, (uint64_t)J, (uint64_t)T, 64)) != BIMASK_OK) return rc;
-  auto kern = gemm_kernel<false, 256, 4>;
+  auto kern = wgrad_pair_kernel<STAGES>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
   p.hw_meta = nullptr; p.tiles_k_meta = 0;
@@ -821,11 +995,14 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
   p.k_tiles_per_split = per;
   p.out = splits > 1 ? partials : dW;
   p.status_word = status_word;
-  p.tiles_m = (I + 127) / 128;
-  p.tiles_n = (J + nt - 1) / nt;
-  p.raster_group = 16;
-  dim3 grid(p.tiles_m * p.tiles_n, 1, splits);
-  kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p);
+  p.tiles_m = ((I + 127) / 128 + 1) / 2;
+  p.tiles_n = (J + 255) / 256;
+  p.raster_group = 8;
+  const int items = p.tiles_m * p.tiles_n * splits;
+  int sms = 148, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int clusters = items < sms / 2 ? items : sms / 2;
+  kern<<<2 * clusters, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p, splits);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   if (splits > 1) {
@@ -834,7 +1011,7 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
     if (blocks > 148 * 8) blocks = 148 * 8;
     splitk_reduce_kernel<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(partials), splits, n4,
                                                          reinterpret_cast<float4*>(dW));
-  count_launch();
+    count_launch();
     BIMASK_CUDA_OK(cudaGetLastError());
   }
   return BIMASK_OK;

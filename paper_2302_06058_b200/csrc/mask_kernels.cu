@@ -214,22 +214,42 @@ bwd_mask_pack_kernel(const float* __restrict__ W, const uint32_t* __restrict__ m
   const uint32_t gmask = 0xFFu << (lane & 24);
   uint32_t vacc[4][8];
   uint32_t cacc[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const int k = kfirst + j;
-    const int4 p4 = __ldg(reinterpret_cast<const int4*>(perm) + k);
-    const int src[4] = {min(max(p4.x, 0), I - 1), min(max(p4.y, 0), I - 1), min(max(p4.z, 0), I - 1),
-                        min(max(p4.w, 0), I - 1)};
-    float4 w[4];
-    uint32_t fn = 0;
+  // software pipeline: the rows of row-block j+1 are in flight while row-block j is processed,
+  // and the permutation entries are fetched two row-blocks ahead (index -> address -> data)
+  auto clamp4 = [&](int4 p4) {
+    return make_int4(min(max(p4.x, 0), I - 1), min(max(p4.y, 0), I - 1), min(max(p4.z, 0), I - 1),
+                     min(max(p4.w, 0), I - 1));
+  };
+  auto load_rows = [&](const int4 src, float4 (&w)[4], uint32_t& fn) {
+    const int r[4] = {src.x, src.y, src.z, src.w};
+    uint32_t f[4];
 #pragma unroll
     for (int m = 0; m < 4; ++m) {
       if (active) {
-        w[m] = __ldg(reinterpret_cast<const float4*>(W + (size_t)src[m] * J + col));
-        fn |= ((__ldg(maskbits_f + (size_t)src[m] * jwords + fword) >> fshift) & 15u) << (4 * m);
+        w[m] = __ldg(reinterpret_cast<const float4*>(W + (size_t)r[m] * J + col));
+        f[m] = __ldg(maskbits_f + (size_t)r[m] * jwords + fword);
       } else {
         w[m] = make_float4(0.f, 0.f, 0.f, 0.f);
+        f[m] = 0u;
       }
+    }
+    fn = ((f[0] >> fshift) & 15u) | (((f[1] >> fshift) & 15u) << 4) | (((f[2] >> fshift) & 15u) << 8) |
+         (((f[3] >> fshift) & 15u) << 12);
+  };
+  const int4* perm4 = reinterpret_cast<const int4*>(perm) + kfirst;
+  int4 p_next = clamp4(__ldg(perm4 + 1));
+  float4 wn[4];
+  uint32_t fnn;
+  load_rows(clamp4(__ldg(perm4)), wn, fnn);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int k = kfirst + j;
+    float4 w[4] = {wn[0], wn[1], wn[2], wn[3]};
+    const uint32_t fn = fnn;
+    if (j + 1 < 8) {
+      const int4 p_use = p_next;
+      if (j + 2 < 8) p_next = clamp4(__ldg(perm4 + j + 2));
+      load_rows(p_use, wn, fnn);
     }
     uint32_t kept = 0;                                    // nibble c = keep mask of column c
 #pragma unroll

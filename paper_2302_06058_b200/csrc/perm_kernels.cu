@@ -19,35 +19,77 @@ __device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
 }
 
 // ---------------------------------------------------------------------------------------
-// Candidate generation: one CTA per candidate sorts the I hashed keys in shared memory
-// (bitonic network on the next power of two, padding keys = all ones sort to the end).
+// Candidate generation: one CTA per candidate sorts the I hashed keys in shared memory.  The
+// keys are uniform 64-bit hashes, so a counting sort on their top log2(I) bits leaves buckets of
+// about one key each: histogram (shared-memory atomics), exclusive scan, scatter, then an
+// insertion sort inside every bucket makes the order exact for the full key.
 // ---------------------------------------------------------------------------------------
 constexpr int GEN_THREADS = 1024;
 
 __global__ void __launch_bounds__(GEN_THREADS)
-gen_candidates_kernel(unsigned long long seed, int I, int n_pow2, int32_t* __restrict__ cands) {
-  extern __shared__ unsigned long long keys[];
+gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int32_t* __restrict__ cands) {
+  extern __shared__ unsigned long long keys[];           // I sorted keys, then nb bucket counters
+  const int nb = 1 << nb_log2;
+  uint32_t* count = reinterpret_cast<uint32_t*>(keys + I);
+  __shared__ uint32_t warp_sums[GEN_THREADS / 32];
   const int c = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned long long stream = mix64(seed + 0x9E3779B97F4A7C15ull * (unsigned long long)(c + 1));
-  for (int i = threadIdx.x; i < n_pow2; i += GEN_THREADS) {
-    unsigned long long v = ~0ull;
-    if (i < I) v = (mix64(stream ^ (unsigned long long)i) & ~0xFFFFFFull) | (unsigned long long)i;
-    keys[i] = v;
+  const int shift = 64 - nb_log2;
+  for (int b = tid; b < nb; b += GEN_THREADS) count[b] = 0;
+  __syncthreads();
+  for (int i = tid; i < I; i += GEN_THREADS) {
+    const unsigned long long v = (mix64(stream ^ (unsigned long long)i) & ~0xFFFFFFull) | (unsigned long long)i;
+    atomicAdd(&count[(uint32_t)(v >> shift)], 1u);
   }
   __syncthreads();
-  for (int k = 2; k <= n_pow2; k <<= 1) {
-    for (int j = k >> 1; j > 0; j >>= 1) {
-      for (int t = threadIdx.x; t < (n_pow2 >> 1); t += GEN_THREADS) {
-        const int lo = ((t & ~(j - 1)) << 1) | (t & (j - 1));   // element with bit j clear
-        const int hi = lo | j;
-        const bool up = (lo & k) == 0;
-        const unsigned long long a = keys[lo], b = keys[hi];
-        if ((a > b) == up) { keys[lo] = b; keys[hi] = a; }
-      }
-      __syncthreads();
+  // exclusive scan of the nb counters: each thread owns a contiguous run of nb / GEN_THREADS
+  const int per = (nb + GEN_THREADS - 1) / GEN_THREADS;
+  const int b0 = tid * per;
+  uint32_t local = 0;
+  for (int b = b0; b < min(nb, b0 + per); ++b) local += count[b];
+  uint32_t incl = local;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+    if (lane >= d) incl += t;
+  }
+  if (lane == 31) warp_sums[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t ws = warp_sums[lane];
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, ws, d);
+      if (lane >= d) ws += t;
+    }
+    warp_sums[lane] = ws;
+  }
+  __syncthreads();
+  uint32_t run = incl - local + (warp > 0 ? warp_sums[warp - 1] : 0u);
+  for (int b = b0; b < min(nb, b0 + per); ++b) {
+    const uint32_t n = count[b];
+    count[b] = run;                                       // start of bucket b
+    run += n;
+  }
+  __syncthreads();
+  for (int i = tid; i < I; i += GEN_THREADS) {
+    const unsigned long long v = (mix64(stream ^ (unsigned long long)i) & ~0xFFFFFFull) | (unsigned long long)i;
+    keys[atomicAdd(&count[(uint32_t)(v >> shift)], 1u)] = v;   // count[b] ends as end of bucket b
+  }
+  __syncthreads();
+  for (int b = b0; b < min(nb, b0 + per); ++b) {
+    const int lo = b == 0 ? 0 : (int)count[b - 1];
+    const int hi = (int)count[b];
+    for (int a = lo + 1; a < hi; ++a) {                   // insertion sort, buckets hold ~1 key
+      const unsigned long long v = keys[a];
+      int q = a - 1;
+      while (q >= lo && keys[q] > v) { keys[q + 1] = keys[q]; --q; }
+      keys[q + 1] = v;
     }
   }
-  for (int i = threadIdx.x; i < I; i += GEN_THREADS)
+  __syncthreads();
+  for (int i = tid; i < I; i += GEN_THREADS)
     cands[(long long)c * I + i] = (int32_t)(keys[i] & 0xFFFFFFull);
 }
 
@@ -186,16 +228,16 @@ __global__ void set_int_kernel(int32_t* p, int32_t v) { *p = v; }
 }  // namespace
 
 int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStream_t s) {
-  int n = 2;
-  while (n < I) n <<= 1;
-  const size_t smem = (size_t)n * sizeof(unsigned long long);
+  int lg = 1;
+  while ((1 << lg) < I) ++lg;                             // one bucket per key on average
+  const size_t smem = (size_t)I * sizeof(unsigned long long) + ((size_t)1 << lg) * sizeof(uint32_t);
   static bool attr_done = false;     // same value every time; a race only repeats the call
   if (!attr_done) {
     BIMASK_CUDA_OK(cudaFuncSetAttribute(gen_candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        16384 * (int)sizeof(unsigned long long)));
+                                        16384 * (int)(sizeof(unsigned long long) + sizeof(uint32_t))));
     attr_done = true;
   }
-  gen_candidates_kernel<<<P, GEN_THREADS, smem, s>>>((unsigned long long)seed, I, n, cands);
+  gen_candidates_kernel<<<P, GEN_THREADS, smem, s>>>((unsigned long long)seed, I, lg, cands);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
