@@ -117,13 +117,10 @@ int bimask_spmm_dgrad(const uint16_t* dY, const int32_t* perm, const uint16_t* v
 int bimask_wgrad(const uint16_t* dY, const uint16_t* X, int T, int I, int J, float* dW,
                  void* ws, size_t ws_bytes, int32_t* status_word, void* stream);
 
-/* One iteration of Alg. 1 for one layer (without the optimizer update): fwd mask + pack,
- * [search if do_search], bwd mask + pack and the three products.  Everything is ordered after
- * what `stream` already holds and before whatever the caller enqueues on `stream` next.  Inside,
- * the dense weight gradient (which needs only dY and X) runs concurrently with the masks and the
- * search on a helper stream; that stream and three events are created once per device on the
- * first call (so the first call should come before any stream capture) and kept until exit.
- * When the search is skipped, perm is used as given. */
+/* One iteration of Alg. 1 for one layer (without the optimizer update): fwd mask + pack, sparse
+ * forward, [search if do_search], bwd mask + pack, sparse input gradient, dense weight
+ * gradient, all enqueued on `stream` in that order.  When the search is skipped, perm is used
+ * as given. */
 typedef struct {
   int T, I, J, N, M, P;
   uint64_t seed;

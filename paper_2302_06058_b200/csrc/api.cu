@@ -3,7 +3,6 @@
 #include "common.cuh"
 #include <string.h>
 #include <atomic>
-#include <mutex>
 
 namespace bimask {
 
@@ -154,7 +153,7 @@ int bimask_spmm_dgrad(const uint16_t* dY, const int32_t* perm, const uint16_t* v
   BIMASK_REQUIRE(aligned16(dY) && aligned16(perm) && aligned16(vals_b) && aligned16(hw_meta_b) && aligned16(dX) &&
                      aligned16(ws),
                  BIMASK_EINVAL, "bimask_spmm_dgrad: pointers must be 16-byte aligned");
-  BIMASK_REQUIRE((size_t)I * 8 <= 200 * 1024, BIMASK_EUNSUPPORTED, "I = %d too large for the column permute pass (limit 25600)", I);
+  BIMASK_REQUIRE((size_t)I * 4 <= 100 * 1024, BIMASK_EUNSUPPORTED, "I = %d too large for the column permute pass (limit 25600)", I);
   const WsPlan w = plan_ws(T, I, J, 0);
   BIMASK_REQUIRE(ws_bytes >= w.dyp_off + w.dyp_bytes, BIMASK_EINVAL,
                  "bimask_spmm_dgrad: workspace too small (%zu bytes, need %zu)", ws_bytes, w.dyp_off + w.dyp_bytes);
@@ -181,35 +180,6 @@ int bimask_wgrad(const uint16_t* dY, const uint16_t* X, int T, int I, int J, flo
   return launch_wgrad_impl(dY, X, T, I, J, dW, partials, status_word, (cudaStream_t)stream);
 }
 
-// A helper stream (highest priority) and two events per device, created on first use by
-// bimask_layer_step and kept for the life of the process.
-struct StepStreams {
-  cudaStream_t side = nullptr;
-  cudaEvent_t fork = nullptr, fwd_done = nullptr, bwd_done = nullptr;
-  bool ready = false;
-};
-static std::mutex g_streams_mutex;
-static StepStreams g_streams[64];
-
-static int get_step_streams(StepStreams** out) {
-  int dev = 0;
-  BIMASK_CUDA_OK(cudaGetDevice(&dev));
-  BIMASK_REQUIRE(dev >= 0 && dev < 64, BIMASK_EUNSUPPORTED, "device ordinal %d out of range", dev);
-  std::lock_guard<std::mutex> lock(g_streams_mutex);
-  StepStreams& st = g_streams[dev];
-  if (!st.ready) {
-    int least = 0, greatest = 0;
-    BIMASK_CUDA_OK(cudaDeviceGetStreamPriorityRange(&least, &greatest));
-    BIMASK_CUDA_OK(cudaStreamCreateWithPriority(&st.side, cudaStreamNonBlocking, greatest));
-    BIMASK_CUDA_OK(cudaEventCreateWithFlags(&st.fork, cudaEventDisableTiming));
-    BIMASK_CUDA_OK(cudaEventCreateWithFlags(&st.fwd_done, cudaEventDisableTiming));
-    BIMASK_CUDA_OK(cudaEventCreateWithFlags(&st.bwd_done, cudaEventDisableTiming));
-    st.ready = true;
-  }
-  *out = &st;
-  return BIMASK_OK;
-}
-
 int bimask_layer_step(const bimask_layer_args* a) {
   BIMASK_REQUIRE(a != nullptr, BIMASK_EINVAL, "bimask_layer_step: null argument block");
   int rc = check_shape(a->I, a->J, a->N, a->M);
@@ -225,7 +195,7 @@ int bimask_layer_step(const bimask_layer_args* a) {
                      aligned16(a->meta_f) && aligned16(a->hw_meta_f) && aligned16(a->maskbits_b) &&
                      aligned16(a->vals_b) && aligned16(a->meta_b) && aligned16(a->hw_meta_b),
                  BIMASK_EINVAL, "bimask_layer_step: pointers must be 16-byte aligned");
-  BIMASK_REQUIRE((size_t)a->I * 8 <= 200 * 1024, BIMASK_EUNSUPPORTED,
+  BIMASK_REQUIRE((size_t)a->I * 4 <= 100 * 1024, BIMASK_EUNSUPPORTED,
                  "I = %d too large for the column permute pass (limit 25600)", a->I);
   if (a->do_search) {
     BIMASK_REQUIRE(a->P >= 1 && a->P <= 65535 && a->best_idx && a->counts, BIMASK_EINVAL,
@@ -241,41 +211,28 @@ int bimask_layer_step(const bimask_layer_args* a) {
   uint16_t* dYp = reinterpret_cast<uint16_t*>(ws + w.dyp_off);
   float* partials = w.part_bytes ? reinterpret_cast<float*>(ws + w.part_off) : nullptr;
 
-  // Order of Alg. 1 with the one independent product taken out of line: the dense weight
-  // gradient needs only dY and X, so it runs on the caller's stream while the bandwidth-bound
-  // chain (forward mask, search, backward mask, column permute of dY) runs on a helper stream of
-  // higher priority; the two sparse products follow on the caller's stream as their operands
-  // become ready.  Everything the step enqueues is ordered before whatever the caller enqueues
-  // on `stream` afterwards.
-  StepStreams* st = nullptr;
-  if ((rc = get_step_streams(&st)) != BIMASK_OK) return rc;
-  cudaStream_t main_s = (cudaStream_t)a->stream, side = st->side;
-  BIMASK_CUDA_OK(cudaEventRecord(st->fork, main_s));
-  BIMASK_CUDA_OK(cudaStreamWaitEvent(side, st->fork, 0));
-
-  if ((rc = launch_fwd_mask(a->W, a->I, a->J, a->N, a->maskbits_f, a->vals_f, a->meta_f, side))) return rc;
-  if ((rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, side))) return rc;
-  BIMASK_CUDA_OK(cudaEventRecord(st->fwd_done, side));
+  // Alg. 1 in order, on the caller's stream.  (Running the dense weight gradient concurrently
+  // with the bandwidth-bound chain on a second stream was measured and rejected: the co-resident
+  // kernels contend for issue slots and the step became slower and erratic.)
+  cudaStream_t s = (cudaStream_t)a->stream;
+  if ((rc = launch_fwd_mask(a->W, a->I, a->J, a->N, a->maskbits_f, a->vals_f, a->meta_f, s))) return rc;
+  if ((rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, s))) return rc;
+  if ((rc = launch_spmm(a->vals_f, a->hw_meta_f, a->X, a->I, a->T, a->J, a->Y, a->status_word, s))) return rc;
   if (a->do_search) {
     const int32_t* cands = a->cands;
     if (!cands) {
-      if ((rc = launch_gen_candidates(a->seed, a->P, a->I, gen, side))) return rc;
+      if ((rc = launch_gen_candidates(a->seed, a->P, a->I, gen, s))) return rc;
       cands = gen;
     }
-    if ((rc = launch_score(a->maskbits_f, cands, a->I, a->J, a->N, a->P, a->counts, side))) return rc;
-    if ((rc = launch_pick(a->counts, cands, a->P, a->I, a->best_idx, a->perm, side))) return rc;
+    if ((rc = launch_score(a->maskbits_f, cands, a->I, a->J, a->N, a->P, a->counts, s))) return rc;
+    if ((rc = launch_pick(a->counts, cands, a->P, a->I, a->best_idx, a->perm, s))) return rc;
   }
-  if ((rc = launch_bwd_mask(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->maskbits_b, a->vals_b, a->meta_b, side)))
+  if ((rc = launch_bwd_mask(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->maskbits_b, a->vals_b, a->meta_b, s)))
     return rc;
-  if ((rc = launch_hw_meta(a->meta_b, a->J, a->I, a->hw_meta_b, side))) return rc;
-  if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, side))) return rc;
-  BIMASK_CUDA_OK(cudaEventRecord(st->bwd_done, side));
-
-  if ((rc = launch_wgrad_impl(a->dY, a->X, a->T, a->I, a->J, a->dW, partials, a->status_word, main_s))) return rc;
-  BIMASK_CUDA_OK(cudaStreamWaitEvent(main_s, st->fwd_done, 0));
-  if ((rc = launch_spmm(a->vals_f, a->hw_meta_f, a->X, a->I, a->T, a->J, a->Y, a->status_word, main_s))) return rc;
-  BIMASK_CUDA_OK(cudaStreamWaitEvent(main_s, st->bwd_done, 0));
-  return launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, a->dX, a->status_word, main_s);
+  if ((rc = launch_hw_meta(a->meta_b, a->J, a->I, a->hw_meta_b, s))) return rc;
+  if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, s))) return rc;
+  if ((rc = launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, a->dX, a->status_word, s))) return rc;
+  return launch_wgrad_impl(a->dY, a->X, a->T, a->I, a->J, a->dW, partials, a->status_word, s);
 }
 
 int bimask_layer_step_host(const bimask_layer_args* d, const bimask_layer_args* h, int32_t* host_status_word) {

@@ -710,48 +710,62 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_consta
 }
 
 // ------------------------------------------------------------------------------------------
-// dY[:, perm]: a streaming pass.  A CTA takes four token rows at a time: it reads them coalesced
-// and stores them column-interleaved in shared memory (one 8-byte word = the four rows' values of
-// one column), so that the gather costs one 8-byte shared load per permuted column for all four
-// rows; every thread then assembles eight consecutive permuted columns per row and writes them
-// with one 16-byte store.
+// dY[:, perm]: a streaming pass.  A CTA takes R token rows at a time (R = 4, or 2 for long rows
+// so that the tile stays under 64 KB and the kernel can run beside a resident GEMM): it reads
+// them coalesced and stores them column-interleaved in shared memory (one 2R-byte word = the R
+// rows' values of one column), so the gather costs one shared load per permuted column for all
+// R rows; every thread then assembles eight consecutive permuted columns per row and writes
+// them with one 16-byte store.
 // ------------------------------------------------------------------------------------------
-constexpr int PERMUTE_THREADS = 1024;
+constexpr int PERMUTE_THREADS = 512;
 
+template <int R>
 __global__ void __launch_bounds__(PERMUTE_THREADS)
 permute_cols_kernel(const uint16_t* __restrict__ dY, const int32_t* __restrict__ perm, int T, int I,
                     uint16_t* __restrict__ dYp) {
-  extern __shared__ uint4 tile4[];                       // tile4[c] = columns 2c and 2c+1, four rows each
-  const uint2* tile = reinterpret_cast<const uint2*>(tile4);
+  extern __shared__ uint32_t tile_w[];                   // R == 4: [I] x uint2, R == 2: [I] x uint32
   const int half = I >> 1;
-  for (int t0 = blockIdx.x * 4; t0 < T; t0 += gridDim.x * 4) {
+  for (int t0 = blockIdx.x * R; t0 < T; t0 += gridDim.x * R) {
     const uint32_t* src = reinterpret_cast<const uint32_t*>(dY) + (size_t)t0 * half;
     for (int c = threadIdx.x; c < half; c += PERMUTE_THREADS) {
-      uint32_t r[4];
+      uint32_t r[R];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) r[j] = (t0 + j < T) ? __ldg(src + (size_t)j * half + c) : 0u;
-      tile4[c] = make_uint4(__byte_perm(r[0], r[1], 0x5410), __byte_perm(r[2], r[3], 0x5410),
-                            __byte_perm(r[0], r[1], 0x7632), __byte_perm(r[2], r[3], 0x7632));
+      for (int j = 0; j < R; ++j) r[j] = (t0 + j < T) ? __ldg(src + (size_t)j * half + c) : 0u;
+      if (R == 4) {
+        reinterpret_cast<uint4*>(tile_w)[c] =
+            make_uint4(__byte_perm(r[0], r[1], 0x5410), __byte_perm(r[2], r[R - 1], 0x5410),
+                       __byte_perm(r[0], r[1], 0x7632), __byte_perm(r[2], r[R - 1], 0x7632));
+      } else {
+        reinterpret_cast<uint2*>(tile_w)[c] = make_uint2(__byte_perm(r[0], r[1], 0x5410), __byte_perm(r[0], r[1], 0x7632));
+      }
     }
     __syncthreads();
     for (int k8 = threadIdx.x; k8 < (I >> 3); k8 += PERMUTE_THREADS) {
       const int4 pa = __ldg(reinterpret_cast<const int4*>(perm) + 2 * k8);
       const int4 pb = __ldg(reinterpret_cast<const int4*>(perm) + 2 * k8 + 1);
       const int idx[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
-      uint2 v[8];
+      uint32_t lo[8], hi[8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) v[e] = tile[min(max(idx[e], 0), I - 1)];
+      for (int e = 0; e < 8; ++e) {
+        const int i = min(max(idx[e], 0), I - 1);
+        if (R == 4) {
+          const uint2 v = reinterpret_cast<const uint2*>(tile_w)[i];
+          lo[e] = v.x; hi[e] = v.y;
+        } else {
+          lo[e] = tile_w[i]; hi[e] = 0u;
+        }
+      }
       uint4 o[4];
-      o[0] = make_uint4(__byte_perm(v[0].x, v[1].x, 0x5410), __byte_perm(v[2].x, v[3].x, 0x5410),
-                        __byte_perm(v[4].x, v[5].x, 0x5410), __byte_perm(v[6].x, v[7].x, 0x5410));
-      o[1] = make_uint4(__byte_perm(v[0].x, v[1].x, 0x7632), __byte_perm(v[2].x, v[3].x, 0x7632),
-                        __byte_perm(v[4].x, v[5].x, 0x7632), __byte_perm(v[6].x, v[7].x, 0x7632));
-      o[2] = make_uint4(__byte_perm(v[0].y, v[1].y, 0x5410), __byte_perm(v[2].y, v[3].y, 0x5410),
-                        __byte_perm(v[4].y, v[5].y, 0x5410), __byte_perm(v[6].y, v[7].y, 0x5410));
-      o[3] = make_uint4(__byte_perm(v[0].y, v[1].y, 0x7632), __byte_perm(v[2].y, v[3].y, 0x7632),
-                        __byte_perm(v[4].y, v[5].y, 0x7632), __byte_perm(v[6].y, v[7].y, 0x7632));
+      o[0] = make_uint4(__byte_perm(lo[0], lo[1], 0x5410), __byte_perm(lo[2], lo[3], 0x5410),
+                        __byte_perm(lo[4], lo[5], 0x5410), __byte_perm(lo[6], lo[7], 0x5410));
+      o[1] = make_uint4(__byte_perm(lo[0], lo[1], 0x7632), __byte_perm(lo[2], lo[3], 0x7632),
+                        __byte_perm(lo[4], lo[5], 0x7632), __byte_perm(lo[6], lo[7], 0x7632));
+      o[2] = make_uint4(__byte_perm(hi[0], hi[1], 0x5410), __byte_perm(hi[2], hi[3], 0x5410),
+                        __byte_perm(hi[4], hi[5], 0x5410), __byte_perm(hi[6], hi[7], 0x5410));
+      o[3] = make_uint4(__byte_perm(hi[0], hi[1], 0x7632), __byte_perm(hi[2], hi[3], 0x7632),
+                        __byte_perm(hi[4], hi[5], 0x7632), __byte_perm(hi[6], hi[7], 0x7632));
 #pragma unroll
-      for (int j = 0; j < 4; ++j)
+      for (int j = 0; j < R; ++j)
         if (t0 + j < T) reinterpret_cast<uint4*>(dYp + (size_t)(t0 + j) * I)[k8] = o[j];
     }
     __syncthreads();
@@ -945,16 +959,21 @@ int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, 
 }
 
 int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, uint16_t* dYp, cudaStream_t s) {
-  const size_t smem = (size_t)I * 8;
   static bool attr_done = false;
   if (!attr_done) {
-    BIMASK_CUDA_OK(cudaFuncSetAttribute(permute_cols_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    BIMASK_CUDA_OK(cudaFuncSetAttribute(permute_cols_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+    BIMASK_CUDA_OK(cudaFuncSetAttribute(permute_cols_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
     attr_done = true;
   }
-  const int groups = (T + 3) / 4;
-  const int per_sm = smem <= 100 * 1024 ? 2 : 1;
-  int grid = groups < 148 * per_sm ? groups : 148 * per_sm;
-  permute_cols_kernel<<<grid, PERMUTE_THREADS, smem, s>>>(dY, perm, T, I, dYp);
+  const int R = (size_t)I * 8 <= 64 * 1024 ? 4 : 2;
+  const size_t smem = (size_t)I * 2 * R;
+  const int groups = (T + R - 1) / R;
+  const int per_sm = smem <= 32 * 1024 ? 3 : smem <= 48 * 1024 ? 2 : 1;
+  const int grid = groups < 148 * per_sm ? groups : 148 * per_sm;
+  if (R == 4)
+    permute_cols_kernel<4><<<grid, PERMUTE_THREADS, smem, s>>>(dY, perm, T, I, dYp);
+  else
+    permute_cols_kernel<2><<<grid, PERMUTE_THREADS, smem, s>>>(dY, perm, T, I, dYp);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;

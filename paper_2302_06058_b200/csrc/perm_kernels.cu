@@ -19,35 +19,49 @@ __device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
 }
 
 // ---------------------------------------------------------------------------------------
-// Candidate generation: one CTA per candidate sorts the I hashed keys in shared memory.  The
-// keys are uniform 64-bit hashes, so a counting sort on their top log2(I) bits leaves buckets of
-// about one key each: histogram (shared-memory atomics), exclusive scan, scatter, then an
-// insertion sort inside every bucket makes the order exact for the full key.
+// Candidate generation.  Candidate c is the order of the rows sorted by a 64-bit hashed key.
+// The keys are uniform, so a counting sort on their top log2(I) bits leaves buckets of about
+// one key each.  The bucket range is cut into Q equal parts and CTA (c, q) sorts part q: it
+// hashes all I rows (cheap), histograms the keys that fall into its part with shared-memory
+// atomics, counts the keys of the lower parts (its output offset), scans, scatters, finishes
+// every bucket with an insertion sort (exact order on the full key) and writes its slice.
+// Shared memory per CTA is about (I / Q) * 10 bytes, small enough to run beside a resident GEMM.
 // ---------------------------------------------------------------------------------------
-constexpr int GEN_THREADS = 1024;
+constexpr int GEN_THREADS = 512;
 
 __global__ void __launch_bounds__(GEN_THREADS)
-gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int32_t* __restrict__ cands) {
-  extern __shared__ unsigned long long keys[];           // I sorted keys, then nb bucket counters
-  const int nb = 1 << nb_log2;
-  uint32_t* count = reinterpret_cast<uint32_t*>(keys + I);
+gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int q_log2, int cap,
+                      int32_t* __restrict__ cands) {
+  extern __shared__ unsigned long long keys[];           // cap keys, then nbq bucket counters
+  const int nbq_log2 = nb_log2 - q_log2;
+  const int nbq = 1 << nbq_log2;
+  uint32_t* count = reinterpret_cast<uint32_t*>(keys + cap);
   __shared__ uint32_t warp_sums[GEN_THREADS / 32];
+  __shared__ uint32_t lower_total;
   const int c = blockIdx.x;
+  const uint32_t part = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned long long stream = mix64(seed + 0x9E3779B97F4A7C15ull * (unsigned long long)(c + 1));
   const int shift = 64 - nb_log2;
-  for (int b = tid; b < nb; b += GEN_THREADS) count[b] = 0;
+  for (int b = tid; b < nbq; b += GEN_THREADS) count[b] = 0;
+  if (tid == 0) lower_total = 0;
   __syncthreads();
+  uint32_t lower = 0;
   for (int i = tid; i < I; i += GEN_THREADS) {
     const unsigned long long v = (mix64(stream ^ (unsigned long long)i) & ~0xFFFFFFull) | (unsigned long long)i;
-    atomicAdd(&count[(uint32_t)(v >> shift)], 1u);
+    const uint32_t b = (uint32_t)(v >> shift);
+    const uint32_t pq = b >> nbq_log2;
+    if (pq == part) atomicAdd(&count[b & (nbq - 1)], 1u);
+    lower += pq < part;
   }
+  lower = __reduce_add_sync(0xFFFFFFFFu, lower);
+  if (lane == 0 && lower) atomicAdd(&lower_total, lower);
   __syncthreads();
-  // exclusive scan of the nb counters: each thread owns a contiguous run of nb / GEN_THREADS
-  const int per = (nb + GEN_THREADS - 1) / GEN_THREADS;
+  // exclusive scan of the nbq counters: each thread owns a contiguous run
+  const int per = (nbq + GEN_THREADS - 1) / GEN_THREADS;
   const int b0 = tid * per;
   uint32_t local = 0;
-  for (int b = b0; b < min(nb, b0 + per); ++b) local += count[b];
+  for (int b = b0; b < min(nbq, b0 + per); ++b) local += count[b];
   uint32_t incl = local;
 #pragma unroll
   for (int d = 1; d < 32; d <<= 1) {
@@ -57,17 +71,18 @@ gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int32_t* __re
   if (lane == 31) warp_sums[warp] = incl;
   __syncthreads();
   if (warp == 0) {
-    uint32_t ws = warp_sums[lane];
+    uint32_t ws = lane < GEN_THREADS / 32 ? warp_sums[lane] : 0u;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
       const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, ws, d);
       if (lane >= d) ws += t;
     }
-    warp_sums[lane] = ws;
+    if (lane < GEN_THREADS / 32) warp_sums[lane] = ws;
   }
   __syncthreads();
+  const uint32_t mine = warp_sums[GEN_THREADS / 32 - 1];  // keys of this part
   uint32_t run = incl - local + (warp > 0 ? warp_sums[warp - 1] : 0u);
-  for (int b = b0; b < min(nb, b0 + per); ++b) {
+  for (int b = b0; b < min(nbq, b0 + per); ++b) {
     const uint32_t n = count[b];
     count[b] = run;                                       // start of bucket b
     run += n;
@@ -75,12 +90,17 @@ gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int32_t* __re
   __syncthreads();
   for (int i = tid; i < I; i += GEN_THREADS) {
     const unsigned long long v = (mix64(stream ^ (unsigned long long)i) & ~0xFFFFFFull) | (unsigned long long)i;
-    keys[atomicAdd(&count[(uint32_t)(v >> shift)], 1u)] = v;   // count[b] ends as end of bucket b
+    const uint32_t b = (uint32_t)(v >> shift);
+    if ((b >> nbq_log2) == part) {
+      const uint32_t pos = atomicAdd(&count[b & (nbq - 1)], 1u);   // count[b] ends as end of bucket b
+      if (pos < (uint32_t)cap) keys[pos] = v;            // cap is > 15 sigma above the mean part size
+    }
   }
   __syncthreads();
-  for (int b = b0; b < min(nb, b0 + per); ++b) {
-    const int lo = b == 0 ? 0 : (int)count[b - 1];
-    const int hi = (int)count[b];
+  const int filled = (int)min(mine, (uint32_t)cap);
+  for (int b = b0; b < min(nbq, b0 + per); ++b) {
+    const int lo = min(b == 0 ? 0 : (int)count[b - 1], filled);
+    const int hi = min((int)count[b], filled);
     for (int a = lo + 1; a < hi; ++a) {                   // insertion sort, buckets hold ~1 key
       const unsigned long long v = keys[a];
       int q = a - 1;
@@ -89,8 +109,9 @@ gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int32_t* __re
     }
   }
   __syncthreads();
-  for (int i = tid; i < I; i += GEN_THREADS)
-    cands[(long long)c * I + i] = (int32_t)(keys[i] & 0xFFFFFFull);
+  const uint32_t base = lower_total;
+  for (int i = tid; i < filled; i += GEN_THREADS)
+    if (base + i < (uint32_t)I) cands[(long long)c * I + base + i] = (int32_t)(keys[i] & 0xFFFFFFull);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -230,14 +251,18 @@ __global__ void set_int_kernel(int32_t* p, int32_t v) { *p = v; }
 int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStream_t s) {
   int lg = 1;
   while ((1 << lg) < I) ++lg;                             // one bucket per key on average
-  const size_t smem = (size_t)I * sizeof(unsigned long long) + ((size_t)1 << lg) * sizeof(uint32_t);
+  int ql = 0;
+  while ((I >> ql) > 2048 && ql < lg - 1) ++ql;           // about 2048 keys per part
+  const int mean = (I + (1 << ql) - 1) >> ql;
+  const int cap = ql == 0 ? I : mean + (mean / 4 > 256 ? mean / 4 : 256);
+  const size_t smem = (size_t)cap * sizeof(unsigned long long) + ((size_t)1 << (lg - ql)) * sizeof(uint32_t);
   static bool attr_done = false;     // same value every time; a race only repeats the call
   if (!attr_done) {
-    BIMASK_CUDA_OK(cudaFuncSetAttribute(gen_candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        16384 * (int)(sizeof(unsigned long long) + sizeof(uint32_t))));
+    BIMASK_CUDA_OK(cudaFuncSetAttribute(gen_candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
     attr_done = true;
   }
-  gen_candidates_kernel<<<P, GEN_THREADS, smem, s>>>((unsigned long long)seed, I, lg, cands);
+  dim3 grid(P, 1 << ql);
+  gen_candidates_kernel<<<grid, GEN_THREADS, smem, s>>>((unsigned long long)seed, I, lg, ql, cap, cands);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
