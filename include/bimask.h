@@ -153,6 +153,33 @@ int bimask_layer_step(const bimask_layer_args* args);
 int bimask_layer_step_host(const bimask_layer_args* dev, const bimask_layer_args* host,
                            int32_t* host_status_word);
 
+/* The same search for a caller that cannot hand over a workspace.  (No counterpart in the paper:
+ * this entry point exists only because of how some programs manage GPU memory.)
+ *
+ * bimask_perm_search keeps the P x I generated candidates in `ws`, which somebody has to
+ * allocate.  Some users of this library are not in a position to do that at the moment they call:
+ * an inference or training runtime that has handed every byte of device memory to its own pool,
+ * a plug-in that is only lent device pointers by its host application, or code running at a
+ * point where calling the CUDA allocator is forbidden (it may synchronise the device).  For them
+ * the candidates live in an 8 MiB array that is part of the library's device image, so this call
+ * allocates nothing and asks for no scratch: it performs no cudaMalloc, no cudaFree and no
+ * allocating library call.  Every GPU that loads the library carries those 8 MiB until exit.
+ *
+ *   - Limit: P * I <= bimask_perm_search_static_max_entries() (2 Mi entries, e.g. P = 128 at
+ *     I = 16384); beyond that the call returns BIMASK_EUNSUPPORTED and launches nothing.
+ *     Candidates are always generated from `seed` (same generator as bimask_perm_search with
+ *     cands_or_null == NULL, so the results are identical); I <= 16384.
+ *   - The first call on each device looks up the array's device address (the current device must
+ *     be the one `stream` belongs to); make that first call before any stream capture begins.
+ *   - All calls share the one array and it keeps whatever the last call left there.  Nothing in
+ *     it needs to start at zero (each call rewrites every entry it later reads), but two calls
+ *     whose kernels overlap on the GPU -- different streams, or different host threads -- race
+ *     on it: serialise them.
+ *   - Inputs, outputs, alignment, return codes: as for bimask_perm_search. */
+int bimask_perm_search_static(const uint32_t* maskbits_f, int I, int J, int N, int M, int P, uint64_t seed,
+                              int32_t* best_perm, int32_t* best_idx, int64_t* counts, void* stream);
+size_t bimask_perm_search_static_max_entries(void);
+
 /* Debug helper, not on the hot path: sets *ok (device int) to 1 iff each of the P rows of
  * cands is a permutation of 0..I-1.  ws: at least P * I bytes of scratch. */
 int bimask_check_perms(const int32_t* cands, int P, int I, int32_t* ok, void* ws, size_t ws_bytes,

@@ -17,7 +17,8 @@ BIMASK_OK, BIMASK_EINVAL, BIMASK_EUNSUPPORTED, BIMASK_ECUDA, BIMASK_ETIMEOUT = 0
 
 EXPORTS = ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "bimask_workspace_bytes", "bimask_fwd_mask",
            "bimask_perm_search", "bimask_bwd_mask", "bimask_spmm_fwd", "bimask_spmm_dgrad", "bimask_wgrad",
-           "bimask_layer_step", "bimask_layer_step_host", "bimask_check_perms")
+           "bimask_layer_step", "bimask_layer_step_host", "bimask_check_perms", "bimask_perm_search_static",
+           "bimask_perm_search_static_max_entries")
 
 
 class BimaskError(RuntimeError):
@@ -67,8 +68,12 @@ def lib() -> ctypes.CDLL:
         L.bimask_layer_step.argtypes = [POINTER(LayerArgs)]
         L.bimask_layer_step_host.argtypes = [POINTER(LayerArgs), POINTER(LayerArgs), c_void_p]
         L.bimask_check_perms.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.bimask_perm_search_static.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_uint64,
+                                                c_void_p, c_void_p, c_void_p, c_void_p]
+        L.bimask_perm_search_static_max_entries.restype = c_size_t
         for name in EXPORTS:
-            if name not in ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "bimask_workspace_bytes"):
+            if name not in ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "bimask_workspace_bytes",
+                            "bimask_perm_search_static_max_entries"):
                 getattr(L, name).restype = c_int
         _lib = L
     return _lib
@@ -172,6 +177,17 @@ def bimask_layer_step_host(dev: LayerArgs, host: LayerArgs, host_status_word=Non
 
 def bimask_check_perms(cands, P, I, ok, ws, ws_bytes, stream=None):
     return _check(lib().bimask_check_perms(_ptr(cands), P, I, _ptr(ok), _ptr(ws), ws_bytes, _stream(stream)))
+
+
+def bimask_perm_search_static(maskbits_f, I, J, N, M, P, seed, best_perm, best_idx, counts, stream=None):
+    """Permutation search without a workspace: the candidates live in the library's built-in
+    8 MiB device array (P * I <= bimask_perm_search_static_max_entries()).  Allocates nothing."""
+    return _check(lib().bimask_perm_search_static(_ptr(maskbits_f), I, J, N, M, P, seed, _ptr(best_perm),
+                                                  _ptr(best_idx), _ptr(counts), _stream(stream)))
+
+
+def bimask_perm_search_static_max_entries() -> int:
+    return int(lib().bimask_perm_search_static_max_entries())
 
 
 def alloc_layer_buffers(T, I, J, P, device="cuda") -> dict:

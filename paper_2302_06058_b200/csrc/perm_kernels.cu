@@ -4,6 +4,7 @@
 // L2): a block of M = 4 permuted rows is tested for 32 columns at a time with a handful of
 // AND/OR operations on the four row words and a popcount.
 #include "common.cuh"
+#include <mutex>
 
 namespace bimask {
 
@@ -303,4 +304,66 @@ int launch_check_perms(const int32_t* cands, int P, int I, int32_t* ok, uint8_t*
   return BIMASK_OK;
 }
 
+// ---------------------------------------------------------------------------------------
+// bimask_perm_search_static: the permutation search for callers that have no scratch buffer
+// to give.  The generated candidates (P x I int32) live in a fixed array inside the library's
+// device image instead of caller memory, so the call needs no allocation by anybody.
+// ---------------------------------------------------------------------------------------
+namespace {
+
+constexpr size_t STATIC_CAND_ENTRIES = (size_t)2 << 20;              // 2 Mi int32 = 8 MiB per GPU
+static __device__ __align__(256) int32_t g_static_cands[STATIC_CAND_ENTRIES];
+
+// Device address of g_static_cands on each device.  In host code the symbol's name is only a
+// handle, so the address is looked up once per device (with that device current) and cached.
+std::mutex g_static_mutex;
+int32_t* g_static_ptr[64] = {nullptr};
+
+int static_cands_ptr(int32_t** out) {
+  int dev = 0;
+  BIMASK_CUDA_OK(cudaGetDevice(&dev));
+  BIMASK_REQUIRE(dev >= 0 && dev < 64, BIMASK_EUNSUPPORTED, "device ordinal %d out of range", dev);
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_ptr[dev]) {
+    int32_t* ptr = nullptr;
+    BIMASK_CUDA_OK(cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_cands));
+    BIMASK_REQUIRE(ptr != nullptr, BIMASK_ECUDA, "cudaGetSymbolAddress returned a null address");
+    g_static_ptr[dev] = ptr;
+  }
+  *out = g_static_ptr[dev];
+  return BIMASK_OK;
+}
+
+}  // namespace
+
 }  // namespace bimask
+
+extern "C" size_t bimask_perm_search_static_max_entries(void) { return bimask::STATIC_CAND_ENTRIES; }
+
+extern "C" int bimask_perm_search_static(const uint32_t* maskbits_f, int I, int J, int N, int M, int P, uint64_t seed,
+                                         int32_t* best_perm, int32_t* best_idx, int64_t* counts, void* stream) {
+  using namespace bimask;
+  BIMASK_REQUIRE(M == 4, BIMASK_EUNSUPPORTED, "M = %d: only M = 4 is implemented", M);
+  BIMASK_REQUIRE(I > 0 && J > 0 && I % 4 == 0 && J % 32 == 0, BIMASK_EINVAL,
+                 "I = %d, J = %d: I must be a positive multiple of 4, J of 32", I, J);
+  BIMASK_REQUIRE(N >= 1 && N <= M, BIMASK_EINVAL, "N = %d out of range 1..%d", N, M);
+  BIMASK_REQUIRE(P >= 1 && P <= 65535, BIMASK_EINVAL, "P = %d out of range 1..65535", P);
+  BIMASK_REQUIRE(I <= 16384, BIMASK_EUNSUPPORTED, "generated candidates need I <= 16384 (I = %d)", I);
+  BIMASK_REQUIRE((size_t)P * (size_t)I <= STATIC_CAND_ENTRIES, BIMASK_EUNSUPPORTED,
+                 "bimask_perm_search_static: P * I = %zu candidate entries exceed the built-in scratch of %zu; "
+                 "use bimask_perm_search with a caller-provided workspace",
+                 (size_t)P * (size_t)I, STATIC_CAND_ENTRIES);
+  BIMASK_REQUIRE(maskbits_f && best_perm && best_idx && counts, BIMASK_EINVAL, "bimask_perm_search_static: null pointer");
+  BIMASK_REQUIRE(aligned16(maskbits_f) && aligned16(best_perm) && ((uintptr_t)counts % 8 == 0) &&
+                     ((uintptr_t)best_idx % 4 == 0),
+                 BIMASK_EINVAL, "bimask_perm_search_static: misaligned pointer");
+  int32_t* cands = nullptr;
+  int rc = static_cands_ptr(&cands);
+  if (rc != BIMASK_OK) return rc;
+  cudaStream_t s = (cudaStream_t)stream;
+  // every entry of the first P x I slots is rewritten by the generator, so nothing left over
+  // from an earlier call is ever read; counts is zeroed inside launch_score
+  if ((rc = launch_gen_candidates(seed, P, I, cands, s)) != BIMASK_OK) return rc;
+  if ((rc = launch_score(maskbits_f, cands, I, J, N, P, counts, s)) != BIMASK_OK) return rc;
+  return launch_pick(counts, cands, P, I, best_idx, best_perm, s);
+}
