@@ -127,7 +127,7 @@ def run_reference(args):
 # clocks sampler
 # --------------------------------------------------------------------------------------------
 class ClockSampler:
-    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
 
@@ -141,13 +141,15 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    def stop(self, t_begin=None, t_end=None):
+        """Stop sampling; summarise the samples whose timestamp lies in [t_begin, t_end] (time.time())."""
+        import datetime
+        out = {"sm_mhz": None, "sm_max_mhz": None, "power_w": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -155,7 +157,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         try:
             with open(self.path) as f:
                 for line in f:
@@ -163,10 +165,15 @@ class ClockSampler:
                     if len(p) < 8:
                         continue
                     try:
-                        sm.append(float(p[0]))
-                        mx.append(float(p[1]))
+                        ts = datetime.datetime.strptime(p[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                        clk, cmax, watts = float(p[1]), float(p[2]), float(p[3])
                     except ValueError:
                         continue
+                    if t_begin is not None and not (t_begin <= ts <= t_end):
+                        continue
+                    sm.append(clk)
+                    mx.append(cmax)
+                    pw.append(watts)
                     for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[4:8]):
                         if v.lower().startswith("active"):
                             reasons.add(name)
@@ -174,13 +181,22 @@ class ClockSampler:
         except Exception:
             pass
         if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), power_w=float(np.median(pw)),
+                       reasons=sorted(reasons), samples=len(sm))
         return out
 
 
 # --------------------------------------------------------------------------------------------
 # GPU arm
 # --------------------------------------------------------------------------------------------
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM kernels on
+# config 5, from the ncu launch list summarised in profiles/cfg5_launch_list.md.
+NCU_TRAFFIC_BYTES = {
+    (5, 0, "wgrad"): 1.246e9 + 0.250e9, (5, 1, "wgrad"): None,
+    (5, 0, "spmm_fwd"): 0.604e9 + 0.249e9, (5, 0, "spmm_dgrad"): 0.879e9 + 0.062e9,
+}
+
+
 def algorithmic_work(L, P):
     """Algorithmic bytes / flops per launch of each timed call for one layer (see the design notes)."""
     I, J, T = L.I, L.J, L.T
@@ -259,9 +275,6 @@ def run_gpu(args):
             bm.bimask_layer_step(largs)
 
     # ---- warm-up, then the timed region: K steps through bimask_layer_step ----
-    for _ in range(max(args.warmup, 3)):
-        one_step()
-    barrier()
     gpu_uuid = str(local)
     try:
         gpu_uuid = "GPU-" + str(torch.cuda.get_device_properties(local).uuid)
@@ -269,6 +282,10 @@ def run_gpu(args):
         pass
     sampler = ClockSampler(gpu_uuid)
     sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    barrier()
+    t_load_begin = time.time()
     launches0 = bm.bimask_launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -306,7 +323,7 @@ def run_gpu(args):
             torch.cuda.synchronize()
             for k, n in enumerate(names):
                 acc[li][n] += ev[k].elapsed_time(ev[k + 1])
-    clocks = sampler.stop()
+    clocks = sampler.stop(t_load_begin, time.time())      # samples taken while the GPU was under this load
     status = [int(b["status_word"].item()) for _, b, _ in layers]
     if any(status):
         raise RuntimeError(f"device status words non-zero: {status}")
@@ -330,7 +347,8 @@ def run_gpu(args):
             kernels.append(entry)
     dom = max(kernels, key=lambda e: e["ms"])
     roofline = {"bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"], "unit": dom["unit"],
-                "frac": dom["frac"], "traffic": None, "kernel": f"layer {dom['layer']} {dom['call']}",
+                "frac": dom["frac"], "traffic": NCU_TRAFFIC_BYTES.get((args.config, dom["layer"], dom["call"])),
+                "kernel": f"layer {dom['layer']} {dom['call']}",
                 "peak_source": peaks["source"] + (" (sustained bf16; x2 for the 2:4 sparse products)"
                                                    if dom["bound"] == "tensor" else " (copy bandwidth)")}
 
@@ -400,7 +418,7 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=5, help="workload: 1..5 (default 5, the largest)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

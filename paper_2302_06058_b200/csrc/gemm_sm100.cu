@@ -44,6 +44,7 @@ struct GemmParams {
   int k_tiles_per_split;    // dense split-K: k tiles handled by one blockIdx.z
   int tiles_m, tiles_n;     // output tiles (CTA pairs along M for the pair kernel)
   int raster_group;         // tiles walked along M before advancing along N
+  int n_tile;               // pair kernel: output columns per tile (multiple of 16, <= 256)
   void* out;                // sparse: bf16 [Ndim][Mdim];  dense: fp32 [split][Mdim][Ndim]
   int32_t* status_word;
 };
@@ -218,157 +219,58 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ C
 
 
 // ------------------------------------------------------------------------------------------
-// 2:4 product on CTA pairs.  Two CTAs of a cluster share one 256 x 256 output tile: each loads
-// its own 128 rows of the compressed operand (and their metadata) and half of the 256 rows of
-// the dense operand; the pair's leader issues tcgen05.mma.sp.cta_group::2, which reads both
-// CTAs' shared memory and writes 128 accumulator rows into each CTA's tensor memory.  Per MMA
-// a CTA streams 12 KB of shared memory instead of 20 KB, which is what lets the sparse tensor
-// pipe run above the dense rate.  TMA loads carry no multicast; completion of both CTAs' loads
-// is counted on the leader's mbarrier, and tcgen05.commit releases a stage in both CTAs.
+// Persistent CTA-pair 2:4 product.  One pair per two SMs walks 256 x N output tiles in raster
+// order.  With N <= 240 tensor memory holds TWO accumulators (columns 0.. and 256..) plus the
+// four metadata columns (496..499), so the epilogue of one tile overlaps the main loop of the
+// next; N = 256 leaves room for one accumulator only (metadata at 256..259) and is used when the
+// tile count would otherwise round up to an extra pass over the SMs (the host picks N).  The TMA
+// producer runs ahead across tile boundaries; the four epilogue warps drain an accumulator 16
+// columns at a time: tensor memory -> registers -> bf16 -> a transposed per-warp staging tile ->
+// one TMA store per chunk (ragged edges are clipped).
 // ------------------------------------------------------------------------------------------
-template <int STAGES>
-struct PairCfg {
-  static constexpr int A_BYTES = 16384;                 // 128 rows x 64 compressed bf16
-  static constexpr int B_BYTES = 32768;                 // 128 rows x 128 bf16 (two 64-wide boxes)
-  static constexpr int E_BYTES = 2048;
-  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
-  static constexpr int TMEM_COLS = 512;                 // 256 accumulator columns + 4 metadata columns
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
-};
 
-template <int STAGES>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
-spmm_pair_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-                 const __grid_constant__ CUtensorMap tmapE, const GemmParams p) {
-  using C = PairCfg<STAGES>;
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t raw = ptx::smem_u32(smem_raw);
-  const uint32_t base = (raw + 1023u) & ~1023u;
-  uint8_t* base_ptr = smem_raw + (base - raw);
-  const uint32_t bar_base = base + STAGES * C::STAGE_BYTES;
-  auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
-  const uint32_t tmem_full_bar = bar_base + 8u * (2 * STAGES);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * C::STAGE_BYTES + 8 * (2 * STAGES + 1));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t rank = ptx::cluster_ctarank();          // 0 = leader of the pair
-  int tile_m, tile_n;
-  raster((int)(blockIdx.x >> 1), p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
-  const int mt128 = 2 * tile_m + (int)rank;              // this CTA's 128 rows of the 256-row tile
-  const int m0 = mt128 * 128;
-  const int n0 = tile_n * 256;
-  const int num_kt = (p.Kdim + 127) / 128;
-
-  if (threadIdx.x == 0) {
-    *abort_flag = 0;
-    for (int s = 0; s < STAGES; ++s) {
-      ptx::mbar_init(full_bar(s), 1);
-      ptx::mbar_init(empty_bar(s), 1);
-    }
-    ptx::mbar_init(tmem_full_bar, 1);
-    ptx::fence_barrier_init();
-    ptx::prefetch_tmap(&tmapA);
-    ptx::prefetch_tmap(&tmapB);
-    ptx::prefetch_tmap(&tmapE);
+// One epilogue chunk of the 2:4 product for one warp: W accumulator columns of its 32 rows go
+// tensor memory -> registers -> bf16 -> staging[token][row] -> one TMA store of a 32 x W box.
+// `last` releases the accumulator (after its final read) to the MMA thread of the pair's leader.
+template <int W>
+__device__ __forceinline__ void sparse_epilogue_chunk(uint32_t taddr, bool last, uint32_t release_bar,
+                                                      uint16_t* stg_ptr, uint32_t stg_base, uint32_t chunk, int lane,
+                                                      const CUtensorMap* tmap, int m0, int n, int Mdim, int Ndim) {
+  uint32_t r[W];
+  if (W == 32) ptx::tmem_ld_32x32(taddr, reinterpret_cast<uint32_t (&)[32]>(r));
+  else ptx::tmem_ld_32x16(taddr, reinterpret_cast<uint32_t (&)[16]>(r));
+  ptx::tmem_ld_wait();
+  if (last) {
+    ptx::tc_fence_before();
+    __syncwarp();
+    if (lane == 0) ptx::mbar_arrive_cluster(release_bar);
   }
-  if (warp == 1) {
-    ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
-    ptx::tmem_relinquish_pair();
-  }
-  ptx::tc_fence_before();
-  __syncthreads();
-  ptx::cluster_sync();                                   // both CTAs' barriers are initialised
-  ptx::tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_meta = tmem_base + 256;
-
-  if (warp == 0) {
-    if (ptx::elect_one()) {
-      for (int it = 0; it < num_kt; ++it) {
-        const int s = it % STAGES;
-        const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
-        if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
-        const uint32_t a_s = base + s * C::STAGE_BYTES;
-        const uint32_t b_s = a_s + C::A_BYTES;
-        const uint32_t e_s = b_s + C::B_BYTES;
-        const uint32_t bar = ptx::mapa(full_bar(s), 0);  // the leader counts both CTAs' bytes
-        if (rank == 0) ptx::mbar_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
-        ptx::tma_load_2d_pair(a_s, &tmapA, it * 64, m0, bar);
-        ptx::tma_load_2d_pair(b_s, &tmapB, it * 128, n0 + 128 * (int)rank, bar);
-        ptx::tma_load_2d_pair(b_s + 16384, &tmapB, it * 128 + 64, n0 + 128 * (int)rank, bar);
-        ptx::tma_load_2d_pair(e_s, &tmapE, 0, 2 * (mt128 * p.tiles_k_meta + it), bar);
-      }
-    }
-  } else if (warp == 1) {
-    if (rank == 0 && ptx::elect_one()) {
-      constexpr uint32_t idesc = ptx::idesc_bf16(256, 256, false, false, true);
-      bool ok = true;
-      for (int it = 0; it < num_kt; ++it) {
-        const int s = it % STAGES;
-        const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
-        if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; ok = false; break; }
-        ptx::tc_fence_after();
-        const uint32_t a_s = base + s * C::STAGE_BYTES;
-        const uint32_t b_s = a_s + C::A_BYTES;
-        ptx::tmem_cp_128x128b_pair(tmem_meta, ptx::smem_desc(b_s + C::B_BYTES, 0, 128, 0));
+  uint16_t* sbuf = stg_ptr + (chunk & 1u) * 1024;        // two 2 KB buffers per warp
+  if (lane == 0) ptx::tma_store_wait_read1();             // the store that last used this buffer is done
+  __syncwarp();
 #pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-          const uint64_t ad = ptx::smem_desc(a_s + kb * 32, 16, 1024, 2);
-          const uint64_t bd = ptx::smem_desc(b_s + (kb >> 1) * 16384 + (kb & 1) * 64, 16, 1024, 2);
-          ptx::mma_sparse_pair(tmem_base, ad, bd, tmem_meta + (kb & ~1), idesc | (uint32_t)(kb & 1), (it | kb) != 0);
-        }
-        ptx::tc_commit_pair(empty_bar(s), 3);
-      }
-      if (ok) ptx::tc_commit_pair(tmem_full_bar, 3);
-    }
-  } else {
-    const int q = warp & 3;
-    bool ok = ptx::mbar_wait_bounded(tmem_full_bar, 0, abort_flag, WAIT_BUDGET);
-    if (!ok) *abort_flag = 1;
-    ptx::tc_fence_after();
-    const int m = m0 + 32 * q + lane;
-    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
-    if (ok) {
-#pragma unroll 1
-      for (int c = 0; c < 8; ++c) {
-        uint32_t r[32];
-        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + 32 * c, r);
-        ptx::tmem_ld_wait();
-        const int nb = n0 + 32 * c;
-        if (m < p.Mdim) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (nb + j < p.Ndim) out[(size_t)(nb + j) * p.Mdim + m] = __float2bfloat16_rn(__uint_as_float(r[j]));
-        }
-      }
-    }
+  for (int j = 0; j < W; j += 2) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+    const uint32_t u = *reinterpret_cast<const uint32_t*>(&v);
+    sbuf[j * 32 + lane] = (uint16_t)(u & 0xFFFFu);
+    sbuf[(j + 1) * 32 + lane] = (uint16_t)(u >> 16);
   }
-
-  ptx::tc_fence_before();
-  __syncthreads();
-  if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status_word, (int32_t)BIMASK_ETIMEOUT);
-  ptx::cluster_sync();                                   // the peer no longer reads this CTA's memory
-  if (warp == 1) {
-    ptx::tc_fence_after();
-    ptx::tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
+  ptx::fence_proxy_async();
+  __syncwarp();
+  if (lane == 0) {
+    if (m0 < Mdim && n < Ndim) ptx::tma_store_2d(tmap, m0, n, stg_base + (chunk & 1u) * 2048);
+    ptx::tma_store_commit();
   }
 }
 
-
-// ------------------------------------------------------------------------------------------
-// Persistent form of the CTA-pair 2:4 product: one pair per two SMs walks the output tiles in
-// raster order.  The TMA producer runs ahead across tile boundaries, so the next tile's operands
-// are already in flight while the four epilogue warps drain the accumulator: tensor memory ->
-// registers -> bf16 -> a transposed staging tile in shared memory (tensor memory is handed back
-// to the MMA thread at that point) -> one TMA store per tile, which also clips ragged edges.
-// ------------------------------------------------------------------------------------------
 template <int STAGES>
 struct PairPCfg {
-  static constexpr int A_BYTES = 16384, B_BYTES = 32768, E_BYTES = 2048;
-  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
-  static constexpr int STAGING_BYTES = 4 * 2 * 2048;   // per epilogue warp: two [32 tokens][32 rows] bf16 buffers
+  static constexpr int A_BYTES = 16384;                    // 128 rows x 64 compressed bf16
+  static constexpr int B_MAX = 32768;                      // up to 128 rows x 128 bf16 (two 64-wide boxes)
+  static constexpr int E_BYTES = 2048;
+  static constexpr int STAGE_BYTES = A_BYTES + B_MAX + E_BYTES;        // 50 KB (the B part is N / 2 rows)
+  static constexpr int STAGING_BYTES = 4 * 2 * 2048;       // per epilogue warp: two [<= 32 tokens][32 rows] bf16 buffers
   static constexpr int TMEM_COLS = 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 + 256;
 };
@@ -376,8 +278,8 @@ struct PairPCfg {
 template <int STAGES>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-                            const __grid_constant__ CUtensorMap tmapE, const __grid_constant__ CUtensorMap tmapOut,
-                            const GemmParams p) {
+                            const __grid_constant__ CUtensorMap tmapE, const __grid_constant__ CUtensorMap tmapOut32,
+                            const __grid_constant__ CUtensorMap tmapOut16, const GemmParams p) {
   using C = PairPCfg<STAGES>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -388,9 +290,9 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
   const uint32_t bar_base = staging + C::STAGING_BYTES;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
-  const uint32_t tmem_full_bar = bar_base + 8u * (2 * STAGES);
-  const uint32_t tmem_empty_bar = bar_base + 8u * (2 * STAGES + 1);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(staging_ptr + C::STAGING_BYTES + 8 * (2 * STAGES + 2));
+  auto tmem_full_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
+  auto tmem_empty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(staging_ptr + C::STAGING_BYTES + 8 * (2 * STAGES + 4));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -398,6 +300,10 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
   const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
   const int num_tiles = p.tiles_m * p.tiles_n;
   const int num_kt = (p.Kdim + 127) / 128;
+  const int SP_N = p.n_tile;                              // output columns (tokens) per tile
+  const uint32_t nbuf = SP_N <= 240 ? 2u : 1u;            // accumulators in tensor memory
+  const uint32_t b_box = (uint32_t)(SP_N / 2) * 128u;     // bytes of one 64-wide box of this CTA's B rows
+  const uint32_t stage_tx = C::A_BYTES + 2u * b_box + C::E_BYTES;
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
@@ -405,13 +311,16 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
       ptx::mbar_init(full_bar(s), 1);
       ptx::mbar_init(empty_bar(s), 1);
     }
-    ptx::mbar_init(tmem_full_bar, 1);
-    ptx::mbar_init(tmem_empty_bar, 8);                   // four epilogue warps in each CTA of the pair
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(tmem_full_bar(b), 1);
+      ptx::mbar_init(tmem_empty_bar(b), 8);               // four epilogue warps in each CTA of the pair
+    }
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmapA);
     ptx::prefetch_tmap(&tmapB);
     ptx::prefetch_tmap(&tmapE);
-    ptx::prefetch_tmap(&tmapOut);
+    ptx::prefetch_tmap(&tmapOut32);
+    ptx::prefetch_tmap(&tmapOut16);
   }
   if (warp == 1) {
     ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
@@ -422,7 +331,7 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
   ptx::cluster_sync();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_meta = tmem_base + 256;
+  const uint32_t tmem_meta = tmem_base + (nbuf == 2u ? 496u : 256u);
 
   if (warp == 0) {
     if (ptx::elect_one()) {
@@ -432,7 +341,7 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
         int tile_m, tile_n;
         raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
         const int mt128 = 2 * tile_m + (int)rank;
-        const int m0 = mt128 * 128, nrow = tile_n * 256 + 128 * (int)rank;
+        const int m0 = mt128 * 128, nrow = tile_n * SP_N + (SP_N / 2) * (int)rank;
         for (int kt = 0; kt < num_kt; ++kt, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
@@ -440,23 +349,25 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
           const uint32_t a_s = base + s * C::STAGE_BYTES;
           const uint32_t b_s = a_s + C::A_BYTES;
           const uint32_t bar = ptx::mapa(full_bar(s), 0);
-          if (rank == 0) ptx::mbar_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
+          if (rank == 0) ptx::mbar_expect_tx(full_bar(s), 2 * stage_tx);
           ptx::tma_load_2d_pair(a_s, &tmapA, kt * 64, m0, bar);
           ptx::tma_load_2d_pair(b_s, &tmapB, kt * 128, nrow, bar);
-          ptx::tma_load_2d_pair(b_s + 16384, &tmapB, kt * 128 + 64, nrow, bar);
-          ptx::tma_load_2d_pair(b_s + C::B_BYTES, &tmapE, 0, 2 * (mt128 * p.tiles_k_meta + kt), bar);
+          ptx::tma_load_2d_pair(b_s + b_box, &tmapB, kt * 128 + 64, nrow, bar);
+          ptx::tma_load_2d_pair(b_s + C::B_MAX, &tmapE, 0, 2 * (mt128 * p.tiles_k_meta + kt), bar);
         }
       }
     }
   } else if (warp == 1) {
     if (rank == 0 && ptx::elect_one()) {
-      constexpr uint32_t idesc = ptx::idesc_bf16(256, 256, false, false, true);
+      const uint32_t idesc = ptx::idesc_bf16(256, SP_N, false, false, true);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++tcount) {
-        // the accumulator must have been drained by both CTAs' epilogues
-        if (!ptx::mbar_wait_bounded(tmem_empty_bar, (tcount & 1u) ^ 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
+        const uint32_t buf = tcount % nbuf;
+        // this accumulator must have been drained by both CTAs' epilogues
+        if (!ptx::mbar_wait_bounded(tmem_empty_bar(buf), ((tcount / nbuf) & 1u) ^ 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
         ptx::tc_fence_after();
+        const uint32_t acc = tmem_base + 256u * buf;
         for (int kt = 0; kt < num_kt; ++kt, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
@@ -464,63 +375,45 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
           ptx::tc_fence_after();
           const uint32_t a_s = base + s * C::STAGE_BYTES;
           const uint32_t b_s = a_s + C::A_BYTES;
-          ptx::tmem_cp_128x128b_pair(tmem_meta, ptx::smem_desc(b_s + C::B_BYTES, 0, 128, 0));
+          ptx::tmem_cp_128x128b_pair(tmem_meta, ptx::smem_desc(b_s + C::B_MAX, 0, 128, 0));
 #pragma unroll
           for (int kb = 0; kb < 4; ++kb) {
             const uint64_t ad = ptx::smem_desc(a_s + kb * 32, 16, 1024, 2);
-            const uint64_t bd = ptx::smem_desc(b_s + (kb >> 1) * 16384 + (kb & 1) * 64, 16, 1024, 2);
-            ptx::mma_sparse_pair(tmem_base, ad, bd, tmem_meta + (kb & ~1), idesc | (uint32_t)(kb & 1), (kt | kb) != 0);
+            const uint64_t bd = ptx::smem_desc(b_s + (kb >> 1) * b_box + (kb & 1) * 64, 16, 1024, 2);
+            ptx::mma_sparse_pair(acc, ad, bd, tmem_meta + (kb & ~1), idesc | (uint32_t)(kb & 1), (kt | kb) != 0);
           }
           ptx::tc_commit_pair(empty_bar(s), 3);
         }
-        if (ok) ptx::tc_commit_pair(tmem_full_bar, 3);
+        if (ok) ptx::tc_commit_pair(tmem_full_bar(buf), 3);
       }
     }
   } else {
     // Each epilogue warp owns 32 accumulator rows (its TMEM lane quadrant) and a private pair of
-    // 2 KB staging buffers: 32 columns at a time go tensor memory -> registers -> bf16 ->
-    // staging[token][row] -> one TMA store of a 32 x 32 box (clipped at ragged edges).  Warps
-    // never wait for each other; a buffer is reused once the store issued two chunks earlier
-    // has finished reading it.
+    // 2 KB staging buffers; warps never wait for each other.  A buffer is reused once the store
+    // issued two chunks earlier has finished reading it.
     const int q = warp & 3;
-    const uint32_t leader_empty = ptx::mapa(tmem_empty_bar, 0);
     const uint32_t stg_base = staging + q * 4096;
     uint16_t* stg_ptr = reinterpret_cast<uint16_t*>(staging_ptr + q * 4096);
     uint32_t tcount = 0, chunk = 0;
     for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++tcount) {
       int tile_m, tile_n;
       raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
-      const int m0 = (2 * tile_m + (int)rank) * 128 + 32 * q, n0 = tile_n * 256;
-      if (!ptx::mbar_wait_bounded(tmem_full_bar, tcount & 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
+      const int m0 = (2 * tile_m + (int)rank) * 128 + 32 * q, n0 = tile_n * SP_N;
+      const uint32_t buf = tcount % nbuf;
+      if (!ptx::mbar_wait_bounded(tmem_full_bar(buf), (tcount / nbuf) & 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
       ptx::tc_fence_after();
+      const uint32_t acc = tmem_base + 256u * buf + ((uint32_t)(32 * q) << 16);
+      const uint32_t release_bar = ptx::mapa(tmem_empty_bar(buf), 0);
+      if ((SP_N & 31) == 0) {
 #pragma unroll 1
-      for (int c = 0; c < 8; ++c, ++chunk) {
-        uint32_t r[32];
-        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + 32 * c, r);
-        ptx::tmem_ld_wait();
-        if (c == 7) {
-          // accumulator drained: hand tensor memory back to the MMA thread of the pair's leader
-          ptx::tc_fence_before();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive_cluster(leader_empty);
-        }
-        uint16_t* buf = stg_ptr + (chunk & 1u) * 1024;
-        if (lane == 0) ptx::tma_store_wait_read1();        // the store that last used this buffer is done
-        __syncwarp();
-#pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-          const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
-          const uint32_t u = *reinterpret_cast<const uint32_t*>(&v);
-          buf[j * 32 + lane] = (uint16_t)(u & 0xFFFFu);
-          buf[(j + 1) * 32 + lane] = (uint16_t)(u >> 16);
-        }
-        ptx::fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) {
-          if (m0 < p.Mdim && n0 + 32 * c < p.Ndim)
-            ptx::tma_store_2d(&tmapOut, m0, n0 + 32 * c, stg_base + (chunk & 1u) * 2048);
-          ptx::tma_store_commit();
-        }
+        for (int c = 0; c < SP_N / 32; ++c, ++chunk)
+          sparse_epilogue_chunk<32>(acc + 32 * c, c == SP_N / 32 - 1, release_bar, stg_ptr, stg_base, chunk, lane,
+                                    &tmapOut32, m0, n0 + 32 * c, p.Mdim, p.Ndim);
+      } else {
+#pragma unroll 1
+        for (int c = 0; c < SP_N / 16; ++c, ++chunk)
+          sparse_epilogue_chunk<16>(acc + 16 * c, c == SP_N / 16 - 1, release_bar, stg_ptr, stg_base, chunk, lane,
+                                    &tmapOut16, m0, n0 + 16 * c, p.Mdim, p.Ndim);
       }
     }
     if (lane == 0) ptx::tma_store_wait_all();
@@ -535,7 +428,6 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
     ptx::tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
   }
 }
-
 
 // ------------------------------------------------------------------------------------------
 // Dense weight gradient on CTA pairs, persistent.  D[i, j] = sum_t dY[t, i] X[t, j]: both
@@ -870,43 +762,13 @@ int make_tmap_meta(CUtensorMap* m, const void* ptr, uint64_t blocks) {
   return BIMASK_OK;
 }
 
-int run_sparse_pair(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim, int Kdim,
-                    uint16_t* out, int32_t* status_word, cudaStream_t s) {
-  constexpr int STAGES = 4;
-  using C = PairCfg<STAGES>;
-  CUtensorMap ta, tb, te;
-  int rc;
-  const int tiles_m = (Mdim + 127) / 128, tiles_k = (Kdim + 127) / 128;
-  if ((rc = make_tmap(&ta, vals, (uint64_t)Kdim / 2, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
-  if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, 128)) != BIMASK_OK) return rc;
-  if ((rc = make_tmap_meta(&te, hw_meta, (uint64_t)tiles_m * tiles_k)) != BIMASK_OK) return rc;
-  auto kern = spmm_pair_kernel<STAGES>;
-  if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
-  GemmParams p;
-  p.hw_meta = reinterpret_cast<const uint8_t*>(hw_meta);
-  p.tiles_k_meta = tiles_k;
-  p.Mdim = Mdim; p.Ndim = Ndim; p.Kdim = Kdim;
-  p.k_tiles_per_split = tiles_k;
-  p.out = out;
-  p.status_word = status_word;
-  p.tiles_m = (tiles_m + 1) / 2;
-  p.tiles_n = (Ndim + 255) / 256;
-  p.raster_group = 8;
-  dim3 grid(2 * p.tiles_m * p.tiles_n, 1, 1);
-  kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, p);
-  count_launch();
-  BIMASK_CUDA_OK(cudaGetLastError());
-  return BIMASK_OK;
-}
-
-
-// bf16 tensor map for TMA stores of 32 x 32 boxes into [rows][inner], no swizzle.
-int make_tmap_out(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t rows) {
+// bf16 tensor map for TMA stores of 32 x box_rows boxes into [rows][inner], no swizzle.
+int make_tmap_out(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t rows, uint32_t box_rows) {
   EncodeTiledFn fn = get_encode_fn();
   BIMASK_REQUIRE(fn != nullptr, BIMASK_ECUDA, "cuTensorMapEncodeTiled entry point not available");
   cuuint64_t dims[2] = {inner, rows};
   cuuint64_t strides[1] = {inner * 2};
-  cuuint32_t box[2] = {32, 32};
+  cuuint32_t box[2] = {32, box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
@@ -915,17 +777,39 @@ int make_tmap_out(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t rows
   return BIMASK_OK;
 }
 
+// Output-tile width of the CTA-pair 2:4 product.  Cost model in SM clocks, fitted to measurements
+// on the 16384 x 4096 / 4096 x 16384 layers: a tile's main loop takes 2 N clocks per 128-deep k
+// tile; N = 256 cannot overlap its epilogue (about 2500 clocks per tile); narrower tiles re-read
+// the compressed operand more often (L2 traffic), 0.3 % per column given up; the kernel's time is
+// the number of passes over the clusters times the tile time.
+int choose_sparse_n(int pair_tiles_m, int Ndim, int k_tiles, int clusters) {
+  int best_n = 256;
+  double best = 1e30;
+  for (int n = 256; n >= 160; n -= 16) {
+    const long long tiles = (long long)pair_tiles_m * ((Ndim + n - 1) / n);
+    const long long rounds = (tiles + clusters - 1) / clusters;
+    const double cost = (double)rounds * ((double)k_tiles * 2.0 * n + (n == 256 ? 2500.0 : 0.0)) *
+                        (1.0 + 0.003 * (256 - n));
+    if (cost < best) { best = cost; best_n = n; }
+  }
+  return best_n;
+}
+
 int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim,
                                int Kdim, uint16_t* out, int32_t* status_word, cudaStream_t s) {
   constexpr int STAGES = 4;
   using C = PairPCfg<STAGES>;
-  CUtensorMap ta, tb, te, to;
+  CUtensorMap ta, tb, te, to32, to16;
   int rc;
   const int tiles_m = (Mdim + 127) / 128, tiles_k = (Kdim + 127) / 128;
+  int sms = 148, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int n_tile = choose_sparse_n((tiles_m + 1) / 2, Ndim, tiles_k, sms / 2);
   if ((rc = make_tmap(&ta, vals, (uint64_t)Kdim / 2, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
-  if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, 128)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, n_tile / 2)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_meta(&te, hw_meta, (uint64_t)tiles_m * tiles_k)) != BIMASK_OK) return rc;
-  if ((rc = make_tmap_out(&to, out, (uint64_t)Mdim, (uint64_t)Ndim)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_out(&to32, out, (uint64_t)Mdim, (uint64_t)Ndim, 32)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_out(&to16, out, (uint64_t)Mdim, (uint64_t)Ndim, 16)) != BIMASK_OK) return rc;
   auto kern = spmm_pair_persistent_kernel<STAGES>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
@@ -935,15 +819,13 @@ int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const 
   p.k_tiles_per_split = tiles_k;
   p.out = out;
   p.status_word = status_word;
+  p.n_tile = n_tile;
   p.tiles_m = (tiles_m + 1) / 2;
-  p.tiles_n = (Ndim + 255) / 256;
+  p.tiles_n = (Ndim + n_tile - 1) / n_tile;
   p.raster_group = 8;
   const int total = p.tiles_m * p.tiles_n;
-  int sms = 148;
-  int dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int clusters = total < sms / 2 ? total : sms / 2;
-  kern<<<2 * clusters, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, to, p);
+  kern<<<2 * clusters, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, to32, to16, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
