@@ -81,8 +81,9 @@ int bimask_fwd_mask(const float* W, int I, int J, int N, int M, uint32_t* maskbi
   BIMASK_REQUIRE(aligned16(W) && aligned16(maskbits_f) && aligned16(vals_f) && aligned16(meta_f) && aligned16(hw_meta_f),
                  BIMASK_EINVAL, "bimask_fwd_mask: pointers must be 16-byte aligned");
   cudaStream_t s = (cudaStream_t)stream;
-  if ((rc = launch_fwd_mask(W, I, J, N, maskbits_f, vals_f, meta_f, s)) != BIMASK_OK) return rc;
-  return launch_hw_meta(meta_f, I, J, hw_meta_f, s);
+  const bool fused = (I % 128 == 0) && (J % 128 == 0);   // no padding in the metadata image
+  if ((rc = launch_fwd_mask(W, I, J, N, maskbits_f, vals_f, meta_f, fused ? hw_meta_f : nullptr, s)) != BIMASK_OK) return rc;
+  return fused ? BIMASK_OK : launch_hw_meta(meta_f, I, J, hw_meta_f, s);
 }
 
 int bimask_perm_search(const uint32_t* maskbits_f, int I, int J, int N, int M, int P, uint64_t seed,
@@ -123,8 +124,11 @@ int bimask_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* p
                      aligned16(vals_b) && aligned16(meta_b) && aligned16(hw_meta_b),
                  BIMASK_EINVAL, "bimask_bwd_mask: pointers must be 16-byte aligned");
   cudaStream_t s = (cudaStream_t)stream;
-  if ((rc = launch_bwd_mask(W, maskbits_f, perm, I, J, N, maskbits_b, vals_b, meta_b, s)) != BIMASK_OK) return rc;
-  return launch_hw_meta(meta_b, J, I, hw_meta_b, s);
+  const bool fused = (I % 128 == 0) && (J % 128 == 0);
+  if ((rc = launch_bwd_mask(W, maskbits_f, perm, I, J, N, maskbits_b, vals_b, meta_b, fused ? hw_meta_b : nullptr, s)) !=
+      BIMASK_OK)
+    return rc;
+  return fused ? BIMASK_OK : launch_hw_meta(meta_b, J, I, hw_meta_b, s);
 }
 
 static int check_gemm(int T, int I, int J) {
@@ -153,7 +157,7 @@ int bimask_spmm_dgrad(const uint16_t* dY, const int32_t* perm, const uint16_t* v
   BIMASK_REQUIRE(aligned16(dY) && aligned16(perm) && aligned16(vals_b) && aligned16(hw_meta_b) && aligned16(dX) &&
                      aligned16(ws),
                  BIMASK_EINVAL, "bimask_spmm_dgrad: pointers must be 16-byte aligned");
-  BIMASK_REQUIRE((size_t)I * 4 <= 100 * 1024, BIMASK_EUNSUPPORTED, "I = %d too large for the column permute pass (limit 25600)", I);
+  BIMASK_REQUIRE((size_t)I * 4 <= 200 * 1024, BIMASK_EUNSUPPORTED, "I = %d too large for the column permute pass (limit 51200)", I);
   const WsPlan w = plan_ws(T, I, J, 0);
   BIMASK_REQUIRE(ws_bytes >= w.dyp_off + w.dyp_bytes, BIMASK_EINVAL,
                  "bimask_spmm_dgrad: workspace too small (%zu bytes, need %zu)", ws_bytes, w.dyp_off + w.dyp_bytes);
@@ -195,8 +199,8 @@ int bimask_layer_step(const bimask_layer_args* a) {
                      aligned16(a->meta_f) && aligned16(a->hw_meta_f) && aligned16(a->maskbits_b) &&
                      aligned16(a->vals_b) && aligned16(a->meta_b) && aligned16(a->hw_meta_b),
                  BIMASK_EINVAL, "bimask_layer_step: pointers must be 16-byte aligned");
-  BIMASK_REQUIRE((size_t)a->I * 4 <= 100 * 1024, BIMASK_EUNSUPPORTED,
-                 "I = %d too large for the column permute pass (limit 25600)", a->I);
+  BIMASK_REQUIRE((size_t)a->I * 4 <= 200 * 1024, BIMASK_EUNSUPPORTED,
+                 "I = %d too large for the column permute pass (limit 51200)", a->I);
   if (a->do_search) {
     BIMASK_REQUIRE(a->P >= 1 && a->P <= 65535 && a->best_idx && a->counts, BIMASK_EINVAL,
                    "bimask_layer_step: search needs 1 <= P <= 65535, best_idx and counts");
@@ -215,8 +219,10 @@ int bimask_layer_step(const bimask_layer_args* a) {
   // with the bandwidth-bound chain on a second stream was measured and rejected: the co-resident
   // kernels contend for issue slots and the step became slower and erratic.)
   cudaStream_t s = (cudaStream_t)a->stream;
-  if ((rc = launch_fwd_mask(a->W, a->I, a->J, a->N, a->maskbits_f, a->vals_f, a->meta_f, s))) return rc;
-  if ((rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, s))) return rc;
+  const bool fused = (a->I % 128 == 0) && (a->J % 128 == 0);   // no padding in the metadata images
+  if ((rc = launch_fwd_mask(a->W, a->I, a->J, a->N, a->maskbits_f, a->vals_f, a->meta_f, fused ? a->hw_meta_f : nullptr, s)))
+    return rc;
+  if (!fused && (rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, s))) return rc;
   if ((rc = launch_spmm(a->vals_f, a->hw_meta_f, a->X, a->I, a->T, a->J, a->Y, a->status_word, s))) return rc;
   if (a->do_search) {
     const int32_t* cands = a->cands;
@@ -227,9 +233,10 @@ int bimask_layer_step(const bimask_layer_args* a) {
     if ((rc = launch_score(a->maskbits_f, cands, a->I, a->J, a->N, a->P, a->counts, s))) return rc;
     if ((rc = launch_pick(a->counts, cands, a->P, a->I, a->best_idx, a->perm, s))) return rc;
   }
-  if ((rc = launch_bwd_mask(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->maskbits_b, a->vals_b, a->meta_b, s)))
+  if ((rc = launch_bwd_mask(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->maskbits_b, a->vals_b, a->meta_b,
+                            fused ? a->hw_meta_b : nullptr, s)))
     return rc;
-  if ((rc = launch_hw_meta(a->meta_b, a->J, a->I, a->hw_meta_b, s))) return rc;
+  if (!fused && (rc = launch_hw_meta(a->meta_b, a->J, a->I, a->hw_meta_b, s))) return rc;
   if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, s))) return rc;
   if ((rc = launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, a->dX, a->status_word, s))) return rc;
   return launch_wgrad_impl(a->dY, a->X, a->T, a->I, a->J, a->dW, partials, a->status_word, s);

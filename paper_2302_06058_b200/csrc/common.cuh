@@ -30,11 +30,14 @@ int cuda_fail(cudaError_t e, const char* what);
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Launchers implemented in the .cu files (all enqueue on `s`, none synchronise).
+// hw_meta_or_null: when given (operand without padding: rows and K multiples of 128) the kernel
+// also writes the tensor-core metadata image; otherwise call launch_hw_meta afterwards.
 int launch_fwd_mask(const float* W, int I, int J, int N, uint32_t* maskbits, uint16_t* vals,
-                    uint32_t* meta, cudaStream_t s);
+                    uint32_t* meta, void* hw_meta_or_null, cudaStream_t s);
 int launch_hw_meta(const uint32_t* meta, int rows, int K, void* hw_meta, cudaStream_t s);
 int launch_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
-                    int N, uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, cudaStream_t s);
+                    int N, uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_or_null,
+                    cudaStream_t s);
 int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStream_t s);
 int launch_score(const uint32_t* maskbits_f, const int32_t* cands, int I, int J, int N, int P,
                  int64_t* counts, cudaStream_t s);

@@ -602,14 +602,14 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_consta
 }
 
 // ------------------------------------------------------------------------------------------
-// dY[:, perm]: a streaming pass.  A CTA takes R token rows at a time (R = 4, or 2 for long rows
-// so that the tile stays under 64 KB and the kernel can run beside a resident GEMM): it reads
+// dY[:, perm]: a streaming pass.  A CTA takes R token rows at a time (R = 4, or 2 for rows too
+// long for a 4-row tile in shared memory): it reads
 // them coalesced and stores them column-interleaved in shared memory (one 2R-byte word = the R
 // rows' values of one column), so the gather costs one shared load per permuted column for all
 // R rows; every thread then assembles eight consecutive permuted columns per row and writes
 // them with one 16-byte store.
 // ------------------------------------------------------------------------------------------
-constexpr int PERMUTE_THREADS = 512;
+constexpr int PERMUTE_THREADS = 1024;
 
 template <int R>
 __global__ void __launch_bounds__(PERMUTE_THREADS)
@@ -843,11 +843,11 @@ int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, 
 int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, uint16_t* dYp, cudaStream_t s) {
   static bool attr_done = false;
   if (!attr_done) {
-    BIMASK_CUDA_OK(cudaFuncSetAttribute(permute_cols_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
-    BIMASK_CUDA_OK(cudaFuncSetAttribute(permute_cols_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+    BIMASK_CUDA_OK(cudaFuncSetAttribute(permute_cols_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    BIMASK_CUDA_OK(cudaFuncSetAttribute(permute_cols_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     attr_done = true;
   }
-  const int R = (size_t)I * 8 <= 64 * 1024 ? 4 : 2;
+  const int R = (size_t)I * 8 <= 200 * 1024 ? 4 : 2;
   const size_t smem = (size_t)I * 2 * R;
   const int groups = (T + R - 1) / R;
   const int per_sm = smem <= 32 * 1024 ? 3 : smem <= 48 * 1024 ? 2 : 1;

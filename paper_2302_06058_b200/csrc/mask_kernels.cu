@@ -92,6 +92,19 @@ __device__ __forceinline__ uint32_t slots(uint32_t e, float w0, float w1, float 
   return v;
 }
 
+// One canonical code word (row r of the packed operand, 32-column word w) scattered into the
+// TMEM image described at hw_meta_kernel below: its low 16 bits (k-half 0) and high 16 bits
+// (k-half 1) land in two different lanes, each as one half of a 32-bit word whose other half
+// comes from the row 8 above or below.  Used when the operand has no padding (rows and K both
+// multiples of 128), so that the separate re-ordering pass is not needed.
+__device__ __forceinline__ void scatter_hw(uint16_t* __restrict__ hw16, int tiles_k, int r, int w, uint32_t word) {
+  const int rr = r & 127;
+  const size_t tile = (size_t)(r >> 7) * tiles_k + (w >> 2);
+  const size_t idx = (tile * 512 + (size_t)((rr & 7) + 16 * (rr >> 4)) * 4 + (w & 3)) * 2 + ((rr >> 3) & 1);
+  hw16[idx] = (uint16_t)(word & 0xFFFFu);
+  hw16[idx + 64] = (uint16_t)(word >> 16);               // lane + 8: 8 lanes x 4 words x 2 halves
+}
+
 // ---------------------------------------------------------------------------------------
 // Forward mask + pack.  W is treated as a flat stream of 4-element blocks (J % 32 == 0, so
 // blocks, 32-column words and rows all nest).  A warp owns chunks of 256 blocks: eight
@@ -105,7 +118,7 @@ template <bool N_IS_2>
 __global__ void __launch_bounds__(FWD_THREADS)
 fwd_mask_pack_kernel(const float4* __restrict__ W4, long long nblk, int N,
                      uint32_t* __restrict__ maskbits, uint4* __restrict__ vals4,
-                     uint32_t* __restrict__ meta) {
+                     uint32_t* __restrict__ meta, uint16_t* __restrict__ hw16, int jwords) {
   __shared__ uint32_t lut[64];
   __shared__ float4 stage[FWD_THREADS / 32][256];
   if (threadIdx.x < 64) lut[threadIdx.x] = lut_entry(threadIdx.x, 0xFu, N);
@@ -140,6 +153,10 @@ fwd_mask_pack_kernel(const float4* __restrict__ W4, long long nblk, int N,
       const long long word = (ch << 5) + lane;
       maskbits[word] = bits;
       meta[word] = codes;
+      if (hw16) {
+        const int r = (int)(word / jwords);
+        scatter_hw(hw16, jwords >> 2, r, (int)(word - (long long)r * jwords), codes);
+      }
       vals4[2 * word] = make_uint4(v[0], v[1], v[2], v[3]);
       vals4[2 * word + 1] = make_uint4(v[4], v[5], v[6], v[7]);
     }
@@ -154,24 +171,30 @@ fwd_mask_pack_kernel(const float4* __restrict__ W4, long long nblk, int N,
 // Rows / k beyond the matrix get the harmless code 0x4 (slots (0,1)), their values are 0.
 // ---------------------------------------------------------------------------------------
 __global__ void hw_meta_kernel(const uint32_t* __restrict__ meta, int rows, int kwords,
-                               int tiles_k, long long total, uint32_t* __restrict__ out) {
+                               int tiles_k, long long total_lanes, uint4* __restrict__ out) {
+  // one thread per (tile, lane): the lane's four columns are one 16-byte store
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= total) return;
-  const int c = (int)(idx & 3);
-  const int L = (int)((idx >> 2) & 127);
-  const long long tile = idx >> 9;
+  if (idx >= total_lanes) return;
+  const int L = (int)(idx & 127);
+  const long long tile = idx >> 7;
   const int kt = (int)(tile % tiles_k);
   const int mt = (int)(tile / tiles_k);
   const int m0 = L & 7, h = (L >> 3) & 1, m2 = L >> 4;
   const int r_lo = mt * 128 + m0 + 16 * m2;
   const int r_hi = r_lo + 8;
-  const int w = kt * 4 + c;
-  uint32_t lo = 0x4444u, hi = 0x4444u;
-  if (w < kwords) {
-    if (r_lo < rows) lo = (__ldg(meta + (long long)r_lo * kwords + w) >> (16 * h)) & 0xFFFFu;
-    if (r_hi < rows) hi = (__ldg(meta + (long long)r_hi * kwords + w) >> (16 * h)) & 0xFFFFu;
+  const uint32_t sel = h ? 0x7632u : 0x5410u;            // low halves or high halves of (lo, hi)
+  uint32_t o[4];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const int w = kt * 4 + c;
+    uint32_t lo = 0x44444444u, hi = 0x44444444u;
+    if (w < kwords) {
+      if (r_lo < rows) lo = __ldg(meta + (long long)r_lo * kwords + w);
+      if (r_hi < rows) hi = __ldg(meta + (long long)r_hi * kwords + w);
+    }
+    o[c] = __byte_perm(lo, hi, sel);
   }
-  out[idx] = lo | (hi << 16);
+  out[idx] = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -192,11 +215,11 @@ __device__ __forceinline__ uint32_t gather4(uint32_t x, int c) {
   return ((((x >> c) & 0x1111u) * 0x1248u) >> 12) & 15u;
 }
 
-__global__ void __launch_bounds__(BWD_THREADS)
+__global__ void __launch_bounds__(BWD_THREADS, 3)
 bwd_mask_pack_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,
                      const int32_t* __restrict__ perm, int I, int J, int N,
                      uint32_t* __restrict__ maskbits_b, uint32_t* __restrict__ vals_b,
-                     uint32_t* __restrict__ meta_b) {
+                     uint32_t* __restrict__ meta_b, uint16_t* __restrict__ hw16) {
   __shared__ uint32_t lut[1024];
   for (int e = threadIdx.x; e < 1024; e += BWD_THREADS) lut[e] = lut_entry(e & 63u, e >> 6, N);
   __syncthreads();
@@ -279,6 +302,7 @@ bwd_mask_pack_kernel(const float* __restrict__ W, const uint32_t* __restrict__ m
       dst[0] = make_uint4(vacc[c][0], vacc[c][1], vacc[c][2], vacc[c][3]);
       dst[1] = make_uint4(vacc[c][4], vacc[c][5], vacc[c][6], vacc[c][7]);
       meta_b[(size_t)(col + c) * mrow + (kfirst >> 3)] = cacc[c];
+      if (hw16) scatter_hw(hw16, I >> 7, col + c, kfirst >> 3, cacc[c]);
     }
   }
 }
@@ -286,7 +310,8 @@ bwd_mask_pack_kernel(const float* __restrict__ W, const uint32_t* __restrict__ m
 }  // namespace
 
 int launch_fwd_mask(const float* W, int I, int J, int N, uint32_t* maskbits, uint16_t* vals,
-                    uint32_t* meta, cudaStream_t s) {
+                    uint32_t* meta, void* hw_meta_or_null, cudaStream_t s) {
+  uint16_t* hw16 = reinterpret_cast<uint16_t*>(hw_meta_or_null);
   const long long nblk = (long long)I * J / 4;
   const long long nchunks = (nblk + 255) >> 8;
   long long ctas = (nchunks + 7) / 8;
@@ -294,10 +319,10 @@ int launch_fwd_mask(const float* W, int I, int J, int N, uint32_t* maskbits, uin
   if (ctas < 1) ctas = 1;
   if (N == 2)
     fwd_mask_pack_kernel<true><<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
-        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta);
+        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32);
   else
     fwd_mask_pack_kernel<false><<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
-        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta);
+        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -305,19 +330,21 @@ int launch_fwd_mask(const float* W, int I, int J, int N, uint32_t* maskbits, uin
 
 int launch_hw_meta(const uint32_t* meta, int rows, int K, void* hw_meta, cudaStream_t s) {
   const int tiles_m = (rows + 127) / 128, tiles_k = (K + 127) / 128;
-  const long long total = (long long)tiles_m * tiles_k * 512;
+  const long long total = (long long)tiles_m * tiles_k * 128;
   hw_meta_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(meta, rows, K / 32, tiles_k, total,
-                                                                 reinterpret_cast<uint32_t*>(hw_meta));
+                                                                 reinterpret_cast<uint4*>(hw_meta));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }
 
 int launch_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
-                    int N, uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, cudaStream_t s) {
+                    int N, uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_or_null,
+                    cudaStream_t s) {
   dim3 grid((I / 4 + BWD_KB - 1) / BWD_KB, (J + BWD_COLS - 1) / BWD_COLS);
   bwd_mask_pack_kernel<<<grid, BWD_THREADS, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b,
-                                                    reinterpret_cast<uint32_t*>(vals_b), meta_b);
+                                                    reinterpret_cast<uint32_t*>(vals_b), meta_b,
+                                                    reinterpret_cast<uint16_t*>(hw_meta_or_null));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;

@@ -28,7 +28,7 @@ __device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
 // every bucket with an insertion sort (exact order on the full key) and writes its slice.
 // Shared memory per CTA is about (I / Q) * 10 bytes, small enough to run beside a resident GEMM.
 // ---------------------------------------------------------------------------------------
-constexpr int GEN_THREADS = 512;
+constexpr int GEN_THREADS = 1024;
 
 __global__ void __launch_bounds__(GEN_THREADS)
 gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int q_log2, int cap,
@@ -253,13 +253,13 @@ int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStrea
   int lg = 1;
   while ((1 << lg) < I) ++lg;                             // one bucket per key on average
   int ql = 0;
-  while ((I >> ql) > 2048 && ql < lg - 1) ++ql;           // about 2048 keys per part
+  while ((I >> ql) > 8192 && ql < lg - 1) ++ql;           // at most 8192 keys per part (measured best)
   const int mean = (I + (1 << ql) - 1) >> ql;
   const int cap = ql == 0 ? I : mean + (mean / 4 > 256 ? mean / 4 : 256);
   const size_t smem = (size_t)cap * sizeof(unsigned long long) + ((size_t)1 << (lg - ql)) * sizeof(uint32_t);
   static bool attr_done = false;     // same value every time; a race only repeats the call
   if (!attr_done) {
-    BIMASK_CUDA_OK(cudaFuncSetAttribute(gen_candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+    BIMASK_CUDA_OK(cudaFuncSetAttribute(gen_candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     attr_done = true;
   }
   dim3 grid(P, 1 << ql);
