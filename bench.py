@@ -190,10 +190,11 @@ class ClockSampler:
 # GPU arm
 # --------------------------------------------------------------------------------------------
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM kernels on
-# config 5, from the ncu launch list summarised in profiles/cfg5_launch_list.md.
+# config 5, from the ncu launch list summarised in profiles/cfg5_launch_list.md (GEMM kernel only).
 NCU_TRAFFIC_BYTES = {
-    (5, 0, "wgrad"): 1.246e9 + 0.250e9, (5, 1, "wgrad"): None,
-    (5, 0, "spmm_fwd"): 0.604e9 + 0.249e9, (5, 0, "spmm_dgrad"): 0.879e9 + 0.062e9,
+    (5, 0, "wgrad"): 1.246e9 + 0.247e9, (5, 1, "wgrad"): 1.015e9 + 0.247e9,
+    (5, 0, "spmm_fwd"): 0.605e9 + 0.244e9, (5, 1, "spmm_fwd"): 0.878e9 + 0.062e9,
+    (5, 0, "spmm_dgrad"): 0.878e9 + 0.058e9, (5, 1, "spmm_dgrad"): 0.604e9 + 0.244e9,
 }
 
 
