@@ -7,6 +7,8 @@
 #include <stdarg.h>
 #include "../../include/bimask.h"
 
+struct CUtensorMap_st;
+
 namespace bimask {
 
 void set_error(const char* fmt, ...);       // defined in api.cu
@@ -28,6 +30,10 @@ int cuda_fail(cudaError_t e, const char* what);
   } while (0)
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// 2-D tensor map without swizzle (gemm_sm100.cu); dtype is a CUtensorMapDataType value.
+int make_tmap_plain(CUtensorMap_st* m, int dtype, const void* ptr, uint64_t inner, uint64_t outer, uint32_t box_inner,
+                    uint32_t box_outer, uint32_t elem_bytes);
 
 // Launchers implemented in the .cu files (all enqueue on `s`, none synchronise).
 // hw_meta_or_null: when given (operand without padding: rows and K multiples of 128) the kernel

@@ -6,6 +6,7 @@
 // selection is done on integer magnitude keys in registers, and the bit/nibble words are
 // assembled with warp reductions / ballots so that every store is a full word.
 #include "common.cuh"
+#include "sm100_ptx.cuh"   // smem_u32
 
 namespace bimask {
 
@@ -198,7 +199,8 @@ __global__ void hw_meta_kernel(const uint32_t* __restrict__ meta, int rows, int 
 }
 
 // ---------------------------------------------------------------------------------------
-// Backward mask + transposed pack.  A CTA owns 128 columns x 64 row-blocks (256 permuted rows);
+// Backward mask + transposed pack, register variant (used when J is not a multiple of 128).
+// A CTA owns 128 columns x 64 row-blocks (256 permuted rows);
 // warp w walks the eight consecutive row-blocks 8w .. 8w+7.  For a row-block it gathers the four
 // source rows perm[4k..4k+3] with one coalesced 128-bit load per row (lane = four columns) and
 // selects per column through the table.  The operand it feeds is transposed (row = column l of
@@ -307,6 +309,127 @@ bwd_mask_pack_kernel(const float* __restrict__ W, const uint32_t* __restrict__ m
   }
 }
 
+
+// ---------------------------------------------------------------------------------------
+// Backward mask + transposed pack, asynchronous-copy variant (J a multiple of 128).  A CTA owns
+// 128 columns x 64 row-blocks (256 permuted rows); warp w walks the eight consecutive row-blocks
+// 8w .. 8w+7.  Each warp runs its own three-deep ring of shared-memory stages filled with
+// cp.async (16 bytes per lane: the 512-byte slices of the four gathered rows, plus their 16 bytes
+// of forward-mask words), so the gather of row-block j+2 is in flight while row-block j is
+// processed and costs no registers.  Compute uses lane = column within each of the tile's four
+// 32-column words: conflict-free shared loads, and a warp ballot yields a complete backward-mask
+// word.  The operand being produced is transposed (row = column l of W, k contiguous): each lane
+// keeps the eight consecutive k results of its four columns in registers and writes them as
+// full 32-byte sectors.
+// ---------------------------------------------------------------------------------------
+constexpr int B4_COLS = 128, B4_KB = 64, B4_WARPS = 8, B4_THREADS = 32 * B4_WARPS, B4_RING = 3;
+constexpr int B4_STAGE = 4 * 512 + 64;                     // four row slices + four x 16 bytes of mask words
+constexpr int B4_SMEM = B4_WARPS * B4_RING * B4_STAGE + 4 * B4_KB * 16 + 1024 * 4 + B4_KB * 16;
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__global__ void __launch_bounds__(B4_THREADS, 3)
+bwd_mask_async_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,
+                      const int32_t* __restrict__ perm, int I, int J, int N,
+                      uint32_t* __restrict__ maskbits_b, uint32_t* __restrict__ vals_b,
+                      uint32_t* __restrict__ meta_b, uint16_t* __restrict__ hw16) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint8_t* ring = smem;                                                          // [warp][stage][B4_STAGE]
+  uint4* mb_s = reinterpret_cast<uint4*>(smem + B4_WARPS * B4_RING * B4_STAGE);  // [256 rows] x 4 mask words
+  uint32_t* lut = reinterpret_cast<uint32_t*>(mb_s + 4 * B4_KB);                 // [1024]
+  int4* perm_s = reinterpret_cast<int4*>(lut + 1024);                            // [64]
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int col0 = blockIdx.y * B4_COLS;                   // J % 128 == 0: the tile is always full
+  const int kb0 = blockIdx.x * B4_KB;
+  const int kb_here = min(B4_KB, (I >> 2) - kb0);          // multiple of 8 (I % 32 == 0)
+  const int jwords = J >> 5;
+  const unsigned last_row = (unsigned)(I - 1);
+
+  for (int e = threadIdx.x; e < 1024; e += B4_THREADS) lut[e] = lut_entry(e & 63u, e >> 6, N);
+  for (int kk = threadIdx.x; kk < kb_here; kk += B4_THREADS) {
+    const int4 p4 = __ldg(reinterpret_cast<const int4*>(perm) + kb0 + kk);
+    perm_s[kk] = make_int4((int)min((unsigned)p4.x, last_row), (int)min((unsigned)p4.y, last_row),
+                           (int)min((unsigned)p4.z, last_row), (int)min((unsigned)p4.w, last_row));
+  }
+  __syncthreads();
+  const int kw = 8 * warp;                                 // this warp's row-blocks kw .. kw+7 of the tile
+  if (kw < kb_here) {
+    uint8_t* my_ring = ring + warp * B4_RING * B4_STAGE;
+    const uint32_t ring_u32 = ptx::smem_u32(my_ring);
+    auto issue = [&](int j) {                              // start the gather of row-block kw + j
+      const int4 p4 = perm_s[kw + j];
+      const int r[4] = {p4.x, p4.y, p4.z, p4.w};
+      const uint32_t dst = ring_u32 + (j % B4_RING) * B4_STAGE;
+#pragma unroll
+      for (int m = 0; m < 4; ++m) cp_async16(dst + m * 512 + 16 * lane, W + (size_t)r[m] * J + col0 + 4 * lane);
+      if (lane < 4) cp_async16(dst + 2048 + 16 * lane, maskbits_f + (size_t)r[lane] * jwords + (col0 >> 5));
+      cp_async_commit();
+    };
+    issue(0);
+    issue(1);
+    uint32_t vacc[4][8];
+    uint32_t cacc[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (j + 2 < 8) issue(j + 2); else cp_async_commit();  // keep the group count uniform
+      cp_async_wait<2>();                                  // row-block j has landed
+      __syncwarp();
+      const float* ws = reinterpret_cast<const float*>(my_ring + (j % B4_RING) * B4_STAGE);
+      const uint4* fs = reinterpret_cast<const uint4*>(my_ring + (j % B4_RING) * B4_STAGE + 2048);
+      float w[4][4];
+      uint4 fw[4];
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        fw[m] = fs[m];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) w[m][c] = ws[m * 128 + 32 * c + lane];
+      }
+      __syncwarp();                                        // all lanes have read the stage
+      const int kk = kw + j;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const uint32_t f0 = c == 0 ? fw[0].x : c == 1 ? fw[0].y : c == 2 ? fw[0].z : fw[0].w;
+        const uint32_t f1 = c == 0 ? fw[1].x : c == 1 ? fw[1].y : c == 2 ? fw[1].z : fw[1].w;
+        const uint32_t f2 = c == 0 ? fw[2].x : c == 1 ? fw[2].y : c == 2 ? fw[2].z : fw[2].w;
+        const uint32_t f3 = c == 0 ? fw[3].x : c == 1 ? fw[3].y : c == 2 ? fw[3].z : fw[3].w;
+        const uint32_t valid = ((f0 >> lane) & 1u) | (((f1 >> lane) & 1u) << 1) | (((f2 >> lane) & 1u) << 2) |
+                               (((f3 >> lane) & 1u) << 3);
+        const uint32_t k0 = mag_key(w[0][c]), k1 = mag_key(w[1][c]), k2 = mag_key(w[2][c]), k3 = mag_key(w[3][c]);
+        const uint32_t e = lut[(valid << 6) | cmp6(k0, k1, k2, k3)];
+        vacc[c][j] = slots<false>(e, w[0][c], w[1][c], w[2][c], w[3][c], k0, k1, k2, k3);
+        cacc[c] |= ((e >> 4) & 15u) << (4 * j);
+        uint32_t b[4];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) b[m] = __ballot_sync(0xFFFFFFFFu, (e >> m) & 1u);
+        if (lane == 0) {
+#pragma unroll
+          for (int m = 0; m < 4; ++m) reinterpret_cast<uint32_t*>(mb_s + 4 * kk + m)[c] = b[m];
+        }
+      }
+    }
+    cp_async_wait<0>();
+    __syncwarp();
+    // this warp's 32 permuted rows of backward-mask words: one 16-byte store per lane
+    *reinterpret_cast<uint4*>(maskbits_b + (size_t)(4 * (kb0 + kw) + lane) * jwords + (col0 >> 5)) = mb_s[4 * kw + lane];
+    const size_t vrow = (size_t)I >> 2;                    // u32 (bf16 pairs) per row of vals_b
+    const size_t mrow = (size_t)I >> 5;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const int l = col0 + 32 * c + lane;
+      uint4* dst = reinterpret_cast<uint4*>(vals_b + (size_t)l * vrow + kb0 + kw);
+      dst[0] = make_uint4(vacc[c][0], vacc[c][1], vacc[c][2], vacc[c][3]);
+      dst[1] = make_uint4(vacc[c][4], vacc[c][5], vacc[c][6], vacc[c][7]);
+      meta_b[(size_t)l * mrow + ((kb0 + kw) >> 3)] = cacc[c];
+      if (hw16) scatter_hw(hw16, I >> 7, l, (kb0 + kw) >> 3, cacc[c]);
+    }
+  }
+}
+
 }  // namespace
 
 int launch_fwd_mask(const float* W, int I, int J, int N, uint32_t* maskbits, uint16_t* vals,
@@ -341,10 +464,25 @@ int launch_hw_meta(const uint32_t* meta, int rows, int K, void* hw_meta, cudaStr
 int launch_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                     int N, uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_or_null,
                     cudaStream_t s) {
-  dim3 grid((I / 4 + BWD_KB - 1) / BWD_KB, (J + BWD_COLS - 1) / BWD_COLS);
-  bwd_mask_pack_kernel<<<grid, BWD_THREADS, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b,
-                                                    reinterpret_cast<uint32_t*>(vals_b), meta_b,
-                                                    reinterpret_cast<uint16_t*>(hw_meta_or_null));
+  if (J % 128 != 0) {
+    // a row of mask words is then not a multiple of 16 bytes: no 16-byte asynchronous copies
+    dim3 grid((I / 4 + BWD_KB - 1) / BWD_KB, (J + BWD_COLS - 1) / BWD_COLS);
+    bwd_mask_pack_kernel<<<grid, BWD_THREADS, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b,
+                                                      reinterpret_cast<uint32_t*>(vals_b), meta_b,
+                                                      reinterpret_cast<uint16_t*>(hw_meta_or_null));
+    count_launch();
+    BIMASK_CUDA_OK(cudaGetLastError());
+    return BIMASK_OK;
+  }
+  static bool attr_done = false;
+  if (!attr_done) {
+    BIMASK_CUDA_OK(cudaFuncSetAttribute(bwd_mask_async_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, B4_SMEM));
+    attr_done = true;
+  }
+  dim3 grid((I / 4 + B4_KB - 1) / B4_KB, J / B4_COLS);
+  bwd_mask_async_kernel<<<grid, B4_THREADS, B4_SMEM, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b,
+                                                         reinterpret_cast<uint32_t*>(vals_b), meta_b,
+                                                         reinterpret_cast<uint16_t*>(hw_meta_or_null));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
