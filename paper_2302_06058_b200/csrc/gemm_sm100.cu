@@ -3,11 +3,13 @@
 //   sparse input grad D[l, t] = sum_k A'[l, k] dYp[t, k]       (Eq. 10; A' 2:4 along permuted k)
 //   dense weight grad D[i, j] = sum_t dY[t, i] X[t, j]         (straight-through estimator)
 //
-// One warp-specialised kernel template: a TMA producer thread fills a ring of shared-memory
-// stages (operands in the 128-byte-swizzled layouts the tensor core reads directly), one thread
-// issues tcgen05.mma (.sp for the 2:4 operand, whose index metadata is copied shared -> tensor
-// memory with tcgen05.cp right before the MMAs that use it), accumulators live in tensor
-// memory, and four epilogue warps drain them with tcgen05.ld and store the result.
+// All kernels are warp-specialised: a TMA producer thread fills a ring of shared-memory stages
+// (operands in the 128-byte-swizzled layouts the tensor core reads directly), one thread issues
+// tcgen05.mma (.sp for the 2:4 operand, whose index metadata is copied shared -> tensor memory
+// with tcgen05.cp right before the MMAs that use it), accumulators live in tensor memory, and
+// four epilogue warps drain them with tcgen05.ld and store the result.  The large-shape kernels
+// (spmm_pair_persistent_kernel, wgrad_pair_kernel) run CTA pairs persistently; spmm_single_kernel
+// is the one-CTA-per-tile form for operands of at most 128 rows or at most 128 tokens.
 //
 // Every wait on an mbarrier carries a cycle budget: when it runs out the kernel writes
 // BIMASK_ETIMEOUT to the caller's status word, all roles unwind, tensor memory is released and
@@ -24,15 +26,15 @@ namespace {
 constexpr long long WAIT_BUDGET = 4000000000ll;      // ~2 s of SM clocks
 constexpr int GEMM_THREADS = 192;                    // warp 0 TMA, warp 1 MMA, warps 2-5 epilogue
 
-template <bool SPARSE, int N_TILE, int STAGES>
+template <int N_TILE, int STAGES>
 struct Cfg {
   static constexpr int M_TILE = 128;
-  static constexpr int K_TILE = SPARSE ? 128 : 64;               // logical reduction elements per stage
+  static constexpr int K_TILE = 128;                             // logical reduction elements per stage
   static constexpr int A_BYTES = 16384;                          // 128 x 64 bf16 either way
   static constexpr int B_BYTES = N_TILE * K_TILE * 2;
-  static constexpr int E_BYTES = SPARSE ? 2048 : 0;
+  static constexpr int E_BYTES = 2048;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
-  static constexpr int META_COLS = SPARSE ? 4 : 0;
+  static constexpr int META_COLS = 4;
   static constexpr int TMEM_COLS = (N_TILE + META_COLS) <= 128 ? 128 : (N_TILE + META_COLS) <= 256 ? 256 : 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 };
@@ -63,11 +65,11 @@ __device__ __forceinline__ void raster(int id, int tiles_m, int tiles_n, int gro
   tn = in / gsize;
 }
 
-template <bool SPARSE, int N_TILE, int STAGES>
+template <int N_TILE, int STAGES>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-            const GemmParams p) {
-  using C = Cfg<SPARSE, N_TILE, STAGES>;
+spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
+                   const GemmParams p) {
+  using C = Cfg<N_TILE, STAGES>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -121,24 +123,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ C
         const uint32_t a_s = base + s * C::STAGE_BYTES;
         const uint32_t b_s = a_s + C::A_BYTES;
         ptx::mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
-        if (SPARSE) {
-          ptx::tma_load_2d(a_s, &tmapA, kt * 64, m0, full_bar(s));                      // 64 compressed x 128 rows
-          ptx::tma_load_2d(b_s, &tmapB, kt * 128, n0, full_bar(s));                     // k 0..63
-          ptx::tma_load_2d(b_s + N_TILE * 128, &tmapB, kt * 128 + 64, n0, full_bar(s)); // k 64..127
-          ptx::bulk_load(b_s + C::B_BYTES,
-                         p.hw_meta + ((size_t)tile_m * p.tiles_k_meta + kt) * 2048, 2048, full_bar(s));
-        } else {
-#pragma unroll
-          for (int b = 0; b < 2; ++b) ptx::tma_load_2d(a_s + b * 8192, &tmapA, m0 + 64 * b, kt * 64, full_bar(s));
-#pragma unroll
-          for (int b = 0; b < N_TILE / 64; ++b) ptx::tma_load_2d(b_s + b * 8192, &tmapB, n0 + 64 * b, kt * 64, full_bar(s));
-        }
+        ptx::tma_load_2d(a_s, &tmapA, kt * 64, m0, full_bar(s));                      // 64 compressed x 128 rows
+        ptx::tma_load_2d(b_s, &tmapB, kt * 128, n0, full_bar(s));                     // k 0..63
+        ptx::tma_load_2d(b_s + N_TILE * 128, &tmapB, kt * 128 + 64, n0, full_bar(s)); // k 64..127
+        ptx::bulk_load(b_s + C::B_BYTES,
+                       p.hw_meta + ((size_t)tile_m * p.tiles_k_meta + kt) * 2048, 2048, full_bar(s));
       }
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
     if (ptx::elect_one()) {
-      constexpr uint32_t idesc = ptx::idesc_bf16(128, N_TILE, !SPARSE, !SPARSE, SPARSE);
+      constexpr uint32_t idesc = ptx::idesc_bf16(128, N_TILE, false, false, true);
       bool ok = true;
       for (int it = 0; it < num_kt && ok; ++it) {
         const int s = it % STAGES;
@@ -147,21 +142,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ C
         ptx::tc_fence_after();
         const uint32_t a_s = base + s * C::STAGE_BYTES;
         const uint32_t b_s = a_s + C::A_BYTES;
-        if (SPARSE) {
-          ptx::tmem_cp_128x128b(tmem_meta, ptx::smem_desc(b_s + C::B_BYTES, 0, 128, 0));
+        ptx::tmem_cp_128x128b(tmem_meta, ptx::smem_desc(b_s + C::B_BYTES, 0, 128, 0));
 #pragma unroll
-          for (int kb = 0; kb < 4; ++kb) {
-            const uint64_t ad = ptx::smem_desc(a_s + kb * 32, 16, 1024, 2);
-            const uint64_t bd = ptx::smem_desc(b_s + (kb >> 1) * (N_TILE * 128) + (kb & 1) * 64, 16, 1024, 2);
-            ptx::mma_sparse(tmem_base, ad, bd, tmem_meta + (kb & ~1), idesc | (uint32_t)(kb & 1), (it | kb) != 0);
-          }
-        } else {
-#pragma unroll
-          for (int kb = 0; kb < 4; ++kb) {
-            const uint64_t ad = ptx::smem_desc(a_s + kb * 2048, 8192, 1024, 2);
-            const uint64_t bd = ptx::smem_desc(b_s + kb * 2048, 8192, 1024, 2);
-            ptx::mma_dense(tmem_base, ad, bd, idesc, (it | kb) != 0);
-          }
+        for (int kb = 0; kb < 4; ++kb) {
+          const uint64_t ad = ptx::smem_desc(a_s + kb * 32, 16, 1024, 2);
+          const uint64_t bd = ptx::smem_desc(b_s + (kb >> 1) * (N_TILE * 128) + (kb & 1) * 64, 16, 1024, 2);
+          ptx::mma_sparse(tmem_base, ad, bd, tmem_meta + (kb & ~1), idesc | (uint32_t)(kb & 1), (it | kb) != 0);
         }
         ptx::tc_commit(empty_bar(s));
       }
@@ -187,22 +173,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ C
           for (int j = 0; j < 32; ++j) r[j] = 0u;
         }
         const int nb = n0 + 32 * c;
-        if (SPARSE) {
-          __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
-          if (m < p.Mdim) {
+        __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
+        if (m < p.Mdim) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (nb + j < p.Ndim) out[(size_t)(nb + j) * p.Mdim + m] = __float2bfloat16_rn(__uint_as_float(r[j]));
-          }
-        } else {
-          float* out = reinterpret_cast<float*>(p.out) + (size_t)blockIdx.z * p.Mdim * p.Ndim;
-          if (m < p.Mdim && nb < p.Ndim) {          // Ndim % 32 == 0: a 32-column chunk is all in or all out
-            float4* dst = reinterpret_cast<float4*>(out + (size_t)m * p.Ndim + nb);
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-              dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                                   __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
-          }
+          for (int j = 0; j < 32; ++j)
+            if (nb + j < p.Ndim) out[(size_t)(nb + j) * p.Mdim + m] = __float2bfloat16_rn(__uint_as_float(r[j]));
         }
       }
     }
@@ -742,12 +717,12 @@ int set_smem_attr(K kernel, int bytes) {
 template <int N_TILE, int STAGES>
 int run_sparse(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim, int Kdim,
                uint16_t* out, int32_t* status_word, cudaStream_t s) {
-  using C = Cfg<true, N_TILE, STAGES>;
+  using C = Cfg<N_TILE, STAGES>;
   CUtensorMap ta, tb;
   int rc;
   if ((rc = make_tmap(&ta, vals, (uint64_t)Kdim / 2, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, N_TILE)) != BIMASK_OK) return rc;
-  auto kern = gemm_kernel<true, N_TILE, STAGES>;
+  auto kern = spmm_single_kernel<N_TILE, STAGES>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
   p.hw_meta = reinterpret_cast<const uint8_t*>(hw_meta);
@@ -902,7 +877,7 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
                       int32_t* status_word, cudaStream_t s) {
   int nt, splits, per;
   wgrad_plan(T, I, J, &nt, &splits, &per);
-  constexpr int STAGES = 4;
+  constexpr int STAGES = 6;
   using C = WgradCfg<STAGES>;
   CUtensorMap ta, tb;
   int rc;

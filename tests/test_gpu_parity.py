@@ -216,3 +216,69 @@ def test_error_paths_launch_nothing():
     assert e.value.code == bm.binding.BIMASK_EINVAL
     assert "workspace" in bm.bimask_last_error()
     torch.cuda.synchronize()
+
+
+def test_layer_step_host_matches_device_path():
+    """The end-to-end entry (host buffers in, host buffers out) gives the same bits as the device
+    path and leaves the status word at zero."""
+    I, J, T, N, P, seed = 256, 384, 200, 2, 5, 77
+    W = inputs.make_weight(I, J, 31)
+    X = inputs.make_activation(T, J, 32)
+    dY = inputs.make_activation(T, I, 33)
+    ref = run_layer_step(W, X, dY, N, 4, P, seed, do_search=True)
+    b = bm.alloc_layer_buffers(T, I, J, P)
+    b["W"] = torch.empty(I, J, device="cuda")
+    b["X"] = torch.empty(T, J, dtype=torch.bfloat16, device="cuda")
+    b["dY"] = torch.empty(T, I, dtype=torch.bfloat16, device="cuda")
+    dev_args = bm.make_layer_args(T, I, J, N, 4, P, seed, True, b)
+    host = {
+        "W": torch.from_numpy(W).pin_memory(),
+        "X": torch.from_numpy(X.view(np.int16)).view(torch.bfloat16).pin_memory(),
+        "dY": torch.from_numpy(dY.view(np.int16)).view(torch.bfloat16).pin_memory(),
+        "Y": torch.empty(T, I, dtype=torch.bfloat16).pin_memory(),
+        "dX": torch.empty(T, J, dtype=torch.bfloat16).pin_memory(),
+        "dW": torch.empty(I, J, dtype=torch.float32).pin_memory(),
+        "perm": torch.empty(I, dtype=torch.int32).pin_memory(),
+        "best_idx": torch.empty(1, dtype=torch.int32).pin_memory(),
+        "counts": torch.empty(P, dtype=torch.int64).pin_memory(),
+        "maskbits_f": torch.empty(I, J // 32, dtype=torch.int32).pin_memory(),
+        "maskbits_b": torch.empty(I, J // 32, dtype=torch.int32).pin_memory(),
+    }
+    hst = torch.full((1,), -9, dtype=torch.int32).pin_memory()
+    bm.bimask_layer_step_host(dev_args, bm.make_layer_args(T, I, J, N, 4, P, seed, True, host), hst)
+    assert int(hst.item()) == 0
+    assert torch.equal(host["Y"], ref["Y"].cpu())
+    assert torch.equal(host["dX"], ref["dX"].cpu())
+    assert torch.equal(host["dW"], ref["dW"].cpu())
+    assert torch.equal(host["perm"], ref["perm"].cpu())
+    assert torch.equal(host["counts"], ref["counts"].cpu())
+    assert int(host["best_idx"].item()) == int(ref["best_idx"].item())
+    assert torch.equal(host["maskbits_f"], ref["maskbits_f"].cpu())
+    assert torch.equal(host["maskbits_b"], ref["maskbits_b"].cpu())
+
+
+def test_layer_step_is_deterministic():
+    """Two runs on the same inputs give identical bits (no atomics on floating-point data)."""
+    I, J, T = 512, 256, 333
+    W = inputs.make_weight(I, J, 41)
+    X = inputs.make_activation(T, J, 42)
+    dY = inputs.make_activation(T, I, 43)
+    a = run_layer_step(W, X, dY, 2, 4, 4, 5, do_search=True)
+    b = run_layer_step(W, X, dY, 2, 4, 4, 5, do_search=True)
+    for name in ("Y", "dX", "dW", "perm", "counts", "maskbits_f", "maskbits_b", "vals_f", "vals_b", "meta_f", "meta_b",
+                 "hw_meta_f", "hw_meta_b"):
+        assert torch.equal(a[name], b[name]), name
+
+
+def test_small_layer_with_split_k_weight_gradient():
+    """Few output tiles and many tokens: the weight gradient is split along the tokens."""
+    I, J, T = 64, 96, 9000
+    W = inputs.make_weight(I, J, 51)
+    X = inputs.make_activation(T, J, 52)
+    dY = inputs.make_activation(T, I, 53)
+    b = run_layer_step(W, X, dY, 2, 4, 3, 6, do_search=True)
+    ref = O.layer_step(W, X, dY, 2, 4, 3, 6, do_search=True)
+    assert int(b["status_word"].item()) == 0
+    assert rel_err(b["dW"].cpu().numpy(), ref["dW"]) <= TOL
+    assert rel_err(b["Y"].float().cpu().numpy(), ref["Y"]) <= TOL
+    assert rel_err(b["dX"].float().cpu().numpy(), ref["dX"]) <= TOL
