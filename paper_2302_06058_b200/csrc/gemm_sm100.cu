@@ -639,6 +639,31 @@ permute_cols_kernel(const uint16_t* __restrict__ dY, const int32_t* __restrict__
   }
 }
 
+// Short rows (I <= 1024): a row is at most 2 KB and stays in L1, so each thread simply gathers
+// its eight permuted columns from global memory; rows are spread over all threads.
+__global__ void __launch_bounds__(256)
+permute_cols_small_kernel(const uint16_t* __restrict__ dY, const int32_t* __restrict__ perm, long long T, int I,
+                          uint16_t* __restrict__ dYp) {
+  const int per_row = I >> 3;
+  const long long total = T * per_row;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+    const long long t = e / per_row;
+    const int k8 = (int)(e - t * per_row);
+    const uint16_t* row = dY + t * I;
+    const int4 pa = __ldg(reinterpret_cast<const int4*>(perm) + 2 * k8);
+    const int4 pb = __ldg(reinterpret_cast<const int4*>(perm) + 2 * k8 + 1);
+    const int idx[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
+    uint32_t v[4];
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+      const uint32_t lo = __ldg(row + min(max(idx[2 * h], 0), I - 1));
+      const uint32_t hi = __ldg(row + min(max(idx[2 * h + 1], 0), I - 1));
+      v[h] = lo | (hi << 16);
+    }
+    reinterpret_cast<uint4*>(dYp + t * I)[k8] = make_uint4(v[0], v[1], v[2], v[3]);
+  }
+}
+
 // Sum of split-K partials: out[e] = sum_s part[s][e].
 __global__ void splitk_reduce_kernel(const float4* __restrict__ part, int splits, long long n4,
                                      float4* __restrict__ out) {
@@ -672,20 +697,71 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
+// Encoding a tensor map costs a few microseconds on the host, which matters when a layer's
+// kernels themselves run for ten.  A training loop passes the same buffers every step, so the
+// encoded maps are kept in a small per-thread cache keyed by everything that went into them.
+struct TmapKey {
+  const void* ptr;
+  uint64_t inner, outer, stride;
+  uint32_t box_inner, box_outer;
+  int dtype, swizzle;
+  bool operator==(const TmapKey& o) const {
+    return ptr == o.ptr && inner == o.inner && outer == o.outer && stride == o.stride && box_inner == o.box_inner &&
+           box_outer == o.box_outer && dtype == o.dtype && swizzle == o.swizzle;
+  }
+};
+
+int encode_cached(CUtensorMap* m, const TmapKey& key) {
+  constexpr int SLOTS = 32;
+  static thread_local TmapKey keys[SLOTS];
+  static thread_local CUtensorMap maps[SLOTS];
+  static thread_local bool used[SLOTS] = {false};
+  static thread_local int next = 0;
+  for (int i = 0; i < SLOTS; ++i)
+    if (used[i] && keys[i] == key) { *m = maps[i]; return BIMASK_OK; }
+  EncodeTiledFn fn = get_encode_fn();
+  BIMASK_REQUIRE(fn != nullptr, BIMASK_ECUDA, "cuTensorMapEncodeTiled entry point not available");
+  cuuint64_t dims[2] = {key.inner, key.outer};
+  cuuint64_t strides[1] = {key.stride};
+  cuuint32_t box[2] = {key.box_inner, key.box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(m, (CUtensorMapDataType)key.dtype, 2, const_cast<void*>(key.ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, (CUtensorMapSwizzle)key.swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  BIMASK_REQUIRE(r == CUDA_SUCCESS, BIMASK_ECUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+  keys[next] = key; maps[next] = *m; used[next] = true;
+  next = (next + 1) % SLOTS;
+  return BIMASK_OK;
+}
+
+int sm_count() {
+  static thread_local int cached_dev = -1, cached = 148;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (dev != cached_dev) {
+    int n = 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess) { cached = n; cached_dev = dev; }
+  }
+  return cached;
+}
+
 // 2-D bf16 tensor map: `inner` contiguous elements per row, `outer` rows, box = 64 x box_rows,
 // 128-byte swizzle, out-of-range elements read as zero.
 int make_tmap(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, uint32_t box_rows) {
-  EncodeTiledFn fn = get_encode_fn();
-  BIMASK_REQUIRE(fn != nullptr, BIMASK_ECUDA, "cuTensorMapEncodeTiled entry point not available");
-  cuuint64_t dims[2] = {inner, outer};
-  cuuint64_t strides[1] = {inner * 2};
-  cuuint32_t box[2] = {64, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  BIMASK_REQUIRE(r == CUDA_SUCCESS, BIMASK_ECUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
-  return BIMASK_OK;
+  return encode_cached(m, TmapKey{ptr, inner, outer, inner * 2, 64, box_rows, (int)CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                                  (int)CU_TENSOR_MAP_SWIZZLE_128B});
+}
+
+// The metadata image as a 2-D tensor of u32: 256 words per row, two rows per 2048-byte block.
+int make_tmap_meta(CUtensorMap* m, const void* ptr, uint64_t blocks) {
+  return encode_cached(m, TmapKey{ptr, 256, blocks * 2, 1024, 256, 2, (int)CU_TENSOR_MAP_DATA_TYPE_UINT32,
+                                  (int)CU_TENSOR_MAP_SWIZZLE_NONE});
+}
+
+// bf16 tensor map for TMA stores of 32 x box_rows boxes into [rows][inner], no swizzle.
+int make_tmap_out(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t rows, uint32_t box_rows) {
+  return encode_cached(m, TmapKey{ptr, inner, rows, inner * 2, 32, box_rows, (int)CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                                  (int)CU_TENSOR_MAP_SWIZZLE_NONE});
 }
 
 }  // namespace
@@ -693,17 +769,8 @@ int make_tmap(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, u
 // Generic 2-D tensor map without swizzle: `inner` contiguous elements of `elem_bytes` per row.
 int make_tmap_plain(CUtensorMap* m, int dtype, const void* ptr, uint64_t inner, uint64_t outer, uint32_t box_inner,
                     uint32_t box_outer, uint32_t elem_bytes) {
-  EncodeTiledFn fn = get_encode_fn();
-  BIMASK_REQUIRE(fn != nullptr, BIMASK_ECUDA, "cuTensorMapEncodeTiled entry point not available");
-  cuuint64_t dims[2] = {inner, outer};
-  cuuint64_t strides[1] = {inner * elem_bytes};
-  cuuint32_t box[2] = {box_inner, box_outer};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(m, (CUtensorMapDataType)dtype, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  BIMASK_REQUIRE(r == CUDA_SUCCESS, BIMASK_ECUDA, "cuTensorMapEncodeTiled (plain) failed with CUresult %d", (int)r);
-  return BIMASK_OK;
+  return encode_cached(m, TmapKey{ptr, inner, outer, inner * elem_bytes, box_inner, box_outer, dtype,
+                                  (int)CU_TENSOR_MAP_SWIZZLE_NONE});
 }
 
 namespace {
@@ -742,35 +809,7 @@ int run_sparse(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, i
 }
 
 
-// The metadata image as a 2-D tensor of u32: 256 words per row, two rows per 2048-byte block.
-int make_tmap_meta(CUtensorMap* m, const void* ptr, uint64_t blocks) {
-  EncodeTiledFn fn = get_encode_fn();
-  BIMASK_REQUIRE(fn != nullptr, BIMASK_ECUDA, "cuTensorMapEncodeTiled entry point not available");
-  cuuint64_t dims[2] = {256, blocks * 2};
-  cuuint64_t strides[1] = {1024};
-  cuuint32_t box[2] = {256, 2};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  BIMASK_REQUIRE(r == CUDA_SUCCESS, BIMASK_ECUDA, "cuTensorMapEncodeTiled (metadata) failed with CUresult %d", (int)r);
-  return BIMASK_OK;
-}
 
-// bf16 tensor map for TMA stores of 32 x box_rows boxes into [rows][inner], no swizzle.
-int make_tmap_out(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t rows, uint32_t box_rows) {
-  EncodeTiledFn fn = get_encode_fn();
-  BIMASK_REQUIRE(fn != nullptr, BIMASK_ECUDA, "cuTensorMapEncodeTiled entry point not available");
-  cuuint64_t dims[2] = {inner, rows};
-  cuuint64_t strides[1] = {inner * 2};
-  cuuint32_t box[2] = {32, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  BIMASK_REQUIRE(r == CUDA_SUCCESS, BIMASK_ECUDA, "cuTensorMapEncodeTiled (output) failed with CUresult %d", (int)r);
-  return BIMASK_OK;
-}
 
 // Output-tile width of the CTA-pair 2:4 product.  Cost model in SM clocks, fitted to measurements
 // on the 16384 x 4096 / 4096 x 16384 layers: a tile's main loop takes 2 N clocks per 128-deep k
@@ -797,8 +836,7 @@ int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const 
   CUtensorMap ta, tb, te, to32, to16;
   int rc;
   const int tiles_m = (Mdim + 127) / 128, tiles_k = (Kdim + 127) / 128;
-  int sms = 148, dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = sm_count();
   const int n_tile = choose_sparse_n((tiles_m + 1) / 2, Ndim, tiles_k, sms / 2);
   if ((rc = make_tmap(&ta, vals, (uint64_t)Kdim / 2, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, n_tile / 2)) != BIMASK_OK) return rc;
@@ -836,6 +874,15 @@ int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, 
 }
 
 int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, uint16_t* dYp, cudaStream_t s) {
+  if (I <= 1024) {
+    const long long total = (long long)T * (I >> 3);
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    permute_cols_small_kernel<<<(unsigned)blocks, 256, 0, s>>>(dY, perm, (long long)T, I, dYp);
+    count_launch();
+    BIMASK_CUDA_OK(cudaGetLastError());
+    return BIMASK_OK;
+  }
   static bool attr_done = false;
   if (!attr_done) {
     BIMASK_CUDA_OK(cudaFuncSetAttribute(permute_cols_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
@@ -895,8 +942,7 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
   p.tiles_n = (J + 255) / 256;
   p.raster_group = 8;
   const int items = p.tiles_m * p.tiles_n * splits;
-  int sms = 148, dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = sm_count();
   const int clusters = items < sms / 2 ? items : sms / 2;
   kern<<<2 * clusters, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p, splits);
   count_launch();
