@@ -275,6 +275,28 @@ def run_gpu(args):
         for _, _, largs in layers:
             bm.bimask_layer_step(largs)
 
+    graph = None
+    launches_per_step = None
+    if args.graph:
+        # capture one pass over all layers in a CUDA graph and replay it: removes the host-side
+        # launch cost, which dominates the small configurations
+        one_step()                                        # first calls set kernel attributes: not capturable
+        torch.cuda.synchronize()
+        cap_stream = torch.cuda.Stream()
+        cap_stream.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        n0 = bm.bimask_launch_count()
+        with torch.cuda.graph(graph, stream=cap_stream):
+            for _, _, largs in layers:
+                largs.stream = torch.cuda.current_stream().cuda_stream
+                bm.bimask_layer_step(largs)
+        launches_per_step = bm.bimask_launch_count() - n0
+        for _, _, largs in layers:
+            largs.stream = stream.cuda_stream
+        step_fn = graph.replay
+    else:
+        step_fn = one_step
+
     # ---- warm-up, then the timed region: K steps through bimask_layer_step ----
     gpu_uuid = str(local)
     try:
@@ -284,7 +306,7 @@ def run_gpu(args):
     sampler = ClockSampler(gpu_uuid)
     sampler.start()
     for _ in range(max(args.warmup, 3)):
-        one_step()
+        step_fn()
     barrier()
     t_load_begin = time.time()
     launches0 = bm.bimask_launch_count()
@@ -292,11 +314,13 @@ def run_gpu(args):
     barrier()
     ev0.record(stream)
     for _ in range(args.steps):
-        one_step()
+        step_fn()
     ev1.record(stream)
     barrier()
     step_ms_total = ev0.elapsed_time(ev1)
     launches = bm.bimask_launch_count() - launches0
+    if graph is not None:
+        launches = launches_per_step * args.steps          # replayed from the graph, counted at capture
 
     # ---- per-call breakdown over the same K steps (CUDA events between the C-ABI calls) ----
     names = ["fwd_mask", "spmm_fwd", "perm_search", "bwd_mask", "spmm_dgrad", "wgrad"]
@@ -399,7 +423,7 @@ def run_gpu(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"config {args.config} ({cfg.name})",
                        "layers": [[L.I, L.J, L.T] for L in cfg.layers], "N": cfg.N, "M": cfg.M, "P": cfg.P,
-                       "search_every_step": True, "parallelism": f"replicas x{world}",
+                       "search_every_step": True, "parallelism": f"replicas x{world}", "cuda_graph": bool(args.graph),
                        "l2": "inputs larger than L2 (W alone is %.0f MB per layer)" % (cfg.layers[0].I * cfg.layers[0].J * 4 / 1e6)
                        if cfg.layers[0].I * cfg.layers[0].J * 4 > 126e6 else "inputs smaller than L2: warm-cache numbers"},
             "clocks": clocks,
@@ -424,6 +448,7 @@ def main():
     ap.add_argument("--config", type=int, default=5, help="workload: 1..5 (default 5, the largest)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--graph", action="store_true", help="replay one captured pass (CUDA graph) in the timed region")
     ap.add_argument("--profile", action="store_true", help="run only the C-ABI calls of one layer (for ncu)")
     ap.add_argument("--layer", type=int, default=0)
     ap.add_argument("--ref-rows", type=int, default=1024)

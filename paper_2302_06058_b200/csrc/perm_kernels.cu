@@ -133,7 +133,7 @@ __device__ __forceinline__ uint32_t ineligible(uint32_t a, uint32_t b, uint32_t 
 }
 
 template <int N>
-__global__ void __launch_bounds__(SCORE_THREADS)
+__global__ void __launch_bounds__(SCORE_THREADS, 4)
 score_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cands, int I, int jwords,
              unsigned long long* __restrict__ counts) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -145,14 +145,22 @@ score_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cand
   uint32_t cnt = 0;
   if ((jwords & 3) == 0) {
     const int jq = jwords >> 2;
+    // the CTA's row indices first (one coalesced load, clamped), so that the row loads below do
+    // not wait on a dependent global load
+    __shared__ int4 idx_s[SCORE_KB_PER_CTA];
+    const unsigned last_row = (unsigned)(I - 1);
+    if (threadIdx.x < kb1 - kb0) {
+      const int4 r = __ldg(cand4 + kb0 + threadIdx.x);
+      idx_s[threadIdx.x] = make_int4((int)min((unsigned)r.x, last_row), (int)min((unsigned)r.y, last_row),
+                                     (int)min((unsigned)r.z, last_row), (int)min((unsigned)r.w, last_row));
+    }
+    __syncthreads();
     // two row blocks per trip: eight independent 128-bit loads in flight per lane
     for (int k = kb0 + warp; k < kb1; k += 2 * (SCORE_THREADS / 32)) {
       const int k2 = k + SCORE_THREADS / 32;
       const bool two = k2 < kb1;
-      int4 r = __ldg(cand4 + k);
-      int4 t = __ldg(cand4 + (two ? k2 : k));
-      r.x = min(max(r.x, 0), I - 1); r.y = min(max(r.y, 0), I - 1); r.z = min(max(r.z, 0), I - 1); r.w = min(max(r.w, 0), I - 1);
-      t.x = min(max(t.x, 0), I - 1); t.y = min(max(t.y, 0), I - 1); t.z = min(max(t.z, 0), I - 1); t.w = min(max(t.w, 0), I - 1);
+      const int4 r = idx_s[k - kb0];
+      const int4 t = idx_s[(two ? k2 : k) - kb0];
       const uint4* r0 = reinterpret_cast<const uint4*>(bits + (long long)r.x * jwords);
       const uint4* r1 = reinterpret_cast<const uint4*>(bits + (long long)r.y * jwords);
       const uint4* r2 = reinterpret_cast<const uint4*>(bits + (long long)r.z * jwords);
