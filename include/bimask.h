@@ -17,8 +17,12 @@
  *   - Return value: BIMASK_OK or a negative bimask_status.  On a negative return caused by
  *     argument validation nothing was launched.  bimask_last_error() gives a text for the
  *     calling thread's last failure.
- *   - Shapes: I % 32 == 0, J % 32 == 0, M == 4, 1 <= N <= 2 (1:4 is stored in the 2:4
- *     container with the spare slot holding +0).
+ *   - Shapes: I % 32 == 0, J % 32 == 0.  Patterns: M in {4, 8, 16}.  With N <= 2 (2:4, 1:4, 2:8,
+ *     1:8, 1:16, ...) every aligned group of four holds at most two survivors, so the result is
+ *     packed into the 2:4 container (a spare slot holds +0) and all calls apply.  With N > 2 (4:8)
+ *     only the mask bits exist: bimask_fwd_mask / bimask_bwd_mask then take NULL for vals, meta
+ *     and hw_meta, bimask_perm_search works as usual, and the products / bimask_layer_step return
+ *     BIMASK_EUNSUPPORTED.  (M = 4 with N > 2 is not implemented.)
  *   - `perm[k]` is the source row of permuted row k (gather: Wp[k,:] = W[perm[k],:]), 0-based.
  *   - Device-side trouble (a bounded wait that ran out) is reported by writing a non-zero
  *     code into *status_word (a device int the caller reads when it chooses to sync);
@@ -82,7 +86,8 @@ int bimask_fwd_mask(const float* W, int I, int J, int N, int M,
  *                       key  mix64(mix64(seed + 0x9E3779B97F4A7C15 (c+1)) ^ i)  (low 24 bits
  *                       replaced by i; mix64 = SplitMix64's output function).  Generated
  *                       candidates need I <= 16384 (BIMASK_EUNSUPPORTED beyond).
- *   This call alone accepts any I % 4 == 0 (the packed operands need I % 32 == 0).
+ *   This call alone accepts any I % M == 0 (the packed operands need I % 32 == 0); for M = 8, 16
+ *   the count kernel handles N <= 4 (and the trivial N == M).
  *   best_perm out I i32, best_idx out 1 i32, counts out P i64
  *   ws: scratch of at least bimask_workspace_bytes(...) bytes (holds the generated candidates). */
 int bimask_perm_search(const uint32_t* maskbits_f, int I, int J, int N, int M, int P, uint64_t seed,

@@ -355,7 +355,7 @@ def layer_step(W, X_bits, dY_bits, N, M, P, seed, do_search=True, perm=None, can
     out = {}
     B = forward_mask(W, N, M)
     out["B"] = B
-    packable = (M == 4 and N <= 2)      # only such masks fit the 2:4 operand format
+    packable = (M % 4 == 0 and N <= 2)  # at most two survivors in every aligned group of four: fits the 2:4 operand
     if packable:
         out["maskbits_f"], out["vals_f"], out["meta_f"] = forward_operand(W, B)
     if do_search:

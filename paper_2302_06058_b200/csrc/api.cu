@@ -25,12 +25,14 @@ int cuda_fail(cudaError_t e, const char* what) {
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-static int check_shape(int I, int J, int N, int M) {
-  BIMASK_REQUIRE(M == 4, BIMASK_EUNSUPPORTED, "M = %d: only M = 4 is implemented", M);
+// Shapes and pattern of the mask calls.  *pack: the pattern fits the 2:4 container (N <= 2).
+static int check_shape(int I, int J, int N, int M, bool* pack) {
+  BIMASK_REQUIRE(M == 4 || M == 8 || M == 16, BIMASK_EUNSUPPORTED, "M = %d: block lengths 4, 8 and 16 are implemented", M);
   BIMASK_REQUIRE(I > 0 && J > 0 && I % 32 == 0 && J % 32 == 0, BIMASK_EINVAL,
                  "I = %d, J = %d: both must be positive multiples of 32", I, J);
   BIMASK_REQUIRE(N >= 1 && N <= M, BIMASK_EINVAL, "N = %d out of range 1..%d", N, M);
-  BIMASK_REQUIRE(N <= 2, BIMASK_EUNSUPPORTED, "N:M = %d:%d does not fit the 2:4 container", N, M);
+  BIMASK_REQUIRE(M != 4 || N <= 2, BIMASK_EUNSUPPORTED, "N:M = %d:%d does not fit the 2:4 container", N, M);
+  *pack = N <= 2;
   return BIMASK_OK;
 }
 
@@ -75,12 +77,24 @@ size_t bimask_workspace_bytes(int T, int I, int J, int P) {
 
 int bimask_fwd_mask(const float* W, int I, int J, int N, int M, uint32_t* maskbits_f, uint16_t* vals_f,
                     uint32_t* meta_f, void* hw_meta_f, void* stream) {
-  int rc = check_shape(I, J, N, M);
+  bool pack = false;
+  int rc = check_shape(I, J, N, M, &pack);
   if (rc != BIMASK_OK) return rc;
-  BIMASK_REQUIRE(W && maskbits_f && vals_f && meta_f && hw_meta_f, BIMASK_EINVAL, "bimask_fwd_mask: null pointer");
+  BIMASK_REQUIRE(W && maskbits_f, BIMASK_EINVAL, "bimask_fwd_mask: null pointer");
+  if (pack) {
+    BIMASK_REQUIRE(vals_f && meta_f && hw_meta_f, BIMASK_EINVAL, "bimask_fwd_mask: null pointer");
+  } else {
+    BIMASK_REQUIRE(!vals_f && !meta_f && !hw_meta_f, BIMASK_EUNSUPPORTED,
+                   "N:M = %d:%d does not fit the 2:4 container: pass vals_f = meta_f = hw_meta_f = NULL for mask bits only",
+                   N, M);
+  }
   BIMASK_REQUIRE(aligned16(W) && aligned16(maskbits_f) && aligned16(vals_f) && aligned16(meta_f) && aligned16(hw_meta_f),
                  BIMASK_EINVAL, "bimask_fwd_mask: pointers must be 16-byte aligned");
   cudaStream_t s = (cudaStream_t)stream;
+  if (M != 4) {
+    if ((rc = launch_fwd_mask_generic(W, I, J, N, M, maskbits_f, vals_f, meta_f, s)) != BIMASK_OK) return rc;
+    return pack ? launch_hw_meta(meta_f, I, J, hw_meta_f, s) : BIMASK_OK;
+  }
   const bool fused = (I % 128 == 0) && (J % 128 == 0);   // no padding in the metadata image
   if ((rc = launch_fwd_mask(W, I, J, N, maskbits_f, vals_f, meta_f, fused ? hw_meta_f : nullptr, s)) != BIMASK_OK) return rc;
   return fused ? BIMASK_OK : launch_hw_meta(meta_f, I, J, hw_meta_f, s);
@@ -89,10 +103,11 @@ int bimask_fwd_mask(const float* W, int I, int J, int N, int M, uint32_t* maskbi
 int bimask_perm_search(const uint32_t* maskbits_f, int I, int J, int N, int M, int P, uint64_t seed,
                        const int32_t* cands_or_null, int32_t* best_perm, int32_t* best_idx, int64_t* counts,
                        void* ws, size_t ws_bytes, void* stream) {
-  BIMASK_REQUIRE(M == 4, BIMASK_EUNSUPPORTED, "M = %d: only M = 4 is implemented", M);
-  BIMASK_REQUIRE(I > 0 && J > 0 && I % 4 == 0 && J % 32 == 0, BIMASK_EINVAL,
-                 "I = %d, J = %d: I must be a positive multiple of 4, J of 32", I, J);
+  BIMASK_REQUIRE(M == 4 || M == 8 || M == 16, BIMASK_EUNSUPPORTED, "M = %d: block lengths 4, 8 and 16 are implemented", M);
+  BIMASK_REQUIRE(I > 0 && J > 0 && I % M == 0 && J % 32 == 0, BIMASK_EINVAL,
+                 "I = %d, J = %d: I must be a positive multiple of M, J of 32", I, J);
   BIMASK_REQUIRE(N >= 1 && N <= M, BIMASK_EINVAL, "N = %d out of range 1..%d", N, M);
+  BIMASK_REQUIRE(M == 4 || N <= 4 || N == M, BIMASK_EUNSUPPORTED, "N:M = %d:%d: the count kernel handles N <= 4", N, M);
   BIMASK_REQUIRE(P >= 1 && P <= 65535, BIMASK_EINVAL, "P = %d out of range 1..65535", P);
   BIMASK_REQUIRE(maskbits_f && best_perm && best_idx && counts, BIMASK_EINVAL, "bimask_perm_search: null pointer");
   BIMASK_REQUIRE(aligned16(maskbits_f) && aligned16(best_perm) && (!cands_or_null || aligned16(cands_or_null)) &&
@@ -110,20 +125,33 @@ int bimask_perm_search(const uint32_t* maskbits_f, int I, int J, int N, int M, i
     if ((rc = launch_gen_candidates(seed, P, I, gen, s)) != BIMASK_OK) return rc;
     cands = gen;
   }
-  if ((rc = launch_score(maskbits_f, cands, I, J, N, P, counts, s)) != BIMASK_OK) return rc;
+  if (M == 4) rc = launch_score(maskbits_f, cands, I, J, N, P, counts, s);
+  else rc = launch_score_generic(maskbits_f, cands, I, J, N, M, P, counts, s);
+  if (rc != BIMASK_OK) return rc;
   return launch_pick(counts, cands, P, I, best_idx, best_perm, s);
 }
 
 int bimask_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J, int N, int M,
                     uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_b, void* stream) {
-  int rc = check_shape(I, J, N, M);
+  bool pack = false;
+  int rc = check_shape(I, J, N, M, &pack);
   if (rc != BIMASK_OK) return rc;
-  BIMASK_REQUIRE(W && maskbits_f && perm && maskbits_b && vals_b && meta_b && hw_meta_b, BIMASK_EINVAL,
-                 "bimask_bwd_mask: null pointer");
+  BIMASK_REQUIRE(W && maskbits_f && perm && maskbits_b, BIMASK_EINVAL, "bimask_bwd_mask: null pointer");
+  if (pack) {
+    BIMASK_REQUIRE(vals_b && meta_b && hw_meta_b, BIMASK_EINVAL, "bimask_bwd_mask: null pointer");
+  } else {
+    BIMASK_REQUIRE(!vals_b && !meta_b && !hw_meta_b, BIMASK_EUNSUPPORTED,
+                   "N:M = %d:%d does not fit the 2:4 container: pass vals_b = meta_b = hw_meta_b = NULL for mask bits only",
+                   N, M);
+  }
   BIMASK_REQUIRE(aligned16(W) && aligned16(maskbits_f) && aligned16(perm) && aligned16(maskbits_b) &&
                      aligned16(vals_b) && aligned16(meta_b) && aligned16(hw_meta_b),
                  BIMASK_EINVAL, "bimask_bwd_mask: pointers must be 16-byte aligned");
   cudaStream_t s = (cudaStream_t)stream;
+  if (M != 4) {
+    if ((rc = launch_bwd_mask_generic(W, maskbits_f, perm, I, J, N, M, maskbits_b, vals_b, meta_b, s)) != BIMASK_OK) return rc;
+    return pack ? launch_hw_meta(meta_b, J, I, hw_meta_b, s) : BIMASK_OK;
+  }
   const bool fused = (I % 128 == 0) && (J % 128 == 0);
   if ((rc = launch_bwd_mask(W, maskbits_f, perm, I, J, N, maskbits_b, vals_b, meta_b, fused ? hw_meta_b : nullptr, s)) !=
       BIMASK_OK)
@@ -186,8 +214,13 @@ int bimask_wgrad(const uint16_t* dY, const uint16_t* X, int T, int I, int J, flo
 
 int bimask_layer_step(const bimask_layer_args* a) {
   BIMASK_REQUIRE(a != nullptr, BIMASK_EINVAL, "bimask_layer_step: null argument block");
-  int rc = check_shape(a->I, a->J, a->N, a->M);
+  bool pack = false;
+  int rc = check_shape(a->I, a->J, a->N, a->M, &pack);
   if (rc != BIMASK_OK) return rc;
+  BIMASK_REQUIRE(pack, BIMASK_EUNSUPPORTED,
+                 "N:M = %d:%d does not fit the 2:4 container, so the sparse products cannot run; the mask and search "
+                 "calls accept it",
+                 a->N, a->M);
   if ((rc = check_gemm(a->T, a->I, a->J)) != BIMASK_OK) return rc;
   BIMASK_REQUIRE(a->perm && a->ws && a->status_word && aligned16(a->ws), BIMASK_EINVAL,
                  "bimask_layer_step: null or misaligned pointer");
@@ -219,9 +252,13 @@ int bimask_layer_step(const bimask_layer_args* a) {
   // with the bandwidth-bound chain on a second stream was measured and rejected: the co-resident
   // kernels contend for issue slots and the step became slower and erratic.)
   cudaStream_t s = (cudaStream_t)a->stream;
-  const bool fused = (a->I % 128 == 0) && (a->J % 128 == 0);   // no padding in the metadata images
-  if ((rc = launch_fwd_mask(a->W, a->I, a->J, a->N, a->maskbits_f, a->vals_f, a->meta_f, fused ? a->hw_meta_f : nullptr, s)))
-    return rc;
+  // M = 4 with unpadded shapes writes the metadata images inside the mask kernels
+  const bool fused = a->M == 4 && (a->I % 128 == 0) && (a->J % 128 == 0);
+  if (a->M == 4)
+    rc = launch_fwd_mask(a->W, a->I, a->J, a->N, a->maskbits_f, a->vals_f, a->meta_f, fused ? a->hw_meta_f : nullptr, s);
+  else
+    rc = launch_fwd_mask_generic(a->W, a->I, a->J, a->N, a->M, a->maskbits_f, a->vals_f, a->meta_f, s);
+  if (rc) return rc;
   if (!fused && (rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, s))) return rc;
   if ((rc = launch_spmm(a->vals_f, a->hw_meta_f, a->X, a->I, a->T, a->J, a->Y, a->status_word, s))) return rc;
   if (a->do_search) {
@@ -230,12 +267,17 @@ int bimask_layer_step(const bimask_layer_args* a) {
       if ((rc = launch_gen_candidates(a->seed, a->P, a->I, gen, s))) return rc;
       cands = gen;
     }
-    if ((rc = launch_score(a->maskbits_f, cands, a->I, a->J, a->N, a->P, a->counts, s))) return rc;
+    if (a->M == 4) rc = launch_score(a->maskbits_f, cands, a->I, a->J, a->N, a->P, a->counts, s);
+    else rc = launch_score_generic(a->maskbits_f, cands, a->I, a->J, a->N, a->M, a->P, a->counts, s);
+    if (rc) return rc;
     if ((rc = launch_pick(a->counts, cands, a->P, a->I, a->best_idx, a->perm, s))) return rc;
   }
-  if ((rc = launch_bwd_mask(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->maskbits_b, a->vals_b, a->meta_b,
-                            fused ? a->hw_meta_b : nullptr, s)))
-    return rc;
+  if (a->M == 4)
+    rc = launch_bwd_mask(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->maskbits_b, a->vals_b, a->meta_b,
+                         fused ? a->hw_meta_b : nullptr, s);
+  else
+    rc = launch_bwd_mask_generic(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->M, a->maskbits_b, a->vals_b, a->meta_b, s);
+  if (rc) return rc;
   if (!fused && (rc = launch_hw_meta(a->meta_b, a->J, a->I, a->hw_meta_b, s))) return rc;
   if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, s))) return rc;
   if ((rc = launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, a->dX, a->status_word, s))) return rc;

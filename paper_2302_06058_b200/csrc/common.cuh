@@ -49,6 +49,13 @@ int launch_score(const uint32_t* maskbits_f, const int32_t* cands, int I, int J,
                  int64_t* counts, cudaStream_t s);
 int launch_pick(const int64_t* counts, const int32_t* cands, int P, int I, int32_t* best_idx,
                 int32_t* best_perm, cudaStream_t s);
+// N:M patterns with M = 8 or 16 (nm_generic_kernels.cu); vals / meta may be null (mask bits only).
+int launch_fwd_mask_generic(const float* W, int I, int J, int N, int M, uint32_t* maskbits, uint16_t* vals_or_null,
+                            uint32_t* meta_or_null, cudaStream_t s);
+int launch_score_generic(const uint32_t* bits, const int32_t* cands, int I, int J, int N, int M, int P,
+                         int64_t* counts, cudaStream_t s);
+int launch_bwd_mask_generic(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J, int N, int M,
+                            uint32_t* maskbits_b, uint16_t* vals_b_or_null, uint32_t* meta_b_or_null, cudaStream_t s);
 int launch_check_perms(const int32_t* cands, int P, int I, int32_t* ok, uint8_t* seen, cudaStream_t s);
 int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, uint16_t* dYp, cudaStream_t s);
 int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim, int Kdim,

@@ -1,0 +1,92 @@
+// Device helpers shared by the mask kernels: magnitude keys, bf16 rounding, and the table-driven
+// selection inside one group of four.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace bimask {
+namespace {
+
+__device__ __forceinline__ uint32_t mag_key(float w) { return __float_as_uint(w) & 0x7FFFFFFFu; }
+
+// fp32 -> bf16, round to nearest even; NaN -> quiet NaN keeping sign and top payload bits.
+__device__ __forceinline__ uint32_t to_bf16(float w) {
+  uint32_t u = __float_as_uint(w);
+  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (u >> 16) | 0x40u;
+  return (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;
+}
+
+// Selection inside one block of four, table driven.  The six pairwise magnitude comparisons
+// (b_qm = key_q >= key_m for q < m) and the four candidate bits index a table whose entry holds
+// everything the block needs:
+//   bits [0,4)   keep mask: element m is kept when it is a candidate and fewer than N candidates
+//                beat it; q beats m when key_q > key_m, or key_q == key_m with q < m
+//   bits [4,8)   index code idx0 | idx1 << 2 of the 2:4 container (pad rule for < 2 kept)
+//   bit 8 / 9    slot 0 / slot 1 holds a kept element (else the slot is +0)
+//   bits [16,32) byte-permute selector that picks the two slots out of the four bf16 values
+// The table (64 entries for "all candidates", 1024 with candidate bits) is rebuilt in shared
+// memory by every CTA from the rule itself.
+__device__ __forceinline__ uint32_t lut_entry(uint32_t cmp, uint32_t valid, int N) {
+  const uint32_t b01 = (cmp >> 5) & 1u, b02 = (cmp >> 4) & 1u, b03 = (cmp >> 3) & 1u;
+  const uint32_t b12 = (cmp >> 2) & 1u, b13 = (cmp >> 1) & 1u, b23 = cmp & 1u;
+  const uint32_t v0 = valid & 1u, v1 = (valid >> 1) & 1u, v2 = (valid >> 2) & 1u, v3 = (valid >> 3) & 1u;
+  const uint32_t r0 = (v1 & (b01 ^ 1u)) + (v2 & (b02 ^ 1u)) + (v3 & (b03 ^ 1u));
+  const uint32_t r1 = (v0 & b01) + (v2 & (b12 ^ 1u)) + (v3 & (b13 ^ 1u));
+  const uint32_t r2 = (v0 & b02) + (v1 & b12) + (v3 & (b23 ^ 1u));
+  const uint32_t r3 = (v0 & b03) + (v1 & b13) + (v2 & b23);
+  const uint32_t n = (uint32_t)N;
+  const uint32_t kb = (v0 & (r0 < n)) | ((v1 & (r1 < n)) << 1) | ((v2 & (r2 < n)) << 2) | ((v3 & (r3 < n)) << 3);
+  const int pop = __popc(kb);
+  uint32_t idx0 = 0u, idx1 = 1u;
+  if (pop >= 2) {
+    idx0 = (uint32_t)(__ffs(kb) - 1);
+    idx1 = 31u - (uint32_t)__clz(kb);
+  } else if (pop == 1) {
+    const uint32_t lo = (uint32_t)(__ffs(kb) - 1);
+    idx1 = lo < 1u ? 1u : lo;
+  }
+  const uint32_t sel = (2u * idx0) | ((2u * idx0 + 1u) << 4) | ((2u * idx1) << 8) | ((2u * idx1 + 1u) << 12);
+  return kb | (idx0 << 4) | (idx1 << 6) | (((kb >> idx0) & 1u) << 8) | (((kb >> idx1) & 1u) << 9) | (sel << 16);
+}
+
+// Six comparison bits of a block, b01 first (bit 5) ... b23 last (bit 0).  Keys are < 2^31, so
+// key_m - key_q - 1 is negative exactly when key_q >= key_m; a funnel shift moves each sign bit in.
+__device__ __forceinline__ uint32_t cmp6(uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3) {
+  uint32_t c = 0;
+  c = __funnelshift_l(k1 - k0 - 1u, c, 1);
+  c = __funnelshift_l(k2 - k0 - 1u, c, 1);
+  c = __funnelshift_l(k3 - k0 - 1u, c, 1);
+  c = __funnelshift_l(k2 - k1 - 1u, c, 1);
+  c = __funnelshift_l(k3 - k1 - 1u, c, 1);
+  c = __funnelshift_l(k3 - k2 - 1u, c, 1);
+  return c;
+}
+
+// {hi, lo} -> packed bf16x2, round to nearest even (NaN comes out as 0x7fff: see slots()).
+__device__ __forceinline__ uint32_t cvt_bf16x2(float hi, float lo) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+
+// The two bf16 slots of a block from its table entry.  Fast path: two packed conversions and
+// one byte permute; a block that holds a NaN takes the exact integer conversion instead so that
+// the NaN payload rule (quiet bit set, sign and top payload bits kept) holds bit for bit.
+template <bool BOTH_KEPT>
+__device__ __forceinline__ uint32_t slots(uint32_t e, float w0, float w1, float w2, float w3,
+                                          uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3) {
+  if (max(max(k0, k1), max(k2, k3)) > 0x7F800000u) {
+    const uint32_t idx0 = (e >> 4) & 3u, idx1 = (e >> 6) & 3u;
+    const float s0 = idx0 == 0 ? w0 : idx0 == 1 ? w1 : w2;      // idx0 is never 3
+    const float s1 = idx1 == 1 ? w1 : idx1 == 2 ? w2 : w3;      // idx1 is never 0
+    const uint32_t a = (e & 0x100u) ? to_bf16(s0) : 0u;
+    const uint32_t b = (e & 0x200u) ? to_bf16(s1) : 0u;
+    return a | (b << 16);
+  }
+  uint32_t v = __byte_perm(cvt_bf16x2(w1, w0), cvt_bf16x2(w3, w2), e >> 16);
+  if (!BOTH_KEPT) v &= (((e >> 8) & 1u) * 0xFFFFu) | (((e >> 9) & 1u) * 0xFFFF0000u);
+  return v;
+}
+
+}  // namespace
+}  // namespace bimask

@@ -1,0 +1,284 @@
+// N:M patterns beyond 2:4 and 1:4 (the paper also trains 4:8, 2:8, 1:8 and 1:16): forward mask,
+// eligible-block count and backward mask for block lengths M = 8 and 16.  Selection is the same
+// rank rule as for M = 4 (an element is kept when fewer than N candidates of its block beat it;
+// ties go to the lower index), evaluated with all M (M - 1) / 2 pairwise comparisons in registers.
+// When N <= 2 every aligned group of four holds at most two survivors, so the result is packed
+// into the same 2:4 tensor-core operand as before (the index code of a group depends on its keep
+// mask alone); patterns with N > 2 (4:8) produce mask bits only.
+#include "common.cuh"
+#include "mask_common.cuh"
+
+namespace bimask {
+
+namespace {
+
+// keep mask of one block of M keys: bit m set iff candidate m is beaten by fewer than N candidates
+template <int M>
+__device__ __forceinline__ uint32_t keep_block(const uint32_t (&key)[M], uint32_t valid, int N) {
+  int rank[M];
+#pragma unroll
+  for (int m = 0; m < M; ++m) rank[m] = 0;
+#pragma unroll
+  for (int m = 1; m < M; ++m)
+#pragma unroll
+    for (int q = 0; q < m; ++q) {
+      const bool q_beats_m = key[q] >= key[m];             // equal keys: the lower index wins
+      rank[m] += (q_beats_m && ((valid >> q) & 1u)) ? 1 : 0;
+      rank[q] += (!q_beats_m && ((valid >> m) & 1u)) ? 1 : 0;
+    }
+  uint32_t kb = 0;
+#pragma unroll
+  for (int m = 0; m < M; ++m) kb |= (((valid >> m) & 1u) && rank[m] < N) ? (1u << m) : 0u;
+  return kb;
+}
+
+// ---------------------------------------------------------------------------------------
+// Forward mask (+ pack when PACK).  One lane per block of M consecutive weights; the 32 / M lanes
+// that share a 32-column word OR their pieces together.
+// ---------------------------------------------------------------------------------------
+template <int M, bool PACK>
+__global__ void __launch_bounds__(256)
+fwd_mask_generic_kernel(const float4* __restrict__ W4, long long nblocks, int N,
+                        uint32_t* __restrict__ maskbits, uint32_t* __restrict__ vals32,
+                        uint32_t* __restrict__ meta) {
+  constexpr int LPW = 32 / M;                               // lanes per 32-column word
+  constexpr int G = M / 4;                                  // groups of four per block
+  __shared__ uint32_t pad16[16];                            // container entry of a group from its keep mask
+  if (threadIdx.x < 16) pad16[threadIdx.x] = lut_entry(0u, threadIdx.x, 4);
+  __syncthreads();
+  const int lane = threadIdx.x & 31;
+  const uint32_t gmask = ((LPW == 4 ? 0xFu : 0x3u)) << (lane & ~(LPW - 1));
+  const int sh = M * (lane & (LPW - 1));
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const long long nround = (nblocks + 31) & ~31ll;          // whole warps stay in the loop together
+  for (long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x; b < nround; b += stride) {
+    const bool live = b < nblocks;
+    float w[M];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const float4 v = live ? __ldg(W4 + b * G + g) : make_float4(0.f, 0.f, 0.f, 0.f);
+      w[4 * g] = v.x; w[4 * g + 1] = v.y; w[4 * g + 2] = v.z; w[4 * g + 3] = v.w;
+    }
+    uint32_t key[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) key[m] = mag_key(w[m]);
+    const uint32_t kb = keep_block<M>(key, (M == 16 ? 0xFFFFu : 0xFFu), N);
+    uint32_t codes = 0;
+    if (PACK) {
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const uint32_t e = pad16[(kb >> (4 * g)) & 15u];
+        if (live)
+          vals32[b * G + g] = slots<false>(e, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3], key[4 * g],
+                                           key[4 * g + 1], key[4 * g + 2], key[4 * g + 3]);
+        codes |= ((e >> 4) & 15u) << (4 * g);
+      }
+    }
+    const uint32_t wb = __reduce_or_sync(gmask, kb << sh);
+    const uint32_t wm = __reduce_or_sync(gmask, codes << sh);
+    if (live && (lane & (LPW - 1)) == 0) {
+      maskbits[b / LPW] = wb;
+      if (PACK) meta[b / LPW] = wm;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Eligible-block count for blocks of M permuted rows: a column is eligible when at most N of the
+// M rows have its bit set.  Bit-sliced saturating counter: level[j] = "at least j rows so far".
+// ---------------------------------------------------------------------------------------
+template <int N>
+struct SatCount {
+  uint32_t lv[N + 1];
+  __device__ __forceinline__ void clear() {
+#pragma unroll
+    for (int j = 0; j <= N; ++j) lv[j] = 0u;
+  }
+  __device__ __forceinline__ void add(uint32_t x) {
+#pragma unroll
+    for (int j = N; j >= 1; --j) lv[j] |= lv[j - 1] & x;
+    lv[0] |= x;
+  }
+  __device__ __forceinline__ uint32_t eligible() const { return ~lv[N]; }   // fewer than N + 1 rows set
+};
+
+template <int N, int M>
+__global__ void __launch_bounds__(256)
+score_generic_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cands, int I, int jwords,
+                     int blocks_per_cta, unsigned long long* __restrict__ counts) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int c = blockIdx.y;
+  const int nblk = I / M;
+  const int b0 = blockIdx.x * blocks_per_cta;
+  const int b1 = min(nblk, b0 + blocks_per_cta);
+  const int32_t* cand = cands + (long long)c * I;
+  const unsigned last_row = (unsigned)(I - 1);
+  uint32_t cnt = 0;
+  for (int b = b0 + warp; b < b1; b += 8) {
+    int rows[M];
+#pragma unroll
+    for (int g = 0; g < M / 4; ++g) {
+      const int4 r = __ldg(reinterpret_cast<const int4*>(cand + (long long)b * M) + g);
+      rows[4 * g] = (int)min((unsigned)r.x, last_row); rows[4 * g + 1] = (int)min((unsigned)r.y, last_row);
+      rows[4 * g + 2] = (int)min((unsigned)r.z, last_row); rows[4 * g + 3] = (int)min((unsigned)r.w, last_row);
+    }
+    for (int q = lane; q < jwords; q += 32) {
+      SatCount<N> s;
+      s.clear();
+#pragma unroll
+      for (int m = 0; m < M; ++m) s.add(__ldg(bits + (long long)rows[m] * jwords + q));
+      cnt += __popc(s.eligible());
+    }
+  }
+  cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+  __shared__ uint32_t part[8];
+  if (lane == 0) part[warp] = cnt;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long s = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) s += part[w];
+    atomicAdd(counts + c, s);
+  }
+}
+
+__global__ void fill_counts_kernel(long long* counts, int P, long long v) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < P) counts[i] = v;
+}
+
+// ---------------------------------------------------------------------------------------
+// Backward mask (+ transposed pack when PACK).  A warp owns 32 permuted rows x 32 columns (lane =
+// column): 32 / M blocks of M rows, which is exactly one metadata word and one 32-byte sector of
+// packed values per column.  Rows are gathered with one coalesced 128-byte load each.
+// ---------------------------------------------------------------------------------------
+template <int M, bool PACK>
+__global__ void __launch_bounds__(256)
+bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,
+                        const int32_t* __restrict__ perm, int I, int J, int N,
+                        uint32_t* __restrict__ maskbits_b, uint32_t* __restrict__ vals_b,
+                        uint32_t* __restrict__ meta_b) {
+  constexpr int NB = 32 / M;                                // blocks per 32-row pass
+  constexpr int G = M / 4;
+  __shared__ uint32_t pad16[16];
+  if (threadIdx.x < 16) pad16[threadIdx.x] = lut_entry(0u, threadIdx.x, 4);
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int jwords = J >> 5;
+  const int cw = blockIdx.y * 8 + warp;                     // column word of this warp
+  const int pass = blockIdx.x;                              // 32 permuted rows
+  if (cw >= jwords) return;
+  const int col = 32 * cw + lane;
+  const unsigned last_row = (unsigned)(I - 1);
+  const int my_src = (int)min((unsigned)__ldg(perm + 32 * pass + lane), last_row);   // lane r: source of permuted row r
+  uint32_t my_word = 0;                                     // lane r ends up with the mask word of permuted row r
+  uint32_t vacc[8];
+  uint32_t cacc = 0;
+#pragma unroll
+  for (int nb = 0; nb < NB; ++nb) {
+    float w[M];
+    uint32_t key[M];
+    uint32_t valid = 0;
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+      const int src = __shfl_sync(0xFFFFFFFFu, my_src, nb * M + m);
+      w[m] = __ldg(W + (size_t)src * J + col);
+      const uint32_t f = __ldg(maskbits_f + (size_t)src * jwords + cw);
+      valid |= ((f >> lane) & 1u) << m;
+      key[m] = mag_key(w[m]);
+    }
+    const uint32_t kb = keep_block<M>(key, valid, N);
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+      const uint32_t word = __ballot_sync(0xFFFFFFFFu, (kb >> m) & 1u);
+      if (lane == nb * M + m) my_word = word;
+    }
+    if (PACK) {
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const uint32_t e = pad16[(kb >> (4 * g)) & 15u];
+        vacc[nb * G + g] = slots<false>(e, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3], key[4 * g],
+                                        key[4 * g + 1], key[4 * g + 2], key[4 * g + 3]);
+        cacc |= ((e >> 4) & 15u) << (4 * (nb * G + g));
+      }
+    }
+  }
+  maskbits_b[(size_t)(32 * pass + lane) * jwords + cw] = my_word;
+  if (PACK) {
+    uint4* dst = reinterpret_cast<uint4*>(vals_b + (size_t)col * (I >> 2) + 8 * pass);
+    dst[0] = make_uint4(vacc[0], vacc[1], vacc[2], vacc[3]);
+    dst[1] = make_uint4(vacc[4], vacc[5], vacc[6], vacc[7]);
+    meta_b[(size_t)col * (I >> 5) + pass] = cacc;
+  }
+}
+
+}  // namespace
+
+int launch_fwd_mask_generic(const float* W, int I, int J, int N, int M, uint32_t* maskbits, uint16_t* vals_or_null,
+                            uint32_t* meta_or_null, cudaStream_t s) {
+  const long long nblocks = (long long)I * J / M;
+  long long ctas = (nblocks + 255) / 256;
+  if (ctas > 148 * 16) ctas = 148 * 16;
+  const float4* W4 = reinterpret_cast<const float4*>(W);
+  uint32_t* v32 = reinterpret_cast<uint32_t*>(vals_or_null);
+  const bool pack = vals_or_null != nullptr;
+  if (M == 8) {
+    if (pack) fwd_mask_generic_kernel<8, true><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
+    else fwd_mask_generic_kernel<8, false><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
+  } else {
+    if (pack) fwd_mask_generic_kernel<16, true><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
+    else fwd_mask_generic_kernel<16, false><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
+  }
+  count_launch();
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
+template <int M>
+static int launch_score_m(const uint32_t* bits, const int32_t* cands, int I, int J, int N, int P, int64_t* counts,
+                          cudaStream_t s) {
+  const int nblk = I / M;
+  const int per_cta = 64;
+  dim3 grid((nblk + per_cta - 1) / per_cta, P);
+  unsigned long long* cnt = reinterpret_cast<unsigned long long*>(counts);
+  switch (N) {
+    case 1: score_generic_kernel<1, M><<<grid, 256, 0, s>>>(bits, cands, I, J / 32, per_cta, cnt); break;
+    case 2: score_generic_kernel<2, M><<<grid, 256, 0, s>>>(bits, cands, I, J / 32, per_cta, cnt); break;
+    case 3: score_generic_kernel<3, M><<<grid, 256, 0, s>>>(bits, cands, I, J / 32, per_cta, cnt); break;
+    default: score_generic_kernel<4, M><<<grid, 256, 0, s>>>(bits, cands, I, J / 32, per_cta, cnt); break;
+  }
+  return BIMASK_OK;
+}
+
+int launch_score_generic(const uint32_t* bits, const int32_t* cands, int I, int J, int N, int M, int P,
+                         int64_t* counts, cudaStream_t s) {
+  if (N >= M) {                                             // every block is eligible
+    fill_counts_kernel<<<(P + 255) / 256, 256, 0, s>>>(reinterpret_cast<long long*>(counts), P, (long long)(I / M) * J);
+  } else {
+    BIMASK_CUDA_OK(cudaMemsetAsync(counts, 0, (size_t)P * sizeof(int64_t), s));
+    if (M == 8) launch_score_m<8>(bits, cands, I, J, N, P, counts, s);
+    else launch_score_m<16>(bits, cands, I, J, N, P, counts, s);
+  }
+  count_launch();
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
+int launch_bwd_mask_generic(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J, int N, int M,
+                            uint32_t* maskbits_b, uint16_t* vals_b_or_null, uint32_t* meta_b_or_null, cudaStream_t s) {
+  dim3 grid(I / 32, (J / 32 + 7) / 8);
+  uint32_t* v32 = reinterpret_cast<uint32_t*>(vals_b_or_null);
+  const bool pack = vals_b_or_null != nullptr;
+  if (M == 8) {
+    if (pack) bwd_mask_generic_kernel<8, true><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null);
+    else bwd_mask_generic_kernel<8, false><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null);
+  } else {
+    if (pack) bwd_mask_generic_kernel<16, true><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null);
+    else bwd_mask_generic_kernel<16, false><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null);
+  }
+  count_launch();
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
+}  // namespace bimask

@@ -197,7 +197,10 @@ def test_error_paths_launch_nothing():
         bm.bimask_fwd_mask(W, 64, 48, 2, 4, b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"])
     assert e.value.code == bm.binding.BIMASK_EINVAL
     with pytest.raises(bm.BimaskError) as e:
-        bm.bimask_fwd_mask(W, 64, 64, 2, 8, b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"])
+        bm.bimask_fwd_mask(W, 64, 64, 2, 32, b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"])
+    assert e.value.code == bm.binding.BIMASK_EUNSUPPORTED
+    with pytest.raises(bm.BimaskError) as e:     # 4:8 has no 2:4 container: packed outputs must be NULL
+        bm.bimask_fwd_mask(W, 64, 64, 4, 8, b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"])
     assert e.value.code == bm.binding.BIMASK_EUNSUPPORTED
     with pytest.raises(bm.BimaskError) as e:
         bm.bimask_fwd_mask(W, 64, 64, 3, 4, b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"])
@@ -282,3 +285,76 @@ def test_small_layer_with_split_k_weight_gradient():
     assert rel_err(b["dW"].cpu().numpy(), ref["dW"]) <= TOL
     assert rel_err(b["Y"].float().cpu().numpy(), ref["Y"]) <= TOL
     assert rel_err(b["dX"].float().cpu().numpy(), ref["dX"]) <= TOL
+
+
+# ---------------------------------------------------------------------------------------------
+# The other N:M patterns the paper trains (4:8, 2:8, 1:8, 1:16): masks, search, backward mask bit
+# for bit; those that fit the 2:4 container (N <= 2) also run the whole layer step.
+# ---------------------------------------------------------------------------------------------
+NM_PATTERNS = [(2, 8), (1, 8), (1, 16), (4, 8), (2, 16)]
+
+
+@pytest.mark.parametrize("N,M", NM_PATTERNS)
+@pytest.mark.parametrize("I,J", [(64, 96), (256, 384), (1024, 1056)])
+def test_other_patterns_masks_and_search(N, M, I, J):
+    W = special_weights(I, J, 7 * I + J + N + M) if I < 1000 else inputs.make_weight(I, J, N + M)
+    pack = N <= 2
+    Wd = dev(W)
+    b = bm.alloc_layer_buffers(1, I, J, 4)
+    opt = (lambda t: t) if pack else (lambda t: None)
+    bm.bimask_fwd_mask(Wd, I, J, N, M, b["maskbits_f"], opt(b["vals_f"]), opt(b["meta_f"]), opt(b["hw_meta_f"]))
+    B = O.forward_mask(W, N, M)
+    assert np.array_equal(u32(b["maskbits_f"]), O.pack_bits(B))
+    if pack:
+        _, vals, meta = O.forward_operand(W, B)
+        assert np.array_equal(u32(b["meta_f"]), meta)
+        assert np.array_equal(u16(b["vals_f"]), vals)
+    # search
+    P, seed = 4, 99 + M
+    ws_bytes = bm.bimask_workspace_bytes(1, I, J, P)
+    bm.bimask_perm_search(b["maskbits_f"], I, J, N, M, P, seed, None, b["perm"], b["best_idx"], b["counts"], b["ws"], ws_bytes)
+    torch.cuda.synchronize()
+    cands = O.candidates(seed, P, I)
+    best, perm, cnt = O.perm_search(B, cands, N, M)
+    assert np.array_equal(b["counts"].cpu().numpy(), cnt)
+    assert int(b["best_idx"].item()) == best
+    assert np.array_equal(b["perm"].cpu().numpy(), perm)
+    # backward mask on the chosen permutation
+    bm.bimask_bwd_mask(Wd, b["maskbits_f"], b["perm"], I, J, N, M, b["maskbits_b"], opt(b["vals_b"]), opt(b["meta_b"]),
+                       opt(b["hw_meta_b"]))
+    torch.cuda.synchronize()
+    Bbar = O.backward_mask(W, B, perm, N, M)
+    assert np.array_equal(u32(b["maskbits_b"]), O.pack_bits(Bbar))
+    if pack:
+        _, vals, meta = O.backward_operand(W, Bbar, perm)
+        assert np.array_equal(u32(b["meta_b"]), meta)
+        assert np.array_equal(u16(b["vals_b"]), vals)
+
+
+@pytest.mark.parametrize("N,M", [(2, 8), (1, 8), (1, 16)])
+def test_other_patterns_layer_step(N, M):
+    I, J, T = 384, 512, 300
+    W = inputs.make_weight(I, J, 100 + N + M)
+    X = inputs.make_activation(T, J, 101)
+    dY = inputs.make_activation(T, I, 102)
+    b = run_layer_step(W, X, dY, N, M, 5, 17, do_search=True)
+    ref = O.layer_step(W, X, dY, N, M, 5, 17, do_search=True)
+    assert int(b["status_word"].item()) == 0
+    assert np.array_equal(u32(b["maskbits_f"]), ref["maskbits_f"])
+    assert np.array_equal(b["counts"].cpu().numpy(), ref["counts"])
+    assert np.array_equal(b["perm"].cpu().numpy(), ref["perm"])
+    assert np.array_equal(u32(b["maskbits_b"]), ref["maskbits_b"])
+    assert np.array_equal(u16(b["vals_b"]), ref["vals_b"])
+    assert rel_err(b["Y"].float().cpu().numpy(), ref["Y"]) <= TOL
+    assert rel_err(b["dX"].float().cpu().numpy(), ref["dX"]) <= TOL
+    assert rel_err(b["dW"].cpu().numpy(), ref["dW"]) <= TOL
+
+
+def test_four_to_eight_layer_step_is_refused():
+    b = bm.alloc_layer_buffers(32, 64, 64, 2)
+    b["W"] = torch.zeros(64, 64, device="cuda")
+    b["X"] = torch.zeros(32, 64, dtype=torch.bfloat16, device="cuda")
+    b["dY"] = torch.zeros(32, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(bm.BimaskError) as e:
+        bm.bimask_layer_step(bm.make_layer_args(32, 64, 64, 4, 8, 2, 1, True, b))
+    assert e.value.code == bm.binding.BIMASK_EUNSUPPORTED
