@@ -1,7 +1,7 @@
 // N:M patterns beyond 2:4 and 1:4 (the paper also trains 4:8, 2:8, 1:8 and 1:16): forward mask,
 // eligible-block count and backward mask for block lengths M = 8 and 16.  Selection is the same
 // rank rule as for M = 4 (an element is kept when fewer than N candidates of its block beat it;
-// ties go to the lower index), evaluated with all M (M - 1) / 2 pairwise comparisons in registers.
+// ties go to the lower index), evaluated in registers (see keep_block).
 // When N <= 2 every aligned group of four holds at most two survivors, so the result is packed
 // into the same 2:4 tensor-core operand as before (the index code of a group depends on its keep
 // mask alone); patterns with N > 2 (4:8) produce mask bits only.
@@ -13,8 +13,36 @@ namespace bimask {
 namespace {
 
 // keep mask of one block of M keys: bit m set iff candidate m is beaten by fewer than N candidates
+// (q beats m when key_q > key_m, or key_q == key_m with q < m).
+//   N <= 2: N rounds of "largest remaining candidate, lowest index on ties" -- about 5 M operations
+//           per round instead of all M (M - 1) / 2 pairwise comparisons;
+//   N  > 2: pairwise ranks.
 template <int M>
 __device__ __forceinline__ uint32_t keep_block(const uint32_t (&key)[M], uint32_t valid, int N) {
+  uint32_t kb = 0;
+  if (N <= 2) {
+    uint32_t k[M];                                        // 0 = not a candidate (keys are < 2^31, so +1 fits)
+#pragma unroll
+    for (int m = 0; m < M; ++m) k[m] = ((valid >> m) & 1u) ? key[m] + 1u : 0u;
+#pragma unroll
+    for (int round = 0; round < 2; ++round) {
+      if (round < N) {
+        uint32_t mx = k[0];
+#pragma unroll
+        for (int m = 1; m < M; ++m) mx = max(mx, k[m]);
+        uint32_t eq = 0;
+#pragma unroll
+        for (int m = 0; m < M; ++m) eq |= (k[m] == mx ? 1u : 0u) << m;
+        const uint32_t pick = mx ? (eq & (0u - eq)) : 0u;  // lowest index among the largest; none if no candidate is left
+        kb |= pick;
+        if (round == 0) {
+#pragma unroll
+          for (int m = 0; m < M; ++m) k[m] = ((pick >> m) & 1u) ? 0u : k[m];
+        }
+      }
+    }
+    return kb;
+  }
   int rank[M];
 #pragma unroll
   for (int m = 0; m < M; ++m) rank[m] = 0;
@@ -26,7 +54,6 @@ __device__ __forceinline__ uint32_t keep_block(const uint32_t (&key)[M], uint32_
       rank[m] += (q_beats_m && ((valid >> q) & 1u)) ? 1 : 0;
       rank[q] += (!q_beats_m && ((valid >> m) & 1u)) ? 1 : 0;
     }
-  uint32_t kb = 0;
 #pragma unroll
   for (int m = 0; m < M; ++m) kb |= (((valid >> m) & 1u) && rank[m] < N) ? (1u << m) : 0u;
   return kb;
