@@ -84,8 +84,7 @@ int bimask_fwd_mask(const float* W, int I, int J, int N, int M,
  *   cands_or_null  in   P x I i32 explicit candidates (each a permutation of 0..I-1), or NULL:
  *                       then candidate c is generated from `seed` by sorting the rows by the
  *                       key  mix64(mix64(seed + 0x9E3779B97F4A7C15 (c+1)) ^ i)  (low 24 bits
- *                       replaced by i; mix64 = SplitMix64's output function).  Generated
- *                       candidates need I <= 16384 (BIMASK_EUNSUPPORTED beyond).
+ *                       replaced by i; mix64 = SplitMix64's output function).  Needs I < 2^24.
  *   This call alone accepts any I % M == 0 (the packed operands need I % 32 == 0); for M = 8, 16
  *   the count kernel handles N <= 4 (and the trivial N == M).
  *   best_perm out I i32, best_idx out 1 i32, counts out P i64
@@ -150,13 +149,24 @@ typedef struct {
 int bimask_layer_step(const bimask_layer_args* args);
 
 /* The same step for a caller whose data lives in HOST memory (pinned memory recommended):
- * copies W, X, dY (and perm when do_search == 0) to the device buffers named in `dev`,
- * runs bimask_layer_step there, copies Y, dX, dW, perm, best_idx, counts and the status word
- * back into the host buffers named in `host`, and synchronises `dev->stream` before it
- * returns.  Pointer fields of `host` that are NULL are skipped (not copied).  `dev` must be
- * fully populated; its sizes/flags are used, those of `host` are ignored. */
+ * copies W, X, dY (and perm when do_search == 0, cands when given) to the device buffers named
+ * in `dev`, runs bimask_layer_step there and copies Y, dX, dW, perm, best_idx, counts, the mask
+ * bits and the status word back into the host buffers named in `host`; pointer fields of `host`
+ * that are NULL are skipped.  `dev` must be fully populated; its sizes / flags are used, those of
+ * `host` are ignored.
+ *   bimask_layer_step_host        returns when the results are in host memory.
+ *   bimask_layer_step_host_async  only enqueues: uploads, the step and downloads run on three
+ *       queues (two copy streams owned by the library -- created with three events on the first
+ *       call on a device, so make that call before any stream capture -- and `dev->stream`), so
+ *       the upload of one call overlaps the download of the previous one.  The host buffers of a
+ *       call must stay valid and untouched until bimask_host_sync() (or a later blocking call)
+ *       has returned; work enqueued on dev->stream afterwards is ordered after the downloads. */
 int bimask_layer_step_host(const bimask_layer_args* dev, const bimask_layer_args* host,
                            int32_t* host_status_word);
+int bimask_layer_step_host_async(const bimask_layer_args* dev, const bimask_layer_args* host,
+                                 int32_t* host_status_word);
+/* Waits for every download enqueued so far by the host-buffer entry points on the current device. */
+int bimask_host_sync(void);
 
 /* The same search for a caller that cannot hand over a workspace.  (No counterpart in the paper:
  * this entry point exists only because of how some programs manage GPU memory.)
@@ -173,7 +183,7 @@ int bimask_layer_step_host(const bimask_layer_args* dev, const bimask_layer_args
  *   - Limit: P * I <= bimask_perm_search_static_max_entries() (2 Mi entries, e.g. P = 128 at
  *     I = 16384); beyond that the call returns BIMASK_EUNSUPPORTED and launches nothing.
  *     Candidates are always generated from `seed` (same generator as bimask_perm_search with
- *     cands_or_null == NULL, so the results are identical); I <= 16384.
+ *     cands_or_null == NULL, so the results are identical).
  *   - The first call on each device looks up the array's device address (the current device must
  *     be the one `stream` belongs to); make that first call before any stream capture begins.
  *   - All calls share the one array and it keeps whatever the last call left there.  Nothing in

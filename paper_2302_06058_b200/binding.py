@@ -17,7 +17,8 @@ BIMASK_OK, BIMASK_EINVAL, BIMASK_EUNSUPPORTED, BIMASK_ECUDA, BIMASK_ETIMEOUT = 0
 
 EXPORTS = ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "bimask_workspace_bytes", "bimask_fwd_mask",
            "bimask_perm_search", "bimask_bwd_mask", "bimask_spmm_fwd", "bimask_spmm_dgrad", "bimask_wgrad",
-           "bimask_layer_step", "bimask_layer_step_host", "bimask_check_perms", "bimask_perm_search_static",
+           "bimask_layer_step", "bimask_layer_step_host", "bimask_layer_step_host_async", "bimask_host_sync",
+           "bimask_check_perms", "bimask_perm_search_static",
            "bimask_perm_search_static_max_entries")
 
 
@@ -67,6 +68,8 @@ def lib() -> ctypes.CDLL:
         L.bimask_wgrad.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
         L.bimask_layer_step.argtypes = [POINTER(LayerArgs)]
         L.bimask_layer_step_host.argtypes = [POINTER(LayerArgs), POINTER(LayerArgs), c_void_p]
+        L.bimask_layer_step_host_async.argtypes = [POINTER(LayerArgs), POINTER(LayerArgs), c_void_p]
+        L.bimask_host_sync.argtypes = []
         L.bimask_check_perms.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_size_t, c_void_p]
         L.bimask_perm_search_static.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_uint64,
                                                 c_void_p, c_void_p, c_void_p, c_void_p]
@@ -173,6 +176,14 @@ def bimask_layer_step(args: LayerArgs):
 
 def bimask_layer_step_host(dev: LayerArgs, host: LayerArgs, host_status_word=None):
     return _check(lib().bimask_layer_step_host(ctypes.byref(dev), ctypes.byref(host), _ptr(host_status_word)))
+
+
+def bimask_layer_step_host_async(dev: LayerArgs, host: LayerArgs, host_status_word=None):
+    return _check(lib().bimask_layer_step_host_async(ctypes.byref(dev), ctypes.byref(host), _ptr(host_status_word)))
+
+
+def bimask_host_sync():
+    return _check(lib().bimask_host_sync())
 
 
 def bimask_check_perms(cands, P, I, ok, ws, ws_bytes, stream=None):

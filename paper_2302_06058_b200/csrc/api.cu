@@ -3,6 +3,7 @@
 #include "common.cuh"
 #include <string.h>
 #include <atomic>
+#include <mutex>
 
 namespace bimask {
 
@@ -117,7 +118,7 @@ int bimask_perm_search(const uint32_t* maskbits_f, int I, int J, int N, int M, i
   const int32_t* cands = cands_or_null;
   int rc;
   if (!cands) {
-    BIMASK_REQUIRE(I <= 16384, BIMASK_EUNSUPPORTED, "generated candidates need I <= 16384 (I = %d)", I);
+    BIMASK_REQUIRE(I < (1 << 24), BIMASK_EUNSUPPORTED, "generated candidates need I < 2^24 (I = %d)", I);
     const WsPlan w = plan_ws(0, I, J, P);
     BIMASK_REQUIRE(ws && aligned16(ws) && ws_bytes >= w.cands_off + w.cands_bytes, BIMASK_EINVAL,
                    "bimask_perm_search: workspace too small (%zu bytes, need %zu)", ws_bytes, w.cands_off + w.cands_bytes);
@@ -237,7 +238,7 @@ int bimask_layer_step(const bimask_layer_args* a) {
   if (a->do_search) {
     BIMASK_REQUIRE(a->P >= 1 && a->P <= 65535 && a->best_idx && a->counts, BIMASK_EINVAL,
                    "bimask_layer_step: search needs 1 <= P <= 65535, best_idx and counts");
-    BIMASK_REQUIRE(a->cands || a->I <= 16384, BIMASK_EUNSUPPORTED, "generated candidates need I <= 16384 (I = %d)", a->I);
+    BIMASK_REQUIRE(a->cands || a->I < (1 << 24), BIMASK_EUNSUPPORTED, "generated candidates need I < 2^24 (I = %d)", a->I);
   }
   // three disjoint scratch regions: generated candidates, permuted dY, split-K partials
   const WsPlan w = plan_ws(a->T, a->I, a->J, a->do_search && !a->cands ? a->P : 0);
@@ -284,36 +285,113 @@ int bimask_layer_step(const bimask_layer_args* a) {
   return launch_wgrad_impl(a->dY, a->X, a->T, a->I, a->J, a->dW, partials, a->status_word, s);
 }
 
-int bimask_layer_step_host(const bimask_layer_args* d, const bimask_layer_args* h, int32_t* host_status_word) {
+}  // extern "C"
+
+namespace bimask {
+
+// Copy streams and events of the host-buffer entry points, one set per device, created on first
+// use and kept until exit.
+struct HostPipe {
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t in_done = nullptr, compute_done = nullptr, out_done = nullptr;
+  bool ready = false, used = false;
+};
+static std::mutex g_pipe_mutex;
+static HostPipe g_pipes[64];
+
+static int get_pipe(HostPipe** out) {
+  int dev = 0;
+  BIMASK_CUDA_OK(cudaGetDevice(&dev));
+  BIMASK_REQUIRE(dev >= 0 && dev < 64, BIMASK_EUNSUPPORTED, "device ordinal %d out of range", dev);
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);
+  HostPipe& p = g_pipes[dev];
+  if (!p.ready) {
+    BIMASK_CUDA_OK(cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking));
+    BIMASK_CUDA_OK(cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking));
+    BIMASK_CUDA_OK(cudaEventCreateWithFlags(&p.in_done, cudaEventDisableTiming));
+    BIMASK_CUDA_OK(cudaEventCreateWithFlags(&p.compute_done, cudaEventDisableTiming));
+    BIMASK_CUDA_OK(cudaEventCreateWithFlags(&p.out_done, cudaEventDisableTiming));
+    p.ready = true;
+  }
+  *out = &p;
+  return BIMASK_OK;
+}
+
+}  // namespace bimask
+
+extern "C" {
+
+int bimask_layer_step_host_async(const bimask_layer_args* d, const bimask_layer_args* h, int32_t* host_status_word) {
   BIMASK_REQUIRE(d && h, BIMASK_EINVAL, "bimask_layer_step_host: null argument block");
+  BIMASK_REQUIRE(h->W && h->X && h->dY, BIMASK_EINVAL, "bimask_layer_step_host: host W, X and dY are required");
+  BIMASK_REQUIRE(d->W && d->X && d->dY && d->status_word, BIMASK_EINVAL, "bimask_layer_step_host: null device pointer");
+  HostPipe* p = nullptr;
+  int rc = get_pipe(&p);
+  if (rc != BIMASK_OK) return rc;
   cudaStream_t s = (cudaStream_t)d->stream;
   const size_t IJ = (size_t)d->I * d->J, TJ = (size_t)d->T * d->J, TI = (size_t)d->T * d->I;
-  BIMASK_REQUIRE(h->W && h->X && h->dY, BIMASK_EINVAL, "bimask_layer_step_host: host W, X and dY are required");
-  BIMASK_CUDA_OK(cudaMemcpyAsync(const_cast<float*>(d->W), h->W, IJ * 4, cudaMemcpyHostToDevice, s));
-  BIMASK_CUDA_OK(cudaMemcpyAsync(const_cast<uint16_t*>(d->X), h->X, TJ * 2, cudaMemcpyHostToDevice, s));
-  BIMASK_CUDA_OK(cudaMemcpyAsync(const_cast<uint16_t*>(d->dY), h->dY, TI * 2, cudaMemcpyHostToDevice, s));
+  // Three queues: inputs go up on `in`, the step runs on the caller's stream, results come down
+  // on `out`.  Consecutive calls therefore overlap the upload of call n with the download of
+  // call n-1 (PCIe is full duplex).  Ordering kept conservative, whatever buffers the caller
+  // re-uses: an upload starts after the previous call's kernels are done, kernels start after
+  // the previous call's download.
+  if (p->used) {
+    BIMASK_CUDA_OK(cudaStreamWaitEvent(p->in, p->compute_done, 0));
+    BIMASK_CUDA_OK(cudaStreamWaitEvent(s, p->out_done, 0));
+  } else {
+    // order behind whatever the caller's stream already holds
+    BIMASK_CUDA_OK(cudaEventRecord(p->compute_done, s));
+    BIMASK_CUDA_OK(cudaStreamWaitEvent(p->in, p->compute_done, 0));
+  }
+  BIMASK_CUDA_OK(cudaMemcpyAsync(const_cast<float*>(d->W), h->W, IJ * 4, cudaMemcpyHostToDevice, p->in));
+  BIMASK_CUDA_OK(cudaMemcpyAsync(const_cast<uint16_t*>(d->X), h->X, TJ * 2, cudaMemcpyHostToDevice, p->in));
+  BIMASK_CUDA_OK(cudaMemcpyAsync(const_cast<uint16_t*>(d->dY), h->dY, TI * 2, cudaMemcpyHostToDevice, p->in));
   if (!d->do_search && h->perm)
-    BIMASK_CUDA_OK(cudaMemcpyAsync(d->perm, h->perm, (size_t)d->I * 4, cudaMemcpyHostToDevice, s));
+    BIMASK_CUDA_OK(cudaMemcpyAsync(d->perm, h->perm, (size_t)d->I * 4, cudaMemcpyHostToDevice, p->in));
   if (d->do_search && d->cands && h->cands)
     BIMASK_CUDA_OK(cudaMemcpyAsync(const_cast<int32_t*>(d->cands), h->cands, (size_t)d->P * d->I * 4,
-                                   cudaMemcpyHostToDevice, s));
-  BIMASK_CUDA_OK(cudaMemsetAsync(d->status_word, 0, sizeof(int32_t), s));
-  int rc = bimask_layer_step(d);
-  if (rc != BIMASK_OK) return rc;
-  if (h->Y) BIMASK_CUDA_OK(cudaMemcpyAsync(h->Y, d->Y, TI * 2, cudaMemcpyDeviceToHost, s));
-  if (h->dX) BIMASK_CUDA_OK(cudaMemcpyAsync(h->dX, d->dX, TJ * 2, cudaMemcpyDeviceToHost, s));
-  if (h->dW) BIMASK_CUDA_OK(cudaMemcpyAsync(h->dW, d->dW, IJ * 4, cudaMemcpyDeviceToHost, s));
-  if (h->perm) BIMASK_CUDA_OK(cudaMemcpyAsync(h->perm, d->perm, (size_t)d->I * 4, cudaMemcpyDeviceToHost, s));
-  if (d->do_search && h->best_idx)
-    BIMASK_CUDA_OK(cudaMemcpyAsync(h->best_idx, d->best_idx, 4, cudaMemcpyDeviceToHost, s));
+                                   cudaMemcpyHostToDevice, p->in));
+  BIMASK_CUDA_OK(cudaMemsetAsync(d->status_word, 0, sizeof(int32_t), p->in));
+  BIMASK_CUDA_OK(cudaEventRecord(p->in_done, p->in));
+  BIMASK_CUDA_OK(cudaStreamWaitEvent(s, p->in_done, 0));
+  rc = bimask_layer_step(d);
+  // even when the step refused to launch, leave the queues in a consistent state
+  BIMASK_CUDA_OK(cudaEventRecord(p->compute_done, s));
+  p->used = true;
+  if (rc != BIMASK_OK) {
+    BIMASK_CUDA_OK(cudaEventRecord(p->out_done, s));
+    return rc;
+  }
+  BIMASK_CUDA_OK(cudaStreamWaitEvent(p->out, p->compute_done, 0));
+  cudaStream_t o = p->out;
+  if (h->Y) BIMASK_CUDA_OK(cudaMemcpyAsync(h->Y, d->Y, TI * 2, cudaMemcpyDeviceToHost, o));
+  if (h->dX) BIMASK_CUDA_OK(cudaMemcpyAsync(h->dX, d->dX, TJ * 2, cudaMemcpyDeviceToHost, o));
+  if (h->dW) BIMASK_CUDA_OK(cudaMemcpyAsync(h->dW, d->dW, IJ * 4, cudaMemcpyDeviceToHost, o));
+  if (h->perm) BIMASK_CUDA_OK(cudaMemcpyAsync(h->perm, d->perm, (size_t)d->I * 4, cudaMemcpyDeviceToHost, o));
+  if (d->do_search && h->best_idx) BIMASK_CUDA_OK(cudaMemcpyAsync(h->best_idx, d->best_idx, 4, cudaMemcpyDeviceToHost, o));
   if (d->do_search && h->counts)
-    BIMASK_CUDA_OK(cudaMemcpyAsync(h->counts, d->counts, (size_t)d->P * 8, cudaMemcpyDeviceToHost, s));
-  if (h->maskbits_f) BIMASK_CUDA_OK(cudaMemcpyAsync(h->maskbits_f, d->maskbits_f, IJ / 8, cudaMemcpyDeviceToHost, s));
-  if (h->maskbits_b) BIMASK_CUDA_OK(cudaMemcpyAsync(h->maskbits_b, d->maskbits_b, IJ / 8, cudaMemcpyDeviceToHost, s));
-  if (host_status_word)
-    BIMASK_CUDA_OK(cudaMemcpyAsync(host_status_word, d->status_word, 4, cudaMemcpyDeviceToHost, s));
-  BIMASK_CUDA_OK(cudaStreamSynchronize(s));
+    BIMASK_CUDA_OK(cudaMemcpyAsync(h->counts, d->counts, (size_t)d->P * 8, cudaMemcpyDeviceToHost, o));
+  if (h->maskbits_f) BIMASK_CUDA_OK(cudaMemcpyAsync(h->maskbits_f, d->maskbits_f, IJ / 8, cudaMemcpyDeviceToHost, o));
+  if (h->maskbits_b) BIMASK_CUDA_OK(cudaMemcpyAsync(h->maskbits_b, d->maskbits_b, IJ / 8, cudaMemcpyDeviceToHost, o));
+  if (host_status_word) BIMASK_CUDA_OK(cudaMemcpyAsync(host_status_word, d->status_word, 4, cudaMemcpyDeviceToHost, o));
+  BIMASK_CUDA_OK(cudaEventRecord(p->out_done, o));
+  // the caller's stream is "done" with this call only once the results are down
+  BIMASK_CUDA_OK(cudaStreamWaitEvent(s, p->out_done, 0));
   return BIMASK_OK;
+}
+
+int bimask_host_sync(void) {
+  HostPipe* p = nullptr;
+  int rc = get_pipe(&p);
+  if (rc != BIMASK_OK) return rc;
+  if (p->used) BIMASK_CUDA_OK(cudaEventSynchronize(p->out_done));
+  return BIMASK_OK;
+}
+
+int bimask_layer_step_host(const bimask_layer_args* d, const bimask_layer_args* h, int32_t* host_status_word) {
+  int rc = bimask_layer_step_host_async(d, h, host_status_word);
+  if (rc != BIMASK_OK) return rc;
+  return bimask_host_sync();
 }
 
 int bimask_check_perms(const int32_t* cands, int P, int I, int32_t* ok, void* ws, size_t ws_bytes, void* stream) {

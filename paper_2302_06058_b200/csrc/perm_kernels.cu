@@ -356,7 +356,6 @@ extern "C" int bimask_perm_search_static(const uint32_t* maskbits_f, int I, int 
                  "I = %d, J = %d: I must be a positive multiple of 4, J of 32", I, J);
   BIMASK_REQUIRE(N >= 1 && N <= M, BIMASK_EINVAL, "N = %d out of range 1..%d", N, M);
   BIMASK_REQUIRE(P >= 1 && P <= 65535, BIMASK_EINVAL, "P = %d out of range 1..65535", P);
-  BIMASK_REQUIRE(I <= 16384, BIMASK_EUNSUPPORTED, "generated candidates need I <= 16384 (I = %d)", I);
   BIMASK_REQUIRE((size_t)P * (size_t)I <= STATIC_CAND_ENTRIES, BIMASK_EUNSUPPORTED,
                  "bimask_perm_search_static: P * I = %zu candidate entries exceed the built-in scratch of %zu; "
                  "use bimask_perm_search with a caller-provided workspace",

@@ -59,7 +59,7 @@ def test_bwd_mask_bit_exact(I, J, N):
 
 
 @pytest.mark.parametrize("I,J,N,P", [(256, 256, 2, 8), (64, 576, 2, 32), (512, 4608, 1, 64), (1152, 384, 2, 32),
-                                     (100, 96, 2, 5), (16384, 64, 2, 3)])
+                                     (100, 96, 2, 5), (16384, 64, 2, 3), (40000, 32, 2, 2)])
 def test_perm_search_generated(I, J, N, P):
     W = inputs.make_weight(I, J, I + P)
     B = O.forward_mask(W, N, 4)
@@ -258,6 +258,18 @@ def test_layer_step_host_matches_device_path():
     assert int(host["best_idx"].item()) == int(ref["best_idx"].item())
     assert torch.equal(host["maskbits_f"], ref["maskbits_f"].cpu())
     assert torch.equal(host["maskbits_b"], ref["maskbits_b"].cpu())
+    # the non-blocking form: two calls in flight (the second re-uses the same buffers), then one wait
+    for name in ("Y", "dX", "dW"):
+        host[name].zero_()
+    hst.fill_(-9)
+    hargs = bm.make_layer_args(T, I, J, N, 4, P, seed, True, host)
+    bm.bimask_layer_step_host_async(dev_args, hargs, hst)
+    bm.bimask_layer_step_host_async(dev_args, hargs, hst)
+    bm.bimask_host_sync()
+    assert int(hst.item()) == 0
+    assert torch.equal(host["Y"], ref["Y"].cpu())
+    assert torch.equal(host["dX"], ref["dX"].cpu())
+    assert torch.equal(host["dW"], ref["dW"].cpu())
 
 
 def test_layer_step_is_deterministic():

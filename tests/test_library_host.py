@@ -66,7 +66,7 @@ def test_validation_happens_before_any_cuda_call(bm):
     assert L.bimask_fwd_mask(16, 64, 64, 0, 4, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_fwd_mask(20, 64, 64, 2, 4, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL   # misaligned
     assert L.bimask_perm_search(16, 64, 64, 2, 4, 0, 1, None, 16, 16, 16, 16, 1 << 20, None) == bm.binding.BIMASK_EINVAL
-    assert L.bimask_perm_search(16, 32768, 64, 2, 4, 2, 1, None, 16, 16, 16, 16, 1 << 30, None) == bm.binding.BIMASK_EUNSUPPORTED
+    assert L.bimask_perm_search(16, 1 << 24, 64, 2, 4, 2, 1, None, 16, 16, 16, 16, 1 << 30, None) == bm.binding.BIMASK_EUNSUPPORTED
     assert L.bimask_perm_search(16, 64, 64, 2, 4, 2, 1, None, 16, 16, 16, 16, 8, None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_spmm_fwd(16, 16, 16, 0, 64, 64, 16, 16, None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_wgrad(16, 16, 8, 64, 64, None, None, 0, 16, None) == bm.binding.BIMASK_EINVAL

@@ -222,13 +222,16 @@ def test_invariants(seed, nm, ib, jb):
 
 
 # ---------------------------------------------------------------- closed forms
-@pytest.mark.parametrize("N,M,elig,ratio", [(2, 4, 11 / 16, 13 / 16), (1, 4, 189 / 256, 175 / 256)])
+@pytest.mark.parametrize("N,M,elig,ratio", [(2, 4, 11 / 16, 13 / 16), (1, 4, 189 / 256, 175 / 256),
+                                            (4, 8, 163 / 256, None), (2, 8, 0.6785431, None), (1, 16, 0.7358865, None)])
 def test_closed_form_eligible_fraction(N, M, elig, ratio):
     """For i.i.d. continuous weights the forward bits of one column over distinct rows are
     i.i.d. Bernoulli(N/M): P(eligible) = P(Bin(M, N/M) <= N), E nnz(B-bar)/nnz(B) =
     E min(Bin, N) / N."""
     binom = [math.comb(M, k) * (N / M) ** k * (1 - N / M) ** (M - k) for k in range(M + 1)]
-    assert abs(sum(binom[:N + 1]) - elig) < 1e-12
+    assert abs(sum(binom[:N + 1]) - elig) < 1e-6
+    if ratio is None:
+        ratio = sum(min(k, N) * binom[k] for k in range(M + 1)) / N
     assert abs(sum(min(k, N) * binom[k] for k in range(M + 1)) / N - ratio) < 1e-12
     W = inputs.make_weight(512, 1024, 7)
     B = O.forward_mask(W, N, M)
