@@ -195,6 +195,12 @@ int bimask_perm_search_static(const uint32_t* maskbits_f, int I, int J, int N, i
                               int32_t* best_perm, int32_t* best_idx, int64_t* counts, void* stream);
 size_t bimask_perm_search_static_max_entries(void);
 
+/* Debug helper, not on the hot path: exercises the bounded wait that every tensor-core kernel
+ * uses on its mbarriers.  One thread waits about a millisecond on a barrier nothing completes; the
+ * wait gives up, *status_word (device int) becomes BIMASK_ETIMEOUT and the kernel returns
+ * normally (no trap: the context stays usable). */
+int bimask_debug_wait_probe(int32_t* status_word, void* stream);
+
 /* Debug helper, not on the hot path: sets *ok (device int) to 1 iff each of the P rows of
  * cands is a permutation of 0..I-1.  ws: at least P * I bytes of scratch. */
 int bimask_check_perms(const int32_t* cands, int P, int I, int32_t* ok, void* ws, size_t ws_bytes,

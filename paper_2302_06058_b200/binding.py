@@ -18,7 +18,7 @@ BIMASK_OK, BIMASK_EINVAL, BIMASK_EUNSUPPORTED, BIMASK_ECUDA, BIMASK_ETIMEOUT = 0
 EXPORTS = ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "bimask_workspace_bytes", "bimask_fwd_mask",
            "bimask_perm_search", "bimask_bwd_mask", "bimask_spmm_fwd", "bimask_spmm_dgrad", "bimask_wgrad",
            "bimask_layer_step", "bimask_layer_step_host", "bimask_layer_step_host_async", "bimask_host_sync",
-           "bimask_check_perms", "bimask_perm_search_static",
+           "bimask_check_perms", "bimask_debug_wait_probe", "bimask_perm_search_static",
            "bimask_perm_search_static_max_entries")
 
 
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
         L.bimask_layer_step_host_async.argtypes = [POINTER(LayerArgs), POINTER(LayerArgs), c_void_p]
         L.bimask_host_sync.argtypes = []
         L.bimask_check_perms.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.bimask_debug_wait_probe.argtypes = [c_void_p, c_void_p]
         L.bimask_perm_search_static.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_uint64,
                                                 c_void_p, c_void_p, c_void_p, c_void_p]
         L.bimask_perm_search_static_max_entries.restype = c_size_t
@@ -184,6 +185,10 @@ def bimask_layer_step_host_async(dev: LayerArgs, host: LayerArgs, host_status_wo
 
 def bimask_host_sync():
     return _check(lib().bimask_host_sync())
+
+
+def bimask_debug_wait_probe(status_word, stream=None):
+    return _check(lib().bimask_debug_wait_probe(_ptr(status_word), _stream(stream)))
 
 
 def bimask_check_perms(cands, P, I, ok, ws, ws_bytes, stream=None):

@@ -394,6 +394,11 @@ int bimask_layer_step_host(const bimask_layer_args* d, const bimask_layer_args* 
   return bimask_host_sync();
 }
 
+int bimask_debug_wait_probe(int32_t* status_word, void* stream) {
+  BIMASK_REQUIRE(status_word != nullptr, BIMASK_EINVAL, "bimask_debug_wait_probe: null pointer");
+  return launch_wait_probe(status_word, (cudaStream_t)stream);
+}
+
 int bimask_check_perms(const int32_t* cands, int P, int I, int32_t* ok, void* ws, size_t ws_bytes, void* stream) {
   BIMASK_REQUIRE(cands && ok && ws && P >= 1 && I >= 1, BIMASK_EINVAL, "bimask_check_perms: bad argument");
   BIMASK_REQUIRE(ws_bytes >= (size_t)P * I, BIMASK_EINVAL, "bimask_check_perms: workspace too small");

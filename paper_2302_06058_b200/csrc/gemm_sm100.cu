@@ -594,16 +594,28 @@ permute_cols_kernel(const uint16_t* __restrict__ dY, const int32_t* __restrict__
   const int half = I >> 1;
   for (int t0 = blockIdx.x * R; t0 < T; t0 += gridDim.x * R) {
     const uint32_t* src = reinterpret_cast<const uint32_t*>(dY) + (size_t)t0 * half;
-    for (int c = threadIdx.x; c < half; c += PERMUTE_THREADS) {
-      uint32_t r[R];
+    // four column chunks per trip: 4 R loads in flight per thread before any is consumed
+    for (int c0 = threadIdx.x; c0 < half; c0 += 4 * PERMUTE_THREADS) {
+      uint32_t r[4][R];
 #pragma unroll
-      for (int j = 0; j < R; ++j) r[j] = (t0 + j < T) ? __ldg(src + (size_t)j * half + c) : 0u;
-      if (R == 4) {
-        reinterpret_cast<uint4*>(tile_w)[c] =
-            make_uint4(__byte_perm(r[0], r[1], 0x5410), __byte_perm(r[2], r[R - 1], 0x5410),
-                       __byte_perm(r[0], r[1], 0x7632), __byte_perm(r[2], r[R - 1], 0x7632));
-      } else {
-        reinterpret_cast<uint2*>(tile_w)[c] = make_uint2(__byte_perm(r[0], r[1], 0x5410), __byte_perm(r[0], r[1], 0x7632));
+      for (int u = 0; u < 4; ++u) {
+        const int c = c0 + u * PERMUTE_THREADS;
+#pragma unroll
+        for (int j = 0; j < R; ++j) r[u][j] = (c < half && t0 + j < T) ? __ldg(src + (size_t)j * half + c) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int c = c0 + u * PERMUTE_THREADS;
+        if (c < half) {
+          if (R == 4) {
+            reinterpret_cast<uint4*>(tile_w)[c] =
+                make_uint4(__byte_perm(r[u][0], r[u][1], 0x5410), __byte_perm(r[u][2], r[u][R - 1], 0x5410),
+                           __byte_perm(r[u][0], r[u][1], 0x7632), __byte_perm(r[u][2], r[u][R - 1], 0x7632));
+          } else {
+            reinterpret_cast<uint2*>(tile_w)[c] =
+                make_uint2(__byte_perm(r[u][0], r[u][1], 0x5410), __byte_perm(r[u][0], r[u][1], 0x7632));
+          }
+        }
       }
     }
     __syncthreads();
@@ -661,6 +673,21 @@ permute_cols_small_kernel(const uint16_t* __restrict__ dY, const int32_t* __rest
       v[h] = lo | (hi << 16);
     }
     reinterpret_cast<uint4*>(dYp + t * I)[k8] = make_uint4(v[0], v[1], v[2], v[3]);
+  }
+}
+
+// Self-test of the bounded wait every GEMM role uses: one thread waits, with a budget of about
+// a millisecond, on an mbarrier that nothing will ever complete.  The wait must give up, the kernel
+// must report BIMASK_ETIMEOUT through the status word and return normally.
+__global__ void wait_probe_kernel(long long budget_cycles, int32_t* __restrict__ status_word) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    ptx::mbar_init(ptx::smem_u32(&bar), 1);
+    ptx::fence_barrier_init();
+    const bool ok = ptx::mbar_wait_bounded(ptx::smem_u32(&bar), 0, &abort_flag, budget_cycles);
+    if (!ok) atomicExch(status_word, (int32_t)BIMASK_ETIMEOUT);
   }
 }
 
@@ -871,6 +898,13 @@ int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, 
   if (Ndim > 128 && Mdim > 128) return run_sparse_pair_persistent(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   if (Ndim > 128) return run_sparse<256, 2>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   return run_sparse<128, 4>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
+}
+
+int launch_wait_probe(int32_t* status_word, cudaStream_t s) {
+  wait_probe_kernel<<<1, 32, 0, s>>>(2000000ll, status_word);
+  count_launch();
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
 }
 
 int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, uint16_t* dYp, cudaStream_t s) {

@@ -370,3 +370,15 @@ def test_four_to_eight_layer_step_is_refused():
     with pytest.raises(bm.BimaskError) as e:
         bm.bimask_layer_step(bm.make_layer_args(32, 64, 64, 4, 8, 2, 1, True, b))
     assert e.value.code == bm.binding.BIMASK_EUNSUPPORTED
+
+
+def test_bounded_wait_reports_timeout_and_context_survives():
+    """A wait on a barrier that nothing completes gives up after its budget (about a millisecond),
+    reports through the status word and leaves the context usable."""
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    bm.bimask_debug_wait_probe(st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == bm.binding.BIMASK_ETIMEOUT
+    W = inputs.make_weight(64, 64, 1)
+    _, b = run_fwd_mask(W, 2)                       # the device still works
+    assert np.array_equal(u32(b["maskbits_f"]), O.pack_bits(O.forward_mask(W, 2, 4)))
