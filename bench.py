@@ -192,7 +192,7 @@ class ClockSampler:
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM kernels on
 # config 5, from the ncu launch list summarised in profiles/cfg5_launch_list.md (GEMM kernel only).
 NCU_TRAFFIC_BYTES = {
-    (5, 0, "wgrad"): 1.246e9 + 0.247e9, (5, 1, "wgrad"): 1.015e9 + 0.247e9,
+    (5, 0, "wgrad"): 1.297e9 + 0.246e9, (5, 1, "wgrad"): 1.024e9 + 0.246e9,
     (5, 0, "spmm_fwd"): 0.605e9 + 0.244e9, (5, 1, "spmm_fwd"): 0.878e9 + 0.062e9,
     (5, 0, "spmm_dgrad"): 0.878e9 + 0.058e9, (5, 1, "spmm_dgrad"): 0.604e9 + 0.244e9,
 }
@@ -322,6 +322,22 @@ def run_gpu(args):
     if graph is not None:
         launches = launches_per_step * args.steps          # replayed from the graph, counted at capture
 
+    # ---- the same step with the search switched off (the permutation of the last search is kept):
+    #      Algorithm 1 searches once per Delta T = 100 iterations, so this is the common iteration.
+    #      Reported beside the headline, never as it.
+    nosearch = [bm.make_layer_args(L.T, L.I, L.J, cfg.N, cfg.M, cfg.P, seed, False, b) for L, b, _ in layers]
+    for a in nosearch:
+        bm.bimask_layer_step(a)
+    barrier()
+    en0, en1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    en0.record(stream)
+    for _ in range(args.steps):
+        for a in nosearch:
+            bm.bimask_layer_step(a)
+    en1.record(stream)
+    barrier()
+    nosearch_ms_total = en0.elapsed_time(en1)
+
     # ---- per-call breakdown over the same K steps (CUDA events between the C-ABI calls) ----
     names = ["fwd_mask", "spmm_fwd", "perm_search", "bwd_mask", "spmm_dgrad", "wgrad"]
     acc = {li: {n: 0.0 for n in names} for li in range(len(layers))}
@@ -408,10 +424,10 @@ def run_gpu(args):
     e2e_ms = max(ee0.elapsed_time(ee1), (time.perf_counter() - t0) * 1e3)
 
     # ---- max over ranks ----
-    t = torch.tensor([step_ms_total, e2e_ms], dtype=torch.float64, device="cuda")
+    t = torch.tensor([step_ms_total, e2e_ms, nosearch_ms_total], dtype=torch.float64, device="cuda")
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    step_ms_total, e2e_ms = float(t[0]), float(t[1])
+    step_ms_total, e2e_ms, nosearch_ms_total = float(t[0]), float(t[1]), float(t[2])
     nl = len(layers)
     value = world * nl * args.steps / (step_ms_total * 1e-3)
     e2e_value = world * nl * e2e_steps / (e2e_ms * 1e-3)
@@ -431,6 +447,11 @@ def run_gpu(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "api": "bimask_layer_step_host_async + bimask_host_sync (pinned host buffers)"},
             "gpu_launches": int(launches),
+            "search_off": {"value": world * nl * args.steps / (nosearch_ms_total * 1e-3), "unit": UNIT,
+                           "ms_per_step": nosearch_ms_total / args.steps,
+                           "note": "do_search=0: permutation kept from the last search; not the headline",
+                           "delta_t_100_value": world * nl * 100.0 /
+                           ((99.0 * nosearch_ms_total + step_ms_total) / args.steps * 1e-3)},
             "roofline": roofline,
             "kernels": kernels,
             "cpu_baseline": {"value": nl / cpu_full, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
