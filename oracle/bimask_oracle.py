@@ -28,7 +28,11 @@ Readings of points the paper leaves open (listed again in the design notes):
   * an "eligible" column block (the quantity the permutation search counts,
     Alg. 1) has at most N forward-mask bits among its M rows;
   * ties between candidate permutations go to the lowest candidate index;
-  * the weight gradient is the dense straight-through one, dW = dY^T X.
+  * the weight gradient is the dense straight-through one, dW = dY^T X;
+  * the optimizer update (`sgd_update`) is float32 in a fixed operation order,
+    because the updated weights decide the next mask; the permutation is the
+    identity before the first search; interval q = t // Delta T draws its
+    candidates from seed + q.
 
 Parity unpinned: the pseudo-random candidate generator (`candidates`).  The
 paper only says the K candidates are random; the generator below is this
@@ -376,3 +380,64 @@ def layer_step(W, X_bits, dY_bits, N, M, P, seed, do_search=True, perm=None, can
         out["dX"] = spmm_dgrad(dY_bits, W, out["M_b"])
         out["dW"] = wgrad(dY_bits, X_bits)
     return out
+
+
+# ---------------------------------------------------------------------------------------
+# Algorithm 1 as a loop: the Delta-T schedule of the search and the optimizer update
+# ---------------------------------------------------------------------------------------
+
+def sgd_update(W, dW, mom, lr, momentum, weight_decay):
+    """'Update via the SGD optimizer' (last line of the loop of Algorithm 1; Sec. 4.1 trains with SGD,
+    momentum and weight decay).  The straight-through estimator hands the gradient of B.W to the dense
+    weights unchanged (Sec. 3.1), so the update runs on all of W:
+
+        g = dW + weight_decay * W ;  mom = momentum * mom + g ;  W = W - lr * mom
+
+    The updated weights decide the next forward mask (an integer result), so the arithmetic is pinned
+    to the precision of the stored weights: float32, every product and sum rounded once, in exactly
+    the order written above (no fused multiply-add).  Returns (W_new, mom_new), float32."""
+    f = np.float32
+    W = np.asarray(W, dtype=f)
+    dW = np.asarray(dW, dtype=f)
+    mom = np.asarray(mom, dtype=f)
+    g = dW + f(weight_decay) * W
+    mom_new = f(momentum) * mom + g
+    W_new = W - f(lr) * mom_new
+    return W_new.astype(f), mom_new.astype(f)
+
+
+def interval_seed(seed, t, delta_t):
+    """Seed of the candidates drawn at iteration t: each interval draws fresh candidates
+    (Sec. 3.2: K new random permutations every Delta T iterations); interval number = t // delta_t."""
+    return (int(seed) + int(t) // int(delta_t)) & MASK64
+
+
+def train_steps(W0, X_bits, dY_bits, N, M, P, seed, delta_t, iters, lr, momentum, weight_decay,
+                with_gemms=True):
+    """Algorithm 1 for one layer: for t = 1 .. iters: forward mask (Eq. 4), forward product (Eq. 3),
+    if t % delta_t == 0 a new search, backward mask (Eq. 11), input gradient (Eq. 10), dense weight
+    gradient, SGD update.  Before the first search the permutation is the identity.  X_bits / dY_bits
+    are lists with one entry per iteration (or a single array used every iteration).
+
+    Returns (history, W_final, mom_final, sparse_final) where history[t-1] is layer_step's dict for
+    iteration t plus 'W' (the weights that iteration saw) and 'searched'; sparse_final = B . W for the
+    mask of the final weights (the algorithm's return value)."""
+    W = np.asarray(W0, dtype=np.float32).copy()
+    mom = np.zeros_like(W)
+    perm = np.arange(W.shape[0], dtype=np.int32)
+    history = []
+    for t in range(1, iters + 1):
+        Xb = X_bits[t - 1] if isinstance(X_bits, (list, tuple)) else X_bits
+        dYb = dY_bits[t - 1] if isinstance(dY_bits, (list, tuple)) else dY_bits
+        searched = (t % delta_t == 0)
+        out = layer_step(W, Xb, dYb, N, M, P, interval_seed(seed, t, delta_t), do_search=searched,
+                         perm=perm, with_gemms=with_gemms)
+        perm = out["perm"]
+        out["W"] = W.copy()
+        out["searched"] = searched
+        dW = out["dW"] if with_gemms else wgrad(dYb, Xb)
+        W, mom = sgd_update(W, np.asarray(dW, dtype=np.float64).astype(np.float32), mom, lr, momentum,
+                            weight_decay)
+        history.append(out)
+    B = forward_mask(W, N, M)
+    return history, W, mom, np.where(B, W, np.float32(0))

@@ -359,3 +359,84 @@ def test_layer_step_identity_when_not_searching():
     assert out2["counts"].shape == (8,)
     assert out2["counts"][out2["best_idx"]] == out2["counts"].max()
     assert np.array_equal(out2["perm"], O.candidates(43, 8, 256)[out2["best_idx"]])
+
+
+# ---------------------------------------------------------------- optimizer update, Delta-T schedule
+def test_sgd_update_matches_torch_optimizer():
+    """Library pin: torch.optim.SGD (momentum, weight decay, no dampening, no Nesterov) on the same
+    float32 data; it may fuse multiply-adds, hence a few-ulp tolerance rather than equality."""
+    rng = np.random.default_rng(3)
+    W0 = rng.standard_normal((16, 24)).astype(np.float32)
+    lr, mu, wd = 0.1, 0.9, 5e-4
+    p = torch.nn.Parameter(torch.from_numpy(W0.copy()))
+    opt = torch.optim.SGD([p], lr=lr, momentum=mu, weight_decay=wd)
+    W, mom = W0.copy(), np.zeros_like(W0)
+    for step in range(5):
+        g = rng.standard_normal(W0.shape).astype(np.float32)
+        p.grad = torch.from_numpy(g.copy())
+        opt.step()
+        W, mom = O.sgd_update(W, g, mom, lr, mu, wd)
+        assert W.dtype == np.float32 and mom.dtype == np.float32
+        assert np.allclose(W, p.detach().numpy(), rtol=2e-6, atol=2e-7), step
+
+
+def test_sgd_update_closed_forms():
+    """Dyadic numbers make every float32 operation exact, so the closed forms hold bit for bit:
+    plain SGD sums the gradients; a constant gradient with momentum mu moves the weight by
+    lr * g * sum_{k=1..n} (1 - mu^k) / (1 - mu); weight decay alone scales by (1 - lr*wd)^n."""
+    W0 = np.array([[1.0, -2.0, 0.5, 8.0]], dtype=np.float32)
+    g = np.array([[0.25, -0.5, 1.0, 2.0]], dtype=np.float32)
+    W, mom = W0.copy(), np.zeros_like(W0)
+    for _ in range(6):
+        W, mom = O.sgd_update(W, g, mom, 0.5, 0.0, 0.0)
+    assert np.array_equal(W, W0 - 6 * 0.5 * g)
+    W, mom = W0.copy(), np.zeros_like(W0)
+    n, mu, lr = 5, 0.5, 0.25
+    for _ in range(n):
+        W, mom = O.sgd_update(W, g, mom, lr, mu, 0.0)
+    coef = sum((1 - mu ** k) / (1 - mu) for k in range(1, n + 1))
+    assert np.array_equal(W, (W0 - lr * coef * g).astype(np.float32))
+    assert np.array_equal(mom, g * np.float32((1 - mu ** n) / (1 - mu)))
+    W, mom = W0.copy(), np.zeros_like(W0)
+    for _ in range(3):
+        W, mom = O.sgd_update(W, np.zeros_like(W0), mom, 0.5, 0.0, 0.25)
+    assert np.array_equal(W, W0 * np.float32((1 - 0.125) ** 3))
+    # the sign of each term: a positive gradient lowers the weight, decay pulls towards zero
+    W1, _ = O.sgd_update(W0, g, np.zeros_like(W0), 0.5, 0.0, 0.0)
+    assert np.all(np.sign(W1 - W0) == -np.sign(g))
+
+
+def test_train_steps_schedule_and_return_value():
+    """Algorithm 1's loop: the search runs exactly when t % Delta T == 0, with a fresh draw per
+    interval; before it the permutation is the identity; every iteration sees the weights the
+    previous update left; the return value is N:M sparse along each row."""
+    N, M, P, seed, dT, iters = 2, 4, 6, 11, 3, 7
+    rng = np.random.default_rng(5)
+    W0 = rng.standard_normal((32, 32)).astype(np.float32)
+    X = O.bf16_bits(rng.integers(-3, 4, size=(8, 32)).astype(np.float32))
+    dY = [O.bf16_bits(rng.integers(-3, 4, size=(8, 32)).astype(np.float32)) for _ in range(iters)]
+    hist, Wf, momf, sparse = O.train_steps(W0, X, dY, N, M, P, seed, dT, iters, 0.125, 0.5, 0.0)
+    assert [h["searched"] for h in hist] == [False, False, True, False, False, True, False]
+    ident = np.arange(32)
+    assert np.array_equal(hist[0]["perm"], ident) and np.array_equal(hist[1]["perm"], ident)
+    best, perm3, _ = O.perm_search(hist[2]["B"], O.candidates(seed + 1, P, 32), N, M)
+    assert np.array_equal(hist[2]["perm"], perm3) and hist[2]["best_idx"] == best
+    assert np.array_equal(hist[3]["perm"], perm3) and np.array_equal(hist[4]["perm"], perm3)
+    best6, perm6, _ = O.perm_search(hist[5]["B"], O.candidates(seed + 2, P, 32), N, M)
+    assert np.array_equal(hist[5]["perm"], perm6) and np.array_equal(hist[6]["perm"], perm6)
+    # the chain of weights, replayed by hand from the recorded gradients (integers: exact)
+    W, mom = W0.copy(), np.zeros_like(W0)
+    for t, h in enumerate(hist):
+        assert np.array_equal(h["W"], W), t
+        assert np.array_equal(h["B"], O.forward_mask(W, N, M))
+        dW = (O.bf16_to_f64(dY[t]).T @ O.bf16_to_f64(X)).astype(np.float32)
+        assert np.array_equal(dW, h["dW"])
+        mom = np.float32(0.5) * mom + dW
+        W = W - np.float32(0.125) * mom
+    assert np.array_equal(W, Wf) and np.array_equal(mom, momf)
+    assert np.all((sparse != 0).reshape(32, 8, 4).sum(axis=2) <= N)
+    assert np.array_equal(sparse != 0, O.forward_mask(Wf, N, M) & (Wf != 0))
+    # lr = 0 freezes the weights: every iteration reproduces the first one's masks
+    hist0, W_same, _, _ = O.train_steps(W0, X, dY[0], N, M, P, seed, dT, 4, 0.0, 0.9, 0.0)
+    assert np.array_equal(W_same, W0)
+    assert all(np.array_equal(h["B"], hist0[0]["B"]) for h in hist0)
