@@ -148,6 +148,50 @@ typedef struct {
 
 int bimask_layer_step(const bimask_layer_args* args);
 
+/* Algorithm 1, last line of the loop ("update via the SGD optimizer"), fused with the first line
+ * of the next iteration (forward mask, Eq. 4): one pass that reads W, dW and the momentum buffer,
+ * writes the updated W and momentum, and emits the forward mask / 2:4 operand of the UPDATED
+ * weights -- so an iteration that follows needs no bimask_fwd_mask of its own.
+ *
+ *   g = dW + weight_decay * W ;  mom = momentum * mom + g ;  W = W - lr * mom
+ *
+ * in float32, every product and sum rounded once in exactly that order (no fused multiply-add):
+ * the updated weight decides mask bits, so the operation order is part of the contract.  The
+ * straight-through estimator (Sec. 3.1) sends the gradient to all of W, masked or not.
+ *   W, dW: device float[I*J]; W is updated in place.  mom: device float[I*J], updated in place;
+ *   NULL means "no momentum buffer": it is read as zero and not stored (use with momentum == 0).
+ *   Mask outputs as for bimask_fwd_mask (vals/meta/hw_meta NULL allowed, and required NULL when
+ *   the pattern does not pack).  M == 4 runs as one kernel; M in {8, 16} as an update pass followed
+ *   by the mask kernel.  All pointers 16-byte aligned.  Errors as for bimask_fwd_mask. */
+int bimask_sgd_fwd_mask(float* W, const float* dW, float* mom_or_null, int I, int J, int N, int M,
+                        float lr, float momentum, float weight_decay,
+                        uint32_t* maskbits_f, uint16_t* vals_f, uint32_t* meta_f, void* hw_meta_f, void* stream);
+
+/* One whole iteration t of Algorithm 1 for one layer, including the Delta-T schedule of the search
+ * and the optimizer update:
+ *   1. forward mask of W (skipped when `premasked`: the previous call's step 6 already wrote it),
+ *   2. Y (Eq. 3),
+ *   3. if t % delta_t == 0: a new search, candidates drawn from seed + t / delta_t (each interval
+ *      draws fresh candidates); otherwise layer.perm is used as it stands -- the caller sets it to
+ *      the identity before the first call, and this call overwrites it whenever it searches,
+ *   4. backward mask (Eq. 11), dX (Eq. 10), dense dW,
+ *   5. (nothing: dW stays available to the caller),
+ *   6. bimask_sgd_fwd_mask: W and mom updated in place, forward mask / operand of the new W written
+ *      to layer.maskbits_f / vals_f / meta_f / hw_meta_f.
+ * `layer` is read as by bimask_layer_step, except that do_search and seed are replaced as in step
+ * 3 and that W is written.  After the last iteration vals_f / meta_f hold B.W of the final weights:
+ * the algorithm's return value.  Only the packable patterns (N <= 2), as for bimask_layer_step. */
+typedef struct bimask_train_args {
+  bimask_layer_args layer;
+  float* mom;              /* device float[I*J] or NULL (see bimask_sgd_fwd_mask) */
+  float lr, momentum, weight_decay;
+  int64_t t;               /* iteration number, counted from 1 as in Algorithm 1 */
+  int32_t delta_t;         /* >= 1 */
+  int32_t premasked;       /* non-zero: the forward mask of the current W is already in place */
+} bimask_train_args;
+
+int bimask_train_step(const bimask_train_args* args);
+
 /* The same step for a caller whose data lives in HOST memory (pinned memory recommended):
  * copies W, X, dY (and perm when do_search == 0, cands when given) to the device buffers named
  * in `dev`, runs bimask_layer_step there and copies Y, dX, dW, perm, best_idx, counts, the mask

@@ -6,7 +6,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from ctypes import c_int, c_int32, c_int64, c_size_t, c_uint64, c_void_p, c_char_p, POINTER, Structure
+from ctypes import c_float, c_int, c_int32, c_int64, c_size_t, c_uint64, c_void_p, c_char_p, POINTER, Structure
 
 import torch
 
@@ -19,7 +19,7 @@ EXPORTS = ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "
            "bimask_perm_search", "bimask_bwd_mask", "bimask_spmm_fwd", "bimask_spmm_dgrad", "bimask_wgrad",
            "bimask_layer_step", "bimask_layer_step_host", "bimask_layer_step_host_async", "bimask_host_sync",
            "bimask_check_perms", "bimask_debug_wait_probe", "bimask_perm_search_static",
-           "bimask_perm_search_static_max_entries")
+           "bimask_perm_search_static_max_entries", "bimask_sgd_fwd_mask", "bimask_train_step")
 
 
 class BimaskError(RuntimeError):
@@ -38,6 +38,12 @@ class LayerArgs(Structure):
                 ("maskbits_b", c_void_p), ("vals_b", c_void_p), ("meta_b", c_void_p), ("hw_meta_b", c_void_p),
                 ("Y", c_void_p), ("dX", c_void_p), ("dW", c_void_p),
                 ("ws", c_void_p), ("ws_bytes", c_size_t), ("status_word", c_void_p), ("stream", c_void_p)]
+
+
+class TrainArgs(Structure):
+    """Mirror of bimask_train_args."""
+    _fields_ = [("layer", LayerArgs), ("mom", c_void_p), ("lr", c_float), ("momentum", c_float),
+                ("weight_decay", c_float), ("t", c_int64), ("delta_t", c_int32), ("premasked", c_int32)]
 
 
 _lib = None
@@ -70,6 +76,9 @@ def lib() -> ctypes.CDLL:
         L.bimask_layer_step_host.argtypes = [POINTER(LayerArgs), POINTER(LayerArgs), c_void_p]
         L.bimask_layer_step_host_async.argtypes = [POINTER(LayerArgs), POINTER(LayerArgs), c_void_p]
         L.bimask_host_sync.argtypes = []
+        L.bimask_sgd_fwd_mask.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_float, c_float,
+                                          c_float, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.bimask_train_step.argtypes = [POINTER(TrainArgs)]
         L.bimask_check_perms.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_size_t, c_void_p]
         L.bimask_debug_wait_probe.argtypes = [c_void_p, c_void_p]
         L.bimask_perm_search_static.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_uint64,
@@ -77,7 +86,7 @@ def lib() -> ctypes.CDLL:
         L.bimask_perm_search_static_max_entries.restype = c_size_t
         for name in EXPORTS:
             if name not in ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "bimask_workspace_bytes",
-                            "bimask_perm_search_static_max_entries"):
+                            "bimask_perm_search_static_max_entries", "bimask_sgd_fwd_mask", "bimask_train_step"):
                 getattr(L, name).restype = c_int
         _lib = L
     return _lib
@@ -173,6 +182,26 @@ def make_layer_args(T, I, J, N, M, P, seed, do_search, bufs: dict, stream=None) 
 
 def bimask_layer_step(args: LayerArgs):
     return _check(lib().bimask_layer_step(ctypes.byref(args)))
+
+
+def bimask_sgd_fwd_mask(W, dW, mom_or_null, I, J, N, M, lr, momentum, weight_decay, maskbits_f, vals_f, meta_f, hw_meta_f,
+                        stream=None):
+    return _check(lib().bimask_sgd_fwd_mask(_ptr(W), _ptr(dW), _ptr(mom_or_null), I, J, N, M, lr, momentum, weight_decay,
+                                            _ptr(maskbits_f), _ptr(vals_f), _ptr(meta_f), _ptr(hw_meta_f),
+                                            _stream(stream)))
+
+
+def make_train_args(layer: LayerArgs, mom, lr, momentum, weight_decay, t, delta_t, premasked) -> TrainArgs:
+    a = TrainArgs()
+    ctypes.memmove(ctypes.byref(a.layer), ctypes.byref(layer), ctypes.sizeof(LayerArgs))
+    a.mom = _ptr(mom)
+    a.lr, a.momentum, a.weight_decay = lr, momentum, weight_decay
+    a.t, a.delta_t, a.premasked = t, delta_t, int(bool(premasked))
+    return a
+
+
+def bimask_train_step(args: TrainArgs):
+    return _check(lib().bimask_train_step(ctypes.byref(args)))
 
 
 def bimask_layer_step_host(dev: LayerArgs, host: LayerArgs, host_status_word=None):

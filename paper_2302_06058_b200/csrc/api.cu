@@ -101,6 +101,38 @@ int bimask_fwd_mask(const float* W, int I, int J, int N, int M, uint32_t* maskbi
   return fused ? BIMASK_OK : launch_hw_meta(meta_f, I, J, hw_meta_f, s);
 }
 
+int bimask_sgd_fwd_mask(float* W, const float* dW, float* mom, int I, int J, int N, int M, float lr, float momentum,
+                        float weight_decay, uint32_t* maskbits_f, uint16_t* vals_f, uint32_t* meta_f, void* hw_meta_f,
+                        void* stream) {
+  bool pack = false;
+  int rc = check_shape(I, J, N, M, &pack);
+  if (rc != BIMASK_OK) return rc;
+  BIMASK_REQUIRE(W && dW && maskbits_f, BIMASK_EINVAL, "bimask_sgd_fwd_mask: null pointer");
+  if (pack) {
+    BIMASK_REQUIRE(vals_f && meta_f && hw_meta_f, BIMASK_EINVAL, "bimask_sgd_fwd_mask: null pointer");
+  } else {
+    BIMASK_REQUIRE(!vals_f && !meta_f && !hw_meta_f, BIMASK_EUNSUPPORTED,
+                   "N:M = %d:%d does not fit the 2:4 container: pass vals_f = meta_f = hw_meta_f = NULL for mask bits only",
+                   N, M);
+  }
+  BIMASK_REQUIRE(aligned16(W) && aligned16(dW) && aligned16(mom) && aligned16(maskbits_f) && aligned16(vals_f) &&
+                     aligned16(meta_f) && aligned16(hw_meta_f),
+                 BIMASK_EINVAL, "bimask_sgd_fwd_mask: pointers must be 16-byte aligned");
+  BIMASK_REQUIRE(lr == lr && momentum == momentum && weight_decay == weight_decay, BIMASK_EINVAL,
+                 "bimask_sgd_fwd_mask: NaN hyper-parameter");
+  cudaStream_t s = (cudaStream_t)stream;
+  if (M != 4) {
+    if ((rc = launch_sgd_update(W, dW, mom, (long long)I * J, lr, momentum, weight_decay, s)) != BIMASK_OK) return rc;
+    if ((rc = launch_fwd_mask_generic(W, I, J, N, M, maskbits_f, vals_f, meta_f, s)) != BIMASK_OK) return rc;
+    return pack ? launch_hw_meta(meta_f, I, J, hw_meta_f, s) : BIMASK_OK;
+  }
+  const bool fused = (I % 128 == 0) && (J % 128 == 0);   // no padding in the metadata image
+  if ((rc = launch_sgd_fwd_mask(W, dW, mom, I, J, N, lr, momentum, weight_decay, maskbits_f, vals_f, meta_f,
+                                fused ? hw_meta_f : nullptr, s)) != BIMASK_OK)
+    return rc;
+  return fused ? BIMASK_OK : launch_hw_meta(meta_f, I, J, hw_meta_f, s);
+}
+
 int bimask_perm_search(const uint32_t* maskbits_f, int I, int J, int N, int M, int P, uint64_t seed,
                        const int32_t* cands_or_null, int32_t* best_perm, int32_t* best_idx, int64_t* counts,
                        void* ws, size_t ws_bytes, void* stream) {
@@ -213,7 +245,10 @@ int bimask_wgrad(const uint16_t* dY, const uint16_t* X, int T, int I, int J, flo
   return launch_wgrad_impl(dY, X, T, I, J, dW, partials, status_word, (cudaStream_t)stream);
 }
 
-int bimask_layer_step(const bimask_layer_args* a) {
+}  // extern "C"
+
+// skip_fwd_mask: the forward mask / operand of the current W is already in place
+static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask) {
   BIMASK_REQUIRE(a != nullptr, BIMASK_EINVAL, "bimask_layer_step: null argument block");
   bool pack = false;
   int rc = check_shape(a->I, a->J, a->N, a->M, &pack);
@@ -255,12 +290,14 @@ int bimask_layer_step(const bimask_layer_args* a) {
   cudaStream_t s = (cudaStream_t)a->stream;
   // M = 4 with unpadded shapes writes the metadata images inside the mask kernels
   const bool fused = a->M == 4 && (a->I % 128 == 0) && (a->J % 128 == 0);
-  if (a->M == 4)
-    rc = launch_fwd_mask(a->W, a->I, a->J, a->N, a->maskbits_f, a->vals_f, a->meta_f, fused ? a->hw_meta_f : nullptr, s);
-  else
-    rc = launch_fwd_mask_generic(a->W, a->I, a->J, a->N, a->M, a->maskbits_f, a->vals_f, a->meta_f, s);
-  if (rc) return rc;
-  if (!fused && (rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, s))) return rc;
+  if (!skip_fwd_mask) {
+    if (a->M == 4)
+      rc = launch_fwd_mask(a->W, a->I, a->J, a->N, a->maskbits_f, a->vals_f, a->meta_f, fused ? a->hw_meta_f : nullptr, s);
+    else
+      rc = launch_fwd_mask_generic(a->W, a->I, a->J, a->N, a->M, a->maskbits_f, a->vals_f, a->meta_f, s);
+    if (rc) return rc;
+    if (!fused && (rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, s))) return rc;
+  }
   if ((rc = launch_spmm(a->vals_f, a->hw_meta_f, a->X, a->I, a->T, a->J, a->Y, a->status_word, s))) return rc;
   if (a->do_search) {
     const int32_t* cands = a->cands;
@@ -283,6 +320,27 @@ int bimask_layer_step(const bimask_layer_args* a) {
   if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, s))) return rc;
   if ((rc = launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, a->dX, a->status_word, s))) return rc;
   return launch_wgrad_impl(a->dY, a->X, a->T, a->I, a->J, a->dW, partials, a->status_word, s);
+}
+
+extern "C" {
+
+int bimask_layer_step(const bimask_layer_args* a) { return layer_step_impl(a, false); }
+
+int bimask_train_step(const bimask_train_args* a) {
+  BIMASK_REQUIRE(a != nullptr, BIMASK_EINVAL, "bimask_train_step: null argument block");
+  BIMASK_REQUIRE(a->t >= 1 && a->delta_t >= 1, BIMASK_EINVAL, "bimask_train_step: t = %lld and delta_t = %d must be >= 1",
+                 (long long)a->t, a->delta_t);
+  BIMASK_REQUIRE(a->lr == a->lr && a->momentum == a->momentum && a->weight_decay == a->weight_decay, BIMASK_EINVAL,
+                 "bimask_train_step: NaN hyper-parameter");
+  BIMASK_REQUIRE(aligned16(a->mom), BIMASK_EINVAL, "bimask_train_step: mom must be 16-byte aligned");
+  bimask_layer_args l = a->layer;
+  l.do_search = (a->t % a->delta_t == 0) ? 1 : 0;
+  l.seed = a->layer.seed + (uint64_t)(a->t / a->delta_t);       // a fresh draw per interval
+  int rc = layer_step_impl(&l, a->premasked != 0);
+  if (rc != BIMASK_OK) return rc;
+  // the update reads dW after the weight-gradient kernel on the same stream, then the next mask
+  return bimask_sgd_fwd_mask(const_cast<float*>(l.W), l.dW, a->mom, l.I, l.J, l.N, l.M, a->lr, a->momentum,
+                             a->weight_decay, l.maskbits_f, l.vals_f, l.meta_f, l.hw_meta_f, l.stream);
 }
 
 }  // extern "C"

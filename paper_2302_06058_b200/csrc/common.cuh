@@ -40,6 +40,12 @@ int make_tmap_plain(CUtensorMap_st* m, int dtype, const void* ptr, uint64_t inne
 // also writes the tensor-core metadata image; otherwise call launch_hw_meta afterwards.
 int launch_fwd_mask(const float* W, int I, int J, int N, uint32_t* maskbits, uint16_t* vals,
                     uint32_t* meta, void* hw_meta_or_null, cudaStream_t s);
+// forward mask of the weights after one SGD step, which the same kernel applies in place
+int launch_sgd_fwd_mask(float* W, const float* dW, float* mom_or_null, int I, int J, int N, float lr, float momentum,
+                        float weight_decay, uint32_t* maskbits, uint16_t* vals, uint32_t* meta,
+                        void* hw_meta_or_null, cudaStream_t s);
+int launch_sgd_update(float* W, const float* dW, float* mom_or_null, long long n, float lr, float momentum,
+                      float weight_decay, cudaStream_t s);
 int launch_hw_meta(const uint32_t* meta, int rows, int K, void* hw_meta, cudaStream_t s);
 int launch_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                     int N, uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_or_null,

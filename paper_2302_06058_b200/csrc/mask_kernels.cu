@@ -35,11 +35,29 @@ __device__ __forceinline__ void scatter_hw(uint16_t* __restrict__ hw16, int tile
 // ---------------------------------------------------------------------------------------
 constexpr int FWD_THREADS = 256;
 
-template <bool N_IS_2>
+// Optimizer update of Algorithm 1 ("update via the SGD optimizer"), applied while the weights
+// stream through the mask kernel so that the next iteration's forward mask costs no second pass
+// over W.  float32, each product and sum rounded once, in this order (the updated weight decides
+// a mask bit, so the operation order is part of the contract):
+//   g = dW + weight_decay * W ;  mom = momentum * mom + g ;  W = W - lr * mom
+struct SgdParams {
+  float4* W4;            // read and written
+  const float4* dW4;
+  float4* mom4;          // nullptr: momentum buffer treated as zero and not stored
+  float lr, momentum, weight_decay;
+};
+
+__device__ __forceinline__ float sgd_one(float w, float dw, float& m, const SgdParams& p) {
+  const float g = __fadd_rn(dw, __fmul_rn(p.weight_decay, w));
+  m = __fadd_rn(__fmul_rn(p.momentum, m), g);
+  return __fsub_rn(w, __fmul_rn(p.lr, m));
+}
+
+template <bool N_IS_2, bool UPDATE>
 __global__ void __launch_bounds__(FWD_THREADS)
 fwd_mask_pack_kernel(const float4* __restrict__ W4, long long nblk, int N,
                      uint32_t* __restrict__ maskbits, uint4* __restrict__ vals4,
-                     uint32_t* __restrict__ meta, uint16_t* __restrict__ hw16, int jwords) {
+                     uint32_t* __restrict__ meta, uint16_t* __restrict__ hw16, int jwords, SgdParams sgd) {
   __shared__ uint32_t lut[64];
   __shared__ float4 stage[FWD_THREADS / 32][256];
   if (threadIdx.x < 64) lut[threadIdx.x] = lut_entry(threadIdx.x, 0xFu, N);
@@ -55,7 +73,23 @@ fwd_mask_pack_kernel(const float4* __restrict__ W4, long long nblk, int N,
 #pragma unroll
     for (int it = 0; it < 8; ++it) {
       const int b = it * 32 + lane;
-      const float4 w = b < left ? __ldg(src + b) : make_float4(0.f, 0.f, 0.f, 0.f);
+      float4 w = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (UPDATE) {
+        if (b < left) {
+          const long long at = (ch << 8) + b;
+          w = sgd.W4[at];
+          const float4 dw = __ldg(sgd.dW4 + at);
+          float4 m = sgd.mom4 ? sgd.mom4[at] : make_float4(0.f, 0.f, 0.f, 0.f);
+          w.x = sgd_one(w.x, dw.x, m.x, sgd);
+          w.y = sgd_one(w.y, dw.y, m.y, sgd);
+          w.z = sgd_one(w.z, dw.z, m.z, sgd);
+          w.w = sgd_one(w.w, dw.w, m.w, sgd);
+          sgd.W4[at] = w;
+          if (sgd.mom4) sgd.mom4[at] = m;
+        }
+      } else if (b < left) {
+        w = __ldg(src + b);
+      }
       st[b ^ ((b >> 3) & 7)] = w;
     }
     __syncwarp();
@@ -360,12 +394,63 @@ int launch_fwd_mask(const float* W, int I, int J, int N, uint32_t* maskbits, uin
   long long ctas = (nchunks + 7) / 8;
   if (ctas > 148 * 8) ctas = 148 * 8;
   if (ctas < 1) ctas = 1;
+  const SgdParams none{nullptr, nullptr, nullptr, 0.f, 0.f, 0.f};
   if (N == 2)
-    fwd_mask_pack_kernel<true><<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
-        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32);
+    fwd_mask_pack_kernel<true, false><<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
+        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, none);
   else
-    fwd_mask_pack_kernel<false><<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
-        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32);
+    fwd_mask_pack_kernel<false, false><<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
+        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, none);
+  count_launch();
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
+int launch_sgd_fwd_mask(float* W, const float* dW, float* mom, int I, int J, int N, float lr, float momentum,
+                        float weight_decay, uint32_t* maskbits, uint16_t* vals, uint32_t* meta,
+                        void* hw_meta_or_null, cudaStream_t s) {
+  const long long nblk = (long long)I * J / 4;
+  uint16_t* hw16 = reinterpret_cast<uint16_t*>(hw_meta_or_null);
+  long long ctas = ((nblk + 255) / 256 + (FWD_THREADS / 32) - 1) / (FWD_THREADS / 32);
+  if (ctas > 148 * 8) ctas = 148 * 8;
+  if (ctas < 1) ctas = 1;
+  const SgdParams p{reinterpret_cast<float4*>(W), reinterpret_cast<const float4*>(dW), reinterpret_cast<float4*>(mom),
+                    lr, momentum, weight_decay};
+  if (N == 2)
+    fwd_mask_pack_kernel<true, true><<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
+        nullptr, nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, p);
+  else
+    fwd_mask_pack_kernel<false, true><<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
+        nullptr, nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, p);
+  count_launch();
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
+// Plain update pass (same arithmetic), for the patterns whose mask kernel is the generic one.
+__global__ void sgd_update_kernel(long long n4, SgdParams p) {
+  for (long long at = (long long)blockIdx.x * blockDim.x + threadIdx.x; at < n4; at += (long long)gridDim.x * blockDim.x) {
+    float4 w = p.W4[at];
+    const float4 dw = __ldg(p.dW4 + at);
+    float4 m = p.mom4 ? p.mom4[at] : make_float4(0.f, 0.f, 0.f, 0.f);
+    w.x = sgd_one(w.x, dw.x, m.x, p);
+    w.y = sgd_one(w.y, dw.y, m.y, p);
+    w.z = sgd_one(w.z, dw.z, m.z, p);
+    w.w = sgd_one(w.w, dw.w, m.w, p);
+    p.W4[at] = w;
+    if (p.mom4) p.mom4[at] = m;
+  }
+}
+
+int launch_sgd_update(float* W, const float* dW, float* mom, long long n, float lr, float momentum, float weight_decay,
+                      cudaStream_t s) {
+  const long long n4 = n / 4;
+  long long ctas = (n4 + 255) / 256;
+  if (ctas > 148 * 8) ctas = 148 * 8;
+  if (ctas < 1) ctas = 1;
+  const SgdParams p{reinterpret_cast<float4*>(W), reinterpret_cast<const float4*>(dW), reinterpret_cast<float4*>(mom),
+                    lr, momentum, weight_decay};
+  sgd_update_kernel<<<(unsigned)ctas, 256, 0, s>>>(n4, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;

@@ -71,6 +71,11 @@ def test_validation_happens_before_any_cuda_call(bm):
     assert L.bimask_spmm_fwd(16, 16, 16, 0, 64, 64, 16, 16, None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_wgrad(16, 16, 8, 64, 64, None, None, 0, 16, None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_layer_step(None) == bm.binding.BIMASK_EINVAL
+    assert L.bimask_train_step(None) == bm.binding.BIMASK_EINVAL
+    assert L.bimask_sgd_fwd_mask(16, None, None, 64, 64, 2, 4, 0.1, 0.9, 0.0, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL
+    assert L.bimask_sgd_fwd_mask(16, 16, 20, 64, 64, 2, 4, 0.1, 0.9, 0.0, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL
+    assert L.bimask_sgd_fwd_mask(16, 16, 16, 64, 64, 2, 4, float("nan"), 0.9, 0.0, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL
+    assert L.bimask_sgd_fwd_mask(16, 16, 16, 64, 64, 4, 8, 0.1, 0.9, 0.0, 16, 16, 16, 16, None) == bm.binding.BIMASK_EUNSUPPORTED
     with pytest.raises(bm.BimaskError):
         bm.bimask_fwd_mask(None, 64, 64, 2, 4, None, None, None, None, stream=0)
 
