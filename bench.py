@@ -423,11 +423,35 @@ def run_gpu(args):
     barrier()
     e2e_ms = max(ee0.elapsed_time(ee1), (time.perf_counter() - t0) * 1e3)
 
+    # ---- whole iterations of Algorithm 1 (search every 100th call, SGD update fused with the next
+    #      forward mask); runs last because it changes W in place.  Reported beside the headline. ----
+    moms = [torch.zeros(L.I, L.J, dtype=torch.float32, device="cuda") for L, _, _ in layers]
+    tstate = {"t": 1}
+
+    def train_pass():
+        for (L, b, largs), mom in zip(layers, moms):
+            bm.bimask_train_step(bm.make_train_args(largs, mom, 1e-6, 0.9, 1e-4, tstate["t"], 100, tstate["t"] > 1))
+        tstate["t"] += 1
+
+    for _ in range(3):
+        train_pass()
+    barrier()
+    et0, et1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    et0.record(stream)
+    for _ in range(args.steps):
+        train_pass()
+    et1.record(stream)
+    barrier()
+    train_ms_total = et0.elapsed_time(et1)
+    status = [int(b["status_word"].item()) for _, b, _ in layers]
+    if any(status):
+        raise RuntimeError(f"device status words non-zero after the training iterations: {status}")
+
     # ---- max over ranks ----
-    t = torch.tensor([step_ms_total, e2e_ms, nosearch_ms_total], dtype=torch.float64, device="cuda")
+    t = torch.tensor([step_ms_total, e2e_ms, nosearch_ms_total, train_ms_total], dtype=torch.float64, device="cuda")
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    step_ms_total, e2e_ms, nosearch_ms_total = float(t[0]), float(t[1]), float(t[2])
+    step_ms_total, e2e_ms, nosearch_ms_total, train_ms_total = float(t[0]), float(t[1]), float(t[2]), float(t[3])
     nl = len(layers)
     value = world * nl * args.steps / (step_ms_total * 1e-3)
     e2e_value = world * nl * e2e_steps / (e2e_ms * 1e-3)
@@ -452,6 +476,10 @@ def run_gpu(args):
                            "note": "do_search=0: permutation kept from the last search; not the headline",
                            "delta_t_100_value": world * nl * 100.0 /
                            ((99.0 * nosearch_ms_total + step_ms_total) / args.steps * 1e-3)},
+            "train_step": {"value": world * nl * args.steps / (train_ms_total * 1e-3), "unit": UNIT,
+                           "ms_per_step": train_ms_total / args.steps,
+                           "note": "bimask_train_step: Algorithm 1 iterations t = 4.., search when t % 100 == 0, SGD "
+                                   "(momentum, weight decay) fused with the next forward mask; not the headline"},
             "roofline": roofline,
             "kernels": kernels,
             "cpu_baseline": {"value": nl / cpu_full, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
