@@ -32,7 +32,10 @@ Readings of points the paper leaves open (listed again in the design notes):
   * the optimizer update (`sgd_update`) is float32 in a fixed operation order,
     because the updated weights decide the next mask; the permutation is the
     identity before the first search; interval q = t // Delta T draws its
-    candidates from seed + q.
+    candidates from seed + q;
+  * the ablation's other backward-mask criteria (`backward_mask_criterion`):
+    "multinomial" is N draws without replacement proportional to |w| by
+    inverse CDF in float32; "random" ranks hashed per-weight keys.
 
 Parity unpinned: the pseudo-random candidate generator (`candidates`).  The
 paper only says the K candidates are random; the generator below is this
@@ -441,3 +444,87 @@ def train_steps(W0, X_bits, dY_bits, N, M, P, seed, delta_t, iters, lr, momentum
         history.append(out)
     B = forward_mask(W, N, M)
     return history, W, mom, np.where(B, W, np.float32(0))
+
+
+# ---------------------------------------------------------------------------------------
+# Other criteria for the backward mask (the ablation on binarization criteria, Sec. 4.4 / Table 8)
+# ---------------------------------------------------------------------------------------
+CRIT_WEIGHT, CRIT_SCORE, CRIT_MULTINOMIAL, CRIT_RANDOM = 0, 1, 2, 3
+_GAMMA = 0x9E3779B97F4A7C15
+
+
+def random_keys(seed: int, I: int, J: int) -> np.ndarray:
+    """31-bit pseudo-random key of every weight (i, j), a function of (seed, i*J + j) only:
+    mix64(mix64(seed) + i*J + j) >> 33."""
+    e = np.arange(I * J, dtype=np.uint64).reshape(I, J)
+    with np.errstate(over="ignore"):
+        return (_mix64_np(np.uint64(_mix64(seed)) + e) >> np.uint64(33)).astype(np.int64)
+
+
+def _uniform24(seed: int, draw: int, index: np.ndarray) -> np.ndarray:
+    """Uniform in [0, 1) with 24 bits, exactly representable in float32: a function of
+    (seed, draw number, block index)."""
+    with np.errstate(over="ignore"):
+        h = _mix64_np(np.uint64(_mix64((seed + _GAMMA * (draw + 1)) & MASK64)) ^ index.astype(np.uint64))
+    return ((h >> np.uint64(40)).astype(np.float32) * np.float32(2.0 ** -24)).astype(np.float32)
+
+
+def backward_mask_criterion(W, B, perm, N, M, criterion, S=None, seed=0):
+    """Backward mask with the N survivors of a column block chosen by another criterion than the
+    weight magnitude (the paper's ablation compares: weight magnitude -- Eq. 11, its choice --,
+    gradient magnitude, multinomial sampling by magnitude, and random).  As in Eq. 11 only entries
+    whose forward bit is set compete, blocks are M consecutive rows of the permuted matrix, and a
+    block with at most N competitors keeps them all.  Returns B-bar in permuted row order.
+
+      CRIT_WEIGHT       Eq. 11 (backward_mask).
+      CRIT_SCORE        rank by |S[perm]| instead of |W[perm]| (S = the weight gradient gives the
+                        gradient-magnitude variant); ties to the lower row of the block.
+      CRIT_RANDOM       rank by random_keys(seed): a uniformly random N-subset of the competitors.
+      CRIT_MULTINOMIAL  N draws without replacement, each proportional to |w| among the remaining
+                        competitors: with a = |w| in float32 and u = _uniform24(seed, draw, block),
+                        x = u * (a_0 + a_1 + ...) summed in row order, the draw takes the first
+                        remaining competitor whose running sum exceeds x; if none does (all zero,
+                        non-finite, or u*total rounded up to the total) the lowest remaining one.
+                        Every product and sum is float32, rounded once, so the draw is reproducible
+                        bit for bit."""
+    I, J = W.shape
+    assert I % M == 0 and 1 <= N <= M
+    p = np.asarray(perm, dtype=np.int64)
+    nb = I // M
+    valid = B[p, :].reshape(nb, M, J).transpose(0, 2, 1)                    # (blocks, J, M)
+    if criterion == CRIT_WEIGHT:
+        return backward_mask(W, B, perm, N, M)
+    if criterion in (CRIT_SCORE, CRIT_RANDOM):
+        full = magnitude_key(S) if criterion == CRIT_SCORE else random_keys(seed, I, J)
+        key = full[p, :].reshape(nb, M, J).transpose(0, 2, 1)
+        return _rank_keep(key, valid, N).transpose(0, 2, 1).reshape(I, J)
+    assert criterion == CRIT_MULTINOMIAL
+    f = np.float32
+    a = np.abs(np.asarray(W, dtype=f))[p, :].reshape(nb, M, J).transpose(0, 2, 1)
+    remaining = valid.copy()
+    keep = np.zeros_like(valid)
+    many = valid.sum(axis=2) > N                                             # blocks that must choose
+    block_index = (np.arange(nb, dtype=np.uint64)[:, None] * np.uint64(J) + np.arange(J, dtype=np.uint64)[None, :])
+    for d in range(N):
+        u = _uniform24(seed, d, block_index)
+        total = np.zeros((nb, J), dtype=f)
+        for m in range(M):
+            total = np.where(remaining[..., m], total + a[..., m], total).astype(f)
+        with np.errstate(invalid="ignore", over="ignore"):
+            x = (u * total).astype(f)
+        chosen = np.full((nb, J), -1, dtype=np.int64)
+        cum = np.zeros((nb, J), dtype=f)
+        for m in range(M):
+            cum = np.where(remaining[..., m], cum + a[..., m], cum).astype(f)
+            with np.errstate(invalid="ignore"):
+                hit = remaining[..., m] & (cum > x) & (chosen < 0)
+            chosen = np.where(hit, m, chosen)
+        lowest = np.argmax(remaining, axis=2)                                # first remaining competitor
+        chosen = np.where(chosen < 0, lowest, chosen)
+        sel = np.zeros_like(valid)
+        np.put_along_axis(sel, chosen[..., None], True, axis=2)
+        sel &= remaining                                                     # (no competitor left: nothing)
+        keep |= sel
+        remaining &= ~sel
+    keep = np.where(many[..., None], keep, valid)
+    return keep.transpose(0, 2, 1).reshape(I, J)

@@ -440,3 +440,103 @@ def test_train_steps_schedule_and_return_value():
     hist0, W_same, _, _ = O.train_steps(W0, X, dY[0], N, M, P, seed, dT, 4, 0.0, 0.9, 0.0)
     assert np.array_equal(W_same, W0)
     assert all(np.array_equal(h["B"], hist0[0]["B"]) for h in hist0)
+
+
+# ---------------------------------------------------------------- backward-mask criteria (ablation variants)
+def _all_valid_case(a_rows, nblocks, J):
+    """W whose every block of 4 permuted rows holds the magnitudes a_rows in every column; B all ones."""
+    W = np.tile(np.asarray(a_rows, dtype=np.float32)[:, None], (nblocks, J))
+    W *= np.where(np.arange(W.shape[0])[:, None] % 3 == 0, -1.0, 1.0).astype(np.float32)   # signs must not matter
+    return W, np.ones(W.shape, dtype=bool), np.arange(W.shape[0])
+
+
+def _subset_histogram(Bbar, nblocks, J):
+    code = (Bbar.reshape(nblocks, 4, J) * np.array([1, 2, 4, 8])[None, :, None]).sum(axis=1)
+    assert set(np.unique(code)) <= {3, 5, 6, 9, 10, 12}                                      # exactly two kept
+    return {c: int((code == c).sum()) for c in (3, 5, 6, 9, 10, 12)}
+
+
+def test_criterion_score_is_the_rank_rule_on_another_matrix():
+    rng = np.random.default_rng(21)
+    for (N, M) in [(2, 4), (1, 4), (2, 8), (4, 8)]:
+        W = rng.standard_normal((32, 16)).astype(np.float32)
+        S = rng.standard_normal((32, 16)).astype(np.float32)
+        S[3, :] = S[7, :]                                            # ties between rows of one block
+        B = O.forward_mask(W, N, M)
+        perm = rng.permutation(32)
+        assert np.array_equal(O.backward_mask_criterion(W, B, perm, N, M, O.CRIT_SCORE, S=W),
+                              O.backward_mask(W, B, perm, N, M))
+        got = O.backward_mask_criterion(W, B, perm, N, M, O.CRIT_SCORE, S=S)
+        Sp, Bp = np.abs(S[perm]), B[perm]
+        for k0 in range(0, 32, M):
+            for l in range(16):
+                comp = [m for m in range(M) if Bp[k0 + m, l]]
+                order = sorted(comp, key=lambda m: (-Sp[k0 + m, l], m))[:N]
+                want = np.zeros(M, dtype=bool)
+                want[order] = True
+                assert np.array_equal(got[k0:k0 + M, l], want)
+
+
+def test_criterion_random_is_uniform_over_subsets():
+    nblocks, J = 512, 64
+    W, B, perm = _all_valid_case([1.0, 2.0, 3.0, 4.0], nblocks, J)
+    got = O.backward_mask_criterion(W, B, perm, 2, 4, O.CRIT_RANDOM, seed=99)
+    hist = _subset_histogram(got, nblocks, J)
+    n = nblocks * J
+    chi2 = sum((v - n / 6) ** 2 / (n / 6) for v in hist.values())
+    assert chi2 < 5 + 6 * math.sqrt(2 * 5)
+    assert not np.array_equal(got, O.backward_mask_criterion(W, B, perm, 2, 4, O.CRIT_RANDOM, seed=100))
+    # the key belongs to the weight, not to its position: permuting rows permutes the keys with them
+    k = O.random_keys(99, 8, 4)
+    assert k.min() >= 0 and k.max() < 2 ** 31 and len(np.unique(k)) == 32
+
+
+def test_criterion_multinomial_matches_exact_subset_probabilities():
+    """Two draws without replacement, each proportional to |w|: P{i,j} = p_i p_j/(1-p_i) + p_j p_i/(1-p_j)."""
+    nblocks, J = 1024, 64
+    a = [1.0, 2.0, 3.0, 4.0]
+    W, B, perm = _all_valid_case(a, nblocks, J)
+    got = O.backward_mask_criterion(W, B, perm, 2, 4, O.CRIT_MULTINOMIAL, seed=5)
+    hist = _subset_histogram(got, nblocks, J)
+    p = np.array(a) / sum(a)
+    n = nblocks * J
+    chi2 = 0.0
+    for i, j in itertools.combinations(range(4), 2):
+        prob = p[i] * p[j] / (1 - p[i]) + p[j] * p[i] / (1 - p[j])
+        chi2 += (hist[(1 << i) | (1 << j)] - n * prob) ** 2 / (n * prob)
+    assert chi2 < 5 + 6 * math.sqrt(2 * 5)
+
+
+def test_criterion_multinomial_first_draw_is_the_inverse_cdf_and_special_cases():
+    nblocks, J = 64, 32
+    W, B, perm = _all_valid_case([1.0, 1.0, 2.0, 4.0], nblocks, J)      # running sums 1, 2, 4, 8: exact
+    got = O.backward_mask_criterion(W, B, perm, 1, 4, O.CRIT_MULTINOMIAL, seed=8)
+    idx = np.arange(nblocks, dtype=np.uint64)[:, None] * np.uint64(J) + np.arange(J, dtype=np.uint64)[None, :]
+    u = O._uniform24(8, 0, idx).astype(np.float64)
+    assert u.min() >= 0 and u.max() < 1 and abs(u.mean() - 0.5) < 0.03
+    want = np.searchsorted(np.array([1.0, 2.0, 4.0, 8.0]), 8 * u.ravel(), side="right").reshape(nblocks, J)
+    assert np.array_equal(np.argmax(got.reshape(nblocks, 4, J), axis=1), want)
+    assert np.all(got.reshape(nblocks, 4, J).sum(axis=1) == 1)
+    # a weight that dwarfs the rest is always drawn; zero weights are drawn only when nothing else is left
+    W2, B2, perm2 = _all_valid_case([1e-30, 0.0, 1e30, 0.0], 16, 32)
+    g2 = O.backward_mask_criterion(W2, B2, perm2, 2, 4, O.CRIT_MULTINOMIAL, seed=1).reshape(16, 4, 32)
+    assert g2[:, 2].all() and g2[:, 0].all() and not g2[:, 1].any() and not g2[:, 3].any()
+    W3, B3, perm3 = _all_valid_case([0.0, 0.0, 0.0, 0.0], 4, 32)
+    g3 = O.backward_mask_criterion(W3, B3, perm3, 2, 4, O.CRIT_MULTINOMIAL, seed=1).reshape(4, 4, 32)
+    assert g3[:, 0].all() and g3[:, 1].all() and not g3[:, 2:].any()
+
+
+@pytest.mark.parametrize("crit", [1, 2, 3])
+def test_criteria_keep_the_structure_of_eq11(crit):
+    """Whatever the criterion: a subset of B[perm], min(N, competitors) survivors per block, and
+    blocks with at most N competitors are untouched (no gradient gap there)."""
+    rng = np.random.default_rng(crit)
+    for (N, M) in [(2, 4), (1, 4), (2, 8), (1, 16), (4, 8)]:
+        W = rng.standard_normal((64, 32)).astype(np.float32)
+        B = O.forward_mask(W, N, M)
+        perm = rng.permutation(64)
+        got = O.backward_mask_criterion(W, B, perm, N, M, crit, S=rng.standard_normal((64, 32)).astype(np.float32), seed=3)
+        Bp = B[perm]
+        assert not (got & ~Bp).any()
+        comp = Bp.reshape(64 // M, M, 32).sum(axis=1)
+        assert np.array_equal(got.reshape(64 // M, M, 32).sum(axis=1), np.minimum(comp, N))
