@@ -105,6 +105,30 @@ int bimask_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* p
                     uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_b,
                     void* stream);
 
+/* The backward mask with another criterion for choosing the N survivors of a column block (the
+ * ablation on binarization criteria, Sec. 4.4 / Table 8, compares these with Eq. 11's weight
+ * magnitude).  As in Eq. 11, only entries whose forward bit is set compete, blocks are M
+ * consecutive rows of the permuted matrix, and a block with at most N competitors keeps them all.
+ *   BIMASK_CRIT_WEIGHT       Eq. 11; identical to bimask_bwd_mask.
+ *   BIMASK_CRIT_SCORE        rank by |S| instead of |W| (S: device float[I*J], original row order;
+ *                            S = the weight gradient of the previous iteration gives the
+ *                            gradient-magnitude variant); ties to the lower row of the block.
+ *   BIMASK_CRIT_MULTINOMIAL  N draws without replacement, each proportional to |w| among the
+ *                            remaining competitors: u = 24 random bits from (seed, draw, block),
+ *                            the draw takes the first remaining competitor whose running sum of
+ *                            |w| (row order) exceeds u * total, else the lowest remaining one;
+ *                            float32, every operation rounded once.
+ *   BIMASK_CRIT_RANDOM       rank by a hashed 31-bit key of (seed, i*J + j): a uniformly random
+ *                            N-subset of the competitors.
+ * S may be NULL unless the criterion is SCORE; seed is ignored by WEIGHT and SCORE.  Everything
+ * else (outputs, packing rules, alignment, errors) as for bimask_bwd_mask.  The variants run one
+ * generic kernel for every M; only Eq. 11 has the tuned M = 4 kernels. */
+enum { BIMASK_CRIT_WEIGHT = 0, BIMASK_CRIT_SCORE = 1, BIMASK_CRIT_MULTINOMIAL = 2, BIMASK_CRIT_RANDOM = 3 };
+int bimask_bwd_mask_criterion(const float* W, const float* S_or_null, const uint32_t* maskbits_f,
+                              const int32_t* perm, int I, int J, int N, int M, int criterion, uint64_t seed,
+                              uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_b,
+                              void* stream);
+
 /* Eq. 3: Y[t, i] = sum_j X[t, j] (B * W)[i, j].  bf16 operands, fp32 accumulation, Y T x I bf16
  * (round to nearest even).  vals_f / hw_meta_f as written by bimask_fwd_mask. */
 int bimask_spmm_fwd(const uint16_t* X, const uint16_t* vals_f, const void* hw_meta_f,

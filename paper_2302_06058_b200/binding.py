@@ -19,7 +19,8 @@ EXPORTS = ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "
            "bimask_perm_search", "bimask_bwd_mask", "bimask_spmm_fwd", "bimask_spmm_dgrad", "bimask_wgrad",
            "bimask_layer_step", "bimask_layer_step_host", "bimask_layer_step_host_async", "bimask_host_sync",
            "bimask_check_perms", "bimask_debug_wait_probe", "bimask_perm_search_static",
-           "bimask_perm_search_static_max_entries", "bimask_sgd_fwd_mask", "bimask_train_step")
+           "bimask_perm_search_static_max_entries", "bimask_sgd_fwd_mask", "bimask_train_step",
+           "bimask_bwd_mask_criterion")
 
 
 class BimaskError(RuntimeError):
@@ -76,6 +77,8 @@ def lib() -> ctypes.CDLL:
         L.bimask_layer_step_host.argtypes = [POINTER(LayerArgs), POINTER(LayerArgs), c_void_p]
         L.bimask_layer_step_host_async.argtypes = [POINTER(LayerArgs), POINTER(LayerArgs), c_void_p]
         L.bimask_host_sync.argtypes = []
+        L.bimask_bwd_mask_criterion.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_int,
+                                                c_uint64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
         L.bimask_sgd_fwd_mask.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_float, c_float,
                                           c_float, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
         L.bimask_train_step.argtypes = [POINTER(TrainArgs)]
@@ -86,7 +89,8 @@ def lib() -> ctypes.CDLL:
         L.bimask_perm_search_static_max_entries.restype = c_size_t
         for name in EXPORTS:
             if name not in ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "bimask_workspace_bytes",
-                            "bimask_perm_search_static_max_entries", "bimask_sgd_fwd_mask", "bimask_train_step"):
+                            "bimask_perm_search_static_max_entries", "bimask_sgd_fwd_mask", "bimask_train_step",
+           "bimask_bwd_mask_criterion"):
                 getattr(L, name).restype = c_int
         _lib = L
     return _lib
@@ -149,6 +153,16 @@ def bimask_perm_search(maskbits_f, I, J, N, M, P, seed, cands_or_null, best_perm
 def bimask_bwd_mask(W, maskbits_f, perm, I, J, N, M, maskbits_b, vals_b, meta_b, hw_meta_b, stream=None):
     return _check(lib().bimask_bwd_mask(_ptr(W), _ptr(maskbits_f), _ptr(perm), I, J, N, M, _ptr(maskbits_b),
                                         _ptr(vals_b), _ptr(meta_b), _ptr(hw_meta_b), _stream(stream)))
+
+
+CRIT_WEIGHT, CRIT_SCORE, CRIT_MULTINOMIAL, CRIT_RANDOM = 0, 1, 2, 3
+
+
+def bimask_bwd_mask_criterion(W, S_or_null, maskbits_f, perm, I, J, N, M, criterion, seed, maskbits_b, vals_b, meta_b,
+                              hw_meta_b, stream=None):
+    return _check(lib().bimask_bwd_mask_criterion(_ptr(W), _ptr(S_or_null), _ptr(maskbits_f), _ptr(perm), I, J, N, M,
+                                                  criterion, seed, _ptr(maskbits_b), _ptr(vals_b), _ptr(meta_b),
+                                                  _ptr(hw_meta_b), _stream(stream)))
 
 
 def bimask_spmm_fwd(X, vals_f, hw_meta_f, T, I, J, Y, status_word, stream=None):

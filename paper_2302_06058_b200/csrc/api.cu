@@ -192,6 +192,35 @@ int bimask_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* p
   return fused ? BIMASK_OK : launch_hw_meta(meta_b, J, I, hw_meta_b, s);
 }
 
+int bimask_bwd_mask_criterion(const float* W, const float* S, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
+                              int N, int M, int criterion, uint64_t seed, uint32_t* maskbits_b, uint16_t* vals_b,
+                              uint32_t* meta_b, void* hw_meta_b, void* stream) {
+  BIMASK_REQUIRE(criterion >= BIMASK_CRIT_WEIGHT && criterion <= BIMASK_CRIT_RANDOM, BIMASK_EINVAL,
+                 "bimask_bwd_mask_criterion: criterion %d out of range 0..3", criterion);
+  if (criterion == BIMASK_CRIT_WEIGHT)
+    return bimask_bwd_mask(W, maskbits_f, perm, I, J, N, M, maskbits_b, vals_b, meta_b, hw_meta_b, stream);
+  bool pack = false;
+  int rc = check_shape(I, J, N, M, &pack);
+  if (rc != BIMASK_OK) return rc;
+  BIMASK_REQUIRE(W && maskbits_f && perm && maskbits_b, BIMASK_EINVAL, "bimask_bwd_mask_criterion: null pointer");
+  BIMASK_REQUIRE(criterion != BIMASK_CRIT_SCORE || S, BIMASK_EINVAL, "bimask_bwd_mask_criterion: the score criterion needs S");
+  if (pack) {
+    BIMASK_REQUIRE(vals_b && meta_b && hw_meta_b, BIMASK_EINVAL, "bimask_bwd_mask_criterion: null pointer");
+  } else {
+    BIMASK_REQUIRE(!vals_b && !meta_b && !hw_meta_b, BIMASK_EUNSUPPORTED,
+                   "N:M = %d:%d does not fit the 2:4 container: pass vals_b = meta_b = hw_meta_b = NULL for mask bits only",
+                   N, M);
+  }
+  BIMASK_REQUIRE(aligned16(W) && aligned16(S) && aligned16(maskbits_f) && aligned16(perm) && aligned16(maskbits_b) &&
+                     aligned16(vals_b) && aligned16(meta_b) && aligned16(hw_meta_b),
+                 BIMASK_EINVAL, "bimask_bwd_mask_criterion: pointers must be 16-byte aligned");
+  cudaStream_t s = (cudaStream_t)stream;
+  if ((rc = launch_bwd_mask_criterion(W, S, maskbits_f, perm, I, J, N, M, criterion, seed, maskbits_b, vals_b, meta_b, s)) !=
+      BIMASK_OK)
+    return rc;
+  return pack ? launch_hw_meta(meta_b, J, I, hw_meta_b, s) : BIMASK_OK;
+}
+
 static int check_gemm(int T, int I, int J) {
   BIMASK_REQUIRE(T > 0 && I > 0 && J > 0 && I % 32 == 0 && J % 32 == 0, BIMASK_EINVAL,
                  "T = %d, I = %d, J = %d: T positive, I and J positive multiples of 32", T, I, J);

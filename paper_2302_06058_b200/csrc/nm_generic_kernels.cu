@@ -179,12 +179,54 @@ __global__ void fill_counts_kernel(long long* counts, int P, long long v) {
 // column): 32 / M blocks of M rows, which is exactly one metadata word and one 32-byte sector of
 // packed values per column.  Rows are gathered with one coalesced 128-byte load each.
 // ---------------------------------------------------------------------------------------
-template <int M, bool PACK>
+// Criteria of the paper's ablation on how the backward mask picks its N survivors (Sec. 4.4):
+// 0 weight magnitude (Eq. 11), 1 magnitude of another matrix S (the weight gradient), 2 N draws
+// without replacement proportional to |w|, 3 random.  Whatever the criterion only entries whose
+// forward bit is set compete, and a block with at most N competitors keeps them all.
+__device__ __forceinline__ uint64_t mix64_dev(uint64_t z) {
+  z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull;
+  z ^= z >> 27; z *= 0x94D049BB133111EBull;
+  z ^= z >> 31;
+  return z;
+}
+
+// Draw number d takes the first remaining competitor whose running sum of |w| exceeds u * total
+// (u: 24 random bits, a function of seed, d and the block index); the lowest remaining one when
+// none does.  float32, each operation rounded once, sums in row order: reproducible bit for bit.
+template <int M>
+__device__ __forceinline__ uint32_t multinomial_block(const float (&w)[M], uint32_t valid, int N, uint64_t seed,
+                                                      uint64_t block_index) {
+  if (__popc(valid) <= N) return valid;
+  uint32_t rem = valid, keep = 0;
+  for (int d = 0; d < N; ++d) {
+    const uint64_t h = mix64_dev(mix64_dev(seed + 0x9E3779B97F4A7C15ull * (uint64_t)(d + 1)) ^ block_index);
+    const float u = __fmul_rn(__uint2float_rn((uint32_t)(h >> 40)), 5.9604644775390625e-8f);   // * 2^-24, exact
+    float total = 0.f;
+#pragma unroll
+    for (int m = 0; m < M; ++m)
+      if ((rem >> m) & 1u) total = __fadd_rn(total, fabsf(w[m]));
+    const float x = __fmul_rn(u, total);
+    float cum = 0.f;
+    int chosen = -1;
+#pragma unroll
+    for (int m = 0; m < M; ++m)
+      if ((rem >> m) & 1u) {
+        cum = __fadd_rn(cum, fabsf(w[m]));
+        if (chosen < 0 && cum > x) chosen = m;
+      }
+    if (chosen < 0) chosen = __ffs(rem) - 1;
+    keep |= 1u << chosen;
+    rem &= ~(1u << chosen);
+  }
+  return keep;
+}
+
+template <int M, bool PACK, int CRIT>
 __global__ void __launch_bounds__(256)
 bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,
                         const int32_t* __restrict__ perm, int I, int J, int N,
                         uint32_t* __restrict__ maskbits_b, uint32_t* __restrict__ vals_b,
-                        uint32_t* __restrict__ meta_b) {
+                        uint32_t* __restrict__ meta_b, const float* __restrict__ S, uint64_t seed) {
   constexpr int NB = 32 / M;                                // blocks per 32-row pass
   constexpr int G = M / 4;
   __shared__ uint32_t pad16[16];
@@ -204,7 +246,8 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
 #pragma unroll
   for (int nb = 0; nb < NB; ++nb) {
     float w[M];
-    uint32_t key[M];
+    uint32_t key[M];                                        // magnitude of the weight (values, NaN handling)
+    uint32_t skey[(CRIT == 1 || CRIT == 3) ? M : 1];        // what the criterion ranks by
     uint32_t valid = 0;
 #pragma unroll
     for (int m = 0; m < M; ++m) {
@@ -213,8 +256,13 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
       const uint32_t f = __ldg(maskbits_f + (size_t)src * jwords + cw);
       valid |= ((f >> lane) & 1u) << m;
       key[m] = mag_key(w[m]);
+      if constexpr (CRIT == 1) skey[m] = mag_key(__ldg(S + (size_t)src * J + col));
+      if constexpr (CRIT == 3) skey[m] = (uint32_t)(mix64_dev(seed + (uint64_t)src * (uint64_t)J + (uint64_t)col) >> 33);
     }
-    const uint32_t kb = keep_block<M>(key, valid, N);
+    uint32_t kb;
+    if constexpr (CRIT == 0) kb = keep_block<M>(key, valid, N);
+    else if constexpr (CRIT == 2) kb = multinomial_block<M>(w, valid, N, seed, (uint64_t)(pass * NB + nb) * (uint64_t)J + (uint64_t)col);
+    else kb = keep_block<M>(skey, valid, N);
 #pragma unroll
     for (int m = 0; m < M; ++m) {
       const uint32_t word = __ballot_sync(0xFFFFFFFFu, (kb >> m) & 1u);
@@ -291,21 +339,50 @@ int launch_score_generic(const uint32_t* bits, const int32_t* cands, int I, int 
   return BIMASK_OK;
 }
 
-int launch_bwd_mask_generic(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J, int N, int M,
-                            uint32_t* maskbits_b, uint16_t* vals_b_or_null, uint32_t* meta_b_or_null, cudaStream_t s) {
+template <int M, int CRIT>
+static void launch_bwd_mc(dim3 grid, bool pack, const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
+                          int N, uint32_t* maskbits_b, uint32_t* v32, uint32_t* meta_b, const float* S, uint64_t seed,
+                          cudaStream_t s) {
+  if (pack) bwd_mask_generic_kernel<M, true, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed);
+  else bwd_mask_generic_kernel<M, false, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed);
+}
+
+template <int M>
+static void launch_bwd_m(int crit, dim3 grid, bool pack, const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I,
+                         int J, int N, uint32_t* maskbits_b, uint32_t* v32, uint32_t* meta_b, const float* S, uint64_t seed,
+                         cudaStream_t s) {
+  switch (crit) {
+    case 1: launch_bwd_mc<M, 1>(grid, pack, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
+    case 2: launch_bwd_mc<M, 2>(grid, pack, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
+    case 3: launch_bwd_mc<M, 3>(grid, pack, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
+    default: launch_bwd_mc<M, 0>(grid, pack, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
+  }
+}
+
+// criterion 0..3 as in the kernel's comment; S is read for criterion 1 only; for criterion 3 `seed`
+// is hashed once here so that the per-weight key is mix64(mix64(seed) + i*J + j) >> 33
+int launch_bwd_mask_criterion(const float* W, const float* S, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
+                              int N, int M, int crit, uint64_t seed, uint32_t* maskbits_b, uint16_t* vals_b_or_null,
+                              uint32_t* meta_b_or_null, cudaStream_t s) {
   dim3 grid(I / 32, (J / 32 + 7) / 8);
   uint32_t* v32 = reinterpret_cast<uint32_t*>(vals_b_or_null);
   const bool pack = vals_b_or_null != nullptr;
-  if (M == 8) {
-    if (pack) bwd_mask_generic_kernel<8, true><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null);
-    else bwd_mask_generic_kernel<8, false><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null);
-  } else {
-    if (pack) bwd_mask_generic_kernel<16, true><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null);
-    else bwd_mask_generic_kernel<16, false><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null);
+  if (crit == 3) {
+    uint64_t z = seed;
+    z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull; z ^= z >> 27; z *= 0x94D049BB133111EBull; z ^= z >> 31;
+    seed = z;
   }
+  if (M == 4) launch_bwd_m<4>(crit, grid, pack, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, s);
+  else if (M == 8) launch_bwd_m<8>(crit, grid, pack, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, s);
+  else launch_bwd_m<16>(crit, grid, pack, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, s);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
+}
+
+int launch_bwd_mask_generic(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J, int N, int M,
+                            uint32_t* maskbits_b, uint16_t* vals_b_or_null, uint32_t* meta_b_or_null, cudaStream_t s) {
+  return launch_bwd_mask_criterion(W, nullptr, maskbits_f, perm, I, J, N, M, 0, 0, maskbits_b, vals_b_or_null, meta_b_or_null, s);
 }
 
 }  // namespace bimask

@@ -72,6 +72,10 @@ def test_validation_happens_before_any_cuda_call(bm):
     assert L.bimask_wgrad(16, 16, 8, 64, 64, None, None, 0, 16, None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_layer_step(None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_train_step(None) == bm.binding.BIMASK_EINVAL
+    assert L.bimask_bwd_mask_criterion(16, None, 16, 16, 64, 64, 2, 4, 7, 0, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL
+    assert L.bimask_bwd_mask_criterion(16, None, 16, 16, 64, 64, 2, 4, 1, 0, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL
+    assert "needs S" in bm.bimask_last_error()
+    assert L.bimask_bwd_mask_criterion(16, None, 16, 16, 64, 64, 4, 8, 3, 0, 16, 16, 16, 16, None) == bm.binding.BIMASK_EUNSUPPORTED
     assert L.bimask_sgd_fwd_mask(16, None, None, 64, 64, 2, 4, 0.1, 0.9, 0.0, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_sgd_fwd_mask(16, 16, 20, 64, 64, 2, 4, 0.1, 0.9, 0.0, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_sgd_fwd_mask(16, 16, 16, 64, 64, 2, 4, float("nan"), 0.9, 0.0, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL
