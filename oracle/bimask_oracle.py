@@ -300,6 +300,18 @@ def unpack_2to4(vals: np.ndarray, meta: np.ndarray) -> np.ndarray:
     return out.reshape(R, 4 * G)
 
 
+def dense_operand(A: np.ndarray, keep: np.ndarray) -> np.ndarray:
+    """Masked operand for patterns the 2:4 tensor-core format cannot hold (more than two survivors
+    in some aligned group of four, e.g. 4:8): bf16 bit patterns of A where `keep`, +0 elsewhere."""
+    return np.where(keep, bf16_bits(A), np.uint16(0)).astype(np.uint16)
+
+
+def dense_backward_operand(W: np.ndarray, Bbar_p: np.ndarray, perm: np.ndarray) -> np.ndarray:
+    """(B-bar * W[perm, :])^T as a dense bf16 J x I matrix (reduction index = permuted rows)."""
+    Wp = np.ascontiguousarray(W[np.asarray(perm, dtype=np.int64), :], dtype=np.float32)
+    return dense_operand(np.ascontiguousarray(Wp.T), np.ascontiguousarray(Bbar_p.T))
+
+
 def forward_operand(W: np.ndarray, B: np.ndarray):
     """Packed forward operand A_f = B*W (I x J, 2:4 along J): (maskbits, vals, meta)."""
     vals, meta = pack_2to4_fast(W, B)

@@ -540,3 +540,26 @@ def test_criteria_keep_the_structure_of_eq11(crit):
         assert not (got & ~Bp).any()
         comp = Bp.reshape(64 // M, M, 32).sum(axis=1)
         assert np.array_equal(got.reshape(64 // M, M, 32).sum(axis=1), np.minimum(comp, N))
+
+
+def test_dense_operand_agrees_with_the_packed_one():
+    """For a packable pattern the dense masked operand is what the 2:4 operand expands to; for 4:8 it
+    carries exactly the kept weights (bf16) and zeros, and the products computed from it are Eq. 3 / Eq. 10."""
+    rng = np.random.default_rng(31)
+    W = rng.standard_normal((32, 64)).astype(np.float32)
+    B = O.forward_mask(W, 2, 8)
+    vals, meta = O.pack_2to4(W, B)
+    assert np.array_equal(O.bf16_to_f64(O.dense_operand(W, B)), O.unpack_2to4(vals, meta))
+    B48 = O.forward_mask(W, 4, 8)
+    D = O.dense_operand(W, B48)
+    assert np.array_equal(D != 0, B48 & (O.bf16_bits(W) != 0))
+    assert np.array_equal(D[B48], O.bf16_bits(W)[B48])
+    X = O.bf16_bits(rng.standard_normal((8, 64)).astype(np.float32))
+    assert np.allclose(O.bf16_to_f64(X) @ O.bf16_to_f64(D).T, O.spmm_fwd(X, W, B48), rtol=1e-12, atol=1e-12)
+    perm = rng.permutation(32)
+    Bbar = O.backward_mask(W, B48, perm, 4, 8)
+    Db = O.dense_backward_operand(W, Bbar, perm)
+    assert Db.shape == (64, 32)
+    dY = O.bf16_bits(rng.standard_normal((8, 32)).astype(np.float32))
+    want = O.spmm_dgrad(dY, W, O.unpermute_rows(Bbar, perm))
+    assert np.allclose(O.bf16_to_f64(dY)[:, perm] @ O.bf16_to_f64(Db).T, want, rtol=1e-12, atol=1e-12)
