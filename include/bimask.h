@@ -19,10 +19,16 @@
  *     calling thread's last failure.
  *   - Shapes: I % 32 == 0, J % 32 == 0.  Patterns: M in {4, 8, 16}.  With N <= 2 (2:4, 1:4, 2:8,
  *     1:8, 1:16, ...) every aligned group of four holds at most two survivors, so the result is
- *     packed into the 2:4 container (a spare slot holds +0) and all calls apply.  With N > 2 (4:8)
- *     only the mask bits exist: bimask_fwd_mask / bimask_bwd_mask then take NULL for vals, meta
- *     and hw_meta, bimask_perm_search works as usual, and the products / bimask_layer_step return
- *     BIMASK_EUNSUPPORTED.  (M = 4 with N > 2 is not implemented.)
+ *     packed into the 2:4 container (a spare slot holds +0) and the products run on the sparse
+ *     tensor cores.  With N > 2 (4:8, the one such pattern in the paper) no hardware format
+ *     exists: there is no index metadata (meta and hw_meta must be NULL in the mask calls), and
+ *     `vals`, when given, receives the DENSE masked operand instead -- I*J bf16, kept weights
+ *     rounded to bf16 and +0 elsewhere, row-major like the matrix it stands for (vals_f: I x J,
+ *     vals_b: J x I in permuted row order).  bimask_spmm_fwd / bimask_spmm_dgrad called with
+ *     hw_meta == NULL take that dense operand and run a dense tensor-core product;
+ *     bimask_layer_step / bimask_train_step do the same by themselves (their meta / hw_meta
+ *     fields are then ignored and vals_f / vals_b must hold I*J bf16).  M = 4 with N > 2 is not
+ *     implemented; the search counts eligible blocks for N <= 4 or N == M.
  *   - `perm[k]` is the source row of permuted row k (gather: Wp[k,:] = W[perm[k],:]), 0-based.
  *   - Device-side trouble (a bounded wait that ran out) is reported by writing a non-zero
  *     code into *status_word (a device int the caller reads when it chooses to sync);
@@ -51,7 +57,7 @@ extern "C" {
 typedef enum {
   BIMASK_OK = 0,
   BIMASK_EINVAL = -1,       /* null / misaligned pointer, bad shape, N or P out of range, workspace too small */
-  BIMASK_EUNSUPPORTED = -2, /* N:M that does not fit the 2:4 container, M != 4, size beyond a kernel limit */
+  BIMASK_EUNSUPPORTED = -2, /* pattern or block length not implemented, metadata asked for a pattern without a 2:4 form, size beyond a kernel limit */
   BIMASK_ECUDA = -3,        /* a CUDA call failed; see bimask_last_error() */
   BIMASK_ETIMEOUT = -4      /* value written to *status_word when a device-side bounded wait ran out */
 } bimask_status;
@@ -184,8 +190,7 @@ int bimask_layer_step(const bimask_layer_args* args);
  * straight-through estimator (Sec. 3.1) sends the gradient to all of W, masked or not.
  *   W, dW: device float[I*J]; W is updated in place.  mom: device float[I*J], updated in place;
  *   NULL means "no momentum buffer": it is read as zero and not stored (use with momentum == 0).
- *   Mask outputs as for bimask_fwd_mask (vals/meta/hw_meta NULL allowed, and required NULL when
- *   the pattern does not pack).  M == 4 runs as one kernel; M in {8, 16} as an update pass followed
+ *   Mask outputs as for bimask_fwd_mask (the same rules for patterns that do not pack).  M == 4 runs as one kernel; M in {8, 16} as an update pass followed
  *   by the mask kernel.  All pointers 16-byte aligned.  Errors as for bimask_fwd_mask. */
 int bimask_sgd_fwd_mask(float* W, const float* dW, float* mom_or_null, int I, int J, int N, int M,
                         float lr, float momentum, float weight_decay,
@@ -204,7 +209,7 @@ int bimask_sgd_fwd_mask(float* W, const float* dW, float* mom_or_null, int I, in
  *      to layer.maskbits_f / vals_f / meta_f / hw_meta_f.
  * `layer` is read as by bimask_layer_step, except that do_search and seed are replaced as in step
  * 3 and that W is written.  After the last iteration vals_f / meta_f hold B.W of the final weights:
- * the algorithm's return value.  Only the packable patterns (N <= 2), as for bimask_layer_step. */
+ * the algorithm's return value (for a pattern that does not pack: vals_f alone, dense). */
 typedef struct bimask_train_args {
   bimask_layer_args layer;
   float* mom;              /* device float[I*J] or NULL (see bimask_sgd_fwd_mask) */

@@ -249,19 +249,21 @@ def bimask_perm_search_static_max_entries() -> int:
     return int(lib().bimask_perm_search_static_max_entries())
 
 
-def alloc_layer_buffers(T, I, J, P, device="cuda") -> dict:
-    """Device buffers for every output of a layer step plus scratch (torch is the allocator)."""
+def alloc_layer_buffers(T, I, J, P, device="cuda", dense=False) -> dict:
+    """Device buffers for every output of a layer step plus scratch (torch is the allocator).
+    dense: size vals_f / vals_b for the dense masked operands of a pattern that does not fit the
+    2:4 container (I*J bf16 each instead of half that)."""
     d = torch.device(device)
     b = {
         "perm": torch.arange(I, dtype=torch.int32, device=d),
         "best_idx": torch.zeros(1, dtype=torch.int32, device=d),
         "counts": torch.zeros(max(P, 1), dtype=torch.int64, device=d),
         "maskbits_f": torch.empty(I, J // 32, dtype=torch.int32, device=d),
-        "vals_f": torch.empty(I, J // 2, dtype=torch.bfloat16, device=d),
+        "vals_f": torch.empty(I, J if dense else J // 2, dtype=torch.bfloat16, device=d),
         "meta_f": torch.empty(I, J // 32, dtype=torch.int32, device=d),
         "hw_meta_f": torch.empty(bimask_hw_meta_bytes(I, J), dtype=torch.uint8, device=d),
         "maskbits_b": torch.empty(I, J // 32, dtype=torch.int32, device=d),
-        "vals_b": torch.empty(J, I // 2, dtype=torch.bfloat16, device=d),
+        "vals_b": torch.empty(J, I if dense else I // 2, dtype=torch.bfloat16, device=d),
         "meta_b": torch.empty(J, I // 32, dtype=torch.int32, device=d),
         "hw_meta_b": torch.empty(bimask_hw_meta_bytes(J, I), dtype=torch.uint8, device=d),
         "Y": torch.empty(T, I, dtype=torch.bfloat16, device=d),

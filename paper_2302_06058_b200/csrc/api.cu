@@ -85,15 +85,17 @@ int bimask_fwd_mask(const float* W, int I, int J, int N, int M, uint32_t* maskbi
   if (pack) {
     BIMASK_REQUIRE(vals_f && meta_f && hw_meta_f, BIMASK_EINVAL, "bimask_fwd_mask: null pointer");
   } else {
-    BIMASK_REQUIRE(!vals_f && !meta_f && !hw_meta_f, BIMASK_EUNSUPPORTED,
-                   "N:M = %d:%d does not fit the 2:4 container: pass vals_f = meta_f = hw_meta_f = NULL for mask bits only",
+    BIMASK_REQUIRE(!meta_f && !hw_meta_f, BIMASK_EUNSUPPORTED,
+                   "N:M = %d:%d does not fit the 2:4 container: pass meta_f = hw_meta_f = NULL (vals_f, when given, receives the "
+                   "dense masked operand)",
                    N, M);
   }
   BIMASK_REQUIRE(aligned16(W) && aligned16(maskbits_f) && aligned16(vals_f) && aligned16(meta_f) && aligned16(hw_meta_f),
                  BIMASK_EINVAL, "bimask_fwd_mask: pointers must be 16-byte aligned");
   cudaStream_t s = (cudaStream_t)stream;
   if (M != 4) {
-    if ((rc = launch_fwd_mask_generic(W, I, J, N, M, maskbits_f, vals_f, meta_f, s)) != BIMASK_OK) return rc;
+    if ((rc = launch_fwd_mask_generic(W, I, J, N, M, maskbits_f, vals_f, meta_f, pack ? 1 : vals_f ? 2 : 0, s)) != BIMASK_OK)
+      return rc;
     return pack ? launch_hw_meta(meta_f, I, J, hw_meta_f, s) : BIMASK_OK;
   }
   const bool fused = (I % 128 == 0) && (J % 128 == 0);   // no padding in the metadata image
@@ -111,8 +113,9 @@ int bimask_sgd_fwd_mask(float* W, const float* dW, float* mom, int I, int J, int
   if (pack) {
     BIMASK_REQUIRE(vals_f && meta_f && hw_meta_f, BIMASK_EINVAL, "bimask_sgd_fwd_mask: null pointer");
   } else {
-    BIMASK_REQUIRE(!vals_f && !meta_f && !hw_meta_f, BIMASK_EUNSUPPORTED,
-                   "N:M = %d:%d does not fit the 2:4 container: pass vals_f = meta_f = hw_meta_f = NULL for mask bits only",
+    BIMASK_REQUIRE(!meta_f && !hw_meta_f, BIMASK_EUNSUPPORTED,
+                   "N:M = %d:%d does not fit the 2:4 container: pass meta_f = hw_meta_f = NULL (vals_f, when given, receives the "
+                   "dense masked operand)",
                    N, M);
   }
   BIMASK_REQUIRE(aligned16(W) && aligned16(dW) && aligned16(mom) && aligned16(maskbits_f) && aligned16(vals_f) &&
@@ -123,7 +126,8 @@ int bimask_sgd_fwd_mask(float* W, const float* dW, float* mom, int I, int J, int
   cudaStream_t s = (cudaStream_t)stream;
   if (M != 4) {
     if ((rc = launch_sgd_update(W, dW, mom, (long long)I * J, lr, momentum, weight_decay, s)) != BIMASK_OK) return rc;
-    if ((rc = launch_fwd_mask_generic(W, I, J, N, M, maskbits_f, vals_f, meta_f, s)) != BIMASK_OK) return rc;
+    if ((rc = launch_fwd_mask_generic(W, I, J, N, M, maskbits_f, vals_f, meta_f, pack ? 1 : vals_f ? 2 : 0, s)) != BIMASK_OK)
+      return rc;
     return pack ? launch_hw_meta(meta_f, I, J, hw_meta_f, s) : BIMASK_OK;
   }
   const bool fused = (I % 128 == 0) && (J % 128 == 0);   // no padding in the metadata image
@@ -173,8 +177,9 @@ int bimask_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* p
   if (pack) {
     BIMASK_REQUIRE(vals_b && meta_b && hw_meta_b, BIMASK_EINVAL, "bimask_bwd_mask: null pointer");
   } else {
-    BIMASK_REQUIRE(!vals_b && !meta_b && !hw_meta_b, BIMASK_EUNSUPPORTED,
-                   "N:M = %d:%d does not fit the 2:4 container: pass vals_b = meta_b = hw_meta_b = NULL for mask bits only",
+    BIMASK_REQUIRE(!meta_b && !hw_meta_b, BIMASK_EUNSUPPORTED,
+                   "N:M = %d:%d does not fit the 2:4 container: pass meta_b = hw_meta_b = NULL (vals_b, when given, receives the "
+                   "dense masked operand)",
                    N, M);
   }
   BIMASK_REQUIRE(aligned16(W) && aligned16(maskbits_f) && aligned16(perm) && aligned16(maskbits_b) &&
@@ -182,7 +187,9 @@ int bimask_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* p
                  BIMASK_EINVAL, "bimask_bwd_mask: pointers must be 16-byte aligned");
   cudaStream_t s = (cudaStream_t)stream;
   if (M != 4) {
-    if ((rc = launch_bwd_mask_generic(W, maskbits_f, perm, I, J, N, M, maskbits_b, vals_b, meta_b, s)) != BIMASK_OK) return rc;
+    if ((rc = launch_bwd_mask_generic(W, maskbits_f, perm, I, J, N, M, maskbits_b, vals_b, meta_b, pack ? 1 : vals_b ? 2 : 0, s)) !=
+        BIMASK_OK)
+      return rc;
     return pack ? launch_hw_meta(meta_b, J, I, hw_meta_b, s) : BIMASK_OK;
   }
   const bool fused = (I % 128 == 0) && (J % 128 == 0);
@@ -207,15 +214,17 @@ int bimask_bwd_mask_criterion(const float* W, const float* S, const uint32_t* ma
   if (pack) {
     BIMASK_REQUIRE(vals_b && meta_b && hw_meta_b, BIMASK_EINVAL, "bimask_bwd_mask_criterion: null pointer");
   } else {
-    BIMASK_REQUIRE(!vals_b && !meta_b && !hw_meta_b, BIMASK_EUNSUPPORTED,
-                   "N:M = %d:%d does not fit the 2:4 container: pass vals_b = meta_b = hw_meta_b = NULL for mask bits only",
+    BIMASK_REQUIRE(!meta_b && !hw_meta_b, BIMASK_EUNSUPPORTED,
+                   "N:M = %d:%d does not fit the 2:4 container: pass meta_b = hw_meta_b = NULL (vals_b, when given, receives the "
+                   "dense masked operand)",
                    N, M);
   }
   BIMASK_REQUIRE(aligned16(W) && aligned16(S) && aligned16(maskbits_f) && aligned16(perm) && aligned16(maskbits_b) &&
                      aligned16(vals_b) && aligned16(meta_b) && aligned16(hw_meta_b),
                  BIMASK_EINVAL, "bimask_bwd_mask_criterion: pointers must be 16-byte aligned");
   cudaStream_t s = (cudaStream_t)stream;
-  if ((rc = launch_bwd_mask_criterion(W, S, maskbits_f, perm, I, J, N, M, criterion, seed, maskbits_b, vals_b, meta_b, s)) !=
+  if ((rc = launch_bwd_mask_criterion(W, S, maskbits_f, perm, I, J, N, M, criterion, seed, maskbits_b, vals_b, meta_b,
+                                      pack ? 1 : vals_b ? 2 : 0, s)) !=
       BIMASK_OK)
     return rc;
   return pack ? launch_hw_meta(meta_b, J, I, hw_meta_b, s) : BIMASK_OK;
@@ -231,9 +240,10 @@ int bimask_spmm_fwd(const uint16_t* X, const uint16_t* vals_f, const void* hw_me
                     uint16_t* Y, int32_t* status_word, void* stream) {
   int rc = check_gemm(T, I, J);
   if (rc != BIMASK_OK) return rc;
-  BIMASK_REQUIRE(X && vals_f && hw_meta_f && Y && status_word, BIMASK_EINVAL, "bimask_spmm_fwd: null pointer");
+  BIMASK_REQUIRE(X && vals_f && Y && status_word, BIMASK_EINVAL, "bimask_spmm_fwd: null pointer");
   BIMASK_REQUIRE(aligned16(X) && aligned16(vals_f) && aligned16(hw_meta_f) && aligned16(Y), BIMASK_EINVAL,
                  "bimask_spmm_fwd: pointers must be 16-byte aligned");
+  if (!hw_meta_f) return launch_dense_nt(vals_f, X, I, T, J, Y, status_word, (cudaStream_t)stream);
   return launch_spmm(vals_f, hw_meta_f, X, I, T, J, Y, status_word, (cudaStream_t)stream);
 }
 
@@ -242,8 +252,7 @@ int bimask_spmm_dgrad(const uint16_t* dY, const int32_t* perm, const uint16_t* v
                       void* stream) {
   int rc = check_gemm(T, I, J);
   if (rc != BIMASK_OK) return rc;
-  BIMASK_REQUIRE(dY && perm && vals_b && hw_meta_b && dX && status_word && ws, BIMASK_EINVAL,
-                 "bimask_spmm_dgrad: null pointer");
+  BIMASK_REQUIRE(dY && perm && vals_b && dX && status_word && ws, BIMASK_EINVAL, "bimask_spmm_dgrad: null pointer");
   BIMASK_REQUIRE(aligned16(dY) && aligned16(perm) && aligned16(vals_b) && aligned16(hw_meta_b) && aligned16(dX) &&
                      aligned16(ws),
                  BIMASK_EINVAL, "bimask_spmm_dgrad: pointers must be 16-byte aligned");
@@ -254,6 +263,7 @@ int bimask_spmm_dgrad(const uint16_t* dY, const int32_t* perm, const uint16_t* v
   uint16_t* dYp = reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(ws) + w.dyp_off);
   cudaStream_t s = (cudaStream_t)stream;
   if ((rc = launch_permute_cols(dY, perm, T, I, dYp, s)) != BIMASK_OK) return rc;
+  if (!hw_meta_b) return launch_dense_nt(vals_b, dYp, J, T, I, dX, status_word, s);
   return launch_spmm(vals_b, hw_meta_b, dYp, J, T, I, dX, status_word, s);
 }
 
@@ -282,16 +292,17 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask) {
   bool pack = false;
   int rc = check_shape(a->I, a->J, a->N, a->M, &pack);
   if (rc != BIMASK_OK) return rc;
-  BIMASK_REQUIRE(pack, BIMASK_EUNSUPPORTED,
-                 "N:M = %d:%d does not fit the 2:4 container, so the sparse products cannot run; the mask and search "
-                 "calls accept it",
-                 a->N, a->M);
+  BIMASK_REQUIRE(pack || a->N <= 4 || a->N == a->M || !a->do_search, BIMASK_EUNSUPPORTED,
+                 "N:M = %d:%d: the count kernel of the search handles N <= 4", a->N, a->M);
   if ((rc = check_gemm(a->T, a->I, a->J)) != BIMASK_OK) return rc;
   BIMASK_REQUIRE(a->perm && a->ws && a->status_word && aligned16(a->ws), BIMASK_EINVAL,
                  "bimask_layer_step: null or misaligned pointer");
-  BIMASK_REQUIRE(a->W && a->X && a->dY && a->Y && a->dX && a->dW && a->maskbits_f && a->vals_f && a->meta_f &&
-                     a->hw_meta_f && a->maskbits_b && a->vals_b && a->meta_b && a->hw_meta_b,
+  BIMASK_REQUIRE(a->W && a->X && a->dY && a->Y && a->dX && a->dW && a->maskbits_f && a->vals_f && a->maskbits_b && a->vals_b,
                  BIMASK_EINVAL, "bimask_layer_step: null pointer");
+  // patterns that fit the 2:4 container need the index metadata buffers; the others run the
+  // products on dense masked operands (vals_f / vals_b then hold I*J bf16) and ignore them
+  BIMASK_REQUIRE(!pack || (a->meta_f && a->hw_meta_f && a->meta_b && a->hw_meta_b), BIMASK_EINVAL,
+                 "bimask_layer_step: null metadata pointer");
   BIMASK_REQUIRE(aligned16(a->W) && aligned16(a->X) && aligned16(a->dY) && aligned16(a->Y) && aligned16(a->dX) &&
                      aligned16(a->dW) && aligned16(a->perm) && aligned16(a->maskbits_f) && aligned16(a->vals_f) &&
                      aligned16(a->meta_f) && aligned16(a->hw_meta_f) && aligned16(a->maskbits_b) &&
@@ -323,11 +334,13 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask) {
     if (a->M == 4)
       rc = launch_fwd_mask(a->W, a->I, a->J, a->N, a->maskbits_f, a->vals_f, a->meta_f, fused ? a->hw_meta_f : nullptr, s);
     else
-      rc = launch_fwd_mask_generic(a->W, a->I, a->J, a->N, a->M, a->maskbits_f, a->vals_f, a->meta_f, s);
+      rc = launch_fwd_mask_generic(a->W, a->I, a->J, a->N, a->M, a->maskbits_f, a->vals_f, a->meta_f, pack ? 1 : 2, s);
     if (rc) return rc;
-    if (!fused && (rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, s))) return rc;
+    if (pack && !fused && (rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, s))) return rc;
   }
-  if ((rc = launch_spmm(a->vals_f, a->hw_meta_f, a->X, a->I, a->T, a->J, a->Y, a->status_word, s))) return rc;
+  if (pack) rc = launch_spmm(a->vals_f, a->hw_meta_f, a->X, a->I, a->T, a->J, a->Y, a->status_word, s);
+  else rc = launch_dense_nt(a->vals_f, a->X, a->I, a->T, a->J, a->Y, a->status_word, s);
+  if (rc) return rc;
   if (a->do_search) {
     const int32_t* cands = a->cands;
     if (!cands) {
@@ -343,11 +356,14 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask) {
     rc = launch_bwd_mask(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->maskbits_b, a->vals_b, a->meta_b,
                          fused ? a->hw_meta_b : nullptr, s);
   else
-    rc = launch_bwd_mask_generic(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->M, a->maskbits_b, a->vals_b, a->meta_b, s);
+    rc = launch_bwd_mask_generic(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->M, a->maskbits_b, a->vals_b, a->meta_b,
+                                 pack ? 1 : 2, s);
   if (rc) return rc;
-  if (!fused && (rc = launch_hw_meta(a->meta_b, a->J, a->I, a->hw_meta_b, s))) return rc;
+  if (pack && !fused && (rc = launch_hw_meta(a->meta_b, a->J, a->I, a->hw_meta_b, s))) return rc;
   if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, s))) return rc;
-  if ((rc = launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, a->dX, a->status_word, s))) return rc;
+  if (pack) rc = launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, a->dX, a->status_word, s);
+  else rc = launch_dense_nt(a->vals_b, dYp, a->J, a->T, a->I, a->dX, a->status_word, s);
+  if (rc) return rc;
   return launch_wgrad_impl(a->dY, a->X, a->T, a->I, a->J, a->dW, partials, a->status_word, s);
 }
 
@@ -368,8 +384,10 @@ int bimask_train_step(const bimask_train_args* a) {
   int rc = layer_step_impl(&l, a->premasked != 0);
   if (rc != BIMASK_OK) return rc;
   // the update reads dW after the weight-gradient kernel on the same stream, then the next mask
+  const bool pack = l.N <= 2;      // otherwise vals_f is the dense masked operand and there is no metadata
   return bimask_sgd_fwd_mask(const_cast<float*>(l.W), l.dW, a->mom, l.I, l.J, l.N, l.M, a->lr, a->momentum,
-                             a->weight_decay, l.maskbits_f, l.vals_f, l.meta_f, l.hw_meta_f, l.stream);
+                             a->weight_decay, l.maskbits_f, l.vals_f, pack ? l.meta_f : nullptr,
+                             pack ? l.hw_meta_f : nullptr, l.stream);
 }
 
 }  // extern "C"

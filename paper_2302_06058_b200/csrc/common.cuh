@@ -56,20 +56,25 @@ int launch_score(const uint32_t* maskbits_f, const int32_t* cands, int I, int J,
 int launch_pick(const int64_t* counts, const int32_t* cands, int P, int I, int32_t* best_idx,
                 int32_t* best_perm, cudaStream_t s);
 // N:M patterns with M = 8 or 16 (nm_generic_kernels.cu); vals / meta may be null (mask bits only).
+// mode (generic mask launchers): 0 mask bits only, 1 the 2:4 operand, 2 the dense masked bf16 operand in `vals`
 int launch_fwd_mask_generic(const float* W, int I, int J, int N, int M, uint32_t* maskbits, uint16_t* vals_or_null,
-                            uint32_t* meta_or_null, cudaStream_t s);
+                            uint32_t* meta_or_null, int mode, cudaStream_t s);
 int launch_score_generic(const uint32_t* bits, const int32_t* cands, int I, int J, int N, int M, int P,
                          int64_t* counts, cudaStream_t s);
 int launch_bwd_mask_generic(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J, int N, int M,
-                            uint32_t* maskbits_b, uint16_t* vals_b_or_null, uint32_t* meta_b_or_null, cudaStream_t s);
+                            uint32_t* maskbits_b, uint16_t* vals_b_or_null, uint32_t* meta_b_or_null, int mode, cudaStream_t s);
 int launch_bwd_mask_criterion(const float* W, const float* S, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                               int N, int M, int crit, uint64_t seed, uint32_t* maskbits_b, uint16_t* vals_b_or_null,
-                              uint32_t* meta_b_or_null, cudaStream_t s);
+                              uint32_t* meta_b_or_null, int mode, cudaStream_t s);
 int launch_check_perms(const int32_t* cands, int P, int I, int32_t* ok, uint8_t* seen, cudaStream_t s);
 int launch_wait_probe(int32_t* status_word, cudaStream_t s);
 int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, uint16_t* dYp, cudaStream_t s);
 int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim, int Kdim,
                 uint16_t* out, int32_t* status_word, cudaStream_t s);
+// Dense product for masked operands that do not fit the 2:4 format: out[n][m] = sum_k A[m][k] B[n][k],
+// A bf16 [Mdim][Kdim], B bf16 [Ndim][Kdim], out bf16 [Ndim][Mdim] (same roles as launch_spmm).
+int launch_dense_nt(const uint16_t* A, const uint16_t* Bop, int Mdim, int Ndim, int Kdim, uint16_t* out,
+                    int32_t* status_word, cudaStream_t s);
 void wgrad_plan(int T, int I, int J, int* n_tile, int* splits, int* k_tiles_per_split);
 int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J, float* dW, float* partials,
                       int32_t* status_word, cudaStream_t s);

@@ -26,15 +26,15 @@ namespace {
 constexpr long long WAIT_BUDGET = 4000000000ll;      // ~2 s of SM clocks
 constexpr int GEMM_THREADS = 192;                    // warp 0 TMA, warp 1 MMA, warps 2-5 epilogue
 
-template <int N_TILE, int STAGES>
+template <int N_TILE, int STAGES, bool SPARSE = true>
 struct Cfg {
   static constexpr int M_TILE = 128;
   static constexpr int K_TILE = 128;                             // logical reduction elements per stage
-  static constexpr int A_BYTES = 16384;                          // 128 x 64 bf16 either way
+  static constexpr int A_BYTES = SPARSE ? 16384 : 32768;         // 128 rows x 64 compressed, or x 128 dense, bf16
   static constexpr int B_BYTES = N_TILE * K_TILE * 2;
-  static constexpr int E_BYTES = 2048;
+  static constexpr int E_BYTES = SPARSE ? 2048 : 0;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
-  static constexpr int META_COLS = 4;
+  static constexpr int META_COLS = SPARSE ? 4 : 0;
   static constexpr int TMEM_COLS = (N_TILE + META_COLS) <= 128 ? 128 : (N_TILE + META_COLS) <= 256 ? 256 : 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 };
@@ -65,11 +65,13 @@ __device__ __forceinline__ void raster(int id, int tiles_m, int tiles_n, int gro
   tn = in / gsize;
 }
 
-template <int N_TILE, int STAGES>
+// SPARSE = false: the same pipeline on a dense bf16 A operand (masked weights of a pattern the
+// 2:4 format cannot hold): 128 x 128 A tile per stage as two 64-wide boxes, eight K = 16 MMAs.
+template <int N_TILE, int STAGES, bool SPARSE>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                    const GemmParams p) {
-  using C = Cfg<N_TILE, STAGES>;
+  using C = Cfg<N_TILE, STAGES, SPARSE>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -123,17 +125,23 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
         const uint32_t a_s = base + s * C::STAGE_BYTES;
         const uint32_t b_s = a_s + C::A_BYTES;
         ptx::mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
-        ptx::tma_load_2d(a_s, &tmapA, kt * 64, m0, full_bar(s));                      // 64 compressed x 128 rows
+        if (SPARSE) {
+          ptx::tma_load_2d(a_s, &tmapA, kt * 64, m0, full_bar(s));                    // 64 compressed x 128 rows
+        } else {
+          ptx::tma_load_2d(a_s, &tmapA, kt * 128, m0, full_bar(s));                   // k 0..63
+          ptx::tma_load_2d(a_s + 16384, &tmapA, kt * 128 + 64, m0, full_bar(s));      // k 64..127
+        }
         ptx::tma_load_2d(b_s, &tmapB, kt * 128, n0, full_bar(s));                     // k 0..63
         ptx::tma_load_2d(b_s + N_TILE * 128, &tmapB, kt * 128 + 64, n0, full_bar(s)); // k 64..127
-        ptx::bulk_load(b_s + C::B_BYTES,
-                       p.hw_meta + ((size_t)tile_m * p.tiles_k_meta + kt) * 2048, 2048, full_bar(s));
+        if (SPARSE)
+          ptx::bulk_load(b_s + C::B_BYTES,
+                         p.hw_meta + ((size_t)tile_m * p.tiles_k_meta + kt) * 2048, 2048, full_bar(s));
       }
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
     if (ptx::elect_one()) {
-      constexpr uint32_t idesc = ptx::idesc_bf16(128, N_TILE, false, false, true);
+      constexpr uint32_t idesc = ptx::idesc_bf16(128, N_TILE, false, false, SPARSE);
       bool ok = true;
       for (int it = 0; it < num_kt && ok; ++it) {
         const int s = it % STAGES;
@@ -142,12 +150,21 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
         ptx::tc_fence_after();
         const uint32_t a_s = base + s * C::STAGE_BYTES;
         const uint32_t b_s = a_s + C::A_BYTES;
-        ptx::tmem_cp_128x128b(tmem_meta, ptx::smem_desc(b_s + C::B_BYTES, 0, 128, 0));
+        if constexpr (SPARSE) {
+          ptx::tmem_cp_128x128b(tmem_meta, ptx::smem_desc(b_s + C::B_BYTES, 0, 128, 0));
 #pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-          const uint64_t ad = ptx::smem_desc(a_s + kb * 32, 16, 1024, 2);
-          const uint64_t bd = ptx::smem_desc(b_s + (kb >> 1) * (N_TILE * 128) + (kb & 1) * 64, 16, 1024, 2);
-          ptx::mma_sparse(tmem_base, ad, bd, tmem_meta + (kb & ~1), idesc | (uint32_t)(kb & 1), (it | kb) != 0);
+          for (int kb = 0; kb < 4; ++kb) {
+            const uint64_t ad = ptx::smem_desc(a_s + kb * 32, 16, 1024, 2);
+            const uint64_t bd = ptx::smem_desc(b_s + (kb >> 1) * (N_TILE * 128) + (kb & 1) * 64, 16, 1024, 2);
+            ptx::mma_sparse(tmem_base, ad, bd, tmem_meta + (kb & ~1), idesc | (uint32_t)(kb & 1), (it | kb) != 0);
+          }
+        } else {
+#pragma unroll
+          for (int kb = 0; kb < 8; ++kb) {                                   // K = 16 each: 32 bytes inside a 128-byte row
+            const uint64_t ad = ptx::smem_desc(a_s + (kb >> 2) * 16384 + (kb & 3) * 32, 16, 1024, 2);
+            const uint64_t bd = ptx::smem_desc(b_s + (kb >> 2) * (N_TILE * 128) + (kb & 3) * 32, 16, 1024, 2);
+            ptx::mma_dense(tmem_base, ad, bd, idesc, (it | kb) != 0);
+          }
         }
         ptx::tc_commit(empty_bar(s));
       }
@@ -808,15 +825,15 @@ int set_smem_attr(K kernel, int bytes) {
   return BIMASK_OK;
 }
 
-template <int N_TILE, int STAGES>
+template <int N_TILE, int STAGES, bool SPARSE = true>
 int run_sparse(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim, int Kdim,
                uint16_t* out, int32_t* status_word, cudaStream_t s) {
-  using C = Cfg<N_TILE, STAGES>;
+  using C = Cfg<N_TILE, STAGES, SPARSE>;
   CUtensorMap ta, tb;
   int rc;
-  if ((rc = make_tmap(&ta, vals, (uint64_t)Kdim / 2, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap(&ta, vals, SPARSE ? (uint64_t)Kdim / 2 : (uint64_t)Kdim, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, N_TILE)) != BIMASK_OK) return rc;
-  auto kern = spmm_single_kernel<N_TILE, STAGES>;
+  auto kern = spmm_single_kernel<N_TILE, STAGES, SPARSE>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
   p.hw_meta = reinterpret_cast<const uint8_t*>(hw_meta);
@@ -898,6 +915,12 @@ int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, 
   if (Ndim > 128 && Mdim > 128) return run_sparse_pair_persistent(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   if (Ndim > 128) return run_sparse<256, 2>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   return run_sparse<128, 4>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
+}
+
+int launch_dense_nt(const uint16_t* A, const uint16_t* Bop, int Mdim, int Ndim, int Kdim, uint16_t* out,
+                    int32_t* status_word, cudaStream_t s) {
+  if (Ndim > 128) return run_sparse<256, 2, false>(A, nullptr, Bop, Mdim, Ndim, Kdim, out, status_word, s);
+  return run_sparse<128, 3, false>(A, nullptr, Bop, Mdim, Ndim, Kdim, out, status_word, s);
 }
 
 int launch_wait_probe(int32_t* status_word, cudaStream_t s) {

@@ -63,7 +63,9 @@ __device__ __forceinline__ uint32_t keep_block(const uint32_t (&key)[M], uint32_
 // Forward mask (+ pack when PACK).  One lane per block of M consecutive weights; the 32 / M lanes
 // that share a 32-column word OR their pieces together.
 // ---------------------------------------------------------------------------------------
-template <int M, bool PACK>
+// MODE 0: mask bits only; 1: 2:4 operand (values + index codes); 2: dense masked bf16 operand
+// (kept weights rounded to bf16, +0 elsewhere) for patterns the 2:4 format cannot hold.
+template <int M, int MODE>
 __global__ void __launch_bounds__(256)
 fwd_mask_generic_kernel(const float4* __restrict__ W4, long long nblocks, int N,
                         uint32_t* __restrict__ maskbits, uint32_t* __restrict__ vals32,
@@ -91,7 +93,7 @@ fwd_mask_generic_kernel(const float4* __restrict__ W4, long long nblocks, int N,
     for (int m = 0; m < M; ++m) key[m] = mag_key(w[m]);
     const uint32_t kb = keep_block<M>(key, (M == 16 ? 0xFFFFu : 0xFFu), N);
     uint32_t codes = 0;
-    if (PACK) {
+    if (MODE == 1) {
 #pragma unroll
       for (int g = 0; g < G; ++g) {
         const uint32_t e = pad16[(kb >> (4 * g)) & 15u];
@@ -101,11 +103,26 @@ fwd_mask_generic_kernel(const float4* __restrict__ W4, long long nblocks, int N,
         codes |= ((e >> 4) & 15u) << (4 * g);
       }
     }
+    if (MODE == 2 && live) {
+      uint4* dst = reinterpret_cast<uint4*>(vals32) + b * (M / 8);
+#pragma unroll
+      for (int h = 0; h < M / 8; ++h) {
+        uint32_t d[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int m = 8 * h + 2 * j;
+          const uint32_t lo = ((kb >> m) & 1u) ? to_bf16(w[m]) : 0u;
+          const uint32_t hi = ((kb >> (m + 1)) & 1u) ? to_bf16(w[m + 1]) : 0u;
+          d[j] = lo | (hi << 16);
+        }
+        dst[h] = make_uint4(d[0], d[1], d[2], d[3]);
+      }
+    }
     const uint32_t wb = __reduce_or_sync(gmask, kb << sh);
     const uint32_t wm = __reduce_or_sync(gmask, codes << sh);
     if (live && (lane & (LPW - 1)) == 0) {
       maskbits[b / LPW] = wb;
-      if (PACK) meta[b / LPW] = wm;
+      if (MODE == 1) meta[b / LPW] = wm;
     }
   }
 }
@@ -221,7 +238,7 @@ __device__ __forceinline__ uint32_t multinomial_block(const float (&w)[M], uint3
   return keep;
 }
 
-template <int M, bool PACK, int CRIT>
+template <int M, int MODE, int CRIT>
 __global__ void __launch_bounds__(256)
 bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,
                         const int32_t* __restrict__ perm, int I, int J, int N,
@@ -242,6 +259,7 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
   const int my_src = (int)min((unsigned)__ldg(perm + 32 * pass + lane), last_row);   // lane r: source of permuted row r
   uint32_t my_word = 0;                                     // lane r ends up with the mask word of permuted row r
   uint32_t vacc[8];
+  uint32_t dacc[MODE == 2 ? 16 : 1];                        // dense: this column's 32 permuted rows as bf16 pairs
   uint32_t cacc = 0;
 #pragma unroll
   for (int nb = 0; nb < NB; ++nb) {
@@ -268,7 +286,15 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
       const uint32_t word = __ballot_sync(0xFFFFFFFFu, (kb >> m) & 1u);
       if (lane == nb * M + m) my_word = word;
     }
-    if (PACK) {
+    if (MODE == 2) {
+#pragma unroll
+      for (int m = 0; m < M; m += 2) {
+        const uint32_t lo = ((kb >> m) & 1u) ? to_bf16(w[m]) : 0u;
+        const uint32_t hi = ((kb >> (m + 1)) & 1u) ? to_bf16(w[m + 1]) : 0u;
+        dacc[(nb * M + m) / 2] = lo | (hi << 16);
+      }
+    }
+    if (MODE == 1) {
 #pragma unroll
       for (int g = 0; g < G; ++g) {
         const uint32_t e = pad16[(kb >> (4 * g)) & 15u];
@@ -279,30 +305,37 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
     }
   }
   maskbits_b[(size_t)(32 * pass + lane) * jwords + cw] = my_word;
-  if (PACK) {
+  if (MODE == 1) {
     uint4* dst = reinterpret_cast<uint4*>(vals_b + (size_t)col * (I >> 2) + 8 * pass);
     dst[0] = make_uint4(vacc[0], vacc[1], vacc[2], vacc[3]);
     dst[1] = make_uint4(vacc[4], vacc[5], vacc[6], vacc[7]);
     meta_b[(size_t)col * (I >> 5) + pass] = cacc;
   }
+  if (MODE == 2) {
+    uint4* dst = reinterpret_cast<uint4*>(vals_b + (size_t)col * (I >> 1) + 16 * pass);   // row `col` of the J x I operand
+#pragma unroll
+    for (int q = 0; q < 4; ++q) dst[q] = make_uint4(dacc[4 * q], dacc[4 * q + 1], dacc[4 * q + 2], dacc[4 * q + 3]);
+  }
 }
 
 }  // namespace
 
+// mode: 0 mask bits only, 1 the 2:4 operand, 2 the dense masked operand (written to `vals`)
 int launch_fwd_mask_generic(const float* W, int I, int J, int N, int M, uint32_t* maskbits, uint16_t* vals_or_null,
-                            uint32_t* meta_or_null, cudaStream_t s) {
+                            uint32_t* meta_or_null, int mode, cudaStream_t s) {
   const long long nblocks = (long long)I * J / M;
   long long ctas = (nblocks + 255) / 256;
   if (ctas > 148 * 16) ctas = 148 * 16;
   const float4* W4 = reinterpret_cast<const float4*>(W);
   uint32_t* v32 = reinterpret_cast<uint32_t*>(vals_or_null);
-  const bool pack = vals_or_null != nullptr;
   if (M == 8) {
-    if (pack) fwd_mask_generic_kernel<8, true><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
-    else fwd_mask_generic_kernel<8, false><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
+    if (mode == 1) fwd_mask_generic_kernel<8, 1><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
+    else if (mode == 2) fwd_mask_generic_kernel<8, 2><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
+    else fwd_mask_generic_kernel<8, 0><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
   } else {
-    if (pack) fwd_mask_generic_kernel<16, true><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
-    else fwd_mask_generic_kernel<16, false><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
+    if (mode == 1) fwd_mask_generic_kernel<16, 1><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
+    else if (mode == 2) fwd_mask_generic_kernel<16, 2><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
+    else fwd_mask_generic_kernel<16, 0><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
   }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
@@ -340,49 +373,51 @@ int launch_score_generic(const uint32_t* bits, const int32_t* cands, int I, int 
 }
 
 template <int M, int CRIT>
-static void launch_bwd_mc(dim3 grid, bool pack, const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
+static void launch_bwd_mc(dim3 grid, int mode, const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                           int N, uint32_t* maskbits_b, uint32_t* v32, uint32_t* meta_b, const float* S, uint64_t seed,
                           cudaStream_t s) {
-  if (pack) bwd_mask_generic_kernel<M, true, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed);
-  else bwd_mask_generic_kernel<M, false, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed);
+  if (mode == 1) bwd_mask_generic_kernel<M, 1, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed);
+  else if (mode == 2) bwd_mask_generic_kernel<M, 2, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed);
+  else bwd_mask_generic_kernel<M, 0, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed);
 }
 
 template <int M>
-static void launch_bwd_m(int crit, dim3 grid, bool pack, const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I,
+static void launch_bwd_m(int crit, dim3 grid, int mode, const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I,
                          int J, int N, uint32_t* maskbits_b, uint32_t* v32, uint32_t* meta_b, const float* S, uint64_t seed,
                          cudaStream_t s) {
   switch (crit) {
-    case 1: launch_bwd_mc<M, 1>(grid, pack, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
-    case 2: launch_bwd_mc<M, 2>(grid, pack, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
-    case 3: launch_bwd_mc<M, 3>(grid, pack, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
-    default: launch_bwd_mc<M, 0>(grid, pack, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
+    case 1: launch_bwd_mc<M, 1>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
+    case 2: launch_bwd_mc<M, 2>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
+    case 3: launch_bwd_mc<M, 3>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
+    default: launch_bwd_mc<M, 0>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
   }
 }
 
 // criterion 0..3 as in the kernel's comment; S is read for criterion 1 only; for criterion 3 `seed`
-// is hashed once here so that the per-weight key is mix64(mix64(seed) + i*J + j) >> 33
+// is hashed once here so that the per-weight key is mix64(mix64(seed) + i*J + j) >> 33.
+// mode: 0 mask bits only, 1 the transposed 2:4 operand, 2 the transposed dense masked operand.
 int launch_bwd_mask_criterion(const float* W, const float* S, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                               int N, int M, int crit, uint64_t seed, uint32_t* maskbits_b, uint16_t* vals_b_or_null,
-                              uint32_t* meta_b_or_null, cudaStream_t s) {
+                              uint32_t* meta_b_or_null, int mode, cudaStream_t s) {
   dim3 grid(I / 32, (J / 32 + 7) / 8);
   uint32_t* v32 = reinterpret_cast<uint32_t*>(vals_b_or_null);
-  const bool pack = vals_b_or_null != nullptr;
   if (crit == 3) {
     uint64_t z = seed;
     z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull; z ^= z >> 27; z *= 0x94D049BB133111EBull; z ^= z >> 31;
     seed = z;
   }
-  if (M == 4) launch_bwd_m<4>(crit, grid, pack, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, s);
-  else if (M == 8) launch_bwd_m<8>(crit, grid, pack, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, s);
-  else launch_bwd_m<16>(crit, grid, pack, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, s);
+  if (M == 4) launch_bwd_m<4>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, s);
+  else if (M == 8) launch_bwd_m<8>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, s);
+  else launch_bwd_m<16>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, s);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }
 
 int launch_bwd_mask_generic(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J, int N, int M,
-                            uint32_t* maskbits_b, uint16_t* vals_b_or_null, uint32_t* meta_b_or_null, cudaStream_t s) {
-  return launch_bwd_mask_criterion(W, nullptr, maskbits_f, perm, I, J, N, M, 0, 0, maskbits_b, vals_b_or_null, meta_b_or_null, s);
+                            uint32_t* maskbits_b, uint16_t* vals_b_or_null, uint32_t* meta_b_or_null, int mode, cudaStream_t s) {
+  return launch_bwd_mask_criterion(W, nullptr, maskbits_f, perm, I, J, N, M, 0, 0, maskbits_b, vals_b_or_null, meta_b_or_null,
+                                   mode, s);
 }
 
 }  // namespace bimask

@@ -199,7 +199,7 @@ def test_error_paths_launch_nothing():
     with pytest.raises(bm.BimaskError) as e:
         bm.bimask_fwd_mask(W, 64, 64, 2, 32, b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"])
     assert e.value.code == bm.binding.BIMASK_EUNSUPPORTED
-    with pytest.raises(bm.BimaskError) as e:     # 4:8 has no 2:4 container: packed outputs must be NULL
+    with pytest.raises(bm.BimaskError) as e:     # 4:8 has no 2:4 container: there is no metadata to write
         bm.bimask_fwd_mask(W, 64, 64, 4, 8, b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"])
     assert e.value.code == bm.binding.BIMASK_EUNSUPPORTED
     with pytest.raises(bm.BimaskError) as e:
@@ -312,15 +312,20 @@ def test_other_patterns_masks_and_search(N, M, I, J):
     W = special_weights(I, J, 7 * I + J + N + M) if I < 1000 else inputs.make_weight(I, J, N + M)
     pack = N <= 2
     Wd = dev(W)
-    b = bm.alloc_layer_buffers(1, I, J, 4)
+    b = bm.alloc_layer_buffers(1, I, J, 4, dense=not pack)
     opt = (lambda t: t) if pack else (lambda t: None)
-    bm.bimask_fwd_mask(Wd, I, J, N, M, b["maskbits_f"], opt(b["vals_f"]), opt(b["meta_f"]), opt(b["hw_meta_f"]))
+    bm.bimask_fwd_mask(Wd, I, J, N, M, b["maskbits_f"], b["vals_f"], opt(b["meta_f"]), opt(b["hw_meta_f"]))
     B = O.forward_mask(W, N, M)
     assert np.array_equal(u32(b["maskbits_f"]), O.pack_bits(B))
     if pack:
         _, vals, meta = O.forward_operand(W, B)
         assert np.array_equal(u32(b["meta_f"]), meta)
         assert np.array_equal(u16(b["vals_f"]), vals)
+    else:                                   # no 2:4 form: the dense masked operand
+        assert np.array_equal(u16(b["vals_f"]), O.dense_operand(W, B))
+        before = b["maskbits_f"].clone()
+        bm.bimask_fwd_mask(Wd, I, J, N, M, b["maskbits_f"], None, None, None)        # mask bits only
+        assert torch.equal(before, b["maskbits_f"])
     # search
     P, seed = 4, 99 + M
     ws_bytes = bm.bimask_workspace_bytes(1, I, J, P)
@@ -332,7 +337,7 @@ def test_other_patterns_masks_and_search(N, M, I, J):
     assert int(b["best_idx"].item()) == best
     assert np.array_equal(b["perm"].cpu().numpy(), perm)
     # backward mask on the chosen permutation
-    bm.bimask_bwd_mask(Wd, b["maskbits_f"], b["perm"], I, J, N, M, b["maskbits_b"], opt(b["vals_b"]), opt(b["meta_b"]),
+    bm.bimask_bwd_mask(Wd, b["maskbits_f"], b["perm"], I, J, N, M, b["maskbits_b"], b["vals_b"], opt(b["meta_b"]),
                        opt(b["hw_meta_b"]))
     torch.cuda.synchronize()
     Bbar = O.backward_mask(W, B, perm, N, M)
@@ -341,6 +346,8 @@ def test_other_patterns_masks_and_search(N, M, I, J):
         _, vals, meta = O.backward_operand(W, Bbar, perm)
         assert np.array_equal(u32(b["meta_b"]), meta)
         assert np.array_equal(u16(b["vals_b"]), vals)
+    else:
+        assert np.array_equal(u16(b["vals_b"]), O.dense_backward_operand(W, Bbar, perm))
 
 
 @pytest.mark.parametrize("N,M", [(2, 8), (1, 8), (1, 16)])
@@ -362,14 +369,37 @@ def test_other_patterns_layer_step(N, M):
     assert rel_err(b["dW"].cpu().numpy(), ref["dW"]) <= TOL
 
 
-def test_four_to_eight_layer_step_is_refused():
-    b = bm.alloc_layer_buffers(32, 64, 64, 2)
-    b["W"] = torch.zeros(64, 64, device="cuda")
-    b["X"] = torch.zeros(32, 64, dtype=torch.bfloat16, device="cuda")
-    b["dY"] = torch.zeros(32, 64, dtype=torch.bfloat16, device="cuda")
-    with pytest.raises(bm.BimaskError) as e:
-        bm.bimask_layer_step(bm.make_layer_args(32, 64, 64, 4, 8, 2, 1, True, b))
-    assert e.value.code == bm.binding.BIMASK_EUNSUPPORTED
+@pytest.mark.parametrize("N,M,I,J,T", [(4, 8, 384, 512, 300), (4, 8, 128, 1056, 100), (3, 8, 1024, 384, 1000),
+                                       (4, 16, 96, 160, 129), (8, 8, 256, 256, 64)])
+def test_unpackable_patterns_run_the_layer_step_on_dense_operands(N, M, I, J, T):
+    """4:8 (and any pattern with more than two survivors in a group of four) has no sparse tensor-core
+    format: the step runs the same masks and search and feeds dense masked operands to the products."""
+    W = inputs.make_weight(I, J, 200 + N + M)
+    X = inputs.make_activation(T, J, 201)
+    dY = inputs.make_activation(T, I, 202)
+    b = bm.alloc_layer_buffers(T, I, J, 5, dense=True)
+    b["W"], b["X"], b["dY"] = dev(W), bits_dev(X), bits_dev(dY)
+    b["meta_f"] = b["hw_meta_f"] = b["meta_b"] = b["hw_meta_b"] = None
+    bm.bimask_layer_step(bm.make_layer_args(T, I, J, N, M, 5, 17, True, b))
+    torch.cuda.synchronize()
+    ref = O.layer_step(W, X, dY, N, M, 5, 17, do_search=True)
+    assert int(b["status_word"].item()) == 0
+    assert np.array_equal(u32(b["maskbits_f"]), O.pack_bits(ref["B"]))
+    assert np.array_equal(u16(b["vals_f"]), O.dense_operand(W, ref["B"]))
+    assert np.array_equal(b["counts"].cpu().numpy(), ref["counts"])
+    assert np.array_equal(b["perm"].cpu().numpy(), ref["perm"])
+    assert np.array_equal(u32(b["maskbits_b"]), O.pack_bits(ref["Bbar_p"]))
+    assert np.array_equal(u16(b["vals_b"]), O.dense_backward_operand(W, ref["Bbar_p"], ref["perm"]))
+    assert rel_err(b["Y"].float().cpu().numpy(), ref["Y"]) <= TOL
+    assert rel_err(b["dX"].float().cpu().numpy(), ref["dX"]) <= TOL
+    assert rel_err(b["dW"].cpu().numpy(), ref["dW"]) <= TOL
+    # the stand-alone products accept the dense operand when no metadata image is given
+    Y2 = torch.empty_like(b["Y"])
+    bm.bimask_spmm_fwd(b["X"], b["vals_f"], None, T, I, J, Y2, b["status_word"])
+    dX2 = torch.empty_like(b["dX"])
+    bm.bimask_spmm_dgrad(b["dY"], b["perm"], b["vals_b"], None, T, I, J, dX2, b["ws"], b["ws"].numel(), b["status_word"])
+    torch.cuda.synchronize()
+    assert torch.equal(Y2, b["Y"]) and torch.equal(dX2, b["dX"])
 
 
 def test_bounded_wait_reports_timeout_and_context_survives():

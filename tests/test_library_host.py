@@ -61,7 +61,7 @@ def test_validation_happens_before_any_cuda_call(bm):
     assert L.bimask_fwd_mask(16, 64, 60, 2, 4, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_fwd_mask(16, 64, 64, 2, 32, 16, 16, 16, 16, None) == bm.binding.BIMASK_EUNSUPPORTED     # M = 32
     assert L.bimask_fwd_mask(16, 64, 64, 4, 8, 16, 16, 16, 16, None) == bm.binding.BIMASK_EUNSUPPORTED      # 4:8 cannot be packed
-    assert "mask bits only" in bm.bimask_last_error()
+    assert "dense masked operand" in bm.bimask_last_error()
     assert L.bimask_fwd_mask(16, 64, 64, 3, 4, 16, 16, 16, 16, None) == bm.binding.BIMASK_EUNSUPPORTED
     assert L.bimask_fwd_mask(16, 64, 64, 0, 4, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_fwd_mask(20, 64, 64, 2, 4, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL   # misaligned
