@@ -540,3 +540,66 @@ def backward_mask_criterion(W, B, perm, N, M, criterion, S=None, seed=0):
         remaining &= ~sel
     keep = np.where(many[..., None], keep, valid)
     return keep.transpose(0, 2, 1).reshape(I, J)
+
+
+# ---------------------------------------------------------------------------------------
+# The same layer step when the layer is a 3x3 convolution (stride 1, zero padding 1) on NHWC
+# activations: "W" of the paper is the I x J matrix view of the filter, J = 9*C, column
+# j = (kh*3 + kw)*C + c (the paper does not state the flatten order; this one keeps the channel
+# index contiguous, as in the NHWC activations).
+# ---------------------------------------------------------------------------------------
+def _pad_hw(a):
+    return np.pad(a, ((0, 0), (1, 1), (1, 1), (0, 0)))
+
+
+def conv_fwd(x_bits, W, B):
+    """y[n, h, w, i] = sum_{kh, kw, c} x[n, h+kh-1, w+kw-1, c] * (B.W)[i, (kh*3+kw)*C + c]  (Eq. 3 for a
+    convolution; out-of-range x is 0).  x_bits: bf16 bit patterns NB x H x W x C.  float64 result."""
+    NB, H, Wd, C = x_bits.shape
+    I = W.shape[0]
+    xp = _pad_hw(bf16_to_f64(x_bits).reshape(NB, H, Wd, C))
+    Wf = (bf16_round(W) * B).reshape(I, 3, 3, C)
+    y = np.zeros((NB, H, Wd, I))
+    for kh in range(3):
+        for kw in range(3):
+            y += xp[:, kh:kh + H, kw:kw + Wd, :] @ Wf[:, kh, kw, :].T
+    return y
+
+
+def conv_dgrad(dy_bits, W, M_b, C):
+    """dx[n, h, w, c] = sum_{kh, kw, i} dy[n, h-kh+1, w-kw+1, i] * (M_b.W)[i, (kh*3+kw)*C + c]: the input
+    gradient of conv_fwd with the backward mask in place of the forward one (Eq. 8 / Eq. 10)."""
+    NB, H, Wd, I = dy_bits.shape
+    dyp = _pad_hw(bf16_to_f64(dy_bits).reshape(NB, H, Wd, I))
+    Wb = (bf16_round(W) * M_b).reshape(I, 3, 3, C)
+    dx = np.zeros((NB, H, Wd, C))
+    for kh in range(3):
+        for kw in range(3):
+            # output pixel (h, w) receives from dy pixel (h-kh+1, w-kw+1): padded index h-kh+2
+            dx += dyp[:, 2 - kh:2 - kh + H, 2 - kw:2 - kw + Wd, :] @ Wb[:, kh, kw, :]
+    return dx
+
+
+def conv_wgrad(dy_bits, x_bits):
+    """dW[i, (kh*3+kw)*C + c] = sum_{n, h, w} dy[n, h, w, i] * x[n, h+kh-1, w+kw-1, c]  (dense, STE)."""
+    NB, H, Wd, C = x_bits.shape
+    I = dy_bits.shape[3]
+    xp = _pad_hw(bf16_to_f64(x_bits).reshape(NB, H, Wd, C))
+    dy = bf16_to_f64(dy_bits).reshape(NB * H * Wd, I)
+    dW = np.zeros((I, 3, 3, C))
+    for kh in range(3):
+        for kw in range(3):
+            dW[:, kh, kw, :] = dy.T @ xp[:, kh:kh + H, kw:kw + Wd, :].reshape(NB * H * Wd, C)
+    return dW.reshape(I, 9 * C)
+
+
+def conv_layer_step(W, x_bits, dy_bits, N, M, P, seed, do_search=True, perm=None):
+    """One iteration of Alg. 1 for a 3x3 convolution layer: masks and search exactly as for a linear
+    layer on the I x 9C matrix view; the three products are convolutions."""
+    C = x_bits.shape[3]
+    assert W.shape[1] == 9 * C
+    out = layer_step(W, None, None, N, M, P, seed, do_search=do_search, perm=perm, with_gemms=False)
+    out["y"] = conv_fwd(x_bits, W, out["B"])
+    out["dx"] = conv_dgrad(dy_bits, W, out["M_b"], C)
+    out["dW"] = conv_wgrad(dy_bits, x_bits)
+    return out

@@ -563,3 +563,56 @@ def test_dense_operand_agrees_with_the_packed_one():
     dY = O.bf16_bits(rng.standard_normal((8, 32)).astype(np.float32))
     want = O.spmm_dgrad(dY, W, O.unpermute_rows(Bbar, perm))
     assert np.allclose(O.bf16_to_f64(dY)[:, perm] @ O.bf16_to_f64(Db).T, want, rtol=1e-12, atol=1e-12)
+
+
+# ---------------------------------------------------------------- convolution layer
+def test_conv_products_match_torch_conv2d_and_autograd():
+    """Library pin: torch's conv2d (float64) and its autograd for the two gradients, on bf16-valued data."""
+    rng = np.random.default_rng(41)
+    NB, H, Wd, C, I = 2, 5, 6, 8, 12
+    W = rng.standard_normal((I, 9 * C)).astype(np.float32)
+    B = O.forward_mask(W, 2, 4)
+    perm = rng.permutation(I)
+    M_b = O.unpermute_rows(O.backward_mask(W, B, perm, 2, 4), perm)
+    x = O.bf16_bits(rng.standard_normal((NB, H, Wd, C)).astype(np.float32))
+    dy = O.bf16_bits(rng.standard_normal((NB, H, Wd, I)).astype(np.float32))
+
+    def filt(mask):        # I x (kh, kw, c)  ->  torch's I x C x kh x kw
+        return torch.from_numpy((O.bf16_round(W) * mask).reshape(I, 3, 3, C)).permute(0, 3, 1, 2).contiguous()
+
+    xt = torch.from_numpy(O.bf16_to_f64(x).reshape(NB, H, Wd, C)).permute(0, 3, 1, 2).contiguous().requires_grad_(True)
+    dyt = torch.from_numpy(O.bf16_to_f64(dy).reshape(NB, H, Wd, I)).permute(0, 3, 1, 2).contiguous()
+    y = torch.nn.functional.conv2d(xt, filt(B), padding=1)
+    assert np.allclose(O.conv_fwd(x, W, B), y.detach().permute(0, 2, 3, 1).numpy(), rtol=1e-12, atol=1e-12)
+    # input gradient through the BACKWARD mask: differentiate a convolution whose filter is M_b . W
+    wb = filt(M_b)
+    (gx,) = torch.autograd.grad(torch.nn.functional.conv2d(xt, wb, padding=1), xt, dyt)
+    assert np.allclose(O.conv_dgrad(dy, W, M_b, C), gx.permute(0, 2, 3, 1).numpy(), rtol=1e-12, atol=1e-12)
+    # dense weight gradient
+    wd = filt(np.ones_like(B)).requires_grad_(True)
+    (gw,) = torch.autograd.grad(torch.nn.functional.conv2d(xt.detach(), wd, padding=1), wd, dyt)
+    assert np.allclose(O.conv_wgrad(dy, x), gw.permute(0, 2, 3, 1).reshape(I, 9 * C).numpy(), rtol=1e-12, atol=1e-12)
+
+
+def test_conv_equals_the_linear_layer_on_the_column_matrix():
+    """im2col identity: the convolution is the linear layer applied to the T x 9C matrix of shifted pixels."""
+    rng = np.random.default_rng(43)
+    NB, H, Wd, C, I = 2, 4, 4, 8, 32
+    W = rng.standard_normal((I, 9 * C)).astype(np.float32)
+    x = O.bf16_bits(rng.standard_normal((NB, H, Wd, C)).astype(np.float32))
+    dy = O.bf16_bits(rng.standard_normal((NB, H, Wd, I)).astype(np.float32))
+    xp = np.pad(x, ((0, 0), (1, 1), (1, 1), (0, 0)))
+    cols = np.concatenate([xp[:, kh:kh + H, kw:kw + Wd, :] for kh in range(3) for kw in range(3)], axis=3)
+    Xcol = cols.reshape(NB * H * Wd, 9 * C)
+    ref = O.layer_step(W, Xcol, dy.reshape(-1, I), 2, 4, 4, 3, do_search=True)
+    got = O.conv_layer_step(W, x, dy, 2, 4, 4, 3, do_search=True)
+    assert np.array_equal(got["perm"], ref["perm"]) and np.array_equal(got["B"], ref["B"])
+    assert np.allclose(got["y"].reshape(-1, I), ref["Y"], rtol=1e-12, atol=1e-12)
+    assert np.allclose(got["dW"], ref["dW"], rtol=1e-12, atol=1e-12)
+    # dX of the linear layer lives in column space; folding it back (sum of the nine shifts) is dx
+    dXcol = ref["dX"].reshape(NB, H, Wd, 9, C)
+    dx = np.zeros((NB, H + 2, Wd + 2, C))
+    for kh in range(3):
+        for kw in range(3):
+            dx[:, kh:kh + H, kw:kw + Wd, :] += dXcol[:, :, :, kh * 3 + kw, :]
+    assert np.allclose(got["dx"], dx[:, 1:-1, 1:-1, :], rtol=1e-12, atol=1e-12)
