@@ -597,7 +597,7 @@ def test_conv_products_match_torch_conv2d_and_autograd():
 def test_conv_equals_the_linear_layer_on_the_column_matrix():
     """im2col identity: the convolution is the linear layer applied to the T x 9C matrix of shifted pixels."""
     rng = np.random.default_rng(43)
-    NB, H, Wd, C, I = 2, 4, 4, 8, 32
+    NB, H, Wd, C, I = 2, 4, 4, 32, 32
     W = rng.standard_normal((I, 9 * C)).astype(np.float32)
     x = O.bf16_bits(rng.standard_normal((NB, H, Wd, C)).astype(np.float32))
     dy = O.bf16_bits(rng.standard_normal((NB, H, Wd, I)).astype(np.float32))
