@@ -20,7 +20,7 @@ EXPORTS = ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "
            "bimask_layer_step", "bimask_layer_step_host", "bimask_layer_step_host_async", "bimask_host_sync",
            "bimask_check_perms", "bimask_debug_wait_probe", "bimask_perm_search_static",
            "bimask_perm_search_static_max_entries", "bimask_sgd_fwd_mask", "bimask_train_step",
-           "bimask_bwd_mask_criterion")
+           "bimask_bwd_mask_criterion", "bimask_conv_workspace_bytes", "bimask_conv_layer_step")
 
 
 class BimaskError(RuntimeError):
@@ -46,6 +46,13 @@ class TrainArgs(Structure):
     _fields_ = [("layer", LayerArgs), ("mom", c_void_p), ("lr", c_float), ("momentum", c_float),
                 ("weight_decay", c_float), ("t", c_int64), ("delta_t", c_int32), ("premasked", c_int32)]
 
+
+class ConvArgs(Structure):
+    """Mirror of bimask_conv_args."""
+    _fields_ = [("layer", LayerArgs), ("NB", c_int), ("H", c_int), ("W", c_int), ("C", c_int), ("mode", c_int)]
+
+
+CONV_AUTO, CONV_EXPLICIT, CONV_IMPLICIT = 0, 1, 2
 
 _lib = None
 
@@ -77,6 +84,9 @@ def lib() -> ctypes.CDLL:
         L.bimask_layer_step_host.argtypes = [POINTER(LayerArgs), POINTER(LayerArgs), c_void_p]
         L.bimask_layer_step_host_async.argtypes = [POINTER(LayerArgs), POINTER(LayerArgs), c_void_p]
         L.bimask_host_sync.argtypes = []
+        L.bimask_conv_workspace_bytes.restype = c_size_t
+        L.bimask_conv_workspace_bytes.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int]
+        L.bimask_conv_layer_step.argtypes = [POINTER(ConvArgs)]
         L.bimask_bwd_mask_criterion.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_int,
                                                 c_uint64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
         L.bimask_sgd_fwd_mask.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_float, c_float,
@@ -90,7 +100,7 @@ def lib() -> ctypes.CDLL:
         for name in EXPORTS:
             if name not in ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "bimask_workspace_bytes",
                             "bimask_perm_search_static_max_entries", "bimask_sgd_fwd_mask", "bimask_train_step",
-           "bimask_bwd_mask_criterion"):
+           "bimask_bwd_mask_criterion", "bimask_conv_workspace_bytes", "bimask_conv_layer_step"):
                 getattr(L, name).restype = c_int
         _lib = L
     return _lib
@@ -203,6 +213,21 @@ def bimask_sgd_fwd_mask(W, dW, mom_or_null, I, J, N, M, lr, momentum, weight_dec
     return _check(lib().bimask_sgd_fwd_mask(_ptr(W), _ptr(dW), _ptr(mom_or_null), I, J, N, M, lr, momentum, weight_decay,
                                             _ptr(maskbits_f), _ptr(vals_f), _ptr(meta_f), _ptr(hw_meta_f),
                                             _stream(stream)))
+
+
+def bimask_conv_workspace_bytes(NB, H, W, C, I, P) -> int:
+    return lib().bimask_conv_workspace_bytes(NB, H, W, C, I, P)
+
+
+def make_conv_args(layer: LayerArgs, NB, H, W, C, mode=CONV_AUTO) -> ConvArgs:
+    a = ConvArgs()
+    ctypes.memmove(ctypes.byref(a.layer), ctypes.byref(layer), ctypes.sizeof(LayerArgs))
+    a.NB, a.H, a.W, a.C, a.mode = NB, H, W, C, mode
+    return a
+
+
+def bimask_conv_layer_step(args: ConvArgs):
+    return _check(lib().bimask_conv_layer_step(ctypes.byref(args)))
 
 
 def make_train_args(layer: LayerArgs, mom, lr, momentum, weight_decay, t, delta_t, premasked) -> TrainArgs:

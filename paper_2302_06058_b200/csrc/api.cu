@@ -286,8 +286,18 @@ int bimask_wgrad(const uint16_t* dY, const uint16_t* X, int T, int I, int J, flo
 
 }  // extern "C"
 
-// skip_fwd_mask: the forward mask / operand of the current W is already in place
-static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask) {
+// A 3x3 convolution layer seen by the layer step: geometry, which products fetch shifted pixel
+// patches themselves (implicit) and the column-space scratch of those that do not.
+struct ConvPlan {
+  int NB, H, W, C;
+  bool imp_fwd, imp_dgrad, imp_wgrad;
+  uint16_t* xcol;     // T x 9C, when the forward or weight-gradient product is explicit
+  uint16_t* dxcol;    // T x 9C, when the input gradient is explicit
+};
+
+// skip_fwd_mask: the forward mask / operand of the current W is already in place.
+// conv: null for a linear layer; otherwise a->X is x (T x C) and a->dX is dx (T x C).
+static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const ConvPlan* conv = nullptr) {
   BIMASK_REQUIRE(a != nullptr, BIMASK_EINVAL, "bimask_layer_step: null argument block");
   bool pack = false;
   int rc = check_shape(a->I, a->J, a->N, a->M, &pack);
@@ -328,6 +338,14 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask) {
   // with the bandwidth-bound chain on a second stream was measured and rejected: the co-resident
   // kernels contend for issue slots and the step became slower and erratic.)
   cudaStream_t s = (cudaStream_t)a->stream;
+  const uint16_t* Xmat = a->X;                       // the T x J activation matrix of the explicit products
+  uint16_t* dXmat = a->dX;
+  if (conv) {
+    Xmat = conv->xcol;
+    dXmat = conv->dxcol;
+    if (!conv->imp_fwd || !conv->imp_wgrad)
+      if ((rc = launch_im2col3x3(a->X, conv->NB, conv->H, conv->W, conv->C, conv->xcol, s))) return rc;
+  }
   // M = 4 with unpadded shapes writes the metadata images inside the mask kernels
   const bool fused = a->M == 4 && (a->I % 128 == 0) && (a->J % 128 == 0);
   if (!skip_fwd_mask) {
@@ -338,8 +356,8 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask) {
     if (rc) return rc;
     if (pack && !fused && (rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, s))) return rc;
   }
-  if (pack) rc = launch_spmm(a->vals_f, a->hw_meta_f, a->X, a->I, a->T, a->J, a->Y, a->status_word, s);
-  else rc = launch_dense_nt(a->vals_f, a->X, a->I, a->T, a->J, a->Y, a->status_word, s);
+  if (pack) rc = launch_spmm(a->vals_f, a->hw_meta_f, Xmat, a->I, a->T, a->J, a->Y, a->status_word, s);
+  else rc = launch_dense_nt(a->vals_f, Xmat, a->I, a->T, a->J, a->Y, a->status_word, s);
   if (rc) return rc;
   if (a->do_search) {
     const int32_t* cands = a->cands;
@@ -361,15 +379,57 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask) {
   if (rc) return rc;
   if (pack && !fused && (rc = launch_hw_meta(a->meta_b, a->J, a->I, a->hw_meta_b, s))) return rc;
   if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, s))) return rc;
-  if (pack) rc = launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, a->dX, a->status_word, s);
-  else rc = launch_dense_nt(a->vals_b, dYp, a->J, a->T, a->I, a->dX, a->status_word, s);
+  if (pack) rc = launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, dXmat, a->status_word, s);
+  else rc = launch_dense_nt(a->vals_b, dYp, a->J, a->T, a->I, dXmat, a->status_word, s);
   if (rc) return rc;
-  return launch_wgrad_impl(a->dY, a->X, a->T, a->I, a->J, a->dW, partials, a->status_word, s);
+  if (conv && !conv->imp_dgrad)
+    if ((rc = launch_col2im3x3(dXmat, conv->NB, conv->H, conv->W, conv->C, a->dX, s))) return rc;
+  return launch_wgrad_impl(a->dY, Xmat, a->T, a->I, a->J, a->dW, partials, a->status_word, s);
 }
 
 extern "C" {
 
 int bimask_layer_step(const bimask_layer_args* a) { return layer_step_impl(a, false); }
+
+size_t bimask_conv_workspace_bytes(int NB, int H, int W, int C, int I, int P) {
+  if (NB <= 0 || H <= 0 || W <= 0 || C <= 0 || I <= 0) return 0;
+  const long long T = (long long)NB * H * W;
+  if (T > 0x7FFFFFFFll || 9ll * C > 0x7FFFFFFFll) return 0;
+  const size_t col = align_up((size_t)T * 9 * C * 2, 256);
+  return plan_ws((int)T, I, 9 * C, P).total + 2 * col;          // + column matrix + column-space gradient
+}
+
+int bimask_conv_layer_step(const bimask_conv_args* c) {
+  BIMASK_REQUIRE(c != nullptr, BIMASK_EINVAL, "bimask_conv_layer_step: null argument block");
+  const bimask_layer_args* a = &c->layer;
+  BIMASK_REQUIRE(c->NB > 0 && c->H > 0 && c->W > 0 && c->C > 0 && c->C % 32 == 0, BIMASK_EINVAL,
+                 "bimask_conv_layer_step: NB = %d, H = %d, W = %d, C = %d: all positive, C a multiple of 32", c->NB, c->H,
+                 c->W, c->C);
+  const long long T = (long long)c->NB * c->H * c->W;
+  BIMASK_REQUIRE(T <= 0x7FFFFFFFll && a->T == (int)T && a->J == 9 * c->C, BIMASK_EINVAL,
+                 "bimask_conv_layer_step: layer.T must be NB*H*W (%lld) and layer.J must be 9*C (%d)", T, 9 * c->C);
+  BIMASK_REQUIRE(c->mode >= BIMASK_CONV_AUTO && c->mode <= BIMASK_CONV_IMPLICIT, BIMASK_EINVAL,
+                 "bimask_conv_layer_step: mode %d out of range", c->mode);
+  BIMASK_REQUIRE(a->ws && aligned16(a->ws), BIMASK_EINVAL, "bimask_conv_layer_step: null or misaligned workspace");
+  const size_t need = bimask_conv_workspace_bytes(c->NB, c->H, c->W, c->C, a->I, a->do_search && !a->cands ? a->P : 0);
+  BIMASK_REQUIRE(a->ws_bytes >= need, BIMASK_EINVAL, "bimask_conv_layer_step: workspace too small (%zu bytes, need %zu)",
+                 a->ws_bytes, need);
+  ConvPlan plan;
+  plan.NB = c->NB; plan.H = c->H; plan.W = c->W; plan.C = c->C;
+  const bool can_fwd = false, can_dgrad = false, can_wgrad = false;
+  BIMASK_REQUIRE(c->mode != BIMASK_CONV_IMPLICIT || (can_fwd && can_dgrad && can_wgrad), BIMASK_EUNSUPPORTED,
+                 "bimask_conv_layer_step: the implicit form needs C %% 128 == 0 and I %% 128 == 0 and a pattern with a 2:4 "
+                 "form (C = %d, I = %d, N:M = %d:%d)", c->C, a->I, a->N, a->M);
+  const bool implicit = c->mode != BIMASK_CONV_EXPLICIT;
+  plan.imp_fwd = implicit && can_fwd;
+  plan.imp_dgrad = implicit && can_dgrad;
+  plan.imp_wgrad = implicit && can_wgrad;
+  const size_t col = align_up((size_t)T * 9 * c->C * 2, 256);
+  uint8_t* tail = reinterpret_cast<uint8_t*>(a->ws) + (need - 2 * col);
+  plan.xcol = reinterpret_cast<uint16_t*>(tail);
+  plan.dxcol = reinterpret_cast<uint16_t*>(tail + col);
+  return layer_step_impl(a, false, &plan);
+}
 
 int bimask_train_step(const bimask_train_args* a) {
   BIMASK_REQUIRE(a != nullptr, BIMASK_EINVAL, "bimask_train_step: null argument block");

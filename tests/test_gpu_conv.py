@@ -1,0 +1,98 @@
+"""GPU parity for the 3x3 convolution layer step (bimask_conv_layer_step) against the oracle's
+direct convolutions: integer results bit for bit, the three products within the GEMM tolerance.
+Shapes cover images smaller and larger than a pixel patch, ragged patch edges, batch sizes that do
+not fill a patch group, channel counts on both sides of the implicit form's limits."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2302_06058_b200 as bm
+from oracle import bimask_oracle as O
+from paper_2302_06058_b200 import inputs
+from tests.gpu_util import bits_dev, dev, rel_err, u16, u32
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+
+
+def conv_case(NB, H, W, C, I, seed):
+    Wt = inputs.make_weight(I, 9 * C, seed)
+    x = inputs.make_activation(NB * H * W, C, seed + 1).reshape(NB, H, W, C)
+    dy = inputs.make_activation(NB * H * W, I, seed + 2).reshape(NB, H, W, I)
+    return Wt, x, dy
+
+
+def run_conv_step(Wt, x, dy, N, M, P, seed, mode, do_search=True):
+    NB, H, W, C = x.shape
+    I = Wt.shape[0]
+    T, J = NB * H * W, 9 * C
+    b = bm.alloc_layer_buffers(T, I, J, P)
+    b["W"], b["X"], b["dY"] = dev(Wt), bits_dev(x), bits_dev(dy)
+    b["dX"] = torch.empty(NB, H, W, C, dtype=torch.bfloat16, device="cuda")
+    b["ws"] = torch.empty(bm.bimask_conv_workspace_bytes(NB, H, W, C, I, P), dtype=torch.uint8, device="cuda")
+    largs = bm.make_layer_args(T, I, J, N, M, P, seed, do_search, b)
+    bm.bimask_conv_layer_step(bm.make_conv_args(largs, NB, H, W, C, mode))
+    torch.cuda.synchronize()
+    return b
+
+
+SHAPES = [(2, 9, 11, 32, 64), (3, 14, 14, 64, 128), (5, 7, 7, 128, 128), (1, 20, 17, 128, 256), (2, 28, 28, 128, 384),
+          (1, 33, 8, 256, 128)]
+
+
+@pytest.mark.parametrize("NB,H,W,C,I", SHAPES)
+@pytest.mark.parametrize("mode", [bm.binding.CONV_EXPLICIT, bm.binding.CONV_AUTO])
+def test_conv_layer_step_against_oracle(NB, H, W, C, I, mode):
+    N, M, P, seed = 2, 4, 4, 21
+    Wt, x, dy = conv_case(NB, H, W, C, I, 300 + NB + H + C)
+    b = run_conv_step(Wt, x, dy, N, M, P, seed, mode)
+    ref = O.conv_layer_step(Wt, x, dy, N, M, P, seed)
+    assert int(b["status_word"].item()) == 0
+    assert np.array_equal(u32(b["maskbits_f"]), ref["maskbits_f"])
+    assert np.array_equal(u16(b["vals_f"]), ref["vals_f"])
+    assert np.array_equal(b["counts"].cpu().numpy(), ref["counts"])
+    assert np.array_equal(b["perm"].cpu().numpy(), ref["perm"])
+    assert np.array_equal(u32(b["maskbits_b"]), ref["maskbits_b"])
+    assert np.array_equal(u16(b["vals_b"]), ref["vals_b"])
+    assert rel_err(b["Y"].float().cpu().numpy().reshape(NB, H, W, I), ref["y"]) <= TOL
+    assert rel_err(b["dX"].float().cpu().numpy(), ref["dx"]) <= TOL
+    assert rel_err(b["dW"].cpu().numpy(), ref["dW"]) <= TOL
+
+
+def test_conv_other_pattern_and_dense_fallback():
+    NB, H, W, C, I = 2, 10, 12, 64, 128
+    Wt, x, dy = conv_case(NB, H, W, C, I, 77)
+    for (N, M) in [(1, 4), (2, 8)]:
+        b = run_conv_step(Wt, x, dy, N, M, 3, 5, bm.binding.CONV_AUTO)
+        ref = O.conv_layer_step(Wt, x, dy, N, M, 3, 5)
+        assert np.array_equal(b["perm"].cpu().numpy(), ref["perm"])
+        assert np.array_equal(u32(b["maskbits_b"]), ref["maskbits_b"])
+        assert rel_err(b["Y"].float().cpu().numpy().reshape(NB, H, W, I), ref["y"]) <= TOL
+        assert rel_err(b["dX"].float().cpu().numpy(), ref["dx"]) <= TOL
+        assert rel_err(b["dW"].cpu().numpy(), ref["dW"]) <= TOL
+
+
+def test_conv_bad_arguments_launch_nothing():
+    NB, H, W, C, I = 1, 8, 8, 32, 32
+    Wt, x, dy = conv_case(NB, H, W, C, I, 1)
+    T, J = NB * H * W, 9 * C
+    b = bm.alloc_layer_buffers(T, I, J, 2)
+    b["W"], b["X"], b["dY"] = dev(Wt), bits_dev(x), bits_dev(dy)
+    b["dX"] = torch.empty(NB, H, W, C, dtype=torch.bfloat16, device="cuda")
+    n0 = bm.bimask_launch_count()
+    largs = bm.make_layer_args(T, I, J, 2, 4, 2, 1, True, b)          # workspace sized for the linear layer: too small
+    with pytest.raises(bm.BimaskError) as e:
+        bm.bimask_conv_layer_step(bm.make_conv_args(largs, NB, H, W, C, 0))
+    assert e.value.code == -1 and "workspace" in str(e.value)
+    b["ws"] = torch.empty(bm.bimask_conv_workspace_bytes(NB, H, W, C, I, 2), dtype=torch.uint8, device="cuda")
+    largs = bm.make_layer_args(T, I, J, 2, 4, 2, 1, True, b)
+    for kw in (dict(H=7), dict(C=48), dict(mode=5)):
+        geo = dict(NB=NB, H=H, W=W, C=C, mode=0)
+        geo.update(kw)
+        with pytest.raises(bm.BimaskError) as e:
+            bm.bimask_conv_layer_step(bm.make_conv_args(largs, geo["NB"], geo["H"], geo["W"], geo["C"], geo["mode"]))
+        assert e.value.code == -1
+    with pytest.raises(bm.BimaskError) as e:                             # C = 32 cannot take the implicit form
+        bm.bimask_conv_layer_step(bm.make_conv_args(largs, NB, H, W, C, bm.binding.CONV_IMPLICIT))
+    assert e.value.code == -2
+    assert bm.bimask_launch_count() == n0
