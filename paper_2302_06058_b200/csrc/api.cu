@@ -356,7 +356,9 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
     if (rc) return rc;
     if (pack && !fused && (rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, s))) return rc;
   }
-  if (pack) rc = launch_spmm(a->vals_f, a->hw_meta_f, Xmat, a->I, a->T, a->J, a->Y, a->status_word, s);
+  if (conv && conv->imp_fwd)
+    rc = launch_spmm_conv(1, a->vals_f, a->hw_meta_f, a->X, conv->NB, conv->H, conv->W, conv->C, a->I, a->Y, a->status_word, s);
+  else if (pack) rc = launch_spmm(a->vals_f, a->hw_meta_f, Xmat, a->I, a->T, a->J, a->Y, a->status_word, s);
   else rc = launch_dense_nt(a->vals_f, Xmat, a->I, a->T, a->J, a->Y, a->status_word, s);
   if (rc) return rc;
   if (a->do_search) {
@@ -379,7 +381,9 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
   if (rc) return rc;
   if (pack && !fused && (rc = launch_hw_meta(a->meta_b, a->J, a->I, a->hw_meta_b, s))) return rc;
   if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, s))) return rc;
-  if (pack) rc = launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, dXmat, a->status_word, s);
+  if (conv && conv->imp_dgrad)
+    rc = launch_spmm_conv(2, a->vals_b, a->hw_meta_b, dYp, conv->NB, conv->H, conv->W, conv->C, a->I, a->dX, a->status_word, s);
+  else if (pack) rc = launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, dXmat, a->status_word, s);
   else rc = launch_dense_nt(a->vals_b, dYp, a->J, a->T, a->I, dXmat, a->status_word, s);
   if (rc) return rc;
   if (conv && !conv->imp_dgrad)
@@ -416,8 +420,11 @@ int bimask_conv_layer_step(const bimask_conv_args* c) {
                  a->ws_bytes, need);
   ConvPlan plan;
   plan.NB = c->NB; plan.H = c->H; plan.W = c->W; plan.C = c->C;
-  const bool can_fwd = false, can_dgrad = false, can_wgrad = false;
-  BIMASK_REQUIRE(c->mode != BIMASK_CONV_IMPLICIT || (can_fwd && can_dgrad && can_wgrad), BIMASK_EUNSUPPORTED,
+  const bool packs = a->N <= 2;
+  const bool can_fwd = packs && c->C % 64 == 0;
+  const bool can_dgrad = packs && c->C % 128 == 0 && a->I % 128 == 0;
+  const bool can_wgrad = false;
+  BIMASK_REQUIRE(c->mode != BIMASK_CONV_IMPLICIT || (can_fwd && can_dgrad), BIMASK_EUNSUPPORTED,
                  "bimask_conv_layer_step: the implicit form needs C %% 128 == 0 and I %% 128 == 0 and a pattern with a 2:4 "
                  "form (C = %d, I = %d, N:M = %d:%d)", c->C, a->I, a->N, a->M);
   const bool implicit = c->mode != BIMASK_CONV_EXPLICIT;

@@ -39,7 +39,51 @@ struct Cfg {
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 };
 
+// A 3x3 convolution as an implicit GEMM: the token operand is an NHWC tensor and a "tile of
+// tokens" is a box of wb x hb pixels of nb images, fetched with one 4-D tensor load per 64
+// channels, shifted by the filter tap the k index belongs to (pixels outside the image read 0).
+//   mode 1 (forward, Eq. 3):        k = (tap, c);  B = x,   shift (+kw-1, +kh-1)
+//   mode 2 (input gradient, Eq. 10): k = (tap, i');  B = dy[:, perm], shift (1-kw, 1-kh); the rows of
+//           the 2:4 operand for tap (kh, kw) are (kh*3+kw)*C + c.
+struct ConvGeom {
+  int mode;                 // 0: plain matrix operand
+  int H, W, NB;             // image
+  int CB;                   // channels of the token operand (x: C; dy: I)
+  int wb, hb, nb;           // pixel box of one load: wb * hb * nb tokens (powers of two)
+  int lg_wb, lg_hb;         // their logarithms
+  int tiles_w, tiles_h;     // boxes per image
+  int kt_per_tap;           // mode 2: 128-wide k tiles per filter tap (I / 128)
+  int rows_per_tap;         // mode 2: rows of the 2:4 operand per tap (C)
+};
+
+__device__ __forceinline__ void conv_box_origin(const ConvGeom& g, int box, int& w0, int& h0, int& n0) {
+  w0 = (box % g.tiles_w) * g.wb;
+  const int r = box / g.tiles_w;
+  h0 = (r % g.tiles_h) * g.hb;
+  n0 = (r / g.tiles_h) * g.nb;
+}
+
+// Channel offset and pixel shift of the 64-wide half q of k tile kt; valid = false: past the
+// reduction length (the loader then reads a box of zeros).
+__device__ __forceinline__ void conv_k_coords(const ConvGeom& g, int kt, int q, int Kdim, int& c0, int& dw, int& dh, bool& valid) {
+  if (g.mode == 1) {
+    const int j = kt * 128 + 64 * q;
+    valid = j < Kdim;
+    const int tap = j / g.CB;
+    c0 = j - tap * g.CB;
+    dh = tap / 3 - 1;
+    dw = tap % 3 - 1;
+  } else {
+    const int tap = kt / g.kt_per_tap;
+    c0 = (kt - tap * g.kt_per_tap) * 128 + 64 * q;
+    valid = true;
+    dh = 1 - tap / 3;
+    dw = 1 - tap % 3;
+  }
+}
+
 struct GemmParams {
+  ConvGeom conv;
   const uint8_t* hw_meta;   // sparse only
   int tiles_k_meta;         // number of 128-wide k tiles in the metadata image
   int Mdim, Ndim, Kdim;     // D is Mdim x Ndim, reduction length Kdim (logical)
@@ -67,7 +111,8 @@ __device__ __forceinline__ void raster(int id, int tiles_m, int tiles_n, int gro
 
 // SPARSE = false: the same pipeline on a dense bf16 A operand (masked weights of a pattern the
 // 2:4 format cannot hold): 128 x 128 A tile per stage as two 64-wide boxes, eight K = 16 MMAs.
-template <int N_TILE, int STAGES, bool SPARSE>
+// CONV: the token operand is fetched as shifted pixel boxes (see ConvGeom); N_TILE tokens = one box.
+template <int N_TILE, int STAGES, bool SPARSE, bool CONV>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                    const GemmParams p) {
@@ -89,6 +134,8 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
   const int m0 = tile_m * C::M_TILE;
   const int n0 = tile_n * N_TILE;
   const int k_tiles_total = (p.Kdim + C::K_TILE - 1) / C::K_TILE;
+  int cw0 = 0, ch0 = 0, cn0 = 0;                       // CONV: origin of this tile's pixel box
+  if (CONV) conv_box_origin(p.conv, tile_n, cw0, ch0, cn0);
   const int kt_begin = blockIdx.z * p.k_tiles_per_split;
   const int kt_end = min(k_tiles_total, kt_begin + p.k_tiles_per_split);
   const int num_kt = kt_end - kt_begin;
@@ -125,6 +172,28 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
         const uint32_t a_s = base + s * C::STAGE_BYTES;
         const uint32_t b_s = a_s + C::A_BYTES;
         ptx::mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
+        if (SPARSE && CONV) {
+          int a_col = kt * 64, a_row = m0, meta_row = tile_m, meta_kt = kt;
+          if (p.conv.mode == 2) {
+            const int tap = kt / p.conv.kt_per_tap;
+            meta_kt = kt - tap * p.conv.kt_per_tap;
+            a_col = meta_kt * 64;
+            a_row = tap * p.conv.rows_per_tap + m0;
+            meta_row = a_row >> 7;
+          }
+          ptx::tma_load_2d(a_s, &tmapA, a_col, a_row, full_bar(s));
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            int c0, dw, dh;
+            bool valid;
+            conv_k_coords(p.conv, kt, q, p.Kdim, c0, dw, dh, valid);
+            ptx::tma_load_4d(b_s + q * (N_TILE * 128), &tmapB, valid ? c0 : 0, cw0 + dw, ch0 + dh, valid ? cn0 : p.conv.NB,
+                             full_bar(s));
+          }
+          ptx::bulk_load(b_s + C::B_BYTES,
+                         p.hw_meta + ((size_t)meta_row * p.tiles_k_meta + meta_kt) * 2048, 2048, full_bar(s));
+          continue;
+        }
         if (SPARSE) {
           ptx::tma_load_2d(a_s, &tmapA, kt * 64, m0, full_bar(s));                    // 64 compressed x 128 rows
         } else {
@@ -191,7 +260,20 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
         }
         const int nb = n0 + 32 * c;
         __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
-        if (m < p.Mdim) {
+        if (CONV) {
+          // token 32c + j of the box is pixel (cn0 + r / (wb*hb), ch0 + (r / wb) % hb, cw0 + r % wb)
+          if (m < p.Mdim) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int rr = 32 * c + j;
+              const int w = cw0 + (rr & (p.conv.wb - 1));
+              const int h = ch0 + ((rr >> p.conv.lg_wb) & (p.conv.hb - 1));
+              const int n = cn0 + (rr >> (p.conv.lg_wb + p.conv.lg_hb));
+              if (w < p.conv.W && h < p.conv.H && n < p.conv.NB)
+                out[(((size_t)n * p.conv.H + h) * p.conv.W + w) * p.Mdim + m] = __float2bfloat16_rn(__uint_as_float(r[j]));
+            }
+          }
+        } else if (m < p.Mdim) {
 #pragma unroll
           for (int j = 0; j < 32; ++j)
             if (nb + j < p.Ndim) out[(size_t)(nb + j) * p.Mdim + m] = __float2bfloat16_rn(__uint_as_float(r[j]));
@@ -225,10 +307,12 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
 // One epilogue chunk of the 2:4 product for one warp: W accumulator columns of its 32 rows go
 // tensor memory -> registers -> bf16 -> staging[token][row] -> one TMA store of a 32 x W box.
 // `last` releases the accumulator (after its final read) to the MMA thread of the pair's leader.
+// cw >= 0: convolution output, the W tokens are pixels (cw.., ch..) of image cn (a 4-D store).
 template <int W>
 __device__ __forceinline__ void sparse_epilogue_chunk(uint32_t taddr, bool last, uint32_t release_bar,
                                                       uint16_t* stg_ptr, uint32_t stg_base, uint32_t chunk, int lane,
-                                                      const CUtensorMap* tmap, int m0, int n, int Mdim, int Ndim) {
+                                                      const CUtensorMap* tmap, int m0, int n, int Mdim, int Ndim,
+                                                      int cw = -1, int ch = 0, int cn = 0, bool cvalid = false) {
   uint32_t r[W];
   if (W == 32) ptx::tmem_ld_32x32(taddr, reinterpret_cast<uint32_t (&)[32]>(r));
   else ptx::tmem_ld_32x16(taddr, reinterpret_cast<uint32_t (&)[16]>(r));
@@ -251,7 +335,11 @@ __device__ __forceinline__ void sparse_epilogue_chunk(uint32_t taddr, bool last,
   ptx::fence_proxy_async();
   __syncwarp();
   if (lane == 0) {
-    if (m0 < Mdim && n < Ndim) ptx::tma_store_2d(tmap, m0, n, stg_base + (chunk & 1u) * 2048);
+    if (cw >= 0) {
+      if (m0 < Mdim && cvalid) ptx::tma_store_4d(tmap, m0, cw, ch, cn, stg_base + (chunk & 1u) * 2048);
+    } else if (m0 < Mdim && n < Ndim) {
+      ptx::tma_store_2d(tmap, m0, n, stg_base + (chunk & 1u) * 2048);
+    }
     ptx::tma_store_commit();
   }
 }
@@ -267,7 +355,7 @@ struct PairPCfg {
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 + 256;
 };
 
-template <int STAGES>
+template <int STAGES, bool CONV>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                             const __grid_constant__ CUtensorMap tmapE, const __grid_constant__ CUtensorMap tmapOut32,
@@ -342,6 +430,29 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
           const uint32_t b_s = a_s + C::A_BYTES;
           const uint32_t bar = ptx::mapa(full_bar(s), 0);
           if (rank == 0) ptx::mbar_expect_tx(full_bar(s), 2 * stage_tx);
+          if (CONV) {
+            // this CTA's SP_N / 2 tokens are pixel box 2 * tile_n + rank
+            int cw0, ch0, cn0;
+            conv_box_origin(p.conv, 2 * tile_n + (int)rank, cw0, ch0, cn0);
+            int a_col = kt * 64, a_row = m0, meta_row = mt128, meta_kt = kt;
+            if (p.conv.mode == 2) {
+              const int tap = kt / p.conv.kt_per_tap;
+              meta_kt = kt - tap * p.conv.kt_per_tap;
+              a_col = meta_kt * 64;
+              a_row = tap * p.conv.rows_per_tap + m0;
+              meta_row = a_row >> 7;
+            }
+            ptx::tma_load_2d_pair(a_s, &tmapA, a_col, a_row, bar);
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              int c0, dw, dh;
+              bool valid;
+              conv_k_coords(p.conv, kt, q, p.Kdim, c0, dw, dh, valid);
+              ptx::tma_load_4d_pair(b_s + q * b_box, &tmapB, valid ? c0 : 0, cw0 + dw, ch0 + dh, valid ? cn0 : p.conv.NB, bar);
+            }
+            ptx::tma_load_2d_pair(b_s + C::B_MAX, &tmapE, 0, 2 * (meta_row * p.tiles_k_meta + meta_kt), bar);
+            continue;
+          }
           ptx::tma_load_2d_pair(a_s, &tmapA, kt * 64, m0, bar);
           ptx::tma_load_2d_pair(b_s, &tmapB, kt * 128, nrow, bar);
           ptx::tma_load_2d_pair(b_s + b_box, &tmapB, kt * 128 + 64, nrow, bar);
@@ -396,7 +507,22 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
       ptx::tc_fence_after();
       const uint32_t acc = tmem_base + 256u * buf + ((uint32_t)(32 * q) << 16);
       const uint32_t release_bar = ptx::mapa(tmem_empty_bar(buf), 0);
-      if ((SP_N & 31) == 0) {
+      if (CONV) {
+        // accumulator columns [0, SP_N/2) are the pixels of box 2*tile_n, the rest those of box 2*tile_n + 1;
+        // a chunk of 32 tokens is 32 / wb consecutive rows of one image of the box
+#pragma unroll 1
+        for (int c = 0; c < SP_N / 32; ++c, ++chunk) {
+          const int half = (32 * c) / (SP_N / 2);
+          const int rr = 32 * c - half * (SP_N / 2);
+          int cw0, ch0, cn0;
+          conv_box_origin(p.conv, 2 * tile_n + half, cw0, ch0, cn0);
+          const int h = ch0 + ((rr >> p.conv.lg_wb) & (p.conv.hb - 1));
+          const int n = cn0 + (rr >> (p.conv.lg_wb + p.conv.lg_hb));
+          sparse_epilogue_chunk<32>(acc + 32 * c, c == SP_N / 32 - 1, release_bar, stg_ptr, stg_base, chunk, lane,
+                                    &tmapOut32, m0, 0, p.Mdim, p.Ndim, cw0, h, n,
+                                    cw0 < p.conv.W && h < p.conv.H && n < p.conv.NB);
+        }
+      } else if ((SP_N & 31) == 0) {
 #pragma unroll 1
         for (int c = 0; c < SP_N / 32; ++c, ++chunk)
           sparse_epilogue_chunk<32>(acc + 32 * c, c == SP_N / 32 - 1, release_bar, stg_ptr, stg_base, chunk, lane,
@@ -749,9 +875,14 @@ struct TmapKey {
   uint64_t inner, outer, stride;
   uint32_t box_inner, box_outer;
   int dtype, swizzle;
+  // rank 4 (NHWC activations: inner = channels, outer = W) when d2 != 0: extents H = d2, NB = d3,
+  // densely packed (stride of H = W * stride, of NB = H * W * stride)
+  uint64_t d2 = 0, d3 = 0;
+  uint32_t box2 = 0, box3 = 0;
   bool operator==(const TmapKey& o) const {
     return ptr == o.ptr && inner == o.inner && outer == o.outer && stride == o.stride && box_inner == o.box_inner &&
-           box_outer == o.box_outer && dtype == o.dtype && swizzle == o.swizzle;
+           box_outer == o.box_outer && dtype == o.dtype && swizzle == o.swizzle && d2 == o.d2 && d3 == o.d3 &&
+           box2 == o.box2 && box3 == o.box3;
   }
 };
 
@@ -765,11 +896,11 @@ int encode_cached(CUtensorMap* m, const TmapKey& key) {
     if (used[i] && keys[i] == key) { *m = maps[i]; return BIMASK_OK; }
   EncodeTiledFn fn = get_encode_fn();
   BIMASK_REQUIRE(fn != nullptr, BIMASK_ECUDA, "cuTensorMapEncodeTiled entry point not available");
-  cuuint64_t dims[2] = {key.inner, key.outer};
-  cuuint64_t strides[1] = {key.stride};
-  cuuint32_t box[2] = {key.box_inner, key.box_outer};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(m, (CUtensorMapDataType)key.dtype, 2, const_cast<void*>(key.ptr), dims, strides, box, estr,
+  cuuint64_t dims[4] = {key.inner, key.outer, key.d2, key.d3};
+  cuuint64_t strides[3] = {key.stride, key.stride * key.outer, key.stride * key.outer * key.d2};
+  cuuint32_t box[4] = {key.box_inner, key.box_outer, key.box2, key.box3};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(m, (CUtensorMapDataType)key.dtype, key.d2 ? 4 : 2, const_cast<void*>(key.ptr), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, (CUtensorMapSwizzle)key.swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   BIMASK_REQUIRE(r == CUDA_SUCCESS, BIMASK_ECUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
@@ -808,6 +939,22 @@ int make_tmap_out(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t rows
                                   (int)CU_TENSOR_MAP_SWIZZLE_NONE});
 }
 
+// 4-D bf16 map of an NHWC tensor (channels, W, H, NB) for loads of 64-channel pixel boxes, 128-byte swizzle.
+int make_tmap_nhwc_load(CUtensorMap* m, const void* ptr, int CH, int W, int H, int NB, int wb, int hb, int nb) {
+  TmapKey k{ptr, (uint64_t)CH, (uint64_t)W, (uint64_t)CH * 2, 64, (uint32_t)wb, (int)CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+            (int)CU_TENSOR_MAP_SWIZZLE_128B};
+  k.d2 = (uint64_t)H; k.d3 = (uint64_t)NB; k.box2 = (uint32_t)hb; k.box3 = (uint32_t)nb;
+  return encode_cached(m, k);
+}
+
+// The same tensor for stores of (32 channels, wb, 32 / wb, 1) boxes, no swizzle.
+int make_tmap_nhwc_store(CUtensorMap* m, const void* ptr, int CH, int W, int H, int NB, int wb) {
+  TmapKey k{ptr, (uint64_t)CH, (uint64_t)W, (uint64_t)CH * 2, 32, (uint32_t)wb, (int)CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+            (int)CU_TENSOR_MAP_SWIZZLE_NONE};
+  k.d2 = (uint64_t)H; k.d3 = (uint64_t)NB; k.box2 = (uint32_t)(32 / wb); k.box3 = 1;
+  return encode_cached(m, k);
+}
+
 }  // namespace
 
 // Generic 2-D tensor map without swizzle: `inner` contiguous elements of `elem_bytes` per row.
@@ -833,9 +980,10 @@ int run_sparse(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, i
   int rc;
   if ((rc = make_tmap(&ta, vals, SPARSE ? (uint64_t)Kdim / 2 : (uint64_t)Kdim, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, N_TILE)) != BIMASK_OK) return rc;
-  auto kern = spmm_single_kernel<N_TILE, STAGES, SPARSE>;
+  auto kern = spmm_single_kernel<N_TILE, STAGES, SPARSE, false>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
+  p.conv.mode = 0;
   p.hw_meta = reinterpret_cast<const uint8_t*>(hw_meta);
   p.tiles_k_meta = (Kdim + 127) / 128;
   p.Mdim = Mdim; p.Ndim = Ndim; p.Kdim = Kdim;
@@ -887,9 +1035,10 @@ int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const 
   if ((rc = make_tmap_meta(&te, hw_meta, (uint64_t)tiles_m * tiles_k)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_out(&to32, out, (uint64_t)Mdim, (uint64_t)Ndim, 32)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_out(&to16, out, (uint64_t)Mdim, (uint64_t)Ndim, 16)) != BIMASK_OK) return rc;
-  auto kern = spmm_pair_persistent_kernel<STAGES>;
+  auto kern = spmm_pair_persistent_kernel<STAGES, false>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
+  p.conv.mode = 0;
   p.hw_meta = reinterpret_cast<const uint8_t*>(hw_meta);
   p.tiles_k_meta = tiles_k;
   p.Mdim = Mdim; p.Ndim = Ndim; p.Kdim = Kdim;
@@ -915,6 +1064,119 @@ int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, 
   if (Ndim > 128 && Mdim > 128) return run_sparse_pair_persistent(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   if (Ndim > 128) return run_sparse<256, 2>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   return run_sparse<128, 4>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
+}
+
+namespace {
+
+int pow2_ceil(int v) { int p = 1; while (p < v) p <<= 1; return p; }
+int log2_exact(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
+
+// Pixel boxes of `tokens` tokens: as wide as the image allows (16 or 8), at least 32 tokens per image of the box.
+void conv_boxes(ConvGeom& g, int tokens) {
+  g.wb = g.W > 8 ? 16 : 8;
+  int hb = tokens / g.wb;
+  const int hp = pow2_ceil(g.H);
+  if (hb > hp) hb = hp;
+  if (hb < 32 / g.wb) hb = 32 / g.wb;
+  g.hb = hb;
+  g.nb = tokens / (g.wb * g.hb);
+  g.lg_wb = log2_exact(g.wb);
+  g.lg_hb = log2_exact(g.hb);
+  g.tiles_w = (g.W + g.wb - 1) / g.wb;
+  g.tiles_h = (g.H + g.hb - 1) / g.hb;
+}
+
+template <int N_TILE, int STAGES>
+int run_conv_single(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_meta, const uint16_t* tok, ConvGeom g,
+                    int Mdim, int Kdim, int tiles_k_meta, uint16_t* out, int32_t* status_word, cudaStream_t s) {
+  using C = Cfg<N_TILE, STAGES, true>;
+  conv_boxes(g, N_TILE);
+  CUtensorMap ta, tb;
+  int rc;
+  if ((rc = make_tmap(&ta, vals, (uint64_t)a_kdim / 2, (uint64_t)a_rows, 128)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_nhwc_load(&tb, tok, g.CB, g.W, g.H, g.NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
+  auto kern = spmm_single_kernel<N_TILE, STAGES, true, true>;
+  if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
+  GemmParams p;
+  p.conv = g;
+  p.hw_meta = reinterpret_cast<const uint8_t*>(hw_meta);
+  p.tiles_k_meta = tiles_k_meta;
+  p.Mdim = Mdim; p.Ndim = g.NB * g.H * g.W; p.Kdim = Kdim;
+  p.k_tiles_per_split = (Kdim + 127) / 128;
+  p.out = out;
+  p.status_word = status_word;
+  p.tiles_m = (Mdim + 127) / 128;
+  p.tiles_n = g.tiles_w * g.tiles_h * ((g.NB + g.nb - 1) / g.nb);
+  p.raster_group = 16;
+  p.n_tile = N_TILE;
+  dim3 grid(p.tiles_m * p.tiles_n, 1, 1);
+  kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p);
+  count_launch();
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
+int run_conv_pair(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_meta, const uint16_t* tok, ConvGeom g,
+                  int Mdim, int Kdim, int tiles_k_meta, uint16_t* out, int32_t* status_word, cudaStream_t s) {
+  constexpr int STAGES = 4;
+  using C = PairPCfg<STAGES>;
+  const int n_tile = 128;                                // two boxes of 64 pixels; two accumulators in tensor memory
+  conv_boxes(g, n_tile / 2);
+  CUtensorMap ta, tb, te, to32;
+  int rc;
+  const int a_tiles_m = (a_rows + 127) / 128;
+  const int sms = sm_count();
+  if ((rc = make_tmap(&ta, vals, (uint64_t)a_kdim / 2, (uint64_t)a_rows, 128)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_nhwc_load(&tb, tok, g.CB, g.W, g.H, g.NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_meta(&te, hw_meta, (uint64_t)a_tiles_m * tiles_k_meta)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_nhwc_store(&to32, out, Mdim, g.W, g.H, g.NB, g.wb)) != BIMASK_OK) return rc;
+  auto kern = spmm_pair_persistent_kernel<STAGES, true>;
+  if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
+  GemmParams p;
+  p.conv = g;
+  p.hw_meta = reinterpret_cast<const uint8_t*>(hw_meta);
+  p.tiles_k_meta = tiles_k_meta;
+  p.Mdim = Mdim; p.Ndim = g.NB * g.H * g.W; p.Kdim = Kdim;
+  p.k_tiles_per_split = (Kdim + 127) / 128;
+  p.out = out;
+  p.status_word = status_word;
+  p.n_tile = n_tile;
+  p.tiles_m = ((Mdim + 127) / 128 + 1) / 2;
+  const int boxes = g.tiles_w * g.tiles_h * ((g.NB + g.nb - 1) / g.nb);
+  p.tiles_n = (boxes + 1) / 2;
+  p.raster_group = 8;
+  const int total = p.tiles_m * p.tiles_n;
+  const int clusters = total < sms / 2 ? total : sms / 2;
+  kern<<<2 * clusters, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, to32, to32, p);
+  count_launch();
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
+}  // namespace
+
+// 3x3 convolution products without a column matrix (see ConvGeom).
+//   forward:        D[i, pixel] = sum_{tap, c} A_f[i, tap*C + c] x[pixel + tap, c];  vals/hw_meta of the I x 9C operand
+//   input gradient: D[c, pixel] = sum_{tap, i'} A'[tap*C + c, i'] dyp[pixel - tap, i'];  vals/hw_meta of the 9C x I operand
+// out is NHWC with Mdim channels.  Needs C % 64 == 0 (forward) or C % 128 == 0 and I % 128 == 0 (input gradient).
+int launch_spmm_conv(int mode, const uint16_t* vals, const void* hw_meta, const uint16_t* tok, int NB, int H, int W, int C,
+                     int I, uint16_t* out, int32_t* status_word, cudaStream_t s) {
+  ConvGeom g{};
+  g.mode = mode; g.H = H; g.W = W; g.NB = NB;
+  const long long T = (long long)NB * H * W;
+  int Mdim, Kdim, a_rows, a_kdim, tiles_k_meta;
+  if (mode == 1) {
+    g.CB = C; g.kt_per_tap = 0; g.rows_per_tap = 0;
+    Mdim = I; Kdim = 9 * C; a_rows = I; a_kdim = 9 * C; tiles_k_meta = (9 * C + 127) / 128;
+  } else {
+    g.CB = I; g.kt_per_tap = I / 128; g.rows_per_tap = C;
+    Mdim = C; Kdim = 9 * I; a_rows = 9 * C; a_kdim = I; tiles_k_meta = I / 128;
+  }
+  if (Mdim > 128 && T > 128)
+    return run_conv_pair(vals, a_rows, a_kdim, hw_meta, tok, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
+  if (T > 128)
+    return run_conv_single<256, 2>(vals, a_rows, a_kdim, hw_meta, tok, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
+  return run_conv_single<128, 4>(vals, a_rows, a_kdim, hw_meta, tok, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
 }
 
 int launch_dense_nt(const uint16_t* A, const uint16_t* Bop, int Mdim, int Ndim, int Kdim, uint16_t* out,
@@ -990,6 +1252,7 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
   auto kern = wgrad_pair_kernel<STAGES>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
+  p.conv.mode = 0;
   p.hw_meta = nullptr; p.tiles_k_meta = 0;
   p.Mdim = I; p.Ndim = J; p.Kdim = T;
   p.k_tiles_per_split = per;
