@@ -293,6 +293,7 @@ struct ConvPlan {
   bool imp_fwd, imp_dgrad, imp_wgrad;
   uint16_t* xcol;     // T x 9C, when the forward or weight-gradient product is explicit
   uint16_t* dxcol;    // T x 9C, when the input gradient is explicit
+  float* wpart;       // split-K partial sums of the implicit weight gradient
 };
 
 // skip_fwd_mask: the forward mask / operand of the current W is already in place.
@@ -388,6 +389,8 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
   if (rc) return rc;
   if (conv && !conv->imp_dgrad)
     if ((rc = launch_col2im3x3(dXmat, conv->NB, conv->H, conv->W, conv->C, a->dX, s))) return rc;
+  if (conv && conv->imp_wgrad)
+    return launch_wgrad_conv(a->dY, a->X, conv->NB, conv->H, conv->W, conv->C, a->I, a->dW, conv->wpart, a->status_word, s);
   return launch_wgrad_impl(a->dY, Xmat, a->T, a->I, a->J, a->dW, partials, a->status_word, s);
 }
 
@@ -395,12 +398,19 @@ extern "C" {
 
 int bimask_layer_step(const bimask_layer_args* a) { return layer_step_impl(a, false); }
 
+static size_t conv_wpart_bytes(int NB, int H, int W, int C, int I) {
+  int splits = 1, per = 0;
+  wgrad_conv_plan(NB, H, W, C, I, &splits, &per);
+  return splits > 1 ? align_up((size_t)splits * I * 9 * C * sizeof(float), 256) : 0;
+}
+
 size_t bimask_conv_workspace_bytes(int NB, int H, int W, int C, int I, int P) {
   if (NB <= 0 || H <= 0 || W <= 0 || C <= 0 || I <= 0) return 0;
   const long long T = (long long)NB * H * W;
   if (T > 0x7FFFFFFFll || 9ll * C > 0x7FFFFFFFll) return 0;
   const size_t col = align_up((size_t)T * 9 * C * 2, 256);
-  return plan_ws((int)T, I, 9 * C, P).total + 2 * col;          // + column matrix + column-space gradient
+  // linear-layer scratch + column matrix + column-space gradient + partial sums of the implicit weight gradient
+  return plan_ws((int)T, I, 9 * C, P).total + 2 * col + conv_wpart_bytes(NB, H, W, C, I);
 }
 
 int bimask_conv_layer_step(const bimask_conv_args* c) {
@@ -423,8 +433,8 @@ int bimask_conv_layer_step(const bimask_conv_args* c) {
   const bool packs = a->N <= 2;
   const bool can_fwd = packs && c->C % 64 == 0;
   const bool can_dgrad = packs && c->C % 128 == 0 && a->I % 128 == 0;
-  const bool can_wgrad = false;
-  BIMASK_REQUIRE(c->mode != BIMASK_CONV_IMPLICIT || (can_fwd && can_dgrad), BIMASK_EUNSUPPORTED,
+  const bool can_wgrad = c->C % 64 == 0;
+  BIMASK_REQUIRE(c->mode != BIMASK_CONV_IMPLICIT || (can_fwd && can_dgrad && can_wgrad), BIMASK_EUNSUPPORTED,
                  "bimask_conv_layer_step: the implicit form needs C %% 128 == 0 and I %% 128 == 0 and a pattern with a 2:4 "
                  "form (C = %d, I = %d, N:M = %d:%d)", c->C, a->I, a->N, a->M);
   const bool implicit = c->mode != BIMASK_CONV_EXPLICIT;
@@ -432,9 +442,11 @@ int bimask_conv_layer_step(const bimask_conv_args* c) {
   plan.imp_dgrad = implicit && can_dgrad;
   plan.imp_wgrad = implicit && can_wgrad;
   const size_t col = align_up((size_t)T * 9 * c->C * 2, 256);
-  uint8_t* tail = reinterpret_cast<uint8_t*>(a->ws) + (need - 2 * col);
+  const size_t wpart = conv_wpart_bytes(c->NB, c->H, c->W, c->C, a->I);
+  uint8_t* tail = reinterpret_cast<uint8_t*>(a->ws) + (need - 2 * col - wpart);
   plan.xcol = reinterpret_cast<uint16_t*>(tail);
   plan.dxcol = reinterpret_cast<uint16_t*>(tail + col);
+  plan.wpart = reinterpret_cast<float*>(tail + 2 * col);
   return layer_step_impl(a, false, &plan);
 }
 

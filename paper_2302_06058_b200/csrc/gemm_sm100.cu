@@ -564,7 +564,9 @@ struct WgradCfg {
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
 };
 
-template <int STAGES>
+// CONV: k tile kt is pixel box kt (64 pixels) of the NHWC tensors; the dy operand is that box, the
+// x operand the same box shifted by the filter tap its 64 columns of dW belong to.
+template <int STAGES, bool CONV>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                   const GemmParams p, int splits) {
@@ -639,6 +641,21 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_consta
           const uint32_t b_s = a_s + C::A_BYTES;
           const uint32_t bar = ptx::mapa(full_bar(s), 0);
           if (rank == 0) ptx::mbar_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
+          if (CONV) {
+            int cw0, ch0, cn0;
+            conv_box_origin(p.conv, kt, cw0, ch0, cn0);
+            ptx::tma_load_4d_pair(a_s, &tmapA, m0, cw0, ch0, cn0, bar);
+            ptx::tma_load_4d_pair(a_s + 8192, &tmapA, m0 + 64, cw0, ch0, cn0, bar);
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              const int j = n0 + 128 * (int)rank + 64 * q;           // first of 64 columns of dW: one tap, 64 channels
+              const bool valid = j < p.Ndim;
+              const int tap = j / p.conv.CB;
+              ptx::tma_load_4d_pair(b_s + q * 8192, &tmapB, valid ? j - tap * p.conv.CB : 0, cw0 + tap % 3 - 1,
+                                    ch0 + tap / 3 - 1, valid ? cn0 : p.conv.NB, bar);
+            }
+            continue;
+          }
           ptx::tma_load_2d_pair(a_s, &tmapA, m0, kt * 64, bar);
           ptx::tma_load_2d_pair(a_s + 8192, &tmapA, m0 + 64, kt * 64, bar);
           ptx::tma_load_2d_pair(b_s, &tmapB, n0 + 128 * (int)rank, kt * 64, bar);
@@ -1222,6 +1239,79 @@ int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, u
   return BIMASK_OK;
 }
 
+// Split-K plan of the dense product for a reduction of k_tiles 64-deep tiles.
+static void wgrad_plan_k(int k_tiles, int I, int J, int* splits, int* k_tiles_per_split) {
+  const int tiles = (((I + 127) / 128 + 1) / 2) * ((J + 255) / 256);     // 256 x 256 pair tiles
+  int sp = 1;
+  if (tiles < 74) {
+    sp = (2 * 74 + tiles - 1) / tiles;
+    const int max_by_k = k_tiles / 8 > 0 ? k_tiles / 8 : 1;        // at least 8 k tiles per split
+    if (sp > max_by_k) sp = max_by_k;
+    if (sp > 64) sp = 64;
+  }
+  int per = (k_tiles + sp - 1) / sp;
+  sp = (k_tiles + per - 1) / per;
+  *splits = sp; *k_tiles_per_split = per;
+}
+
+// The same for the implicit convolution: one k tile per 64-pixel box.
+static ConvGeom conv_wgrad_geom(int NB, int H, int W, int C) {
+  ConvGeom g{};
+  g.mode = 1; g.H = H; g.W = W; g.NB = NB; g.CB = C;
+  conv_boxes(g, 64);
+  return g;
+}
+
+void wgrad_conv_plan(int NB, int H, int W, int C, int I, int* splits, int* k_tiles_per_split) {
+  const ConvGeom g = conv_wgrad_geom(NB, H, W, C);
+  wgrad_plan_k(g.tiles_w * g.tiles_h * ((NB + g.nb - 1) / g.nb), I, 9 * C, splits, k_tiles_per_split);
+}
+
+// dW[i, tap*C + c] = sum over pixels of dy[pixel, i] x[pixel + tap, c] without a column matrix (C % 64 == 0).
+// partials: splits * I * 9C floats when wgrad_conv_plan gives more than one split.
+int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int W, int C, int I, float* dW, float* partials,
+                      int32_t* status_word, cudaStream_t s) {
+  const ConvGeom g = conv_wgrad_geom(NB, H, W, C);
+  const int boxes = g.tiles_w * g.tiles_h * ((NB + g.nb - 1) / g.nb);
+  const int J = 9 * C;
+  int splits, per;
+  wgrad_plan_k(boxes, I, J, &splits, &per);
+  constexpr int STAGES = 6;
+  using Cf = WgradCfg<STAGES>;
+  CUtensorMap ta, tb;
+  int rc;
+  if ((rc = make_tmap_nhwc_load(&ta, dy, I, W, H, NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_nhwc_load(&tb, x, C, W, H, NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
+  auto kern = wgrad_pair_kernel<STAGES, true>;
+  if ((rc = set_smem_attr(kern, Cf::SMEM_BYTES)) != BIMASK_OK) return rc;
+  GemmParams p;
+  p.conv = g;
+  p.hw_meta = nullptr; p.tiles_k_meta = 0;
+  p.Mdim = I; p.Ndim = J; p.Kdim = boxes * 64;
+  p.k_tiles_per_split = per;
+  p.out = splits > 1 ? partials : dW;
+  p.status_word = status_word;
+  p.tiles_m = ((I + 127) / 128 + 1) / 2;
+  p.tiles_n = (J + 255) / 256;
+  p.raster_group = 8;
+  const int items = p.tiles_m * p.tiles_n * splits;
+  const int sms = sm_count();
+  const int clusters = items < sms / 2 ? items : sms / 2;
+  kern<<<2 * clusters, GEMM_THREADS, Cf::SMEM_BYTES, s>>>(ta, tb, p, splits);
+  count_launch();
+  BIMASK_CUDA_OK(cudaGetLastError());
+  if (splits > 1) {
+    const long long n4 = (long long)I * J / 4;
+    long long blocks = (n4 + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    splitk_reduce_kernel<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(partials), splits, n4,
+                                                         reinterpret_cast<float4*>(dW));
+    count_launch();
+    BIMASK_CUDA_OK(cudaGetLastError());
+  }
+  return BIMASK_OK;
+}
+
 // Split-K plan of the dense product, shared by the launcher and the workspace-size query.
 void wgrad_plan(int T, int I, int J, int* n_tile, int* splits, int* k_tiles_per_split) {
   const int nt = 256;
@@ -1249,7 +1339,7 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
   int rc;
   if ((rc = make_tmap(&ta, dY, (uint64_t)I, (uint64_t)T, 64)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, X, (uint64_t)J, (uint64_t)T, 64)) != BIMASK_OK) return rc;
-  auto kern = wgrad_pair_kernel<STAGES>;
+  auto kern = wgrad_pair_kernel<STAGES, false>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
   p.conv.mode = 0;

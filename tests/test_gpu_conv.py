@@ -96,3 +96,24 @@ def test_conv_bad_arguments_launch_nothing():
         bm.bimask_conv_layer_step(bm.make_conv_args(largs, NB, H, W, C, bm.binding.CONV_IMPLICIT))
     assert e.value.code == -2
     assert bm.bimask_launch_count() == n0
+
+
+@pytest.mark.parametrize("NB,H,W,C,I", [(5, 7, 7, 128, 128), (1, 20, 17, 128, 256), (2, 28, 28, 128, 384),
+                                        (1, 33, 8, 256, 128), (1, 14, 14, 256, 512), (4, 56, 56, 128, 128)])
+def test_conv_implicit_form_builds_no_column_matrix(NB, H, W, C, I):
+    N, M, P, seed = 2, 4, 4, 33
+    Wt, x, dy = conv_case(NB, H, W, C, I, 500 + H + C)
+    n0 = bm.bimask_launch_count()
+    b = run_conv_step(Wt, x, dy, N, M, P, seed, bm.binding.CONV_IMPLICIT)
+    n_imp = bm.bimask_launch_count() - n0
+    b2 = run_conv_step(Wt, x, dy, N, M, P, seed, bm.binding.CONV_EXPLICIT)
+    n_exp = bm.bimask_launch_count() - n0 - n_imp
+    assert n_exp - n_imp >= 2                      # the unfold and fold passes are gone
+    ref = O.conv_layer_step(Wt, x, dy, N, M, P, seed)
+    assert int(b["status_word"].item()) == 0
+    assert np.array_equal(b["perm"].cpu().numpy(), ref["perm"])
+    assert np.array_equal(u16(b["vals_b"]), ref["vals_b"])
+    for got in (b, b2):
+        assert rel_err(got["Y"].float().cpu().numpy().reshape(NB, H, W, I), ref["y"]) <= TOL
+        assert rel_err(got["dX"].float().cpu().numpy(), ref["dx"]) <= TOL
+        assert rel_err(got["dW"].cpu().numpy(), ref["dW"]) <= TOL
