@@ -239,8 +239,11 @@ int bimask_train_step(const bimask_train_args* args);
  * BIMASK_CONV_IMPLICIT never builds the column matrix: the GEMM kernels fetch shifted pixel
  * patches with 4-D tensor loads (out-of-image pixels read as zero); BIMASK_CONV_AUTO takes the
  * implicit form for every product whose shape allows it (C % 64 == 0; the input gradient also
- * needs C % 128 == 0 and I % 128 == 0) and the explicit form for the rest.  IMPLICIT with a shape
- * that does not allow it returns BIMASK_EUNSUPPORTED.  C % 32 == 0 and I % 32 == 0 always. */
+ * needs C % 128 == 0 and I % 128 == 0; patterns with a 2:4 form) when the column matrix would
+ * exceed 16 MiB, and the explicit form otherwise.  IMPLICIT with a shape that does not allow it
+ * returns BIMASK_EUNSUPPORTED.  C % 32 == 0 and I % 32 == 0 always.  The two forms round the
+ * input gradient differently (explicit: nine bf16 partial results summed in fp32; implicit: one
+ * fp32 accumulation), both within the products' tolerance. */
 enum { BIMASK_CONV_AUTO = 0, BIMASK_CONV_EXPLICIT = 1, BIMASK_CONV_IMPLICIT = 2 };
 typedef struct bimask_conv_args {
   bimask_layer_args layer;

@@ -36,7 +36,8 @@ struct Cfg {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
   static constexpr int META_COLS = SPARSE ? 4 : 0;
   static constexpr int TMEM_COLS = (N_TILE + META_COLS) <= 128 ? 128 : (N_TILE + META_COLS) <= 256 ? 256 : 512;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */ +
+                                    16384 /* epilogue staging */;
 };
 
 // A 3x3 convolution as an implicit GEMM: the token operand is an NHWC tensor and a "tile of
@@ -115,7 +116,7 @@ __device__ __forceinline__ void raster(int id, int tiles_m, int tiles_n, int gro
 template <int N_TILE, int STAGES, bool SPARSE, bool CONV>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-                   const GemmParams p) {
+                   const __grid_constant__ CUtensorMap tmapOut, const GemmParams p) {
   using C = Cfg<N_TILE, STAGES, SPARSE>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -127,6 +128,8 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
   const uint32_t tmem_full_bar = bar_base + 8u * (2 * STAGES);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * C::STAGE_BYTES + 8 * (2 * STAGES + 1));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t staging = bar_base + 256;             // epilogue staging, 4 KB per epilogue warp
+  uint8_t* staging_ptr = base_ptr + STAGES * C::STAGE_BYTES + 256;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int tile_m, tile_n;
@@ -150,6 +153,7 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmapA);
     ptx::prefetch_tmap(&tmapB);
+    ptx::prefetch_tmap(&tmapOut);
   }
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
@@ -246,7 +250,8 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     if (num_kt > 0) ok = ptx::mbar_wait_bounded(tmem_full_bar, 0, abort_flag, WAIT_BUDGET);
     if (!ok) *abort_flag = 1;
     ptx::tc_fence_after();
-    const int m = m0 + 32 * q + lane;
+    const uint32_t stg_base = staging + q * 4096;       // two 2 KB buffers per warp
+    uint16_t* stg_ptr = reinterpret_cast<uint16_t*>(staging_ptr + q * 4096);
     if (ok) {
 #pragma unroll 1
       for (int c = 0; c < N_TILE / 32; ++c) {
@@ -258,27 +263,35 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
 #pragma unroll
           for (int j = 0; j < 32; ++j) r[j] = 0u;
         }
-        const int nb = n0 + 32 * c;
-        __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
-        if (CONV) {
-          // token 32c + j of the box is pixel (cn0 + r / (wb*hb), ch0 + (r / wb) % hb, cw0 + r % wb)
-          if (m < p.Mdim) {
+        // registers -> bf16 -> this warp's staging tile [token][row] -> one TMA store of a 32 x 32 box
+        uint16_t* sbuf = stg_ptr + (c & 1) * 1024;
+        if (lane == 0) ptx::tma_store_wait_read1();         // the store that last used this buffer has read it
+        __syncwarp();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const int rr = 32 * c + j;
-              const int w = cw0 + (rr & (p.conv.wb - 1));
-              const int h = ch0 + ((rr >> p.conv.lg_wb) & (p.conv.hb - 1));
-              const int n = cn0 + (rr >> (p.conv.lg_wb + p.conv.lg_hb));
-              if (w < p.conv.W && h < p.conv.H && n < p.conv.NB)
-                out[(((size_t)n * p.conv.H + h) * p.conv.W + w) * p.Mdim + m] = __float2bfloat16_rn(__uint_as_float(r[j]));
-            }
+        for (int j = 0; j < 32; j += 2) {
+          const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+          const uint32_t u = *reinterpret_cast<const uint32_t*>(&v);
+          sbuf[j * 32 + lane] = (uint16_t)(u & 0xFFFFu);
+          sbuf[(j + 1) * 32 + lane] = (uint16_t)(u >> 16);
+        }
+        ptx::fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) {
+          const int mq = m0 + 32 * q;
+          const uint32_t src = stg_base + (uint32_t)(c & 1) * 2048u;
+          if (CONV) {
+            // tokens 32c .. 32c+31 of the box: 32 / wb consecutive image rows starting at (h, cw0) of image n
+            const int rr = 32 * c;
+            const int h = ch0 + ((rr >> p.conv.lg_wb) & (p.conv.hb - 1));
+            const int n = cn0 + (rr >> (p.conv.lg_wb + p.conv.lg_hb));
+            if (mq < p.Mdim && cw0 < p.conv.W && h < p.conv.H && n < p.conv.NB) ptx::tma_store_4d(&tmapOut, mq, cw0, h, n, src);
+          } else if (mq < p.Mdim && n0 + 32 * c < p.Ndim) {
+            ptx::tma_store_2d(&tmapOut, mq, n0 + 32 * c, src);
           }
-        } else if (m < p.Mdim) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (nb + j < p.Ndim) out[(size_t)(nb + j) * p.Mdim + m] = __float2bfloat16_rn(__uint_as_float(r[j]));
+          ptx::tma_store_commit();
         }
       }
+      if (lane == 0) ptx::tma_store_wait_all();
     }
   }
 
@@ -997,6 +1010,8 @@ int run_sparse(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, i
   int rc;
   if ((rc = make_tmap(&ta, vals, SPARSE ? (uint64_t)Kdim / 2 : (uint64_t)Kdim, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, N_TILE)) != BIMASK_OK) return rc;
+  CUtensorMap to;
+  if ((rc = make_tmap_out(&to, out, (uint64_t)Mdim, (uint64_t)Ndim, 32)) != BIMASK_OK) return rc;
   auto kern = spmm_single_kernel<N_TILE, STAGES, SPARSE, false>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
@@ -1011,14 +1026,11 @@ int run_sparse(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, i
   p.tiles_n = (Ndim + N_TILE - 1) / N_TILE;
   p.raster_group = 16;
   dim3 grid(p.tiles_m * p.tiles_n, 1, 1);
-  kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p);
+  kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, to, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }
-
-
-
 
 // Output-tile width of the CTA-pair 2:4 product.  Cost model in SM clocks, fitted to measurements
 // on the 16384 x 4096 / 4096 x 16384 layers: a tile's main loop takes 2 N clocks per 128-deep k
@@ -1112,6 +1124,8 @@ int run_conv_single(const uint16_t* vals, int a_rows, int a_kdim, const void* hw
   int rc;
   if ((rc = make_tmap(&ta, vals, (uint64_t)a_kdim / 2, (uint64_t)a_rows, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_nhwc_load(&tb, tok, g.CB, g.W, g.H, g.NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
+  CUtensorMap to;
+  if ((rc = make_tmap_nhwc_store(&to, out, Mdim, g.W, g.H, g.NB, g.wb)) != BIMASK_OK) return rc;
   auto kern = spmm_single_kernel<N_TILE, STAGES, true, true>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
@@ -1127,7 +1141,7 @@ int run_conv_single(const uint16_t* vals, int a_rows, int a_kdim, const void* hw
   p.raster_group = 16;
   p.n_tile = N_TILE;
   dim3 grid(p.tiles_m * p.tiles_n, 1, 1);
-  kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p);
+  kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, to, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;

@@ -37,7 +37,9 @@ def run_conv_step(Wt, x, dy, N, M, P, seed, mode, do_search=True):
 
 
 SHAPES = [(2, 9, 11, 32, 64), (3, 14, 14, 64, 128), (5, 7, 7, 128, 128), (1, 20, 17, 128, 256), (2, 28, 28, 128, 384),
-          (1, 33, 8, 256, 128), (2, 7, 7, 128, 128), (1, 14, 14, 256, 512), (3, 5, 4, 192, 320)]
+          (1, 33, 8, 256, 128), (2, 7, 7, 128, 128), (1, 14, 14, 256, 512), (3, 5, 4, 192, 320),
+          # column matrices above 16 MiB: AUTO takes the implicit form where the channel counts allow it
+          (20, 28, 28, 64, 128), (8, 28, 28, 192, 320), (6, 40, 36, 128, 256)]
 
 
 @pytest.mark.parametrize("NB,H,W,C,I", SHAPES)

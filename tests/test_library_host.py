@@ -72,6 +72,9 @@ def test_validation_happens_before_any_cuda_call(bm):
     assert L.bimask_wgrad(16, 16, 8, 64, 64, None, None, 0, 16, None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_layer_step(None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_train_step(None) == bm.binding.BIMASK_EINVAL
+    assert L.bimask_conv_layer_step(None) == bm.binding.BIMASK_EINVAL
+    assert bm.bimask_conv_workspace_bytes(32, 56, 56, 64, 64, 100) > 2 * 32 * 56 * 56 * 576 * 2
+    assert bm.bimask_conv_workspace_bytes(0, 56, 56, 64, 64, 100) == 0
     assert L.bimask_bwd_mask_criterion(16, None, 16, 16, 64, 64, 2, 4, 7, 0, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_bwd_mask_criterion(16, None, 16, 16, 64, 64, 2, 4, 1, 0, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL
     assert "needs S" in bm.bimask_last_error()
