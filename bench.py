@@ -490,6 +490,51 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+CONV_LAYERS = [(56, 56, 64, 64), (28, 28, 128, 128), (14, 14, 256, 256), (7, 7, 512, 512)]   # ResNet-50's 3x3 convolutions
+
+
+def run_conv(args):
+    """Side measurement, not the headline: the convolution form of the layer step (bimask_conv_layer_step) on
+    ResNet-50's 3x3 layers at batch --conv-batch, explicit and automatic form, CUDA events per step."""
+    import torch
+    import paper_2302_06058_b200 as bm
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    N, M, P, NB = 2, 4, 100, args.conv_batch
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    rows = []
+    for (H, W, C, I) in CONV_LAYERS:
+        T, J = NB * H * W, 9 * C
+        b = bm.alloc_layer_buffers(T, I, J, P)
+        b["W"] = torch.randn(I, J, device="cuda", generator=gen) * (2.0 / J) ** 0.5
+        b["X"] = torch.randn(NB, H, W, C, device="cuda", generator=gen).bfloat16()
+        b["dY"] = torch.randn(NB, H, W, I, device="cuda", generator=gen).bfloat16()
+        b["dX"] = torch.empty(NB, H, W, C, dtype=torch.bfloat16, device="cuda")
+        b["ws"] = torch.empty(bm.bimask_conv_workspace_bytes(NB, H, W, C, I, P), dtype=torch.uint8, device="cuda")
+        largs = bm.make_layer_args(T, I, J, N, M, P, 43, True, b)
+        row = {"layer": [NB, H, W, C, I]}
+        for name, mode in (("explicit", 1), ("auto", 0)):
+            ca = bm.make_conv_args(largs, NB, H, W, C, mode)
+            n0 = bm.bimask_launch_count()
+            for _ in range(max(args.warmup, 3)):
+                bm.bimask_conv_layer_step(ca)
+            launches = (bm.bimask_launch_count() - n0) // max(args.warmup, 3)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(args.steps):
+                bm.bimask_conv_layer_step(ca)
+            e1.record()
+            torch.cuda.synchronize()
+            row[name] = {"us_per_step": e0.elapsed_time(e1) * 1e3 / args.steps, "launches": int(launches)}
+        if int(b["status_word"].item()):
+            raise RuntimeError("device status word non-zero")
+        rows.append(row)
+    print(json.dumps({"workload": "3x3 convolution layer steps (ResNet-50 shapes), 2:4, P = 100, search on",
+                      "conv": rows, "steps": args.steps, "note": "inputs smaller than L2: warm-cache numbers"}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -503,7 +548,12 @@ def main():
     ap.add_argument("--layer", type=int, default=0)
     ap.add_argument("--ref-rows", type=int, default=1024)
     ap.add_argument("--ref-tokens", type=int, default=256)
+    ap.add_argument("--conv", action="store_true", help="time the convolution form of the layer step instead")
+    ap.add_argument("--conv-batch", type=int, default=32)
     args = ap.parse_args()
+    if args.conv and args.impl != "reference":
+        run_conv(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
