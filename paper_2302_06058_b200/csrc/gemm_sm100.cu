@@ -1258,7 +1258,7 @@ static void wgrad_plan_k(int k_tiles, int I, int J, int* splits, int* k_tiles_pe
   const int tiles = (((I + 127) / 128 + 1) / 2) * ((J + 255) / 256);     // 256 x 256 pair tiles
   int sp = 1;
   if (tiles < 74) {
-    sp = (2 * 74 + tiles - 1) / tiles;
+    sp = 74 / tiles;                                              // one round of work items over the 74 CTA pairs
     const int max_by_k = k_tiles / 8 > 0 ? k_tiles / 8 : 1;        // at least 8 k tiles per split
     if (sp > max_by_k) sp = max_by_k;
     if (sp > 64) sp = 64;
@@ -1328,19 +1328,8 @@ int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int 
 
 // Split-K plan of the dense product, shared by the launcher and the workspace-size query.
 void wgrad_plan(int T, int I, int J, int* n_tile, int* splits, int* k_tiles_per_split) {
-  const int nt = 256;
-  const int tiles = (((I + 127) / 128 + 1) / 2) * ((J + nt - 1) / nt);     // 256 x 256 pair tiles
-  const int k_tiles = (T + 63) / 64;
-  int sp = 1;
-  if (tiles < 74) {
-    sp = (2 * 74 + tiles - 1) / tiles;
-    const int max_by_k = k_tiles / 8 > 0 ? k_tiles / 8 : 1;        // at least 8 k tiles per split
-    if (sp > max_by_k) sp = max_by_k;
-    if (sp > 64) sp = 64;
-  }
-  int per = (k_tiles + sp - 1) / sp;
-  sp = (k_tiles + per - 1) / per;
-  *n_tile = nt; *splits = sp; *k_tiles_per_split = per;
+  *n_tile = 256;
+  wgrad_plan_k((T + 63) / 64, I, J, splits, k_tiles_per_split);
 }
 
 int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J, float* dW, float* partials,
