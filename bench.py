@@ -490,6 +490,80 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def run_per_call(args):
+    """Side measurement: every C-ABI call of the path alone, 5 warm-up + --steps timed launches each, CUDA events,
+    min and median; "cold" = a 256 MB buffer is overwritten before every launch (L2 flushed, clocks near burst because
+    of the gaps), "warm" = back to back.  Fractions are against the burst peaks (copy bandwidth, bf16 burst)."""
+    import torch
+    import paper_2302_06058_b200 as bm
+    from paper_2302_06058_b200 import inputs
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    cfg = inputs.CONFIGS[args.config]
+    seed = inputs.perm_seed(args.config)
+    peaks = load_peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    reps = max(args.steps, 20) if args.steps != 100 else 20
+    out = []
+    for li, L in enumerate(cfg.layers):
+        W, X, dY = inputs.make_layer(args.config, li)
+        b = bm.alloc_layer_buffers(L.T, L.I, L.J, cfg.P)
+        b["W"] = torch.from_numpy(W).cuda()
+        b["X"] = torch.from_numpy(X.view(np.int16)).cuda().view(torch.bfloat16)
+        b["dY"] = torch.from_numpy(dY.view(np.int16)).cuda().view(torch.bfloat16)
+        wsb = b["ws"].numel()
+        mom = torch.zeros(L.I, L.J, device="cuda")
+        calls = {
+            "fwd_mask": lambda: bm.bimask_fwd_mask(b["W"], L.I, L.J, cfg.N, cfg.M, b["maskbits_f"], b["vals_f"], b["meta_f"],
+                                                   b["hw_meta_f"]),
+            "spmm_fwd": lambda: bm.bimask_spmm_fwd(b["X"], b["vals_f"], b["hw_meta_f"], L.T, L.I, L.J, b["Y"], b["status_word"]),
+            "perm_search": lambda: bm.bimask_perm_search(b["maskbits_f"], L.I, L.J, cfg.N, cfg.M, cfg.P, seed, None, b["perm"],
+                                                         b["best_idx"], b["counts"], b["ws"], wsb),
+            "bwd_mask": lambda: bm.bimask_bwd_mask(b["W"], b["maskbits_f"], b["perm"], L.I, L.J, cfg.N, cfg.M, b["maskbits_b"],
+                                                   b["vals_b"], b["meta_b"], b["hw_meta_b"]),
+            "spmm_dgrad": lambda: bm.bimask_spmm_dgrad(b["dY"], b["perm"], b["vals_b"], b["hw_meta_b"], L.T, L.I, L.J, b["dX"],
+                                                       b["ws"], wsb, b["status_word"]),
+            "wgrad": lambda: bm.bimask_wgrad(b["dY"], b["X"], L.T, L.I, L.J, b["dW"], b["ws"], wsb, b["status_word"]),
+            "sgd_fwd_mask": lambda: bm.bimask_sgd_fwd_mask(b["W"], b["dW"], mom, L.I, L.J, cfg.N, cfg.M, 1e-9, 0.9, 1e-4,
+                                                           b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"]),
+        }
+        work = algorithmic_work(L, cfg.P)
+        work["sgd_fwd_mask"] = {"bound": "hbm", "bytes": 21.4 * L.I * L.J}
+        for name, fn in calls.items():
+            res = {"layer": li, "call": name}
+            for kind in ("cold", "warm"):
+                for _ in range(5):
+                    fn()
+                torch.cuda.synchronize()
+                ts = []
+                for _ in range(reps):
+                    if kind == "cold":
+                        flush.zero_()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    fn()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    ts.append(e0.elapsed_time(e1) * 1e3)
+                res[kind + "_us_min"] = min(ts)
+                res[kind + "_us_median"] = float(np.median(ts))
+            w = work[name]
+            t = res["cold_us_median"] * 1e-6
+            if w["bound"] == "hbm":
+                res.update(bound="hbm", achieved=w["bytes"] / t / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
+            else:
+                pk = peaks["bf16_tflops"] * (1.0 if name == "wgrad" else 2.0)
+                res.update(bound="tensor", achieved=w["flops"] / t / 1e12, peak=pk, unit="TFLOP/s")
+            res["frac"] = res["achieved"] / res["peak"]
+            out.append(res)
+        if int(b["status_word"].item()):
+            raise RuntimeError("device status word non-zero")
+        del b
+    print(json.dumps({"per_call": out, "config": args.config, "launches_per_kind": reps, "peak_source": peaks["source"],
+                      "note": "fractions of the burst peaks from the cold median"}), flush=True)
+
+
 CONV_LAYERS = [(56, 56, 64, 64), (28, 28, 128, 128), (14, 14, 256, 256), (7, 7, 512, 512)]   # ResNet-50's 3x3 convolutions
 
 
@@ -548,11 +622,15 @@ def main():
     ap.add_argument("--layer", type=int, default=0)
     ap.add_argument("--ref-rows", type=int, default=1024)
     ap.add_argument("--ref-tokens", type=int, default=256)
+    ap.add_argument("--per-call", action="store_true", help="time every C-ABI call alone (cold and warm L2, min and median)")
     ap.add_argument("--conv", action="store_true", help="time the convolution form of the layer step instead")
     ap.add_argument("--conv-batch", type=int, default=32)
     args = ap.parse_args()
     if args.conv and args.impl != "reference":
         run_conv(args)
+        return
+    if args.per_call and args.impl != "reference":
+        run_per_call(args)
         return
     if args.impl == "reference":
         run_reference(args)
