@@ -561,6 +561,208 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
 }
 
 // ------------------------------------------------------------------------------------------
+// CTA-pair 2:4 product, two row tiles per token tile.  The kernel above streams, per 128-deep k
+// tile and CTA, 16 KB of compressed weights + up to 32 KB of activations + 2 KB of metadata for
+// 512 tensor-pipe clocks -- about 1.5 x the bytes per clock of the dense kernel, and measurement
+// puts it at the L2 -> shared-memory feed rate (tensor pipe 79 % busy, L2 at 60-70 %).  Here a pair
+// owns 512 x N outputs: TWO 256-row MMA tiles that share the activation tile in shared memory, so
+// a stage carries 2 x 16 KB + <= 30 KB + 2 x 2 KB for twice the tensor-pipe work (a third fewer
+// bytes per clock).  Both accumulators (tensor-memory columns 0.. and 256.., N <= 240) belong to
+// the same token tile, so the epilogue cannot overlap the next main loop; instead eight epilogue
+// warps per CTA drain the two accumulators side by side.  Metadata: columns 496..499 and 500..503.
+// Roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 accumulator 0, warps 6-9 accumulator 1.
+// ------------------------------------------------------------------------------------------
+constexpr int GEMM2M_THREADS = 320;
+
+template <int STAGES>
+struct Pair2MCfg {
+  static constexpr int A_BYTES = 16384;                    // per row tile: 128 rows x 64 compressed bf16
+  static constexpr int B_MAX = 30720;                      // 120 rows x 128 bf16 (two 64-wide boxes), N <= 240
+  static constexpr int E_BYTES = 2048;
+  static constexpr int STAGE_BYTES = 2 * A_BYTES + B_MAX + 2 * E_BYTES;      // 66 KB
+  static constexpr int STAGING_BYTES = 8 * 2 * 1024;       // per epilogue warp: two [16 tokens][32 rows] bf16 buffers
+  static constexpr int TMEM_COLS = 512;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 + 256;
+};
+
+template <int STAGES>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2M_THREADS, 1)
+spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
+                   const __grid_constant__ CUtensorMap tmapE, const __grid_constant__ CUtensorMap tmapOut16,
+                   const GemmParams p) {
+  using C = Pair2MCfg<STAGES>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = ptx::smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - raw);
+  const uint32_t staging = base + STAGES * C::STAGE_BYTES;
+  uint8_t* staging_ptr = base_ptr + STAGES * C::STAGE_BYTES;
+  const uint32_t bar_base = staging + C::STAGING_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  const uint32_t tmem_full_bar = bar_base + 8u * (2 * STAGES);
+  const uint32_t tmem_empty_bar = bar_base + 8u * (2 * STAGES + 1);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(staging_ptr + C::STAGING_BYTES + 8 * (2 * STAGES + 2));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = ptx::cluster_ctarank();
+  const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+  const int num_tiles = p.tiles_m * p.tiles_n;            // tiles_m counts 512-row tiles
+  const int num_kt = (p.Kdim + 127) / 128;
+  const int SP_N = p.n_tile;                              // tokens per tile, multiple of 16, <= 240
+  const uint32_t b_box = (uint32_t)(SP_N / 2) * 128u;     // bytes of one 64-wide box of this CTA's activation rows
+  const uint32_t stage_tx = 2u * C::A_BYTES + 2u * b_box + 2u * C::E_BYTES;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    ptx::mbar_init(tmem_full_bar, 1);
+    ptx::mbar_init(tmem_empty_bar, 16);                   // eight epilogue warps in each CTA of the pair
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmapA);
+    ptx::prefetch_tmap(&tmapB);
+    ptx::prefetch_tmap(&tmapE);
+    ptx::prefetch_tmap(&tmapOut16);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
+    ptx::tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_meta = tmem_base + 496u;            // + 4 * row tile
+
+  // 128-row block of row tile mt (0 / 1) of this CTA inside 512-row tile tile_m
+  auto mt128_of = [&](int tile_m, int mt) { return 4 * tile_m + 2 * mt + (int)rank; };
+
+  if (warp == 0) {
+    if (ptx::elect_one()) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+        int tile_m, tile_n;
+        raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
+        const int nrow = tile_n * SP_N + (SP_N / 2) * (int)rank;
+        for (int kt = 0; kt < num_kt; ++kt, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; ok = false; break; }
+          const uint32_t a_s = base + s * C::STAGE_BYTES;
+          const uint32_t b_s = a_s + 2 * C::A_BYTES;
+          const uint32_t e_s = b_s + C::B_MAX;
+          const uint32_t bar = ptx::mapa(full_bar(s), 0);
+          if (rank == 0) ptx::mbar_expect_tx(full_bar(s), 2 * stage_tx);
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) {
+            const int mt128 = mt128_of(tile_m, mt);
+            ptx::tma_load_2d_pair(a_s + mt * C::A_BYTES, &tmapA, kt * 64, mt128 * 128, bar);
+            ptx::tma_load_2d_pair(e_s + mt * C::E_BYTES, &tmapE, 0, 2 * (mt128 * p.tiles_k_meta + kt), bar);
+          }
+          ptx::tma_load_2d_pair(b_s, &tmapB, kt * 128, nrow, bar);
+          ptx::tma_load_2d_pair(b_s + b_box, &tmapB, kt * 128 + 64, nrow, bar);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (rank == 0 && ptx::elect_one()) {
+      const uint32_t idesc = ptx::idesc_bf16(256, SP_N, false, false, true);
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++tcount) {
+        // both accumulators must have been drained by all sixteen epilogue warps of the pair
+        if (!ptx::mbar_wait_bounded(tmem_empty_bar, (tcount & 1u) ^ 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
+        ptx::tc_fence_after();
+        for (int kt = 0; kt < num_kt; ++kt, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t a_s = base + s * C::STAGE_BYTES;
+          const uint32_t b_s = a_s + 2 * C::A_BYTES;
+          const uint32_t e_s = b_s + C::B_MAX;
+          ptx::tmem_cp_128x128b_pair(tmem_meta, ptx::smem_desc(e_s, 0, 128, 0));
+          ptx::tmem_cp_128x128b_pair(tmem_meta + 4u, ptx::smem_desc(e_s + C::E_BYTES, 0, 128, 0));
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) {
+#pragma unroll
+            for (int kb = 0; kb < 4; ++kb) {
+              const uint64_t ad = ptx::smem_desc(a_s + mt * C::A_BYTES + kb * 32, 16, 1024, 2);
+              const uint64_t bd = ptx::smem_desc(b_s + (kb >> 1) * b_box + (kb & 1) * 64, 16, 1024, 2);
+              ptx::mma_sparse_pair(tmem_base + 256u * mt, ad, bd, tmem_meta + 4u * mt + (kb & ~1), idesc | (uint32_t)(kb & 1),
+                                   (kt | kb) != 0);
+            }
+          }
+          ptx::tc_commit_pair(empty_bar(s), 3);
+        }
+        if (ok) ptx::tc_commit_pair(tmem_full_bar, 3);
+      }
+    }
+  } else {
+    // warps 2-5 drain accumulator 0 (row tile 0), warps 6-9 accumulator 1; a warp reads its own
+    // tensor-memory lane quadrant and owns two 1 KB staging buffers
+    const int q = warp & 3;
+    const int mt = warp >= 6 ? 1 : 0;
+    const int ew = warp - 2;                               // 0..7
+    const uint32_t stg_base = staging + ew * 2048;
+    uint16_t* stg_ptr = reinterpret_cast<uint16_t*>(staging_ptr + ew * 2048);
+    const uint32_t release_bar = ptx::mapa(tmem_empty_bar, 0);
+    uint32_t tcount = 0, chunk = 0;
+    for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++tcount) {
+      int tile_m, tile_n;
+      raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
+      const int m0 = mt128_of(tile_m, mt) * 128 + 32 * q, n0 = tile_n * SP_N;
+      if (!ptx::mbar_wait_bounded(tmem_full_bar, tcount & 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
+      ptx::tc_fence_after();
+      const uint32_t acc = tmem_base + 256u * mt + ((uint32_t)(32 * q) << 16);
+#pragma unroll 1
+      for (int c = 0; c < SP_N / 16; ++c, ++chunk) {
+        uint32_t r[16];
+        ptx::tmem_ld_32x16(acc + 16 * c, r);
+        ptx::tmem_ld_wait();
+        if (c == SP_N / 16 - 1) {                          // last read of this accumulator quadrant: release it
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive_cluster(release_bar);
+        }
+        uint16_t* sbuf = stg_ptr + (chunk & 1u) * 512;     // two 1 KB buffers
+        if (lane == 0) ptx::tma_store_wait_read1();
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 16; j += 2) {
+          const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+          const uint32_t u = *reinterpret_cast<const uint32_t*>(&v);
+          sbuf[j * 32 + lane] = (uint16_t)(u & 0xFFFFu);
+          sbuf[(j + 1) * 32 + lane] = (uint16_t)(u >> 16);
+        }
+        ptx::fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) {
+          if (m0 < p.Mdim && n0 + 16 * c < p.Ndim) ptx::tma_store_2d(&tmapOut16, m0, n0 + 16 * c, stg_base + (chunk & 1u) * 1024);
+          ptx::tma_store_commit();
+        }
+      }
+    }
+    if (lane == 0) ptx::tma_store_wait_all();
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status_word, (int32_t)BIMASK_ETIMEOUT);
+  ptx::cluster_sync();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Dense weight gradient on CTA pairs, persistent.  D[i, j] = sum_t dY[t, i] X[t, j]: both
 // operands are read MN-major straight from the row-major activations (no transpose pass).  A
 // pair owns a 256 x 256 tile; each CTA loads its 128 rows of dY^T and 128 of the 256 columns of
@@ -1086,10 +1288,65 @@ int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const 
   return BIMASK_OK;
 }
 
+// Token-tile width of the two-row-tile kernel: per 128-deep k tile a pair issues eight MMAs of N / 2
+// clocks; the epilogue (not overlapped) costs about 2500 clocks per tile.
+int choose_sparse_n_2m(int tiles_m512, int Ndim, int k_tiles, int clusters) {
+  int best_n = 240;
+  double best = 1e30;
+  for (int n = 240; n >= 160; n -= 16) {
+    const long long tiles = (long long)tiles_m512 * ((Ndim + n - 1) / n);
+    const long long rounds = (tiles + clusters - 1) / clusters;
+    const double cost = (double)rounds * ((double)k_tiles * 4.0 * n + 2500.0) * (1.0 + 0.003 * (240 - n));
+    if (cost < best) { best = cost; best_n = n; }
+  }
+  return best_n;
+}
+
+int run_sparse_pair2m(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim, int Kdim,
+                      uint16_t* out, int32_t* status_word, cudaStream_t s) {
+  constexpr int STAGES = 3;
+  using C = Pair2MCfg<STAGES>;
+  CUtensorMap ta, tb, te, to16;
+  int rc;
+  const int tiles_m = (Mdim + 127) / 128, tiles_k = (Kdim + 127) / 128;
+  const int sms = sm_count();
+  const int tiles_m512 = (tiles_m + 3) / 4;
+  const int n_tile = choose_sparse_n_2m(tiles_m512, Ndim, tiles_k, sms / 2);
+  if ((rc = make_tmap(&ta, vals, (uint64_t)Kdim / 2, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, n_tile / 2)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_meta(&te, hw_meta, (uint64_t)tiles_m * tiles_k)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_out(&to16, out, (uint64_t)Mdim, (uint64_t)Ndim, 16)) != BIMASK_OK) return rc;
+  auto kern = spmm_pair2m_kernel<STAGES>;
+  if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
+  GemmParams p;
+  p.conv.mode = 0;
+  p.hw_meta = reinterpret_cast<const uint8_t*>(hw_meta);
+  p.tiles_k_meta = tiles_k;
+  p.Mdim = Mdim; p.Ndim = Ndim; p.Kdim = Kdim;
+  p.k_tiles_per_split = tiles_k;
+  p.out = out;
+  p.status_word = status_word;
+  p.n_tile = n_tile;
+  p.tiles_m = tiles_m512;
+  p.tiles_n = (Ndim + n_tile - 1) / n_tile;
+  p.raster_group = 4;
+  const int total = p.tiles_m * p.tiles_n;
+  const int clusters = total < sms / 2 ? total : sms / 2;
+  kern<<<2 * clusters, GEMM2M_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, to16, p);
+  count_launch();
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
 }  // namespace
 
 int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim, int Kdim,
                 uint16_t* out, int32_t* status_word, cudaStream_t s) {
+  // large operands with a long reduction: two row tiles per token tile (fewer bytes per tensor-pipe clock; its
+  // epilogue is not overlapped, which only pays off from about 48 k tiles: measured 7-10 % faster at k = 16384,
+  // 2 % slower at k = 4096)
+  if (Ndim >= 1024 && Mdim >= 2048 && Kdim >= 6144)
+    return run_sparse_pair2m(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   if (Ndim > 128 && Mdim > 128) return run_sparse_pair_persistent(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   if (Ndim > 128) return run_sparse<256, 2>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   return run_sparse<128, 4>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);

@@ -412,3 +412,22 @@ def test_bounded_wait_reports_timeout_and_context_survives():
     W = inputs.make_weight(64, 64, 1)
     _, b = run_fwd_mask(W, 2)                       # the device still works
     assert np.array_equal(u32(b["maskbits_f"]), O.pack_bits(O.forward_mask(W, 2, 4)))
+
+
+@pytest.mark.parametrize("I,J,T", [(2176, 6176, 1040), (2048, 6144, 1024), (6400, 2080, 1265)])
+def test_large_operand_sparse_kernel_ragged_shapes(I, J, T):
+    """Operands of >= 2048 rows with >= 1024 tokens and k >= 6144 run on the kernel that pairs two row tiles per
+    token tile: rows that do not fill the last 512-row tile, a ragged token tail and a k tail, forward and input gradient."""
+    N, M = 2, 4
+    W = inputs.make_weight(I, J, 900 + I % 97)
+    X = inputs.make_activation(T, J, 901)
+    dY = inputs.make_activation(T, I, 902)
+    rng = np.random.default_rng(I + J)
+    perm = rng.permutation(I).astype(np.int32)
+    b = run_layer_step(W, X, dY, N, M, 2, 5, do_search=False, perm=perm)
+    assert int(b["status_word"].item()) == 0
+    B = O.forward_mask(W, N, M)
+    Bbar = O.backward_mask(W, B, perm, N, M)
+    assert np.array_equal(u32(b["maskbits_b"]), O.pack_bits(Bbar))
+    assert rel_err(b["Y"].float().cpu().numpy(), O.spmm_fwd(X, W, B)) <= TOL
+    assert rel_err(b["dX"].float().cpu().numpy(), O.spmm_dgrad(dY, W, O.unpermute_rows(Bbar, perm))) <= TOL
