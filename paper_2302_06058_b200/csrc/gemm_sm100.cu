@@ -566,8 +566,8 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
 // 512 tensor-pipe clocks -- about 1.5 x the bytes per clock of the dense kernel, and measurement
 // puts it at the L2 -> shared-memory feed rate (tensor pipe 79 % busy, L2 at 60-70 %).  Here a pair
 // owns 512 x N outputs: TWO 256-row MMA tiles that share the activation tile in shared memory, so
-// a stage carries 2 x 16 KB + <= 30 KB + 2 x 2 KB for twice the tensor-pipe work (a third fewer
-// bytes per clock).  Both accumulators (tensor-memory columns 0.. and 256.., N <= 240) belong to
+// a stage carries 2 x 16 KB + <= 28 KB + 2 x 2 KB for twice the tensor-pipe work (a third fewer
+// bytes per clock).  Both accumulators (tensor-memory columns 0.. and 256.., N <= 224) belong to
 // the same token tile, so the epilogue cannot overlap the next main loop; instead eight epilogue
 // warps per CTA drain the two accumulators side by side.  Metadata: columns 496..499 and 500..503.
 // Roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 accumulator 0, warps 6-9 accumulator 1.
@@ -577,10 +577,10 @@ constexpr int GEMM2M_THREADS = 320;
 template <int STAGES>
 struct Pair2MCfg {
   static constexpr int A_BYTES = 16384;                    // per row tile: 128 rows x 64 compressed bf16
-  static constexpr int B_MAX = 30720;                      // 120 rows x 128 bf16 (two 64-wide boxes), N <= 240
+  static constexpr int B_MAX = 28672;                      // 112 rows x 128 bf16 (two 64-wide boxes), N <= 224
   static constexpr int E_BYTES = 2048;
-  static constexpr int STAGE_BYTES = 2 * A_BYTES + B_MAX + 2 * E_BYTES;      // 66 KB
-  static constexpr int STAGING_BYTES = 8 * 2 * 1024;       // per epilogue warp: two [16 tokens][32 rows] bf16 buffers
+  static constexpr int STAGE_BYTES = 2 * A_BYTES + B_MAX + 2 * E_BYTES;      // 64 KB
+  static constexpr int STAGING_BYTES = 8 * 2 * 2048;       // per epilogue warp: two [32 tokens][32 rows] bf16 buffers
   static constexpr int TMEM_COLS = 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 + 256;
 };
@@ -588,7 +588,7 @@ struct Pair2MCfg {
 template <int STAGES>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2M_THREADS, 1)
 spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-                   const __grid_constant__ CUtensorMap tmapE, const __grid_constant__ CUtensorMap tmapOut16,
+                   const __grid_constant__ CUtensorMap tmapE, const __grid_constant__ CUtensorMap tmapOut32,
                    const GemmParams p) {
   using C = Pair2MCfg<STAGES>;
   extern __shared__ uint8_t smem_raw[];
@@ -610,7 +610,7 @@ spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
   const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
   const int num_tiles = p.tiles_m * p.tiles_n;            // tiles_m counts 512-row tiles
   const int num_kt = (p.Kdim + 127) / 128;
-  const int SP_N = p.n_tile;                              // tokens per tile, multiple of 16, <= 240
+  const int SP_N = p.n_tile;                              // tokens per tile, multiple of 32, <= 224
   const uint32_t b_box = (uint32_t)(SP_N / 2) * 128u;     // bytes of one 64-wide box of this CTA's activation rows
   const uint32_t stage_tx = 2u * C::A_BYTES + 2u * b_box + 2u * C::E_BYTES;
 
@@ -626,7 +626,7 @@ spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     ptx::prefetch_tmap(&tmapA);
     ptx::prefetch_tmap(&tmapB);
     ptx::prefetch_tmap(&tmapE);
-    ptx::prefetch_tmap(&tmapOut16);
+    ptx::prefetch_tmap(&tmapOut32);
   }
   if (warp == 1) {
     ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
@@ -710,8 +710,8 @@ spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     const int q = warp & 3;
     const int mt = warp >= 6 ? 1 : 0;
     const int ew = warp - 2;                               // 0..7
-    const uint32_t stg_base = staging + ew * 2048;
-    uint16_t* stg_ptr = reinterpret_cast<uint16_t*>(staging_ptr + ew * 2048);
+    const uint32_t stg_base = staging + ew * 4096;
+    uint16_t* stg_ptr = reinterpret_cast<uint16_t*>(staging_ptr + ew * 4096);
     const uint32_t release_bar = ptx::mapa(tmem_empty_bar, 0);
     uint32_t tcount = 0, chunk = 0;
     for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++tcount) {
@@ -722,20 +722,20 @@ spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
       ptx::tc_fence_after();
       const uint32_t acc = tmem_base + 256u * mt + ((uint32_t)(32 * q) << 16);
 #pragma unroll 1
-      for (int c = 0; c < SP_N / 16; ++c, ++chunk) {
-        uint32_t r[16];
-        ptx::tmem_ld_32x16(acc + 16 * c, r);
+      for (int c = 0; c < SP_N / 32; ++c, ++chunk) {
+        uint32_t r[32];
+        ptx::tmem_ld_32x32(acc + 32 * c, r);
         ptx::tmem_ld_wait();
-        if (c == SP_N / 16 - 1) {                          // last read of this accumulator quadrant: release it
+        if (c == SP_N / 32 - 1) {                          // last read of this accumulator quadrant: release it
           ptx::tc_fence_before();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive_cluster(release_bar);
         }
-        uint16_t* sbuf = stg_ptr + (chunk & 1u) * 512;     // two 1 KB buffers
+        uint16_t* sbuf = stg_ptr + (chunk & 1u) * 1024;    // two 2 KB buffers
         if (lane == 0) ptx::tma_store_wait_read1();
         __syncwarp();
 #pragma unroll
-        for (int j = 0; j < 16; j += 2) {
+        for (int j = 0; j < 32; j += 2) {
           const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
           const uint32_t u = *reinterpret_cast<const uint32_t*>(&v);
           sbuf[j * 32 + lane] = (uint16_t)(u & 0xFFFFu);
@@ -744,7 +744,7 @@ spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
         ptx::fence_proxy_async();
         __syncwarp();
         if (lane == 0) {
-          if (m0 < p.Mdim && n0 + 16 * c < p.Ndim) ptx::tma_store_2d(&tmapOut16, m0, n0 + 16 * c, stg_base + (chunk & 1u) * 1024);
+          if (m0 < p.Mdim && n0 + 32 * c < p.Ndim) ptx::tma_store_2d(&tmapOut32, m0, n0 + 32 * c, stg_base + (chunk & 1u) * 2048);
           ptx::tma_store_commit();
         }
       }
@@ -1291,12 +1291,12 @@ int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const 
 // Token-tile width of the two-row-tile kernel: per 128-deep k tile a pair issues eight MMAs of N / 2
 // clocks; the epilogue (not overlapped) costs about 2500 clocks per tile.
 int choose_sparse_n_2m(int tiles_m512, int Ndim, int k_tiles, int clusters) {
-  int best_n = 240;
+  int best_n = 224;
   double best = 1e30;
-  for (int n = 240; n >= 160; n -= 16) {
+  for (int n = 224; n >= 160; n -= 32) {
     const long long tiles = (long long)tiles_m512 * ((Ndim + n - 1) / n);
     const long long rounds = (tiles + clusters - 1) / clusters;
-    const double cost = (double)rounds * ((double)k_tiles * 4.0 * n + 2500.0) * (1.0 + 0.003 * (240 - n));
+    const double cost = (double)rounds * ((double)k_tiles * 4.0 * n + 2500.0) * (1.0 + 0.003 * (224 - n));
     if (cost < best) { best = cost; best_n = n; }
   }
   return best_n;
@@ -1306,7 +1306,7 @@ int run_sparse_pair2m(const uint16_t* vals, const void* hw_meta, const uint16_t*
                       uint16_t* out, int32_t* status_word, cudaStream_t s) {
   constexpr int STAGES = 3;
   using C = Pair2MCfg<STAGES>;
-  CUtensorMap ta, tb, te, to16;
+  CUtensorMap ta, tb, te, to32;
   int rc;
   const int tiles_m = (Mdim + 127) / 128, tiles_k = (Kdim + 127) / 128;
   const int sms = sm_count();
@@ -1315,7 +1315,7 @@ int run_sparse_pair2m(const uint16_t* vals, const void* hw_meta, const uint16_t*
   if ((rc = make_tmap(&ta, vals, (uint64_t)Kdim / 2, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, n_tile / 2)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_meta(&te, hw_meta, (uint64_t)tiles_m * tiles_k)) != BIMASK_OK) return rc;
-  if ((rc = make_tmap_out(&to16, out, (uint64_t)Mdim, (uint64_t)Ndim, 16)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_out(&to32, out, (uint64_t)Mdim, (uint64_t)Ndim, 32)) != BIMASK_OK) return rc;
   auto kern = spmm_pair2m_kernel<STAGES>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
@@ -1332,7 +1332,7 @@ int run_sparse_pair2m(const uint16_t* vals, const void* hw_meta, const uint16_t*
   p.raster_group = 4;
   const int total = p.tiles_m * p.tiles_n;
   const int clusters = total < sms / 2 ? total : sms / 2;
-  kern<<<2 * clusters, GEMM2M_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, to16, p);
+  kern<<<2 * clusters, GEMM2M_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, to32, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -1343,9 +1343,9 @@ int run_sparse_pair2m(const uint16_t* vals, const void* hw_meta, const uint16_t*
 int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim, int Kdim,
                 uint16_t* out, int32_t* status_word, cudaStream_t s) {
   // large operands with a long reduction: two row tiles per token tile (fewer bytes per tensor-pipe clock; its
-  // epilogue is not overlapped, which only pays off from about 48 k tiles: measured 7-10 % faster at k = 16384,
-  // 2 % slower at k = 4096)
-  if (Ndim >= 1024 && Mdim >= 2048 && Kdim >= 6144)
+  // epilogue is not overlapped, which pays off from about 28 k tiles: measured 2 % faster at k = 4096, 8-10 % at
+  // k = 16384)
+  if (Ndim >= 1024 && Mdim >= 2048 && Kdim >= 4096)
     return run_sparse_pair2m(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   if (Ndim > 128 && Mdim > 128) return run_sparse_pair_persistent(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   if (Ndim > 128) return run_sparse<256, 2>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
