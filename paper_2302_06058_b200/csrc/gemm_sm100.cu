@@ -967,20 +967,21 @@ permute_cols_kernel(const uint16_t* __restrict__ dY, const int32_t* __restrict__
                     uint16_t* __restrict__ dYp) {
   extern __shared__ uint32_t tile_w[];                   // R == 4: [I] x uint2, R == 2: [I] x uint32
   const int half = I >> 1;
+  const int nthreads = (int)blockDim.x;                  // 256 .. 1024: short rows run more, smaller CTAs per SM
   for (int t0 = blockIdx.x * R; t0 < T; t0 += gridDim.x * R) {
     const uint32_t* src = reinterpret_cast<const uint32_t*>(dY) + (size_t)t0 * half;
     // four column chunks per trip: 4 R loads in flight per thread before any is consumed
-    for (int c0 = threadIdx.x; c0 < half; c0 += 4 * PERMUTE_THREADS) {
+    for (int c0 = threadIdx.x; c0 < half; c0 += 4 * nthreads) {
       uint32_t r[4][R];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const int c = c0 + u * PERMUTE_THREADS;
+        const int c = c0 + u * nthreads;
 #pragma unroll
         for (int j = 0; j < R; ++j) r[u][j] = (c < half && t0 + j < T) ? __ldg(src + (size_t)j * half + c) : 0u;
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const int c = c0 + u * PERMUTE_THREADS;
+        const int c = c0 + u * nthreads;
         if (c < half) {
           if (R == 4) {
             reinterpret_cast<uint4*>(tile_w)[c] =
@@ -994,7 +995,7 @@ permute_cols_kernel(const uint16_t* __restrict__ dY, const int32_t* __restrict__
       }
     }
     __syncthreads();
-    for (int k8 = threadIdx.x; k8 < (I >> 3); k8 += PERMUTE_THREADS) {
+    for (int k8 = threadIdx.x; k8 < (I >> 3); k8 += nthreads) {
       const int4 pa = __ldg(reinterpret_cast<const int4*>(perm) + 2 * k8);
       const int4 pb = __ldg(reinterpret_cast<const int4*>(perm) + 2 * k8 + 1);
       const int idx[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
@@ -1499,12 +1500,16 @@ int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, u
   const int R = (size_t)I * 8 <= 200 * 1024 ? 4 : 2;
   const size_t smem = (size_t)I * 2 * R;
   const int groups = (T + R - 1) / R;
-  const int per_sm = smem <= 32 * 1024 ? 3 : smem <= 48 * 1024 ? 2 : 1;
+  // a thread stages 16 row loads per trip and gathers 8 columns per trip: rows of I columns keep I / 8 threads busy
+  const int threads = I >= 8192 ? PERMUTE_THREADS : I >= 4096 ? 512 : 256;
+  int per_sm = (int)((200 * 1024) / smem);
+  if (per_sm > 2048 / threads) per_sm = 2048 / threads;
+  if (per_sm < 1) per_sm = 1;
   const int grid = groups < 148 * per_sm ? groups : 148 * per_sm;
   if (R == 4)
-    permute_cols_kernel<4><<<grid, PERMUTE_THREADS, smem, s>>>(dY, perm, T, I, dYp);
+    permute_cols_kernel<4><<<grid, threads, smem, s>>>(dY, perm, T, I, dYp);
   else
-    permute_cols_kernel<2><<<grid, PERMUTE_THREADS, smem, s>>>(dY, perm, T, I, dYp);
+    permute_cols_kernel<2><<<grid, threads, smem, s>>>(dY, perm, T, I, dYp);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
