@@ -261,11 +261,17 @@ int bimask_conv_layer_step(const bimask_conv_args* args);
  * `host` are ignored.
  *   bimask_layer_step_host        returns when the results are in host memory.
  *   bimask_layer_step_host_async  only enqueues: uploads, the step and downloads run on three
- *       queues (two copy streams owned by the library -- created with three events on the first
- *       call on a device, so make that call before any stream capture -- and `dev->stream`), so
- *       the upload of one call overlaps the download of the previous one.  The host buffers of a
- *       call must stay valid and untouched until bimask_host_sync() (or a later blocking call)
- *       has returned; work enqueued on dev->stream afterwards is ordered after the downloads. */
+ *       queues (two copy streams owned by the library -- created with their events on the first
+ *       call on a device, so make that call before any stream capture -- and `dev->stream`).  The
+ *       library remembers the device buffers of the last four calls and orders a new call only
+ *       behind earlier calls it shares device buffers with: a caller that alternates between two
+ *       or more sets of device buffers gets the upload of one call, the kernels of another and the
+ *       download of a third running at the same time (PCIe is full duplex); re-using one set
+ *       serialises upload -> kernels -> download -> next upload, which is always correct.
+ *       The host buffers of a call must stay valid and untouched until bimask_host_sync() (or a
+ *       later blocking call) has returned.  Work the caller enqueues on dev->stream afterwards is
+ *       ordered after this call's kernels but NOT after its downloads: do not overwrite the device
+ *       outputs with other work before bimask_host_sync(). */
 int bimask_layer_step_host(const bimask_layer_args* dev, const bimask_layer_args* host,
                            int32_t* host_status_word);
 int bimask_layer_step_host_async(const bimask_layer_args* dev, const bimask_layer_args* host,

@@ -478,10 +478,21 @@ int bimask_train_step(const bimask_train_args* a) {
 namespace bimask {
 
 // Copy streams and events of the host-buffer entry points, one set per device, created on first
-// use and kept until exit.
+// use and kept until exit.  The last four calls are remembered (which device buffers they read and
+// wrote, and their three events) so that a new call waits only for earlier calls it shares buffers
+// with: a caller that alternates between buffer sets gets uploads, kernels and downloads of
+// different calls running at the same time.
+struct HostSlot {
+  const void* in[4];                 // device buffers the upload writes: W, X, dY, perm
+  const void* out[12];               // device buffers the kernels write / the download reads
+  cudaEvent_t in_done = nullptr, compute_done = nullptr, out_done = nullptr;
+  cudaStream_t stream = nullptr;
+  bool used = false;
+};
 struct HostPipe {
   cudaStream_t in = nullptr, out = nullptr;
-  cudaEvent_t in_done = nullptr, compute_done = nullptr, out_done = nullptr;
+  HostSlot slots[4];
+  int next = 0;
   bool ready = false, used = false;
 };
 static std::mutex g_pipe_mutex;
@@ -496,13 +507,22 @@ static int get_pipe(HostPipe** out) {
   if (!p.ready) {
     BIMASK_CUDA_OK(cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking));
     BIMASK_CUDA_OK(cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking));
-    BIMASK_CUDA_OK(cudaEventCreateWithFlags(&p.in_done, cudaEventDisableTiming));
-    BIMASK_CUDA_OK(cudaEventCreateWithFlags(&p.compute_done, cudaEventDisableTiming));
-    BIMASK_CUDA_OK(cudaEventCreateWithFlags(&p.out_done, cudaEventDisableTiming));
+    for (HostSlot& sl : p.slots) {
+      BIMASK_CUDA_OK(cudaEventCreateWithFlags(&sl.in_done, cudaEventDisableTiming));
+      BIMASK_CUDA_OK(cudaEventCreateWithFlags(&sl.compute_done, cudaEventDisableTiming));
+      BIMASK_CUDA_OK(cudaEventCreateWithFlags(&sl.out_done, cudaEventDisableTiming));
+    }
     p.ready = true;
   }
   *out = &p;
   return BIMASK_OK;
+}
+
+static bool shares(const void* const* a, int na, const void* const* b, int nb) {
+  for (int i = 0; i < na; ++i)
+    for (int k = 0; k < nb; ++k)
+      if (a[i] != nullptr && a[i] == b[k]) return true;
+  return false;
 }
 
 }  // namespace bimask
@@ -519,17 +539,27 @@ int bimask_layer_step_host_async(const bimask_layer_args* d, const bimask_layer_
   cudaStream_t s = (cudaStream_t)d->stream;
   const size_t IJ = (size_t)d->I * d->J, TJ = (size_t)d->T * d->J, TI = (size_t)d->T * d->I;
   // Three queues: inputs go up on `in`, the step runs on the caller's stream, results come down
-  // on `out`.  Consecutive calls therefore overlap the upload of call n with the download of
-  // call n-1 (PCIe is full duplex).  Ordering kept conservative, whatever buffers the caller
-  // re-uses: an upload starts after the previous call's kernels are done, kernels start after
-  // the previous call's download.
-  if (p->used) {
-    BIMASK_CUDA_OK(cudaStreamWaitEvent(p->in, p->compute_done, 0));
-    BIMASK_CUDA_OK(cudaStreamWaitEvent(s, p->out_done, 0));
-  } else {
+  // on `out` (PCIe is full duplex).  An upload waits for the kernels of earlier calls that used the
+  // device buffers it overwrites; the kernels wait for their own upload and for the downloads of
+  // earlier calls that read the buffers they overwrite.
+  HostSlot* me = &p->slots[p->next];
+  const void* ins[4] = {d->W, d->X, d->dY, d->perm};
+  const void* outs[12] = {d->Y, d->dX, d->dW, d->perm, d->counts, d->best_idx, d->maskbits_f, d->maskbits_b,
+                          d->status_word, d->vals_f, d->vals_b, d->ws};
+  if (!p->used) {
     // order behind whatever the caller's stream already holds
-    BIMASK_CUDA_OK(cudaEventRecord(p->compute_done, s));
-    BIMASK_CUDA_OK(cudaStreamWaitEvent(p->in, p->compute_done, 0));
+    BIMASK_CUDA_OK(cudaEventRecord(me->compute_done, s));
+    BIMASK_CUDA_OK(cudaStreamWaitEvent(p->in, me->compute_done, 0));
+  }
+  for (HostSlot& o : p->slots) {
+    if (!o.used) continue;
+    const bool evicted = &o == me;                       // its record is about to be overwritten: depend on it
+    const bool in_hit = evicted || shares(ins, 4, o.in, 4) || shares(ins, 4, o.out, 12);
+    const bool out_hit = evicted || shares(outs, 12, o.out, 12) || shares(outs, 12, o.in, 4);
+    if (in_hit) BIMASK_CUDA_OK(cudaStreamWaitEvent(p->in, o.compute_done, 0));
+    if (in_hit && shares(ins, 4, o.out, 12)) BIMASK_CUDA_OK(cudaStreamWaitEvent(p->in, o.out_done, 0));
+    if (out_hit) BIMASK_CUDA_OK(cudaStreamWaitEvent(s, o.out_done, 0));
+    if ((in_hit || out_hit) && o.stream != s) BIMASK_CUDA_OK(cudaStreamWaitEvent(s, o.compute_done, 0));
   }
   BIMASK_CUDA_OK(cudaMemcpyAsync(const_cast<float*>(d->W), h->W, IJ * 4, cudaMemcpyHostToDevice, p->in));
   BIMASK_CUDA_OK(cudaMemcpyAsync(const_cast<uint16_t*>(d->X), h->X, TJ * 2, cudaMemcpyHostToDevice, p->in));
@@ -539,18 +569,23 @@ int bimask_layer_step_host_async(const bimask_layer_args* d, const bimask_layer_
   if (d->do_search && d->cands && h->cands)
     BIMASK_CUDA_OK(cudaMemcpyAsync(const_cast<int32_t*>(d->cands), h->cands, (size_t)d->P * d->I * 4,
                                    cudaMemcpyHostToDevice, p->in));
-  BIMASK_CUDA_OK(cudaMemsetAsync(d->status_word, 0, sizeof(int32_t), p->in));
-  BIMASK_CUDA_OK(cudaEventRecord(p->in_done, p->in));
-  BIMASK_CUDA_OK(cudaStreamWaitEvent(s, p->in_done, 0));
+  BIMASK_CUDA_OK(cudaEventRecord(me->in_done, p->in));
+  BIMASK_CUDA_OK(cudaStreamWaitEvent(s, me->in_done, 0));
+  BIMASK_CUDA_OK(cudaMemsetAsync(d->status_word, 0, sizeof(int32_t), s));
   rc = bimask_layer_step(d);
   // even when the step refused to launch, leave the queues in a consistent state
-  BIMASK_CUDA_OK(cudaEventRecord(p->compute_done, s));
+  BIMASK_CUDA_OK(cudaEventRecord(me->compute_done, s));
+  for (int i = 0; i < 4; ++i) me->in[i] = ins[i];
+  for (int i = 0; i < 12; ++i) me->out[i] = outs[i];
+  me->stream = s;
+  me->used = true;
   p->used = true;
+  p->next = (p->next + 1) % 4;
   if (rc != BIMASK_OK) {
-    BIMASK_CUDA_OK(cudaEventRecord(p->out_done, s));
+    BIMASK_CUDA_OK(cudaEventRecord(me->out_done, s));
     return rc;
   }
-  BIMASK_CUDA_OK(cudaStreamWaitEvent(p->out, p->compute_done, 0));
+  BIMASK_CUDA_OK(cudaStreamWaitEvent(p->out, me->compute_done, 0));
   cudaStream_t o = p->out;
   if (h->Y) BIMASK_CUDA_OK(cudaMemcpyAsync(h->Y, d->Y, TI * 2, cudaMemcpyDeviceToHost, o));
   if (h->dX) BIMASK_CUDA_OK(cudaMemcpyAsync(h->dX, d->dX, TJ * 2, cudaMemcpyDeviceToHost, o));
@@ -562,17 +597,16 @@ int bimask_layer_step_host_async(const bimask_layer_args* d, const bimask_layer_
   if (h->maskbits_f) BIMASK_CUDA_OK(cudaMemcpyAsync(h->maskbits_f, d->maskbits_f, IJ / 8, cudaMemcpyDeviceToHost, o));
   if (h->maskbits_b) BIMASK_CUDA_OK(cudaMemcpyAsync(h->maskbits_b, d->maskbits_b, IJ / 8, cudaMemcpyDeviceToHost, o));
   if (host_status_word) BIMASK_CUDA_OK(cudaMemcpyAsync(host_status_word, d->status_word, 4, cudaMemcpyDeviceToHost, o));
-  BIMASK_CUDA_OK(cudaEventRecord(p->out_done, o));
-  // the caller's stream is "done" with this call only once the results are down
-  BIMASK_CUDA_OK(cudaStreamWaitEvent(s, p->out_done, 0));
+  BIMASK_CUDA_OK(cudaEventRecord(me->out_done, o));
   return BIMASK_OK;
 }
 
+// Waits until every download enqueued so far on this device is in host memory.
 int bimask_host_sync(void) {
   HostPipe* p = nullptr;
   int rc = get_pipe(&p);
   if (rc != BIMASK_OK) return rc;
-  if (p->used) BIMASK_CUDA_OK(cudaEventSynchronize(p->out_done));
+  if (p->used) BIMASK_CUDA_OK(cudaStreamSynchronize(p->out));
   return BIMASK_OK;
 }
 

@@ -431,3 +431,47 @@ def test_large_operand_sparse_kernel_ragged_shapes(I, J, T):
     assert np.array_equal(u32(b["maskbits_b"]), O.pack_bits(Bbar))
     assert rel_err(b["Y"].float().cpu().numpy(), O.spmm_fwd(X, W, B)) <= TOL
     assert rel_err(b["dX"].float().cpu().numpy(), O.spmm_dgrad(dY, W, O.unpermute_rows(Bbar, perm))) <= TOL
+
+
+def test_async_host_calls_with_alternating_buffer_sets():
+    """Three device buffer sets used in turn, ten calls in flight before one wait, every call with its own
+    inputs and its own host outputs: uploads, kernels and downloads of different calls overlap, and a set
+    that comes round again must wait for the call that used it last.  Every result equals the blocking one."""
+    shapes = [(1024, 1536, 900), (1536, 1024, 700), (2048, 512, 1100)]
+    N, P = 2, 4
+    sets, refs, outs = [], [], []
+    for k, (I, J, T) in enumerate(shapes):
+        b = bm.alloc_layer_buffers(T, I, J, P)
+        b["W"] = torch.empty(I, J, device="cuda")
+        b["X"] = torch.empty(T, J, dtype=torch.bfloat16, device="cuda")
+        b["dY"] = torch.empty(T, I, dtype=torch.bfloat16, device="cuda")
+        sets.append(b)
+    calls = []
+    for c in range(10):
+        k = c % 3
+        I, J, T = shapes[k]
+        W = inputs.make_weight(I, J, 700 + c)
+        X = inputs.make_activation(T, J, 800 + c)
+        dY = inputs.make_activation(T, I, 900 + c)
+        host = {"W": torch.from_numpy(W).pin_memory(),
+                "X": torch.from_numpy(X.view(np.int16)).view(torch.bfloat16).pin_memory(),
+                "dY": torch.from_numpy(dY.view(np.int16)).view(torch.bfloat16).pin_memory(),
+                "Y": torch.zeros(T, I, dtype=torch.bfloat16).pin_memory(),
+                "dX": torch.zeros(T, J, dtype=torch.bfloat16).pin_memory(),
+                "dW": torch.zeros(I, J, dtype=torch.float32).pin_memory(),
+                "perm": torch.zeros(I, dtype=torch.int32).pin_memory(),
+                "counts": torch.zeros(P, dtype=torch.int64).pin_memory()}
+        calls.append((k, W, X, dY, host, torch.full((1,), -9, dtype=torch.int32).pin_memory()))
+    for c, (k, W, X, dY, host, hst) in enumerate(calls):
+        I, J, T = shapes[k]
+        bm.bimask_layer_step_host_async(bm.make_layer_args(T, I, J, N, 4, P, 50 + c, True, sets[k]),
+                                        bm.make_layer_args(T, I, J, N, 4, P, 50 + c, True, host), hst)
+    bm.bimask_host_sync()
+    for c, (k, W, X, dY, host, hst) in enumerate(calls):
+        ref = run_layer_step(W, X, dY, N, 4, P, 50 + c, do_search=True)
+        assert int(hst.item()) == 0, c
+        assert torch.equal(host["perm"], ref["perm"].cpu()), c
+        assert torch.equal(host["counts"], ref["counts"].cpu()), c
+        assert torch.equal(host["Y"], ref["Y"].cpu()), c
+        assert torch.equal(host["dX"], ref["dX"].cpu()), c
+        assert torch.equal(host["dW"], ref["dW"].cpu()), c
