@@ -351,6 +351,13 @@ def test_candidates_are_permutations_and_uniform():
     assert [k & 0xFFFFFF for k in keys] == list(O.candidates(seed, 3, I)[2])
 
 
+def test_candidates_match_the_independent_test_vector():
+    """Seed 42, I = 8: the first three candidates as computed, independently of this oracle, from the written
+    definition of the generator when the interface was drawn up."""
+    want = [[5, 4, 2, 3, 7, 0, 1, 6], [2, 5, 6, 7, 0, 1, 3, 4], [7, 0, 2, 1, 5, 4, 6, 3]]
+    assert O.candidates(42, 3, 8).tolist() == want
+
+
 def test_layer_step_identity_when_not_searching():
     W, X, dY = inputs.make_layer(1, 0, T=8)
     out = O.layer_step(W, X, dY, 2, 4, 8, 43, do_search=False)
