@@ -40,7 +40,8 @@ Readings of points the paper leaves open (listed again in the design notes):
 Parity unpinned: the pseudo-random candidate generator (`candidates`).  The
 paper only says the K candidates are random; the generator below is this
 build's contract (its mixing function is pinned to the published SplitMix64
-test vector, the rest by permutation validity and a uniformity test).
+test vector, the rest by permutation validity, a uniformity test and a
+three-candidate vector computed independently from the written definition).
 """
 from __future__ import annotations
 
