@@ -623,3 +623,66 @@ def test_conv_equals_the_linear_layer_on_the_column_matrix():
         for kw in range(3):
             dx[:, kh:kh + H, kw:kw + Wd, :] += dXcol[:, :, :, kh * 3 + kw, :]
     assert np.allclose(got["dx"], dx[:, 1:-1, 1:-1, :], rtol=1e-12, atol=1e-12)
+
+
+# ---------------------------------------------------------------- greedy refinement of the permutation
+def test_refine_perm_never_loses_and_matches_a_recount():
+    """Every round's accepted swaps are re-derived here by brute force (full recount of the eligible blocks for
+    each proposed swap), and the total must equal the sum of the accepted gains."""
+    rng = np.random.default_rng(51)
+    for (N, M, I, J) in [(2, 4, 32, 64), (1, 4, 32, 32), (2, 8, 64, 32)]:
+        W = rng.standard_normal((I, J)).astype(np.float32)
+        B = O.forward_mask(W, N, M)
+        perm0 = rng.permutation(I).astype(np.int32)
+        seed = 9
+        counts = [O.eligible_blocks(B, perm0, N, M)]
+        perm = perm0.copy()
+        for r in range(1, 5):
+            got, cnt = O.refine_perm(B, perm0, N, M, r, seed)
+            assert np.array_equal(np.sort(got), np.arange(I)) and cnt == O.eligible_blocks(B, got, N, M)
+            # one more round, by hand, from the previous result
+            order = O.candidates(seed + O.REFINE_SEED_OFFSET, r, I)[r - 1]
+            base = O.eligible_blocks(B, perm, N, M)
+            cand = []
+            for i in range(I // 2):
+                a, b = int(order[2 * i]), int(order[2 * i + 1])
+                if a // M == b // M:
+                    continue
+                q = perm.copy()
+                q[a], q[b] = q[b], q[a]
+                g = O.eligible_blocks(B, q, N, M) - base
+                if g > 0:
+                    cand.append((g, -i, a, b))
+            accepted, nxt = [], perm.copy()
+            for (g, ni, a, b) in cand:
+                rivals = [c for c in cand if {c[2] // M, c[3] // M} & {a // M, b // M}]
+                if all((g, ni) >= (c[0], c[1]) for c in rivals):
+                    accepted.append(g)
+                    nxt[a], nxt[b] = nxt[b], nxt[a]
+            assert np.array_equal(nxt, got), (N, M, r)
+            assert cnt == base + sum(accepted)
+            counts.append(cnt)
+            perm = nxt
+        assert all(y >= x for x, y in zip(counts, counts[1:])) and counts[-1] > counts[0]
+
+
+def test_refine_perm_fixed_point_and_improvement():
+    # a permutation that already makes every block eligible cannot be improved
+    W, Q = inputs.planted_transposable(64, 32, 2, 4, 3)
+    B = O.forward_mask(W, 2, 4)
+    assert O.eligible_blocks(B, Q, 2, 4) == (64 // 4) * 32
+    got, cnt = O.refine_perm(B, Q, 2, 4, 6, 1)
+    assert np.array_equal(got, Q) and cnt == 16 * 32
+    # zero rounds: unchanged
+    p = np.random.default_rng(1).permutation(64).astype(np.int32)
+    got, cnt = O.refine_perm(B, p, 2, 4, 0, 1)
+    assert np.array_equal(got, p)
+    # i.i.d. weights: best-of-K sits at 11/16 of the blocks; hill climbing clearly beats it
+    rng = np.random.default_rng(2)
+    W = rng.standard_normal((128, 128)).astype(np.float32)
+    B = O.forward_mask(W, 2, 4)
+    best, perm, counts = O.perm_search(B, O.candidates(7, 16, 128), 2, 4)
+    got, cnt = O.refine_perm(B, perm, 2, 4, 24, 7)
+    total = (128 // 4) * 128
+    assert abs(counts.mean() / total - 11 / 16) < 0.02
+    assert cnt / total > 0.73 and cnt > counts.max() + 0.02 * total
