@@ -20,7 +20,8 @@ EXPORTS = ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "
            "bimask_layer_step", "bimask_layer_step_host", "bimask_layer_step_host_async", "bimask_host_sync",
            "bimask_check_perms", "bimask_debug_wait_probe", "bimask_perm_search_static",
            "bimask_perm_search_static_max_entries", "bimask_sgd_fwd_mask", "bimask_train_step",
-           "bimask_bwd_mask_criterion", "bimask_conv_workspace_bytes", "bimask_conv_layer_step")
+           "bimask_bwd_mask_criterion", "bimask_conv_workspace_bytes", "bimask_conv_layer_step",
+           "bimask_refine_workspace_bytes", "bimask_perm_refine")
 
 
 class BimaskError(RuntimeError):
@@ -84,6 +85,10 @@ def lib() -> ctypes.CDLL:
         L.bimask_layer_step_host.argtypes = [POINTER(LayerArgs), POINTER(LayerArgs), c_void_p]
         L.bimask_layer_step_host_async.argtypes = [POINTER(LayerArgs), POINTER(LayerArgs), c_void_p]
         L.bimask_host_sync.argtypes = []
+        L.bimask_refine_workspace_bytes.restype = c_size_t
+        L.bimask_refine_workspace_bytes.argtypes = [c_int, c_int, c_int]
+        L.bimask_perm_refine.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_uint64, c_void_p, c_void_p, c_void_p,
+                                         c_size_t, c_void_p]
         L.bimask_conv_workspace_bytes.restype = c_size_t
         L.bimask_conv_workspace_bytes.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int]
         L.bimask_conv_layer_step.argtypes = [POINTER(ConvArgs)]
@@ -100,7 +105,8 @@ def lib() -> ctypes.CDLL:
         for name in EXPORTS:
             if name not in ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "bimask_workspace_bytes",
                             "bimask_perm_search_static_max_entries", "bimask_sgd_fwd_mask", "bimask_train_step",
-           "bimask_bwd_mask_criterion", "bimask_conv_workspace_bytes", "bimask_conv_layer_step"):
+           "bimask_bwd_mask_criterion", "bimask_conv_workspace_bytes", "bimask_conv_layer_step",
+           "bimask_refine_workspace_bytes", "bimask_perm_refine"):
                 getattr(L, name).restype = c_int
         _lib = L
     return _lib
@@ -166,6 +172,15 @@ def bimask_bwd_mask(W, maskbits_f, perm, I, J, N, M, maskbits_b, vals_b, meta_b,
 
 
 CRIT_WEIGHT, CRIT_SCORE, CRIT_MULTINOMIAL, CRIT_RANDOM = 0, 1, 2, 3
+
+
+def bimask_refine_workspace_bytes(I, M, rounds) -> int:
+    return lib().bimask_refine_workspace_bytes(I, M, rounds)
+
+
+def bimask_perm_refine(maskbits_f, I, J, N, M, rounds, seed, perm_inout, count_out, ws, ws_bytes, stream=None):
+    return _check(lib().bimask_perm_refine(_ptr(maskbits_f), I, J, N, M, rounds, seed, _ptr(perm_inout), _ptr(count_out),
+                                           _ptr(ws), ws_bytes, _stream(stream)))
 
 
 def bimask_bwd_mask_criterion(W, S_or_null, maskbits_f, perm, I, J, N, M, criterion, seed, maskbits_b, vals_b, meta_b,

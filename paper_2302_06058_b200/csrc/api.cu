@@ -103,6 +103,45 @@ int bimask_fwd_mask(const float* W, int I, int J, int N, int M, uint32_t* maskbi
   return fused ? BIMASK_OK : launch_hw_meta(meta_f, I, J, hw_meta_f, s);
 }
 
+size_t bimask_refine_workspace_bytes(int I, int M, int rounds) {
+  if (I <= 0 || rounds < 0 || (M != 4 && M != 8 && M != 16)) return 0;
+  return align_up((size_t)rounds * I * sizeof(int32_t), 256) + align_up((size_t)(I / 2) * sizeof(int32_t), 256) +
+         align_up((size_t)(I / M) * sizeof(unsigned long long), 256);
+}
+
+int bimask_perm_refine(const uint32_t* maskbits_f, int I, int J, int N, int M, int rounds, uint64_t seed,
+                       int32_t* perm_inout, int64_t* count_out, void* ws, size_t ws_bytes, void* stream) {
+  BIMASK_REQUIRE(M == 4 || M == 8 || M == 16, BIMASK_EUNSUPPORTED, "M = %d: block lengths 4, 8 and 16 are implemented", M);
+  BIMASK_REQUIRE(I > 0 && J > 0 && I % M == 0 && I % 2 == 0 && J % 32 == 0, BIMASK_EINVAL,
+                 "I = %d, J = %d: I must be a positive even multiple of M, J of 32", I, J);
+  BIMASK_REQUIRE(N >= 1 && N <= M, BIMASK_EINVAL, "N = %d out of range 1..%d", N, M);
+  BIMASK_REQUIRE(N <= 4 && (M != 4 || N <= 2), BIMASK_EUNSUPPORTED, "N:M = %d:%d: the refinement counts blocks for N <= 4 (N <= 2 at M = 4)", N, M);
+  BIMASK_REQUIRE(rounds >= 0 && rounds <= 4096, BIMASK_EINVAL, "rounds = %d out of range 0..4096", rounds);
+  BIMASK_REQUIRE(I < (1 << 24), BIMASK_EUNSUPPORTED, "the pairing generator needs I < 2^24 (I = %d)", I);
+  BIMASK_REQUIRE(maskbits_f && perm_inout && ws, BIMASK_EINVAL, "bimask_perm_refine: null pointer");
+  BIMASK_REQUIRE(aligned16(maskbits_f) && aligned16(perm_inout) && aligned16(ws) && (!count_out || (uintptr_t)count_out % 8 == 0),
+                 BIMASK_EINVAL, "bimask_perm_refine: misaligned pointer");
+  const size_t need = bimask_refine_workspace_bytes(I, M, rounds);
+  BIMASK_REQUIRE(ws_bytes >= need, BIMASK_EINVAL, "bimask_perm_refine: workspace too small (%zu bytes, need %zu)", ws_bytes, need);
+  cudaStream_t s = (cudaStream_t)stream;
+  uint8_t* w8 = reinterpret_cast<uint8_t*>(ws);
+  int32_t* orders = reinterpret_cast<int32_t*>(w8);
+  int32_t* gains = reinterpret_cast<int32_t*>(w8 + align_up((size_t)rounds * I * sizeof(int32_t), 256));
+  unsigned long long* best = reinterpret_cast<unsigned long long*>(reinterpret_cast<uint8_t*>(gains) +
+                                                                   align_up((size_t)(I / 2) * sizeof(int32_t), 256));
+  int rc;
+  if (rounds > 0) {
+    // the random pairings of all rounds: `rounds` permutations of the positions, same generator as the candidates
+    if ((rc = launch_gen_candidates(seed + 0x5EED5EEDull, rounds, I, orders, s)) != BIMASK_OK) return rc;
+    if ((rc = launch_refine(maskbits_f, I, J, N, M, rounds, orders, perm_inout, gains, best, s)) != BIMASK_OK) return rc;
+  }
+  if (count_out) {
+    if (M == 4) return launch_score(maskbits_f, perm_inout, I, J, N, 1, count_out, s);
+    return launch_score_generic(maskbits_f, perm_inout, I, J, N, M, 1, count_out, s);
+  }
+  return BIMASK_OK;
+}
+
 int bimask_sgd_fwd_mask(float* W, const float* dW, float* mom, int I, int J, int N, int M, float lr, float momentum,
                         float weight_decay, uint32_t* maskbits_f, uint16_t* vals_f, uint32_t* meta_f, void* hw_meta_f,
                         void* stream) {

@@ -69,6 +69,8 @@ int launch_bwd_mask_generic(const float* W, const uint32_t* maskbits_f, const in
 int launch_bwd_mask_criterion(const float* W, const float* S, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                               int N, int M, int crit, uint64_t seed, uint32_t* maskbits_b, uint16_t* vals_b_or_null,
                               uint32_t* meta_b_or_null, int mode, cudaStream_t s);
+int launch_refine(const uint32_t* bits, int I, int J, int N, int M, int rounds, const int32_t* orders, int32_t* perm,
+                  int32_t* gains, unsigned long long* block_best, cudaStream_t s);
 int launch_check_perms(const int32_t* cands, int P, int I, int32_t* ok, uint8_t* seen, cudaStream_t s);
 int launch_wait_probe(int32_t* status_word, cudaStream_t s);
 int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, uint16_t* dYp, cudaStream_t s);

@@ -186,6 +186,90 @@ score_generic_kernel(const uint32_t* __restrict__ bits, const int32_t* __restric
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// Greedy refinement of a permutation by pairwise swaps (hill climbing on the eligible-block
+// count; not part of the paper's Algorithm 1, which stops at the best random candidate).
+// A round pairs the positions of the permutation at random: pair i = (order[2i], order[2i+1]).
+// gain kernel: one warp per pair; lanes stride over the 32-column words; for each word the M
+// mask words of both row blocks are loaded once and the eligible columns counted before and after
+// exchanging the two rows.  A pair with positive gain bids for both of its blocks with
+// (gain << 32 | ~pair index) through a 64-bit atomic maximum.
+// apply kernel: a pair that won BOTH of its blocks exchanges its two entries of perm; winners never
+// share a block, so their gains add up and a round never lowers the count.
+// ---------------------------------------------------------------------------------------
+template <int N, int M>
+__global__ void __launch_bounds__(256)
+refine_gain_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ perm, const int32_t* __restrict__ order,
+                   int I, int jwords, int32_t* __restrict__ gains, unsigned long long* __restrict__ block_best) {
+  const int lane = threadIdx.x & 31;
+  const int pair = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (pair >= (I >> 1)) return;
+  const int a = __ldg(order + 2 * pair), b = __ldg(order + 2 * pair + 1);
+  const int ka = a / M, kb = b / M;
+  if (ka == kb) {
+    if (lane == 0) gains[pair] = 0;
+    return;
+  }
+  const unsigned last_row = (unsigned)(I - 1);
+  int ra[M], rb[M];
+#pragma unroll
+  for (int m = 0; m < M; ++m) {
+    ra[m] = (int)min((unsigned)__ldg(perm + ka * M + m), last_row);
+    rb[m] = (int)min((unsigned)__ldg(perm + kb * M + m), last_row);
+  }
+  const int ma = a - ka * M, mb = b - kb * M;
+  int gain = 0;
+  for (int q = lane; q < jwords; q += 32) {
+    uint32_t wa[M], wb[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+      wa[m] = __ldg(bits + (long long)ra[m] * jwords + q);
+      wb[m] = __ldg(bits + (long long)rb[m] * jwords + q);
+    }
+    uint32_t xa = 0, xb = 0;                                 // the two rows that change places
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+      xa = m == ma ? wa[m] : xa;
+      xb = m == mb ? wb[m] : xb;
+    }
+    SatCount<N> s0, s1, s2, s3;
+    s0.clear(); s1.clear(); s2.clear(); s3.clear();
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+      s0.add(wa[m]);
+      s1.add(wb[m]);
+      s2.add(m == ma ? xb : wa[m]);
+      s3.add(m == mb ? xa : wb[m]);
+    }
+    gain += __popc(s2.eligible()) + __popc(s3.eligible()) - __popc(s0.eligible()) - __popc(s1.eligible());
+  }
+  gain = __reduce_add_sync(0xFFFFFFFFu, gain);
+  if (lane == 0) {
+    gains[pair] = gain;
+    if (gain > 0) {
+      const unsigned long long key = ((unsigned long long)(unsigned)gain << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned)pair);
+      atomicMax(block_best + ka, key);
+      atomicMax(block_best + kb, key);
+    }
+  }
+}
+
+template <int M>
+__global__ void refine_apply_kernel(const int32_t* __restrict__ order, const int32_t* __restrict__ gains,
+                                    const unsigned long long* __restrict__ block_best, int I, int32_t* __restrict__ perm) {
+  const int pair = blockIdx.x * blockDim.x + threadIdx.x;
+  if (pair >= (I >> 1)) return;
+  const int gain = gains[pair];
+  if (gain <= 0) return;
+  const int a = __ldg(order + 2 * pair), b = __ldg(order + 2 * pair + 1);
+  const unsigned long long key = ((unsigned long long)(unsigned)gain << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned)pair);
+  if (block_best[a / M] == key && block_best[b / M] == key) {
+    const int32_t pa = perm[a], pb = perm[b];
+    perm[a] = pb;
+    perm[b] = pa;
+  }
+}
+
 __global__ void fill_counts_kernel(long long* counts, int P, long long v) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < P) counts[i] = v;
@@ -411,6 +495,46 @@ int launch_bwd_mask_criterion(const float* W, const float* S, const uint32_t* ma
   else launch_bwd_m<16>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, s);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
+template <int N, int M>
+static void refine_round(const uint32_t* bits, int32_t* perm, const int32_t* order, int I, int J, int32_t* gains,
+                         unsigned long long* block_best, cudaStream_t s) {
+  const int pairs = I / 2;
+  refine_gain_kernel<N, M><<<(pairs + 7) / 8, 256, 0, s>>>(bits, perm, order, I, J / 32, gains, block_best);
+  refine_apply_kernel<M><<<(pairs + 255) / 256, 256, 0, s>>>(order, gains, block_best, I, perm);
+}
+
+// rounds of greedy pairwise swaps on perm (in place).  orders: rounds x I position permutations; scratch:
+// gains (I / 2 ints) and block_best (I / M 64-bit words, zeroed here before every round).
+int launch_refine(const uint32_t* bits, int I, int J, int N, int M, int rounds, const int32_t* orders, int32_t* perm,
+                  int32_t* gains, unsigned long long* block_best, cudaStream_t s) {
+  for (int r = 0; r < rounds; ++r) {
+    BIMASK_CUDA_OK(cudaMemsetAsync(block_best, 0, (size_t)(I / M) * sizeof(unsigned long long), s));
+    const int32_t* order = orders + (size_t)r * I;
+    if (M == 4) {
+      if (N == 1) refine_round<1, 4>(bits, perm, order, I, J, gains, block_best, s);
+      else refine_round<2, 4>(bits, perm, order, I, J, gains, block_best, s);
+    } else if (M == 8) {
+      switch (N) {
+        case 1: refine_round<1, 8>(bits, perm, order, I, J, gains, block_best, s); break;
+        case 2: refine_round<2, 8>(bits, perm, order, I, J, gains, block_best, s); break;
+        case 3: refine_round<3, 8>(bits, perm, order, I, J, gains, block_best, s); break;
+        default: refine_round<4, 8>(bits, perm, order, I, J, gains, block_best, s); break;
+      }
+    } else {
+      switch (N) {
+        case 1: refine_round<1, 16>(bits, perm, order, I, J, gains, block_best, s); break;
+        case 2: refine_round<2, 16>(bits, perm, order, I, J, gains, block_best, s); break;
+        case 3: refine_round<3, 16>(bits, perm, order, I, J, gains, block_best, s); break;
+        default: refine_round<4, 16>(bits, perm, order, I, J, gains, block_best, s); break;
+      }
+    }
+    count_launch();
+    count_launch();
+    BIMASK_CUDA_OK(cudaGetLastError());
+  }
   return BIMASK_OK;
 }
 

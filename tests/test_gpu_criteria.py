@@ -106,3 +106,70 @@ def test_random_and_multinomial_statistics_at_scale():
     for c in out:
         assert not (out[c] & ~Bp).any()
         assert np.array_equal(out[c].reshape(I // M, M, J).sum(axis=1), np.minimum(comp, N))
+
+
+# ---------------------------------------------------------------------------------------------
+# Greedy refinement of the permutation (bimask_perm_refine)
+# ---------------------------------------------------------------------------------------------
+def _refine_gpu(B, perm, N, M, rounds, seed):
+    I, J = B.shape
+    bits = dev(O.pack_bits(B).view(np.int32))
+    p = dev(np.asarray(perm, dtype=np.int32))
+    cnt = torch.zeros(1, dtype=torch.int64, device="cuda")
+    nbytes = bm.bimask_refine_workspace_bytes(I, M, rounds)
+    ws = torch.empty(max(nbytes, 16), dtype=torch.uint8, device="cuda")
+    bm.bimask_perm_refine(bits, I, J, N, M, rounds, seed, p, cnt, ws, ws.numel())
+    torch.cuda.synchronize()
+    return p.cpu().numpy(), int(cnt.item())
+
+
+@pytest.mark.parametrize("I,J,N,M,rounds", [(256, 256, 2, 4, 8), (128, 512, 1, 4, 5), (256, 128, 2, 8, 6),
+                                            (128, 64, 1, 16, 4), (64, 96, 4, 8, 3), (96, 160, 2, 4, 7), (64, 64, 2, 4, 0)])
+def test_perm_refine_bit_exact(I, J, N, M, rounds):
+    rng = np.random.default_rng(I + J + N + M)
+    W = rng.standard_normal((I, J)).astype(np.float32)
+    B = O.forward_mask(W, N, M)
+    perm0 = rng.permutation(I).astype(np.int32)
+    seed = 1000 + rounds
+    got, cnt = _refine_gpu(B, perm0, N, M, rounds, seed)
+    ref, ref_cnt = O.refine_perm(B, perm0, N, M, rounds, seed)
+    assert np.array_equal(got, ref)
+    assert cnt == ref_cnt
+    assert cnt >= O.eligible_blocks(B, perm0, N, M)
+
+
+def test_perm_refine_at_scale_properties():
+    """Too large for the oracle's loops: the result is a permutation, the count equals an independent score of
+    the result, grows with the number of rounds and beats the best of the random candidates."""
+    I, J, N, M, P = 4096, 2048, 2, 4, 64
+    rng = np.random.default_rng(4)
+    W = rng.standard_normal((I, J)).astype(np.float32)
+    B = O.forward_mask(W, N, M)
+    bits = dev(O.pack_bits(B).view(np.int32))
+    b = bm.alloc_layer_buffers(1, I, J, P)
+    bm.bimask_perm_search(bits, I, J, N, M, P, 7, None, b["perm"], b["best_idx"], b["counts"], b["ws"], b["ws"].numel())
+    torch.cuda.synchronize()
+    start = b["perm"].cpu().numpy()
+    best_random = int(b["counts"].max().item())
+    prev = best_random
+    for rounds in (4, 16, 48):
+        got, cnt = _refine_gpu(B, start, N, M, rounds, 3)
+        assert np.array_equal(np.sort(got), np.arange(I))
+        assert cnt == O.eligible_blocks(B, got, N, M)
+        assert cnt > prev
+        prev = cnt
+    total = (I // M) * J
+    assert best_random / total < 0.70 and prev / total > best_random / total + 0.005
+
+
+def test_perm_refine_rejects_bad_arguments():
+    bits = torch.zeros(64, 2, dtype=torch.int32, device="cuda")
+    p = torch.arange(64, dtype=torch.int32, device="cuda")
+    ws = torch.empty(1 << 16, dtype=torch.uint8, device="cuda")
+    n0 = bm.bimask_launch_count()
+    for kw in (dict(rounds=-1), dict(N=3), dict(ws_bytes=8), dict(M=32)):
+        a = dict(I=64, J=64, N=2, M=4, rounds=2, ws_bytes=ws.numel())
+        a.update(kw)
+        with pytest.raises(bm.BimaskError):
+            bm.bimask_perm_refine(bits, a["I"], a["J"], a["N"], a["M"], a["rounds"], 1, p, None, ws, a["ws_bytes"])
+    assert bm.bimask_launch_count() == n0

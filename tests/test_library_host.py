@@ -73,6 +73,10 @@ def test_validation_happens_before_any_cuda_call(bm):
     assert L.bimask_layer_step(None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_train_step(None) == bm.binding.BIMASK_EINVAL
     assert L.bimask_conv_layer_step(None) == bm.binding.BIMASK_EINVAL
+    assert L.bimask_perm_refine(16, 64, 64, 2, 4, 2, 1, 16, None, None, 1 << 20, None) == bm.binding.BIMASK_EINVAL
+    assert L.bimask_perm_refine(16, 64, 64, 2, 4, 2, 1, 16, None, 16, 8, None) == bm.binding.BIMASK_EINVAL
+    assert L.bimask_perm_refine(16, 64, 64, 5, 8, 2, 1, 16, None, 16, 1 << 20, None) == bm.binding.BIMASK_EUNSUPPORTED
+    assert bm.bimask_refine_workspace_bytes(16384, 4, 32) >= 32 * 16384 * 4 + 8192 * 4 + 4096 * 8
     assert bm.bimask_conv_workspace_bytes(32, 56, 56, 64, 64, 100) > 2 * 32 * 56 * 56 * 576 * 2
     assert bm.bimask_conv_workspace_bytes(0, 56, 56, 64, 64, 100) == 0
     assert L.bimask_bwd_mask_criterion(16, None, 16, 16, 64, 64, 2, 4, 7, 0, 16, 16, 16, 16, None) == bm.binding.BIMASK_EINVAL
