@@ -104,9 +104,8 @@ def lib() -> ctypes.CDLL:
         L.bimask_perm_search_static_max_entries.restype = c_size_t
         for name in EXPORTS:
             if name not in ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "bimask_workspace_bytes",
-                            "bimask_perm_search_static_max_entries", "bimask_sgd_fwd_mask", "bimask_train_step",
-           "bimask_bwd_mask_criterion", "bimask_conv_workspace_bytes", "bimask_conv_layer_step",
-           "bimask_refine_workspace_bytes", "bimask_perm_refine"):
+                            "bimask_perm_search_static_max_entries", "bimask_conv_workspace_bytes",
+                            "bimask_refine_workspace_bytes"):
                 getattr(L, name).restype = c_int
         _lib = L
     return _lib
