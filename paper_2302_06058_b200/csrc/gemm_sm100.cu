@@ -1206,7 +1206,7 @@ int set_smem_attr(K kernel, int bytes) {
 }
 
 template <int N_TILE, int STAGES, bool SPARSE = true>
-int run_sparse(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim, int Kdim,
+int run_single(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim, int Kdim,
                uint16_t* out, int32_t* status_word, cudaStream_t s) {
   using C = Cfg<N_TILE, STAGES, SPARSE>;
   CUtensorMap ta, tb;
@@ -1349,8 +1349,8 @@ int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, 
   if (Ndim >= 1024 && Mdim >= 2048 && Kdim >= 4096)
     return run_sparse_pair2m(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   if (Ndim > 128 && Mdim > 128) return run_sparse_pair_persistent(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
-  if (Ndim > 128) return run_sparse<256, 2>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
-  return run_sparse<128, 4>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
+  if (Ndim > 128) return run_single<256, 2>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
+  return run_single<128, 4>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
 }
 
 namespace {
@@ -1470,8 +1470,8 @@ int launch_spmm_conv(int mode, const uint16_t* vals, const void* hw_meta, const 
 
 int launch_dense_nt(const uint16_t* A, const uint16_t* Bop, int Mdim, int Ndim, int Kdim, uint16_t* out,
                     int32_t* status_word, cudaStream_t s) {
-  if (Ndim > 128) return run_sparse<256, 2, false>(A, nullptr, Bop, Mdim, Ndim, Kdim, out, status_word, s);
-  return run_sparse<128, 3, false>(A, nullptr, Bop, Mdim, Ndim, Kdim, out, status_word, s);
+  if (Ndim > 128) return run_single<256, 2, false>(A, nullptr, Bop, Mdim, Ndim, Kdim, out, status_word, s);
+  return run_single<128, 3, false>(A, nullptr, Bop, Mdim, Ndim, Kdim, out, status_word, s);
 }
 
 int launch_wait_probe(int32_t* status_word, cudaStream_t s) {
