@@ -291,7 +291,9 @@ int bimask_conv_layer_step(const bimask_conv_args* args);
  *       The host buffers of a call must stay valid and untouched until bimask_host_sync() (or a
  *       later blocking call) has returned.  Work the caller enqueues on dev->stream afterwards is
  *       ordered after this call's kernels but NOT after its downloads: do not overwrite the device
- *       outputs with other work before bimask_host_sync(). */
+ *       outputs with other work before bimask_host_sync().  The host-buffer entry points keep
+ *       per-device state (copy streams, the record of recent calls): call them from one host
+ *       thread per device at a time.  The device-pointer entry points have no such state. */
 int bimask_layer_step_host(const bimask_layer_args* dev, const bimask_layer_args* host,
                            int32_t* host_status_word);
 int bimask_layer_step_host_async(const bimask_layer_args* dev, const bimask_layer_args* host,
