@@ -952,6 +952,184 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_consta
 }
 
 // ------------------------------------------------------------------------------------------
+// Dense weight gradient, one CTA per 128 x 256 tile: for layers of at most 128 output rows the
+// pair kernel above would leave half of every 256-row MMA tile empty.  Same pipeline without the
+// cluster: 16 KB of dY^T and 32 KB of X per stage, tcgen05.mma.cta_group::1 128 x 256 x 16, two
+// accumulators in tensor memory, persistent over (tile, k-split) work items.
+// ------------------------------------------------------------------------------------------
+template <int STAGES>
+struct WgradSingleCfg {
+  static constexpr int A_BYTES = 16384, B_BYTES = 32768;     // 128 and 256 columns x 64 tokens, 64-wide boxes
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int TMEM_COLS = 512;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+};
+
+template <int STAGES, bool CONV>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+wgrad_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
+                    const GemmParams p, int splits) {
+  using C = WgradSingleCfg<STAGES>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = ptx::smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - raw);
+  const uint32_t bar_base = base + STAGES * C::STAGE_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tmem_full_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
+  auto tmem_empty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * C::STAGE_BYTES + 8 * (2 * STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_tiles = p.tiles_m * p.tiles_n;            // tiles_m counts 128-row tiles
+  const int num_items = num_tiles * splits;
+  const int k_tiles_total = (p.Kdim + 63) / 64;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(tmem_full_bar(b), 1);
+      ptx::mbar_init(tmem_empty_bar(b), 4);               // four epilogue warps
+    }
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmapA);
+    ptx::prefetch_tmap(&tmapB);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  auto item_coords = [&](int item, int& m0, int& n0, int& kt0, int& nkt, int& split) {
+    const int tile = item % num_tiles;
+    split = item / num_tiles;
+    int tile_m, tile_n;
+    raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
+    m0 = tile_m * 128;
+    n0 = tile_n * 256;
+    kt0 = split * p.k_tiles_per_split;
+    nkt = min(k_tiles_total, kt0 + p.k_tiles_per_split) - kt0;
+  };
+
+  if (warp == 0) {
+    if (ptx::elect_one()) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+        int m0, n0, kt0, nkt, split;
+        item_coords(item, m0, n0, kt0, nkt, split);
+        for (int kt = kt0; kt < kt0 + nkt; ++kt, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; ok = false; break; }
+          const uint32_t a_s = base + s * C::STAGE_BYTES;
+          const uint32_t b_s = a_s + C::A_BYTES;
+          ptx::mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
+          if (CONV) {
+            int cw0, ch0, cn0;
+            conv_box_origin(p.conv, kt, cw0, ch0, cn0);
+            ptx::tma_load_4d(a_s, &tmapA, m0, cw0, ch0, cn0, full_bar(s));
+            ptx::tma_load_4d(a_s + 8192, &tmapA, m0 + 64, cw0, ch0, cn0, full_bar(s));
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const int j = n0 + 64 * q;                   // first of 64 columns of dW: one tap, 64 channels
+              const bool valid = j < p.Ndim;
+              const int tap = j / p.conv.CB;
+              ptx::tma_load_4d(b_s + q * 8192, &tmapB, valid ? j - tap * p.conv.CB : 0, cw0 + tap % 3 - 1, ch0 + tap / 3 - 1,
+                               valid ? cn0 : p.conv.NB, full_bar(s));
+            }
+            continue;
+          }
+          ptx::tma_load_2d(a_s, &tmapA, m0, kt * 64, full_bar(s));
+          ptx::tma_load_2d(a_s + 8192, &tmapA, m0 + 64, kt * 64, full_bar(s));
+#pragma unroll
+          for (int q = 0; q < 4; ++q) ptx::tma_load_2d(b_s + q * 8192, &tmapB, n0 + 64 * q, kt * 64, full_bar(s));
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (ptx::elect_one()) {
+      constexpr uint32_t idesc = ptx::idesc_bf16(128, 256, true, true, false);
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x, ++tcount) {
+        int m0, n0, kt0, nkt, split;
+        item_coords(item, m0, n0, kt0, nkt, split);
+        const uint32_t buf = tcount & 1u;
+        if (!ptx::mbar_wait_bounded(tmem_empty_bar(buf), ((tcount >> 1) & 1u) ^ 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
+        ptx::tc_fence_after();
+        const uint32_t acc = tmem_base + 256u * buf;
+        for (int k = 0; k < nkt; ++k, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t a_s = base + s * C::STAGE_BYTES;
+          const uint32_t b_s = a_s + C::A_BYTES;
+#pragma unroll
+          for (int kb = 0; kb < 4; ++kb) {
+            const uint64_t ad = ptx::smem_desc(a_s + kb * 2048, 8192, 1024, 2);
+            const uint64_t bd = ptx::smem_desc(b_s + kb * 2048, 8192, 1024, 2);
+            ptx::mma_dense(acc, ad, bd, idesc, (k | kb) != 0);
+          }
+          ptx::tc_commit(empty_bar(s));
+        }
+        if (ok) ptx::tc_commit(tmem_full_bar(buf));
+      }
+    }
+  } else {
+    const int q = warp & 3;
+    uint32_t tcount = 0;
+    for (int item = blockIdx.x; item < num_items; item += gridDim.x, ++tcount) {
+      int m0, n0, kt0, nkt, split;
+      item_coords(item, m0, n0, kt0, nkt, split);
+      const uint32_t buf = tcount & 1u;
+      if (!ptx::mbar_wait_bounded(tmem_full_bar(buf), (tcount >> 1) & 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
+      ptx::tc_fence_after();
+      const int m = m0 + 32 * q + lane;
+      float* out = reinterpret_cast<float*>(p.out) + (size_t)split * p.Mdim * p.Ndim;
+#pragma unroll 1
+      for (int c = 0; c < 8; ++c) {
+        uint32_t r[32];
+        ptx::tmem_ld_32x32(tmem_base + 256u * buf + ((uint32_t)(32 * q) << 16) + 32 * c, r);
+        ptx::tmem_ld_wait();
+        if (c == 7) {                                      // accumulator drained: release it
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(tmem_empty_bar(buf));
+        }
+        const int nb = n0 + 32 * c;
+        if (m < p.Mdim && nb < p.Ndim) {                  // Ndim % 32 == 0: a chunk is all in or all out
+          float4* dst = reinterpret_cast<float4*>(out + (size_t)m * p.Ndim + nb);
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                 __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+        }
+      }
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status_word, (int32_t)BIMASK_ETIMEOUT);
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, C::TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // dY[:, perm]: a streaming pass.  A CTA takes R token rows at a time (R = 4, or 2 for rows too
 // long for a 4-row tile in shared memory): it reads
 // them coalesced and stores them column-interleaved in shared memory (one 2R-byte word = the R
@@ -1516,11 +1694,15 @@ int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, u
 }
 
 // Split-K plan of the dense product for a reduction of k_tiles 64-deep tiles.
+static bool wgrad_uses_single(int I) { return I <= 128; }       // one 128-row tile: no CTA pairs
+
 static void wgrad_plan_k(int k_tiles, int I, int J, int* splits, int* k_tiles_per_split) {
-  const int tiles = (((I + 127) / 128 + 1) / 2) * ((J + 255) / 256);     // 256 x 256 pair tiles
+  const bool single = wgrad_uses_single(I);
+  const int tiles = single ? (J + 255) / 256 : (((I + 127) / 128 + 1) / 2) * ((J + 255) / 256);   // 128 / 256 x 256 tiles
+  const int workers = single ? 148 : 74;                          // CTAs or CTA pairs
   int sp = 1;
-  if (tiles < 74) {
-    sp = 74 / tiles;                                              // one round of work items over the 74 CTA pairs
+  if (tiles < workers) {
+    sp = workers / tiles;                                         // one round of work items over the workers
     const int max_by_k = k_tiles / 8 > 0 ? k_tiles / 8 : 1;        // at least 8 k tiles per split
     if (sp > max_by_k) sp = max_by_k;
     if (sp > 64) sp = 64;
@@ -1558,8 +1740,6 @@ int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int 
   int rc;
   if ((rc = make_tmap_nhwc_load(&ta, dy, I, W, H, NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_nhwc_load(&tb, x, C, W, H, NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
-  auto kern = wgrad_pair_kernel<STAGES, true>;
-  if ((rc = set_smem_attr(kern, Cf::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
   p.conv = g;
   p.hw_meta = nullptr; p.tiles_k_meta = 0;
@@ -1567,13 +1747,23 @@ int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int 
   p.k_tiles_per_split = per;
   p.out = splits > 1 ? partials : dW;
   p.status_word = status_word;
-  p.tiles_m = ((I + 127) / 128 + 1) / 2;
   p.tiles_n = (J + 255) / 256;
   p.raster_group = 8;
-  const int items = p.tiles_m * p.tiles_n * splits;
   const int sms = sm_count();
-  const int clusters = items < sms / 2 ? items : sms / 2;
-  kern<<<2 * clusters, GEMM_THREADS, Cf::SMEM_BYTES, s>>>(ta, tb, p, splits);
+  if (wgrad_uses_single(I)) {
+    auto kern1 = wgrad_single_kernel<4, true>;
+    if ((rc = set_smem_attr(kern1, WgradSingleCfg<4>::SMEM_BYTES)) != BIMASK_OK) return rc;
+    p.tiles_m = 1;
+    const int items = p.tiles_n * splits;
+    kern1<<<items < sms ? items : sms, GEMM_THREADS, WgradSingleCfg<4>::SMEM_BYTES, s>>>(ta, tb, p, splits);
+  } else {
+    auto kern = wgrad_pair_kernel<STAGES, true>;
+    if ((rc = set_smem_attr(kern, Cf::SMEM_BYTES)) != BIMASK_OK) return rc;
+    p.tiles_m = ((I + 127) / 128 + 1) / 2;
+    const int items = p.tiles_m * p.tiles_n * splits;
+    const int clusters = items < sms / 2 ? items : sms / 2;
+    kern<<<2 * clusters, GEMM_THREADS, Cf::SMEM_BYTES, s>>>(ta, tb, p, splits);
+  }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   if (splits > 1) {
@@ -1604,8 +1794,6 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
   int rc;
   if ((rc = make_tmap(&ta, dY, (uint64_t)I, (uint64_t)T, 64)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, X, (uint64_t)J, (uint64_t)T, 64)) != BIMASK_OK) return rc;
-  auto kern = wgrad_pair_kernel<STAGES, false>;
-  if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
   p.conv.mode = 0;
   p.hw_meta = nullptr; p.tiles_k_meta = 0;
@@ -1613,13 +1801,23 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
   p.k_tiles_per_split = per;
   p.out = splits > 1 ? partials : dW;
   p.status_word = status_word;
-  p.tiles_m = ((I + 127) / 128 + 1) / 2;
   p.tiles_n = (J + 255) / 256;
   p.raster_group = 8;
-  const int items = p.tiles_m * p.tiles_n * splits;
   const int sms = sm_count();
-  const int clusters = items < sms / 2 ? items : sms / 2;
-  kern<<<2 * clusters, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p, splits);
+  if (wgrad_uses_single(I)) {
+    auto kern1 = wgrad_single_kernel<4, false>;
+    if ((rc = set_smem_attr(kern1, WgradSingleCfg<4>::SMEM_BYTES)) != BIMASK_OK) return rc;
+    p.tiles_m = 1;
+    const int items = p.tiles_n * splits;
+    kern1<<<items < sms ? items : sms, GEMM_THREADS, WgradSingleCfg<4>::SMEM_BYTES, s>>>(ta, tb, p, splits);
+  } else {
+    auto kern = wgrad_pair_kernel<STAGES, false>;
+    if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
+    p.tiles_m = ((I + 127) / 128 + 1) / 2;
+    const int items = p.tiles_m * p.tiles_n * splits;
+    const int clusters = items < sms / 2 ? items : sms / 2;
+    kern<<<2 * clusters, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p, splits);
+  }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   if (splits > 1) {
