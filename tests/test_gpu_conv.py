@@ -74,6 +74,20 @@ def test_conv_other_pattern_and_dense_fallback():
         assert rel_err(b["dW"].cpu().numpy(), ref["dW"]) <= TOL
 
 
+@pytest.mark.parametrize("N,M", [(1, 4), (2, 8), (1, 16)])
+def test_conv_implicit_form_other_patterns(N, M):
+    NB, H, W, C, I = 2, 10, 12, 128, 128
+    Wt, x, dy = conv_case(NB, H, W, C, I, 78)
+    b = run_conv_step(Wt, x, dy, N, M, 3, 5, bm.binding.CONV_IMPLICIT)
+    ref = O.conv_layer_step(Wt, x, dy, N, M, 3, 5)
+    assert int(b["status_word"].item()) == 0
+    assert np.array_equal(b["perm"].cpu().numpy(), ref["perm"])
+    assert np.array_equal(u16(b["vals_b"]), ref["vals_b"])
+    assert rel_err(b["Y"].float().cpu().numpy().reshape(NB, H, W, I), ref["y"]) <= TOL
+    assert rel_err(b["dX"].float().cpu().numpy(), ref["dx"]) <= TOL
+    assert rel_err(b["dW"].cpu().numpy(), ref["dW"]) <= TOL
+
+
 def test_conv_bad_arguments_launch_nothing():
     NB, H, W, C, I = 1, 8, 8, 32, 32
     Wt, x, dy = conv_case(NB, H, W, C, I, 1)
