@@ -137,3 +137,25 @@ def test_config5_layer_on_samples(li):
     assert rel_err(dW[is_], ref) <= TOL
     ref = dYf.T @ Xf[:, js]                                    # dW[:, js]
     assert rel_err(dW[:, js], ref) <= TOL
+
+
+@pytest.mark.parametrize("I,J,T", [(256, 64, 100352), (64, 256, 100352), (2048, 512, 1568), (512, 2048, 1568)])
+def test_resnet_bottleneck_1x1_shapes(I, J, T):
+    """The 1x1 convolutions of ResNet-50's bottleneck blocks (c x 4c and 4c x c at the same pixel counts as
+    config 2) are plain linear layers on the NHWC activations: narrow reduction or narrow output, very many tokens."""
+    N, M, P, seed = 2, 4, 32, 44
+    W = inputs.make_weight(I, J, 600 + I)
+    X = inputs.make_activation(T, J, 601)
+    dY = inputs.make_activation(T, I, 602)
+    b = run_layer_step(W, X, dY, N, M, P, seed, do_search=True)
+    ref = O.layer_step(W, X, dY, N, M, P, seed, do_search=True)
+    assert int(b["status_word"].item()) == 0
+    assert np.array_equal(u32(b["maskbits_f"]), ref["maskbits_f"])
+    assert np.array_equal(u16(b["vals_f"]), ref["vals_f"])
+    assert np.array_equal(b["counts"].cpu().numpy(), ref["counts"])
+    assert np.array_equal(b["perm"].cpu().numpy(), ref["perm"])
+    assert np.array_equal(u32(b["maskbits_b"]), ref["maskbits_b"])
+    assert np.array_equal(u16(b["vals_b"]), ref["vals_b"])
+    assert rel_err(b["Y"].float().cpu().numpy(), ref["Y"]) <= TOL
+    assert rel_err(b["dX"].float().cpu().numpy(), ref["dX"]) <= TOL
+    assert rel_err(b["dW"].cpu().numpy(), ref["dW"]) <= TOL
