@@ -616,7 +616,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=5, help="workload: 1..5 (default 5, the largest)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--graph", action="store_true", help="replay one captured pass (CUDA graph) in the timed region")
     ap.add_argument("--profile", action="store_true", help="run only the C-ABI calls of one layer (for ncu)")
     ap.add_argument("--layer", type=int, default=0)
