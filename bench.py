@@ -102,11 +102,27 @@ def run_reference(args):
     cfg = inputs.CONFIGS[args.config]
     for _ in range(args.warmup):
         oracle_sample_time(args.config, rows=128, tokens=32, cands=1)
+    # Size the per-step sample so that the whole run stays within a few minutes whatever --steps and the host are:
+    # a time budget for the run, each step's sample sized from what the previous one cost (cost grows faster
+    # than linearly in the rows, hence the margin); every step's result is scaled to the full layer anyway.
+    budget = 150.0
+    t_cal = time.perf_counter()
+    oracle_sample_time(args.config, rows=128, tokens=args.ref_tokens, cands=2)
+    last_rows, last_cost = 128, time.perf_counter() - t_cal
     per_pass = []
+    rows_used = []
     t_begin = time.perf_counter()
-    for _ in range(args.steps):
-        full, _, desc = oracle_sample_time(args.config, rows=args.ref_rows, tokens=args.ref_tokens, cands=2)
+    for k in range(args.steps):
+        share = max(budget - (time.perf_counter() - t_begin), 0.0) / (args.steps - k)
+        rows = int(last_rows * (share / max(last_cost, 1e-3)) ** 0.75) // 32 * 32
+        rows = max(128, min(args.ref_rows, rows))
+        t0 = time.perf_counter()
+        full, _, desc = oracle_sample_time(args.config, rows=rows, tokens=args.ref_tokens, cands=2)
+        last_rows, last_cost = rows, time.perf_counter() - t0
         per_pass.append(full)
+        rows_used.append(rows)
+    if len(set(rows_used)) > 1:
+        desc += f"; rows per step adapted to a {budget:.0f} s budget: {min(rows_used)}..{max(rows_used)}"
     wall = time.perf_counter() - t_begin
     sec = float(np.mean(per_pass))
     value = len(cfg.layers) / sec
