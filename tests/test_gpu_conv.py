@@ -133,3 +133,22 @@ def test_conv_implicit_form_builds_no_column_matrix(NB, H, W, C, I):
         assert rel_err(got["Y"].float().cpu().numpy().reshape(NB, H, W, I), ref["y"]) <= TOL
         assert rel_err(got["dX"].float().cpu().numpy(), ref["dx"]) <= TOL
         assert rel_err(got["dW"].cpu().numpy(), ref["dW"]) <= TOL
+
+
+@pytest.mark.parametrize("H,W,C,I", [(56, 56, 64, 64), (28, 28, 128, 128), (14, 14, 256, 256), (7, 7, 512, 512)])
+def test_conv_resnet50_layers_at_batch_32(H, W, C, I):
+    """ResNet-50's four 3x3 layer shapes at the batch size bench.py --conv times, automatic form (implicit for the
+    first three, whose column matrices exceed 16 MiB; explicit for 7 x 7)."""
+    NB, N, M, P, seed = 32, 2, 4, 32, 45
+    Wt, x, dy = conv_case(NB, H, W, C, I, 640 + H)
+    b = run_conv_step(Wt, x, dy, N, M, P, seed, bm.binding.CONV_AUTO)
+    ref = O.conv_layer_step(Wt, x, dy, N, M, P, seed)
+    assert int(b["status_word"].item()) == 0
+    assert np.array_equal(u32(b["maskbits_f"]), ref["maskbits_f"])
+    assert np.array_equal(b["counts"].cpu().numpy(), ref["counts"])
+    assert np.array_equal(b["perm"].cpu().numpy(), ref["perm"])
+    assert np.array_equal(u32(b["maskbits_b"]), ref["maskbits_b"])
+    assert np.array_equal(u16(b["vals_b"]), ref["vals_b"])
+    assert rel_err(b["Y"].float().cpu().numpy().reshape(NB, H, W, I), ref["y"]) <= TOL
+    assert rel_err(b["dX"].float().cpu().numpy(), ref["dx"]) <= TOL
+    assert rel_err(b["dW"].cpu().numpy(), ref["dW"]) <= TOL
