@@ -124,10 +124,15 @@ gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int q_log2, i
 constexpr int SCORE_THREADS = 256;
 constexpr int SCORE_KB_PER_CTA = 64;
 
+// Columns (bits) where more than N of the four rows are set.  a + b + c = 2 * maj + par (a full adder per bit,
+// two three-input logic operations); adding d: at least two  <=>  maj | (par & d), at least three  <=>
+// maj & (par | d) -- one more three-input operation.
 template <int N>
 __device__ __forceinline__ uint32_t ineligible(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  if (N == 1) return (a & b) | (c & d) | ((a | b) & (c | d));     // two or more set
-  if (N == 2) return (a & b & (c | d)) | (c & d & (a | b));       // three or more set
+  const uint32_t par = a ^ b ^ c;
+  const uint32_t maj = (a & b) | (a & c) | (b & c);
+  if (N == 1) return maj | (par & d);
+  if (N == 2) return maj & (par | d);
   if (N == 3) return a & b & c & d;
   return 0u;
 }
@@ -169,16 +174,18 @@ score_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cand
       const uint4* t1 = reinterpret_cast<const uint4*>(bits + (long long)t.y * jwords);
       const uint4* t2 = reinterpret_cast<const uint4*>(bits + (long long)t.z * jwords);
       const uint4* t3 = reinterpret_cast<const uint4*>(bits + (long long)t.w * jwords);
-      uint32_t c1 = 0, c2 = 0;
+      uint32_t c1 = 0, c2 = 0, words = 0;
       for (int q = lane; q < jq; q += 32) {
         const uint4 a = __ldg(r0 + q), b = __ldg(r1 + q), cc = __ldg(r2 + q), d = __ldg(r3 + q);
         const uint4 e = __ldg(t0 + q), f = __ldg(t1 + q), g = __ldg(t2 + q), h = __ldg(t3 + q);
-        c1 += __popc(~ineligible<N>(a.x, b.x, cc.x, d.x)) + __popc(~ineligible<N>(a.y, b.y, cc.y, d.y)) +
-              __popc(~ineligible<N>(a.z, b.z, cc.z, d.z)) + __popc(~ineligible<N>(a.w, b.w, cc.w, d.w));
-        c2 += __popc(~ineligible<N>(e.x, f.x, g.x, h.x)) + __popc(~ineligible<N>(e.y, f.y, g.y, h.y)) +
-              __popc(~ineligible<N>(e.z, f.z, g.z, h.z)) + __popc(~ineligible<N>(e.w, f.w, g.w, h.w));
+        c1 += __popc(ineligible<N>(a.x, b.x, cc.x, d.x)) + __popc(ineligible<N>(a.y, b.y, cc.y, d.y)) +
+              __popc(ineligible<N>(a.z, b.z, cc.z, d.z)) + __popc(ineligible<N>(a.w, b.w, cc.w, d.w));
+        c2 += __popc(ineligible<N>(e.x, f.x, g.x, h.x)) + __popc(ineligible<N>(e.y, f.y, g.y, h.y)) +
+              __popc(ineligible<N>(e.z, f.z, g.z, h.z)) + __popc(ineligible<N>(e.w, f.w, g.w, h.w));
+        words += 4;
       }
-      cnt += c1 + (two ? c2 : 0u);
+      // eligible = all columns this lane looked at minus the ineligible ones
+      cnt += (32u * words - c1) + (two ? 32u * words - c2 : 0u);
     }
   } else {
     for (int k = kb0 + warp; k < kb1; k += SCORE_THREADS / 32) {
