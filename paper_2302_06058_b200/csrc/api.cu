@@ -94,9 +94,11 @@ int bimask_fwd_mask(const float* W, int I, int J, int N, int M, uint32_t* maskbi
                  BIMASK_EINVAL, "bimask_fwd_mask: pointers must be 16-byte aligned");
   cudaStream_t s = (cudaStream_t)stream;
   if (M != 4) {
-    if ((rc = launch_fwd_mask_generic(W, I, J, N, M, maskbits_f, vals_f, meta_f, pack ? 1 : vals_f ? 2 : 0, s)) != BIMASK_OK)
+    const bool gfused = pack && (I % 128 == 0) && (J % 128 == 0);   // unpadded: the mask kernel writes the metadata image
+    if ((rc = launch_fwd_mask_generic(W, I, J, N, M, maskbits_f, vals_f, meta_f, pack ? 1 : vals_f ? 2 : 0,
+                                      gfused ? hw_meta_f : nullptr, s)) != BIMASK_OK)
       return rc;
-    return pack ? launch_hw_meta(meta_f, I, J, hw_meta_f, s) : BIMASK_OK;
+    return pack && !gfused ? launch_hw_meta(meta_f, I, J, hw_meta_f, s) : BIMASK_OK;
   }
   const bool fused = (I % 128 == 0) && (J % 128 == 0);   // no padding in the metadata image
   if ((rc = launch_fwd_mask(W, I, J, N, maskbits_f, vals_f, meta_f, fused ? hw_meta_f : nullptr, s)) != BIMASK_OK) return rc;
@@ -165,9 +167,11 @@ int bimask_sgd_fwd_mask(float* W, const float* dW, float* mom, int I, int J, int
   cudaStream_t s = (cudaStream_t)stream;
   if (M != 4) {
     if ((rc = launch_sgd_update(W, dW, mom, (long long)I * J, lr, momentum, weight_decay, s)) != BIMASK_OK) return rc;
-    if ((rc = launch_fwd_mask_generic(W, I, J, N, M, maskbits_f, vals_f, meta_f, pack ? 1 : vals_f ? 2 : 0, s)) != BIMASK_OK)
+    const bool gfused = pack && (I % 128 == 0) && (J % 128 == 0);   // unpadded: the mask kernel writes the metadata image
+    if ((rc = launch_fwd_mask_generic(W, I, J, N, M, maskbits_f, vals_f, meta_f, pack ? 1 : vals_f ? 2 : 0,
+                                      gfused ? hw_meta_f : nullptr, s)) != BIMASK_OK)
       return rc;
-    return pack ? launch_hw_meta(meta_f, I, J, hw_meta_f, s) : BIMASK_OK;
+    return pack && !gfused ? launch_hw_meta(meta_f, I, J, hw_meta_f, s) : BIMASK_OK;
   }
   const bool fused = (I % 128 == 0) && (J % 128 == 0);   // no padding in the metadata image
   if ((rc = launch_sgd_fwd_mask(W, dW, mom, I, J, N, lr, momentum, weight_decay, maskbits_f, vals_f, meta_f,
@@ -226,10 +230,11 @@ int bimask_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* p
                  BIMASK_EINVAL, "bimask_bwd_mask: pointers must be 16-byte aligned");
   cudaStream_t s = (cudaStream_t)stream;
   if (M != 4) {
-    if ((rc = launch_bwd_mask_generic(W, maskbits_f, perm, I, J, N, M, maskbits_b, vals_b, meta_b, pack ? 1 : vals_b ? 2 : 0, s)) !=
-        BIMASK_OK)
+    const bool gfused = pack && (I % 128 == 0) && (J % 128 == 0);
+    if ((rc = launch_bwd_mask_generic(W, maskbits_f, perm, I, J, N, M, maskbits_b, vals_b, meta_b, pack ? 1 : vals_b ? 2 : 0,
+                                      gfused ? hw_meta_b : nullptr, s)) != BIMASK_OK)
       return rc;
-    return pack ? launch_hw_meta(meta_b, J, I, hw_meta_b, s) : BIMASK_OK;
+    return pack && !gfused ? launch_hw_meta(meta_b, J, I, hw_meta_b, s) : BIMASK_OK;
   }
   const bool fused = (I % 128 == 0) && (J % 128 == 0);
   if ((rc = launch_bwd_mask(W, maskbits_f, perm, I, J, N, maskbits_b, vals_b, meta_b, fused ? hw_meta_b : nullptr, s)) !=
@@ -262,11 +267,11 @@ int bimask_bwd_mask_criterion(const float* W, const float* S, const uint32_t* ma
                      aligned16(vals_b) && aligned16(meta_b) && aligned16(hw_meta_b),
                  BIMASK_EINVAL, "bimask_bwd_mask_criterion: pointers must be 16-byte aligned");
   cudaStream_t s = (cudaStream_t)stream;
+  const bool gfused = pack && (I % 128 == 0) && (J % 128 == 0);
   if ((rc = launch_bwd_mask_criterion(W, S, maskbits_f, perm, I, J, N, M, criterion, seed, maskbits_b, vals_b, meta_b,
-                                      pack ? 1 : vals_b ? 2 : 0, s)) !=
-      BIMASK_OK)
+                                      pack ? 1 : vals_b ? 2 : 0, gfused ? hw_meta_b : nullptr, s)) != BIMASK_OK)
     return rc;
-  return pack ? launch_hw_meta(meta_b, J, I, hw_meta_b, s) : BIMASK_OK;
+  return pack && !gfused ? launch_hw_meta(meta_b, J, I, hw_meta_b, s) : BIMASK_OK;
 }
 
 static int check_gemm(int T, int I, int J) {
@@ -386,13 +391,14 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
     if (!conv->imp_fwd || !conv->imp_wgrad)
       if ((rc = launch_im2col3x3(a->X, conv->NB, conv->H, conv->W, conv->C, conv->xcol, s))) return rc;
   }
-  // M = 4 with unpadded shapes writes the metadata images inside the mask kernels
-  const bool fused = a->M == 4 && (a->I % 128 == 0) && (a->J % 128 == 0);
+  // unpadded shapes: the mask kernels write the metadata images themselves
+  const bool fused = pack && (a->I % 128 == 0) && (a->J % 128 == 0);
   if (!skip_fwd_mask) {
     if (a->M == 4)
       rc = launch_fwd_mask(a->W, a->I, a->J, a->N, a->maskbits_f, a->vals_f, a->meta_f, fused ? a->hw_meta_f : nullptr, s);
     else
-      rc = launch_fwd_mask_generic(a->W, a->I, a->J, a->N, a->M, a->maskbits_f, a->vals_f, a->meta_f, pack ? 1 : 2, s);
+      rc = launch_fwd_mask_generic(a->W, a->I, a->J, a->N, a->M, a->maskbits_f, a->vals_f, a->meta_f, pack ? 1 : 2,
+                                   fused ? a->hw_meta_f : nullptr, s);
     if (rc) return rc;
     if (pack && !fused && (rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, s))) return rc;
   }
@@ -417,7 +423,7 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
                          fused ? a->hw_meta_b : nullptr, s);
   else
     rc = launch_bwd_mask_generic(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->M, a->maskbits_b, a->vals_b, a->meta_b,
-                                 pack ? 1 : 2, s);
+                                 pack ? 1 : 2, fused ? a->hw_meta_b : nullptr, s);
   if (rc) return rc;
   if (pack && !fused && (rc = launch_hw_meta(a->meta_b, a->J, a->I, a->hw_meta_b, s))) return rc;
   if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, s))) return rc;

@@ -61,14 +61,15 @@ int launch_pick(const int64_t* counts, const int32_t* cands, int P, int I, int32
 // N:M patterns with M = 8 or 16 (nm_generic_kernels.cu); vals / meta may be null (mask bits only).
 // mode (generic mask launchers): 0 mask bits only, 1 the 2:4 operand, 2 the dense masked bf16 operand in `vals`
 int launch_fwd_mask_generic(const float* W, int I, int J, int N, int M, uint32_t* maskbits, uint16_t* vals_or_null,
-                            uint32_t* meta_or_null, int mode, cudaStream_t s);
+                            uint32_t* meta_or_null, int mode, void* hw_meta_or_null, cudaStream_t s);
 int launch_score_generic(const uint32_t* bits, const int32_t* cands, int I, int J, int N, int M, int P,
                          int64_t* counts, cudaStream_t s);
 int launch_bwd_mask_generic(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J, int N, int M,
-                            uint32_t* maskbits_b, uint16_t* vals_b_or_null, uint32_t* meta_b_or_null, int mode, cudaStream_t s);
+                            uint32_t* maskbits_b, uint16_t* vals_b_or_null, uint32_t* meta_b_or_null, int mode,
+                            void* hw_meta_or_null, cudaStream_t s);
 int launch_bwd_mask_criterion(const float* W, const float* S, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                               int N, int M, int crit, uint64_t seed, uint32_t* maskbits_b, uint16_t* vals_b_or_null,
-                              uint32_t* meta_b_or_null, int mode, cudaStream_t s);
+                              uint32_t* meta_b_or_null, int mode, void* hw_meta_or_null, cudaStream_t s);
 int launch_refine(const uint32_t* bits, int I, int J, int N, int M, int rounds, const int32_t* orders, int32_t* perm,
                   int32_t* gains, unsigned long long* block_best, cudaStream_t s);
 int launch_check_perms(const int32_t* cands, int P, int I, int32_t* ok, uint8_t* seen, cudaStream_t s);

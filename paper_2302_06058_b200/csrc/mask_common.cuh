@@ -88,5 +88,19 @@ __device__ __forceinline__ uint32_t slots(uint32_t e, float w0, float w1, float 
   return v;
 }
 
+// One canonical code word (row r of the packed operand, 32-column word w) scattered into the
+// tensor-memory image of the metadata (one 2048-byte block per 128 rows x 128 k: 128 lanes x 4
+// columns of u32, lane = m0 + 8*h + 16*m2 holding rows m0 + 16*m2 / + 8 of k-half h): its low 16 bits (k-half 0) and high 16 bits
+// (k-half 1) land in two different lanes, each as one half of a 32-bit word whose other half
+// comes from the row 8 above or below.  Used when the operand has no padding (rows and K both
+// multiples of 128), so that the separate re-ordering pass is not needed.
+__device__ __forceinline__ void scatter_hw(uint16_t* __restrict__ hw16, int tiles_k, int r, int w, uint32_t word) {
+  const int rr = r & 127;
+  const size_t tile = (size_t)(r >> 7) * tiles_k + (w >> 2);
+  const size_t idx = (tile * 512 + (size_t)((rr & 7) + 16 * (rr >> 4)) * 4 + (w & 3)) * 2 + ((rr >> 3) & 1);
+  hw16[idx] = (uint16_t)(word & 0xFFFFu);
+  hw16[idx + 64] = (uint16_t)(word >> 16);               // lane + 8: 8 lanes x 4 words x 2 halves
+}
+
 }  // namespace
 }  // namespace bimask

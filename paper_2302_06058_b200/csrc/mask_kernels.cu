@@ -13,19 +13,6 @@ namespace bimask {
 
 namespace {
 
-// One canonical code word (row r of the packed operand, 32-column word w) scattered into the
-// TMEM image described at hw_meta_kernel below: its low 16 bits (k-half 0) and high 16 bits
-// (k-half 1) land in two different lanes, each as one half of a 32-bit word whose other half
-// comes from the row 8 above or below.  Used when the operand has no padding (rows and K both
-// multiples of 128), so that the separate re-ordering pass is not needed.
-__device__ __forceinline__ void scatter_hw(uint16_t* __restrict__ hw16, int tiles_k, int r, int w, uint32_t word) {
-  const int rr = r & 127;
-  const size_t tile = (size_t)(r >> 7) * tiles_k + (w >> 2);
-  const size_t idx = (tile * 512 + (size_t)((rr & 7) + 16 * (rr >> 4)) * 4 + (w & 3)) * 2 + ((rr >> 3) & 1);
-  hw16[idx] = (uint16_t)(word & 0xFFFFu);
-  hw16[idx + 64] = (uint16_t)(word >> 16);               // lane + 8: 8 lanes x 4 words x 2 halves
-}
-
 // ---------------------------------------------------------------------------------------
 // Forward mask + pack.  W is treated as a flat stream of 4-element blocks (J % 32 == 0, so
 // blocks, 32-column words and rows all nest).  A warp owns chunks of 256 blocks: eight

@@ -69,7 +69,7 @@ template <int M, int MODE>
 __global__ void __launch_bounds__(256)
 fwd_mask_generic_kernel(const float4* __restrict__ W4, long long nblocks, int N,
                         uint32_t* __restrict__ maskbits, uint32_t* __restrict__ vals32,
-                        uint32_t* __restrict__ meta) {
+                        uint32_t* __restrict__ meta, uint16_t* __restrict__ hw16, int jwords) {
   constexpr int LPW = 32 / M;                               // lanes per 32-column word
   constexpr int G = M / 4;                                  // groups of four per block
   __shared__ uint32_t pad16[16];                            // container entry of a group from its keep mask
@@ -80,13 +80,25 @@ fwd_mask_generic_kernel(const float4* __restrict__ W4, long long nblocks, int N,
   const int sh = M * (lane & (LPW - 1));
   const long long stride = (long long)gridDim.x * blockDim.x;
   const long long nround = (nblocks + 31) & ~31ll;          // whole warps stay in the loop together
+  // the next trip's block is loaded before this trip's is worked on (one block of loads always in flight)
+  float4 nxt[G];
+  {
+    const long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+#pragma unroll
+    for (int g = 0; g < G; ++g) nxt[g] = b < nblocks ? __ldg(W4 + b * G + g) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
   for (long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x; b < nround; b += stride) {
     const bool live = b < nblocks;
     float w[M];
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      const float4 v = live ? __ldg(W4 + b * G + g) : make_float4(0.f, 0.f, 0.f, 0.f);
+      const float4 v = nxt[g];
       w[4 * g] = v.x; w[4 * g + 1] = v.y; w[4 * g + 2] = v.z; w[4 * g + 3] = v.w;
+    }
+    {
+      const long long bn = b + stride;
+#pragma unroll
+      for (int g = 0; g < G; ++g) nxt[g] = bn < nblocks ? __ldg(W4 + bn * G + g) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     uint32_t key[M];
 #pragma unroll
@@ -121,8 +133,15 @@ fwd_mask_generic_kernel(const float4* __restrict__ W4, long long nblocks, int N,
     const uint32_t wb = __reduce_or_sync(gmask, kb << sh);
     const uint32_t wm = __reduce_or_sync(gmask, codes << sh);
     if (live && (lane & (LPW - 1)) == 0) {
-      maskbits[b / LPW] = wb;
-      if (MODE == 1) meta[b / LPW] = wm;
+      const long long word = b / LPW;
+      maskbits[word] = wb;
+      if (MODE == 1) {
+        meta[word] = wm;
+        if (hw16) {                                         // unpadded operand: write the tensor-memory image here
+          const int r = (int)(word / jwords);
+          scatter_hw(hw16, jwords >> 2, r, (int)(word - (long long)r * jwords), wm);
+        }
+      }
     }
   }
 }
@@ -166,12 +185,27 @@ score_generic_kernel(const uint32_t* __restrict__ bits, const int32_t* __restric
       rows[4 * g] = (int)min((unsigned)r.x, last_row); rows[4 * g + 1] = (int)min((unsigned)r.y, last_row);
       rows[4 * g + 2] = (int)min((unsigned)r.z, last_row); rows[4 * g + 3] = (int)min((unsigned)r.w, last_row);
     }
-    for (int q = lane; q < jwords; q += 32) {
-      SatCount<N> s;
-      s.clear();
+    if ((jwords & 3) == 0) {
+      // 128-bit loads: four words of every row at once (a quarter of the load instructions)
+      const int jq = jwords >> 2;
+      for (int q = lane; q < jq; q += 32) {
+        SatCount<N> s0, s1, s2, s3;
+        s0.clear(); s1.clear(); s2.clear(); s3.clear();
 #pragma unroll
-      for (int m = 0; m < M; ++m) s.add(__ldg(bits + (long long)rows[m] * jwords + q));
-      cnt += __popc(s.eligible());
+        for (int m = 0; m < M; ++m) {
+          const uint4 v = __ldg(reinterpret_cast<const uint4*>(bits + (long long)rows[m] * jwords) + q);
+          s0.add(v.x); s1.add(v.y); s2.add(v.z); s3.add(v.w);
+        }
+        cnt += __popc(s0.eligible()) + __popc(s1.eligible()) + __popc(s2.eligible()) + __popc(s3.eligible());
+      }
+    } else {
+      for (int q = lane; q < jwords; q += 32) {
+        SatCount<N> s;
+        s.clear();
+#pragma unroll
+        for (int m = 0; m < M; ++m) s.add(__ldg(bits + (long long)rows[m] * jwords + q));
+        cnt += __popc(s.eligible());
+      }
     }
   }
   cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
@@ -327,7 +361,8 @@ __global__ void __launch_bounds__(256)
 bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,
                         const int32_t* __restrict__ perm, int I, int J, int N,
                         uint32_t* __restrict__ maskbits_b, uint32_t* __restrict__ vals_b,
-                        uint32_t* __restrict__ meta_b, const float* __restrict__ S, uint64_t seed) {
+                        uint32_t* __restrict__ meta_b, const float* __restrict__ S, uint64_t seed,
+                        uint16_t* __restrict__ hw16) {
   constexpr int NB = 32 / M;                                // blocks per 32-row pass
   constexpr int G = M / 4;
   __shared__ uint32_t pad16[16];
@@ -394,6 +429,7 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
     dst[0] = make_uint4(vacc[0], vacc[1], vacc[2], vacc[3]);
     dst[1] = make_uint4(vacc[4], vacc[5], vacc[6], vacc[7]);
     meta_b[(size_t)col * (I >> 5) + pass] = cacc;
+    if (hw16) scatter_hw(hw16, I >> 7, col, pass, cacc);
   }
   if (MODE == 2) {
     uint4* dst = reinterpret_cast<uint4*>(vals_b + (size_t)col * (I >> 1) + 16 * pass);   // row `col` of the J x I operand
@@ -406,20 +442,22 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
 
 // mode: 0 mask bits only, 1 the 2:4 operand, 2 the dense masked operand (written to `vals`)
 int launch_fwd_mask_generic(const float* W, int I, int J, int N, int M, uint32_t* maskbits, uint16_t* vals_or_null,
-                            uint32_t* meta_or_null, int mode, cudaStream_t s) {
+                            uint32_t* meta_or_null, int mode, void* hw_meta_or_null, cudaStream_t s) {
+  uint16_t* hw16 = reinterpret_cast<uint16_t*>(hw_meta_or_null);
+  const int jw = J / 32;
   const long long nblocks = (long long)I * J / M;
   long long ctas = (nblocks + 255) / 256;
   if (ctas > 148 * 16) ctas = 148 * 16;
   const float4* W4 = reinterpret_cast<const float4*>(W);
   uint32_t* v32 = reinterpret_cast<uint32_t*>(vals_or_null);
   if (M == 8) {
-    if (mode == 1) fwd_mask_generic_kernel<8, 1><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
-    else if (mode == 2) fwd_mask_generic_kernel<8, 2><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
-    else fwd_mask_generic_kernel<8, 0><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
+    if (mode == 1) fwd_mask_generic_kernel<8, 1><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw);
+    else if (mode == 2) fwd_mask_generic_kernel<8, 2><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw);
+    else fwd_mask_generic_kernel<8, 0><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw);
   } else {
-    if (mode == 1) fwd_mask_generic_kernel<16, 1><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
-    else if (mode == 2) fwd_mask_generic_kernel<16, 2><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
-    else fwd_mask_generic_kernel<16, 0><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null);
+    if (mode == 1) fwd_mask_generic_kernel<16, 1><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw);
+    else if (mode == 2) fwd_mask_generic_kernel<16, 2><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw);
+    else fwd_mask_generic_kernel<16, 0><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw);
   }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
@@ -459,21 +497,21 @@ int launch_score_generic(const uint32_t* bits, const int32_t* cands, int I, int 
 template <int M, int CRIT>
 static void launch_bwd_mc(dim3 grid, int mode, const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                           int N, uint32_t* maskbits_b, uint32_t* v32, uint32_t* meta_b, const float* S, uint64_t seed,
-                          cudaStream_t s) {
-  if (mode == 1) bwd_mask_generic_kernel<M, 1, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed);
-  else if (mode == 2) bwd_mask_generic_kernel<M, 2, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed);
-  else bwd_mask_generic_kernel<M, 0, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed);
+                          uint16_t* hw16, cudaStream_t s) {
+  if (mode == 1) bwd_mask_generic_kernel<M, 1, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16);
+  else if (mode == 2) bwd_mask_generic_kernel<M, 2, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16);
+  else bwd_mask_generic_kernel<M, 0, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16);
 }
 
 template <int M>
 static void launch_bwd_m(int crit, dim3 grid, int mode, const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I,
                          int J, int N, uint32_t* maskbits_b, uint32_t* v32, uint32_t* meta_b, const float* S, uint64_t seed,
-                         cudaStream_t s) {
+                         uint16_t* hw16, cudaStream_t s) {
   switch (crit) {
-    case 1: launch_bwd_mc<M, 1>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
-    case 2: launch_bwd_mc<M, 2>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
-    case 3: launch_bwd_mc<M, 3>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
-    default: launch_bwd_mc<M, 0>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, s); break;
+    case 1: launch_bwd_mc<M, 1>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16, s); break;
+    case 2: launch_bwd_mc<M, 2>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16, s); break;
+    case 3: launch_bwd_mc<M, 3>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16, s); break;
+    default: launch_bwd_mc<M, 0>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16, s); break;
   }
 }
 
@@ -482,17 +520,18 @@ static void launch_bwd_m(int crit, dim3 grid, int mode, const float* W, const ui
 // mode: 0 mask bits only, 1 the transposed 2:4 operand, 2 the transposed dense masked operand.
 int launch_bwd_mask_criterion(const float* W, const float* S, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                               int N, int M, int crit, uint64_t seed, uint32_t* maskbits_b, uint16_t* vals_b_or_null,
-                              uint32_t* meta_b_or_null, int mode, cudaStream_t s) {
+                              uint32_t* meta_b_or_null, int mode, void* hw_meta_or_null, cudaStream_t s) {
   dim3 grid(I / 32, (J / 32 + 7) / 8);
   uint32_t* v32 = reinterpret_cast<uint32_t*>(vals_b_or_null);
+  uint16_t* hw16 = reinterpret_cast<uint16_t*>(hw_meta_or_null);
   if (crit == 3) {
     uint64_t z = seed;
     z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull; z ^= z >> 27; z *= 0x94D049BB133111EBull; z ^= z >> 31;
     seed = z;
   }
-  if (M == 4) launch_bwd_m<4>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, s);
-  else if (M == 8) launch_bwd_m<8>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, s);
-  else launch_bwd_m<16>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, s);
+  if (M == 4) launch_bwd_m<4>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, hw16, s);
+  else if (M == 8) launch_bwd_m<8>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, hw16, s);
+  else launch_bwd_m<16>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, hw16, s);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -539,9 +578,10 @@ int launch_refine(const uint32_t* bits, int I, int J, int N, int M, int rounds, 
 }
 
 int launch_bwd_mask_generic(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J, int N, int M,
-                            uint32_t* maskbits_b, uint16_t* vals_b_or_null, uint32_t* meta_b_or_null, int mode, cudaStream_t s) {
+                            uint32_t* maskbits_b, uint16_t* vals_b_or_null, uint32_t* meta_b_or_null, int mode,
+                            void* hw_meta_or_null, cudaStream_t s) {
   return launch_bwd_mask_criterion(W, nullptr, maskbits_f, perm, I, J, N, M, 0, 0, maskbits_b, vals_b_or_null, meta_b_or_null,
-                                   mode, s);
+                                   mode, hw_meta_or_null, s);
 }
 
 }  // namespace bimask
