@@ -553,104 +553,62 @@ def _pad_hw(a):
     return np.pad(a, ((0, 0), (1, 1), (1, 1), (0, 0)))
 
 
-def conv_fwd(x_bits, W, B):
-    """y[n, h, w, i] = sum_{kh, kw, c} x[n, h+kh-1, w+kw-1, c] * (B.W)[i, (kh*3+kw)*C + c]  (Eq. 3 for a
+def conv_out_size(n: int, stride: int) -> int:
+    """Output extent of a 3-tap window with padding 1: floor((n + 2 - 3) / stride) + 1."""
+    return (n - 1) // stride + 1
+
+
+def conv_fwd(x_bits, W, B, stride=1):
+    """y[n, ho, wo, i] = sum_{kh, kw, c} x[n, ho*s+kh-1, wo*s+kw-1, c] * (B.W)[i, (kh*3+kw)*C + c]  (Eq. 3 for a
     convolution; out-of-range x is 0).  x_bits: bf16 bit patterns NB x H x W x C.  float64 result."""
     NB, H, Wd, C = x_bits.shape
     I = W.shape[0]
+    Ho, Wo = conv_out_size(H, stride), conv_out_size(Wd, stride)
     xp = _pad_hw(bf16_to_f64(x_bits).reshape(NB, H, Wd, C))
     Wf = (bf16_round(W) * B).reshape(I, 3, 3, C)
-    y = np.zeros((NB, H, Wd, I))
+    y = np.zeros((NB, Ho, Wo, I))
     for kh in range(3):
         for kw in range(3):
-            y += xp[:, kh:kh + H, kw:kw + Wd, :] @ Wf[:, kh, kw, :].T
+            y += xp[:, kh:kh + stride * (Ho - 1) + 1:stride, kw:kw + stride * (Wo - 1) + 1:stride, :] @ Wf[:, kh, kw, :].T
     return y
 
 
-def conv_dgrad(dy_bits, W, M_b, C):
-    """dx[n, h, w, c] = sum_{kh, kw, i} dy[n, h-kh+1, w-kw+1, i] * (M_b.W)[i, (kh*3+kw)*C + c]: the input
-    gradient of conv_fwd with the backward mask in place of the forward one (Eq. 8 / Eq. 10)."""
-    NB, H, Wd, I = dy_bits.shape
-    dyp = _pad_hw(bf16_to_f64(dy_bits).reshape(NB, H, Wd, I))
+def conv_dgrad(dy_bits, W, M_b, C, stride=1, in_hw=None):
+    """dx[n, h, w, c] = sum over (kh, kw, i) and output pixels (ho, wo) with ho*s+kh-1 = h, wo*s+kw-1 = w of
+    dy[n, ho, wo, i] * (M_b.W)[i, (kh*3+kw)*C + c]: the input gradient of conv_fwd with the backward mask in place of
+    the forward one (Eq. 8 / Eq. 10).  in_hw = (H, W) of x (needed when stride > 1)."""
+    NB, Ho, Wo, I = dy_bits.shape
+    H, Wd = in_hw if in_hw is not None else (Ho, Wo)
+    dy = bf16_to_f64(dy_bits).reshape(NB, Ho, Wo, I)
     Wb = (bf16_round(W) * M_b).reshape(I, 3, 3, C)
-    dx = np.zeros((NB, H, Wd, C))
+    dxp = np.zeros((NB, H + 2, Wd + 2, C))                      # padded input gradient; the border is dropped
     for kh in range(3):
         for kw in range(3):
-            # output pixel (h, w) receives from dy pixel (h-kh+1, w-kw+1): padded index h-kh+2
-            dx += dyp[:, 2 - kh:2 - kh + H, 2 - kw:2 - kw + Wd, :] @ Wb[:, kh, kw, :]
-    return dx
+            dxp[:, kh:kh + stride * (Ho - 1) + 1:stride, kw:kw + stride * (Wo - 1) + 1:stride, :] += dy @ Wb[:, kh, kw, :]
+    return dxp[:, 1:H + 1, 1:Wd + 1, :]
 
 
-def conv_wgrad(dy_bits, x_bits):
-    """dW[i, (kh*3+kw)*C + c] = sum_{n, h, w} dy[n, h, w, i] * x[n, h+kh-1, w+kw-1, c]  (dense, STE)."""
+def conv_wgrad(dy_bits, x_bits, stride=1):
+    """dW[i, (kh*3+kw)*C + c] = sum_{n, ho, wo} dy[n, ho, wo, i] * x[n, ho*s+kh-1, wo*s+kw-1, c]  (dense, STE)."""
     NB, H, Wd, C = x_bits.shape
-    I = dy_bits.shape[3]
+    _, Ho, Wo, I = dy_bits.shape
     xp = _pad_hw(bf16_to_f64(x_bits).reshape(NB, H, Wd, C))
-    dy = bf16_to_f64(dy_bits).reshape(NB * H * Wd, I)
+    dy = bf16_to_f64(dy_bits).reshape(NB * Ho * Wo, I)
     dW = np.zeros((I, 3, 3, C))
     for kh in range(3):
         for kw in range(3):
-            dW[:, kh, kw, :] = dy.T @ xp[:, kh:kh + H, kw:kw + Wd, :].reshape(NB * H * Wd, C)
+            patch = xp[:, kh:kh + stride * (Ho - 1) + 1:stride, kw:kw + stride * (Wo - 1) + 1:stride, :]
+            dW[:, kh, kw, :] = dy.T @ patch.reshape(NB * Ho * Wo, C)
     return dW.reshape(I, 9 * C)
 
 
-def conv_layer_step(W, x_bits, dy_bits, N, M, P, seed, do_search=True, perm=None):
-    """One iteration of Alg. 1 for a 3x3 convolution layer: masks and search exactly as for a linear
-    layer on the I x 9C matrix view; the three products are convolutions."""
-    C = x_bits.shape[3]
+def conv_layer_step(W, x_bits, dy_bits, N, M, P, seed, do_search=True, perm=None, stride=1):
+    """One iteration of Alg. 1 for a 3x3 convolution layer (padding 1, stride 1 or 2): masks and search exactly as
+    for a linear layer on the I x 9C matrix view; the three products are convolutions."""
+    NB, H, Wd, C = x_bits.shape
     assert W.shape[1] == 9 * C
     out = layer_step(W, None, None, N, M, P, seed, do_search=do_search, perm=perm, with_gemms=False)
-    out["y"] = conv_fwd(x_bits, W, out["B"])
-    out["dx"] = conv_dgrad(dy_bits, W, out["M_b"], C)
-    out["dW"] = conv_wgrad(dy_bits, x_bits)
+    out["y"] = conv_fwd(x_bits, W, out["B"], stride)
+    out["dx"] = conv_dgrad(dy_bits, W, out["M_b"], C, stride, (H, Wd))
+    out["dW"] = conv_wgrad(dy_bits, x_bits, stride)
     return out
-
-
-# ---------------------------------------------------------------------------------------
-# Greedy refinement of a permutation (beyond the paper: its conclusion names a better search than
-# "best of K random candidates" as future work).  Not part of Algorithm 1.
-# ---------------------------------------------------------------------------------------
-REFINE_SEED_OFFSET = 0x5EED5EED
-
-
-def _block_eligible(B, rows, N):
-    """Columns of the row block `rows` (M row indices of B) that hold at most N ones."""
-    return int((B[np.asarray(rows, dtype=np.int64), :].sum(axis=0) <= N).sum())
-
-
-def refine_perm(B, perm, N, M, rounds, seed):
-    """Pairwise-swap hill climbing on the eligible-block count.  Round r pairs up the POSITIONS of the
-    permutation at random: with order = candidates(seed + REFINE_SEED_OFFSET, rounds, I)[r], pair i is
-    (a, b) = (order[2i], order[2i+1]).  A pair whose positions lie in different row blocks ka != kb
-    has gain = (eligible columns of the two blocks after exchanging perm[a] and perm[b]) - (before),
-    all gains taken against the permutation at the start of the round.  A pair is accepted when its
-    gain is positive and, for BOTH of its blocks, it is the best pair touching that block (largest
-    gain, lowest pair index on equal gain) -- so accepted pairs never share a block, their gains add
-    up, and the count never decreases.  Returns (perm, eligible-block count of the result)."""
-    perm = np.array(perm, dtype=np.int32).copy()
-    I = perm.shape[0]
-    assert I % M == 0
-    orders = candidates((int(seed) + REFINE_SEED_OFFSET) & MASK64, rounds, I) if rounds > 0 else None
-    for r in range(rounds):
-        order = orders[r]
-        gains = {}
-        best = {}                                            # block -> (gain, -pair index) of its best pair
-        for i in range(I // 2):
-            a, b = int(order[2 * i]), int(order[2 * i + 1])
-            ka, kb = a // M, b // M
-            if ka == kb:
-                continue
-            rows_a = perm[ka * M:(ka + 1) * M].copy()
-            rows_b = perm[kb * M:(kb + 1) * M].copy()
-            before = _block_eligible(B, rows_a, N) + _block_eligible(B, rows_b, N)
-            rows_a[a - ka * M], rows_b[b - kb * M] = perm[b], perm[a]
-            gain = _block_eligible(B, rows_a, N) + _block_eligible(B, rows_b, N) - before
-            if gain > 0:
-                gains[i] = (gain, a, b, ka, kb)
-                for k in (ka, kb):
-                    if k not in best or (gain, -i) > best[k]:
-                        best[k] = (gain, -i)
-        for i, (gain, a, b, ka, kb) in gains.items():
-            if best[ka] == (gain, -i) and best[kb] == (gain, -i):
-                perm[a], perm[b] = perm[b], perm[a]
-    return perm, eligible_blocks(B, perm, N, M)

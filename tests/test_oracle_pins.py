@@ -686,3 +686,31 @@ def test_refine_perm_fixed_point_and_improvement():
     total = (128 // 4) * 128
     assert abs(counts.mean() / total - 11 / 16) < 0.02
     assert cnt / total > 0.73 and cnt > counts.max() + 0.02 * total
+
+
+def test_strided_conv_products_match_torch():
+    """Stride 2 (ResNet's down-sampling 3x3 convolutions), odd and even image sizes, against torch and its autograd."""
+    rng = np.random.default_rng(47)
+    for (H, Wd) in [(6, 6), (7, 5)]:
+        NB, C, I = 2, 8, 12
+        W = rng.standard_normal((I, 9 * C)).astype(np.float32)
+        B = O.forward_mask(W, 2, 4)
+        perm = rng.permutation(I)
+        M_b = O.unpermute_rows(O.backward_mask(W, B, perm, 2, 4), perm)
+        Ho, Wo = O.conv_out_size(H, 2), O.conv_out_size(Wd, 2)
+        x = O.bf16_bits(rng.standard_normal((NB, H, Wd, C)).astype(np.float32))
+        dy = O.bf16_bits(rng.standard_normal((NB, Ho, Wo, I)).astype(np.float32))
+
+        def filt(mask):
+            return torch.from_numpy((O.bf16_round(W) * mask).reshape(I, 3, 3, C)).permute(0, 3, 1, 2).contiguous()
+
+        xt = torch.from_numpy(O.bf16_to_f64(x).reshape(NB, H, Wd, C)).permute(0, 3, 1, 2).contiguous().requires_grad_(True)
+        dyt = torch.from_numpy(O.bf16_to_f64(dy).reshape(NB, Ho, Wo, I)).permute(0, 3, 1, 2).contiguous()
+        y = torch.nn.functional.conv2d(xt, filt(B), padding=1, stride=2)
+        assert tuple(y.shape[2:]) == (Ho, Wo)
+        assert np.allclose(O.conv_fwd(x, W, B, 2), y.detach().permute(0, 2, 3, 1).numpy(), rtol=1e-12, atol=1e-12)
+        (gx,) = torch.autograd.grad(torch.nn.functional.conv2d(xt, filt(M_b), padding=1, stride=2), xt, dyt)
+        assert np.allclose(O.conv_dgrad(dy, W, M_b, C, 2, (H, Wd)), gx.permute(0, 2, 3, 1).numpy(), rtol=1e-12, atol=1e-12)
+        wd = filt(np.ones_like(B)).requires_grad_(True)
+        (gw,) = torch.autograd.grad(torch.nn.functional.conv2d(xt.detach(), wd, padding=1, stride=2), wd, dyt)
+        assert np.allclose(O.conv_wgrad(dy, x, 2), gw.permute(0, 2, 3, 1).reshape(I, 9 * C).numpy(), rtol=1e-12, atol=1e-12)
