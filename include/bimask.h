@@ -241,7 +241,7 @@ typedef struct bimask_train_args {
 
 int bimask_train_step(const bimask_train_args* args);
 
-/* The layer step for a 3x3 convolution (stride 1, zero padding 1) on NHWC activations -- the
+/* The layer step for a 3x3 convolution (zero padding 1, stride 1 or 2) on NHWC activations -- the
  * ResNet layers the paper trains.  The paper's W is the I x J matrix view of the filter with
  * J = 9*C and column j = (kh*3 + kw)*C + c (flatten order: the paper does not state one; this
  * keeps the channel index contiguous as in the activations), so masks, search and backward mask
@@ -249,10 +249,12 @@ int bimask_train_step(const bimask_train_args* args);
  *   y [n,h,w,i] = sum_{kh,kw,c} x [n,h+kh-1,w+kw-1,c] (B.W)[i,(kh,kw,c)]                      (Eq. 3)
  *   dx[n,h,w,c] = sum_{kh,kw,i} dy[n,h-kh+1,w-kw+1,i] (B-bar.W[perm])...[i,(kh,kw,c)]         (Eq. 10)
  *   dW[i,(kh,kw,c)] = sum_{n,h,w} dy[n,h,w,i] x[n,h+kh-1,w+kw-1,c]                  (dense, Sec. 3.1)
- * `layer` is filled as for bimask_layer_step with T = NB*H*W and J = 9*C, except that
- *   layer.X  = x,  bf16 NB x H x W x C      (T x C, not T x J),
+ * (written for stride 1; with stride s the input pixel of tap (kh, kw) of output pixel (ho, wo) is
+ * (ho*s + kh - 1, wo*s + kw - 1) and the output is Ho x Wo with Ho = (H - 1) / s + 1, Wo likewise).
+ * `layer` is filled as for bimask_layer_step with T = NB*Ho*Wo (output pixels) and J = 9*C, except that
+ *   layer.X  = x,  bf16 NB x H x W x C      (not T x J),
  *   layer.dX = dx, bf16 NB x H x W x C      (out),
- *   layer.dY = dy and layer.Y = y, bf16 NB x H x W x I (the same memory layout as T x I),
+ *   layer.dY = dy and layer.Y = y, bf16 NB x Ho x Wo x I (the same memory layout as T x I),
  *   layer.ws holds bimask_conv_workspace_bytes(...) bytes.
  * mode: BIMASK_CONV_EXPLICIT unfolds x into the T x 9C column matrix, runs the linear-layer
  * products and folds the column-space input gradient back (sum of the nine shifts, fp32);
@@ -261,7 +263,8 @@ int bimask_train_step(const bimask_train_args* args);
  * implicit form for every product whose shape allows it (C % 64 == 0; the input gradient also
  * needs C % 128 == 0 and I % 128 == 0; patterns with a 2:4 form) when the column matrix would
  * exceed 16 MiB, and the explicit form otherwise.  IMPLICIT with a shape that does not allow it
- * returns BIMASK_EUNSUPPORTED.  C % 32 == 0 and I % 32 == 0 always.  The two forms round the
+ * returns BIMASK_EUNSUPPORTED; so does stride 2, for which only the explicit form is built (AUTO
+ * takes it).  C % 32 == 0 and I % 32 == 0 always.  The two forms round the
  * input gradient differently (explicit: nine bf16 partial results summed in fp32; implicit: one
  * fp32 accumulation), both within the products' tolerance. */
 enum { BIMASK_CONV_AUTO = 0, BIMASK_CONV_EXPLICIT = 1, BIMASK_CONV_IMPLICIT = 2 };
@@ -269,8 +272,9 @@ typedef struct bimask_conv_args {
   bimask_layer_args layer;
   int NB, H, W, C;
   int mode;
+  int stride;               /* 1 or 2 */
 } bimask_conv_args;
-size_t bimask_conv_workspace_bytes(int NB, int H, int W, int C, int I, int P);
+size_t bimask_conv_workspace_bytes(int NB, int H, int W, int C, int I, int P, int stride);
 int bimask_conv_layer_step(const bimask_conv_args* args);
 
 /* The same step for a caller whose data lives in HOST memory (pinned memory recommended):

@@ -50,7 +50,8 @@ class TrainArgs(Structure):
 
 class ConvArgs(Structure):
     """Mirror of bimask_conv_args."""
-    _fields_ = [("layer", LayerArgs), ("NB", c_int), ("H", c_int), ("W", c_int), ("C", c_int), ("mode", c_int)]
+    _fields_ = [("layer", LayerArgs), ("NB", c_int), ("H", c_int), ("W", c_int), ("C", c_int), ("mode", c_int),
+                ("stride", c_int)]
 
 
 CONV_AUTO, CONV_EXPLICIT, CONV_IMPLICIT = 0, 1, 2
@@ -90,7 +91,7 @@ def lib() -> ctypes.CDLL:
         L.bimask_perm_refine.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_uint64, c_void_p, c_void_p, c_void_p,
                                          c_size_t, c_void_p]
         L.bimask_conv_workspace_bytes.restype = c_size_t
-        L.bimask_conv_workspace_bytes.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int]
+        L.bimask_conv_workspace_bytes.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int, c_int]
         L.bimask_conv_layer_step.argtypes = [POINTER(ConvArgs)]
         L.bimask_bwd_mask_criterion.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_int,
                                                 c_uint64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
@@ -229,14 +230,14 @@ def bimask_sgd_fwd_mask(W, dW, mom_or_null, I, J, N, M, lr, momentum, weight_dec
                                             _stream(stream)))
 
 
-def bimask_conv_workspace_bytes(NB, H, W, C, I, P) -> int:
-    return lib().bimask_conv_workspace_bytes(NB, H, W, C, I, P)
+def bimask_conv_workspace_bytes(NB, H, W, C, I, P, stride=1) -> int:
+    return lib().bimask_conv_workspace_bytes(NB, H, W, C, I, P, stride)
 
 
-def make_conv_args(layer: LayerArgs, NB, H, W, C, mode=CONV_AUTO) -> ConvArgs:
+def make_conv_args(layer: LayerArgs, NB, H, W, C, mode=CONV_AUTO, stride=1) -> ConvArgs:
     a = ConvArgs()
     ctypes.memmove(ctypes.byref(a.layer), ctypes.byref(layer), ctypes.sizeof(LayerArgs))
-    a.NB, a.H, a.W, a.C, a.mode = NB, H, W, C, mode
+    a.NB, a.H, a.W, a.C, a.mode, a.stride = NB, H, W, C, mode, stride
     return a
 
 

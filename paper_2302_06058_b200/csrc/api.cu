@@ -333,7 +333,7 @@ int bimask_wgrad(const uint16_t* dY, const uint16_t* X, int T, int I, int J, flo
 // A 3x3 convolution layer seen by the layer step: geometry, which products fetch shifted pixel
 // patches themselves (implicit) and the column-space scratch of those that do not.
 struct ConvPlan {
-  int NB, H, W, C;
+  int NB, H, W, C, stride;
   bool imp_fwd, imp_dgrad, imp_wgrad;
   uint16_t* xcol;     // T x 9C, when the forward or weight-gradient product is explicit
   uint16_t* dxcol;    // T x 9C, when the input gradient is explicit
@@ -389,7 +389,7 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
     Xmat = conv->xcol;
     dXmat = conv->dxcol;
     if (!conv->imp_fwd || !conv->imp_wgrad)
-      if ((rc = launch_im2col3x3(a->X, conv->NB, conv->H, conv->W, conv->C, conv->xcol, s))) return rc;
+      if ((rc = launch_im2col3x3(a->X, conv->NB, conv->H, conv->W, conv->C, conv->stride, conv->xcol, s))) return rc;
   }
   // unpadded shapes: the mask kernels write the metadata images themselves
   const bool fused = pack && (a->I % 128 == 0) && (a->J % 128 == 0);
@@ -433,7 +433,7 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
   else rc = launch_dense_nt(a->vals_b, dYp, a->J, a->T, a->I, dXmat, a->status_word, s);
   if (rc) return rc;
   if (conv && !conv->imp_dgrad)
-    if ((rc = launch_col2im3x3(dXmat, conv->NB, conv->H, conv->W, conv->C, a->dX, s))) return rc;
+    if ((rc = launch_col2im3x3(dXmat, conv->NB, conv->H, conv->W, conv->C, conv->stride, a->dX, s))) return rc;
   if (conv && conv->imp_wgrad)
     return launch_wgrad_conv(a->dY, a->X, conv->NB, conv->H, conv->W, conv->C, a->I, a->dW, conv->wpart, a->status_word, s);
   return launch_wgrad_impl(a->dY, Xmat, a->T, a->I, a->J, a->dW, partials, a->status_word, s);
@@ -449,13 +449,13 @@ static size_t conv_wpart_bytes(int NB, int H, int W, int C, int I) {
   return splits > 1 ? align_up((size_t)splits * I * 9 * C * sizeof(float), 256) : 0;
 }
 
-size_t bimask_conv_workspace_bytes(int NB, int H, int W, int C, int I, int P) {
-  if (NB <= 0 || H <= 0 || W <= 0 || C <= 0 || I <= 0) return 0;
-  const long long T = (long long)NB * H * W;
+size_t bimask_conv_workspace_bytes(int NB, int H, int W, int C, int I, int P, int stride) {
+  if (NB <= 0 || H <= 0 || W <= 0 || C <= 0 || I <= 0 || (stride != 1 && stride != 2)) return 0;
+  const long long T = (long long)NB * ((H - 1) / stride + 1) * ((W - 1) / stride + 1);     // output pixels
   if (T > 0x7FFFFFFFll || 9ll * C > 0x7FFFFFFFll) return 0;
   const size_t col = align_up((size_t)T * 9 * C * 2, 256);
   // linear-layer scratch + column matrix + column-space gradient + partial sums of the implicit weight gradient
-  return plan_ws((int)T, I, 9 * C, P).total + 2 * col + conv_wpart_bytes(NB, H, W, C, I);
+  return plan_ws((int)T, I, 9 * C, P).total + 2 * col + (stride == 1 ? conv_wpart_bytes(NB, H, W, C, I) : 0);
 }
 
 int bimask_conv_layer_step(const bimask_conv_args* c) {
@@ -464,24 +464,27 @@ int bimask_conv_layer_step(const bimask_conv_args* c) {
   BIMASK_REQUIRE(c->NB > 0 && c->H > 0 && c->W > 0 && c->C > 0 && c->C % 32 == 0, BIMASK_EINVAL,
                  "bimask_conv_layer_step: NB = %d, H = %d, W = %d, C = %d: all positive, C a multiple of 32", c->NB, c->H,
                  c->W, c->C);
-  const long long T = (long long)c->NB * c->H * c->W;
+  BIMASK_REQUIRE(c->stride == 1 || c->stride == 2, BIMASK_EUNSUPPORTED, "bimask_conv_layer_step: stride %d (1 and 2 are implemented)",
+                 c->stride);
+  const long long T = (long long)c->NB * ((c->H - 1) / c->stride + 1) * ((c->W - 1) / c->stride + 1);
   BIMASK_REQUIRE(T <= 0x7FFFFFFFll && a->T == (int)T && a->J == 9 * c->C, BIMASK_EINVAL,
-                 "bimask_conv_layer_step: layer.T must be NB*H*W (%lld) and layer.J must be 9*C (%d)", T, 9 * c->C);
+                 "bimask_conv_layer_step: layer.T must be the number of output pixels (%lld) and layer.J must be 9*C (%d)", T,
+                 9 * c->C);
   BIMASK_REQUIRE(c->mode >= BIMASK_CONV_AUTO && c->mode <= BIMASK_CONV_IMPLICIT, BIMASK_EINVAL,
                  "bimask_conv_layer_step: mode %d out of range", c->mode);
   BIMASK_REQUIRE(a->ws && aligned16(a->ws), BIMASK_EINVAL, "bimask_conv_layer_step: null or misaligned workspace");
-  const size_t need = bimask_conv_workspace_bytes(c->NB, c->H, c->W, c->C, a->I, a->do_search && !a->cands ? a->P : 0);
+  const size_t need = bimask_conv_workspace_bytes(c->NB, c->H, c->W, c->C, a->I, a->do_search && !a->cands ? a->P : 0, c->stride);
   BIMASK_REQUIRE(a->ws_bytes >= need, BIMASK_EINVAL, "bimask_conv_layer_step: workspace too small (%zu bytes, need %zu)",
                  a->ws_bytes, need);
   ConvPlan plan;
-  plan.NB = c->NB; plan.H = c->H; plan.W = c->W; plan.C = c->C;
-  const bool packs = a->N <= 2;
-  const bool can_fwd = packs && c->C % 64 == 0;
-  const bool can_dgrad = packs && c->C % 128 == 0 && a->I % 128 == 0;
-  const bool can_wgrad = c->C % 64 == 0;
+  plan.NB = c->NB; plan.H = c->H; plan.W = c->W; plan.C = c->C; plan.stride = c->stride;
+  const bool packs = a->N <= 2, unit = c->stride == 1;          // the implicit form is built for stride 1
+  const bool can_fwd = unit && packs && c->C % 64 == 0;
+  const bool can_dgrad = unit && packs && c->C % 128 == 0 && a->I % 128 == 0;
+  const bool can_wgrad = unit && c->C % 64 == 0;
   BIMASK_REQUIRE(c->mode != BIMASK_CONV_IMPLICIT || (can_fwd && can_dgrad && can_wgrad), BIMASK_EUNSUPPORTED,
-                 "bimask_conv_layer_step: the implicit form needs C %% 128 == 0 and I %% 128 == 0 and a pattern with a 2:4 "
-                 "form (C = %d, I = %d, N:M = %d:%d)", c->C, a->I, a->N, a->M);
+                 "bimask_conv_layer_step: the implicit form needs stride 1, C %% 128 == 0, I %% 128 == 0 and a pattern with a "
+                 "2:4 form (stride %d, C = %d, I = %d, N:M = %d:%d)", c->stride, c->C, a->I, a->N, a->M);
   // AUTO: a column matrix that fits comfortably in L2 costs little, and the explicit form then has
   // fewer, denser k tiles (measured: 7x7 images of 512 channels are faster explicit, 14x14 of 256
   // channels faster implicit); above 16 MiB the implicit form wins by the HBM traffic it avoids.
@@ -491,7 +494,7 @@ int bimask_conv_layer_step(const bimask_conv_args* c) {
   plan.imp_dgrad = implicit && can_dgrad;
   plan.imp_wgrad = implicit && can_wgrad;
   const size_t col = align_up((size_t)T * 9 * c->C * 2, 256);
-  const size_t wpart = conv_wpart_bytes(c->NB, c->H, c->W, c->C, a->I);
+  const size_t wpart = unit ? conv_wpart_bytes(c->NB, c->H, c->W, c->C, a->I) : 0;
   uint8_t* tail = reinterpret_cast<uint8_t*>(a->ws) + (need - 2 * col - wpart);
   plan.xcol = reinterpret_cast<uint16_t*>(tail);
   plan.dxcol = reinterpret_cast<uint16_t*>(tail + col);

@@ -48,8 +48,8 @@ int launch_sgd_update(float* W, const float* dW, float* mom_or_null, long long n
                       float weight_decay, cudaStream_t s);
 int launch_hw_meta(const uint32_t* meta, int rows, int K, void* hw_meta, cudaStream_t s);
 // 3x3 convolution, explicit form: x (NHWC) -> column matrix [T][9C]; column-space gradient -> dx (NHWC)
-int launch_im2col3x3(const uint16_t* x, int NB, int H, int W, int C, uint16_t* cols, cudaStream_t s);
-int launch_col2im3x3(const uint16_t* dcols, int NB, int H, int W, int C, uint16_t* dx, cudaStream_t s);
+int launch_im2col3x3(const uint16_t* x, int NB, int H, int W, int C, int stride, uint16_t* cols, cudaStream_t s);
+int launch_col2im3x3(const uint16_t* dcols, int NB, int H, int W, int C, int stride, uint16_t* dx, cudaStream_t s);
 int launch_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                     int N, uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_or_null,
                     cudaStream_t s);

@@ -1,4 +1,4 @@
-// 3x3 convolution layers (stride 1, zero padding 1, NHWC activations) for the layer step.
+// 3x3 convolution layers (zero padding 1, stride 1 or 2, NHWC activations) for the layer step.
 // The filter is the paper's I x J weight matrix with J = 9*C and column j = (kh*3 + kw)*C + c, so
 // masks and search are unchanged.  This file holds the "explicit" form of the three products:
 // the activations are unfolded into the T x 9C column matrix (T = NB*H*W pixels), the linear-layer
@@ -12,19 +12,19 @@ namespace bimask {
 namespace {
 
 // One thread per 16-byte chunk (eight channels) of the column matrix.
-__global__ void im2col3x3_kernel(const uint4* __restrict__ x, int NB, int H, int W, int C8, long long total,
-                                 uint4* __restrict__ cols) {
+__global__ void im2col3x3_kernel(const uint4* __restrict__ x, int NB, int H, int W, int Ho, int Wo, int stride, int C8,
+                                 long long total, uint4* __restrict__ cols) {
   for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
        idx += (long long)gridDim.x * blockDim.x) {
     const int c8 = (int)(idx % C8);
     long long r = idx / C8;
     const int khw = (int)(r % 9);
-    r /= 9;                                              // pixel index t = (n*H + h)*W + w
-    const int w = (int)(r % W);
-    const long long nh = r / W;
-    const int h = (int)(nh % H);
-    const long long n = nh / H;
-    const int hs = h + khw / 3 - 1, ws = w + khw % 3 - 1;
+    r /= 9;                                              // output pixel index t = (n*Ho + ho)*Wo + wo
+    const int wo = (int)(r % Wo);
+    const long long nh = r / Wo;
+    const int ho = (int)(nh % Ho);
+    const long long n = nh / Ho;
+    const int hs = ho * stride + khw / 3 - 1, ws = wo * stride + khw % 3 - 1;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (hs >= 0 && hs < H && ws >= 0 && ws < W) v = __ldg(x + ((n * H + hs) * W + ws) * C8 + c8);
     cols[idx] = v;
@@ -42,9 +42,10 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return d;
 }
 
-// dx[n, h, w, c] = sum over the nine taps of dXcol[(n, h-kh+1, w-kw+1), (kh*3+kw)*C + c]; fp32 sums.
-__global__ void col2im3x3_kernel(const uint4* __restrict__ dcols, int NB, int H, int W, int C8, long long total,
-                                 uint4* __restrict__ dx) {
+// dx[n, h, w, c] = sum over the nine taps of dXcol[(n, ho, wo), (kh*3+kw)*C + c] with ho*stride + kh - 1 = h and
+// wo*stride + kw - 1 = w (taps with no such output pixel contribute nothing); fp32 sums.
+__global__ void col2im3x3_kernel(const uint4* __restrict__ dcols, int NB, int H, int W, int Ho, int Wo, int stride, int C8,
+                                 long long total, uint4* __restrict__ dx) {
   for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
        idx += (long long)gridDim.x * blockDim.x) {
     const int c8 = (int)(idx % C8);
@@ -58,9 +59,10 @@ __global__ void col2im3x3_kernel(const uint4* __restrict__ dcols, int NB, int H,
     for (int j = 0; j < 8; ++j) acc[j] = 0.f;
 #pragma unroll
     for (int khw = 0; khw < 9; ++khw) {
-      const int hs = h - khw / 3 + 1, ws = w - khw % 3 + 1;
-      if (hs >= 0 && hs < H && ws >= 0 && ws < W) {
-        const uint4 v = __ldg(dcols + (((n * H + hs) * W + ws) * 9 + khw) * C8 + c8);
+      const int hn = h - khw / 3 + 1, wn = w - khw % 3 + 1;       // = ho * stride, wo * stride
+      const int hs = hn / stride, ws = wn / stride;
+      if (hn >= 0 && wn >= 0 && hs * stride == hn && ws * stride == wn && hs < Ho && ws < Wo) {
+        const uint4 v = __ldg(dcols + (((n * Ho + hs) * Wo + ws) * 9 + khw) * C8 + c8);
         add_bf16x2(acc[0], acc[1], v.x);
         add_bf16x2(acc[2], acc[3], v.y);
         add_bf16x2(acc[4], acc[5], v.z);
@@ -74,22 +76,24 @@ __global__ void col2im3x3_kernel(const uint4* __restrict__ dcols, int NB, int H,
 
 }  // namespace
 
-int launch_im2col3x3(const uint16_t* x, int NB, int H, int W, int C, uint16_t* cols, cudaStream_t s) {
-  const long long total = (long long)NB * H * W * 9 * (C / 8);
+int launch_im2col3x3(const uint16_t* x, int NB, int H, int W, int C, int stride, uint16_t* cols, cudaStream_t s) {
+  const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+  const long long total = (long long)NB * Ho * Wo * 9 * (C / 8);
   long long ctas = (total + 255) / 256;
   if (ctas > 148 * 16) ctas = 148 * 16;
-  im2col3x3_kernel<<<(unsigned)ctas, 256, 0, s>>>(reinterpret_cast<const uint4*>(x), NB, H, W, C / 8, total,
+  im2col3x3_kernel<<<(unsigned)ctas, 256, 0, s>>>(reinterpret_cast<const uint4*>(x), NB, H, W, Ho, Wo, stride, C / 8, total,
                                                   reinterpret_cast<uint4*>(cols));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }
 
-int launch_col2im3x3(const uint16_t* dcols, int NB, int H, int W, int C, uint16_t* dx, cudaStream_t s) {
+int launch_col2im3x3(const uint16_t* dcols, int NB, int H, int W, int C, int stride, uint16_t* dx, cudaStream_t s) {
+  const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
   const long long total = (long long)NB * H * W * (C / 8);
   long long ctas = (total + 255) / 256;
   if (ctas > 148 * 16) ctas = 148 * 16;
-  col2im3x3_kernel<<<(unsigned)ctas, 256, 0, s>>>(reinterpret_cast<const uint4*>(dcols), NB, H, W, C / 8, total,
+  col2im3x3_kernel<<<(unsigned)ctas, 256, 0, s>>>(reinterpret_cast<const uint4*>(dcols), NB, H, W, Ho, Wo, stride, C / 8, total,
                                                   reinterpret_cast<uint4*>(dx));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());

@@ -22,16 +22,16 @@ def conv_case(NB, H, W, C, I, seed):
     return Wt, x, dy
 
 
-def run_conv_step(Wt, x, dy, N, M, P, seed, mode, do_search=True):
+def run_conv_step(Wt, x, dy, N, M, P, seed, mode, do_search=True, stride=1):
     NB, H, W, C = x.shape
     I = Wt.shape[0]
-    T, J = NB * H * W, 9 * C
+    T, J = dy.shape[0] * dy.shape[1] * dy.shape[2], 9 * C
     b = bm.alloc_layer_buffers(T, I, J, P)
     b["W"], b["X"], b["dY"] = dev(Wt), bits_dev(x), bits_dev(dy)
     b["dX"] = torch.empty(NB, H, W, C, dtype=torch.bfloat16, device="cuda")
-    b["ws"] = torch.empty(bm.bimask_conv_workspace_bytes(NB, H, W, C, I, P), dtype=torch.uint8, device="cuda")
+    b["ws"] = torch.empty(bm.bimask_conv_workspace_bytes(NB, H, W, C, I, P, stride), dtype=torch.uint8, device="cuda")
     largs = bm.make_layer_args(T, I, J, N, M, P, seed, do_search, b)
-    bm.bimask_conv_layer_step(bm.make_conv_args(largs, NB, H, W, C, mode))
+    bm.bimask_conv_layer_step(bm.make_conv_args(largs, NB, H, W, C, mode, stride))
     torch.cuda.synchronize()
     return b
 
@@ -88,6 +88,29 @@ def test_conv_implicit_form_other_patterns(N, M):
     assert rel_err(b["dW"].cpu().numpy(), ref["dW"]) <= TOL
 
 
+@pytest.mark.parametrize("NB,H,W,C,I", [(2, 9, 11, 32, 64), (3, 14, 14, 64, 128), (2, 56, 56, 128, 128), (4, 28, 27, 256, 256)])
+def test_conv_stride_2(NB, H, W, C, I):
+    """ResNet's down-sampling 3x3 convolutions (stride 2): odd and even image sizes; the explicit form serves them,
+    and the automatic mode must choose it."""
+    N, M, P, seed = 2, 4, 4, 23
+    Ho, Wo = O.conv_out_size(H, 2), O.conv_out_size(W, 2)
+    Wt = inputs.make_weight(I, 9 * C, 330 + H)
+    x = inputs.make_activation(NB * H * W, C, 331).reshape(NB, H, W, C)
+    dy = inputs.make_activation(NB * Ho * Wo, I, 332).reshape(NB, Ho, Wo, I)
+    ref = O.conv_layer_step(Wt, x, dy, N, M, P, seed, stride=2)
+    for mode in (bm.binding.CONV_EXPLICIT, bm.binding.CONV_AUTO):
+        b = run_conv_step(Wt, x, dy, N, M, P, seed, mode, stride=2)
+        assert int(b["status_word"].item()) == 0
+        assert np.array_equal(b["perm"].cpu().numpy(), ref["perm"])
+        assert np.array_equal(u16(b["vals_b"]), ref["vals_b"])
+        assert rel_err(b["Y"].float().cpu().numpy().reshape(NB, Ho, Wo, I), ref["y"]) <= TOL
+        assert rel_err(b["dX"].float().cpu().numpy(), ref["dx"]) <= TOL
+        assert rel_err(b["dW"].cpu().numpy(), ref["dW"]) <= TOL
+    with pytest.raises(bm.BimaskError) as e:
+        run_conv_step(Wt, x, dy, N, M, P, seed, bm.binding.CONV_IMPLICIT, stride=2)
+    assert e.value.code == -2
+
+
 def test_conv_bad_arguments_launch_nothing():
     NB, H, W, C, I = 1, 8, 8, 32, 32
     Wt, x, dy = conv_case(NB, H, W, C, I, 1)
@@ -102,11 +125,11 @@ def test_conv_bad_arguments_launch_nothing():
     assert e.value.code == -1 and "workspace" in str(e.value)
     b["ws"] = torch.empty(bm.bimask_conv_workspace_bytes(NB, H, W, C, I, 2), dtype=torch.uint8, device="cuda")
     largs = bm.make_layer_args(T, I, J, 2, 4, 2, 1, True, b)
-    for kw in (dict(H=7), dict(C=48), dict(mode=5)):
-        geo = dict(NB=NB, H=H, W=W, C=C, mode=0)
+    for kw in (dict(H=7), dict(C=48), dict(mode=5), dict(stride=2)):
+        geo = dict(NB=NB, H=H, W=W, C=C, mode=0, stride=1)
         geo.update(kw)
         with pytest.raises(bm.BimaskError) as e:
-            bm.bimask_conv_layer_step(bm.make_conv_args(largs, geo["NB"], geo["H"], geo["W"], geo["C"], geo["mode"]))
+            bm.bimask_conv_layer_step(bm.make_conv_args(largs, geo["NB"], geo["H"], geo["W"], geo["C"], geo["mode"], geo["stride"]))
         assert e.value.code == -1
     with pytest.raises(bm.BimaskError) as e:                             # C = 32 cannot take the implicit form
         bm.bimask_conv_layer_step(bm.make_conv_args(largs, NB, H, W, C, bm.binding.CONV_IMPLICIT))
