@@ -612,3 +612,53 @@ def conv_layer_step(W, x_bits, dy_bits, N, M, P, seed, do_search=True, perm=None
     out["dx"] = conv_dgrad(dy_bits, W, out["M_b"], C, stride, (H, Wd))
     out["dW"] = conv_wgrad(dy_bits, x_bits, stride)
     return out
+
+
+# ---------------------------------------------------------------------------------------
+# Greedy refinement of a permutation (beyond the paper: its conclusion names a better search than
+# "best of K random candidates" as future work).  Not part of Algorithm 1.
+# ---------------------------------------------------------------------------------------
+REFINE_SEED_OFFSET = 0x5EED5EED
+
+
+def _block_eligible(B, rows, N):
+    """Columns of the row block `rows` (M row indices of B) that hold at most N ones."""
+    return int((B[np.asarray(rows, dtype=np.int64), :].sum(axis=0) <= N).sum())
+
+
+def refine_perm(B, perm, N, M, rounds, seed):
+    """Pairwise-swap hill climbing on the eligible-block count.  Round r pairs up the POSITIONS of the
+    permutation at random: with order = candidates(seed + REFINE_SEED_OFFSET, rounds, I)[r], pair i is
+    (a, b) = (order[2i], order[2i+1]).  A pair whose positions lie in different row blocks ka != kb
+    has gain = (eligible columns of the two blocks after exchanging perm[a] and perm[b]) - (before),
+    all gains taken against the permutation at the start of the round.  A pair is accepted when its
+    gain is positive and, for BOTH of its blocks, it is the best pair touching that block (largest
+    gain, lowest pair index on equal gain) -- so accepted pairs never share a block, their gains add
+    up, and the count never decreases.  Returns (perm, eligible-block count of the result)."""
+    perm = np.array(perm, dtype=np.int32).copy()
+    I = perm.shape[0]
+    assert I % M == 0
+    orders = candidates((int(seed) + REFINE_SEED_OFFSET) & MASK64, rounds, I) if rounds > 0 else None
+    for r in range(rounds):
+        order = orders[r]
+        gains = {}
+        best = {}                                            # block -> (gain, -pair index) of its best pair
+        for i in range(I // 2):
+            a, b = int(order[2 * i]), int(order[2 * i + 1])
+            ka, kb = a // M, b // M
+            if ka == kb:
+                continue
+            rows_a = perm[ka * M:(ka + 1) * M].copy()
+            rows_b = perm[kb * M:(kb + 1) * M].copy()
+            before = _block_eligible(B, rows_a, N) + _block_eligible(B, rows_b, N)
+            rows_a[a - ka * M], rows_b[b - kb * M] = perm[b], perm[a]
+            gain = _block_eligible(B, rows_a, N) + _block_eligible(B, rows_b, N) - before
+            if gain > 0:
+                gains[i] = (gain, a, b, ka, kb)
+                for k in (ka, kb):
+                    if k not in best or (gain, -i) > best[k]:
+                        best[k] = (gain, -i)
+        for i, (gain, a, b, ka, kb) in gains.items():
+            if best[ka] == (gain, -i) and best[kb] == (gain, -i):
+                perm[a], perm[b] = perm[b], perm[a]
+    return perm, eligible_blocks(B, perm, N, M)
