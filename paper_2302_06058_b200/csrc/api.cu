@@ -202,12 +202,13 @@ int bimask_perm_search(const uint32_t* maskbits_f, int I, int J, int N, int M, i
     BIMASK_REQUIRE(ws && aligned16(ws) && ws_bytes >= w.cands_off + w.cands_bytes, BIMASK_EINVAL,
                    "bimask_perm_search: workspace too small (%zu bytes, need %zu)", ws_bytes, w.cands_off + w.cands_bytes);
     int32_t* gen = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(ws) + w.cands_off);
-    if ((rc = launch_gen_candidates(seed, P, I, gen, s)) != BIMASK_OK) return rc;
+    // M = 4: the generator zeroes counts and the pick's CTA counter, the count kernel picks the winner itself
+    if ((rc = launch_gen_candidates(seed, P, I, gen, s, M == 4 ? counts : nullptr, M == 4 ? best_idx : nullptr)) != BIMASK_OK)
+      return rc;
     cands = gen;
   }
-  if (M == 4) rc = launch_score(maskbits_f, cands, I, J, N, P, counts, s);
-  else rc = launch_score_generic(maskbits_f, cands, I, J, N, M, P, counts, s);
-  if (rc != BIMASK_OK) return rc;
+  if (M == 4) return launch_score(maskbits_f, cands, I, J, N, P, counts, s, cands_or_null == nullptr, best_idx, best_perm);
+  if ((rc = launch_score_generic(maskbits_f, cands, I, J, N, M, P, counts, s)) != BIMASK_OK) return rc;
   return launch_pick(counts, cands, P, I, best_idx, best_perm, s);
 }
 
@@ -410,13 +411,19 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
   if (a->do_search) {
     const int32_t* cands = a->cands;
     if (!cands) {
-      if ((rc = launch_gen_candidates(a->seed, a->P, a->I, gen, s))) return rc;
+      if ((rc = launch_gen_candidates(a->seed, a->P, a->I, gen, s, a->M == 4 ? a->counts : nullptr,
+                                      a->M == 4 ? a->best_idx : nullptr)))
+        return rc;
       cands = gen;
     }
-    if (a->M == 4) rc = launch_score(a->maskbits_f, cands, a->I, a->J, a->N, a->P, a->counts, s);
-    else rc = launch_score_generic(a->maskbits_f, cands, a->I, a->J, a->N, a->M, a->P, a->counts, s);
-    if (rc) return rc;
-    if ((rc = launch_pick(a->counts, cands, a->P, a->I, a->best_idx, a->perm, s))) return rc;
+    if (a->M == 4) {
+      // the count kernel's last CTA picks the winner and copies it into perm
+      if ((rc = launch_score(a->maskbits_f, cands, a->I, a->J, a->N, a->P, a->counts, s, a->cands == nullptr, a->best_idx, a->perm)))
+        return rc;
+    } else {
+      if ((rc = launch_score_generic(a->maskbits_f, cands, a->I, a->J, a->N, a->M, a->P, a->counts, s))) return rc;
+      if ((rc = launch_pick(a->counts, cands, a->P, a->I, a->best_idx, a->perm, s))) return rc;
+    }
   }
   if (a->M == 4)
     rc = launch_bwd_mask(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->maskbits_b, a->vals_b, a->meta_b,

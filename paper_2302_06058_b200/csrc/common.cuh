@@ -53,9 +53,13 @@ int launch_col2im3x3(const uint16_t* dcols, int NB, int H, int W, int C, int str
 int launch_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                     int N, uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_or_null,
                     cudaStream_t s);
-int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStream_t s);
+// zero_counts / zero_ticket (optional): the generator also zeroes counts[0..P) and *zero_ticket for the count kernel
+int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStream_t s, int64_t* zero_counts = nullptr,
+                          int32_t* zero_ticket = nullptr);
+// best_idx / best_perm (optional): fused pick by the kernel's last CTA; zeroed: counts and *best_idx are already zero
 int launch_score(const uint32_t* maskbits_f, const int32_t* cands, int I, int J, int N, int P,
-                 int64_t* counts, cudaStream_t s);
+                 int64_t* counts, cudaStream_t s, bool zeroed = false, int32_t* best_idx = nullptr,
+                 int32_t* best_perm = nullptr);
 int launch_pick(const int64_t* counts, const int32_t* cands, int P, int I, int32_t* best_idx,
                 int32_t* best_perm, cudaStream_t s);
 // N:M patterns with M = 8 or 16 (nm_generic_kernels.cu); vals / meta may be null (mask bits only).

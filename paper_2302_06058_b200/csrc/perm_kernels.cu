@@ -32,7 +32,8 @@ constexpr int GEN_THREADS = 1024;
 
 __global__ void __launch_bounds__(GEN_THREADS)
 gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int q_log2, int cap,
-                      int32_t* __restrict__ cands) {
+                      int32_t* __restrict__ cands, unsigned long long* __restrict__ zero_counts,
+                      int32_t* __restrict__ zero_ticket) {
   extern __shared__ unsigned long long keys[];           // cap keys, then nbq bucket counters
   const int nbq_log2 = nb_log2 - q_log2;
   const int nbq = 1 << nbq_log2;
@@ -45,7 +46,12 @@ gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int q_log2, i
   const unsigned long long stream = mix64(seed + 0x9E3779B97F4A7C15ull * (unsigned long long)(c + 1));
   const int shift = 64 - nb_log2;
   for (int b = tid; b < nbq; b += GEN_THREADS) count[b] = 0;
-  if (tid == 0) lower_total = 0;
+  if (tid == 0) {
+    lower_total = 0;
+    // the count kernel that follows adds into counts[c] and uses *zero_ticket as its "CTAs done" counter
+    if (part == 0 && zero_counts) zero_counts[c] = 0ull;
+    if (part == 0 && c == 0 && zero_ticket) *zero_ticket = 0;
+  }
   __syncthreads();
   uint32_t lower = 0;
   for (int i = tid; i < I; i += GEN_THREADS) {
@@ -116,6 +122,47 @@ gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int q_log2, i
 }
 
 // ---------------------------------------------------------------------------------------
+// Pick: arg-max of counts with ties to the lowest candidate index, then copy that candidate.
+// ---------------------------------------------------------------------------------------
+constexpr int PICK_THREADS = 256;
+
+// One CTA of PICK_THREADS threads; counts are read around L1 (they were written by atomics of other CTAs).
+__device__ __forceinline__ void pick_body(const long long* counts, const int32_t* __restrict__ cands, int P, int I,
+                                          int32_t* best_idx, int32_t* __restrict__ best_perm) {
+  __shared__ long long s_cnt[PICK_THREADS];
+  __shared__ int s_idx[PICK_THREADS];
+  long long bc = -1;
+  int bi = 0x7FFFFFFF;
+  for (int c = threadIdx.x; c < P; c += PICK_THREADS) {
+    const long long v = __ldcg(counts + c);
+    if (v > bc) { bc = v; bi = c; }      // ascending c per thread: first maximum is kept
+  }
+  s_cnt[threadIdx.x] = bc;
+  s_idx[threadIdx.x] = bi;
+  __syncthreads();
+  for (int s = PICK_THREADS / 2; s > 0; s >>= 1) {
+    if (threadIdx.x < s) {
+      const long long oc = s_cnt[threadIdx.x + s];
+      const int oi = s_idx[threadIdx.x + s];
+      if (oc > s_cnt[threadIdx.x] || (oc == s_cnt[threadIdx.x] && oi < s_idx[threadIdx.x])) {
+        s_cnt[threadIdx.x] = oc;
+        s_idx[threadIdx.x] = oi;
+      }
+    }
+    __syncthreads();
+  }
+  const int best = s_idx[0];
+  if (threadIdx.x == 0) *best_idx = best;
+  for (int i = threadIdx.x; i < I; i += PICK_THREADS) best_perm[i] = cands[(long long)best * I + i];
+}
+
+__global__ void __launch_bounds__(PICK_THREADS)
+pick_kernel(const long long* __restrict__ counts, const int32_t* __restrict__ cands, int P, int I,
+            int32_t* __restrict__ best_idx, int32_t* __restrict__ best_perm) {
+  pick_body(counts, cands, P, I, best_idx, best_perm);
+}
+
+// ---------------------------------------------------------------------------------------
 // Eligible-block count.  grid = (row-block chunks, P).  A warp takes one row block of a
 // candidate at a time: the four row indices are one 16-byte load, each lane then reads its
 // slice of the four mask rows (128-bit loads when J % 128 == 0) and counts columns whose
@@ -140,7 +187,7 @@ __device__ __forceinline__ uint32_t ineligible(uint32_t a, uint32_t b, uint32_t 
 template <int N>
 __global__ void __launch_bounds__(SCORE_THREADS, 4)
 score_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cands, int I, int jwords,
-             unsigned long long* __restrict__ counts) {
+             unsigned long long* __restrict__ counts, int P, int32_t* best_idx, int32_t* __restrict__ best_perm) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int c = blockIdx.y;
   const int nkb = I >> 2;
@@ -203,47 +250,26 @@ score_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cand
   __shared__ uint32_t part[SCORE_THREADS / 32];
   if (lane == 0) part[warp] = cnt;
   __syncthreads();
+  __shared__ bool last_cta;
   if (threadIdx.x == 0) {
     unsigned long long s = 0;
 #pragma unroll
     for (int w = 0; w < SCORE_THREADS / 32; ++w) s += part[w];
     atomicAdd(counts + c, s);
-  }
-}
-
-// ---------------------------------------------------------------------------------------
-// Pick: arg-max of counts with ties to the lowest candidate index, then copy that candidate.
-// ---------------------------------------------------------------------------------------
-constexpr int PICK_THREADS = 256;
-
-__global__ void __launch_bounds__(PICK_THREADS)
-pick_kernel(const long long* __restrict__ counts, const int32_t* __restrict__ cands, int P, int I,
-            int32_t* __restrict__ best_idx, int32_t* __restrict__ best_perm) {
-  __shared__ long long s_cnt[PICK_THREADS];
-  __shared__ int s_idx[PICK_THREADS];
-  long long bc = -1;
-  int bi = 0x7FFFFFFF;
-  for (int c = threadIdx.x; c < P; c += PICK_THREADS) {
-    const long long v = counts[c];
-    if (v > bc) { bc = v; bi = c; }      // ascending c per thread: first maximum is kept
-  }
-  s_cnt[threadIdx.x] = bc;
-  s_idx[threadIdx.x] = bi;
-  __syncthreads();
-  for (int s = PICK_THREADS / 2; s > 0; s >>= 1) {
-    if (threadIdx.x < s) {
-      const long long oc = s_cnt[threadIdx.x + s];
-      const int oi = s_idx[threadIdx.x + s];
-      if (oc > s_cnt[threadIdx.x] || (oc == s_cnt[threadIdx.x] && oi < s_idx[threadIdx.x])) {
-        s_cnt[threadIdx.x] = oc;
-        s_idx[threadIdx.x] = oi;
-      }
+    last_cta = false;
+    if (best_idx) {
+      // fused pick: *best_idx counts the CTAs that have added their share (zeroed before the launch); the CTA that
+      // completes the grid sees every sum (fence on both sides of the counter) and picks the winner
+      __threadfence();
+      const unsigned done = atomicAdd(reinterpret_cast<unsigned*>(best_idx), 1u);
+      last_cta = done == gridDim.x * gridDim.y - 1u;
     }
-    __syncthreads();
   }
-  const int best = s_idx[0];
-  if (threadIdx.x == 0) *best_idx = best;
-  for (int i = threadIdx.x; i < I; i += PICK_THREADS) best_perm[i] = cands[(long long)best * I + i];
+  __syncthreads();
+  if (last_cta) {
+    __threadfence();
+    pick_body(reinterpret_cast<const long long*>(counts), cands, P, I, best_idx, best_perm);
+  }
 }
 
 // Debug: every row of cands is a permutation of 0..I-1.
@@ -264,7 +290,8 @@ __global__ void set_int_kernel(int32_t* p, int32_t v) { *p = v; }
 
 }  // namespace
 
-int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStream_t s) {
+int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStream_t s, int64_t* zero_counts,
+                          int32_t* zero_ticket) {
   int lg = 1;
   while ((1 << lg) < I) ++lg;                             // one bucket per key on average
   int ql = 0;
@@ -278,25 +305,43 @@ int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStrea
     attr_done = true;
   }
   dim3 grid(P, 1 << ql);
-  gen_candidates_kernel<<<grid, GEN_THREADS, smem, s>>>((unsigned long long)seed, I, lg, ql, cap, cands);
+  gen_candidates_kernel<<<grid, GEN_THREADS, smem, s>>>((unsigned long long)seed, I, lg, ql, cap, cands,
+                                                        reinterpret_cast<unsigned long long*>(zero_counts), zero_ticket);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }
 
+// best_idx / best_perm given: the kernel also picks the winner (its last CTA), so no pick launch is needed.
+// zeroed: counts (and *best_idx, the fused pick's CTA counter) were already zeroed on the stream, e.g. by the
+// candidate generator.
 int launch_score(const uint32_t* maskbits_f, const int32_t* cands, int I, int J, int N, int P,
-                 int64_t* counts, cudaStream_t s) {
-  BIMASK_CUDA_OK(cudaMemsetAsync(counts, 0, (size_t)P * sizeof(int64_t), s));
+                 int64_t* counts, cudaStream_t s, bool zeroed, int32_t* best_idx, int32_t* best_perm) {
   dim3 grid((I / 4 + SCORE_KB_PER_CTA - 1) / SCORE_KB_PER_CTA, P);
+  // The fused pick costs every CTA a fence and an atomic on one counter: a win for small grids (it saves a launch
+  // of a few microseconds), a loss for thousands of CTAs (measured: +8 us on 2048 CTAs, +24 us on 8192), which keep the
+  // separate pick kernel.
+  int32_t* pick_idx = best_idx, *pick_perm = best_perm;
+  const bool fuse = best_idx != nullptr && (long long)grid.x * grid.y <= 1024;
+  if (!fuse) best_idx = nullptr;
+  if (!zeroed) {
+    BIMASK_CUDA_OK(cudaMemsetAsync(counts, 0, (size_t)P * sizeof(int64_t), s));
+    if (best_idx) BIMASK_CUDA_OK(cudaMemsetAsync(best_idx, 0, sizeof(int32_t), s));
+  }
   unsigned long long* cnt = reinterpret_cast<unsigned long long*>(counts);
   switch (N) {
-    case 1: score_kernel<1><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt); break;
-    case 2: score_kernel<2><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt); break;
-    case 3: score_kernel<3><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt); break;
-    default: score_kernel<4><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt); break;
+    case 1: score_kernel<1><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm); break;
+    case 2: score_kernel<2><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm); break;
+    case 3: score_kernel<3><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm); break;
+    default: score_kernel<4><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm); break;
   }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
+  if (pick_idx && !fuse) {
+    pick_kernel<<<1, PICK_THREADS, 0, s>>>(reinterpret_cast<const long long*>(counts), cands, P, I, pick_idx, pick_perm);
+    count_launch();
+    BIMASK_CUDA_OK(cudaGetLastError());
+  }
   return BIMASK_OK;
 }
 
