@@ -260,8 +260,8 @@ int bimask_train_step(const bimask_train_args* args);
  * products and folds the column-space input gradient back (sum of the nine shifts, fp32);
  * BIMASK_CONV_IMPLICIT never builds the column matrix: the GEMM kernels fetch shifted pixel
  * patches with 4-D tensor loads (out-of-image pixels read as zero); BIMASK_CONV_AUTO takes the
- * implicit form for every product whose shape allows it (C % 64 == 0; the input gradient also
- * needs C % 128 == 0 and I % 128 == 0; patterns with a 2:4 form) when the column matrix would
+ * implicit form for every product whose shape allows it (C % 64 == 0; the input gradient needs
+ * C == 64 or C % 128 == 0; patterns with a 2:4 form) when the column matrix would
  * exceed 16 MiB, and the explicit form otherwise.  IMPLICIT with a shape that does not allow it
  * returns BIMASK_EUNSUPPORTED; so does stride 2, for which only the explicit form is built (AUTO
  * takes it).  C % 32 == 0 and I % 32 == 0 always.  The two forms round the

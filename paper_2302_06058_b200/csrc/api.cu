@@ -487,11 +487,11 @@ int bimask_conv_layer_step(const bimask_conv_args* c) {
   plan.NB = c->NB; plan.H = c->H; plan.W = c->W; plan.C = c->C; plan.stride = c->stride;
   const bool packs = a->N <= 2, unit = c->stride == 1;          // the implicit form is built for stride 1
   const bool can_fwd = unit && packs && c->C % 64 == 0;
-  const bool can_dgrad = unit && packs && c->C % 128 == 0 && a->I % 128 == 0;
+  const bool can_dgrad = unit && packs && (c->C % 128 == 0 || c->C == 64);
   const bool can_wgrad = unit && c->C % 64 == 0;
   BIMASK_REQUIRE(c->mode != BIMASK_CONV_IMPLICIT || (can_fwd && can_dgrad && can_wgrad), BIMASK_EUNSUPPORTED,
-                 "bimask_conv_layer_step: the implicit form needs stride 1, C %% 128 == 0, I %% 128 == 0 and a pattern with a "
-                 "2:4 form (stride %d, C = %d, I = %d, N:M = %d:%d)", c->stride, c->C, a->I, a->N, a->M);
+                 "bimask_conv_layer_step: the implicit form needs stride 1, C = 64 or a multiple of 128, and a pattern with "
+                 "a 2:4 form (stride %d, C = %d, I = %d, N:M = %d:%d)", c->stride, c->C, a->I, a->N, a->M);
   // AUTO: a column matrix that fits comfortably in L2 costs little, and the explicit form then has
   // fewer, denser k tiles (measured: 7x7 images of 512 channels are faster explicit, 14x14 of 256
   // channels faster implicit); above 16 MiB the implicit form wins by the HBM traffic it avoids.

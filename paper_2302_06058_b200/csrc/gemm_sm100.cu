@@ -194,8 +194,18 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
             ptx::tma_load_4d(b_s + q * (N_TILE * 128), &tmapB, valid ? c0 : 0, cw0 + dw, ch0 + dh, valid ? cn0 : p.conv.NB,
                              full_bar(s));
           }
-          ptx::bulk_load(b_s + C::B_BYTES,
-                         p.hw_meta + ((size_t)meta_row * p.tiles_k_meta + meta_kt) * 2048, 2048, full_bar(s));
+          {
+            // 64 rows per tap (C = 64): every other tap starts in the middle of a 128-row metadata block; its rows
+            // are that block's lanes 64..127 (the second KiB), which must land in lanes 0..63 of the tile.  The
+            // tile's other 64 rows belong to another tap and are never stored: they get the block's other half.
+            const uint8_t* blk = p.hw_meta + ((size_t)meta_row * p.tiles_k_meta + meta_kt) * 2048;
+            if (a_row & 64) {
+              ptx::bulk_load(b_s + C::B_BYTES, blk + 1024, 1024, full_bar(s));
+              ptx::bulk_load(b_s + C::B_BYTES + 1024, blk, 1024, full_bar(s));
+            } else {
+              ptx::bulk_load(b_s + C::B_BYTES, blk, 2048, full_bar(s));
+            }
+          }
           continue;
         }
         if (SPARSE) {
@@ -1625,7 +1635,7 @@ int run_conv_pair(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_m
 // 3x3 convolution products without a column matrix (see ConvGeom).
 //   forward:        D[i, pixel] = sum_{tap, c} A_f[i, tap*C + c] x[pixel + tap, c];  vals/hw_meta of the I x 9C operand
 //   input gradient: D[c, pixel] = sum_{tap, i'} A'[tap*C + c, i'] dyp[pixel - tap, i'];  vals/hw_meta of the 9C x I operand
-// out is NHWC with Mdim channels.  Needs C % 64 == 0 (forward) or C % 128 == 0 and I % 128 == 0 (input gradient).
+// out is NHWC with Mdim channels.  Needs C % 64 == 0 (forward); C % 128 == 0 or C == 64 (input gradient).
 int launch_spmm_conv(int mode, const uint16_t* vals, const void* hw_meta, const uint16_t* tok, int NB, int H, int W, int C,
                      int I, uint16_t* out, int32_t* status_word, cudaStream_t s) {
   ConvGeom g{};
@@ -1636,8 +1646,8 @@ int launch_spmm_conv(int mode, const uint16_t* vals, const void* hw_meta, const 
     g.CB = C; g.kt_per_tap = 0; g.rows_per_tap = 0;
     Mdim = I; Kdim = 9 * C; a_rows = I; a_kdim = 9 * C; tiles_k_meta = (9 * C + 127) / 128;
   } else {
-    g.CB = I; g.kt_per_tap = I / 128; g.rows_per_tap = C;
-    Mdim = C; Kdim = 9 * I; a_rows = 9 * C; a_kdim = I; tiles_k_meta = I / 128;
+    g.CB = I; g.kt_per_tap = (I + 127) / 128; g.rows_per_tap = C;
+    Mdim = C; Kdim = 9 * g.kt_per_tap * 128; a_rows = 9 * C; a_kdim = I; tiles_k_meta = g.kt_per_tap;
   }
   if (Mdim > 128 && T > 128)
     return run_conv_pair(vals, a_rows, a_kdim, hw_meta, tok, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
