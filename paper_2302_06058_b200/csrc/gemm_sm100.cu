@@ -373,13 +373,17 @@ struct PairPCfg {
   static constexpr int B_MAX = 32768;                      // up to 128 rows x 128 bf16 (two 64-wide boxes)
   static constexpr int E_BYTES = 2048;
   static constexpr int STAGE_BYTES = A_BYTES + B_MAX + E_BYTES;        // 50 KB (the B part is N / 2 rows)
-  static constexpr int STAGING_BYTES = 4 * 2 * 2048;       // per epilogue warp: two [<= 32 tokens][32 rows] bf16 buffers
+  static constexpr int STAGING_BYTES = 8 * 2 * 2048;       // per epilogue warp: two [<= 32 tokens][32 rows] bf16 buffers
   static constexpr int TMEM_COLS = 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 + 256;
 };
 
+// Eight epilogue warps (two per tensor-memory lane quadrant, taking alternate column chunks): products with
+// a short reduction are bound by the drain of the accumulator, not by the tensor pipe.
+constexpr int PAIR_THREADS = 320;
+
 template <int STAGES, bool CONV>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PAIR_THREADS, 1)
 spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                             const __grid_constant__ CUtensorMap tmapE, const __grid_constant__ CUtensorMap tmapOut32,
                             const __grid_constant__ CUtensorMap tmapOut16, const GemmParams p) {
@@ -416,7 +420,7 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(tmem_full_bar(b), 1);
-      ptx::mbar_init(tmem_empty_bar(b), 8);               // four epilogue warps in each CTA of the pair
+      ptx::mbar_init(tmem_empty_bar(b), 16);              // eight epilogue warps in each CTA of the pair
     }
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmapA);
@@ -518,8 +522,9 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
     // 2 KB staging buffers; warps never wait for each other.  A buffer is reused once the store
     // issued two chunks earlier has finished reading it.
     const int q = warp & 3;
-    const uint32_t stg_base = staging + q * 4096;
-    uint16_t* stg_ptr = reinterpret_cast<uint16_t*>(staging_ptr + q * 4096);
+    const int eg = (warp - 2) >> 2;                        // 0: even chunks, 1: odd chunks of this lane quadrant
+    const uint32_t stg_base = staging + (warp - 2) * 4096;
+    uint16_t* stg_ptr = reinterpret_cast<uint16_t*>(staging_ptr + (warp - 2) * 4096);
     uint32_t tcount = 0, chunk = 0;
     for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++tcount) {
       int tile_m, tile_n;
@@ -530,30 +535,38 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
       ptx::tc_fence_after();
       const uint32_t acc = tmem_base + 256u * buf + ((uint32_t)(32 * q) << 16);
       const uint32_t release_bar = ptx::mapa(tmem_empty_bar(buf), 0);
+      // this warp's chunks: eg, eg + 2, ...; `last_c` is the one after which it has no more reads of the accumulator
+      const int nchunks = (CONV || (SP_N & 31) == 0) ? SP_N / 32 : SP_N / 16;
+      const int last_c = ((nchunks - 1 - eg) & ~1) + eg;   // largest c < nchunks with c % 2 == eg (negative: none)
+      if (last_c < 0) {                                    // nothing to drain: release at once
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive_cluster(release_bar);
+      }
       if (CONV) {
         // accumulator columns [0, SP_N/2) are the pixels of box 2*tile_n, the rest those of box 2*tile_n + 1;
         // a chunk of 32 tokens is 32 / wb consecutive rows of one image of the box
 #pragma unroll 1
-        for (int c = 0; c < SP_N / 32; ++c, ++chunk) {
+        for (int c = eg; c < nchunks; c += 2, ++chunk) {
           const int half = (32 * c) / (SP_N / 2);
           const int rr = 32 * c - half * (SP_N / 2);
           int cw0, ch0, cn0;
           conv_box_origin(p.conv, 2 * tile_n + half, cw0, ch0, cn0);
           const int h = ch0 + ((rr >> p.conv.lg_wb) & (p.conv.hb - 1));
           const int n = cn0 + (rr >> (p.conv.lg_wb + p.conv.lg_hb));
-          sparse_epilogue_chunk<32>(acc + 32 * c, c == SP_N / 32 - 1, release_bar, stg_ptr, stg_base, chunk, lane,
+          sparse_epilogue_chunk<32>(acc + 32 * c, c == last_c, release_bar, stg_ptr, stg_base, chunk, lane,
                                     &tmapOut32, m0, 0, p.Mdim, p.Ndim, cw0, h, n,
                                     cw0 < p.conv.W && h < p.conv.H && n < p.conv.NB);
         }
       } else if ((SP_N & 31) == 0) {
 #pragma unroll 1
-        for (int c = 0; c < SP_N / 32; ++c, ++chunk)
-          sparse_epilogue_chunk<32>(acc + 32 * c, c == SP_N / 32 - 1, release_bar, stg_ptr, stg_base, chunk, lane,
+        for (int c = eg; c < nchunks; c += 2, ++chunk)
+          sparse_epilogue_chunk<32>(acc + 32 * c, c == last_c, release_bar, stg_ptr, stg_base, chunk, lane,
                                     &tmapOut32, m0, n0 + 32 * c, p.Mdim, p.Ndim);
       } else {
 #pragma unroll 1
-        for (int c = 0; c < SP_N / 16; ++c, ++chunk)
-          sparse_epilogue_chunk<16>(acc + 16 * c, c == SP_N / 16 - 1, release_bar, stg_ptr, stg_base, chunk, lane,
+        for (int c = eg; c < nchunks; c += 2, ++chunk)
+          sparse_epilogue_chunk<16>(acc + 16 * c, c == last_c, release_bar, stg_ptr, stg_base, chunk, lane,
                                     &tmapOut16, m0, n0 + 16 * c, p.Mdim, p.Ndim);
       }
     }
@@ -1443,7 +1456,7 @@ int choose_sparse_n(int pair_tiles_m, int Ndim, int k_tiles, int clusters) {
 
 int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim,
                                int Kdim, uint16_t* out, int32_t* status_word, cudaStream_t s) {
-  constexpr int STAGES = 4;
+  constexpr int STAGES = 3;
   using C = PairPCfg<STAGES>;
   CUtensorMap ta, tb, te, to32, to16;
   int rc;
@@ -1471,7 +1484,7 @@ int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const 
   p.raster_group = 8;
   const int total = p.tiles_m * p.tiles_n;
   const int clusters = total < sms / 2 ? total : sms / 2;
-  kern<<<2 * clusters, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, to32, to16, p);
+  kern<<<2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, to32, to16, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -1595,7 +1608,7 @@ int run_conv_single(const uint16_t* vals, int a_rows, int a_kdim, const void* hw
 
 int run_conv_pair(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_meta, const uint16_t* tok, ConvGeom g,
                   int Mdim, int Kdim, int tiles_k_meta, uint16_t* out, int32_t* status_word, cudaStream_t s) {
-  constexpr int STAGES = 4;
+  constexpr int STAGES = 3;
   using C = PairPCfg<STAGES>;
   const int n_tile = 128;                                // two boxes of 64 pixels; two accumulators in tensor memory
   conv_boxes(g, n_tile / 2);
@@ -1624,7 +1637,7 @@ int run_conv_pair(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_m
   p.raster_group = 8;
   const int total = p.tiles_m * p.tiles_n;
   const int clusters = total < sms / 2 ? total : sms / 2;
-  kern<<<2 * clusters, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, to32, to32, p);
+  kern<<<2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, to32, to32, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
