@@ -25,6 +25,9 @@ namespace {
 
 constexpr long long WAIT_BUDGET = 4000000000ll;      // ~2 s of SM clocks
 constexpr int GEMM_THREADS = 192;                    // warp 0 TMA, warp 1 MMA, warps 2-5 epilogue
+// The sparse kernels that drain bf16 results use eight epilogue warps (two per tensor-memory lane quadrant, taking
+// alternate column chunks): products with a short reduction are bound by that drain, not by the tensor pipe.
+constexpr int PAIR_THREADS = 320;
 
 template <int N_TILE, int STAGES, bool SPARSE = true>
 struct Cfg {
@@ -37,7 +40,7 @@ struct Cfg {
   static constexpr int META_COLS = SPARSE ? 4 : 0;
   static constexpr int TMEM_COLS = (N_TILE + META_COLS) <= 128 ? 128 : (N_TILE + META_COLS) <= 256 ? 256 : 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */ +
-                                    16384 /* epilogue staging */;
+                                    32768 /* epilogue staging: eight warps x two 2 KB buffers */;
 };
 
 // A 3x3 convolution as an implicit GEMM: the token operand is an NHWC tensor and a "tile of
@@ -114,7 +117,7 @@ __device__ __forceinline__ void raster(int id, int tiles_m, int tiles_n, int gro
 // 2:4 format cannot hold): 128 x 128 A tile per stage as two 64-wide boxes, eight K = 16 MMAs.
 // CONV: the token operand is fetched as shifted pixel boxes (see ConvGeom); N_TILE tokens = one box.
 template <int N_TILE, int STAGES, bool SPARSE, bool CONV>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __launch_bounds__(PAIR_THREADS, 1)
 spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                    const __grid_constant__ CUtensorMap tmapOut, const GemmParams p) {
   using C = Cfg<N_TILE, STAGES, SPARSE>;
@@ -260,11 +263,13 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     if (num_kt > 0) ok = ptx::mbar_wait_bounded(tmem_full_bar, 0, abort_flag, WAIT_BUDGET);
     if (!ok) *abort_flag = 1;
     ptx::tc_fence_after();
-    const uint32_t stg_base = staging + q * 4096;       // two 2 KB buffers per warp
-    uint16_t* stg_ptr = reinterpret_cast<uint16_t*>(staging_ptr + q * 4096);
+    const int eg = (warp - 2) >> 2;                      // eight epilogue warps: two per lane quadrant, alternate chunks
+    const uint32_t stg_base = staging + (warp - 2) * 4096;       // two 2 KB buffers per warp
+    uint16_t* stg_ptr = reinterpret_cast<uint16_t*>(staging_ptr + (warp - 2) * 4096);
     if (ok) {
+      int nbuf = 0;                                      // this warp's chunk counter (staging buffer parity)
 #pragma unroll 1
-      for (int c = 0; c < N_TILE / 32; ++c) {
+      for (int c = eg; c < N_TILE / 32; c += 2, ++nbuf) {
         uint32_t r[32];
         if (num_kt > 0) {
           ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + 32 * c, r);
@@ -274,7 +279,7 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
           for (int j = 0; j < 32; ++j) r[j] = 0u;
         }
         // registers -> bf16 -> this warp's staging tile [token][row] -> one TMA store of a 32 x 32 box
-        uint16_t* sbuf = stg_ptr + (c & 1) * 1024;
+        uint16_t* sbuf = stg_ptr + (nbuf & 1) * 1024;
         if (lane == 0) ptx::tma_store_wait_read1();         // the store that last used this buffer has read it
         __syncwarp();
 #pragma unroll
@@ -288,7 +293,7 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
         __syncwarp();
         if (lane == 0) {
           const int mq = m0 + 32 * q;
-          const uint32_t src = stg_base + (uint32_t)(c & 1) * 2048u;
+          const uint32_t src = stg_base + (uint32_t)(nbuf & 1) * 2048u;
           if (CONV) {
             // tokens 32c .. 32c+31 of the box: 32 / wb consecutive image rows starting at (h, cw0) of image n
             const int rr = 32 * c;
@@ -377,10 +382,6 @@ struct PairPCfg {
   static constexpr int TMEM_COLS = 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 + 256;
 };
-
-// Eight epilogue warps (two per tensor-memory lane quadrant, taking alternate column chunks): products with
-// a short reduction are bound by the drain of the accumulator, not by the tensor pipe.
-constexpr int PAIR_THREADS = 320;
 
 template <int STAGES, bool CONV>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PAIR_THREADS, 1)
@@ -1430,7 +1431,7 @@ int run_single(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, i
   p.tiles_n = (Ndim + N_TILE - 1) / N_TILE;
   p.raster_group = 16;
   dim3 grid(p.tiles_m * p.tiles_n, 1, 1);
-  kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, to, p);
+  kern<<<grid, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, to, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -1551,7 +1552,7 @@ int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, 
     return run_sparse_pair2m(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   if (Ndim > 128 && Mdim > 128) return run_sparse_pair_persistent(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   if (Ndim > 128) return run_single<256, 2>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
-  return run_single<128, 4>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
+  return run_single<128, 3>(vals, hw_meta, Bop, Mdim, Ndim, Kdim, out, status_word, s);
 }
 
 namespace {
@@ -1600,7 +1601,7 @@ int run_conv_single(const uint16_t* vals, int a_rows, int a_kdim, const void* hw
   p.raster_group = 16;
   p.n_tile = N_TILE;
   dim3 grid(p.tiles_m * p.tiles_n, 1, 1);
-  kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, to, p);
+  kern<<<grid, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, to, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -1666,7 +1667,7 @@ int launch_spmm_conv(int mode, const uint16_t* vals, const void* hw_meta, const 
     return run_conv_pair(vals, a_rows, a_kdim, hw_meta, tok, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
   if (T > 128)
     return run_conv_single<256, 2>(vals, a_rows, a_kdim, hw_meta, tok, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
-  return run_conv_single<128, 4>(vals, a_rows, a_kdim, hw_meta, tok, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
+  return run_conv_single<128, 3>(vals, a_rows, a_kdim, hw_meta, tok, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
 }
 
 int launch_dense_nt(const uint16_t* A, const uint16_t* Bop, int Mdim, int Ndim, int Kdim, uint16_t* out,
