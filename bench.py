@@ -208,9 +208,9 @@ class ClockSampler:
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM kernels on
 # config 5, from the ncu launch list summarised in profiles/cfg5_launch_list.md (GEMM kernel only).
 NCU_TRAFFIC_BYTES = {
-    (5, 0, "wgrad"): 1.297e9 + 0.246e9, (5, 1, "wgrad"): 1.024e9 + 0.246e9,
-    (5, 0, "spmm_fwd"): 0.605e9 + 0.244e9, (5, 1, "spmm_fwd"): 0.878e9 + 0.062e9,
-    (5, 0, "spmm_dgrad"): 0.878e9 + 0.058e9, (5, 1, "spmm_dgrad"): 0.604e9 + 0.244e9,
+    (5, 0, "wgrad"): 1.245e9 + 0.245e9, (5, 1, "wgrad"): 1.012e9 + 0.245e9,
+    (5, 0, "spmm_fwd"): 0.613e9 + 0.242e9, (5, 1, "spmm_fwd"): 0.703e9 + 0.055e9,
+    (5, 0, "spmm_dgrad"): 0.703e9 + 0.051e9, (5, 1, "spmm_dgrad"): 0.616e9 + 0.243e9,
 }
 
 
