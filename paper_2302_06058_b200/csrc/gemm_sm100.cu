@@ -17,6 +17,7 @@
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 #include <cuda_bf16.h>
+#include <atomic>
 #include <mutex>
 
 namespace bimask {
@@ -1401,9 +1402,27 @@ int make_tmap_plain(CUtensorMap* m, int dtype, const void* ptr, uint64_t inner, 
 
 namespace {
 
+// The dynamic shared-memory limit of a kernel is set once per (device, kernel): the call costs a microsecond or two
+// on the host, which a layer step of ten short launches would notice.  A kernel is always launched with the same size.
 template <typename K>
 int set_smem_attr(K kernel, int bytes) {
+  constexpr int SLOTS = 64;
+  static std::atomic<const void*> done[16][SLOTS];       // [device][slot]; zero-initialised
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 16) dev = -1;
+  const void* key = reinterpret_cast<const void*>(kernel);
+  if (dev >= 0)
+    for (int i = 0; i < SLOTS; ++i) {
+      const void* seen = done[dev][i].load(std::memory_order_acquire);
+      if (seen == key) return BIMASK_OK;
+      if (seen == nullptr) break;
+    }
   BIMASK_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  if (dev >= 0)
+    for (int i = 0; i < SLOTS; ++i) {
+      const void* expect = nullptr;
+      if (done[dev][i].compare_exchange_strong(expect, key, std::memory_order_acq_rel) || expect == key) break;
+    }
   return BIMASK_OK;
 }
 
