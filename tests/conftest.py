@@ -24,3 +24,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_sessionstart(session):
+    """The shared library is a build artefact (not in version control): compile it when it is missing or older than
+    its sources, so that neither the CPU nor the GPU suite depends on an earlier build step."""
+    try:
+        from paper_2302_06058_b200 import build
+        build.build()
+    except Exception as exc:                                 # the tests that need the library will say so themselves
+        sys.stderr.write(f"[conftest] building libbimask.so failed: {exc}\n")
