@@ -26,9 +26,11 @@ namespace {
 
 constexpr long long WAIT_BUDGET = 4000000000ll;      // ~2 s of SM clocks
 constexpr int GEMM_THREADS = 192;                    // warp 0 TMA, warp 1 MMA, warps 2-5 epilogue
-// The sparse kernels that drain bf16 results use eight epilogue warps (two per tensor-memory lane quadrant, taking
-// alternate column chunks): products with a short reduction are bound by that drain, not by the tensor pipe.
-constexpr int PAIR_THREADS = 320;
+// The sparse kernels that drain bf16 results use eight epilogue warps (two groups of four, one warp per
+// tensor-memory lane quadrant, taking alternate column chunks): products with a short reduction are bound by
+// that drain, not by the tensor pipe.
+constexpr int EPI_WARPS = 8;
+constexpr int PAIR_THREADS = 64 + 32 * EPI_WARPS;
 
 template <int N_TILE, int STAGES, bool SPARSE = true>
 struct Cfg {
@@ -41,7 +43,7 @@ struct Cfg {
   static constexpr int META_COLS = SPARSE ? 4 : 0;
   static constexpr int TMEM_COLS = (N_TILE + META_COLS) <= 128 ? 128 : (N_TILE + META_COLS) <= 256 ? 256 : 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */ +
-                                    32768 /* epilogue staging: eight warps x two 2 KB buffers */;
+                                    EPI_WARPS * 2048 /* epilogue staging: one [32 tokens][128 rows] bf16 tile per group of four warps */;
 };
 
 // A 3x3 convolution as an implicit GEMM: the token operand is an NHWC tensor and a "tile of
@@ -114,26 +116,114 @@ __device__ __forceinline__ void raster(int id, int tiles_m, int tiles_n, int gro
   tn = in / gsize;
 }
 
+// Epilogue of the 2:4 products.  The accumulator holds D[row][token] (row = tensor-memory lane), the result is
+// stored token-major, so a chunk of W tokens x the CTA's 128 rows is transposed on its way out by a GROUP of four
+// warps, one per tensor-memory lane quadrant:
+//   tensor memory -> registers in the accumulator-fragment layout (two 16-lane loads per warp) -> bf16 pairs ->
+//   stmatrix.trans into the group's staging tile [token][128 rows] (256-byte rows; the 16-byte unit index is
+//   XOR-ed with the token index mod 8, so the eight rows of a matrix fall into eight different bank groups) ->
+//   named barrier -> each warp reads W/4 whole token rows back and writes them with 16-byte stores, 256 contiguous
+//   bytes per token (whole 128-byte lines: half-line writes were bound by the number of write requests).
+// The tensor-memory load of the next chunk is issued before the current one is converted and stored.
+template <int W>
+__device__ __forceinline__ void epi_load(uint32_t taddr, uint32_t (&r)[W], bool zero) {
+  if (zero) {
+#pragma unroll
+    for (int j = 0; j < W; ++j) r[j] = 0u;
+  } else if (W == 32) {
+    ptx::tmem_ld_16x256b_x4(taddr, &r[0]);                 // lanes 0-15 of the quadrant
+    ptx::tmem_ld_16x256b_x4(taddr + (16u << 16), &r[16]);  // lanes 16-31
+  } else {
+    ptx::tmem_ld_16x256b_x2(taddr, &r[0]);
+    ptx::tmem_ld_16x256b_x2(taddr + (16u << 16), &r[W / 2]);
+  }
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(uint32_t lo, uint32_t hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(lo), __uint_as_float(hi));
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// `dst`: this lane's row address for token group 0 (see drain_chunks); token group g is 2048 bytes further.
+template <int W>
+__device__ __forceinline__ void epi_stage(const uint32_t (&r)[W], uint32_t dst) {
+#pragma unroll
+  for (int g = 0; g < W / 8; ++g)
+    ptx::stmatrix_x4_trans(dst + 2048u * g, pack_bf16(r[4 * g], r[4 * g + 1]), pack_bf16(r[4 * g + 2], r[4 * g + 3]),
+                           pack_bf16(r[W / 2 + 4 * g], r[W / 2 + 4 * g + 1]),
+                           pack_bf16(r[W / 2 + 4 * g + 2], r[W / 2 + 4 * g + 3]));
+}
+
+// Drains chunks c0, c0 + cstep, ... (< nchunks) of one accumulator; called by the four warps of a group with the
+// same arguments except `acc` (the warp's lane quadrant q = warp % 4, column of chunk c: W * c).  After its last
+// tensor-memory read each warp arrives once on `release_bar` (0: nobody waits for the accumulator).
+// row_of(c, t) returns where token t of chunk c starts in the result (the CTA's first row), or nullptr when that
+// token lies outside; rows_valid = how many of the CTA's 128 rows exist (a multiple of 32).
+// `stg`: the group's staging tile (W * 256 bytes, 1 KB aligned); `bar_id`: its named barrier.
+template <int W, typename RowOf>
+__device__ __forceinline__ void drain_chunks(uint32_t acc, int c0, int cstep, int nchunks, bool zero, uint32_t release_bar,
+                                             uint32_t stg, uint32_t bar_id, int q, int lane, int rows_valid, RowOf&& row_of) {
+  auto release = [&]() {
+    if (release_bar != 0u) {
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive_cluster(release_bar);
+    }
+  };
+  if (c0 >= nchunks) { release(); return; }
+  // stmatrix: lane 8 i + k addresses token k (of a group of eight) of matrix i = rows 32 q + 8 i .. + 7, i.e. unit
+  // 4 q + i of the token's 256-byte row
+  const uint32_t dst = stg + (uint32_t)(lane & 7) * 256u + ((((uint32_t)(4 * q) + ((uint32_t)lane >> 3)) ^ ((uint32_t)lane & 7u)) << 4);
+  // reading back: this warp owns tokens (W/4) q .. (W/4) q + W/4 - 1; per step lanes 0-15 take one token, lanes 16-31
+  // the next, 16 bytes (eight rows) per lane
+  const int unit = lane & 15;
+  const bool unit_ok = 8 * unit < rows_valid;
+  auto emit = [&](const uint32_t (&r)[W], int c) {
+    ptx::named_bar_sync(bar_id, 128);                     // the group has read the previous chunk out of the tile
+    epi_stage<W>(r, dst);
+    ptx::named_bar_sync(bar_id, 128);
+#pragma unroll
+    for (int i = 0; i < W / 8; ++i) {
+      const int t = (W / 4) * q + 2 * i + (lane >> 4);
+      const uint4 v = ptx::ld_shared_v4(stg + (uint32_t)t * 256u + (((uint32_t)unit ^ ((uint32_t)t & 7u)) << 4));
+      uint16_t* row = row_of(c, t);
+      if (row != nullptr && unit_ok) *reinterpret_cast<uint4*>(row + 8 * unit) = v;
+    }
+  };
+  uint32_t ra[W], rb[W];
+  epi_load<W>(acc + W * c0, ra, zero);
+#pragma unroll 1
+  for (int c = c0; c < nchunks; c += 2 * cstep) {
+    if (!zero) ptx::tmem_ld_wait();
+    const bool more1 = c + cstep < nchunks;
+    if (more1) epi_load<W>(acc + W * (c + cstep), rb, zero); else release();
+    emit(ra, c);
+    if (!more1) break;
+    if (!zero) ptx::tmem_ld_wait();
+    if (c + 2 * cstep < nchunks) epi_load<W>(acc + W * (c + 2 * cstep), ra, zero); else release();
+    emit(rb, c + cstep);
+  }
+}
+
 // SPARSE = false: the same pipeline on a dense bf16 A operand (masked weights of a pattern the
 // 2:4 format cannot hold): 128 x 128 A tile per stage as two 64-wide boxes, eight K = 16 MMAs.
 // CONV: the token operand is fetched as shifted pixel boxes (see ConvGeom); N_TILE tokens = one box.
 template <int N_TILE, int STAGES, bool SPARSE, bool CONV>
 __global__ void __launch_bounds__(PAIR_THREADS, 1)
 spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-                   const __grid_constant__ CUtensorMap tmapOut, const GemmParams p) {
+                   const GemmParams p) {
   using C = Cfg<N_TILE, STAGES, SPARSE>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - raw);
-  const uint32_t bar_base = base + STAGES * C::STAGE_BYTES;
+  const uint32_t staging = base + STAGES * C::STAGE_BYTES;      // epilogue staging, 8 KB per group of four warps
+  const uint32_t bar_base = staging + EPI_WARPS * 2048;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   const uint32_t tmem_full_bar = bar_base + 8u * (2 * STAGES);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * C::STAGE_BYTES + 8 * (2 * STAGES + 1));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * C::STAGE_BYTES + EPI_WARPS * 2048 + 8 * (2 * STAGES + 1));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  const uint32_t staging = bar_base + 256;             // epilogue staging, 4 KB per epilogue warp
-  uint8_t* staging_ptr = base_ptr + STAGES * C::STAGE_BYTES + 256;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int tile_m, tile_n;
@@ -157,7 +247,6 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmapA);
     ptx::prefetch_tmap(&tmapB);
-    ptx::prefetch_tmap(&tmapOut);
   }
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
@@ -264,50 +353,24 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     if (num_kt > 0) ok = ptx::mbar_wait_bounded(tmem_full_bar, 0, abort_flag, WAIT_BUDGET);
     if (!ok) *abort_flag = 1;
     ptx::tc_fence_after();
-    const int eg = (warp - 2) >> 2;                      // eight epilogue warps: two per lane quadrant, alternate chunks
-    const uint32_t stg_base = staging + (warp - 2) * 4096;       // two 2 KB buffers per warp
-    uint16_t* stg_ptr = reinterpret_cast<uint16_t*>(staging_ptr + (warp - 2) * 4096);
+    const int eg = (warp - 2) >> 2;                      // EPI_WARPS / 4 groups of four warps take chunks in turn
+    ok = ptx::named_bar_and(1 + eg, 128, ok);            // the four warps of a group go on or give up together
     if (ok) {
-      int nbuf = 0;                                      // this warp's chunk counter (staging buffer parity)
-#pragma unroll 1
-      for (int c = eg; c < N_TILE / 32; c += 2, ++nbuf) {
-        uint32_t r[32];
-        if (num_kt > 0) {
-          ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + 32 * c, r);
-          ptx::tmem_ld_wait();
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) r[j] = 0u;
+      uint16_t* outp = reinterpret_cast<uint16_t*>(p.out);
+      drain_chunks<32>(tmem_base + ((uint32_t)(32 * q) << 16), eg, EPI_WARPS / 4, N_TILE / 32, num_kt <= 0, 0u,
+                       staging + eg * 8192, 1 + eg, q, lane, p.Mdim - m0, [&](int c, int t) -> uint16_t* {
+        if (CONV) {
+          // token 32c + t of the box: pixel (cw0 + ., ch0 + .) of image cn0 + .
+          const int rr = 32 * c + t;
+          const int w = cw0 + (rr & (p.conv.wb - 1));
+          const int h = ch0 + ((rr >> p.conv.lg_wb) & (p.conv.hb - 1));
+          const int n = cn0 + (rr >> (p.conv.lg_wb + p.conv.lg_hb));
+          if (w >= p.conv.W || h >= p.conv.H || n >= p.conv.NB) return nullptr;
+          return outp + ((size_t)(n * p.conv.H + h) * p.conv.W + w) * p.Mdim + m0;
         }
-        // registers -> bf16 -> this warp's staging tile [token][row] -> one TMA store of a 32 x 32 box
-        uint16_t* sbuf = stg_ptr + (nbuf & 1) * 1024;
-        if (lane == 0) ptx::tma_store_wait_read1();         // the store that last used this buffer has read it
-        __syncwarp();
-#pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-          const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
-          const uint32_t u = *reinterpret_cast<const uint32_t*>(&v);
-          sbuf[j * 32 + lane] = (uint16_t)(u & 0xFFFFu);
-          sbuf[(j + 1) * 32 + lane] = (uint16_t)(u >> 16);
-        }
-        ptx::fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) {
-          const int mq = m0 + 32 * q;
-          const uint32_t src = stg_base + (uint32_t)(nbuf & 1) * 2048u;
-          if (CONV) {
-            // tokens 32c .. 32c+31 of the box: 32 / wb consecutive image rows starting at (h, cw0) of image n
-            const int rr = 32 * c;
-            const int h = ch0 + ((rr >> p.conv.lg_wb) & (p.conv.hb - 1));
-            const int n = cn0 + (rr >> (p.conv.lg_wb + p.conv.lg_hb));
-            if (mq < p.Mdim && cw0 < p.conv.W && h < p.conv.H && n < p.conv.NB) ptx::tma_store_4d(&tmapOut, mq, cw0, h, n, src);
-          } else if (mq < p.Mdim && n0 + 32 * c < p.Ndim) {
-            ptx::tma_store_2d(&tmapOut, mq, n0 + 32 * c, src);
-          }
-          ptx::tma_store_commit();
-        }
-      }
-      if (lane == 0) ptx::tma_store_wait_all();
+        const int n = n0 + 32 * c + t;
+        return n < p.Ndim ? outp + (size_t)n * p.Mdim + m0 : nullptr;
+      });
     }
   }
 
@@ -327,51 +390,10 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
 // four metadata columns (496..499), so the epilogue of one tile overlaps the main loop of the
 // next; N = 256 leaves room for one accumulator only (metadata at 256..259) and is used when the
 // tile count would otherwise round up to an extra pass over the SMs (the host picks N).  The TMA
-// producer runs ahead across tile boundaries; the four epilogue warps drain an accumulator 16
-// columns at a time: tensor memory -> registers -> bf16 -> a transposed per-warp staging tile ->
-// one TMA store per chunk (ragged edges are clipped).
+// producer runs ahead across tile boundaries; two groups of four epilogue warps drain an accumulator
+// in chunks of 32 (16) columns, taking chunks in turn (see drain_chunks).
 // ------------------------------------------------------------------------------------------
 
-
-// One epilogue chunk of the 2:4 product for one warp: W accumulator columns of its 32 rows go
-// tensor memory -> registers -> bf16 -> staging[token][row] -> one TMA store of a 32 x W box.
-// `last` releases the accumulator (after its final read) to the MMA thread of the pair's leader.
-// cw >= 0: convolution output, the W tokens are pixels (cw.., ch..) of image cn (a 4-D store).
-template <int W>
-__device__ __forceinline__ void sparse_epilogue_chunk(uint32_t taddr, bool last, uint32_t release_bar,
-                                                      uint16_t* stg_ptr, uint32_t stg_base, uint32_t chunk, int lane,
-                                                      const CUtensorMap* tmap, int m0, int n, int Mdim, int Ndim,
-                                                      int cw = -1, int ch = 0, int cn = 0, bool cvalid = false) {
-  uint32_t r[W];
-  if (W == 32) ptx::tmem_ld_32x32(taddr, reinterpret_cast<uint32_t (&)[32]>(r));
-  else ptx::tmem_ld_32x16(taddr, reinterpret_cast<uint32_t (&)[16]>(r));
-  ptx::tmem_ld_wait();
-  if (last) {
-    ptx::tc_fence_before();
-    __syncwarp();
-    if (lane == 0) ptx::mbar_arrive_cluster(release_bar);
-  }
-  uint16_t* sbuf = stg_ptr + (chunk & 1u) * 1024;        // two 2 KB buffers per warp
-  if (lane == 0) ptx::tma_store_wait_read1();             // the store that last used this buffer is done
-  __syncwarp();
-#pragma unroll
-  for (int j = 0; j < W; j += 2) {
-    const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
-    const uint32_t u = *reinterpret_cast<const uint32_t*>(&v);
-    sbuf[j * 32 + lane] = (uint16_t)(u & 0xFFFFu);
-    sbuf[(j + 1) * 32 + lane] = (uint16_t)(u >> 16);
-  }
-  ptx::fence_proxy_async();
-  __syncwarp();
-  if (lane == 0) {
-    if (cw >= 0) {
-      if (m0 < Mdim && cvalid) ptx::tma_store_4d(tmap, m0, cw, ch, cn, stg_base + (chunk & 1u) * 2048);
-    } else if (m0 < Mdim && n < Ndim) {
-      ptx::tma_store_2d(tmap, m0, n, stg_base + (chunk & 1u) * 2048);
-    }
-    ptx::tma_store_commit();
-  }
-}
 
 template <int STAGES>
 struct PairPCfg {
@@ -379,7 +401,7 @@ struct PairPCfg {
   static constexpr int B_MAX = 32768;                      // up to 128 rows x 128 bf16 (two 64-wide boxes)
   static constexpr int E_BYTES = 2048;
   static constexpr int STAGE_BYTES = A_BYTES + B_MAX + E_BYTES;        // 50 KB (the B part is N / 2 rows)
-  static constexpr int STAGING_BYTES = 8 * 2 * 2048;       // per epilogue warp: two [<= 32 tokens][32 rows] bf16 buffers
+  static constexpr int STAGING_BYTES = EPI_WARPS * 2048;   // per group of four epilogue warps: one [32 tokens][128 rows] bf16 tile
   static constexpr int TMEM_COLS = 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 + 256;
 };
@@ -387,8 +409,7 @@ struct PairPCfg {
 template <int STAGES, bool CONV>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PAIR_THREADS, 1)
 spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-                            const __grid_constant__ CUtensorMap tmapE, const __grid_constant__ CUtensorMap tmapOut32,
-                            const __grid_constant__ CUtensorMap tmapOut16, const GemmParams p) {
+                            const __grid_constant__ CUtensorMap tmapE, const GemmParams p) {
   using C = PairPCfg<STAGES>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -422,14 +443,12 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(tmem_full_bar(b), 1);
-      ptx::mbar_init(tmem_empty_bar(b), 16);              // eight epilogue warps in each CTA of the pair
+      ptx::mbar_init(tmem_empty_bar(b), 2 * EPI_WARPS);   // the epilogue warps of both CTAs of the pair
     }
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmapA);
     ptx::prefetch_tmap(&tmapB);
     ptx::prefetch_tmap(&tmapE);
-    ptx::prefetch_tmap(&tmapOut32);
-    ptx::prefetch_tmap(&tmapOut16);
   }
   if (warp == 1) {
     ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
@@ -520,59 +539,53 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
       }
     }
   } else {
-    // Each epilogue warp owns 32 accumulator rows (its TMEM lane quadrant) and a private pair of
-    // 2 KB staging buffers; warps never wait for each other.  A buffer is reused once the store
-    // issued two chunks earlier has finished reading it.
+    // Each epilogue warp reads 32 accumulator rows (its TMEM lane quadrant); the four warps of a group share
+    // one staging tile.
     const int q = warp & 3;
-    const int eg = (warp - 2) >> 2;                        // 0: even chunks, 1: odd chunks of this lane quadrant
-    const uint32_t stg_base = staging + (warp - 2) * 4096;
-    uint16_t* stg_ptr = reinterpret_cast<uint16_t*>(staging_ptr + (warp - 2) * 4096);
-    uint32_t tcount = 0, chunk = 0;
+    const int eg = (warp - 2) >> 2;                        // EPI_WARPS / 4 groups of four warps take chunks in turn
+    const uint32_t stg = staging + eg * 8192;
+    uint16_t* outp = reinterpret_cast<uint16_t*>(p.out);
+    uint32_t tcount = 0;
     for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++tcount) {
       int tile_m, tile_n;
       raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
-      const int m0 = (2 * tile_m + (int)rank) * 128 + 32 * q, n0 = tile_n * SP_N;
+      const int m0 = (2 * tile_m + (int)rank) * 128, n0 = tile_n * SP_N;
       const uint32_t buf = tcount % nbuf;
-      if (!ptx::mbar_wait_bounded(tmem_full_bar(buf), (tcount / nbuf) & 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
+      bool ok = ptx::mbar_wait_bounded(tmem_full_bar(buf), (tcount / nbuf) & 1u, abort_flag, WAIT_BUDGET);
+      ok = ptx::named_bar_and(1 + eg, 128, ok);            // the four warps of a group go on or give up together
+      if (!ok) { *abort_flag = 1; break; }
       ptx::tc_fence_after();
       const uint32_t acc = tmem_base + 256u * buf + ((uint32_t)(32 * q) << 16);
       const uint32_t release_bar = ptx::mapa(tmem_empty_bar(buf), 0);
-      // this warp's chunks: eg, eg + 2, ...; `last_c` is the one after which it has no more reads of the accumulator
       const int nchunks = (CONV || (SP_N & 31) == 0) ? SP_N / 32 : SP_N / 16;
-      const int last_c = ((nchunks - 1 - eg) & ~1) + eg;   // largest c < nchunks with c % 2 == eg (negative: none)
-      if (last_c < 0) {                                    // nothing to drain: release at once
-        ptx::tc_fence_before();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive_cluster(release_bar);
-      }
       if (CONV) {
-        // accumulator columns [0, SP_N/2) are the pixels of box 2*tile_n, the rest those of box 2*tile_n + 1;
-        // a chunk of 32 tokens is 32 / wb consecutive rows of one image of the box
-#pragma unroll 1
-        for (int c = eg; c < nchunks; c += 2, ++chunk) {
+        // accumulator columns [0, SP_N/2) are the pixels of box 2*tile_n, the rest those of box 2*tile_n + 1
+        drain_chunks<32>(acc, eg, EPI_WARPS / 4, nchunks, false, release_bar, stg, 1 + eg, q, lane, p.Mdim - m0,
+                         [&](int c, int t) -> uint16_t* {
           const int half = (32 * c) / (SP_N / 2);
-          const int rr = 32 * c - half * (SP_N / 2);
+          const int rr = 32 * c - half * (SP_N / 2) + t;
           int cw0, ch0, cn0;
           conv_box_origin(p.conv, 2 * tile_n + half, cw0, ch0, cn0);
+          const int w = cw0 + (rr & (p.conv.wb - 1));
           const int h = ch0 + ((rr >> p.conv.lg_wb) & (p.conv.hb - 1));
           const int n = cn0 + (rr >> (p.conv.lg_wb + p.conv.lg_hb));
-          sparse_epilogue_chunk<32>(acc + 32 * c, c == last_c, release_bar, stg_ptr, stg_base, chunk, lane,
-                                    &tmapOut32, m0, 0, p.Mdim, p.Ndim, cw0, h, n,
-                                    cw0 < p.conv.W && h < p.conv.H && n < p.conv.NB);
-        }
+          if (w >= p.conv.W || h >= p.conv.H || n >= p.conv.NB) return nullptr;
+          return outp + ((size_t)(n * p.conv.H + h) * p.conv.W + w) * p.Mdim + m0;
+        });
       } else if ((SP_N & 31) == 0) {
-#pragma unroll 1
-        for (int c = eg; c < nchunks; c += 2, ++chunk)
-          sparse_epilogue_chunk<32>(acc + 32 * c, c == last_c, release_bar, stg_ptr, stg_base, chunk, lane,
-                                    &tmapOut32, m0, n0 + 32 * c, p.Mdim, p.Ndim);
+        drain_chunks<32>(acc, eg, EPI_WARPS / 4, nchunks, false, release_bar, stg, 1 + eg, q, lane, p.Mdim - m0,
+                         [&](int c, int t) -> uint16_t* {
+          const int n = n0 + 32 * c + t;
+          return n < p.Ndim ? outp + (size_t)n * p.Mdim + m0 : nullptr;
+        });
       } else {
-#pragma unroll 1
-        for (int c = eg; c < nchunks; c += 2, ++chunk)
-          sparse_epilogue_chunk<16>(acc + 16 * c, c == last_c, release_bar, stg_ptr, stg_base, chunk, lane,
-                                    &tmapOut16, m0, n0 + 16 * c, p.Mdim, p.Ndim);
+        drain_chunks<16>(acc, eg, EPI_WARPS / 4, nchunks, false, release_bar, stg, 1 + eg, q, lane, p.Mdim - m0,
+                         [&](int c, int t) -> uint16_t* {
+          const int n = n0 + 16 * c + t;
+          return n < p.Ndim ? outp + (size_t)n * p.Mdim + m0 : nullptr;
+        });
       }
     }
-    if (lane == 0) ptx::tma_store_wait_all();
   }
 
   ptx::tc_fence_before();
@@ -593,11 +606,11 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
 // owns 512 x N outputs: TWO 256-row MMA tiles that share the activation tile in shared memory, so
 // a stage carries 2 x 16 KB + <= 28 KB + 2 x 2 KB for twice the tensor-pipe work (a third fewer
 // bytes per clock).  Both accumulators (tensor-memory columns 0.. and 256.., N <= 224) belong to
-// the same token tile, so the epilogue cannot overlap the next main loop; instead eight epilogue
-// warps per CTA drain the two accumulators side by side.  Metadata: columns 496..499 and 500..503.
+// the same token tile, so the epilogue cannot overlap the next main loop; instead two groups of four
+// epilogue warps per CTA drain the two accumulators side by side.  Metadata: columns 496..499 and 500..503.
 // Roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 accumulator 0, warps 6-9 accumulator 1.
 // ------------------------------------------------------------------------------------------
-constexpr int GEMM2M_THREADS = 320;
+constexpr int GEMM2M_THREADS = PAIR_THREADS;
 
 template <int STAGES>
 struct Pair2MCfg {
@@ -605,7 +618,7 @@ struct Pair2MCfg {
   static constexpr int B_MAX = 28672;                      // 112 rows x 128 bf16 (two 64-wide boxes), N <= 224
   static constexpr int E_BYTES = 2048;
   static constexpr int STAGE_BYTES = 2 * A_BYTES + B_MAX + 2 * E_BYTES;      // 64 KB
-  static constexpr int STAGING_BYTES = 8 * 2 * 2048;       // per epilogue warp: two [32 tokens][32 rows] bf16 buffers
+  static constexpr int STAGING_BYTES = EPI_WARPS * 2048;   // per group of four epilogue warps: one [32 tokens][128 rows] bf16 tile
   static constexpr int TMEM_COLS = 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 + 256;
 };
@@ -613,7 +626,7 @@ struct Pair2MCfg {
 template <int STAGES>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2M_THREADS, 1)
 spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-                   const __grid_constant__ CUtensorMap tmapE, const __grid_constant__ CUtensorMap tmapOut32,
+                   const __grid_constant__ CUtensorMap tmapE,
                    const GemmParams p) {
   using C = Pair2MCfg<STAGES>;
   extern __shared__ uint8_t smem_raw[];
@@ -646,12 +659,11 @@ spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
       ptx::mbar_init(empty_bar(s), 1);
     }
     ptx::mbar_init(tmem_full_bar, 1);
-    ptx::mbar_init(tmem_empty_bar, 16);                   // eight epilogue warps in each CTA of the pair
+    ptx::mbar_init(tmem_empty_bar, 2 * EPI_WARPS);        // the epilogue warps of both CTAs of the pair
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmapA);
     ptx::prefetch_tmap(&tmapB);
     ptx::prefetch_tmap(&tmapE);
-    ptx::prefetch_tmap(&tmapOut32);
   }
   if (warp == 1) {
     ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
@@ -731,50 +743,28 @@ spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     }
   } else {
     // warps 2-5 drain accumulator 0 (row tile 0), warps 6-9 accumulator 1; a warp reads its own
-    // tensor-memory lane quadrant and owns two 1 KB staging buffers
+    // tensor-memory lane quadrant, a group shares one staging tile
     const int q = warp & 3;
-    const int mt = warp >= 6 ? 1 : 0;
-    const int ew = warp - 2;                               // 0..7
-    const uint32_t stg_base = staging + ew * 4096;
-    uint16_t* stg_ptr = reinterpret_cast<uint16_t*>(staging_ptr + ew * 4096);
+    const int mt = (warp - 2) >> 2;                        // the group of four warps that drains accumulator mt
+    const uint32_t stg = staging + mt * 8192;
+    uint16_t* outp = reinterpret_cast<uint16_t*>(p.out);
     const uint32_t release_bar = ptx::mapa(tmem_empty_bar, 0);
-    uint32_t tcount = 0, chunk = 0;
+    uint32_t tcount = 0;
     for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++tcount) {
       int tile_m, tile_n;
       raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
-      const int m0 = mt128_of(tile_m, mt) * 128 + 32 * q, n0 = tile_n * SP_N;
-      if (!ptx::mbar_wait_bounded(tmem_full_bar, tcount & 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
+      const int m0 = mt128_of(tile_m, mt) * 128, n0 = tile_n * SP_N;
+      bool ok = ptx::mbar_wait_bounded(tmem_full_bar, tcount & 1u, abort_flag, WAIT_BUDGET);
+      ok = ptx::named_bar_and(1 + mt, 128, ok);            // the four warps of a group go on or give up together
+      if (!ok) { *abort_flag = 1; break; }
       ptx::tc_fence_after();
       const uint32_t acc = tmem_base + 256u * mt + ((uint32_t)(32 * q) << 16);
-#pragma unroll 1
-      for (int c = 0; c < SP_N / 32; ++c, ++chunk) {
-        uint32_t r[32];
-        ptx::tmem_ld_32x32(acc + 32 * c, r);
-        ptx::tmem_ld_wait();
-        if (c == SP_N / 32 - 1) {                          // last read of this accumulator quadrant: release it
-          ptx::tc_fence_before();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive_cluster(release_bar);
-        }
-        uint16_t* sbuf = stg_ptr + (chunk & 1u) * 1024;    // two 2 KB buffers
-        if (lane == 0) ptx::tma_store_wait_read1();
-        __syncwarp();
-#pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-          const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
-          const uint32_t u = *reinterpret_cast<const uint32_t*>(&v);
-          sbuf[j * 32 + lane] = (uint16_t)(u & 0xFFFFu);
-          sbuf[(j + 1) * 32 + lane] = (uint16_t)(u >> 16);
-        }
-        ptx::fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) {
-          if (m0 < p.Mdim && n0 + 32 * c < p.Ndim) ptx::tma_store_2d(&tmapOut32, m0, n0 + 32 * c, stg_base + (chunk & 1u) * 2048);
-          ptx::tma_store_commit();
-        }
-      }
+      drain_chunks<32>(acc, 0, 1, SP_N / 32, false, release_bar, stg, 1 + mt, q, lane, p.Mdim - m0,
+                       [&](int c, int t) -> uint16_t* {
+        const int n = n0 + 32 * c + t;
+        return n < p.Ndim ? outp + (size_t)n * p.Mdim + m0 : nullptr;
+      });
     }
-    if (lane == 0) ptx::tma_store_wait_all();
   }
 
   ptx::tc_fence_before();
@@ -1369,25 +1359,11 @@ int make_tmap_meta(CUtensorMap* m, const void* ptr, uint64_t blocks) {
                                   (int)CU_TENSOR_MAP_SWIZZLE_NONE});
 }
 
-// bf16 tensor map for TMA stores of 32 x box_rows boxes into [rows][inner], no swizzle.
-int make_tmap_out(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t rows, uint32_t box_rows) {
-  return encode_cached(m, TmapKey{ptr, inner, rows, inner * 2, 32, box_rows, (int)CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
-                                  (int)CU_TENSOR_MAP_SWIZZLE_NONE});
-}
-
 // 4-D bf16 map of an NHWC tensor (channels, W, H, NB) for loads of 64-channel pixel boxes, 128-byte swizzle.
 int make_tmap_nhwc_load(CUtensorMap* m, const void* ptr, int CH, int W, int H, int NB, int wb, int hb, int nb) {
   TmapKey k{ptr, (uint64_t)CH, (uint64_t)W, (uint64_t)CH * 2, 64, (uint32_t)wb, (int)CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
             (int)CU_TENSOR_MAP_SWIZZLE_128B};
   k.d2 = (uint64_t)H; k.d3 = (uint64_t)NB; k.box2 = (uint32_t)hb; k.box3 = (uint32_t)nb;
-  return encode_cached(m, k);
-}
-
-// The same tensor for stores of (32 channels, wb, 32 / wb, 1) boxes, no swizzle.
-int make_tmap_nhwc_store(CUtensorMap* m, const void* ptr, int CH, int W, int H, int NB, int wb) {
-  TmapKey k{ptr, (uint64_t)CH, (uint64_t)W, (uint64_t)CH * 2, 32, (uint32_t)wb, (int)CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
-            (int)CU_TENSOR_MAP_SWIZZLE_NONE};
-  k.d2 = (uint64_t)H; k.d3 = (uint64_t)NB; k.box2 = (uint32_t)(32 / wb); k.box3 = 1;
   return encode_cached(m, k);
 }
 
@@ -1434,8 +1410,6 @@ int run_single(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, i
   int rc;
   if ((rc = make_tmap(&ta, vals, SPARSE ? (uint64_t)Kdim / 2 : (uint64_t)Kdim, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, N_TILE)) != BIMASK_OK) return rc;
-  CUtensorMap to;
-  if ((rc = make_tmap_out(&to, out, (uint64_t)Mdim, (uint64_t)Ndim, 32)) != BIMASK_OK) return rc;
   auto kern = spmm_single_kernel<N_TILE, STAGES, SPARSE, false>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
@@ -1450,7 +1424,7 @@ int run_single(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, i
   p.tiles_n = (Ndim + N_TILE - 1) / N_TILE;
   p.raster_group = 16;
   dim3 grid(p.tiles_m * p.tiles_n, 1, 1);
-  kern<<<grid, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, to, p);
+  kern<<<grid, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -1481,7 +1455,7 @@ int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const 
                                int Kdim, uint16_t* out, int32_t* status_word, cudaStream_t s) {
   constexpr int STAGES = 3;
   using C = PairPCfg<STAGES>;
-  CUtensorMap ta, tb, te, to32, to16;
+  CUtensorMap ta, tb, te;
   int rc;
   const int tiles_m = (Mdim + 127) / 128, tiles_k = (Kdim + 127) / 128;
   const int sms = sm_count();
@@ -1489,8 +1463,6 @@ int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const 
   if ((rc = make_tmap(&ta, vals, (uint64_t)Kdim / 2, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, n_tile / 2)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_meta(&te, hw_meta, (uint64_t)tiles_m * tiles_k)) != BIMASK_OK) return rc;
-  if ((rc = make_tmap_out(&to32, out, (uint64_t)Mdim, (uint64_t)Ndim, 32)) != BIMASK_OK) return rc;
-  if ((rc = make_tmap_out(&to16, out, (uint64_t)Mdim, (uint64_t)Ndim, 16)) != BIMASK_OK) return rc;
   auto kern = spmm_pair_persistent_kernel<STAGES, false>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
@@ -1507,7 +1479,7 @@ int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const 
   p.raster_group = 8;
   const int total = p.tiles_m * p.tiles_n;
   const int clusters = total < sms / 2 ? total : sms / 2;
-  kern<<<2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, to32, to16, p);
+  kern<<<2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -1531,7 +1503,7 @@ int run_sparse_pair2m(const uint16_t* vals, const void* hw_meta, const uint16_t*
                       uint16_t* out, int32_t* status_word, cudaStream_t s) {
   constexpr int STAGES = 3;
   using C = Pair2MCfg<STAGES>;
-  CUtensorMap ta, tb, te, to32;
+  CUtensorMap ta, tb, te;
   int rc;
   const int tiles_m = (Mdim + 127) / 128, tiles_k = (Kdim + 127) / 128;
   const int sms = sm_count();
@@ -1540,7 +1512,6 @@ int run_sparse_pair2m(const uint16_t* vals, const void* hw_meta, const uint16_t*
   if ((rc = make_tmap(&ta, vals, (uint64_t)Kdim / 2, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, n_tile / 2)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_meta(&te, hw_meta, (uint64_t)tiles_m * tiles_k)) != BIMASK_OK) return rc;
-  if ((rc = make_tmap_out(&to32, out, (uint64_t)Mdim, (uint64_t)Ndim, 32)) != BIMASK_OK) return rc;
   auto kern = spmm_pair2m_kernel<STAGES>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
@@ -1557,7 +1528,7 @@ int run_sparse_pair2m(const uint16_t* vals, const void* hw_meta, const uint16_t*
   p.raster_group = 4;
   const int total = p.tiles_m * p.tiles_n;
   const int clusters = total < sms / 2 ? total : sms / 2;
-  kern<<<2 * clusters, GEMM2M_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, to32, p);
+  kern<<<2 * clusters, GEMM2M_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -1606,8 +1577,6 @@ int run_conv_single(const uint16_t* vals, int a_rows, int a_kdim, const void* hw
   int rc;
   if ((rc = make_tmap(&ta, vals, (uint64_t)a_kdim / 2, (uint64_t)a_rows, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_nhwc_load(&tb, tok, g.CB, g.W, g.H, g.NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
-  CUtensorMap to;
-  if ((rc = make_tmap_nhwc_store(&to, out, Mdim, g.W, g.H, g.NB, g.wb)) != BIMASK_OK) return rc;
   auto kern = spmm_single_kernel<N_TILE, STAGES, true, true>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
@@ -1623,7 +1592,7 @@ int run_conv_single(const uint16_t* vals, int a_rows, int a_kdim, const void* hw
   p.raster_group = 16;
   p.n_tile = N_TILE;
   dim3 grid(p.tiles_m * p.tiles_n, 1, 1);
-  kern<<<grid, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, to, p);
+  kern<<<grid, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -1635,14 +1604,13 @@ int run_conv_pair(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_m
   using C = PairPCfg<STAGES>;
   const int n_tile = 128;                                // two boxes of 64 pixels; two accumulators in tensor memory
   conv_boxes(g, n_tile / 2);
-  CUtensorMap ta, tb, te, to32;
+  CUtensorMap ta, tb, te;
   int rc;
   const int a_tiles_m = (a_rows + 127) / 128;
   const int sms = sm_count();
   if ((rc = make_tmap(&ta, vals, (uint64_t)a_kdim / 2, (uint64_t)a_rows, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_nhwc_load(&tb, tok, g.CB, g.W, g.H, g.NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_meta(&te, hw_meta, (uint64_t)a_tiles_m * tiles_k_meta)) != BIMASK_OK) return rc;
-  if ((rc = make_tmap_nhwc_store(&to32, out, Mdim, g.W, g.H, g.NB, g.wb)) != BIMASK_OK) return rc;
   auto kern = spmm_pair_persistent_kernel<STAGES, true>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
@@ -1660,7 +1628,7 @@ int run_conv_pair(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_m
   p.raster_group = 8;
   const int total = p.tiles_m * p.tiles_n;
   const int clusters = total < sms / 2 ? total : sms / 2;
-  kern<<<2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, to32, to32, p);
+  kern<<<2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, p);
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
