@@ -1121,7 +1121,7 @@ wgrad_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_cons
         if (c == 7) {                                      // accumulator drained: release it
           ptx::tc_fence_before();
           __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(tmem_empty_bar(buf));
+          if (lane == 0) ptx::mbar_arrive_relaxed(tmem_empty_bar(buf));
         }
         const int nb = n0 + 32 * c;
         if (m < p.Mdim && nb < p.Ndim) {                  // Ndim % 32 == 0: a chunk is all in or all out
@@ -1260,7 +1260,8 @@ __global__ void wait_probe_kernel(long long budget_cycles, int32_t* __restrict__
   }
 }
 
-// Sum of split-K partials: out[e] = sum_s part[s][e].
+// Sum of split-K partials: out[e] = sum_s part[s][e], one thread per float4 -- for outputs large enough to fill
+// the GPU that way.
 __global__ void splitk_reduce_kernel(const float4* __restrict__ part, int splits, long long n4,
                                      float4* __restrict__ out) {
   for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < n4; e += (long long)gridDim.x * blockDim.x) {
@@ -1270,6 +1271,37 @@ __global__ void splitk_reduce_kernel(const float4* __restrict__ part, int splits
       acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
     }
     out[e] = acc;
+  }
+}
+
+// The same sum for small outputs with many splits (a 64 x 576 gradient cut 49 ways): a CTA covers 32 consecutive
+// float4 columns, its eight warps take the splits in turn (warp w: splits w, w + 8, ...) and the eight partial sums
+// are added in warp order through shared memory.
+__global__ void __launch_bounds__(256)
+splitk_reduce_wide_kernel(const float4* __restrict__ part, int splits, long long n4, float4* __restrict__ out) {
+  __shared__ float4 red[8][32];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  for (long long e0 = (long long)blockIdx.x * 32; e0 < n4; e0 += (long long)gridDim.x * 32) {
+    const long long e = e0 + lane;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (e < n4) {
+#pragma unroll 4
+      for (int sp = w; sp < splits; sp += 8) {
+        const float4 v = __ldg(part + (long long)sp * n4 + e);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+      }
+    }
+    red[w][lane] = acc;
+    __syncthreads();
+    if (w == 0 && e < n4) {
+#pragma unroll
+      for (int k = 1; k < 8; ++k) {
+        const float4 v = red[k][lane];
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+      }
+      out[e] = acc;
+    }
+    __syncthreads();
   }
 }
 
@@ -1707,6 +1739,23 @@ int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, u
   return BIMASK_OK;
 }
 
+// Adds up the split-K partial results into dW.
+static int launch_splitk_reduce(const float* partials, int splits, long long n4, float* dW, cudaStream_t s) {
+  const float4* part = reinterpret_cast<const float4*>(partials);
+  float4* out = reinterpret_cast<float4*>(dW);
+  if (n4 >= 148 * 1024 || splits < 8) {
+    long long blocks = (n4 + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    splitk_reduce_kernel<<<(unsigned)blocks, 256, 0, s>>>(part, splits, n4, out);
+  } else {
+    const long long blocks = (n4 + 31) / 32;               // < 148 * 32
+    splitk_reduce_wide_kernel<<<(unsigned)blocks, 256, 0, s>>>(part, splits, n4, out);
+  }
+  count_launch();
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
 // Split-K plan of the dense product for a reduction of k_tiles 64-deep tiles.
 static bool wgrad_uses_single(int I) { return I <= 128; }       // one 128-row tile: no CTA pairs
 
@@ -1782,12 +1831,7 @@ int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int 
   BIMASK_CUDA_OK(cudaGetLastError());
   if (splits > 1) {
     const long long n4 = (long long)I * J / 4;
-    long long blocks = (n4 + 255) / 256;
-    if (blocks > 148 * 8) blocks = 148 * 8;
-    splitk_reduce_kernel<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(partials), splits, n4,
-                                                         reinterpret_cast<float4*>(dW));
-    count_launch();
-    BIMASK_CUDA_OK(cudaGetLastError());
+    if ((rc = launch_splitk_reduce(partials, splits, n4, dW, s)) != BIMASK_OK) return rc;
   }
   return BIMASK_OK;
 }
@@ -1836,12 +1880,7 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
   BIMASK_CUDA_OK(cudaGetLastError());
   if (splits > 1) {
     const long long n4 = (long long)I * J / 4;
-    long long blocks = (n4 + 255) / 256;
-    if (blocks > 148 * 8) blocks = 148 * 8;
-    splitk_reduce_kernel<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(partials), splits, n4,
-                                                         reinterpret_cast<float4*>(dW));
-    count_launch();
-    BIMASK_CUDA_OK(cudaGetLastError());
+    if ((rc = launch_splitk_reduce(partials, splits, n4, dW, s)) != BIMASK_OK) return rc;
   }
   return BIMASK_OK;
 }

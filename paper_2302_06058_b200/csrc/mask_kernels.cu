@@ -140,152 +140,49 @@ __global__ void hw_meta_kernel(const uint32_t* __restrict__ meta, int rows, int 
 }
 
 // ---------------------------------------------------------------------------------------
-// Backward mask + transposed pack, register variant (used when J is not a multiple of 128).
-// A CTA owns 128 columns x 64 row-blocks (256 permuted rows);
-// warp w walks the eight consecutive row-blocks 8w .. 8w+7.  For a row-block it gathers the four
-// source rows perm[4k..4k+3] with one coalesced 128-bit load per row (lane = four columns) and
-// selects per column through the table.  The operand it feeds is transposed (row = column l of
-// W, k contiguous), so each lane keeps the eight consecutive k results of its four columns in
-// registers and writes them as full 32-byte sectors -- no shared-memory transpose.  Mask words
-// (32 columns of one permuted row) are assembled with 4x4 bit transposes and an 8-lane OR.
+// Backward mask + transposed pack, asynchronous-copy variant.  A CTA owns 32 CW columns x 64 row-blocks (256
+// permuted rows); warp w walks the eight consecutive row-blocks 8w .. 8w+7.  Each warp runs its own three-deep
+// ring of shared-memory stages filled with cp.async (the slices of the four gathered rows plus their forward-mask
+// words), so the gather of row-block j+2 is in flight while row-block j is processed and costs no registers.
+// Compute uses lane = column within each of the tile's CW 32-column words: conflict-free shared loads, and a warp
+// ballot yields a complete backward-mask word.  The operand being produced is transposed (row = column l of W,
+// k contiguous): each lane keeps the eight consecutive k results of its CW columns in registers and writes them
+// as full 32-byte sectors.
+// CW = 4 (J a multiple of 128) is the variant for large matrices: 512-byte row slices, 16-byte mask-word copies.
+// CW = 1 has four times as many warps for the same matrix; it serves small matrices, where the per-warp chain of
+// eight row-blocks is what takes the time, and any J % 32 == 0.
 // ---------------------------------------------------------------------------------------
-constexpr int BWD_COLS = 128;
-constexpr int BWD_KB = 64;
-constexpr int BWD_THREADS = 256;
-
-// bit c of each of the four nibbles of x (bits c, c+4, c+8, c+12) gathered into a nibble
-__device__ __forceinline__ uint32_t gather4(uint32_t x, int c) {
-  return ((((x >> c) & 0x1111u) * 0x1248u) >> 12) & 15u;
-}
-
-__global__ void __launch_bounds__(BWD_THREADS, 3)
-bwd_mask_pack_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,
-                     const int32_t* __restrict__ perm, int I, int J, int N,
-                     uint32_t* __restrict__ maskbits_b, uint32_t* __restrict__ vals_b,
-                     uint32_t* __restrict__ meta_b, uint16_t* __restrict__ hw16) {
-  __shared__ uint32_t lut[1024];
-  for (int e = threadIdx.x; e < 1024; e += BWD_THREADS) lut[e] = lut_entry(e & 63u, e >> 6, N);
-  __syncthreads();
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  // row-block tiles vary fastest over the grid: CTAs resident together write neighbouring
-  // pieces of the same operand rows, which L2 merges into long bursts
-  const int col0 = blockIdx.y * BWD_COLS;
-  const int jwords = J >> 5;
-  const int kfirst = blockIdx.x * BWD_KB + 8 * warp;      // this warp's eight row-blocks
-  if (kfirst >= (I >> 2)) return;                         // I % 32 == 0: all eight or none
-  const int col = col0 + 4 * lane;                        // this lane's four columns
-  const bool active = col < J;
-  const int fword = (col0 >> 5) + (lane >> 3);            // mask word holding those columns
-  const int fshift = 4 * (lane & 7);
-  const uint32_t gmask = 0xFFu << (lane & 24);
-  uint32_t vacc[4][8];
-  uint32_t cacc[4] = {0u, 0u, 0u, 0u};
-  // software pipeline: the rows of row-block j+1 are in flight while row-block j is processed,
-  // and the permutation entries are fetched two row-blocks ahead (index -> address -> data)
-  auto clamp4 = [&](int4 p4) {
-    return make_int4(min(max(p4.x, 0), I - 1), min(max(p4.y, 0), I - 1), min(max(p4.z, 0), I - 1),
-                     min(max(p4.w, 0), I - 1));
-  };
-  auto load_rows = [&](const int4 src, float4 (&w)[4], uint32_t& fn) {
-    const int r[4] = {src.x, src.y, src.z, src.w};
-    uint32_t f[4];
-#pragma unroll
-    for (int m = 0; m < 4; ++m) {
-      if (active) {
-        w[m] = __ldg(reinterpret_cast<const float4*>(W + (size_t)r[m] * J + col));
-        f[m] = __ldg(maskbits_f + (size_t)r[m] * jwords + fword);
-      } else {
-        w[m] = make_float4(0.f, 0.f, 0.f, 0.f);
-        f[m] = 0u;
-      }
-    }
-    fn = ((f[0] >> fshift) & 15u) | (((f[1] >> fshift) & 15u) << 4) | (((f[2] >> fshift) & 15u) << 8) |
-         (((f[3] >> fshift) & 15u) << 12);
-  };
-  const int4* perm4 = reinterpret_cast<const int4*>(perm) + kfirst;
-  int4 p_next = clamp4(__ldg(perm4 + 1));
-  float4 wn[4];
-  uint32_t fnn;
-  load_rows(clamp4(__ldg(perm4)), wn, fnn);
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const int k = kfirst + j;
-    float4 w[4] = {wn[0], wn[1], wn[2], wn[3]};
-    const uint32_t fn = fnn;
-    if (j + 1 < 8) {
-      const int4 p_use = p_next;
-      if (j + 2 < 8) p_next = clamp4(__ldg(perm4 + j + 2));
-      load_rows(p_use, wn, fnn);
-    }
-    uint32_t kept = 0;                                    // nibble c = keep mask of column c
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const float w0 = c == 0 ? w[0].x : c == 1 ? w[0].y : c == 2 ? w[0].z : w[0].w;
-      const float w1 = c == 0 ? w[1].x : c == 1 ? w[1].y : c == 2 ? w[1].z : w[1].w;
-      const float w2 = c == 0 ? w[2].x : c == 1 ? w[2].y : c == 2 ? w[2].z : w[2].w;
-      const float w3 = c == 0 ? w[3].x : c == 1 ? w[3].y : c == 2 ? w[3].z : w[3].w;
-      const uint32_t k0 = mag_key(w0), k1 = mag_key(w1), k2 = mag_key(w2), k3 = mag_key(w3);
-      const uint32_t e = lut[(gather4(fn, c) << 6) | cmp6(k0, k1, k2, k3)];
-      vacc[c][j] = slots<false>(e, w0, w1, w2, w3, k0, k1, k2, k3);
-      cacc[c] |= ((e >> 4) & 15u) << (4 * j);
-      kept |= (e & 15u) << (4 * c);
-    }
-#pragma unroll
-    for (int m = 0; m < 4; ++m) {
-      const uint32_t word = __reduce_or_sync(gmask, gather4(kept, m) << fshift);
-      if (active && (lane & 7) == 0) maskbits_b[(size_t)(4 * k + m) * jwords + fword] = word;
-    }
-  }
-  if (active) {
-    const size_t vrow = (size_t)I >> 2;                   // u32 (bf16 pairs) per row of vals_b
-    const size_t mrow = (size_t)I >> 5;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      uint4* dst = reinterpret_cast<uint4*>(vals_b + (size_t)(col + c) * vrow + kfirst);
-      dst[0] = make_uint4(vacc[c][0], vacc[c][1], vacc[c][2], vacc[c][3]);
-      dst[1] = make_uint4(vacc[c][4], vacc[c][5], vacc[c][6], vacc[c][7]);
-      meta_b[(size_t)(col + c) * mrow + (kfirst >> 3)] = cacc[c];
-      if (hw16) scatter_hw(hw16, I >> 7, col + c, kfirst >> 3, cacc[c]);
-    }
-  }
-}
-
-
-// ---------------------------------------------------------------------------------------
-// Backward mask + transposed pack, asynchronous-copy variant (J a multiple of 128).  A CTA owns
-// 128 columns x 64 row-blocks (256 permuted rows); warp w walks the eight consecutive row-blocks
-// 8w .. 8w+7.  Each warp runs its own three-deep ring of shared-memory stages filled with
-// cp.async (16 bytes per lane: the 512-byte slices of the four gathered rows, plus their 16 bytes
-// of forward-mask words), so the gather of row-block j+2 is in flight while row-block j is
-// processed and costs no registers.  Compute uses lane = column within each of the tile's four
-// 32-column words: conflict-free shared loads, and a warp ballot yields a complete backward-mask
-// word.  The operand being produced is transposed (row = column l of W, k contiguous): each lane
-// keeps the eight consecutive k results of its four columns in registers and writes them as
-// full 32-byte sectors.
-// ---------------------------------------------------------------------------------------
-constexpr int B4_COLS = 128, B4_KB = 64, B4_WARPS = 8, B4_THREADS = 32 * B4_WARPS, B4_RING = 3;
-constexpr int B4_STAGE = 4 * 512 + 64;                     // four row slices + four x 16 bytes of mask words
-constexpr int B4_SMEM = B4_WARPS * B4_RING * B4_STAGE + 4 * B4_KB * 16 + 1024 * 4 + B4_KB * 16;
+constexpr int B4_KB = 64, B4_WARPS = 8, B4_THREADS = 32 * B4_WARPS, B4_RING = 3;
+template <int CW>
+struct B4Cfg {
+  static constexpr int STAGE = 4 * 128 * CW + 64;          // four row slices + four x 16 bytes for the mask words
+  static constexpr int SMEM = B4_WARPS * B4_RING * STAGE + 4 * B4_KB * 16 + 1024 * 4 + B4_KB * 16;
+};
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
+template <int CW>
 __global__ void __launch_bounds__(B4_THREADS, 3)
 bwd_mask_async_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,
                       const int32_t* __restrict__ perm, int I, int J, int N,
                       uint32_t* __restrict__ maskbits_b, uint32_t* __restrict__ vals_b,
                       uint32_t* __restrict__ meta_b, uint16_t* __restrict__ hw16) {
+  using C = B4Cfg<CW>;
   extern __shared__ __align__(128) uint8_t smem[];
-  uint8_t* ring = smem;                                                          // [warp][stage][B4_STAGE]
-  uint4* mb_s = reinterpret_cast<uint4*>(smem + B4_WARPS * B4_RING * B4_STAGE);  // [256 rows] x 4 mask words
+  uint8_t* ring = smem;                                                          // [warp][stage][C::STAGE]
+  uint4* mb_s = reinterpret_cast<uint4*>(smem + B4_WARPS * B4_RING * C::STAGE);  // [256 rows] x up to 4 mask words
   uint32_t* lut = reinterpret_cast<uint32_t*>(mb_s + 4 * B4_KB);                 // [1024]
   int4* perm_s = reinterpret_cast<int4*>(lut + 1024);                            // [64]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int col0 = blockIdx.y * B4_COLS;                   // J % 128 == 0: the tile is always full
+  const int col0 = blockIdx.y * 32 * CW;                   // J % (32 CW) == 0: the tile is always full
   const int kb0 = blockIdx.x * B4_KB;
   const int kb_here = min(B4_KB, (I >> 2) - kb0);          // multiple of 8 (I % 32 == 0)
   const int jwords = J >> 5;
@@ -300,40 +197,47 @@ bwd_mask_async_kernel(const float* __restrict__ W, const uint32_t* __restrict__ 
   __syncthreads();
   const int kw = 8 * warp;                                 // this warp's row-blocks kw .. kw+7 of the tile
   if (kw < kb_here) {
-    uint8_t* my_ring = ring + warp * B4_RING * B4_STAGE;
+    uint8_t* my_ring = ring + warp * B4_RING * C::STAGE;
     const uint32_t ring_u32 = ptx::smem_u32(my_ring);
     auto issue = [&](int j) {                              // start the gather of row-block kw + j
       const int4 p4 = perm_s[kw + j];
       const int r[4] = {p4.x, p4.y, p4.z, p4.w};
-      const uint32_t dst = ring_u32 + (j % B4_RING) * B4_STAGE;
+      const uint32_t dst = ring_u32 + (j % B4_RING) * C::STAGE;
+      if (CW == 4) {
 #pragma unroll
-      for (int m = 0; m < 4; ++m) cp_async16(dst + m * 512 + 16 * lane, W + (size_t)r[m] * J + col0 + 4 * lane);
-      if (lane < 4) cp_async16(dst + 2048 + 16 * lane, maskbits_f + (size_t)r[lane] * jwords + (col0 >> 5));
+        for (int m = 0; m < 4; ++m) cp_async16(dst + m * 512 + 16 * lane, W + (size_t)r[m] * J + col0 + 4 * lane);
+        if (lane < 4) cp_async16(dst + 2048 + 16 * lane, maskbits_f + (size_t)r[lane] * jwords + (col0 >> 5));
+      } else {                                             // 128-byte slices: eight lanes per row
+        cp_async16(dst + 16 * lane, W + (size_t)r[lane >> 3] * J + col0 + 4 * (lane & 7));
+        if (lane < 4) cp_async4(dst + 512 + 16 * lane, maskbits_f + (size_t)r[lane] * jwords + (col0 >> 5));
+      }
       cp_async_commit();
     };
     issue(0);
     issue(1);
-    uint32_t vacc[4][8];
-    uint32_t cacc[4] = {0u, 0u, 0u, 0u};
+    uint32_t vacc[CW][8];
+    uint32_t cacc[CW];
+#pragma unroll
+    for (int c = 0; c < CW; ++c) cacc[c] = 0u;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       if (j + 2 < 8) issue(j + 2); else cp_async_commit();  // keep the group count uniform
       cp_async_wait<2>();                                  // row-block j has landed
       __syncwarp();
-      const float* ws = reinterpret_cast<const float*>(my_ring + (j % B4_RING) * B4_STAGE);
-      const uint4* fs = reinterpret_cast<const uint4*>(my_ring + (j % B4_RING) * B4_STAGE + 2048);
-      float w[4][4];
+      const float* ws = reinterpret_cast<const float*>(my_ring + (j % B4_RING) * C::STAGE);
+      const uint4* fs = reinterpret_cast<const uint4*>(my_ring + (j % B4_RING) * C::STAGE + 128 * CW * 4);
+      float w[4][CW];
       uint4 fw[4];
 #pragma unroll
       for (int m = 0; m < 4; ++m) {
-        fw[m] = fs[m];
+        if (CW == 4) fw[m] = fs[m]; else fw[m].x = reinterpret_cast<const uint32_t*>(fs + m)[0];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) w[m][c] = ws[m * 128 + 32 * c + lane];
+        for (int c = 0; c < CW; ++c) w[m][c] = ws[m * 32 * CW + 32 * c + lane];
       }
       __syncwarp();                                        // all lanes have read the stage
       const int kk = kw + j;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < CW; ++c) {
         const uint32_t f0 = c == 0 ? fw[0].x : c == 1 ? fw[0].y : c == 2 ? fw[0].z : fw[0].w;
         const uint32_t f1 = c == 0 ? fw[1].x : c == 1 ? fw[1].y : c == 2 ? fw[1].z : fw[1].w;
         const uint32_t f2 = c == 0 ? fw[2].x : c == 1 ? fw[2].y : c == 2 ? fw[2].z : fw[2].w;
@@ -355,12 +259,15 @@ bwd_mask_async_kernel(const float* __restrict__ W, const uint32_t* __restrict__ 
     }
     cp_async_wait<0>();
     __syncwarp();
-    // this warp's 32 permuted rows of backward-mask words: one 16-byte store per lane
-    *reinterpret_cast<uint4*>(maskbits_b + (size_t)(4 * (kb0 + kw) + lane) * jwords + (col0 >> 5)) = mb_s[4 * kw + lane];
+    // this warp's 32 permuted rows of backward-mask words: one store of CW words per lane
+    if (CW == 4)
+      *reinterpret_cast<uint4*>(maskbits_b + (size_t)(4 * (kb0 + kw) + lane) * jwords + (col0 >> 5)) = mb_s[4 * kw + lane];
+    else
+      maskbits_b[(size_t)(4 * (kb0 + kw) + lane) * jwords + (col0 >> 5)] = reinterpret_cast<const uint32_t*>(mb_s + 4 * kw + lane)[0];
     const size_t vrow = (size_t)I >> 2;                    // u32 (bf16 pairs) per row of vals_b
     const size_t mrow = (size_t)I >> 5;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
+    for (int c = 0; c < CW; ++c) {
       const int l = col0 + 32 * c + lane;
       uint4* dst = reinterpret_cast<uint4*>(vals_b + (size_t)l * vrow + kb0 + kw);
       dst[0] = make_uint4(vacc[c][0], vacc[c][1], vacc[c][2], vacc[c][3]);
@@ -456,25 +363,24 @@ int launch_hw_meta(const uint32_t* meta, int rows, int K, void* hw_meta, cudaStr
 int launch_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                     int N, uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_or_null,
                     cudaStream_t s) {
-  if (J % 128 != 0) {
-    // a row of mask words is then not a multiple of 16 bytes: no 16-byte asynchronous copies
-    dim3 grid((I / 4 + BWD_KB - 1) / BWD_KB, (J + BWD_COLS - 1) / BWD_COLS);
-    bwd_mask_pack_kernel<<<grid, BWD_THREADS, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b,
-                                                      reinterpret_cast<uint32_t*>(vals_b), meta_b,
-                                                      reinterpret_cast<uint16_t*>(hw_meta_or_null));
-    count_launch();
-    BIMASK_CUDA_OK(cudaGetLastError());
-    return BIMASK_OK;
-  }
+  // the wide tile (128 columns per warp) once it gives every SM a few CTAs, the narrow one otherwise
+  const long long wide_ctas = (long long)((I / 4 + B4_KB - 1) / B4_KB) * (J / 128);
+  const bool wide = J % 128 == 0 && wide_ctas >= 2 * 148;
   static bool attr_done = false;
   if (!attr_done) {
-    BIMASK_CUDA_OK(cudaFuncSetAttribute(bwd_mask_async_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, B4_SMEM));
+    BIMASK_CUDA_OK(cudaFuncSetAttribute(bwd_mask_async_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, B4Cfg<4>::SMEM));
+    BIMASK_CUDA_OK(cudaFuncSetAttribute(bwd_mask_async_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, B4Cfg<1>::SMEM));
     attr_done = true;
   }
-  dim3 grid((I / 4 + B4_KB - 1) / B4_KB, J / B4_COLS);
-  bwd_mask_async_kernel<<<grid, B4_THREADS, B4_SMEM, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b,
-                                                         reinterpret_cast<uint32_t*>(vals_b), meta_b,
-                                                         reinterpret_cast<uint16_t*>(hw_meta_or_null));
+  uint32_t* vals32 = reinterpret_cast<uint32_t*>(vals_b);
+  uint16_t* hw16 = reinterpret_cast<uint16_t*>(hw_meta_or_null);
+  if (wide) {
+    dim3 grid((I / 4 + B4_KB - 1) / B4_KB, J / 128);
+    bwd_mask_async_kernel<4><<<grid, B4_THREADS, B4Cfg<4>::SMEM, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, vals32, meta_b, hw16);
+  } else {
+    dim3 grid((I / 4 + B4_KB - 1) / B4_KB, J / 32);
+    bwd_mask_async_kernel<1><<<grid, B4_THREADS, B4Cfg<1>::SMEM, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, vals32, meta_b, hw16);
+  }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
