@@ -31,6 +31,33 @@ int cuda_fail(cudaError_t e, const char* what);
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Programmatic dependent launch.  Every kernel of the library is launched with the attribute below, tells the
+// runtime at its very start that the next kernel in the stream may be scheduled (pdl_launch_dependents) and
+// waits for the kernels before it (pdl_wait) only after the part of its prologue that touches no global memory:
+// barrier initialisation, tensor-memory allocation, table building.  So the launch latency and the prologue of a
+// kernel overlap the tail of its predecessor; pdl_wait returns once the preceding grid has completed and its
+// writes are visible, and since every kernel calls it, completion is transitive along the stream.
+// Rule for kernel code: no global-memory access (read or write) before pdl_wait().
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // 2-D tensor map without swizzle (gemm_sm100.cu); dtype is a CUtensorMapDataType value.
 int make_tmap_plain(CUtensorMap_st* m, int dtype, const void* ptr, uint64_t inner, uint64_t outer, uint32_t box_inner,
                     uint32_t box_outer, uint32_t elem_bytes);

@@ -14,6 +14,8 @@ namespace {
 // One thread per 16-byte chunk (eight channels) of the column matrix.
 __global__ void im2col3x3_kernel(const uint4* __restrict__ x, int NB, int H, int W, int Ho, int Wo, int stride, int C8,
                                  long long total, uint4* __restrict__ cols) {
+  pdl_launch_dependents();
+  pdl_wait();
   for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
        idx += (long long)gridDim.x * blockDim.x) {
     const int c8 = (int)(idx % C8);
@@ -46,6 +48,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // wo*stride + kw - 1 = w (taps with no such output pixel contribute nothing); fp32 sums.
 __global__ void col2im3x3_kernel(const uint4* __restrict__ dcols, int NB, int H, int W, int Ho, int Wo, int stride, int C8,
                                  long long total, uint4* __restrict__ dx) {
+  pdl_launch_dependents();
+  pdl_wait();
   for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
        idx += (long long)gridDim.x * blockDim.x) {
     const int c8 = (int)(idx % C8);
@@ -81,8 +85,8 @@ int launch_im2col3x3(const uint16_t* x, int NB, int H, int W, int C, int stride,
   const long long total = (long long)NB * Ho * Wo * 9 * (C / 8);
   long long ctas = (total + 255) / 256;
   if (ctas > 148 * 16) ctas = 148 * 16;
-  im2col3x3_kernel<<<(unsigned)ctas, 256, 0, s>>>(reinterpret_cast<const uint4*>(x), NB, H, W, Ho, Wo, stride, C / 8, total,
-                                                  reinterpret_cast<uint4*>(cols));
+  BIMASK_CUDA_OK(launch_pdl(im2col3x3_kernel, (unsigned)ctas, 256, 0, s, reinterpret_cast<const uint4*>(x), NB, H, W, Ho, Wo, stride, C / 8, total,
+                                                  reinterpret_cast<uint4*>(cols)));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -93,8 +97,8 @@ int launch_col2im3x3(const uint16_t* dcols, int NB, int H, int W, int C, int str
   const long long total = (long long)NB * H * W * (C / 8);
   long long ctas = (total + 255) / 256;
   if (ctas > 148 * 16) ctas = 148 * 16;
-  col2im3x3_kernel<<<(unsigned)ctas, 256, 0, s>>>(reinterpret_cast<const uint4*>(dcols), NB, H, W, Ho, Wo, stride, C / 8, total,
-                                                  reinterpret_cast<uint4*>(dx));
+  BIMASK_CUDA_OK(launch_pdl(col2im3x3_kernel, (unsigned)ctas, 256, 0, s, reinterpret_cast<const uint4*>(dcols), NB, H, W, Ho, Wo, stride, C / 8, total,
+                                                  reinterpret_cast<uint4*>(dx)));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;

@@ -212,6 +212,7 @@ template <int N_TILE, int STAGES, bool SPARSE, bool CONV>
 __global__ void __launch_bounds__(PAIR_THREADS, 1)
 spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                    const GemmParams p) {
+  pdl_launch_dependents();
   using C = Cfg<N_TILE, STAGES, SPARSE>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -256,6 +257,7 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                                            // barriers, tensor memory and tensor-map prefetch needed no global memory
   const uint32_t tmem_meta = tmem_base + N_TILE;     // 4 columns after the accumulator (multiple of 4)
 
   if (warp == 0) {
@@ -410,6 +412,7 @@ template <int STAGES, bool CONV>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PAIR_THREADS, 1)
 spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                             const __grid_constant__ CUtensorMap tmapE, const GemmParams p) {
+  pdl_launch_dependents();
   using C = PairPCfg<STAGES>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -459,6 +462,7 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
   ptx::cluster_sync();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                                            // barriers, tensor memory and tensor-map prefetch needed no global memory
   const uint32_t tmem_meta = tmem_base + (nbuf == 2u ? 496u : 256u);
 
   if (warp == 0) {
@@ -628,6 +632,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2M_THREADS, 1)
 spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                    const __grid_constant__ CUtensorMap tmapE,
                    const GemmParams p) {
+  pdl_launch_dependents();
   using C = Pair2MCfg<STAGES>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -674,6 +679,7 @@ spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
   ptx::cluster_sync();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                                            // barriers, tensor memory and tensor-map prefetch needed no global memory
   const uint32_t tmem_meta = tmem_base + 496u;            // + 4 * row tile
 
   // 128-row block of row tile mt (0 / 1) of this CTA inside 512-row tile tile_m
@@ -800,6 +806,7 @@ template <int STAGES, bool CONV>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                   const GemmParams p, int splits) {
+  pdl_launch_dependents();
   using C = WgradCfg<STAGES>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -843,6 +850,7 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_consta
   ptx::cluster_sync();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                                            // barriers, tensor memory and tensor-map prefetch needed no global memory
 
   // item -> (tile, split) -> coordinates; identical in every role
   auto item_coords = [&](int item, int& m0, int& n0, int& kt0, int& nkt, int& split) {
@@ -984,6 +992,7 @@ template <int STAGES, bool CONV>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 wgrad_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                     const GemmParams p, int splits) {
+  pdl_launch_dependents();
   using C = WgradSingleCfg<STAGES>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -1024,6 +1033,7 @@ wgrad_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_cons
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                                            // barriers, tensor memory and tensor-map prefetch needed no global memory
 
   auto item_coords = [&](int item, int& m0, int& n0, int& kt0, int& nkt, int& split) {
     const int tile = item % num_tiles;
@@ -1158,6 +1168,8 @@ template <int R>
 __global__ void __launch_bounds__(PERMUTE_THREADS)
 permute_cols_kernel(const uint16_t* __restrict__ dY, const int32_t* __restrict__ perm, int T, int I,
                     uint16_t* __restrict__ dYp) {
+  pdl_launch_dependents();
+  pdl_wait();
   extern __shared__ uint32_t tile_w[];                   // R == 4: [I] x uint2, R == 2: [I] x uint32
   const int half = I >> 1;
   const int nthreads = (int)blockDim.x;                  // 256 .. 1024: short rows run more, smaller CTAs per SM
@@ -1225,6 +1237,8 @@ permute_cols_kernel(const uint16_t* __restrict__ dY, const int32_t* __restrict__
 __global__ void __launch_bounds__(256)
 permute_cols_small_kernel(const uint16_t* __restrict__ dY, const int32_t* __restrict__ perm, long long T, int I,
                           uint16_t* __restrict__ dYp) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int per_row = I >> 3;
   const long long total = T * per_row;
   for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
@@ -1249,6 +1263,8 @@ permute_cols_small_kernel(const uint16_t* __restrict__ dY, const int32_t* __rest
 // a millisecond, on an mbarrier that nothing will ever complete.  The wait must give up, the kernel
 // must report BIMASK_ETIMEOUT through the status word and return normally.
 __global__ void wait_probe_kernel(long long budget_cycles, int32_t* __restrict__ status_word) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ __align__(8) unsigned long long bar;
   __shared__ int abort_flag;
   if (threadIdx.x == 0) {
@@ -1264,6 +1280,8 @@ __global__ void wait_probe_kernel(long long budget_cycles, int32_t* __restrict__
 // the GPU that way.
 __global__ void splitk_reduce_kernel(const float4* __restrict__ part, int splits, long long n4,
                                      float4* __restrict__ out) {
+  pdl_launch_dependents();
+  pdl_wait();
   for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < n4; e += (long long)gridDim.x * blockDim.x) {
     float4 acc = part[e];
     for (int s = 1; s < splits; ++s) {
@@ -1279,6 +1297,8 @@ __global__ void splitk_reduce_kernel(const float4* __restrict__ part, int splits
 // are added in warp order through shared memory.
 __global__ void __launch_bounds__(256)
 splitk_reduce_wide_kernel(const float4* __restrict__ part, int splits, long long n4, float4* __restrict__ out) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ float4 red[8][32];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   for (long long e0 = (long long)blockIdx.x * 32; e0 < n4; e0 += (long long)gridDim.x * 32) {
@@ -1456,7 +1476,7 @@ int run_single(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, i
   p.tiles_n = (Ndim + N_TILE - 1) / N_TILE;
   p.raster_group = 16;
   dim3 grid(p.tiles_m * p.tiles_n, 1, 1);
-  kern<<<grid, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p);
+  BIMASK_CUDA_OK(launch_pdl(kern, grid, PAIR_THREADS, C::SMEM_BYTES, s, ta, tb, p));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -1511,7 +1531,7 @@ int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const 
   p.raster_group = 8;
   const int total = p.tiles_m * p.tiles_n;
   const int clusters = total < sms / 2 ? total : sms / 2;
-  kern<<<2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, p);
+  BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s, ta, tb, te, p));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -1560,7 +1580,7 @@ int run_sparse_pair2m(const uint16_t* vals, const void* hw_meta, const uint16_t*
   p.raster_group = 4;
   const int total = p.tiles_m * p.tiles_n;
   const int clusters = total < sms / 2 ? total : sms / 2;
-  kern<<<2 * clusters, GEMM2M_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, p);
+  BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, GEMM2M_THREADS, C::SMEM_BYTES, s, ta, tb, te, p));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -1624,7 +1644,7 @@ int run_conv_single(const uint16_t* vals, int a_rows, int a_kdim, const void* hw
   p.raster_group = 16;
   p.n_tile = N_TILE;
   dim3 grid(p.tiles_m * p.tiles_n, 1, 1);
-  kern<<<grid, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p);
+  BIMASK_CUDA_OK(launch_pdl(kern, grid, PAIR_THREADS, C::SMEM_BYTES, s, ta, tb, p));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -1660,7 +1680,7 @@ int run_conv_pair(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_m
   p.raster_group = 8;
   const int total = p.tiles_m * p.tiles_n;
   const int clusters = total < sms / 2 ? total : sms / 2;
-  kern<<<2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s>>>(ta, tb, te, p);
+  BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s, ta, tb, te, p));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -1699,7 +1719,7 @@ int launch_dense_nt(const uint16_t* A, const uint16_t* Bop, int Mdim, int Ndim, 
 }
 
 int launch_wait_probe(int32_t* status_word, cudaStream_t s) {
-  wait_probe_kernel<<<1, 32, 0, s>>>(2000000ll, status_word);
+  BIMASK_CUDA_OK(launch_pdl(wait_probe_kernel, 1, 32, 0, s, 2000000ll, status_word));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -1710,7 +1730,7 @@ int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, u
     const long long total = (long long)T * (I >> 3);
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    permute_cols_small_kernel<<<(unsigned)blocks, 256, 0, s>>>(dY, perm, (long long)T, I, dYp);
+    BIMASK_CUDA_OK(launch_pdl(permute_cols_small_kernel, (unsigned)blocks, 256, 0, s, dY, perm, (long long)T, I, dYp));
     count_launch();
     BIMASK_CUDA_OK(cudaGetLastError());
     return BIMASK_OK;
@@ -1731,9 +1751,9 @@ int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, u
   if (per_sm < 1) per_sm = 1;
   const int grid = groups < 148 * per_sm ? groups : 148 * per_sm;
   if (R == 4)
-    permute_cols_kernel<4><<<grid, threads, smem, s>>>(dY, perm, T, I, dYp);
+    BIMASK_CUDA_OK(launch_pdl(permute_cols_kernel<4>, grid, threads, smem, s, dY, perm, T, I, dYp));
   else
-    permute_cols_kernel<2><<<grid, threads, smem, s>>>(dY, perm, T, I, dYp);
+    BIMASK_CUDA_OK(launch_pdl(permute_cols_kernel<2>, grid, threads, smem, s, dY, perm, T, I, dYp));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -1746,10 +1766,10 @@ static int launch_splitk_reduce(const float* partials, int splits, long long n4,
   if (n4 >= 148 * 1024 || splits < 8) {
     long long blocks = (n4 + 255) / 256;
     if (blocks > 148 * 8) blocks = 148 * 8;
-    splitk_reduce_kernel<<<(unsigned)blocks, 256, 0, s>>>(part, splits, n4, out);
+    BIMASK_CUDA_OK(launch_pdl(splitk_reduce_kernel, (unsigned)blocks, 256, 0, s, part, splits, n4, out));
   } else {
     const long long blocks = (n4 + 31) / 32;               // < 148 * 32
-    splitk_reduce_wide_kernel<<<(unsigned)blocks, 256, 0, s>>>(part, splits, n4, out);
+    BIMASK_CUDA_OK(launch_pdl(splitk_reduce_wide_kernel, (unsigned)blocks, 256, 0, s, part, splits, n4, out));
   }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
@@ -1818,14 +1838,14 @@ int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int 
     if ((rc = set_smem_attr(kern1, WgradSingleCfg<4>::SMEM_BYTES)) != BIMASK_OK) return rc;
     p.tiles_m = 1;
     const int items = p.tiles_n * splits;
-    kern1<<<items < sms ? items : sms, GEMM_THREADS, WgradSingleCfg<4>::SMEM_BYTES, s>>>(ta, tb, p, splits);
+    BIMASK_CUDA_OK(launch_pdl(kern1, items < sms ? items : sms, GEMM_THREADS, WgradSingleCfg<4>::SMEM_BYTES, s, ta, tb, p, splits));
   } else {
     auto kern = wgrad_pair_kernel<STAGES, true>;
     if ((rc = set_smem_attr(kern, Cf::SMEM_BYTES)) != BIMASK_OK) return rc;
     p.tiles_m = ((I + 127) / 128 + 1) / 2;
     const int items = p.tiles_m * p.tiles_n * splits;
     const int clusters = items < sms / 2 ? items : sms / 2;
-    kern<<<2 * clusters, GEMM_THREADS, Cf::SMEM_BYTES, s>>>(ta, tb, p, splits);
+    BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, GEMM_THREADS, Cf::SMEM_BYTES, s, ta, tb, p, splits));
   }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
@@ -1867,14 +1887,14 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
     if ((rc = set_smem_attr(kern1, WgradSingleCfg<4>::SMEM_BYTES)) != BIMASK_OK) return rc;
     p.tiles_m = 1;
     const int items = p.tiles_n * splits;
-    kern1<<<items < sms ? items : sms, GEMM_THREADS, WgradSingleCfg<4>::SMEM_BYTES, s>>>(ta, tb, p, splits);
+    BIMASK_CUDA_OK(launch_pdl(kern1, items < sms ? items : sms, GEMM_THREADS, WgradSingleCfg<4>::SMEM_BYTES, s, ta, tb, p, splits));
   } else {
     auto kern = wgrad_pair_kernel<STAGES, false>;
     if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
     p.tiles_m = ((I + 127) / 128 + 1) / 2;
     const int items = p.tiles_m * p.tiles_n * splits;
     const int clusters = items < sms / 2 ? items : sms / 2;
-    kern<<<2 * clusters, GEMM_THREADS, C::SMEM_BYTES, s>>>(ta, tb, p, splits);
+    BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, GEMM_THREADS, C::SMEM_BYTES, s, ta, tb, p, splits));
   }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());

@@ -45,6 +45,8 @@ __global__ void __launch_bounds__(FWD_THREADS)
 fwd_mask_pack_kernel(const float4* __restrict__ W4, long long nblk, int N,
                      uint32_t* __restrict__ maskbits, uint4* __restrict__ vals4,
                      uint32_t* __restrict__ meta, uint16_t* __restrict__ hw16, int jwords, SgdParams sgd) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ uint32_t lut[64];
   __shared__ float4 stage[FWD_THREADS / 32][256];
   if (threadIdx.x < 64) lut[threadIdx.x] = lut_entry(threadIdx.x, 0xFu, N);
@@ -114,6 +116,8 @@ fwd_mask_pack_kernel(const float4* __restrict__ W4, long long nblk, int N,
 // ---------------------------------------------------------------------------------------
 __global__ void hw_meta_kernel(const uint32_t* __restrict__ meta, int rows, int kwords,
                                int tiles_k, long long total_lanes, uint4* __restrict__ out) {
+  pdl_launch_dependents();
+  pdl_wait();
   // one thread per (tile, lane): the lane's four columns are one 16-byte store
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total_lanes) return;
@@ -175,6 +179,7 @@ bwd_mask_async_kernel(const float* __restrict__ W, const uint32_t* __restrict__ 
                       const int32_t* __restrict__ perm, int I, int J, int N,
                       uint32_t* __restrict__ maskbits_b, uint32_t* __restrict__ vals_b,
                       uint32_t* __restrict__ meta_b, uint16_t* __restrict__ hw16) {
+  pdl_launch_dependents();
   using C = B4Cfg<CW>;
   extern __shared__ __align__(128) uint8_t smem[];
   uint8_t* ring = smem;                                                          // [warp][stage][C::STAGE]
@@ -189,6 +194,7 @@ bwd_mask_async_kernel(const float* __restrict__ W, const uint32_t* __restrict__ 
   const unsigned last_row = (unsigned)(I - 1);
 
   for (int e = threadIdx.x; e < 1024; e += B4_THREADS) lut[e] = lut_entry(e & 63u, e >> 6, N);
+  pdl_wait();                                              // the table needed no global memory
   for (int kk = threadIdx.x; kk < kb_here; kk += B4_THREADS) {
     const int4 p4 = __ldg(reinterpret_cast<const int4*>(perm) + kb0 + kk);
     perm_s[kk] = make_int4((int)min((unsigned)p4.x, last_row), (int)min((unsigned)p4.y, last_row),
@@ -290,11 +296,11 @@ int launch_fwd_mask(const float* W, int I, int J, int N, uint32_t* maskbits, uin
   if (ctas < 1) ctas = 1;
   const SgdParams none{nullptr, nullptr, nullptr, 0.f, 0.f, 0.f};
   if (N == 2)
-    fwd_mask_pack_kernel<true, false><<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
-        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, none);
+    BIMASK_CUDA_OK(launch_pdl(fwd_mask_pack_kernel<true, false>, (unsigned)ctas, FWD_THREADS, 0, s,
+        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, none));
   else
-    fwd_mask_pack_kernel<false, false><<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
-        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, none);
+    BIMASK_CUDA_OK(launch_pdl(fwd_mask_pack_kernel<false, false>, (unsigned)ctas, FWD_THREADS, 0, s,
+        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, none));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -311,11 +317,11 @@ int launch_sgd_fwd_mask(float* W, const float* dW, float* mom, int I, int J, int
   const SgdParams p{reinterpret_cast<float4*>(W), reinterpret_cast<const float4*>(dW), reinterpret_cast<float4*>(mom),
                     lr, momentum, weight_decay};
   if (N == 2)
-    fwd_mask_pack_kernel<true, true><<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
-        nullptr, nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, p);
+    BIMASK_CUDA_OK(launch_pdl(fwd_mask_pack_kernel<true, true>, (unsigned)ctas, FWD_THREADS, 0, s,
+        nullptr, nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, p));
   else
-    fwd_mask_pack_kernel<false, true><<<(unsigned)ctas, FWD_THREADS, 0, s>>>(
-        nullptr, nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, p);
+    BIMASK_CUDA_OK(launch_pdl(fwd_mask_pack_kernel<false, true>, (unsigned)ctas, FWD_THREADS, 0, s,
+        nullptr, nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, p));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -323,6 +329,8 @@ int launch_sgd_fwd_mask(float* W, const float* dW, float* mom, int I, int J, int
 
 // Plain update pass (same arithmetic), for the patterns whose mask kernel is the generic one.
 __global__ void sgd_update_kernel(long long n4, SgdParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   for (long long at = (long long)blockIdx.x * blockDim.x + threadIdx.x; at < n4; at += (long long)gridDim.x * blockDim.x) {
     float4 w = p.W4[at];
     const float4 dw = __ldg(p.dW4 + at);
@@ -344,7 +352,7 @@ int launch_sgd_update(float* W, const float* dW, float* mom, long long n, float 
   if (ctas < 1) ctas = 1;
   const SgdParams p{reinterpret_cast<float4*>(W), reinterpret_cast<const float4*>(dW), reinterpret_cast<float4*>(mom),
                     lr, momentum, weight_decay};
-  sgd_update_kernel<<<(unsigned)ctas, 256, 0, s>>>(n4, p);
+  BIMASK_CUDA_OK(launch_pdl(sgd_update_kernel, (unsigned)ctas, 256, 0, s, n4, p));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -353,8 +361,8 @@ int launch_sgd_update(float* W, const float* dW, float* mom, long long n, float 
 int launch_hw_meta(const uint32_t* meta, int rows, int K, void* hw_meta, cudaStream_t s) {
   const int tiles_m = (rows + 127) / 128, tiles_k = (K + 127) / 128;
   const long long total = (long long)tiles_m * tiles_k * 128;
-  hw_meta_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(meta, rows, K / 32, tiles_k, total,
-                                                                 reinterpret_cast<uint4*>(hw_meta));
+  BIMASK_CUDA_OK(launch_pdl(hw_meta_kernel, (unsigned)((total + 255) / 256), 256, 0, s, meta, rows, K / 32, tiles_k, total,
+                                                                 reinterpret_cast<uint4*>(hw_meta)));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -376,10 +384,10 @@ int launch_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* p
   uint16_t* hw16 = reinterpret_cast<uint16_t*>(hw_meta_or_null);
   if (wide) {
     dim3 grid((I / 4 + B4_KB - 1) / B4_KB, J / 128);
-    bwd_mask_async_kernel<4><<<grid, B4_THREADS, B4Cfg<4>::SMEM, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, vals32, meta_b, hw16);
+    BIMASK_CUDA_OK(launch_pdl(bwd_mask_async_kernel<4>, grid, B4_THREADS, B4Cfg<4>::SMEM, s, W, maskbits_f, perm, I, J, N, maskbits_b, vals32, meta_b, hw16));
   } else {
     dim3 grid((I / 4 + B4_KB - 1) / B4_KB, J / 32);
-    bwd_mask_async_kernel<1><<<grid, B4_THREADS, B4Cfg<1>::SMEM, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, vals32, meta_b, hw16);
+    BIMASK_CUDA_OK(launch_pdl(bwd_mask_async_kernel<1>, grid, B4_THREADS, B4Cfg<1>::SMEM, s, W, maskbits_f, perm, I, J, N, maskbits_b, vals32, meta_b, hw16));
   }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());

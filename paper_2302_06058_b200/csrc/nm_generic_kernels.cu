@@ -70,6 +70,8 @@ __global__ void __launch_bounds__(256)
 fwd_mask_generic_kernel(const float4* __restrict__ W4, long long nblocks, int N,
                         uint32_t* __restrict__ maskbits, uint32_t* __restrict__ vals32,
                         uint32_t* __restrict__ meta, uint16_t* __restrict__ hw16, int jwords) {
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr int LPW = 32 / M;                               // lanes per 32-column word
   constexpr int G = M / 4;                                  // groups of four per block
   __shared__ uint32_t pad16[16];                            // container entry of a group from its keep mask
@@ -169,6 +171,8 @@ template <int N, int M>
 __global__ void __launch_bounds__(256)
 score_generic_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cands, int I, int jwords,
                      int blocks_per_cta, unsigned long long* __restrict__ counts) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int c = blockIdx.y;
   const int nblk = I / M;
@@ -235,6 +239,8 @@ template <int N, int M>
 __global__ void __launch_bounds__(256)
 refine_gain_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ perm, const int32_t* __restrict__ order,
                    int I, int jwords, int32_t* __restrict__ gains, unsigned long long* __restrict__ block_best) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int pair = blockIdx.x * 8 + (threadIdx.x >> 5);
   if (pair >= (I >> 1)) return;
@@ -291,6 +297,8 @@ refine_gain_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict_
 template <int M>
 __global__ void refine_apply_kernel(const int32_t* __restrict__ order, const int32_t* __restrict__ gains,
                                     const unsigned long long* __restrict__ block_best, int I, int32_t* __restrict__ perm) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int pair = blockIdx.x * blockDim.x + threadIdx.x;
   if (pair >= (I >> 1)) return;
   const int gain = gains[pair];
@@ -305,6 +313,8 @@ __global__ void refine_apply_kernel(const int32_t* __restrict__ order, const int
 }
 
 __global__ void fill_counts_kernel(long long* counts, int P, long long v) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < P) counts[i] = v;
 }
@@ -363,6 +373,8 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
                         uint32_t* __restrict__ maskbits_b, uint32_t* __restrict__ vals_b,
                         uint32_t* __restrict__ meta_b, const float* __restrict__ S, uint64_t seed,
                         uint16_t* __restrict__ hw16) {
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr int NB = 32 / M;                                // blocks per 32-row pass
   constexpr int G = M / 4;
   __shared__ uint32_t pad16[16];
@@ -451,13 +463,13 @@ int launch_fwd_mask_generic(const float* W, int I, int J, int N, int M, uint32_t
   const float4* W4 = reinterpret_cast<const float4*>(W);
   uint32_t* v32 = reinterpret_cast<uint32_t*>(vals_or_null);
   if (M == 8) {
-    if (mode == 1) fwd_mask_generic_kernel<8, 1><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw);
-    else if (mode == 2) fwd_mask_generic_kernel<8, 2><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw);
-    else fwd_mask_generic_kernel<8, 0><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw);
+    if (mode == 1) BIMASK_CUDA_OK(launch_pdl(fwd_mask_generic_kernel<8, 1>, (unsigned)ctas, 256, 0, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw));
+    else if (mode == 2) BIMASK_CUDA_OK(launch_pdl(fwd_mask_generic_kernel<8, 2>, (unsigned)ctas, 256, 0, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw));
+    else BIMASK_CUDA_OK(launch_pdl(fwd_mask_generic_kernel<8, 0>, (unsigned)ctas, 256, 0, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw));
   } else {
-    if (mode == 1) fwd_mask_generic_kernel<16, 1><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw);
-    else if (mode == 2) fwd_mask_generic_kernel<16, 2><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw);
-    else fwd_mask_generic_kernel<16, 0><<<(unsigned)ctas, 256, 0, s>>>(W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw);
+    if (mode == 1) BIMASK_CUDA_OK(launch_pdl(fwd_mask_generic_kernel<16, 1>, (unsigned)ctas, 256, 0, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw));
+    else if (mode == 2) BIMASK_CUDA_OK(launch_pdl(fwd_mask_generic_kernel<16, 2>, (unsigned)ctas, 256, 0, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw));
+    else BIMASK_CUDA_OK(launch_pdl(fwd_mask_generic_kernel<16, 0>, (unsigned)ctas, 256, 0, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw));
   }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
@@ -472,10 +484,10 @@ static int launch_score_m(const uint32_t* bits, const int32_t* cands, int I, int
   dim3 grid((nblk + per_cta - 1) / per_cta, P);
   unsigned long long* cnt = reinterpret_cast<unsigned long long*>(counts);
   switch (N) {
-    case 1: score_generic_kernel<1, M><<<grid, 256, 0, s>>>(bits, cands, I, J / 32, per_cta, cnt); break;
-    case 2: score_generic_kernel<2, M><<<grid, 256, 0, s>>>(bits, cands, I, J / 32, per_cta, cnt); break;
-    case 3: score_generic_kernel<3, M><<<grid, 256, 0, s>>>(bits, cands, I, J / 32, per_cta, cnt); break;
-    default: score_generic_kernel<4, M><<<grid, 256, 0, s>>>(bits, cands, I, J / 32, per_cta, cnt); break;
+    case 1: BIMASK_CUDA_OK(launch_pdl(score_generic_kernel<1, M>, grid, 256, 0, s, bits, cands, I, J / 32, per_cta, cnt)); break;
+    case 2: BIMASK_CUDA_OK(launch_pdl(score_generic_kernel<2, M>, grid, 256, 0, s, bits, cands, I, J / 32, per_cta, cnt)); break;
+    case 3: BIMASK_CUDA_OK(launch_pdl(score_generic_kernel<3, M>, grid, 256, 0, s, bits, cands, I, J / 32, per_cta, cnt)); break;
+    default: BIMASK_CUDA_OK(launch_pdl(score_generic_kernel<4, M>, grid, 256, 0, s, bits, cands, I, J / 32, per_cta, cnt)); break;
   }
   return BIMASK_OK;
 }
@@ -483,11 +495,11 @@ static int launch_score_m(const uint32_t* bits, const int32_t* cands, int I, int
 int launch_score_generic(const uint32_t* bits, const int32_t* cands, int I, int J, int N, int M, int P,
                          int64_t* counts, cudaStream_t s) {
   if (N >= M) {                                             // every block is eligible
-    fill_counts_kernel<<<(P + 255) / 256, 256, 0, s>>>(reinterpret_cast<long long*>(counts), P, (long long)(I / M) * J);
+    BIMASK_CUDA_OK(launch_pdl(fill_counts_kernel, (P + 255) / 256, 256, 0, s, reinterpret_cast<long long*>(counts), P, (long long)(I / M) * J));
   } else {
     BIMASK_CUDA_OK(cudaMemsetAsync(counts, 0, (size_t)P * sizeof(int64_t), s));
-    if (M == 8) launch_score_m<8>(bits, cands, I, J, N, P, counts, s);
-    else launch_score_m<16>(bits, cands, I, J, N, P, counts, s);
+    const int rc = M == 8 ? launch_score_m<8>(bits, cands, I, J, N, P, counts, s) : launch_score_m<16>(bits, cands, I, J, N, P, counts, s);
+    if (rc != BIMASK_OK) return rc;
   }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
@@ -495,23 +507,24 @@ int launch_score_generic(const uint32_t* bits, const int32_t* cands, int I, int 
 }
 
 template <int M, int CRIT>
-static void launch_bwd_mc(dim3 grid, int mode, const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
+static int launch_bwd_mc(dim3 grid, int mode, const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                           int N, uint32_t* maskbits_b, uint32_t* v32, uint32_t* meta_b, const float* S, uint64_t seed,
                           uint16_t* hw16, cudaStream_t s) {
-  if (mode == 1) bwd_mask_generic_kernel<M, 1, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16);
-  else if (mode == 2) bwd_mask_generic_kernel<M, 2, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16);
-  else bwd_mask_generic_kernel<M, 0, CRIT><<<grid, 256, 0, s>>>(W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16);
+  if (mode == 1) BIMASK_CUDA_OK(launch_pdl(bwd_mask_generic_kernel<M, 1, CRIT>, grid, 256, 0, s, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16));
+  else if (mode == 2) BIMASK_CUDA_OK(launch_pdl(bwd_mask_generic_kernel<M, 2, CRIT>, grid, 256, 0, s, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16));
+  else BIMASK_CUDA_OK(launch_pdl(bwd_mask_generic_kernel<M, 0, CRIT>, grid, 256, 0, s, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16));
+  return BIMASK_OK;
 }
 
 template <int M>
-static void launch_bwd_m(int crit, dim3 grid, int mode, const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I,
+static int launch_bwd_m(int crit, dim3 grid, int mode, const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I,
                          int J, int N, uint32_t* maskbits_b, uint32_t* v32, uint32_t* meta_b, const float* S, uint64_t seed,
                          uint16_t* hw16, cudaStream_t s) {
   switch (crit) {
-    case 1: launch_bwd_mc<M, 1>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16, s); break;
-    case 2: launch_bwd_mc<M, 2>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16, s); break;
-    case 3: launch_bwd_mc<M, 3>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16, s); break;
-    default: launch_bwd_mc<M, 0>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16, s); break;
+    case 1: return launch_bwd_mc<M, 1>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16, s);
+    case 2: return launch_bwd_mc<M, 2>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16, s);
+    case 3: return launch_bwd_mc<M, 3>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16, s);
+    default: return launch_bwd_mc<M, 0>(grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b, S, seed, hw16, s);
   }
 }
 
@@ -529,20 +542,23 @@ int launch_bwd_mask_criterion(const float* W, const float* S, const uint32_t* ma
     z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull; z ^= z >> 27; z *= 0x94D049BB133111EBull; z ^= z >> 31;
     seed = z;
   }
-  if (M == 4) launch_bwd_m<4>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, hw16, s);
-  else if (M == 8) launch_bwd_m<8>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, hw16, s);
-  else launch_bwd_m<16>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, hw16, s);
+  int rc;
+  if (M == 4) rc = launch_bwd_m<4>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, hw16, s);
+  else if (M == 8) rc = launch_bwd_m<8>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, hw16, s);
+  else rc = launch_bwd_m<16>(crit, grid, mode, W, maskbits_f, perm, I, J, N, maskbits_b, v32, meta_b_or_null, S, seed, hw16, s);
+  if (rc != BIMASK_OK) return rc;
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }
 
 template <int N, int M>
-static void refine_round(const uint32_t* bits, int32_t* perm, const int32_t* order, int I, int J, int32_t* gains,
+static int refine_round(const uint32_t* bits, int32_t* perm, const int32_t* order, int I, int J, int32_t* gains,
                          unsigned long long* block_best, cudaStream_t s) {
   const int pairs = I / 2;
-  refine_gain_kernel<N, M><<<(pairs + 7) / 8, 256, 0, s>>>(bits, perm, order, I, J / 32, gains, block_best);
-  refine_apply_kernel<M><<<(pairs + 255) / 256, 256, 0, s>>>(order, gains, block_best, I, perm);
+  BIMASK_CUDA_OK(launch_pdl(refine_gain_kernel<N, M>, (pairs + 7) / 8, 256, 0, s, bits, perm, order, I, J / 32, gains, block_best));
+  BIMASK_CUDA_OK(launch_pdl(refine_apply_kernel<M>, (pairs + 255) / 256, 256, 0, s, order, gains, block_best, I, perm));
+  return BIMASK_OK;
 }
 
 // rounds of greedy pairwise swaps on perm (in place).  orders: rounds x I position permutations; scratch:
@@ -552,24 +568,26 @@ int launch_refine(const uint32_t* bits, int I, int J, int N, int M, int rounds, 
   for (int r = 0; r < rounds; ++r) {
     BIMASK_CUDA_OK(cudaMemsetAsync(block_best, 0, (size_t)(I / M) * sizeof(unsigned long long), s));
     const int32_t* order = orders + (size_t)r * I;
+    int rc;
     if (M == 4) {
-      if (N == 1) refine_round<1, 4>(bits, perm, order, I, J, gains, block_best, s);
-      else refine_round<2, 4>(bits, perm, order, I, J, gains, block_best, s);
+      if (N == 1) rc = refine_round<1, 4>(bits, perm, order, I, J, gains, block_best, s);
+      else rc = refine_round<2, 4>(bits, perm, order, I, J, gains, block_best, s);
     } else if (M == 8) {
       switch (N) {
-        case 1: refine_round<1, 8>(bits, perm, order, I, J, gains, block_best, s); break;
-        case 2: refine_round<2, 8>(bits, perm, order, I, J, gains, block_best, s); break;
-        case 3: refine_round<3, 8>(bits, perm, order, I, J, gains, block_best, s); break;
-        default: refine_round<4, 8>(bits, perm, order, I, J, gains, block_best, s); break;
+        case 1: rc = refine_round<1, 8>(bits, perm, order, I, J, gains, block_best, s); break;
+        case 2: rc = refine_round<2, 8>(bits, perm, order, I, J, gains, block_best, s); break;
+        case 3: rc = refine_round<3, 8>(bits, perm, order, I, J, gains, block_best, s); break;
+        default: rc = refine_round<4, 8>(bits, perm, order, I, J, gains, block_best, s); break;
       }
     } else {
       switch (N) {
-        case 1: refine_round<1, 16>(bits, perm, order, I, J, gains, block_best, s); break;
-        case 2: refine_round<2, 16>(bits, perm, order, I, J, gains, block_best, s); break;
-        case 3: refine_round<3, 16>(bits, perm, order, I, J, gains, block_best, s); break;
-        default: refine_round<4, 16>(bits, perm, order, I, J, gains, block_best, s); break;
+        case 1: rc = refine_round<1, 16>(bits, perm, order, I, J, gains, block_best, s); break;
+        case 2: rc = refine_round<2, 16>(bits, perm, order, I, J, gains, block_best, s); break;
+        case 3: rc = refine_round<3, 16>(bits, perm, order, I, J, gains, block_best, s); break;
+        default: rc = refine_round<4, 16>(bits, perm, order, I, J, gains, block_best, s); break;
       }
     }
+    if (rc != BIMASK_OK) return rc;
     count_launch();
     count_launch();
     BIMASK_CUDA_OK(cudaGetLastError());

@@ -34,6 +34,7 @@ __global__ void __launch_bounds__(GEN_THREADS)
 gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int q_log2, int cap,
                       int32_t* __restrict__ cands, unsigned long long* __restrict__ zero_counts,
                       int32_t* __restrict__ zero_ticket) {
+  pdl_launch_dependents();                               // the candidates depend on the seed alone: no wait up here
   extern __shared__ unsigned long long keys[];           // cap keys, then nbq bucket counters
   const int nbq_log2 = nb_log2 - q_log2;
   const int nbq = 1 << nbq_log2;
@@ -46,12 +47,7 @@ gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int q_log2, i
   const unsigned long long stream = mix64(seed + 0x9E3779B97F4A7C15ull * (unsigned long long)(c + 1));
   const int shift = 64 - nb_log2;
   for (int b = tid; b < nbq; b += GEN_THREADS) count[b] = 0;
-  if (tid == 0) {
-    lower_total = 0;
-    // the count kernel that follows adds into counts[c] and uses *zero_ticket as its "CTAs done" counter
-    if (part == 0 && zero_counts) zero_counts[c] = 0ull;
-    if (part == 0 && c == 0 && zero_ticket) *zero_ticket = 0;
-  }
+  if (tid == 0) lower_total = 0;
   __syncthreads();
   uint32_t lower = 0;
   for (int i = tid; i < I; i += GEN_THREADS) {
@@ -116,6 +112,12 @@ gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int q_log2, i
     }
   }
   __syncthreads();
+  pdl_wait();                                            // first global access: earlier kernels may still read these buffers
+  if (tid == 0) {
+    // the count kernel that follows adds into counts[c] and uses *zero_ticket as its "CTAs done" counter
+    if (part == 0 && zero_counts) zero_counts[c] = 0ull;
+    if (part == 0 && c == 0 && zero_ticket) *zero_ticket = 0;
+  }
   const uint32_t base = lower_total;
   for (int i = tid; i < filled; i += GEN_THREADS)
     if (base + i < (uint32_t)I) cands[(long long)c * I + base + i] = (int32_t)(keys[i] & 0xFFFFFFull);
@@ -159,6 +161,8 @@ __device__ __forceinline__ void pick_body(const long long* counts, const int32_t
 __global__ void __launch_bounds__(PICK_THREADS)
 pick_kernel(const long long* __restrict__ counts, const int32_t* __restrict__ cands, int P, int I,
             int32_t* __restrict__ best_idx, int32_t* __restrict__ best_perm) {
+  pdl_launch_dependents();
+  pdl_wait();
   pick_body(counts, cands, P, I, best_idx, best_perm);
 }
 
@@ -188,6 +192,8 @@ template <int N>
 __global__ void __launch_bounds__(SCORE_THREADS, 4)
 score_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cands, int I, int jwords,
              unsigned long long* __restrict__ counts, int P, int32_t* best_idx, int32_t* __restrict__ best_perm) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int c = blockIdx.y;
   const int nkb = I >> 2;
@@ -275,6 +281,8 @@ score_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cand
 // Debug: every row of cands is a permutation of 0..I-1.
 __global__ void check_perms_kernel(const int32_t* __restrict__ cands, int P, int I,
                                    uint8_t* __restrict__ seen, int32_t* __restrict__ ok) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int c = blockIdx.x;
   for (int i = threadIdx.x; i < I; i += blockDim.x) {
     const int v = cands[(long long)c * I + i];
@@ -286,7 +294,11 @@ __global__ void check_perms_kernel(const int32_t* __restrict__ cands, int P, int
     if (!seen[(long long)c * I + i]) atomicExch(ok, 0);
 }
 
-__global__ void set_int_kernel(int32_t* p, int32_t v) { *p = v; }
+__global__ void set_int_kernel(int32_t* p, int32_t v) {
+  pdl_launch_dependents();
+  pdl_wait();
+  *p = v;
+}
 
 }  // namespace
 
@@ -305,8 +317,8 @@ int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStrea
     attr_done = true;
   }
   dim3 grid(P, 1 << ql);
-  gen_candidates_kernel<<<grid, GEN_THREADS, smem, s>>>((unsigned long long)seed, I, lg, ql, cap, cands,
-                                                        reinterpret_cast<unsigned long long*>(zero_counts), zero_ticket);
+  BIMASK_CUDA_OK(launch_pdl(gen_candidates_kernel, grid, GEN_THREADS, smem, s, (unsigned long long)seed, I, lg, ql, cap, cands,
+                                                        reinterpret_cast<unsigned long long*>(zero_counts), zero_ticket));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -330,15 +342,15 @@ int launch_score(const uint32_t* maskbits_f, const int32_t* cands, int I, int J,
   }
   unsigned long long* cnt = reinterpret_cast<unsigned long long*>(counts);
   switch (N) {
-    case 1: score_kernel<1><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm); break;
-    case 2: score_kernel<2><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm); break;
-    case 3: score_kernel<3><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm); break;
-    default: score_kernel<4><<<grid, SCORE_THREADS, 0, s>>>(maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm); break;
+    case 1: BIMASK_CUDA_OK(launch_pdl(score_kernel<1>, grid, SCORE_THREADS, 0, s, maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm)); break;
+    case 2: BIMASK_CUDA_OK(launch_pdl(score_kernel<2>, grid, SCORE_THREADS, 0, s, maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm)); break;
+    case 3: BIMASK_CUDA_OK(launch_pdl(score_kernel<3>, grid, SCORE_THREADS, 0, s, maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm)); break;
+    default: BIMASK_CUDA_OK(launch_pdl(score_kernel<4>, grid, SCORE_THREADS, 0, s, maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm)); break;
   }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   if (pick_idx && !fuse) {
-    pick_kernel<<<1, PICK_THREADS, 0, s>>>(reinterpret_cast<const long long*>(counts), cands, P, I, pick_idx, pick_perm);
+    BIMASK_CUDA_OK(launch_pdl(pick_kernel, 1, PICK_THREADS, 0, s, reinterpret_cast<const long long*>(counts), cands, P, I, pick_idx, pick_perm));
     count_launch();
     BIMASK_CUDA_OK(cudaGetLastError());
   }
@@ -347,8 +359,8 @@ int launch_score(const uint32_t* maskbits_f, const int32_t* cands, int I, int J,
 
 int launch_pick(const int64_t* counts, const int32_t* cands, int P, int I, int32_t* best_idx,
                 int32_t* best_perm, cudaStream_t s) {
-  pick_kernel<<<1, PICK_THREADS, 0, s>>>(reinterpret_cast<const long long*>(counts), cands, P, I,
-                                         best_idx, best_perm);
+  BIMASK_CUDA_OK(launch_pdl(pick_kernel, 1, PICK_THREADS, 0, s, reinterpret_cast<const long long*>(counts), cands, P, I,
+                                         best_idx, best_perm));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -356,9 +368,9 @@ int launch_pick(const int64_t* counts, const int32_t* cands, int P, int I, int32
 
 int launch_check_perms(const int32_t* cands, int P, int I, int32_t* ok, uint8_t* seen, cudaStream_t s) {
   BIMASK_CUDA_OK(cudaMemsetAsync(seen, 0, (size_t)P * I, s));
-  set_int_kernel<<<1, 1, 0, s>>>(ok, 1);
+  BIMASK_CUDA_OK(launch_pdl(set_int_kernel, 1, 1, 0, s, ok, 1));
   count_launch();
-  check_perms_kernel<<<P, 256, 0, s>>>(cands, P, I, seen, ok);
+  BIMASK_CUDA_OK(launch_pdl(check_perms_kernel, P, 256, 0, s, cands, P, I, seen, ok));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
