@@ -12,7 +12,10 @@
  *     X is T x J bf16, dY is T x I bf16 (bf16 is passed as uint16_t bit patterns).
  *   - Every pointer is a DEVICE pointer owned by the caller, 16-byte aligned.  The library
  *     allocates nothing, frees nothing and never synchronises: work is enqueued on `stream`
- *     (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *     (a cudaStream_t passed as void*; NULL = the legacy default stream).  Kernels are launched
+ *     with programmatic stream serialization and wait for the work before them on the stream
+ *     before they touch global memory: relative to other work of the caller on the same
+ *     stream they behave like ordinary launches, and every call may be captured in a CUDA graph.
  *   - Outputs are fully overwritten, inputs are never modified.
  *   - Return value: BIMASK_OK or a negative bimask_status.  On a negative return caused by
  *     argument validation nothing was launched.  bimask_last_error() gives a text for the
