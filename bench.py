@@ -514,8 +514,10 @@ def run_gpu(args):
 
 def run_per_call(args):
     """Side measurement: every C-ABI call of the path alone, 5 warm-up + --steps timed launches each, CUDA events,
-    min and median; "cold" = a 256 MB buffer is overwritten before every launch (L2 flushed, clocks near burst because
-    of the gaps), "warm" = back to back.  Fractions are against the burst peaks (copy bandwidth, bf16 burst)."""
+    min and median; "cold" = a 256 MB buffer is overwritten and a second one read before every launch (L2 flushed and
+    left clean: after the write alone the timed kernel would also pay for the write-back of up to 126 MB of dirty
+    lines, about 19 us; clocks near burst because of the gaps), "warm" = back to back.  Fractions are against the
+    burst peaks (copy bandwidth, bf16 burst)."""
     import torch
     import paper_2302_06058_b200 as bm
     from paper_2302_06058_b200 import inputs
@@ -526,6 +528,7 @@ def run_per_call(args):
     seed = inputs.perm_seed(args.config)
     peaks = load_peaks()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    flush_rd = torch.zeros(64 << 20, dtype=torch.int32, device="cuda")
     reps = max(args.steps, 20) if args.steps != 100 else 20
     out = []
     for li, L in enumerate(cfg.layers):
@@ -562,6 +565,7 @@ def run_per_call(args):
                 for _ in range(reps):
                     if kind == "cold":
                         flush.zero_()
+                        flush_rd.max()
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     e0.record()
                     fn()
