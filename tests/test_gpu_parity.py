@@ -475,3 +475,39 @@ def test_async_host_calls_with_alternating_buffer_sets():
         assert torch.equal(host["Y"], ref["Y"].cpu()), c
         assert torch.equal(host["dX"], ref["dX"].cpu()), c
         assert torch.equal(host["dW"], ref["dW"].cpu()), c
+
+
+@pytest.mark.parametrize("I,J,T", [(256, 384, 512), (64, 576, 3000)])
+def test_back_to_back_steps_on_reused_buffers(I, J, T):
+    """Every kernel is launched as a programmatic dependent of the one before it and may begin before that one
+    has finished.  Steps on alternating inputs, enqueued back to back into the same buffers with no synchronisation
+    in between, must give each step's own results: a kernel that read or wrote ahead of its dependency would pick
+    up the other input's data."""
+    N, M, P = 2, 4, 6
+    sets = []
+    for k in range(2):
+        W = inputs.make_weight(I, J, 500 + k)
+        X = inputs.make_activation(T, J, 510 + k)
+        dY = inputs.make_activation(T, I, 520 + k)
+        sets.append((W, X, dY, dev(W), bits_dev(X), bits_dev(dY), O.layer_step(W, X, dY, N, M, P, 40 + k)))
+    b = bm.alloc_layer_buffers(T, I, J, P)
+    b["W"], b["X"], b["dY"] = torch.empty_like(sets[0][3]), torch.empty_like(sets[0][4]), torch.empty_like(sets[0][5])
+    keep = {}
+    for it in range(24):
+        k = it & 1
+        b["W"].copy_(sets[k][3]); b["X"].copy_(sets[k][4]); b["dY"].copy_(sets[k][5])
+        bm.bimask_layer_step(bm.make_layer_args(T, I, J, N, M, P, 40 + k, True, b))
+        if it >= 22:                                      # device-side copies of the last two steps' results
+            keep[k] = {n: b[n].clone() for n in ("maskbits_f", "meta_f", "counts", "perm", "maskbits_b", "meta_b", "Y", "dX", "dW")}
+    torch.cuda.synchronize()
+    assert int(b["status_word"].item()) == 0
+    for k in range(2):
+        ref, got = sets[k][6], keep[k]
+        assert np.array_equal(u32(got["maskbits_f"]), ref["maskbits_f"])
+        assert np.array_equal(u32(got["meta_f"]), ref["meta_f"])
+        assert np.array_equal(got["counts"].cpu().numpy(), ref["counts"])
+        assert np.array_equal(got["perm"].cpu().numpy(), ref["perm"])
+        assert np.array_equal(u32(got["maskbits_b"]), ref["maskbits_b"])
+        assert np.array_equal(u32(got["meta_b"]), ref["meta_b"])
+        for n in ("Y", "dX", "dW"):
+            assert rel_err(got[n].float().cpu().numpy(), ref[n]) <= TOL, (k, n)
