@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbimask.so")
-SOURCES = ["api.cu", "mask_kernels.cu", "nm_generic_kernels.cu", "perm_kernels.cu", "gemm_sm100.cu", "conv_kernels.cu"]
+SOURCES = ["api.cu", "mask_kernels.cu", "nm_generic_kernels.cu", "perm_kernels.cu", "spmm_sm100.cu", "wgrad_sm100.cu", "gemm_host.cu", "conv_kernels.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-O2"]
 

@@ -58,7 +58,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 }
 #endif
 
-// 2-D tensor map without swizzle (gemm_sm100.cu); dtype is a CUtensorMapDataType value.
+// 2-D tensor map without swizzle (gemm_host.cu); dtype is a CUtensorMapDataType value.
 int make_tmap_plain(CUtensorMap_st* m, int dtype, const void* ptr, uint64_t inner, uint64_t outer, uint32_t box_inner,
                     uint32_t box_outer, uint32_t elem_bytes);
 

@@ -1,0 +1,248 @@
+// What the tensor-core kernels share: tile configurations, the convolution geometry, kernel parameters, the tile
+// order, the accumulator drain of the 2:4 products, and the host helpers (tensor maps, SM count, shared-memory
+// attribute) implemented in gemm_host.cu.
+#pragma once
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <atomic>
+
+namespace bimask {
+
+
+constexpr long long WAIT_BUDGET = 4000000000ll;      // ~2 s of SM clocks
+constexpr int GEMM_THREADS = 192;                    // warp 0 TMA, warp 1 MMA, warps 2-5 epilogue
+// The sparse kernels that drain bf16 results use eight epilogue warps (two groups of four, one warp per
+// tensor-memory lane quadrant, taking alternate column chunks): products with a short reduction are bound by
+// that drain, not by the tensor pipe.
+constexpr int EPI_WARPS = 8;
+constexpr int PAIR_THREADS = 64 + 32 * EPI_WARPS;
+
+template <int N_TILE, int STAGES, bool SPARSE = true>
+struct Cfg {
+  static constexpr int M_TILE = 128;
+  static constexpr int K_TILE = 128;                             // logical reduction elements per stage
+  static constexpr int A_BYTES = SPARSE ? 16384 : 32768;         // 128 rows x 64 compressed, or x 128 dense, bf16
+  static constexpr int B_BYTES = N_TILE * K_TILE * 2;
+  static constexpr int E_BYTES = SPARSE ? 2048 : 0;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
+  static constexpr int META_COLS = SPARSE ? 4 : 0;
+  static constexpr int TMEM_COLS = (N_TILE + META_COLS) <= 128 ? 128 : (N_TILE + META_COLS) <= 256 ? 256 : 512;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */ +
+                                    EPI_WARPS * 2048 /* epilogue staging: one [32 tokens][128 rows] bf16 tile per group of four warps */;
+};
+
+// A 3x3 convolution as an implicit GEMM: the token operand is an NHWC tensor and a "tile of
+// tokens" is a box of wb x hb pixels of nb images, fetched with one 4-D tensor load per 64
+// channels, shifted by the filter tap the k index belongs to (pixels outside the image read 0).
+//   mode 1 (forward, Eq. 3):        k = (tap, c);  B = x,   shift (+kw-1, +kh-1)
+//   mode 2 (input gradient, Eq. 10): k = (tap, i');  B = dy[:, perm], shift (1-kw, 1-kh); the rows of
+//           the 2:4 operand for tap (kh, kw) are (kh*3+kw)*C + c.
+struct ConvGeom {
+  int mode;                 // 0: plain matrix operand
+  int H, W, NB;             // image
+  int CB;                   // channels of the token operand (x: C; dy: I)
+  int wb, hb, nb;           // pixel box of one load: wb * hb * nb tokens (powers of two)
+  int lg_wb, lg_hb;         // their logarithms
+  int tiles_w, tiles_h;     // boxes per image
+  int kt_per_tap;           // mode 2: 128-wide k tiles per filter tap (I / 128)
+  int rows_per_tap;         // mode 2: rows of the 2:4 operand per tap (C)
+};
+
+__device__ __forceinline__ void conv_box_origin(const ConvGeom& g, int box, int& w0, int& h0, int& n0) {
+  w0 = (box % g.tiles_w) * g.wb;
+  const int r = box / g.tiles_w;
+  h0 = (r % g.tiles_h) * g.hb;
+  n0 = (r / g.tiles_h) * g.nb;
+}
+
+// Channel offset and pixel shift of the 64-wide half q of k tile kt; valid = false: past the
+// reduction length (the loader then reads a box of zeros).
+__device__ __forceinline__ void conv_k_coords(const ConvGeom& g, int kt, int q, int Kdim, int& c0, int& dw, int& dh, bool& valid) {
+  if (g.mode == 1) {
+    const int j = kt * 128 + 64 * q;
+    valid = j < Kdim;
+    const int tap = j / g.CB;
+    c0 = j - tap * g.CB;
+    dh = tap / 3 - 1;
+    dw = tap % 3 - 1;
+  } else {
+    const int tap = kt / g.kt_per_tap;
+    c0 = (kt - tap * g.kt_per_tap) * 128 + 64 * q;
+    valid = true;
+    dh = 1 - tap / 3;
+    dw = 1 - tap % 3;
+  }
+}
+
+struct GemmParams {
+  ConvGeom conv;
+  const uint8_t* hw_meta;   // sparse only
+  int tiles_k_meta;         // number of 128-wide k tiles in the metadata image
+  int Mdim, Ndim, Kdim;     // D is Mdim x Ndim, reduction length Kdim (logical)
+  int k_tiles_per_split;    // dense split-K: k tiles handled by one blockIdx.z
+  int tiles_m, tiles_n;     // output tiles (CTA pairs along M for the pair kernel)
+  int raster_group;         // tiles walked along M before advancing along N
+  int n_tile;               // pair kernel: output columns per tile (multiple of 16, <= 256)
+  void* out;                // sparse: bf16 [Ndim][Mdim];  dense: fp32 [split][Mdim][Ndim]
+  int32_t* status_word;
+};
+
+
+// Tile order.  A linear id walks `group` tiles along M before it advances along N, so that the
+// CTAs resident at one time cover a near-square patch of the output and both operands are
+// re-used out of L2 instead of being streamed from HBM once per wave.
+__device__ __forceinline__ void raster(int id, int tiles_m, int tiles_n, int group, int& tm, int& tn) {
+  const int per_group = group * tiles_n;
+  const int g = id / per_group;
+  const int first = g * group;
+  const int gsize = min(group, tiles_m - first);
+  const int in = id - g * per_group;
+  tm = first + in % gsize;
+  tn = in / gsize;
+}
+
+// Epilogue of the 2:4 products.  The accumulator holds D[row][token] (row = tensor-memory lane), the result is
+// stored token-major, so a chunk of W tokens x the CTA's 128 rows is transposed on its way out by a GROUP of four
+// warps, one per tensor-memory lane quadrant:
+//   tensor memory -> registers in the accumulator-fragment layout (two 16-lane loads per warp) -> bf16 pairs ->
+//   stmatrix.trans into the group's staging tile [token][128 rows] (256-byte rows; the 16-byte unit index is
+//   XOR-ed with the token index mod 8, so the eight rows of a matrix fall into eight different bank groups) ->
+//   named barrier -> each warp reads W/4 whole token rows back and writes them with 16-byte stores, 256 contiguous
+//   bytes per token (whole 128-byte lines: half-line writes were bound by the number of write requests).
+// The tensor-memory load of the next chunk is issued before the current one is converted and stored.
+template <int W>
+__device__ __forceinline__ void epi_load(uint32_t taddr, uint32_t (&r)[W], bool zero) {
+  if (zero) {
+#pragma unroll
+    for (int j = 0; j < W; ++j) r[j] = 0u;
+  } else if (W == 32) {
+    ptx::tmem_ld_16x256b_x4(taddr, &r[0]);                 // lanes 0-15 of the quadrant
+    ptx::tmem_ld_16x256b_x4(taddr + (16u << 16), &r[16]);  // lanes 16-31
+  } else {
+    ptx::tmem_ld_16x256b_x2(taddr, &r[0]);
+    ptx::tmem_ld_16x256b_x2(taddr + (16u << 16), &r[W / 2]);
+  }
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(uint32_t lo, uint32_t hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(lo), __uint_as_float(hi));
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// `dst`: this lane's row address for token group 0 (see drain_chunks); token group g is 2048 bytes further.
+template <int W>
+__device__ __forceinline__ void epi_stage(const uint32_t (&r)[W], uint32_t dst) {
+#pragma unroll
+  for (int g = 0; g < W / 8; ++g)
+    ptx::stmatrix_x4_trans(dst + 2048u * g, pack_bf16(r[4 * g], r[4 * g + 1]), pack_bf16(r[4 * g + 2], r[4 * g + 3]),
+                           pack_bf16(r[W / 2 + 4 * g], r[W / 2 + 4 * g + 1]),
+                           pack_bf16(r[W / 2 + 4 * g + 2], r[W / 2 + 4 * g + 3]));
+}
+
+// Drains chunks c0, c0 + cstep, ... (< nchunks) of one accumulator; called by the four warps of a group with the
+// same arguments except `acc` (the warp's lane quadrant q = warp % 4, column of chunk c: W * c).  After its last
+// tensor-memory read each warp arrives once on `release_bar` (0: nobody waits for the accumulator).
+// row_of(c, t) returns where token t of chunk c starts in the result (the CTA's first row), or nullptr when that
+// token lies outside; rows_valid = how many of the CTA's 128 rows exist (a multiple of 32).
+// `stg`: the group's staging tile (W * 256 bytes, 1 KB aligned); `bar_id`: its named barrier.
+template <int W, typename RowOf>
+__device__ __forceinline__ void drain_chunks(uint32_t acc, int c0, int cstep, int nchunks, bool zero, uint32_t release_bar,
+                                             uint32_t stg, uint32_t bar_id, int q, int lane, int rows_valid, RowOf&& row_of) {
+  auto release = [&]() {
+    if (release_bar != 0u) {
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive_cluster(release_bar);
+    }
+  };
+  if (c0 >= nchunks) { release(); return; }
+  // stmatrix: lane 8 i + k addresses token k (of a group of eight) of matrix i = rows 32 q + 8 i .. + 7, i.e. unit
+  // 4 q + i of the token's 256-byte row
+  const uint32_t dst = stg + (uint32_t)(lane & 7) * 256u + ((((uint32_t)(4 * q) + ((uint32_t)lane >> 3)) ^ ((uint32_t)lane & 7u)) << 4);
+  // reading back: this warp owns tokens (W/4) q .. (W/4) q + W/4 - 1; per step lanes 0-15 take one token, lanes 16-31
+  // the next, 16 bytes (eight rows) per lane
+  const int unit = lane & 15;
+  const bool unit_ok = 8 * unit < rows_valid;
+  auto emit = [&](const uint32_t (&r)[W], int c) {
+    ptx::named_bar_sync(bar_id, 128);                     // the group has read the previous chunk out of the tile
+    epi_stage<W>(r, dst);
+    ptx::named_bar_sync(bar_id, 128);
+#pragma unroll
+    for (int i = 0; i < W / 8; ++i) {
+      const int t = (W / 4) * q + 2 * i + (lane >> 4);
+      const uint4 v = ptx::ld_shared_v4(stg + (uint32_t)t * 256u + (((uint32_t)unit ^ ((uint32_t)t & 7u)) << 4));
+      uint16_t* row = row_of(c, t);
+      if (row != nullptr && unit_ok) *reinterpret_cast<uint4*>(row + 8 * unit) = v;
+    }
+  };
+  uint32_t ra[W], rb[W];
+  epi_load<W>(acc + W * c0, ra, zero);
+#pragma unroll 1
+  for (int c = c0; c < nchunks; c += 2 * cstep) {
+    if (!zero) ptx::tmem_ld_wait();
+    const bool more1 = c + cstep < nchunks;
+    if (more1) epi_load<W>(acc + W * (c + cstep), rb, zero); else release();
+    emit(ra, c);
+    if (!more1) break;
+    if (!zero) ptx::tmem_ld_wait();
+    if (c + 2 * cstep < nchunks) epi_load<W>(acc + W * (c + 2 * cstep), ra, zero); else release();
+    emit(rb, c + cstep);
+  }
+}
+
+// ---- host helpers (gemm_host.cu) -----------------------------------------------------------
+int sm_count();
+// 2-D bf16 tensor map: `inner` contiguous elements per row, `outer` rows, box = 64 x box_rows, 128-byte swizzle,
+// out-of-range elements read as zero.
+int make_tmap(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, uint32_t box_rows);
+// The metadata image as a 2-D tensor of u32: 256 words per row, two rows per 2048-byte block.
+int make_tmap_meta(CUtensorMap* m, const void* ptr, uint64_t blocks);
+// 4-D bf16 map of an NHWC tensor (channels, W, H, NB) for loads of 64-channel pixel boxes, 128-byte swizzle.
+int make_tmap_nhwc_load(CUtensorMap* m, const void* ptr, int CH, int W, int H, int NB, int wb, int hb, int nb);
+
+// The dynamic shared-memory limit of a kernel is set once per (device, kernel): the call costs a microsecond or two
+// on the host, which a layer step of ten short launches would notice.  A kernel is always launched with the same size.
+template <typename K>
+inline int set_smem_attr(K kernel, int bytes) {
+  constexpr int SLOTS = 64;
+  static std::atomic<const void*> done[16][SLOTS];       // [device][slot]; zero-initialised
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 16) dev = -1;
+  const void* key = reinterpret_cast<const void*>(kernel);
+  if (dev >= 0)
+    for (int i = 0; i < SLOTS; ++i) {
+      const void* seen = done[dev][i].load(std::memory_order_acquire);
+      if (seen == key) return BIMASK_OK;
+      if (seen == nullptr) break;
+    }
+  BIMASK_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  if (dev >= 0)
+    for (int i = 0; i < SLOTS; ++i) {
+      const void* expect = nullptr;
+      if (done[dev][i].compare_exchange_strong(expect, key, std::memory_order_acq_rel) || expect == key) break;
+    }
+  return BIMASK_OK;
+}
+
+// ---- pixel boxes of the implicit convolution ------------------------------------------------
+inline int pow2_ceil(int v) { int p = 1; while (p < v) p <<= 1; return p; }
+inline int log2_exact(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
+
+// Pixel boxes of `tokens` tokens: as wide as the image allows (16 or 8), at least 32 tokens per image of the box.
+inline void conv_boxes(ConvGeom& g, int tokens) {
+  g.wb = g.W > 8 ? 16 : 8;
+  int hb = tokens / g.wb;
+  const int hp = pow2_ceil(g.H);
+  if (hb > hp) hb = hp;
+  if (hb < 32 / g.wb) hb = 32 / g.wb;
+  g.hb = hb;
+  g.nb = tokens / (g.wb * g.hb);
+  g.lg_wb = log2_exact(g.wb);
+  g.lg_hb = log2_exact(g.hb);
+  g.tiles_w = (g.W + g.wb - 1) / g.wb;
+  g.tiles_h = (g.H + g.hb - 1) / g.hb;
+}
+
+}  // namespace bimask
