@@ -152,9 +152,10 @@ __global__ void hw_meta_kernel(const uint32_t* __restrict__ meta, int rows, int 
 // ballot yields a complete backward-mask word.  The operand being produced is transposed (row = column l of W,
 // k contiguous): each lane keeps the eight consecutive k results of its CW columns in registers and writes them
 // as full 32-byte sectors.
-// CW = 4 (J a multiple of 128) is the variant for large matrices: 512-byte row slices, 16-byte mask-word copies.
-// CW = 1 has four times as many warps for the same matrix; it serves small matrices, where the per-warp chain of
-// eight row-blocks is what takes the time, and any J % 32 == 0.
+// CW = 2 (J a multiple of 64) is the variant for large matrices: 256-byte row slices, 64 registers, four CTAs
+// per SM (CW = 4 needs 80 registers, runs three and measured 4 % slower).
+// CW = 1 has twice as many warps again for the same matrix; it serves small matrices, where the per-warp chain
+// of eight row-blocks is what takes the time, and any J % 32 == 0.
 // ---------------------------------------------------------------------------------------
 constexpr int B4_KB = 64, B4_WARPS = 8, B4_THREADS = 32 * B4_WARPS, B4_RING = 3;
 template <int CW>
@@ -166,15 +167,18 @@ struct B4Cfg {
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
-__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+template <int WORDS>                                       // 1, 2 or 4 32-bit words
+__device__ __forceinline__ void cp_async_words(uint32_t dst, const void* src) {
+  if (WORDS == 4) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+  else if (WORDS == 2) asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
+  else asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 template <int CW>
-__global__ void __launch_bounds__(B4_THREADS, 3)
+__global__ void __launch_bounds__(B4_THREADS, 4)
 bwd_mask_async_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,
                       const int32_t* __restrict__ perm, int I, int J, int N,
                       uint32_t* __restrict__ maskbits_b, uint32_t* __restrict__ vals_b,
@@ -209,14 +213,13 @@ bwd_mask_async_kernel(const float* __restrict__ W, const uint32_t* __restrict__ 
       const int4 p4 = perm_s[kw + j];
       const int r[4] = {p4.x, p4.y, p4.z, p4.w};
       const uint32_t dst = ring_u32 + (j % B4_RING) * C::STAGE;
-      if (CW == 4) {
+      // a row slice is 128 CW bytes = 8 CW lanes x 16 bytes: CW passes of 4 / CW rows each
 #pragma unroll
-        for (int m = 0; m < 4; ++m) cp_async16(dst + m * 512 + 16 * lane, W + (size_t)r[m] * J + col0 + 4 * lane);
-        if (lane < 4) cp_async16(dst + 2048 + 16 * lane, maskbits_f + (size_t)r[lane] * jwords + (col0 >> 5));
-      } else {                                             // 128-byte slices: eight lanes per row
-        cp_async16(dst + 16 * lane, W + (size_t)r[lane >> 3] * J + col0 + 4 * (lane & 7));
-        if (lane < 4) cp_async4(dst + 512 + 16 * lane, maskbits_f + (size_t)r[lane] * jwords + (col0 >> 5));
+      for (int ps = 0; ps < CW; ++ps) {
+        const int m = ps * (4 / CW) + lane / (8 * CW), piece = lane % (8 * CW);
+        cp_async16(dst + m * 128 * CW + 16 * piece, W + (size_t)r[m] * J + col0 + 4 * piece);
       }
+      if (lane < 4) cp_async_words<CW>(dst + 512 * CW + 16 * lane, maskbits_f + (size_t)r[lane] * jwords + (col0 >> 5));
       cp_async_commit();
     };
     issue(0);
@@ -236,7 +239,9 @@ bwd_mask_async_kernel(const float* __restrict__ W, const uint32_t* __restrict__ 
       uint4 fw[4];
 #pragma unroll
       for (int m = 0; m < 4; ++m) {
-        if (CW == 4) fw[m] = fs[m]; else fw[m].x = reinterpret_cast<const uint32_t*>(fs + m)[0];
+        if (CW == 4) fw[m] = fs[m];
+        else if (CW == 2) { const uint2 t = reinterpret_cast<const uint2*>(fs + m)[0]; fw[m].x = t.x; fw[m].y = t.y; }
+        else fw[m].x = reinterpret_cast<const uint32_t*>(fs + m)[0];
 #pragma unroll
         for (int c = 0; c < CW; ++c) w[m][c] = ws[m * 32 * CW + 32 * c + lane];
       }
@@ -266,10 +271,10 @@ bwd_mask_async_kernel(const float* __restrict__ W, const uint32_t* __restrict__ 
     cp_async_wait<0>();
     __syncwarp();
     // this warp's 32 permuted rows of backward-mask words: one store of CW words per lane
-    if (CW == 4)
-      *reinterpret_cast<uint4*>(maskbits_b + (size_t)(4 * (kb0 + kw) + lane) * jwords + (col0 >> 5)) = mb_s[4 * kw + lane];
-    else
-      maskbits_b[(size_t)(4 * (kb0 + kw) + lane) * jwords + (col0 >> 5)] = reinterpret_cast<const uint32_t*>(mb_s + 4 * kw + lane)[0];
+    uint32_t* mrow_out = maskbits_b + (size_t)(4 * (kb0 + kw) + lane) * jwords + (col0 >> 5);
+    if (CW == 4) *reinterpret_cast<uint4*>(mrow_out) = mb_s[4 * kw + lane];
+    else if (CW == 2) *reinterpret_cast<uint2*>(mrow_out) = reinterpret_cast<const uint2*>(mb_s + 4 * kw + lane)[0];
+    else *mrow_out = reinterpret_cast<const uint32_t*>(mb_s + 4 * kw + lane)[0];
     const size_t vrow = (size_t)I >> 2;                    // u32 (bf16 pairs) per row of vals_b
     const size_t mrow = (size_t)I >> 5;
 #pragma unroll
@@ -371,22 +376,22 @@ int launch_hw_meta(const uint32_t* meta, int rows, int K, void* hw_meta, cudaStr
 int launch_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                     int N, uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_or_null,
                     cudaStream_t s) {
-  // the wide tile (128 columns per warp) once it gives every SM a few CTAs, the narrow one otherwise
-  const long long wide_ctas = (long long)((I / 4 + B4_KB - 1) / B4_KB) * (J / 128);
-  const bool wide = J % 128 == 0 && wide_ctas >= 2 * 148;
+  // the wide tile (64 columns per warp) once it gives every SM a few CTAs, the narrow one otherwise
+  const int row_tiles = (I / 4 + B4_KB - 1) / B4_KB;
+  const bool wide = J % 64 == 0 && (long long)row_tiles * (J / 64) >= 4 * 148;
   static bool attr_done = false;
   if (!attr_done) {
-    BIMASK_CUDA_OK(cudaFuncSetAttribute(bwd_mask_async_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, B4Cfg<4>::SMEM));
+    BIMASK_CUDA_OK(cudaFuncSetAttribute(bwd_mask_async_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, B4Cfg<2>::SMEM));
     BIMASK_CUDA_OK(cudaFuncSetAttribute(bwd_mask_async_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, B4Cfg<1>::SMEM));
     attr_done = true;
   }
   uint32_t* vals32 = reinterpret_cast<uint32_t*>(vals_b);
   uint16_t* hw16 = reinterpret_cast<uint16_t*>(hw_meta_or_null);
   if (wide) {
-    dim3 grid((I / 4 + B4_KB - 1) / B4_KB, J / 128);
-    BIMASK_CUDA_OK(launch_pdl(bwd_mask_async_kernel<4>, grid, B4_THREADS, B4Cfg<4>::SMEM, s, W, maskbits_f, perm, I, J, N, maskbits_b, vals32, meta_b, hw16));
+    dim3 grid(row_tiles, J / 64);
+    BIMASK_CUDA_OK(launch_pdl(bwd_mask_async_kernel<2>, grid, B4_THREADS, B4Cfg<2>::SMEM, s, W, maskbits_f, perm, I, J, N, maskbits_b, vals32, meta_b, hw16));
   } else {
-    dim3 grid((I / 4 + B4_KB - 1) / B4_KB, J / 32);
+    dim3 grid(row_tiles, J / 32);
     BIMASK_CUDA_OK(launch_pdl(bwd_mask_async_kernel<1>, grid, B4_THREADS, B4Cfg<1>::SMEM, s, W, maskbits_f, perm, I, J, N, maskbits_b, vals32, meta_b, hw16));
   }
   count_launch();
