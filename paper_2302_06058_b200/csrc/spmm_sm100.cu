@@ -213,23 +213,27 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
 // ------------------------------------------------------------------------------------------
 
 
-template <int STAGES>
+template <int STAGES, bool SPARSE = true>
 struct PairPCfg {
-  static constexpr int A_BYTES = 16384;                    // 128 rows x 64 compressed bf16
+  static constexpr int A_BYTES = SPARSE ? 16384 : 32768;   // 128 rows x 64 compressed bf16, or x 128 dense (two boxes)
   static constexpr int B_MAX = 32768;                      // up to 128 rows x 128 bf16 (two 64-wide boxes)
-  static constexpr int E_BYTES = 2048;
-  static constexpr int STAGE_BYTES = A_BYTES + B_MAX + E_BYTES;        // 50 KB (the B part is N / 2 rows)
+  static constexpr int E_BYTES = SPARSE ? 2048 : 0;
+  static constexpr int STAGE_BYTES = A_BYTES + B_MAX + E_BYTES;        // 50 KB / 64 KB (the B part is N / 2 rows)
   static constexpr int STAGING_BYTES = EPI_WARPS * 2048;   // per group of four epilogue warps: one [32 tokens][128 rows] bf16 tile
   static constexpr int TMEM_COLS = 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 + 256;
 };
 
-template <int STAGES, bool CONV>
+// SPARSE = false: the same kernel on a dense bf16 A operand (masked weights of a pattern the 2:4 format cannot
+// hold): a 256 x 128 A tile per stage as two 64-wide boxes per CTA, eight K = 16 MMAs, no metadata, and two
+// accumulators at every N (tmapE is not used).
+template <int STAGES, bool CONV, bool SPARSE = true>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PAIR_THREADS, 1)
 spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                             const __grid_constant__ CUtensorMap tmapE, const GemmParams p) {
+  static_assert(SPARSE || !CONV, "the implicit convolution runs on 2:4 operands only");
   pdl_launch_dependents();
-  using C = PairPCfg<STAGES>;
+  using C = PairPCfg<STAGES, SPARSE>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -250,7 +254,7 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
   const int num_tiles = p.tiles_m * p.tiles_n;
   const int num_kt = (p.Kdim + 127) / 128;
   const int SP_N = p.n_tile;                              // output columns (tokens) per tile
-  const uint32_t nbuf = SP_N <= 240 ? 2u : 1u;            // accumulators in tensor memory
+  const uint32_t nbuf = (!SPARSE || SP_N <= 240) ? 2u : 1u;   // accumulators in tensor memory
   const uint32_t b_box = (uint32_t)(SP_N / 2) * 128u;     // bytes of one 64-wide box of this CTA's B rows
   const uint32_t stage_tx = C::A_BYTES + 2u * b_box + C::E_BYTES;
 
@@ -321,16 +325,21 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
             ptx::tma_load_2d_pair(b_s + C::B_MAX, &tmapE, 0, 2 * (meta_row * p.tiles_k_meta + meta_kt), bar);
             continue;
           }
-          ptx::tma_load_2d_pair(a_s, &tmapA, kt * 64, m0, bar);
+          if (SPARSE) {
+            ptx::tma_load_2d_pair(a_s, &tmapA, kt * 64, m0, bar);
+          } else {
+            ptx::tma_load_2d_pair(a_s, &tmapA, kt * 128, m0, bar);
+            ptx::tma_load_2d_pair(a_s + 16384, &tmapA, kt * 128 + 64, m0, bar);
+          }
           ptx::tma_load_2d_pair(b_s, &tmapB, kt * 128, nrow, bar);
           ptx::tma_load_2d_pair(b_s + b_box, &tmapB, kt * 128 + 64, nrow, bar);
-          ptx::tma_load_2d_pair(b_s + C::B_MAX, &tmapE, 0, 2 * (mt128 * p.tiles_k_meta + kt), bar);
+          if (SPARSE) ptx::tma_load_2d_pair(b_s + C::B_MAX, &tmapE, 0, 2 * (mt128 * p.tiles_k_meta + kt), bar);
         }
       }
     }
   } else if (warp == 1) {
     if (rank == 0 && ptx::elect_one()) {
-      const uint32_t idesc = ptx::idesc_bf16(256, SP_N, false, false, true);
+      const uint32_t idesc = ptx::idesc_bf16(256, SP_N, false, false, SPARSE);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++tcount) {
@@ -346,12 +355,21 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
           ptx::tc_fence_after();
           const uint32_t a_s = base + s * C::STAGE_BYTES;
           const uint32_t b_s = a_s + C::A_BYTES;
-          ptx::tmem_cp_128x128b_pair(tmem_meta, ptx::smem_desc(b_s + C::B_MAX, 0, 128, 0));
+          if constexpr (SPARSE) {
+            ptx::tmem_cp_128x128b_pair(tmem_meta, ptx::smem_desc(b_s + C::B_MAX, 0, 128, 0));
 #pragma unroll
-          for (int kb = 0; kb < 4; ++kb) {
-            const uint64_t ad = ptx::smem_desc(a_s + kb * 32, 16, 1024, 2);
-            const uint64_t bd = ptx::smem_desc(b_s + (kb >> 1) * b_box + (kb & 1) * 64, 16, 1024, 2);
-            ptx::mma_sparse_pair(acc, ad, bd, tmem_meta + (kb & ~1), idesc | (uint32_t)(kb & 1), (kt | kb) != 0);
+            for (int kb = 0; kb < 4; ++kb) {
+              const uint64_t ad = ptx::smem_desc(a_s + kb * 32, 16, 1024, 2);
+              const uint64_t bd = ptx::smem_desc(b_s + (kb >> 1) * b_box + (kb & 1) * 64, 16, 1024, 2);
+              ptx::mma_sparse_pair(acc, ad, bd, tmem_meta + (kb & ~1), idesc | (uint32_t)(kb & 1), (kt | kb) != 0);
+            }
+          } else {
+#pragma unroll
+            for (int kb = 0; kb < 8; ++kb) {                                 // K = 16 each: 32 bytes inside a 128-byte row
+              const uint64_t ad = ptx::smem_desc(a_s + (kb >> 2) * 16384 + (kb & 3) * 32, 16, 1024, 2);
+              const uint64_t bd = ptx::smem_desc(b_s + (kb >> 2) * b_box + (kb & 3) * 32, 16, 1024, 2);
+              ptx::mma_dense_pair(acc, ad, bd, idesc, (kt | kb) != 0);
+            }
           }
           ptx::tc_commit_pair(empty_bar(s), 3);
         }
@@ -839,8 +857,55 @@ int launch_spmm_conv(int mode, const uint16_t* vals, const void* hw_meta, const 
   return run_conv_single<128, 3>(vals, a_rows, a_kdim, hw_meta, tok, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
 }
 
+namespace {
+
+// Dense operand, CTA pairs: 256 x N tiles, N the multiple of 32 (at most 256) that wastes the fewest token columns
+// among those with the fewest rounds over the pairs.
+int run_dense_pair_persistent(const uint16_t* A, const uint16_t* Bop, int Mdim, int Ndim, int Kdim, uint16_t* out,
+                              int32_t* status_word, cudaStream_t s) {
+  constexpr int STAGES = 3;
+  using C = PairPCfg<STAGES, false>;
+  CUtensorMap ta, tb;
+  int rc;
+  const int tiles_m = (Mdim + 127) / 128, tiles_k = (Kdim + 127) / 128;
+  const int sms = sm_count();
+  int n_tile = 256;
+  double best = 1e30;
+  for (int n = 256; n >= 160; n -= 32) {
+    const long long tiles = (long long)((tiles_m + 1) / 2) * ((Ndim + n - 1) / n);
+    const long long rounds = (tiles + sms / 2 - 1) / (sms / 2);
+    const double cost = (double)rounds * n * (1.0 + 0.002 * (256 - n));
+    if (cost < best) { best = cost; n_tile = n; }
+  }
+  if ((rc = make_tmap(&ta, A, (uint64_t)Kdim, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, n_tile / 2)) != BIMASK_OK) return rc;
+  auto kern = spmm_pair_persistent_kernel<STAGES, false, false>;
+  if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
+  GemmParams p;
+  p.conv.mode = 0;
+  p.hw_meta = nullptr;
+  p.tiles_k_meta = tiles_k;
+  p.Mdim = Mdim; p.Ndim = Ndim; p.Kdim = Kdim;
+  p.k_tiles_per_split = tiles_k;
+  p.out = out;
+  p.status_word = status_word;
+  p.n_tile = n_tile;
+  p.tiles_m = (tiles_m + 1) / 2;
+  p.tiles_n = (Ndim + n_tile - 1) / n_tile;
+  p.raster_group = 8;
+  const int total = p.tiles_m * p.tiles_n;
+  const int clusters = total < sms / 2 ? total : sms / 2;
+  BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s, ta, tb, ta, p));
+  count_launch();
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+
+}  // namespace
+
 int launch_dense_nt(const uint16_t* A, const uint16_t* Bop, int Mdim, int Ndim, int Kdim, uint16_t* out,
                     int32_t* status_word, cudaStream_t s) {
+  if (Ndim > 128 && Mdim > 128) return run_dense_pair_persistent(A, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   if (Ndim > 128) return run_single<256, 2, false>(A, nullptr, Bop, Mdim, Ndim, Kdim, out, status_word, s);
   return run_single<128, 3, false>(A, nullptr, Bop, Mdim, Ndim, Kdim, out, status_word, s);
 }
