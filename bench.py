@@ -208,9 +208,9 @@ class ClockSampler:
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM kernels on
 # config 5, from the ncu launch list summarised in profiles/cfg5_launch_list.md (GEMM kernel only).
 NCU_TRAFFIC_BYTES = {
-    (5, 0, "wgrad"): 1.245e9 + 0.245e9, (5, 1, "wgrad"): 1.012e9 + 0.245e9,
-    (5, 0, "spmm_fwd"): 0.613e9 + 0.242e9, (5, 1, "spmm_fwd"): 0.703e9 + 0.055e9,
-    (5, 0, "spmm_dgrad"): 0.703e9 + 0.051e9, (5, 1, "spmm_dgrad"): 0.616e9 + 0.243e9,
+    (5, 0, "wgrad"): 1.274e9 + 0.247e9, (5, 1, "wgrad"): 1.003e9 + 0.247e9,
+    (5, 0, "spmm_fwd"): 0.616e9 + 0.239e9, (5, 1, "spmm_fwd"): 0.703e9 + 0.054e9,
+    (5, 0, "spmm_dgrad"): 0.703e9 + 0.051e9, (5, 1, "spmm_dgrad"): 0.620e9 + 0.240e9,
 }
 
 
