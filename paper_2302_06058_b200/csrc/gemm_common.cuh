@@ -30,7 +30,7 @@ struct Cfg {
   static constexpr int META_COLS = SPARSE ? 4 : 0;
   static constexpr int TMEM_COLS = (N_TILE + META_COLS) <= 128 ? 128 : (N_TILE + META_COLS) <= 256 ? 256 : 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */ +
-                                    EPI_WARPS * 2048 /* epilogue staging: one [32 tokens][128 rows] bf16 tile per group of four warps */;
+                                    EPI_WARPS * 4096 /* epilogue staging: two [32 tokens][128 rows] bf16 tiles per group of four warps */;
 };
 
 // A 3x3 convolution as an implicit GEMM: the token operand is an NHWC tensor and a "tile of
@@ -146,7 +146,7 @@ __device__ __forceinline__ void epi_stage(const uint32_t (&r)[W], uint32_t dst) 
 // tensor-memory read each warp arrives once on `release_bar` (0: nobody waits for the accumulator).
 // row_of(c, t) returns where token t of chunk c starts in the result (the CTA's first row), or nullptr when that
 // token lies outside; rows_valid = how many of the CTA's 128 rows exist (a multiple of 32).
-// `stg`: the group's staging tile (W * 256 bytes, 1 KB aligned); `bar_id`: its named barrier.
+// `stg`: the group's two staging tiles (2 x W * 256 bytes, 1 KB aligned); `bar_id`: its named barrier.
 template <int W, typename RowOf>
 __device__ __forceinline__ void drain_chunks(uint32_t acc, int c0, int cstep, int nchunks, bool zero, uint32_t release_bar,
                                              uint32_t stg, uint32_t bar_id, int q, int lane, int rows_valid, RowOf&& row_of) {
@@ -165,17 +165,29 @@ __device__ __forceinline__ void drain_chunks(uint32_t acc, int c0, int cstep, in
   // the next, 16 bytes (eight rows) per lane
   const int unit = lane & 15;
   const bool unit_ok = 8 * unit < rows_valid;
+  uint32_t parity = 0;                                    // which of the group's two tiles this chunk goes through
   auto emit = [&](const uint32_t (&r)[W], int c) {
-    ptx::named_bar_sync(bar_id, 128);                     // the group has read the previous chunk out of the tile
-    epi_stage<W>(r, dst);
+    // Two tiles, one barrier per chunk: a tile is staged again two chunks later, and between the read-back of this
+    // chunk and that staging every warp of the group passes the barrier of the chunk in between.
+    const uint32_t tile = parity * (uint32_t)(W * 256);
+    parity ^= 1u;
+    uint16_t* row[W / 8];                                 // where this lane's tokens go: worked out ahead of the barrier
+#pragma unroll
+    for (int i = 0; i < W / 8; ++i) {
+      uint16_t* r0 = row_of(c, (W / 4) * q + 2 * i + (lane >> 4));
+      row[i] = (r0 != nullptr && unit_ok) ? r0 + 8 * unit : nullptr;
+    }
+    epi_stage<W>(r, dst + tile);
     ptx::named_bar_sync(bar_id, 128);
+    uint4 v[W / 8];
 #pragma unroll
     for (int i = 0; i < W / 8; ++i) {
       const int t = (W / 4) * q + 2 * i + (lane >> 4);
-      const uint4 v = ptx::ld_shared_v4(stg + (uint32_t)t * 256u + (((uint32_t)unit ^ ((uint32_t)t & 7u)) << 4));
-      uint16_t* row = row_of(c, t);
-      if (row != nullptr && unit_ok) *reinterpret_cast<uint4*>(row + 8 * unit) = v;
+      v[i] = ptx::ld_shared_v4(stg + tile + (uint32_t)t * 256u + (((uint32_t)unit ^ ((uint32_t)t & 7u)) << 4));
     }
+#pragma unroll
+    for (int i = 0; i < W / 8; ++i)
+      if (row[i] != nullptr) *reinterpret_cast<uint4*>(row[i]) = v[i];
   };
   uint32_t ra[W], rb[W];
   epi_load<W>(acc + W * c0, ra, zero);

@@ -35,11 +35,11 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - raw);
   const uint32_t staging = base + STAGES * C::STAGE_BYTES;      // epilogue staging, 8 KB per group of four warps
-  const uint32_t bar_base = staging + EPI_WARPS * 2048;
+  const uint32_t bar_base = staging + EPI_WARPS * 4096;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   const uint32_t tmem_full_bar = bar_base + 8u * (2 * STAGES);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * C::STAGE_BYTES + EPI_WARPS * 2048 + 8 * (2 * STAGES + 1));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * C::STAGE_BYTES + EPI_WARPS * 4096 + 8 * (2 * STAGES + 1));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -176,7 +176,7 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     if (ok) {
       uint16_t* outp = reinterpret_cast<uint16_t*>(p.out);
       drain_chunks<32>(tmem_base + ((uint32_t)(32 * q) << 16), eg, EPI_WARPS / 4, N_TILE / 32, num_kt <= 0, 0u,
-                       staging + eg * 8192, 1 + eg, q, lane, p.Mdim - m0, [&](int c, int t) -> uint16_t* {
+                       staging + eg * 16384, 1 + eg, q, lane, p.Mdim - m0, [&](int c, int t) -> uint16_t* {
         if (CONV) {
           // token 32c + t of the box: pixel (cw0 + ., ch0 + .) of image cn0 + .
           const int rr = 32 * c + t;
@@ -219,7 +219,7 @@ struct PairPCfg {
   static constexpr int B_MAX = 32768;                      // up to 128 rows x 128 bf16 (two 64-wide boxes)
   static constexpr int E_BYTES = SPARSE ? 2048 : 0;
   static constexpr int STAGE_BYTES = A_BYTES + B_MAX + E_BYTES;        // 50 KB / 64 KB (the B part is N / 2 rows)
-  static constexpr int STAGING_BYTES = EPI_WARPS * 2048;   // per group of four epilogue warps: one [32 tokens][128 rows] bf16 tile
+  static constexpr int STAGING_BYTES = EPI_WARPS * 4096;   // per group of four epilogue warps: two [32 tokens][128 rows] bf16 tiles
   static constexpr int TMEM_COLS = 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 + 256;
 };
@@ -381,7 +381,7 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
     // one staging tile.
     const int q = warp & 3;
     const int eg = (warp - 2) >> 2;                        // EPI_WARPS / 4 groups of four warps take chunks in turn
-    const uint32_t stg = staging + eg * 8192;
+    const uint32_t stg = staging + eg * 16384;
     uint16_t* outp = reinterpret_cast<uint16_t*>(p.out);
     uint32_t tcount = 0;
     for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++tcount) {
@@ -456,7 +456,7 @@ struct Pair2MCfg {
   static constexpr int B_MAX = 28672;                      // 112 rows x 128 bf16 (two 64-wide boxes), N <= 224
   static constexpr int E_BYTES = 2048;
   static constexpr int STAGE_BYTES = 2 * A_BYTES + B_MAX + 2 * E_BYTES;      // 64 KB
-  static constexpr int STAGING_BYTES = EPI_WARPS * 2048;   // per group of four epilogue warps: one [32 tokens][128 rows] bf16 tile
+  static constexpr int STAGING_BYTES = EPI_WARPS * 4096;   // per group of four epilogue warps: two [32 tokens][128 rows] bf16 tiles
   static constexpr int TMEM_COLS = 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 + 256;
 };
@@ -586,7 +586,7 @@ spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     // tensor-memory lane quadrant, a group shares one staging tile
     const int q = warp & 3;
     const int mt = (warp - 2) >> 2;                        // the group of four warps that drains accumulator mt
-    const uint32_t stg = staging + mt * 8192;
+    const uint32_t stg = staging + mt * 16384;
     uint16_t* outp = reinterpret_cast<uint16_t*>(p.out);
     const uint32_t release_bar = ptx::mapa(tmem_empty_bar, 0);
     uint32_t tcount = 0;
