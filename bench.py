@@ -590,7 +590,9 @@ def run_per_call(args):
                       "note": "fractions of the burst peaks from the cold median"}), flush=True)
 
 
-CONV_LAYERS = [(56, 56, 64, 64), (28, 28, 128, 128), (14, 14, 256, 256), (7, 7, 512, 512)]   # ResNet-50's 3x3 convolutions
+# ResNet-50's 3x3 convolutions (H, W, C, I, stride): the stride-1 layers of the four stages, then the three down-sampling ones
+CONV_LAYERS = [(56, 56, 64, 64, 1), (28, 28, 128, 128, 1), (14, 14, 256, 256, 1), (7, 7, 512, 512, 1),
+               (56, 56, 128, 128, 2), (28, 28, 256, 256, 2), (14, 14, 512, 512, 2)]
 
 
 def run_conv(args):
@@ -604,18 +606,19 @@ def run_conv(args):
     N, M, P, NB = 2, 4, 100, args.conv_batch
     gen = torch.Generator(device="cuda").manual_seed(7)
     rows = []
-    for (H, W, C, I) in CONV_LAYERS:
-        T, J = NB * H * W, 9 * C
+    for (H, W, C, I, stride) in CONV_LAYERS:
+        Ho, Wo = (H - 1) // stride + 1, (W - 1) // stride + 1
+        T, J = NB * Ho * Wo, 9 * C
         b = bm.alloc_layer_buffers(T, I, J, P)
         b["W"] = torch.randn(I, J, device="cuda", generator=gen) * (2.0 / J) ** 0.5
         b["X"] = torch.randn(NB, H, W, C, device="cuda", generator=gen).bfloat16()
-        b["dY"] = torch.randn(NB, H, W, I, device="cuda", generator=gen).bfloat16()
+        b["dY"] = torch.randn(NB, Ho, Wo, I, device="cuda", generator=gen).bfloat16()
         b["dX"] = torch.empty(NB, H, W, C, dtype=torch.bfloat16, device="cuda")
-        b["ws"] = torch.empty(bm.bimask_conv_workspace_bytes(NB, H, W, C, I, P), dtype=torch.uint8, device="cuda")
+        b["ws"] = torch.empty(bm.bimask_conv_workspace_bytes(NB, H, W, C, I, P, stride), dtype=torch.uint8, device="cuda")
         largs = bm.make_layer_args(T, I, J, N, M, P, 43, True, b)
-        row = {"layer": [NB, H, W, C, I]}
-        for name, mode in (("explicit", 1), ("auto", 0)):
-            ca = bm.make_conv_args(largs, NB, H, W, C, mode)
+        row = {"layer": [NB, H, W, C, I], "stride": stride}
+        for name, mode in (("explicit", 1), ("auto", 0), ("implicit", 2)):
+            ca = bm.make_conv_args(largs, NB, H, W, C, mode, stride)
             n0 = bm.bimask_launch_count()
             for _ in range(max(args.warmup, 3)):
                 bm.bimask_conv_layer_step(ca)

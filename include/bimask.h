@@ -265,9 +265,10 @@ int bimask_train_step(const bimask_train_args* args);
  * patches with 4-D tensor loads (out-of-image pixels read as zero); BIMASK_CONV_AUTO takes the
  * implicit form for every product whose shape allows it (C % 64 == 0; the input gradient needs
  * C == 64 or C % 128 == 0; patterns with a 2:4 form) when the column matrix would
- * exceed 16 MiB, and the explicit form otherwise.  IMPLICIT with a shape that does not allow it
- * returns BIMASK_EUNSUPPORTED; so does stride 2, for which only the explicit form is built (AUTO
- * takes it).  C % 32 == 0 and I % 32 == 0 always.  The two forms round the
+ * exceed 16 MiB and an output image has more than 64 pixels, and the explicit form otherwise.  With stride 2 the forward product and the
+ * weight gradient have an implicit form (the tensor loads take every second pixel), the input
+ * gradient always takes the explicit one.  IMPLICIT with a shape that does not allow it returns
+ * BIMASK_EUNSUPPORTED.  C % 32 == 0 and I % 32 == 0 always.  The two forms round the
  * input gradient differently (explicit: nine bf16 partial results summed in fp32; implicit: one
  * fp32 accumulation), both within the products' tolerance. */
 enum { BIMASK_CONV_AUTO = 0, BIMASK_CONV_EXPLICIT = 1, BIMASK_CONV_IMPLICIT = 2 };

@@ -404,7 +404,8 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
     if (pack && !fused && (rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, s))) return rc;
   }
   if (conv && conv->imp_fwd)
-    rc = launch_spmm_conv(1, a->vals_f, a->hw_meta_f, a->X, conv->NB, conv->H, conv->W, conv->C, a->I, a->Y, a->status_word, s);
+    rc = launch_spmm_conv(1, a->vals_f, a->hw_meta_f, a->X, conv->NB, conv->H, conv->W, conv->C, a->I, conv->stride, a->Y,
+                          a->status_word, s);
   else if (pack) rc = launch_spmm(a->vals_f, a->hw_meta_f, Xmat, a->I, a->T, a->J, a->Y, a->status_word, s);
   else rc = launch_dense_nt(a->vals_f, Xmat, a->I, a->T, a->J, a->Y, a->status_word, s);
   if (rc) return rc;
@@ -435,14 +436,15 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
   if (pack && !fused && (rc = launch_hw_meta(a->meta_b, a->J, a->I, a->hw_meta_b, s))) return rc;
   if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, s))) return rc;
   if (conv && conv->imp_dgrad)
-    rc = launch_spmm_conv(2, a->vals_b, a->hw_meta_b, dYp, conv->NB, conv->H, conv->W, conv->C, a->I, a->dX, a->status_word, s);
+    rc = launch_spmm_conv(2, a->vals_b, a->hw_meta_b, dYp, conv->NB, conv->H, conv->W, conv->C, a->I, 1, a->dX, a->status_word, s);
   else if (pack) rc = launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, dXmat, a->status_word, s);
   else rc = launch_dense_nt(a->vals_b, dYp, a->J, a->T, a->I, dXmat, a->status_word, s);
   if (rc) return rc;
   if (conv && !conv->imp_dgrad)
     if ((rc = launch_col2im3x3(dXmat, conv->NB, conv->H, conv->W, conv->C, conv->stride, a->dX, s))) return rc;
   if (conv && conv->imp_wgrad)
-    return launch_wgrad_conv(a->dY, a->X, conv->NB, conv->H, conv->W, conv->C, a->I, a->dW, conv->wpart, a->status_word, s);
+    return launch_wgrad_conv(a->dY, a->X, conv->NB, conv->H, conv->W, conv->C, a->I, conv->stride, a->dW, conv->wpart,
+                             a->status_word, s);
   return launch_wgrad_impl(a->dY, Xmat, a->T, a->I, a->J, a->dW, partials, a->status_word, s);
 }
 
@@ -450,9 +452,9 @@ extern "C" {
 
 int bimask_layer_step(const bimask_layer_args* a) { return layer_step_impl(a, false); }
 
-static size_t conv_wpart_bytes(int NB, int H, int W, int C, int I) {
+static size_t conv_wpart_bytes(int NB, int H, int W, int C, int I, int stride) {
   int splits = 1, per = 0;
-  wgrad_conv_plan(NB, H, W, C, I, &splits, &per);
+  wgrad_conv_plan(NB, H, W, C, I, stride, &splits, &per);
   return splits > 1 ? align_up((size_t)splits * I * 9 * C * sizeof(float), 256) : 0;
 }
 
@@ -462,7 +464,7 @@ size_t bimask_conv_workspace_bytes(int NB, int H, int W, int C, int I, int P, in
   if (T > 0x7FFFFFFFll || 9ll * C > 0x7FFFFFFFll) return 0;
   const size_t col = align_up((size_t)T * 9 * C * 2, 256);
   // linear-layer scratch + column matrix + column-space gradient + partial sums of the implicit weight gradient
-  return plan_ws((int)T, I, 9 * C, P).total + 2 * col + (stride == 1 ? conv_wpart_bytes(NB, H, W, C, I) : 0);
+  return plan_ws((int)T, I, 9 * C, P).total + 2 * col + conv_wpart_bytes(NB, H, W, C, I, stride);
 }
 
 int bimask_conv_layer_step(const bimask_conv_args* c) {
@@ -485,23 +487,28 @@ int bimask_conv_layer_step(const bimask_conv_args* c) {
                  a->ws_bytes, need);
   ConvPlan plan;
   plan.NB = c->NB; plan.H = c->H; plan.W = c->W; plan.C = c->C; plan.stride = c->stride;
-  const bool packs = a->N <= 2, unit = c->stride == 1;          // the implicit form is built for stride 1
-  const bool can_fwd = unit && packs && c->C % 64 == 0;
+  // the forward product and the weight gradient have an implicit form for both strides (strided tensor-map
+  // traversal), the input gradient for stride 1 only: with stride 2 it always takes the explicit form
+  const bool packs = a->N <= 2, unit = c->stride == 1;
+  const bool can_fwd = packs && c->C % 64 == 0;
   const bool can_dgrad = unit && packs && (c->C % 128 == 0 || c->C == 64);
-  const bool can_wgrad = unit && c->C % 64 == 0;
-  BIMASK_REQUIRE(c->mode != BIMASK_CONV_IMPLICIT || (can_fwd && can_dgrad && can_wgrad), BIMASK_EUNSUPPORTED,
-                 "bimask_conv_layer_step: the implicit form needs stride 1, C = 64 or a multiple of 128, and a pattern with "
-                 "a 2:4 form (stride %d, C = %d, I = %d, N:M = %d:%d)", c->stride, c->C, a->I, a->N, a->M);
+  const bool can_wgrad = c->C % 64 == 0;
+  BIMASK_REQUIRE(c->mode != BIMASK_CONV_IMPLICIT || (can_fwd && can_wgrad && (can_dgrad || !unit)), BIMASK_EUNSUPPORTED,
+                 "bimask_conv_layer_step: the implicit form needs C = 64 or a multiple of 128 (a multiple of 64 with stride 2) "
+                 "and a pattern with a 2:4 form (stride %d, C = %d, I = %d, N:M = %d:%d)", c->stride, c->C, a->I, a->N, a->M);
   // AUTO: a column matrix that fits comfortably in L2 costs little, and the explicit form then has
   // fewer, denser k tiles (measured: 7x7 images of 512 channels are faster explicit, 14x14 of 256
   // channels faster implicit); above 16 MiB the implicit form wins by the HBM traffic it avoids.
+  // Images of at most 8 x 8 output pixels leave a quarter of every pixel box empty, more than the unfold and fold
+  // passes cost (measured at batch 256, 7x7 x 512 channels: 256 us explicit, 295 us implicit).
   const bool small_cols = (size_t)T * 9 * c->C * 2 < ((size_t)16 << 20);
-  const bool implicit = c->mode == BIMASK_CONV_IMPLICIT || (c->mode == BIMASK_CONV_AUTO && !small_cols);
+  const bool small_image = T / c->NB <= 64;
+  const bool implicit = c->mode == BIMASK_CONV_IMPLICIT || (c->mode == BIMASK_CONV_AUTO && !small_cols && !small_image);
   plan.imp_fwd = implicit && can_fwd;
   plan.imp_dgrad = implicit && can_dgrad;
   plan.imp_wgrad = implicit && can_wgrad;
   const size_t col = align_up((size_t)T * 9 * c->C * 2, 256);
-  const size_t wpart = unit ? conv_wpart_bytes(c->NB, c->H, c->W, c->C, a->I) : 0;
+  const size_t wpart = conv_wpart_bytes(c->NB, c->H, c->W, c->C, a->I, c->stride);
   uint8_t* tail = reinterpret_cast<uint8_t*>(a->ws) + (need - 2 * col - wpart);
   plan.xcol = reinterpret_cast<uint16_t*>(tail);
   plan.dxcol = reinterpret_cast<uint16_t*>(tail + col);

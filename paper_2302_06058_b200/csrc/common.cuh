@@ -110,12 +110,13 @@ int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, 
                 uint16_t* out, int32_t* status_word, cudaStream_t s);
 // 3x3 convolution products on shifted pixel boxes (no column matrix): mode 1 forward (tok = x, out = y with I
 // channels), mode 2 input gradient (tok = permuted dy, out = dx with C channels); NHWC bf16 throughout.
+// H x W is the INPUT image; stride 2 (forward only) gives an output of ((H-1)/2+1) x ((W-1)/2+1) pixels.
 int launch_spmm_conv(int mode, const uint16_t* vals, const void* hw_meta, const uint16_t* tok, int NB, int H, int W, int C,
-                     int I, uint16_t* out, int32_t* status_word, cudaStream_t s);
+                     int I, int stride, uint16_t* out, int32_t* status_word, cudaStream_t s);
 // Dense weight gradient of the 3x3 convolution on shifted pixel boxes; partials as sized by wgrad_conv_plan.
-void wgrad_conv_plan(int NB, int H, int W, int C, int I, int* splits, int* k_tiles_per_split);
-int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int W, int C, int I, float* dW, float* partials,
-                      int32_t* status_word, cudaStream_t s);
+void wgrad_conv_plan(int NB, int H, int W, int C, int I, int stride, int* splits, int* k_tiles_per_split);
+int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int W, int C, int I, int stride, float* dW,
+                      float* partials, int32_t* status_word, cudaStream_t s);
 // Dense product for masked operands that do not fit the 2:4 format: out[n][m] = sum_k A[m][k] B[n][k],
 // A bf16 [Mdim][Kdim], B bf16 [Ndim][Kdim], out bf16 [Ndim][Mdim] (same roles as launch_spmm).
 int launch_dense_nt(const uint16_t* A, const uint16_t* Bop, int Mdim, int Ndim, int Kdim, uint16_t* out,

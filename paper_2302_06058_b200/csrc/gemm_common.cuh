@@ -41,7 +41,9 @@ struct Cfg {
 //           the 2:4 operand for tap (kh, kw) are (kh*3+kw)*C + c.
 struct ConvGeom {
   int mode;                 // 0: plain matrix operand
-  int H, W, NB;             // image
+  int H, W, NB;             // grid of the tokens (the convolution's OUTPUT pixels)
+  int stride;               // mode 1 / weight gradient: input pixel of output pixel (h, w), tap (kh, kw) is
+                            // (stride * h + kh - 1, stride * w + kw - 1); the input tensor map strides by it
   int CB;                   // channels of the token operand (x: C; dy: I)
   int wb, hb, nb;           // pixel box of one load: wb * hb * nb tokens (powers of two)
   int lg_wb, lg_hb;         // their logarithms
@@ -212,7 +214,8 @@ int make_tmap(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, u
 // The metadata image as a 2-D tensor of u32: 256 words per row, two rows per 2048-byte block.
 int make_tmap_meta(CUtensorMap* m, const void* ptr, uint64_t blocks);
 // 4-D bf16 map of an NHWC tensor (channels, W, H, NB) for loads of 64-channel pixel boxes, 128-byte swizzle.
-int make_tmap_nhwc_load(CUtensorMap* m, const void* ptr, int CH, int W, int H, int NB, int wb, int hb, int nb);
+// estride 2: a box takes every second pixel along W and H (wb x hb pixels all the same).
+int make_tmap_nhwc_load(CUtensorMap* m, const void* ptr, int CH, int W, int H, int NB, int wb, int hb, int nb, int estride = 1);
 
 // The dynamic shared-memory limit of a kernel is set once per (device, kernel): the call costs a microsecond or two
 // on the host, which a layer step of ten short launches would notice.  A kernel is always launched with the same size.

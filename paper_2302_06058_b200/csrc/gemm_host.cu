@@ -163,10 +163,11 @@ struct TmapKey {
   // densely packed (stride of H = W * stride, of NB = H * W * stride)
   uint64_t d2 = 0, d3 = 0;
   uint32_t box2 = 0, box3 = 0;
+  uint32_t estride = 1;     // rank 4: traversal stride along W and H (the box spans estride * box pixels, takes `box`)
   bool operator==(const TmapKey& o) const {
     return ptr == o.ptr && inner == o.inner && outer == o.outer && stride == o.stride && box_inner == o.box_inner &&
            box_outer == o.box_outer && dtype == o.dtype && swizzle == o.swizzle && d2 == o.d2 && d3 == o.d3 &&
-           box2 == o.box2 && box3 == o.box3;
+           box2 == o.box2 && box3 == o.box3 && estride == o.estride;
   }
 };
 
@@ -182,8 +183,9 @@ int encode_cached(CUtensorMap* m, const TmapKey& key) {
   BIMASK_REQUIRE(fn != nullptr, BIMASK_ECUDA, "cuTensorMapEncodeTiled entry point not available");
   cuuint64_t dims[4] = {key.inner, key.outer, key.d2, key.d3};
   cuuint64_t strides[3] = {key.stride, key.stride * key.outer, key.stride * key.outer * key.d2};
-  cuuint32_t box[4] = {key.box_inner, key.box_outer, key.box2, key.box3};
-  cuuint32_t estr[4] = {1, 1, 1, 1};
+  const cuuint32_t es = key.d2 ? key.estride : 1u;
+  cuuint32_t box[4] = {key.box_inner, key.box_outer * es, key.box2 * es, key.box3};
+  cuuint32_t estr[4] = {1, es, es, 1};
   CUresult r = fn(m, (CUtensorMapDataType)key.dtype, key.d2 ? 4 : 2, const_cast<void*>(key.ptr), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, (CUtensorMapSwizzle)key.swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -220,10 +222,11 @@ int make_tmap_meta(CUtensorMap* m, const void* ptr, uint64_t blocks) {
 }
 
 // 4-D bf16 map of an NHWC tensor (channels, W, H, NB) for loads of 64-channel pixel boxes, 128-byte swizzle.
-int make_tmap_nhwc_load(CUtensorMap* m, const void* ptr, int CH, int W, int H, int NB, int wb, int hb, int nb) {
+int make_tmap_nhwc_load(CUtensorMap* m, const void* ptr, int CH, int W, int H, int NB, int wb, int hb, int nb, int estride) {
   TmapKey k{ptr, (uint64_t)CH, (uint64_t)W, (uint64_t)CH * 2, 64, (uint32_t)wb, (int)CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
             (int)CU_TENSOR_MAP_SWIZZLE_128B};
   k.d2 = (uint64_t)H; k.d3 = (uint64_t)NB; k.box2 = (uint32_t)hb; k.box3 = (uint32_t)nb;
+  k.estride = (uint32_t)estride;
   return encode_cached(m, k);
 }
 

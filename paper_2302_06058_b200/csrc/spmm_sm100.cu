@@ -102,7 +102,7 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
             int c0, dw, dh;
             bool valid;
             conv_k_coords(p.conv, kt, q, p.Kdim, c0, dw, dh, valid);
-            ptx::tma_load_4d(b_s + q * (N_TILE * 128), &tmapB, valid ? c0 : 0, cw0 + dw, ch0 + dh, valid ? cn0 : p.conv.NB,
+            ptx::tma_load_4d(b_s + q * (N_TILE * 128), &tmapB, valid ? c0 : 0, p.conv.stride * cw0 + dw, p.conv.stride * ch0 + dh, valid ? cn0 : p.conv.NB,
                              full_bar(s));
           }
           {
@@ -320,7 +320,7 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
               int c0, dw, dh;
               bool valid;
               conv_k_coords(p.conv, kt, q, p.Kdim, c0, dw, dh, valid);
-              ptx::tma_load_4d_pair(b_s + q * b_box, &tmapB, valid ? c0 : 0, cw0 + dw, ch0 + dh, valid ? cn0 : p.conv.NB, bar);
+              ptx::tma_load_4d_pair(b_s + q * b_box, &tmapB, valid ? c0 : 0, p.conv.stride * cw0 + dw, p.conv.stride * ch0 + dh, valid ? cn0 : p.conv.NB, bar);
             }
             ptx::tma_load_2d_pair(b_s + C::B_MAX, &tmapE, 0, 2 * (meta_row * p.tiles_k_meta + meta_kt), bar);
             continue;
@@ -766,14 +766,14 @@ int launch_spmm(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, 
 namespace {
 
 template <int N_TILE, int STAGES>
-int run_conv_single(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_meta, const uint16_t* tok, ConvGeom g,
+int run_conv_single(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_meta, const uint16_t* tok, int in_h, int in_w, ConvGeom g,
                     int Mdim, int Kdim, int tiles_k_meta, uint16_t* out, int32_t* status_word, cudaStream_t s) {
   using C = Cfg<N_TILE, STAGES, true>;
   conv_boxes(g, N_TILE);
   CUtensorMap ta, tb;
   int rc;
   if ((rc = make_tmap(&ta, vals, (uint64_t)a_kdim / 2, (uint64_t)a_rows, 128)) != BIMASK_OK) return rc;
-  if ((rc = make_tmap_nhwc_load(&tb, tok, g.CB, g.W, g.H, g.NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_nhwc_load(&tb, tok, g.CB, in_w, in_h, g.NB, g.wb, g.hb, g.nb, g.stride)) != BIMASK_OK) return rc;
   auto kern = spmm_single_kernel<N_TILE, STAGES, true, true>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
@@ -795,7 +795,7 @@ int run_conv_single(const uint16_t* vals, int a_rows, int a_kdim, const void* hw
   return BIMASK_OK;
 }
 
-int run_conv_pair(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_meta, const uint16_t* tok, ConvGeom g,
+int run_conv_pair(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_meta, const uint16_t* tok, int in_h, int in_w, ConvGeom g,
                   int Mdim, int Kdim, int tiles_k_meta, uint16_t* out, int32_t* status_word, cudaStream_t s) {
   constexpr int STAGES = 3;
   using C = PairPCfg<STAGES>;
@@ -806,7 +806,7 @@ int run_conv_pair(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_m
   const int a_tiles_m = (a_rows + 127) / 128;
   const int sms = sm_count();
   if ((rc = make_tmap(&ta, vals, (uint64_t)a_kdim / 2, (uint64_t)a_rows, 128)) != BIMASK_OK) return rc;
-  if ((rc = make_tmap_nhwc_load(&tb, tok, g.CB, g.W, g.H, g.NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_nhwc_load(&tb, tok, g.CB, in_w, in_h, g.NB, g.wb, g.hb, g.nb, g.stride)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_meta(&te, hw_meta, (uint64_t)a_tiles_m * tiles_k_meta)) != BIMASK_OK) return rc;
   auto kern = spmm_pair_persistent_kernel<STAGES, true>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
@@ -838,23 +838,26 @@ int run_conv_pair(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_m
 //   input gradient: D[c, pixel] = sum_{tap, i'} A'[tap*C + c, i'] dyp[pixel - tap, i'];  vals/hw_meta of the 9C x I operand
 // out is NHWC with Mdim channels.  Needs C % 64 == 0 (forward); C % 128 == 0 or C == 64 (input gradient).
 int launch_spmm_conv(int mode, const uint16_t* vals, const void* hw_meta, const uint16_t* tok, int NB, int H, int W, int C,
-                     int I, uint16_t* out, int32_t* status_word, cudaStream_t s) {
+                     int I, int stride, uint16_t* out, int32_t* status_word, cudaStream_t s) {
   ConvGeom g{};
-  g.mode = mode; g.H = H; g.W = W; g.NB = NB;
-  const long long T = (long long)NB * H * W;
+  // the tokens are the output pixels; with stride 2 (forward only) the input tensor is H x W, the output Ho x Wo
+  g.mode = mode; g.NB = NB; g.stride = stride;
+  g.H = (H - 1) / stride + 1; g.W = (W - 1) / stride + 1;
+  const long long T = (long long)NB * g.H * g.W;
   int Mdim, Kdim, a_rows, a_kdim, tiles_k_meta;
   if (mode == 1) {
     g.CB = C; g.kt_per_tap = 0; g.rows_per_tap = 0;
     Mdim = I; Kdim = 9 * C; a_rows = I; a_kdim = 9 * C; tiles_k_meta = (9 * C + 127) / 128;
   } else {
+    BIMASK_REQUIRE(stride == 1, BIMASK_EUNSUPPORTED, "implicit input gradient: stride %d", stride);
     g.CB = I; g.kt_per_tap = (I + 127) / 128; g.rows_per_tap = C;
     Mdim = C; Kdim = 9 * g.kt_per_tap * 128; a_rows = 9 * C; a_kdim = I; tiles_k_meta = g.kt_per_tap;
   }
   if (Mdim > 128 && T > 128)
-    return run_conv_pair(vals, a_rows, a_kdim, hw_meta, tok, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
+    return run_conv_pair(vals, a_rows, a_kdim, hw_meta, tok, H, W, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
   if (T > 128)
-    return run_conv_single<256, 2>(vals, a_rows, a_kdim, hw_meta, tok, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
-  return run_conv_single<128, 3>(vals, a_rows, a_kdim, hw_meta, tok, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
+    return run_conv_single<256, 2>(vals, a_rows, a_kdim, hw_meta, tok, H, W, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
+  return run_conv_single<128, 3>(vals, a_rows, a_kdim, hw_meta, tok, H, W, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
 }
 
 namespace {

@@ -113,8 +113,8 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_consta
               const int j = n0 + 128 * (int)rank + 64 * q;           // first of 64 columns of dW: one tap, 64 channels
               const bool valid = j < p.Ndim;
               const int tap = j / p.conv.CB;
-              ptx::tma_load_4d_pair(b_s + q * 8192, &tmapB, valid ? j - tap * p.conv.CB : 0, cw0 + tap % 3 - 1,
-                                    ch0 + tap / 3 - 1, valid ? cn0 : p.conv.NB, bar);
+              ptx::tma_load_4d_pair(b_s + q * 8192, &tmapB, valid ? j - tap * p.conv.CB : 0, p.conv.stride * cw0 + tap % 3 - 1,
+                                    p.conv.stride * ch0 + tap / 3 - 1, valid ? cn0 : p.conv.NB, bar);
             }
             continue;
           }
@@ -294,7 +294,7 @@ wgrad_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_cons
               const int j = n0 + 64 * q;                   // first of 64 columns of dW: one tap, 64 channels
               const bool valid = j < p.Ndim;
               const int tap = j / p.conv.CB;
-              ptx::tma_load_4d(b_s + q * 8192, &tmapB, valid ? j - tap * p.conv.CB : 0, cw0 + tap % 3 - 1, ch0 + tap / 3 - 1,
+              ptx::tma_load_4d(b_s + q * 8192, &tmapB, valid ? j - tap * p.conv.CB : 0, p.conv.stride * cw0 + tap % 3 - 1, p.conv.stride * ch0 + tap / 3 - 1,
                                valid ? cn0 : p.conv.NB, full_bar(s));
             }
             continue;
@@ -466,23 +466,25 @@ static void wgrad_plan_k(int k_tiles, int I, int J, int* splits, int* k_tiles_pe
 }
 
 // The same for the implicit convolution: one k tile per 64-pixel box.
-static ConvGeom conv_wgrad_geom(int NB, int H, int W, int C) {
+// H, W: the input image; the k tiles are boxes of OUTPUT pixels.
+static ConvGeom conv_wgrad_geom(int NB, int H, int W, int C, int stride) {
   ConvGeom g{};
-  g.mode = 1; g.H = H; g.W = W; g.NB = NB; g.CB = C;
+  g.mode = 1; g.NB = NB; g.CB = C; g.stride = stride;
+  g.H = (H - 1) / stride + 1; g.W = (W - 1) / stride + 1;
   conv_boxes(g, 64);
   return g;
 }
 
-void wgrad_conv_plan(int NB, int H, int W, int C, int I, int* splits, int* k_tiles_per_split) {
-  const ConvGeom g = conv_wgrad_geom(NB, H, W, C);
+void wgrad_conv_plan(int NB, int H, int W, int C, int I, int stride, int* splits, int* k_tiles_per_split) {
+  const ConvGeom g = conv_wgrad_geom(NB, H, W, C, stride);
   wgrad_plan_k(g.tiles_w * g.tiles_h * ((NB + g.nb - 1) / g.nb), I, 9 * C, splits, k_tiles_per_split);
 }
 
-// dW[i, tap*C + c] = sum over pixels of dy[pixel, i] x[pixel + tap, c] without a column matrix (C % 64 == 0).
-// partials: splits * I * 9C floats when wgrad_conv_plan gives more than one split.
-int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int W, int C, int I, float* dW, float* partials,
-                      int32_t* status_word, cudaStream_t s) {
-  const ConvGeom g = conv_wgrad_geom(NB, H, W, C);
+// dW[i, tap*C + c] = sum over output pixels of dy[pixel, i] x[stride * pixel + tap, c] without a column matrix
+// (C % 64 == 0).  partials: splits * I * 9C floats when wgrad_conv_plan gives more than one split.
+int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int W, int C, int I, int stride, float* dW,
+                      float* partials, int32_t* status_word, cudaStream_t s) {
+  const ConvGeom g = conv_wgrad_geom(NB, H, W, C, stride);
   const int boxes = g.tiles_w * g.tiles_h * ((NB + g.nb - 1) / g.nb);
   const int J = 9 * C;
   int splits, per;
@@ -491,8 +493,8 @@ int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int 
   using Cf = WgradCfg<STAGES>;
   CUtensorMap ta, tb;
   int rc;
-  if ((rc = make_tmap_nhwc_load(&ta, dy, I, W, H, NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
-  if ((rc = make_tmap_nhwc_load(&tb, x, C, W, H, NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_nhwc_load(&ta, dy, I, g.W, g.H, NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_nhwc_load(&tb, x, C, W, H, NB, g.wb, g.hb, g.nb, stride)) != BIMASK_OK) return rc;
   GemmParams p;
   p.conv = g;
   p.hw_meta = nullptr; p.tiles_k_meta = 0;
