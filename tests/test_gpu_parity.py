@@ -511,3 +511,42 @@ def test_back_to_back_steps_on_reused_buffers(I, J, T):
         assert np.array_equal(u32(got["meta_b"]), ref["meta_b"])
         for n in ("Y", "dX", "dW"):
             assert rel_err(got[n].float().cpu().numpy(), ref[n]) <= TOL, (k, n)
+
+
+def _random_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(n):
+        I = 32 * int(rng.integers(1, 41))                 # 32 .. 1280
+        J = 32 * int(rng.integers(1, 41))
+        T = int(rng.integers(1, 2600))
+        NM = [(2, 4), (1, 4), (2, 8), (1, 16), (4, 8)][int(rng.integers(0, 5))]
+        out.append((I, J, T) + NM)
+    return out
+
+
+@pytest.mark.parametrize("I,J,T,N,M", _random_shapes(16, 20240607))
+def test_layer_step_parity_on_drawn_shapes(I, J, T, N, M):
+    """Shapes drawn at random (seeded): every kernel choice the dispatchers make below the large-operand kernels,
+    ragged tiles in all three dimensions, packed and dense operands."""
+    if J % M or I % M:
+        J, I = J + (-J) % 64, I + (-I) % 64
+    W = inputs.make_weight(I, J, I + 3 * J)
+    X = inputs.make_activation(T, J, T + I)
+    dY = inputs.make_activation(T, I, T + J)
+    P, seed = 5, 77 + T
+    b = run_layer_step(W, X, dY, N, M, P, seed, do_search=True) if N <= 2 else None
+    if b is None:                                         # dense masked operands (no 2:4 form)
+        b = bm.alloc_layer_buffers(T, I, J, P, dense=True)
+        b["W"], b["X"], b["dY"] = dev(W), bits_dev(X), bits_dev(dY)
+        b["meta_f"] = b["hw_meta_f"] = b["meta_b"] = b["hw_meta_b"] = None
+        bm.bimask_layer_step(bm.make_layer_args(T, I, J, N, M, P, seed, True, b))
+        torch.cuda.synchronize()
+    ref = O.layer_step(W, X, dY, N, M, P, seed, do_search=True)
+    assert int(b["status_word"].item()) == 0
+    assert np.array_equal(u32(b["maskbits_f"]), O.pack_bits(ref["B"]))
+    assert np.array_equal(b["counts"].cpu().numpy(), ref["counts"])
+    assert np.array_equal(b["perm"].cpu().numpy(), ref["perm"])
+    assert np.array_equal(u32(b["maskbits_b"]), O.pack_bits(ref["Bbar_p"]))
+    for n in ("Y", "dX", "dW"):
+        assert rel_err(b[n].float().cpu().numpy(), ref[n]) <= TOL, n
