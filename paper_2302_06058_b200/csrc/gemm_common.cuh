@@ -109,10 +109,10 @@ __device__ __forceinline__ void raster(int id, int tiles_m, int tiles_n, int gro
 // stored token-major, so a chunk of W tokens x the CTA's 128 rows is transposed on its way out by a GROUP of four
 // warps, one per tensor-memory lane quadrant:
 //   tensor memory -> registers in the accumulator-fragment layout (two 16-lane loads per warp) -> bf16 pairs ->
-//   stmatrix.trans into the group's staging tile [token][128 rows] (256-byte rows; the 16-byte unit index is
-//   XOR-ed with the token index mod 8, so the eight rows of a matrix fall into eight different bank groups) ->
-//   named barrier -> each warp reads W/4 whole token rows back and writes them with 16-byte stores, 256 contiguous
-//   bytes per token (whole 128-byte lines: half-line writes were bound by the number of write requests).
+//   stmatrix.trans into one of the group's two staging tiles [token][128 rows] (256-byte rows; the 16-byte unit
+//   index is XOR-ed with the token index mod 8, so the eight rows of a matrix fall into eight different bank
+//   groups) -> named barrier -> each warp reads W/4 whole token rows back and writes them with 16-byte stores,
+//   256 contiguous bytes per token (whole 128-byte lines).
 // The tensor-memory load of the next chunk is issued before the current one is converted and stored.
 template <int W>
 __device__ __forceinline__ void epi_load(uint32_t taddr, uint32_t (&r)[W], bool zero) {
@@ -148,7 +148,9 @@ __device__ __forceinline__ void epi_stage(const uint32_t (&r)[W], uint32_t dst) 
 // tensor-memory read each warp arrives once on `release_bar` (0: nobody waits for the accumulator).
 // row_of(c, t) returns where token t of chunk c starts in the result (the CTA's first row), or nullptr when that
 // token lies outside; rows_valid = how many of the CTA's 128 rows exist (a multiple of 32).
-// `stg`: the group's two staging tiles (2 x W * 256 bytes, 1 KB aligned); `bar_id`: its named barrier.
+// `stg`: the group's two staging tiles (2 x W * 256 bytes, 1 KB aligned); `bar_id`: its named barrier.  Every call
+// starts with the first tile: the callers synchronise the group between two calls (the barrier on which the group
+// agrees that the next accumulator is ready), so the last read-back of one call is over before the next one stages.
 template <int W, typename RowOf>
 __device__ __forceinline__ void drain_chunks(uint32_t acc, int c0, int cstep, int nchunks, bool zero, uint32_t release_bar,
                                              uint32_t stg, uint32_t bar_id, int q, int lane, int rows_valid, RowOf&& row_of) {
