@@ -550,3 +550,35 @@ def test_layer_step_parity_on_drawn_shapes(I, J, T, N, M):
     assert np.array_equal(u32(b["maskbits_b"]), O.pack_bits(ref["Bbar_p"]))
     for n in ("Y", "dX", "dW"):
         assert rel_err(b[n].float().cpu().numpy(), ref[n]) <= TOL, n
+
+
+def test_layer_step_captured_in_a_cuda_graph():
+    """The entry points enqueue kernels only (programmatic dependent launches included), so a step can be captured
+    once and replayed: the replay on new contents of the same buffers must give that input's results."""
+    I, J, T, N, M, P = 256, 384, 700, 2, 4, 6
+    sets = [(inputs.make_weight(I, J, 600 + k), inputs.make_activation(T, J, 610 + k), inputs.make_activation(T, I, 620 + k))
+            for k in range(2)]
+    b = bm.alloc_layer_buffers(T, I, J, P)
+    b["W"], b["X"], b["dY"] = dev(sets[0][0]), bits_dev(sets[0][1]), bits_dev(sets[0][2])
+    args = bm.make_layer_args(T, I, J, N, M, P, 9, True, b)
+    bm.bimask_layer_step(args)                            # first call: kernel attributes and tensor maps
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        args.stream = torch.cuda.current_stream().cuda_stream
+        bm.bimask_layer_step(args)
+    for k in (1, 0, 1):
+        b["W"].copy_(dev(sets[k][0])); b["X"].copy_(bits_dev(sets[k][1])); b["dY"].copy_(bits_dev(sets[k][2]))
+        graph.replay()
+    torch.cuda.synchronize()
+    ref = O.layer_step(sets[1][0], sets[1][1], sets[1][2], N, M, P, 9)
+    assert int(b["status_word"].item()) == 0
+    assert np.array_equal(u32(b["maskbits_f"]), ref["maskbits_f"])
+    assert np.array_equal(b["counts"].cpu().numpy(), ref["counts"])
+    assert np.array_equal(b["perm"].cpu().numpy(), ref["perm"])
+    assert np.array_equal(u32(b["maskbits_b"]), ref["maskbits_b"])
+    assert np.array_equal(u16(b["vals_b"]), ref["vals_b"])
+    for n in ("Y", "dX", "dW"):
+        assert rel_err(b[n].float().cpu().numpy(), ref[n]) <= TOL, n
