@@ -108,13 +108,17 @@ fwd_mask_generic_kernel(const float4* __restrict__ W4, long long nblocks, int N,
     const uint32_t kb = keep_block<M>(key, (M == 16 ? 0xFFFFu : 0xFFu), N);
     uint32_t codes = 0;
     if (MODE == 1) {
+      uint32_t pv[G];                                     // the block's G packed pairs: one 8- or 16-byte store
 #pragma unroll
       for (int g = 0; g < G; ++g) {
         const uint32_t e = pad16[(kb >> (4 * g)) & 15u];
-        if (live)
-          vals32[b * G + g] = slots<false>(e, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3], key[4 * g],
-                                           key[4 * g + 1], key[4 * g + 2], key[4 * g + 3]);
+        pv[g] = slots<false>(e, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3], key[4 * g], key[4 * g + 1],
+                             key[4 * g + 2], key[4 * g + 3]);
         codes |= ((e >> 4) & 15u) << (4 * g);
+      }
+      if (live) {
+        if (G == 2) reinterpret_cast<uint2*>(vals32)[b] = make_uint2(pv[0], pv[1]);
+        else reinterpret_cast<uint4*>(vals32)[b] = make_uint4(pv[0], pv[1], pv[G > 2 ? 2 : 0], pv[G > 3 ? 3 : 0]);
       }
     }
     if (MODE == 2 && live) {
