@@ -143,34 +143,28 @@ __device__ __forceinline__ void epi_stage(const uint32_t (&r)[W], uint32_t dst) 
                            pack_bf16(r[W / 2 + 4 * g + 2], r[W / 2 + 4 * g + 3]));
 }
 
-// Drains chunks c0, c0 + cstep, ... (< nchunks) of one accumulator; called by the four warps of a group with the
-// same arguments except `acc` (the warp's lane quadrant q = warp % 4, column of chunk c: W * c).  After its last
-// tensor-memory read each warp arrives once on `release_bar` (0: nobody waits for the accumulator).
+// The staging and store half of the drain, shared by the two schedules below: state of one warp of a group.
+// `stg`: the group's two staging tiles (2 x W * 256 bytes, 1 KB aligned); `bar_id`: its named barrier.  Every tile
+// of the accumulator loop starts with the first staging tile: the callers synchronise the group between two tiles
+// (the barrier on which the group agrees that the next accumulator is ready), so the last read-back of one tile is
+// over before the next one stages.
 // row_of(c, t) returns where token t of chunk c starts in the result (the CTA's first row), or nullptr when that
 // token lies outside; rows_valid = how many of the CTA's 128 rows exist (a multiple of 32).
-// `stg`: the group's two staging tiles (2 x W * 256 bytes, 1 KB aligned); `bar_id`: its named barrier.  Every call
-// starts with the first tile: the callers synchronise the group between two calls (the barrier on which the group
-// agrees that the next accumulator is ready), so the last read-back of one call is over before the next one stages.
-template <int W, typename RowOf>
-__device__ __forceinline__ void drain_chunks(uint32_t acc, int c0, int cstep, int nchunks, bool zero, uint32_t release_bar,
-                                             uint32_t stg, uint32_t bar_id, int q, int lane, int rows_valid, RowOf&& row_of) {
-  auto release = [&]() {
-    if (release_bar != 0u) {
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive_cluster(release_bar);
-    }
-  };
-  if (c0 >= nchunks) { release(); return; }
-  // stmatrix: lane 8 i + k addresses token k (of a group of eight) of matrix i = rows 32 q + 8 i .. + 7, i.e. unit
-  // 4 q + i of the token's 256-byte row
-  const uint32_t dst = stg + (uint32_t)(lane & 7) * 256u + ((((uint32_t)(4 * q) + ((uint32_t)lane >> 3)) ^ ((uint32_t)lane & 7u)) << 4);
+template <int W>
+struct DrainWarp {
+  uint32_t stg, bar_id, dst, parity;
+  int q, lane, unit;
+  bool unit_ok;
+  __device__ __forceinline__ DrainWarp(uint32_t stg_, uint32_t bar_id_, int q_, int lane_, int rows_valid)
+      : stg(stg_), bar_id(bar_id_), parity(0), q(q_), lane(lane_), unit(lane_ & 15), unit_ok(8 * (lane_ & 15) < rows_valid) {
+    // stmatrix: lane 8 i + k addresses token k (of a group of eight) of matrix i = rows 32 q + 8 i .. + 7, i.e. unit
+    // 4 q + i of the token's 256-byte row
+    dst = stg + (uint32_t)(lane & 7) * 256u + ((((uint32_t)(4 * q) + ((uint32_t)lane >> 3)) ^ ((uint32_t)lane & 7u)) << 4);
+  }
   // reading back: this warp owns tokens (W/4) q .. (W/4) q + W/4 - 1; per step lanes 0-15 take one token, lanes 16-31
   // the next, 16 bytes (eight rows) per lane
-  const int unit = lane & 15;
-  const bool unit_ok = 8 * unit < rows_valid;
-  uint32_t parity = 0;                                    // which of the group's two tiles this chunk goes through
-  auto emit = [&](const uint32_t (&r)[W], int c) {
+  template <typename RowOf>
+  __device__ __forceinline__ void emit(const uint32_t (&r)[W], int c, RowOf& row_of) {
     // Two tiles, one barrier per chunk: a tile is staged again two chunks later, and between the read-back of this
     // chunk and that staging every warp of the group passes the barrier of the chunk in between.
     const uint32_t tile = parity * (uint32_t)(W * 256);
@@ -192,19 +186,38 @@ __device__ __forceinline__ void drain_chunks(uint32_t acc, int c0, int cstep, in
 #pragma unroll
     for (int i = 0; i < W / 8; ++i)
       if (row[i] != nullptr) *reinterpret_cast<uint4*>(row[i]) = v[i];
-  };
+  }
+};
+
+// After its last tensor-memory read a warp arrives once on `release_bar` (0: nobody waits for the accumulator).
+__device__ __forceinline__ void release_accumulator(uint32_t release_bar, int lane) {
+  if (release_bar != 0u) {
+    ptx::tc_fence_before();
+    __syncwarp();
+    if (lane == 0) ptx::mbar_arrive_cluster(release_bar);
+  }
+}
+
+// Drains chunks c0, c0 + cstep, ... (< nchunks) of one accumulator; called by the four warps of a group with the
+// same arguments except `acc` (the warp's lane quadrant q = warp % 4, column of chunk c: W * c).  One chunk is
+// converted and stored while the tensor-memory load of the next is in flight.
+template <int W, typename RowOf>
+__device__ __forceinline__ void drain_chunks(uint32_t acc, int c0, int cstep, int nchunks, bool zero, uint32_t release_bar,
+                                             uint32_t stg, uint32_t bar_id, int q, int lane, int rows_valid, RowOf&& row_of) {
+  if (c0 >= nchunks) { release_accumulator(release_bar, lane); return; }
+  DrainWarp<W> d(stg, bar_id, q, lane, rows_valid);
   uint32_t ra[W], rb[W];
   epi_load<W>(acc + W * c0, ra, zero);
 #pragma unroll 1
   for (int c = c0; c < nchunks; c += 2 * cstep) {
     if (!zero) ptx::tmem_ld_wait();
     const bool more1 = c + cstep < nchunks;
-    if (more1) epi_load<W>(acc + W * (c + cstep), rb, zero); else release();
-    emit(ra, c);
+    if (more1) epi_load<W>(acc + W * (c + cstep), rb, zero); else release_accumulator(release_bar, lane);
+    d.emit(ra, c, row_of);
     if (!more1) break;
     if (!zero) ptx::tmem_ld_wait();
-    if (c + 2 * cstep < nchunks) epi_load<W>(acc + W * (c + 2 * cstep), ra, zero); else release();
-    emit(rb, c + cstep);
+    if (c + 2 * cstep < nchunks) epi_load<W>(acc + W * (c + 2 * cstep), ra, zero); else release_accumulator(release_bar, lane);
+    d.emit(rb, c + cstep, row_of);
   }
 }
 
