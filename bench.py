@@ -527,34 +527,42 @@ def run_per_call(args):
     cfg = inputs.CONFIGS[args.config]
     seed = inputs.perm_seed(args.config)
     peaks = load_peaks()
+    pN, pM = cfg.N, cfg.M
+    if args.pattern:                                          # another N:M pattern on the same shapes, e.g. 4:8 or 2:8
+        pN, pM = (int(v) for v in args.pattern.split(":"))
+    pack = pN <= 2                                            # N > 2: dense masked operands, dense products
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     flush_rd = torch.zeros(64 << 20, dtype=torch.int32, device="cuda")
     reps = max(args.steps, 20) if args.steps != 100 else 20
     out = []
     for li, L in enumerate(cfg.layers):
         W, X, dY = inputs.make_layer(args.config, li)
-        b = bm.alloc_layer_buffers(L.T, L.I, L.J, cfg.P)
+        b = bm.alloc_layer_buffers(L.T, L.I, L.J, cfg.P, dense=not pack)
         b["W"] = torch.from_numpy(W).cuda()
         b["X"] = torch.from_numpy(X.view(np.int16)).cuda().view(torch.bfloat16)
         b["dY"] = torch.from_numpy(dY.view(np.int16)).cuda().view(torch.bfloat16)
+        if not pack:
+            b["meta_f"] = b["hw_meta_f"] = b["meta_b"] = b["hw_meta_b"] = None
         wsb = b["ws"].numel()
         mom = torch.zeros(L.I, L.J, device="cuda")
         calls = {
-            "fwd_mask": lambda: bm.bimask_fwd_mask(b["W"], L.I, L.J, cfg.N, cfg.M, b["maskbits_f"], b["vals_f"], b["meta_f"],
+            "fwd_mask": lambda: bm.bimask_fwd_mask(b["W"], L.I, L.J, pN, pM, b["maskbits_f"], b["vals_f"], b["meta_f"],
                                                    b["hw_meta_f"]),
             "spmm_fwd": lambda: bm.bimask_spmm_fwd(b["X"], b["vals_f"], b["hw_meta_f"], L.T, L.I, L.J, b["Y"], b["status_word"]),
-            "perm_search": lambda: bm.bimask_perm_search(b["maskbits_f"], L.I, L.J, cfg.N, cfg.M, cfg.P, seed, None, b["perm"],
+            "perm_search": lambda: bm.bimask_perm_search(b["maskbits_f"], L.I, L.J, pN, pM, cfg.P, seed, None, b["perm"],
                                                          b["best_idx"], b["counts"], b["ws"], wsb),
-            "bwd_mask": lambda: bm.bimask_bwd_mask(b["W"], b["maskbits_f"], b["perm"], L.I, L.J, cfg.N, cfg.M, b["maskbits_b"],
+            "bwd_mask": lambda: bm.bimask_bwd_mask(b["W"], b["maskbits_f"], b["perm"], L.I, L.J, pN, pM, b["maskbits_b"],
                                                    b["vals_b"], b["meta_b"], b["hw_meta_b"]),
             "spmm_dgrad": lambda: bm.bimask_spmm_dgrad(b["dY"], b["perm"], b["vals_b"], b["hw_meta_b"], L.T, L.I, L.J, b["dX"],
                                                        b["ws"], wsb, b["status_word"]),
             "wgrad": lambda: bm.bimask_wgrad(b["dY"], b["X"], L.T, L.I, L.J, b["dW"], b["ws"], wsb, b["status_word"]),
-            "sgd_fwd_mask": lambda: bm.bimask_sgd_fwd_mask(b["W"], b["dW"], mom, L.I, L.J, cfg.N, cfg.M, 1e-9, 0.9, 1e-4,
+            "sgd_fwd_mask": lambda: bm.bimask_sgd_fwd_mask(b["W"], b["dW"], mom, L.I, L.J, pN, pM, 1e-9, 0.9, 1e-4,
                                                            b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"]),
+            "layer_step": lambda: bm.bimask_layer_step(bm.make_layer_args(L.T, L.I, L.J, pN, pM, cfg.P, seed, True, b)),
         }
         work = algorithmic_work(L, cfg.P)
         work["sgd_fwd_mask"] = {"bound": "hbm", "bytes": 21.4 * L.I * L.J}
+        work["layer_step"] = {"bound": "tensor", "flops": 6.0 * L.T * L.I * L.J}
         for name, fn in calls.items():
             res = {"layer": li, "call": name}
             for kind in ("cold", "warm"):
@@ -579,14 +587,15 @@ def run_per_call(args):
             if w["bound"] == "hbm":
                 res.update(bound="hbm", achieved=w["bytes"] / t / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
             else:
-                pk = peaks["bf16_tflops"] * (1.0 if name == "wgrad" else 2.0)
+                pk = peaks["bf16_tflops"] * (1.0 if (name in ("wgrad", "layer_step") or not pack) else 2.0)
                 res.update(bound="tensor", achieved=w["flops"] / t / 1e12, peak=pk, unit="TFLOP/s")
             res["frac"] = res["achieved"] / res["peak"]
             out.append(res)
         if int(b["status_word"].item()):
             raise RuntimeError("device status word non-zero")
         del b
-    print(json.dumps({"per_call": out, "config": args.config, "launches_per_kind": reps, "peak_source": peaks["source"],
+    print(json.dumps({"per_call": out, "config": args.config, "pattern": f"{pN}:{pM}", "launches_per_kind": reps,
+                      "peak_source": peaks["source"],
                       "note": "fractions of the burst peaks from the cold median"}), flush=True)
 
 
@@ -652,6 +661,7 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=1024)
     ap.add_argument("--ref-tokens", type=int, default=256)
     ap.add_argument("--per-call", action="store_true", help="time every C-ABI call alone (cold and warm L2, min and median)")
+    ap.add_argument("--pattern", default=None, help="with --per-call: another N:M pattern on the config's shapes, e.g. 4:8")
     ap.add_argument("--conv", action="store_true", help="time the convolution form of the layer step instead")
     ap.add_argument("--conv-batch", type=int, default=32)
     args = ap.parse_args()
