@@ -59,7 +59,8 @@ def test_bwd_mask_bit_exact(I, J, N):
 
 
 @pytest.mark.parametrize("I,J,N,P", [(256, 256, 2, 8), (64, 576, 2, 32), (512, 4608, 1, 64), (1152, 384, 2, 32),
-                                     (100, 96, 2, 5), (16384, 64, 2, 3), (40000, 32, 2, 2)])
+                                     (100, 96, 2, 5), (16384, 64, 2, 3), (40000, 32, 2, 2),
+                                     (128, 128, 2, 1), (96, 64, 1, 300), (2048, 2048, 2, 130)])
 def test_perm_search_generated(I, J, N, P):
     W = inputs.make_weight(I, J, I + P)
     B = O.forward_mask(W, N, 4)
