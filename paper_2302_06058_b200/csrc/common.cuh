@@ -5,6 +5,7 @@
 #include <stdint.h>
 #include <stdio.h>
 #include <stdarg.h>
+#include <atomic>
 #include "../../include/bimask.h"
 
 struct CUtensorMap_st;
@@ -57,6 +58,34 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 #endif
+
+}  // namespace bimask
+
+namespace bimask {
+
+// The dynamic shared-memory limit of a kernel is set once per (device, kernel): the call costs a microsecond or two
+// on the host, which a layer step of ten short launches would notice.  A kernel is always launched with the same size.
+template <typename K>
+inline int set_smem_attr(K kernel, int bytes) {
+  constexpr int SLOTS = 64;
+  static std::atomic<const void*> done[64][SLOTS];       // [device][slot]; zero-initialised
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = -1;
+  const void* key = reinterpret_cast<const void*>(kernel);
+  if (dev >= 0)
+    for (int i = 0; i < SLOTS; ++i) {
+      const void* seen = done[dev][i].load(std::memory_order_acquire);
+      if (seen == key) return BIMASK_OK;
+      if (seen == nullptr) break;
+    }
+  BIMASK_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  if (dev >= 0)
+    for (int i = 0; i < SLOTS; ++i) {
+      const void* expect = nullptr;
+      if (done[dev][i].compare_exchange_strong(expect, key, std::memory_order_acq_rel) || expect == key) break;
+    }
+  return BIMASK_OK;
+}
 
 // 2-D tensor map without swizzle (gemm_host.cu); dtype is a CUtensorMapDataType value.
 int make_tmap_plain(CUtensorMap_st* m, int dtype, const void* ptr, uint64_t inner, uint64_t outer, uint32_t box_inner,

@@ -232,30 +232,6 @@ int make_tmap_meta(CUtensorMap* m, const void* ptr, uint64_t blocks);
 // estride 2: a box takes every second pixel along W and H (wb x hb pixels all the same).
 int make_tmap_nhwc_load(CUtensorMap* m, const void* ptr, int CH, int W, int H, int NB, int wb, int hb, int nb, int estride = 1);
 
-// The dynamic shared-memory limit of a kernel is set once per (device, kernel): the call costs a microsecond or two
-// on the host, which a layer step of ten short launches would notice.  A kernel is always launched with the same size.
-template <typename K>
-inline int set_smem_attr(K kernel, int bytes) {
-  constexpr int SLOTS = 64;
-  static std::atomic<const void*> done[16][SLOTS];       // [device][slot]; zero-initialised
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 16) dev = -1;
-  const void* key = reinterpret_cast<const void*>(kernel);
-  if (dev >= 0)
-    for (int i = 0; i < SLOTS; ++i) {
-      const void* seen = done[dev][i].load(std::memory_order_acquire);
-      if (seen == key) return BIMASK_OK;
-      if (seen == nullptr) break;
-    }
-  BIMASK_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  if (dev >= 0)
-    for (int i = 0; i < SLOTS; ++i) {
-      const void* expect = nullptr;
-      if (done[dev][i].compare_exchange_strong(expect, key, std::memory_order_acq_rel) || expect == key) break;
-    }
-  return BIMASK_OK;
-}
-
 // ---- pixel boxes of the implicit convolution ------------------------------------------------
 inline int pow2_ceil(int v) { int p = 1; while (p < v) p <<= 1; return p; }
 inline int log2_exact(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }

@@ -254,12 +254,8 @@ int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, u
     BIMASK_CUDA_OK(cudaGetLastError());
     return BIMASK_OK;
   }
-  static bool attr_done = false;
-  if (!attr_done) {
-    BIMASK_CUDA_OK(cudaFuncSetAttribute(permute_cols_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    BIMASK_CUDA_OK(cudaFuncSetAttribute(permute_cols_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    attr_done = true;
-  }
+  if (int rc = set_smem_attr(permute_cols_kernel<4>, 200 * 1024)) return rc;
+  if (int rc = set_smem_attr(permute_cols_kernel<2>, 200 * 1024)) return rc;
   const int R = (size_t)I * 8 <= 200 * 1024 ? 4 : 2;
   const size_t smem = (size_t)I * 2 * R;
   const int groups = (T + R - 1) / R;

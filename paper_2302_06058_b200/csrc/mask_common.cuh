@@ -49,6 +49,15 @@ __device__ __forceinline__ uint32_t lut_entry(uint32_t cmp, uint32_t valid, int 
   return kb | (idx0 << 4) | (idx1 << 6) | (((kb >> idx0) & 1u) << 8) | (((kb >> idx1) & 1u) << 9) | (sel << 16);
 }
 
+// The same entry laid out for the backward-mask kernel, which reads it as one 64-bit word:
+//   x bits [0,16)  byte-permute selector of the two slots (the permute reads its low 16 bits in place)
+//   x bits [16,20) keep mask, bits [20,24) index code
+//   y              0xFFFF in each half whose slot holds a kept element (the slot is +0 otherwise)
+__device__ __forceinline__ uint2 lut_entry_masked(uint32_t cmp, uint32_t valid, int N) {
+  const uint32_t e = lut_entry(cmp, valid, N);
+  return make_uint2((e >> 16) | ((e & 0xFFu) << 16), (((e >> 8) & 1u) * 0xFFFFu) | (((e >> 9) & 1u) * 0xFFFF0000u));
+}
+
 // Six comparison bits of a block, b01 first (bit 5) ... b23 last (bit 0).  Keys are < 2^31, so
 // key_m - key_q - 1 is negative exactly when key_q >= key_m; a funnel shift moves each sign bit in.
 __device__ __forceinline__ uint32_t cmp6(uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3) {
@@ -86,6 +95,19 @@ __device__ __forceinline__ uint32_t slots(uint32_t e, float w0, float w1, float 
   uint32_t v = __byte_perm(cvt_bf16x2(w1, w0), cvt_bf16x2(w3, w2), e >> 16);
   if (!BOTH_KEPT) v &= (((e >> 8) & 1u) * 0xFFFFu) | (((e >> 9) & 1u) * 0xFFFF0000u);
   return v;
+}
+
+// The two bf16 slots of a block from the 64-bit table entry: two packed conversions, one byte permute, one AND.
+// A block that holds a NaN takes the exact integer conversion (see slots()).
+__device__ __forceinline__ uint32_t slots_masked(uint2 e, float w0, float w1, float w2, float w3,
+                                                 uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3) {
+  if (max(max(k0, k1), max(k2, k3)) > 0x7F800000u) {
+    const uint32_t idx0 = (e.x >> 20) & 3u, idx1 = (e.x >> 22) & 3u;
+    const float s0 = idx0 == 0 ? w0 : idx0 == 1 ? w1 : w2;      // idx0 is never 3
+    const float s1 = idx1 == 1 ? w1 : idx1 == 2 ? w2 : w3;      // idx1 is never 0
+    return ((to_bf16(s0) | (to_bf16(s1) << 16))) & e.y;
+  }
+  return __byte_perm(cvt_bf16x2(w1, w0), cvt_bf16x2(w3, w2), e.x) & e.y;
 }
 
 // One canonical code word (row r of the packed operand, 32-column word w) scattered into the

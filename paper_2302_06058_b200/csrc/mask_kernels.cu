@@ -144,149 +144,176 @@ __global__ void hw_meta_kernel(const uint32_t* __restrict__ meta, int rows, int 
 }
 
 // ---------------------------------------------------------------------------------------
-// Backward mask + transposed pack, asynchronous-copy variant.  A CTA owns 32 CW columns x 64 row-blocks (256
-// permuted rows); warp w walks the eight consecutive row-blocks 8w .. 8w+7.  Each warp runs its own three-deep
-// ring of shared-memory stages filled with cp.async (the slices of the four gathered rows plus their forward-mask
-// words), so the gather of row-block j+2 is in flight while row-block j is processed and costs no registers.
-// Compute uses lane = column within each of the tile's CW 32-column words: conflict-free shared loads, and a warp
-// ballot yields a complete backward-mask word.  The operand being produced is transposed (row = column l of W,
-// k contiguous): each lane keeps the eight consecutive k results of its CW columns in registers and writes them
-// as full 32-byte sectors.
-// CW = 2 (J a multiple of 64) is the variant for large matrices: 256-byte row slices, 64 registers, four CTAs
-// per SM (CW = 4 needs 80 registers, runs three and measured 4 % slower).
-// CW = 1 has twice as many warps again for the same matrix; it serves small matrices, where the per-warp chain
-// of eight row-blocks is what takes the time, and any J % 32 == 0.
+// Backward mask + transposed pack (Eq. 11).  The unit of work is one warp item: 32 permuted rows (eight
+// row-blocks) x 32 CW columns.  Persistent CTAs; every warp walks its own items (column tiles fastest, so the warps
+// that run together read whole stretches of the same gathered rows) with its own four-deep ring of shared-memory
+// stages filled by cp.async: the four row slices of row-block j+3 are in flight while row-block j is processed,
+// also across the boundary between two items, and the ring costs no registers.
+// Compute uses lane = column within each 32-column word (conflict-free shared loads).  The bit matrices at both
+// ends are turned by a 32 x 32 shuffle transpose instead of per-block ballots: lane r loads the forward-mask word
+// of its permuted row, after the transpose lane l holds the 32 candidate bits of its column, one nibble per
+// row-block; the kept bits are collected the same way and transposed back into one backward-mask word per row.
+// The operand being produced is transposed (row = column l of W, k contiguous): a lane keeps the eight
+// consecutive k results of its columns in registers and writes them as full 32-byte sectors; the two halves of
+// a code word go to the tensor-memory image as 32-bit words shared with the lane eight columns away.
+// The selection table (1024 entries: six comparison bits x four candidate bits) is built once per CTA.
+// CW = 2 (J a multiple of 64) for large matrices, CW = 1 for small ones (twice the items) and any J % 32 == 0.
 // ---------------------------------------------------------------------------------------
-constexpr int B4_KB = 64, B4_WARPS = 8, B4_THREADS = 32 * B4_WARPS, B4_RING = 3;
+constexpr int BM_WARPS = 8, BM_THREADS = 32 * BM_WARPS, BM_RING = 4, BM_CTAS_PER_SM = 4;
 template <int CW>
-struct B4Cfg {
-  static constexpr int STAGE = 4 * 128 * CW + 64;          // four row slices + four x 16 bytes for the mask words
-  static constexpr int SMEM = B4_WARPS * B4_RING * STAGE + 4 * B4_KB * 16 + 1024 * 4 + B4_KB * 16;
+struct BMCfg {
+  static constexpr int STAGE = 4 * 128 * CW;               // four row slices of 32 CW floats
+  static constexpr int LUT_BYTES = 1024 * 8;
+  static constexpr int SMEM = LUT_BYTES + BM_WARPS * BM_RING * STAGE;
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
-template <int WORDS>                                       // 1, 2 or 4 32-bit words
-__device__ __forceinline__ void cp_async_words(uint32_t dst, const void* src) {
-  if (WORDS == 4) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-  else if (WORDS == 2) asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
-  else asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
-}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
+// Transpose of a 32 x 32 bit matrix held one row per lane (bit b of lane r = element (r, b)): five exchange
+// stages, each swapping the off-diagonal quadrants of every 2s x 2s block; afterwards lane c holds column c.
+__device__ __forceinline__ uint32_t transpose32(uint32_t x, int lane) {
+  {
+    const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, 16);
+    x = __byte_perm(x, y, (lane & 16) ? 0x3276u : 0x5410u);
+  }
+  {
+    const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, 8);
+    x = __byte_perm(x, y, (lane & 8) ? 0x3715u : 0x6240u);
+  }
+#pragma unroll
+  for (int s = 4; s >= 1; s >>= 1) {
+    const uint32_t m = s == 4 ? 0x0F0F0F0Fu : s == 2 ? 0x33333333u : 0x55555555u;
+    const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, s);
+    const bool low = (lane & s) == 0;                      // this lane keeps its low half of every 2s group
+    const uint32_t keep = low ? m : ~m;
+    const uint32_t moved = low ? (y << s) : (y >> s);
+    x = (x & keep) | (moved & ~keep);
+  }
+  return x;
+}
+
 template <int CW>
-__global__ void __launch_bounds__(B4_THREADS, 4)
-bwd_mask_async_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,
-                      const int32_t* __restrict__ perm, int I, int J, int N,
-                      uint32_t* __restrict__ maskbits_b, uint32_t* __restrict__ vals_b,
-                      uint32_t* __restrict__ meta_b, uint16_t* __restrict__ hw16) {
+__global__ void __launch_bounds__(BM_THREADS, BM_CTAS_PER_SM)
+bwd_mask_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,
+                const int32_t* __restrict__ perm, int I, int J, int N,
+                uint32_t* __restrict__ maskbits_b, uint32_t* __restrict__ vals_b,
+                uint32_t* __restrict__ meta_b, uint32_t* __restrict__ hw32, int col_tiles, int n_items) {
   pdl_launch_dependents();
-  using C = B4Cfg<CW>;
+  using C = BMCfg<CW>;
   extern __shared__ __align__(128) uint8_t smem[];
-  uint8_t* ring = smem;                                                          // [warp][stage][C::STAGE]
-  uint4* mb_s = reinterpret_cast<uint4*>(smem + B4_WARPS * B4_RING * C::STAGE);  // [256 rows] x up to 4 mask words
-  uint32_t* lut = reinterpret_cast<uint32_t*>(mb_s + 4 * B4_KB);                 // [1024]
-  int4* perm_s = reinterpret_cast<int4*>(lut + 1024);                            // [64]
+  uint2* lut = reinterpret_cast<uint2*>(smem);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int col0 = blockIdx.y * 32 * CW;                   // J % (32 CW) == 0: the tile is always full
-  const int kb0 = blockIdx.x * B4_KB;
-  const int kb_here = min(B4_KB, (I >> 2) - kb0);          // multiple of 8 (I % 32 == 0)
+  for (int e = threadIdx.x; e < 1024; e += BM_THREADS) lut[e] = lut_entry_masked(e & 63u, e >> 6, N);
+  pdl_wait();                                              // the table needed no global memory
+  __syncthreads();
+  const int nw = gridDim.x * BM_WARPS;
+  int item = blockIdx.x * BM_WARPS + warp;
+  if (item >= n_items) return;
+  uint8_t* my_ring = smem + C::LUT_BYTES + warp * BM_RING * C::STAGE;
+  const uint32_t ring_u32 = ptx::smem_u32(my_ring);
   const int jwords = J >> 5;
   const unsigned last_row = (unsigned)(I - 1);
+  const int step_rg = nw / col_tiles, step_ct = nw % col_tiles;
+  int rg = item / col_tiles, ct = item % col_tiles;        // 32-row group and column tile of the item
 
-  for (int e = threadIdx.x; e < 1024; e += B4_THREADS) lut[e] = lut_entry(e & 63u, e >> 6, N);
-  pdl_wait();                                              // the table needed no global memory
-  for (int kk = threadIdx.x; kk < kb_here; kk += B4_THREADS) {
-    const int4 p4 = __ldg(reinterpret_cast<const int4*>(perm) + kb0 + kk);
-    perm_s[kk] = make_int4((int)min((unsigned)p4.x, last_row), (int)min((unsigned)p4.y, last_row),
-                           (int)min((unsigned)p4.z, last_row), (int)min((unsigned)p4.w, last_row));
-  }
-  __syncthreads();
-  const int kw = 8 * warp;                                 // this warp's row-blocks kw .. kw+7 of the tile
-  if (kw < kb_here) {
-    uint8_t* my_ring = ring + warp * B4_RING * C::STAGE;
-    const uint32_t ring_u32 = ptx::smem_u32(my_ring);
-    auto issue = [&](int j) {                              // start the gather of row-block kw + j
-      const int4 p4 = perm_s[kw + j];
-      const int r[4] = {p4.x, p4.y, p4.z, p4.w};
-      const uint32_t dst = ring_u32 + (j % B4_RING) * C::STAGE;
-      // a row slice is 128 CW bytes = 8 CW lanes x 16 bytes: CW passes of 4 / CW rows each
+  // the gather of row-block j of an item whose 32 row indices the lanes hold in `rows`
+  auto issue = [&](int rows, int ctile, int j) {
+    const uint32_t dst = ring_u32 + (j % BM_RING) * C::STAGE;
+    // a row slice is 128 CW bytes = 8 CW lanes x 16 bytes: CW passes of 4 / CW rows each
 #pragma unroll
-      for (int ps = 0; ps < CW; ++ps) {
-        const int m = ps * (4 / CW) + lane / (8 * CW), piece = lane % (8 * CW);
-        cp_async16(dst + m * 128 * CW + 16 * piece, W + (size_t)r[m] * J + col0 + 4 * piece);
-      }
-      if (lane < 4) cp_async_words<CW>(dst + 512 * CW + 16 * lane, maskbits_f + (size_t)r[lane] * jwords + (col0 >> 5));
-      cp_async_commit();
-    };
-    issue(0);
-    issue(1);
+    for (int ps = 0; ps < CW; ++ps) {
+      const int m = ps * (4 / CW) + lane / (8 * CW), piece = lane % (8 * CW);
+      const int r = __shfl_sync(0xFFFFFFFFu, rows, 4 * j + m);
+      cp_async16(dst + m * 128 * CW + 16 * piece, W + (size_t)r * J + ctile * 32 * CW + 4 * piece);
+    }
+    cp_async_commit();
+  };
+  auto load_rows = [&](int rgroup) { return (int)min((unsigned)__ldg(perm + 32 * rgroup + lane), last_row); };
+  auto load_fwd = [&](int rows, int ctile, uint32_t (&f)[CW]) {
+    const uint32_t* src = maskbits_f + (size_t)rows * jwords + ctile * CW;
+    if (CW == 2) { const uint2 t = __ldg(reinterpret_cast<const uint2*>(src)); f[0] = t.x; f[1] = t.y; }
+    else f[0] = __ldg(src);
+  };
+
+  int rows_nxt = load_rows(rg);
+  uint32_t f_nxt[CW];
+  load_fwd(rows_nxt, ct, f_nxt);
+  issue(rows_nxt, ct, 0);
+  issue(rows_nxt, ct, 1);
+  issue(rows_nxt, ct, 2);
+  const size_t vrow = (size_t)I >> 2;                      // u32 (bf16 pairs) per row of vals_b
+  const size_t mrow = (size_t)I >> 5;
+  while (true) {
+    const int rows_cur = rows_nxt;
+    uint32_t cand[CW];                                     // candidate bits of this lane's columns, by row
+#pragma unroll
+    for (int c = 0; c < CW; ++c) cand[c] = transpose32(f_nxt[c], lane);
+    int rg_n = rg + step_rg, ct_n = ct + step_ct;
+    if (ct_n >= col_tiles) { ct_n -= col_tiles; ++rg_n; }
+    const bool has_next = item + nw < n_items;             // warp uniform
+    if (has_next) rows_nxt = load_rows(rg_n);
     uint32_t vacc[CW][8];
-    uint32_t cacc[CW];
+    uint32_t cacc[CW], kacc[CW];
 #pragma unroll
-    for (int c = 0; c < CW; ++c) cacc[c] = 0u;
+    for (int c = 0; c < CW; ++c) cacc[c] = kacc[c] = 0u;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      if (j + 2 < 8) issue(j + 2); else cp_async_commit();  // keep the group count uniform
-      cp_async_wait<2>();                                  // row-block j has landed
+      if (j + 3 < 8) issue(rows_cur, ct, j + 3);
+      else if (has_next) issue(rows_nxt, ct_n, j + 3 - 8);  // the ring runs on into the next item
+      else cp_async_commit();                              // keep the group count uniform
+      if (j == 4 && has_next) load_fwd(rows_nxt, ct_n, f_nxt);
+      cp_async_wait<3>();                                  // row-block j has landed
       __syncwarp();
-      const float* ws = reinterpret_cast<const float*>(my_ring + (j % B4_RING) * C::STAGE);
-      const uint4* fs = reinterpret_cast<const uint4*>(my_ring + (j % B4_RING) * C::STAGE + 128 * CW * 4);
+      const float* ws = reinterpret_cast<const float*>(my_ring + (j % BM_RING) * C::STAGE);
       float w[4][CW];
-      uint4 fw[4];
 #pragma unroll
-      for (int m = 0; m < 4; ++m) {
-        if (CW == 4) fw[m] = fs[m];
-        else if (CW == 2) { const uint2 t = reinterpret_cast<const uint2*>(fs + m)[0]; fw[m].x = t.x; fw[m].y = t.y; }
-        else fw[m].x = reinterpret_cast<const uint32_t*>(fs + m)[0];
+      for (int m = 0; m < 4; ++m)
 #pragma unroll
         for (int c = 0; c < CW; ++c) w[m][c] = ws[m * 32 * CW + 32 * c + lane];
-      }
       __syncwarp();                                        // all lanes have read the stage
-      const int kk = kw + j;
 #pragma unroll
       for (int c = 0; c < CW; ++c) {
-        const uint32_t f0 = c == 0 ? fw[0].x : c == 1 ? fw[0].y : c == 2 ? fw[0].z : fw[0].w;
-        const uint32_t f1 = c == 0 ? fw[1].x : c == 1 ? fw[1].y : c == 2 ? fw[1].z : fw[1].w;
-        const uint32_t f2 = c == 0 ? fw[2].x : c == 1 ? fw[2].y : c == 2 ? fw[2].z : fw[2].w;
-        const uint32_t f3 = c == 0 ? fw[3].x : c == 1 ? fw[3].y : c == 2 ? fw[3].z : fw[3].w;
-        const uint32_t valid = ((f0 >> lane) & 1u) | (((f1 >> lane) & 1u) << 1) | (((f2 >> lane) & 1u) << 2) |
-                               (((f3 >> lane) & 1u) << 3);
         const uint32_t k0 = mag_key(w[0][c]), k1 = mag_key(w[1][c]), k2 = mag_key(w[2][c]), k3 = mag_key(w[3][c]);
-        const uint32_t e = lut[(valid << 6) | cmp6(k0, k1, k2, k3)];
-        vacc[c][j] = slots<false>(e, w[0][c], w[1][c], w[2][c], w[3][c], k0, k1, k2, k3);
-        cacc[c] |= ((e >> 4) & 15u) << (4 * j);
-        uint32_t b[4];
-#pragma unroll
-        for (int m = 0; m < 4; ++m) b[m] = __ballot_sync(0xFFFFFFFFu, (e >> m) & 1u);
-        if (lane == 0) {
-#pragma unroll
-          for (int m = 0; m < 4; ++m) reinterpret_cast<uint32_t*>(mb_s + 4 * kk + m)[c] = b[m];
-        }
+        const uint32_t valid = (cand[c] >> (4 * j)) & 15u;
+        const uint2 e = lut[(valid << 6) | cmp6(k0, k1, k2, k3)];
+        vacc[c][j] = slots_masked(e, w[0][c], w[1][c], w[2][c], w[3][c], k0, k1, k2, k3);
+        kacc[c] |= ((e.x >> 16) & 15u) << (4 * j);
+        cacc[c] |= ((e.x >> 20) & 15u) << (4 * j);
       }
     }
-    cp_async_wait<0>();
-    __syncwarp();
     // this warp's 32 permuted rows of backward-mask words: one store of CW words per lane
-    uint32_t* mrow_out = maskbits_b + (size_t)(4 * (kb0 + kw) + lane) * jwords + (col0 >> 5);
-    if (CW == 4) *reinterpret_cast<uint4*>(mrow_out) = mb_s[4 * kw + lane];
-    else if (CW == 2) *reinterpret_cast<uint2*>(mrow_out) = reinterpret_cast<const uint2*>(mb_s + 4 * kw + lane)[0];
-    else *mrow_out = reinterpret_cast<const uint32_t*>(mb_s + 4 * kw + lane)[0];
-    const size_t vrow = (size_t)I >> 2;                    // u32 (bf16 pairs) per row of vals_b
-    const size_t mrow = (size_t)I >> 5;
+    uint32_t* mrow_out = maskbits_b + (size_t)(32 * rg + lane) * jwords + ct * CW;
+    if (CW == 2) *reinterpret_cast<uint2*>(mrow_out) = make_uint2(transpose32(kacc[0], lane), transpose32(kacc[1], lane));
+    else *mrow_out = transpose32(kacc[0], lane);
 #pragma unroll
     for (int c = 0; c < CW; ++c) {
-      const int l = col0 + 32 * c + lane;
-      uint4* dst = reinterpret_cast<uint4*>(vals_b + (size_t)l * vrow + kb0 + kw);
+      const int l = (ct * CW + c) * 32 + lane;
+      uint4* dst = reinterpret_cast<uint4*>(vals_b + (size_t)l * vrow + 8 * rg);
       dst[0] = make_uint4(vacc[c][0], vacc[c][1], vacc[c][2], vacc[c][3]);
       dst[1] = make_uint4(vacc[c][4], vacc[c][5], vacc[c][6], vacc[c][7]);
-      meta_b[(size_t)l * mrow + ((kb0 + kw) >> 3)] = cacc[c];
-      if (hw16) scatter_hw(hw16, I >> 7, l, (kb0 + kw) >> 3, cacc[c]);
+      meta_b[(size_t)l * mrow + rg] = cacc[c];
+      if (hw32) {
+        // image word (rows l and l ^ 8 of the operand, k word rg): its low-half lane stores the two low halves of
+        // the code words, its high-half lane the two high halves
+        const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, cacc[c], 8);
+        const int rr = l & 127;
+        const size_t tile = (size_t)(l >> 7) * (I >> 7) + (rg >> 2);
+        const size_t at = tile * 512 + (size_t)((rr & 7) + 16 * (rr >> 4)) * 4 + (rg & 3);
+        if (rr & 8) hw32[at + 32] = __byte_perm(other, cacc[c], 0x7632u);
+        else hw32[at] = __byte_perm(cacc[c], other, 0x5410u);
+      }
     }
+    if (!has_next) break;
+    item += nw;
+    rg = rg_n;
+    ct = ct_n;
   }
+  cp_async_wait<0>();
 }
 
 }  // namespace
@@ -376,23 +403,25 @@ int launch_hw_meta(const uint32_t* meta, int rows, int K, void* hw_meta, cudaStr
 int launch_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                     int N, uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_or_null,
                     cudaStream_t s) {
-  // the wide tile (64 columns per warp) once it gives every SM a few CTAs, the narrow one otherwise
-  const int row_tiles = (I / 4 + B4_KB - 1) / B4_KB;
-  const bool wide = J % 64 == 0 && (long long)row_tiles * (J / 64) >= 4 * 148;
-  static bool attr_done = false;
-  if (!attr_done) {
-    BIMASK_CUDA_OK(cudaFuncSetAttribute(bwd_mask_async_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, B4Cfg<2>::SMEM));
-    BIMASK_CUDA_OK(cudaFuncSetAttribute(bwd_mask_async_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, B4Cfg<1>::SMEM));
-    attr_done = true;
-  }
+  // 64-column items once they keep every resident warp busy, 32-column items (twice as many) otherwise
+  const long long items_wide = (long long)(I / 32) * (J / 64);
+  const bool wide = J % 64 == 0 && items_wide >= (long long)BM_CTAS_PER_SM * 148 * BM_WARPS;
+  const int col_tiles = wide ? J / 64 : J / 32;
+  const long long n_items = (long long)(I / 32) * col_tiles;
+  BIMASK_REQUIRE(n_items < (1ll << 31), BIMASK_EUNSUPPORTED, "bimask_bwd_mask: I * J = %lld is beyond the kernel's item index",
+                 (long long)I * J);
+  long long ctas = (n_items + BM_WARPS - 1) / BM_WARPS;
+  if (ctas > BM_CTAS_PER_SM * 148) ctas = BM_CTAS_PER_SM * 148;
   uint32_t* vals32 = reinterpret_cast<uint32_t*>(vals_b);
-  uint16_t* hw16 = reinterpret_cast<uint16_t*>(hw_meta_or_null);
+  uint32_t* hw32 = reinterpret_cast<uint32_t*>(hw_meta_or_null);
   if (wide) {
-    dim3 grid(row_tiles, J / 64);
-    BIMASK_CUDA_OK(launch_pdl(bwd_mask_async_kernel<2>, grid, B4_THREADS, B4Cfg<2>::SMEM, s, W, maskbits_f, perm, I, J, N, maskbits_b, vals32, meta_b, hw16));
+    if (int rc = set_smem_attr(bwd_mask_kernel<2>, BMCfg<2>::SMEM)) return rc;
+    BIMASK_CUDA_OK(launch_pdl(bwd_mask_kernel<2>, (unsigned)ctas, BM_THREADS, BMCfg<2>::SMEM, s, W, maskbits_f, perm, I, J, N,
+                              maskbits_b, vals32, meta_b, hw32, col_tiles, (int)n_items));
   } else {
-    dim3 grid(row_tiles, J / 32);
-    BIMASK_CUDA_OK(launch_pdl(bwd_mask_async_kernel<1>, grid, B4_THREADS, B4Cfg<1>::SMEM, s, W, maskbits_f, perm, I, J, N, maskbits_b, vals32, meta_b, hw16));
+    if (int rc = set_smem_attr(bwd_mask_kernel<1>, BMCfg<1>::SMEM)) return rc;
+    BIMASK_CUDA_OK(launch_pdl(bwd_mask_kernel<1>, (unsigned)ctas, BM_THREADS, BMCfg<1>::SMEM, s, W, maskbits_f, perm, I, J, N,
+                              maskbits_b, vals32, meta_b, hw32, col_tiles, (int)n_items));
   }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());

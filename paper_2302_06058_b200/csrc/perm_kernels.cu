@@ -311,11 +311,7 @@ int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStrea
   const int mean = (I + (1 << ql) - 1) >> ql;
   const int cap = ql == 0 ? I : mean + (mean / 4 > 256 ? mean / 4 : 256);
   const size_t smem = (size_t)cap * sizeof(unsigned long long) + ((size_t)1 << (lg - ql)) * sizeof(uint32_t);
-  static bool attr_done = false;     // same value every time; a race only repeats the call
-  if (!attr_done) {
-    BIMASK_CUDA_OK(cudaFuncSetAttribute(gen_candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    attr_done = true;
-  }
+  if (int rc = set_smem_attr(gen_candidates_kernel, 200 * 1024)) return rc;
   dim3 grid(P, 1 << ql);
   BIMASK_CUDA_OK(launch_pdl(gen_candidates_kernel, grid, GEN_THREADS, smem, s, (unsigned long long)seed, I, lg, ql, cap, cands,
                                                         reinterpret_cast<unsigned long long*>(zero_counts), zero_ticket));
