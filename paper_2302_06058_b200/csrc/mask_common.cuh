@@ -49,13 +49,14 @@ __device__ __forceinline__ uint32_t lut_entry(uint32_t cmp, uint32_t valid, int 
   return kb | (idx0 << 4) | (idx1 << 6) | (((kb >> idx0) & 1u) << 8) | (((kb >> idx1) & 1u) << 9) | (sel << 16);
 }
 
-// The same entry laid out for the backward-mask kernel, which reads it as one 64-bit word:
-//   x bits [0,16)  byte-permute selector of the two slots (the permute reads its low 16 bits in place)
-//   x bits [16,20) keep mask, bits [20,24) index code
-//   y              0xFFFF in each half whose slot holds a kept element (the slot is +0 otherwise)
-__device__ __forceinline__ uint2 lut_entry_masked(uint32_t cmp, uint32_t valid, int N) {
+// The same entry laid out for the backward-mask kernel:
+//   bits [0,16)  byte-permute selector of the two slots (the permute reads its low 16 bits in place)
+//   bits [16,20) keep mask, bits [24,28) index code
+//   bit 31 / 23  slot 0 / slot 1 holds a kept element: the top bits of bytes 3 and 2, so that one byte permute in
+//                sign-replication mode expands them into the 0xFFFF / 0 halves of the slot mask
+__device__ __forceinline__ uint32_t lut_entry_signs(uint32_t cmp, uint32_t valid, int N) {
   const uint32_t e = lut_entry(cmp, valid, N);
-  return make_uint2((e >> 16) | ((e & 0xFFu) << 16), (((e >> 8) & 1u) * 0xFFFFu) | (((e >> 9) & 1u) * 0xFFFF0000u));
+  return (e >> 16) | ((e & 0xFu) << 16) | (((e >> 4) & 0xFu) << 24) | (((e >> 8) & 1u) << 31) | (((e >> 9) & 1u) << 23);
 }
 
 // Six comparison bits of a block, b01 first (bit 5) ... b23 last (bit 0).  Keys are < 2^31, so
@@ -97,17 +98,20 @@ __device__ __forceinline__ uint32_t slots(uint32_t e, float w0, float w1, float 
   return v;
 }
 
-// The two bf16 slots of a block from the 64-bit table entry: two packed conversions, one byte permute, one AND.
-// A block that holds a NaN takes the exact integer conversion (see slots()).
-__device__ __forceinline__ uint32_t slots_masked(uint2 e, float w0, float w1, float w2, float w3,
-                                                 uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3) {
+// The two bf16 slots of a block from an entry of lut_entry_signs: two packed conversions and three byte permutes
+// (select the slots; expand the two "kept" bits into a mask).  A block that holds a NaN takes the exact integer
+// conversion (see slots()).
+__device__ __forceinline__ uint32_t slots_signs(uint32_t e, float w0, float w1, float w2, float w3,
+                                                uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3) {
+  uint32_t keep;                                           // bytes 0-1: sign of byte 3, bytes 2-3: sign of byte 2
+  asm("prmt.b32 %0, %1, %1, 0xAABB;" : "=r"(keep) : "r"(e));
   if (max(max(k0, k1), max(k2, k3)) > 0x7F800000u) {
-    const uint32_t idx0 = (e.x >> 20) & 3u, idx1 = (e.x >> 22) & 3u;
+    const uint32_t idx0 = (e >> 24) & 3u, idx1 = (e >> 26) & 3u;
     const float s0 = idx0 == 0 ? w0 : idx0 == 1 ? w1 : w2;      // idx0 is never 3
     const float s1 = idx1 == 1 ? w1 : idx1 == 2 ? w2 : w3;      // idx1 is never 0
-    return ((to_bf16(s0) | (to_bf16(s1) << 16))) & e.y;
+    return (to_bf16(s0) | (to_bf16(s1) << 16)) & keep;
   }
-  return __byte_perm(cvt_bf16x2(w1, w0), cvt_bf16x2(w3, w2), e.x) & e.y;
+  return __byte_perm(cvt_bf16x2(w1, w0), cvt_bf16x2(w3, w2), e) & keep;
 }
 
 // One canonical code word (row r of the packed operand, 32-column word w) scattered into the

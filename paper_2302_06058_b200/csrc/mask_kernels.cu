@@ -144,27 +144,37 @@ __global__ void hw_meta_kernel(const uint32_t* __restrict__ meta, int rows, int 
 }
 
 // ---------------------------------------------------------------------------------------
-// Backward mask + transposed pack (Eq. 11).  The unit of work is one warp item: 32 permuted rows (eight
-// row-blocks) x 32 CW columns.  Persistent CTAs; every warp walks its own items (column tiles fastest, so the warps
-// that run together read whole stretches of the same gathered rows) with its own four-deep ring of shared-memory
-// stages filled by cp.async: the four row slices of row-block j+3 are in flight while row-block j is processed,
-// also across the boundary between two items, and the ring costs no registers.
+// Backward mask + transposed pack (Eq. 11).  Persistent CTAs walk tiles of 128 permuted rows x 64 CW columns
+// (column tiles fastest, so the CTAs that run together read whole stretches of the same gathered rows).  Inside
+// a tile warp w owns one item: the 32 rows (eight row-blocks) of row group w & 3 and the 32 CW columns of column
+// item w >> 2.  Every warp runs its own three-deep ring of shared-memory stages filled by cp.async: the four row
+// slices of row-block j+2 are in flight while row-block j is processed, also across the boundary between two
+// tiles, and the ring costs no registers.
 // Compute uses lane = column within each 32-column word (conflict-free shared loads).  The bit matrices at both
 // ends are turned by a 32 x 32 shuffle transpose instead of per-block ballots: lane r loads the forward-mask word
 // of its permuted row, after the transpose lane l holds the 32 candidate bits of its column, one nibble per
 // row-block; the kept bits are collected the same way and transposed back into one backward-mask word per row.
-// The operand being produced is transposed (row = column l of W, k contiguous): a lane keeps the eight
-// consecutive k results of its columns in registers and writes them as full 32-byte sectors; the two halves of
-// a code word go to the tensor-memory image as 32-bit words shared with the lane eight columns away.
+// The operand being produced is transposed (row = column l of W, k contiguous), so a lane's results are 32 bytes
+// of one operand row, a code word and a few mask bits: stored from the registers, every store instruction would
+// touch 32 different 128-byte lines, and the load/store unit, not HBM, set the kernel's time.  The eight warps
+// therefore put their results into a shared staging tile and the CTA writes it out in whole lines: 128 bytes per
+// operand row, 16 bytes per code row and mask row, and the tile's 128 x 128 block of the tensor-memory image of
+// the codes as one contiguous run.
 // The selection table (1024 entries: six comparison bits x four candidate bits) is built once per CTA.
-// CW = 2 (J a multiple of 64) for large matrices, CW = 1 for small ones (twice the items) and any J % 32 == 0.
+// CW = 2 (J a multiple of 64) for large matrices, CW = 1 for small ones (twice the tiles) and any J % 32 == 0.
 // ---------------------------------------------------------------------------------------
-constexpr int BM_WARPS = 8, BM_THREADS = 32 * BM_WARPS, BM_RING = 4, BM_CTAS_PER_SM = 4;
+constexpr int BM_WARPS = 8, BM_THREADS = 32 * BM_WARPS, BM_RING = 3, BM_CTAS_PER_SM = 4;
+constexpr int BM_SV_PITCH = 36;                            // words per staged operand row: 32 + 4, conflict-free 16-byte accesses
 template <int CW>
 struct BMCfg {
+  static constexpr int COLS = 64 * CW;                     // columns of a tile
   static constexpr int STAGE = 4 * 128 * CW;               // four row slices of 32 CW floats
-  static constexpr int LUT_BYTES = 1024 * 8;
-  static constexpr int SMEM = LUT_BYTES + BM_WARPS * BM_RING * STAGE;
+  static constexpr int LUT_BYTES = 1024 * 4;
+  static constexpr int RING_BYTES = BM_WARPS * BM_RING * STAGE;
+  static constexpr int SV_BYTES = COLS * BM_SV_PITCH * 4;  // operand values [column][32 k pairs]
+  static constexpr int SM_BYTES = 128 * 2 * CW * 4;        // backward-mask words [row][2 CW]
+  static constexpr int SC_BYTES = COLS * 4 * 4;            // code words [column][4]
+  static constexpr int SMEM = LUT_BYTES + RING_BYTES + SV_BYTES + SM_BYTES + SC_BYTES;
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -202,116 +212,169 @@ __global__ void __launch_bounds__(BM_THREADS, BM_CTAS_PER_SM)
 bwd_mask_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,
                 const int32_t* __restrict__ perm, int I, int J, int N,
                 uint32_t* __restrict__ maskbits_b, uint32_t* __restrict__ vals_b,
-                uint32_t* __restrict__ meta_b, uint32_t* __restrict__ hw32, int col_tiles, int n_items) {
+                uint32_t* __restrict__ meta_b, uint32_t* __restrict__ hw32, int tiles_c, int n_tiles) {
   pdl_launch_dependents();
   using C = BMCfg<CW>;
   extern __shared__ __align__(128) uint8_t smem[];
-  uint2* lut = reinterpret_cast<uint2*>(smem);
+  uint32_t* lut = reinterpret_cast<uint32_t*>(smem);
+  uint8_t* ring_all = smem + C::LUT_BYTES;
+  uint32_t* sv = reinterpret_cast<uint32_t*>(ring_all + C::RING_BYTES);
+  uint32_t* sm = sv + C::SV_BYTES / 4;
+  uint32_t* sc = sm + C::SM_BYTES / 4;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int e = threadIdx.x; e < 1024; e += BM_THREADS) lut[e] = lut_entry_masked(e & 63u, e >> 6, N);
+  for (int e = threadIdx.x; e < 1024; e += BM_THREADS) lut[e] = lut_entry_signs(e & 63u, e >> 6, N);
   pdl_wait();                                              // the table needed no global memory
   __syncthreads();
-  const int nw = gridDim.x * BM_WARPS;
-  int item = blockIdx.x * BM_WARPS + warp;
-  if (item >= n_items) return;
-  uint8_t* my_ring = smem + C::LUT_BYTES + warp * BM_RING * C::STAGE;
+  uint8_t* my_ring = ring_all + warp * BM_RING * C::STAGE;
   const uint32_t ring_u32 = ptx::smem_u32(my_ring);
   const int jwords = J >> 5;
+  const int nrg = I >> 5;                                  // groups of 32 permuted rows
+  const int items = jwords / CW;                           // column items of 32 CW columns
   const unsigned last_row = (unsigned)(I - 1);
-  const int step_rg = nw / col_tiles, step_ct = nw % col_tiles;
-  int rg = item / col_tiles, ct = item % col_tiles;        // 32-row group and column tile of the item
+  const int rgi = warp & 3, cti = warp >> 2;               // this warp's row group and column item inside a tile
+  const size_t vrow = (size_t)I >> 2;                      // u32 (bf16 pairs) per row of vals_b
+  const size_t mrow = (size_t)I >> 5;
 
-  // the gather of row-block j of an item whose 32 row indices the lanes hold in `rows`
-  auto issue = [&](int rows, int ctile, int j) {
-    const uint32_t dst = ring_u32 + (j % BM_RING) * C::STAGE;
+  // the gather of row-block j of an item whose 32 row indices the lanes hold in `rows`, into the stage at `soff`
+  auto issue = [&](int rows, int item, int j, int soff) {
     // a row slice is 128 CW bytes = 8 CW lanes x 16 bytes: CW passes of 4 / CW rows each
 #pragma unroll
     for (int ps = 0; ps < CW; ++ps) {
       const int m = ps * (4 / CW) + lane / (8 * CW), piece = lane % (8 * CW);
       const int r = __shfl_sync(0xFFFFFFFFu, rows, 4 * j + m);
-      cp_async16(dst + m * 128 * CW + 16 * piece, W + (size_t)r * J + ctile * 32 * CW + 4 * piece);
+      cp_async16(ring_u32 + soff + m * 128 * CW + 16 * piece, W + (size_t)r * J + item * 32 * CW + 4 * piece);
     }
     cp_async_commit();
   };
   auto load_rows = [&](int rgroup) { return (int)min((unsigned)__ldg(perm + 32 * rgroup + lane), last_row); };
-  auto load_fwd = [&](int rows, int ctile, uint32_t (&f)[CW]) {
-    const uint32_t* src = maskbits_f + (size_t)rows * jwords + ctile * CW;
+  auto load_fwd = [&](int rows, int item, uint32_t (&f)[CW]) {
+    const uint32_t* src = maskbits_f + (size_t)rows * jwords + item * CW;
     if (CW == 2) { const uint2 t = __ldg(reinterpret_cast<const uint2*>(src)); f[0] = t.x; f[1] = t.y; }
     else f[0] = __ldg(src);
   };
 
-  int rows_nxt = load_rows(rg);
+  bool primed = false;                                     // the first two row-blocks of the coming item are in flight
+  int off = 0;                                             // ring offset of the stage that holds the next row-block
+  int rows_nxt = 0;
   uint32_t f_nxt[CW];
-  load_fwd(rows_nxt, ct, f_nxt);
-  issue(rows_nxt, ct, 0);
-  issue(rows_nxt, ct, 1);
-  issue(rows_nxt, ct, 2);
-  const size_t vrow = (size_t)I >> 2;                      // u32 (bf16 pairs) per row of vals_b
-  const size_t mrow = (size_t)I >> 5;
-  while (true) {
-    const int rows_cur = rows_nxt;
-    uint32_t cand[CW];                                     // candidate bits of this lane's columns, by row
 #pragma unroll
-    for (int c = 0; c < CW; ++c) cand[c] = transpose32(f_nxt[c], lane);
-    int rg_n = rg + step_rg, ct_n = ct + step_ct;
-    if (ct_n >= col_tiles) { ct_n -= col_tiles; ++rg_n; }
-    const bool has_next = item + nw < n_items;             // warp uniform
-    if (has_next) rows_nxt = load_rows(rg_n);
-    uint32_t vacc[CW][8];
-    uint32_t cacc[CW], kacc[CW];
+  for (int c = 0; c < CW; ++c) f_nxt[c] = 0u;
+  for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const int tr = tile / tiles_c, tc = tile - tr * tiles_c;
+    const int rg = 4 * tr + rgi, item = 2 * tc + cti;
+    const bool active = rg < nrg && item < items;          // warp uniform
+    const int tile_n = tile + gridDim.x;
+    const int tr_n = tile_n / tiles_c, tc_n = tile_n - tr_n * tiles_c;
+    const int rg_n = 4 * tr_n + rgi, item_n = 2 * tc_n + cti;
+    const bool active_n = tile_n < n_tiles && rg_n < nrg && item_n < items;
+    if (active) {
+      if (!primed) {
+        rows_nxt = load_rows(rg);
+        load_fwd(rows_nxt, item, f_nxt);
+        off = 0;
+        issue(rows_nxt, item, 0, 0);
+        issue(rows_nxt, item, 1, C::STAGE);
+      }
+      const int rows_cur = rows_nxt;
+      uint32_t cand[CW];                                   // candidate bits of this lane's columns, by row
 #pragma unroll
-    for (int c = 0; c < CW; ++c) cacc[c] = kacc[c] = 0u;
+      for (int c = 0; c < CW; ++c) cand[c] = transpose32(f_nxt[c], lane);
+      if (active_n) rows_nxt = load_rows(rg_n);
+      uint32_t vacc[CW][8];
+      uint32_t cacc[CW], kacc[CW];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      if (j + 3 < 8) issue(rows_cur, ct, j + 3);
-      else if (has_next) issue(rows_nxt, ct_n, j + 3 - 8);  // the ring runs on into the next item
-      else cp_async_commit();                              // keep the group count uniform
-      if (j == 4 && has_next) load_fwd(rows_nxt, ct_n, f_nxt);
-      cp_async_wait<3>();                                  // row-block j has landed
-      __syncwarp();
-      const float* ws = reinterpret_cast<const float*>(my_ring + (j % BM_RING) * C::STAGE);
-      float w[4][CW];
+      for (int c = 0; c < CW; ++c) cacc[c] = kacc[c] = 0u;
 #pragma unroll
-      for (int m = 0; m < 4; ++m)
+      for (int j = 0; j < 8; ++j) {
+        int ioff = off + 2 * C::STAGE;                     // the stage read in the previous step
+        if (ioff >= BM_RING * C::STAGE) ioff -= BM_RING * C::STAGE;
+        if (j + 2 < 8) issue(rows_cur, item, j + 2, ioff);
+        else if (active_n) issue(rows_nxt, item_n, j + 2 - 8, ioff);   // the ring runs on into the next tile
+        else cp_async_commit();                            // keep the group count uniform
+        if (j == 4 && active_n) load_fwd(rows_nxt, item_n, f_nxt);
+        cp_async_wait<2>();                                // row-block j has landed
+        __syncwarp();
+        const float* ws = reinterpret_cast<const float*>(my_ring + off);
+        float w[4][CW];
 #pragma unroll
-        for (int c = 0; c < CW; ++c) w[m][c] = ws[m * 32 * CW + 32 * c + lane];
-      __syncwarp();                                        // all lanes have read the stage
+        for (int m = 0; m < 4; ++m)
+#pragma unroll
+          for (int c = 0; c < CW; ++c) w[m][c] = ws[m * 32 * CW + 32 * c + lane];
+        __syncwarp();                                      // all lanes have read the stage
+        off += C::STAGE;
+        if (off == BM_RING * C::STAGE) off = 0;
+#pragma unroll
+        for (int c = 0; c < CW; ++c) {
+          const uint32_t k0 = mag_key(w[0][c]), k1 = mag_key(w[1][c]), k2 = mag_key(w[2][c]), k3 = mag_key(w[3][c]);
+          const uint32_t valid = (cand[c] >> (4 * j)) & 15u;
+          const uint32_t e = lut[(valid << 6) | cmp6(k0, k1, k2, k3)];
+          vacc[c][j] = slots_signs(e, w[0][c], w[1][c], w[2][c], w[3][c], k0, k1, k2, k3);
+          kacc[c] |= ((e >> 16) & 15u) << (4 * j);
+          cacc[c] |= ((e >> 24) & 15u) << (4 * j);
+        }
+      }
+      primed = active_n;
+      // results into the staging tile: 32 bytes of each operand row, its code word, and the mask words by row
 #pragma unroll
       for (int c = 0; c < CW; ++c) {
-        const uint32_t k0 = mag_key(w[0][c]), k1 = mag_key(w[1][c]), k2 = mag_key(w[2][c]), k3 = mag_key(w[3][c]);
-        const uint32_t valid = (cand[c] >> (4 * j)) & 15u;
-        const uint2 e = lut[(valid << 6) | cmp6(k0, k1, k2, k3)];
-        vacc[c][j] = slots_masked(e, w[0][c], w[1][c], w[2][c], w[3][c], k0, k1, k2, k3);
-        kacc[c] |= ((e.x >> 16) & 15u) << (4 * j);
-        cacc[c] |= ((e.x >> 20) & 15u) << (4 * j);
+        const int col = (cti * CW + c) * 32 + lane;
+        uint4* dst = reinterpret_cast<uint4*>(sv + col * BM_SV_PITCH + 8 * rgi);
+        dst[0] = make_uint4(vacc[c][0], vacc[c][1], vacc[c][2], vacc[c][3]);
+        dst[1] = make_uint4(vacc[c][4], vacc[c][5], vacc[c][6], vacc[c][7]);
+        sc[col * 4 + rgi] = cacc[c];
+        sm[(32 * rgi + lane) * (2 * CW) + cti * CW + c] = transpose32(kacc[c], lane);
       }
     }
-    // this warp's 32 permuted rows of backward-mask words: one store of CW words per lane
-    uint32_t* mrow_out = maskbits_b + (size_t)(32 * rg + lane) * jwords + ct * CW;
-    if (CW == 2) *reinterpret_cast<uint2*>(mrow_out) = make_uint2(transpose32(kacc[0], lane), transpose32(kacc[1], lane));
-    else *mrow_out = transpose32(kacc[0], lane);
+    __syncthreads();
+    // ---- the CTA writes the tile out in whole lines ----
+    const int rg0 = 4 * tr, item0 = 2 * tc;
+    const int rgs_here = min(4, nrg - rg0), items_here = min(2, items - item0);
+    const int col0 = item0 * 32 * CW, cols_here = items_here * 32 * CW;
 #pragma unroll
-    for (int c = 0; c < CW; ++c) {
-      const int l = (ct * CW + c) * 32 + lane;
-      uint4* dst = reinterpret_cast<uint4*>(vals_b + (size_t)l * vrow + 8 * rg);
-      dst[0] = make_uint4(vacc[c][0], vacc[c][1], vacc[c][2], vacc[c][3]);
-      dst[1] = make_uint4(vacc[c][4], vacc[c][5], vacc[c][6], vacc[c][7]);
-      meta_b[(size_t)l * mrow + rg] = cacc[c];
-      if (hw32) {
-        // image word (rows l and l ^ 8 of the operand, k word rg): its low-half lane stores the two low halves of
-        // the code words, its high-half lane the two high halves
-        const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, cacc[c], 8);
-        const int rr = l & 127;
-        const size_t tile = (size_t)(l >> 7) * (I >> 7) + (rg >> 2);
-        const size_t at = tile * 512 + (size_t)((rr & 7) + 16 * (rr >> 4)) * 4 + (rg & 3);
-        if (rr & 8) hw32[at + 32] = __byte_perm(other, cacc[c], 0x7632u);
-        else hw32[at] = __byte_perm(cacc[c], other, 0x5410u);
+    for (int it = 0; it < C::COLS * 8 / BM_THREADS; ++it) {
+      const int idx = it * BM_THREADS + threadIdx.x;       // (column, 16-byte chunk of its 128 bytes)
+      const int col = idx >> 3, chunk = idx & 7;
+      if (col < cols_here && (chunk >> 1) < rgs_here)
+        *reinterpret_cast<uint4*>(vals_b + (size_t)(col0 + col) * vrow + 8 * rg0 + 4 * chunk) =
+            *reinterpret_cast<const uint4*>(sv + col * BM_SV_PITCH + 4 * chunk);
+    }
+    if (threadIdx.x < 128) {                               // backward-mask words of row rg0 * 32 + threadIdx.x
+      const int row = threadIdx.x;
+      if (row < 32 * rgs_here) {
+        uint32_t* dst = maskbits_b + (size_t)(32 * rg0 + row) * jwords + item0 * CW;
+        const uint32_t* src = sm + row * (2 * CW);
+        if (CW == 2 && (jwords & 3) == 0) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+        else if ((jwords & 1) == 0 && items_here * CW >= 2) {
+#pragma unroll
+          for (int q = 0; q < CW; ++q)
+            if (2 * q < items_here * CW) reinterpret_cast<uint2*>(dst)[q] = reinterpret_cast<const uint2*>(src)[q];
+        } else {
+          for (int q = 0; q < items_here * CW; ++q) dst[q] = src[q];
+        }
+      }
+    } else {                                               // code words of operand row col0 + (threadIdx.x - 128)
+      for (int col = threadIdx.x - 128; col < cols_here; col += 128) {
+        uint32_t* dst = meta_b + (size_t)(col0 + col) * mrow + rg0;
+        const uint32_t* src = sc + col * 4;
+        if (rgs_here == 4 && (mrow & 3) == 0) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+        else for (int q = 0; q < rgs_here; ++q) dst[q] = src[q];
       }
     }
-    if (!has_next) break;
-    item += nw;
-    rg = rg_n;
-    ct = ct_n;
+    if (hw32) {
+      // tensor-memory image (I and J multiples of 128): the tile's codes fill a contiguous run of the 2048-byte
+      // block (operand rows col0 .., k words rg0 ..): image lane L = m0 + 8 h + 16 m2 holds half h of the code
+      // words of rows m0 + 16 m2 (low 16 bits) and m0 + 8 + 16 m2 (high 16 bits)
+      uint32_t* blk = hw32 + ((size_t)(col0 >> 7) * (I >> 7) + tr) * 512 + (col0 & 127) * 4;
+#pragma unroll
+      for (int it = 0; it < C::COLS * 4 / BM_THREADS; ++it) {
+        const int idx = it * BM_THREADS + threadIdx.x;
+        const int L = idx >> 2, kc = idx & 3;
+        const int r_lo = (L & 7) + 16 * (L >> 4);
+        const uint32_t lo = sc[r_lo * 4 + kc], hi = sc[(r_lo + 8) * 4 + kc];
+        blk[idx] = __byte_perm(lo, hi, (L & 8) ? 0x7632u : 0x5410u);
+      }
+    }
+    __syncthreads();                                       // the staging tile is free again
   }
   cp_async_wait<0>();
 }
@@ -403,25 +466,25 @@ int launch_hw_meta(const uint32_t* meta, int rows, int K, void* hw_meta, cudaStr
 int launch_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                     int N, uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_or_null,
                     cudaStream_t s) {
-  // 64-column items once they keep every resident warp busy, 32-column items (twice as many) otherwise
-  const long long items_wide = (long long)(I / 32) * (J / 64);
-  const bool wide = J % 64 == 0 && items_wide >= (long long)BM_CTAS_PER_SM * 148 * BM_WARPS;
-  const int col_tiles = wide ? J / 64 : J / 32;
-  const long long n_items = (long long)(I / 32) * col_tiles;
-  BIMASK_REQUIRE(n_items < (1ll << 31), BIMASK_EUNSUPPORTED, "bimask_bwd_mask: I * J = %lld is beyond the kernel's item index",
+  // tiles of 128 rows x 128 columns once they fill the resident CTAs, 128 x 64 (twice as many) otherwise
+  const long long tiles_r = (I / 32 + 3) / 4;
+  const bool wide = J % 64 == 0 && tiles_r * ((J / 64 + 1) / 2) >= (long long)BM_CTAS_PER_SM * 148;
+  const int items = wide ? J / 64 : J / 32;
+  const int tiles_c = (items + 1) / 2;
+  const long long n_tiles = tiles_r * tiles_c;
+  BIMASK_REQUIRE(n_tiles < (1ll << 30), BIMASK_EUNSUPPORTED, "bimask_bwd_mask: I * J = %lld is beyond the kernel's tile index",
                  (long long)I * J);
-  long long ctas = (n_items + BM_WARPS - 1) / BM_WARPS;
-  if (ctas > BM_CTAS_PER_SM * 148) ctas = BM_CTAS_PER_SM * 148;
+  const long long ctas = n_tiles < BM_CTAS_PER_SM * 148 ? n_tiles : BM_CTAS_PER_SM * 148;
   uint32_t* vals32 = reinterpret_cast<uint32_t*>(vals_b);
   uint32_t* hw32 = reinterpret_cast<uint32_t*>(hw_meta_or_null);
   if (wide) {
     if (int rc = set_smem_attr(bwd_mask_kernel<2>, BMCfg<2>::SMEM)) return rc;
     BIMASK_CUDA_OK(launch_pdl(bwd_mask_kernel<2>, (unsigned)ctas, BM_THREADS, BMCfg<2>::SMEM, s, W, maskbits_f, perm, I, J, N,
-                              maskbits_b, vals32, meta_b, hw32, col_tiles, (int)n_items));
+                              maskbits_b, vals32, meta_b, hw32, tiles_c, (int)n_tiles));
   } else {
     if (int rc = set_smem_attr(bwd_mask_kernel<1>, BMCfg<1>::SMEM)) return rc;
     BIMASK_CUDA_OK(launch_pdl(bwd_mask_kernel<1>, (unsigned)ctas, BM_THREADS, BMCfg<1>::SMEM, s, W, maskbits_f, perm, I, J, N,
-                              maskbits_b, vals32, meta_b, hw32, col_tiles, (int)n_items));
+                              maskbits_b, vals32, meta_b, hw32, tiles_c, (int)n_tiles));
   }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
