@@ -124,19 +124,170 @@ gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int q_log2, i
 }
 
 // ---------------------------------------------------------------------------------------
+// Candidate generation for I <= 16384: one CTA per candidate, every key hashed once, KPT keys per thread.
+// Counting sort on the top log2(I) bits as above, with three differences that matter on one SM:
+//  * one atomic per key: the histogram pass keeps the value the atomic returned (the key's arrival number in its
+//    bucket), so after the scan the key goes to start[bucket] + arrival without a second atomic;
+//  * the order inside a bucket is settled by ranking, not by a per-bucket insertion sort: every thread counts, for
+//    each of its keys, the keys of the same bucket that are smaller (buckets hold about one key);
+//  * shared memory holds one 32-bit word per key: the 32 - log2(I) hash bits that follow the bucket bits, then the
+//    row index.  Two keys of a bucket that agree in those hash bits (the eight lower hash bits are not stored) are
+//    compared on the full key, recomputed from the row index.
+// The counters are padded by one word per 32 so that the scan, where a thread walks a contiguous run of counters,
+// is free of bank conflicts.  The sorted row indices are collected in shared memory (in place of the counters) and
+// written out in one coalesced pass.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ int pad32(int b) { return b + (b >> 5); }
+
+// Position of the key `mine` (packed form) among the keys of its bucket, keys[lo, hi): ordered by the stored hash
+// bits, and by the full 64-bit key, recomputed from the row indices, where those agree.
+__device__ __noinline__ uint32_t rank_exact(const uint32_t* keys, uint32_t lo, uint32_t hi, uint32_t mine,
+                                            unsigned long long stream, int nb_log2) {
+  const uint32_t idx_mask = (1u << nb_log2) - 1u;
+  uint32_t rank = lo;
+  for (uint32_t a = lo; a < hi; ++a) {
+    const uint32_t o = keys[a];
+    if (((o ^ mine) >> nb_log2) != 0u || o == mine) {
+      rank += o < mine;
+    } else {
+      const unsigned long long oi = o & idx_mask, mi = mine & idx_mask;
+      const unsigned long long vo = (mix64(stream ^ oi) & ~0xFFFFFFull) | oi;
+      const unsigned long long vm = (mix64(stream ^ mi) & ~0xFFFFFFull) | mi;
+      rank += vo < vm;
+    }
+  }
+  return rank;
+}
+
+template <int KPT>
+__global__ void __launch_bounds__(1024)
+gen_candidates_reg_kernel(unsigned long long seed, int I, int nb_log2, int32_t* __restrict__ cands,
+                          unsigned long long* __restrict__ zero_counts, int32_t* __restrict__ zero_ticket) {
+  pdl_launch_dependents();                               // the candidates depend on the seed alone: no wait up here
+  extern __shared__ uint32_t gen_smem[];                 // I packed keys, then the padded bucket counters
+  const int nb = 1 << nb_log2;
+  uint32_t* keys = gen_smem;
+  uint32_t* count = gen_smem + I;
+  __shared__ uint32_t warp_sums[32];
+  const int c = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthreads = blockDim.x, nwarps = nthreads >> 5;
+  const unsigned long long stream = mix64(seed + 0x9E3779B97F4A7C15ull * (unsigned long long)(c + 1));
+  const int shift = 64 - nb_log2;
+  const uint32_t idx_mask = (1u << nb_log2) - 1u;
+  for (int b = tid; b < nb + (nb >> 5); b += nthreads) count[b] = 0;
+  __syncthreads();
+  uint32_t k32[KPT], where[KPT];                         // packed key; bucket << 16 | arrival, later the final position
+#pragma unroll
+  for (int q = 0; q < KPT; ++q) {
+    const int i = tid + q * nthreads;
+    const unsigned long long v = (mix64(stream ^ (unsigned long long)i) & ~0xFFFFFFull) | (unsigned long long)i;
+    const uint32_t b = (uint32_t)(v >> shift);
+    k32[q] = ((uint32_t)((v << nb_log2) >> 32) & ~idx_mask) | (uint32_t)i;
+    where[q] = 0u;
+    if (i < I) where[q] = (b << 16) | atomicAdd(&count[pad32(b)], 1u);
+  }
+  __syncthreads();
+  // exclusive scan of the counters: each thread owns a contiguous run
+  const int per = (nb + nthreads - 1) / nthreads;
+  const int b0 = tid * per;
+  uint32_t local = 0;
+  for (int b = b0; b < min(nb, b0 + per); ++b) local += count[pad32(b)];
+  uint32_t incl = local;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+    if (lane >= d) incl += t;
+  }
+  if (lane == 31) warp_sums[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t ws = lane < nwarps ? warp_sums[lane] : 0u;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, ws, d);
+      if (lane >= d) ws += t;
+    }
+    if (lane < nwarps) warp_sums[lane] = ws;
+  }
+  __syncthreads();
+  uint32_t run = incl - local + (warp > 0 ? warp_sums[warp - 1] : 0u);
+  for (int b = b0; b < min(nb, b0 + per); ++b) {
+    const uint32_t n = count[pad32(b)];
+    count[pad32(b)] = run;                                // start of bucket b
+    run += n;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int q = 0; q < KPT; ++q) {
+    const int i = tid + q * nthreads;
+    if (i < I) keys[count[pad32(where[q] >> 16)] + (where[q] & 0xFFFFu)] = k32[q];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int q = 0; q < KPT; ++q) {
+    const int i = tid + q * nthreads;
+    if (i < I) {
+      const int b = (int)(where[q] >> 16);
+      const uint32_t lo = count[pad32(b)], hi = b + 1 < nb ? count[pad32(b + 1)] : (uint32_t)I;
+      // the first six keys of the bucket without a loop (a bucket holds one key on average); longer buckets and
+      // keys that agree in the stored hash bits take the exact walk
+      uint32_t rank = lo;
+      bool again = hi - lo > 6u;
+#pragma unroll
+      for (uint32_t t = 0; t < 6u; ++t) {
+        if (lo + t < hi) {
+          const uint32_t o = keys[lo + t];
+          rank += o < k32[q];
+          again |= ((o ^ k32[q]) >> nb_log2) == 0u && o != k32[q];
+        }
+      }
+      if (again) rank = rank_exact(keys, lo, hi, k32[q], stream, nb_log2);
+      where[q] = rank;
+    }
+  }
+  __syncthreads();                                       // every thread has read the bucket starts
+  int32_t* sorted = reinterpret_cast<int32_t*>(count);   // more than I entries
+#pragma unroll
+  for (int q = 0; q < KPT; ++q) {
+    const int i = tid + q * nthreads;
+    if (i < I) sorted[where[q]] = i;
+  }
+  __syncthreads();
+  pdl_wait();                                            // first global access: earlier kernels may still read these buffers
+  if (tid == 0) {
+    if (zero_counts) zero_counts[c] = 0ull;
+    if (c == 0 && zero_ticket) *zero_ticket = 0;
+  }
+  int32_t* out = cands + (long long)c * I;
+  if ((I & 3) == 0) {
+    for (int i = tid; i < (I >> 2); i += nthreads) reinterpret_cast<int4*>(out)[i] = reinterpret_cast<const int4*>(sorted)[i];
+  } else {
+    for (int i = tid; i < I; i += nthreads) out[i] = sorted[i];
+  }
+}
+
+// ---------------------------------------------------------------------------------------
 // Pick: arg-max of counts with ties to the lowest candidate index, then copy that candidate.
 // ---------------------------------------------------------------------------------------
 constexpr int PICK_THREADS = 256;
 
 // One CTA of PICK_THREADS threads; counts are read around L1 (they were written by atomics of other CTAs).
-__device__ __forceinline__ void pick_body(const long long* counts, const int32_t* __restrict__ cands, int P, int I,
+// PACKED: bits [48,64) of a count hold the number of CTAs that have added their share (the fused pick of the count
+// kernel); they are stripped here and the plain count is written back.
+constexpr unsigned long long COUNT_MASK = (1ull << 48) - 1ull;
+template <bool PACKED>
+__device__ __forceinline__ void pick_body(long long* counts, const int32_t* __restrict__ cands, int P, int I,
                                           int32_t* best_idx, int32_t* __restrict__ best_perm) {
   __shared__ long long s_cnt[PICK_THREADS];
   __shared__ int s_idx[PICK_THREADS];
   long long bc = -1;
   int bi = 0x7FFFFFFF;
   for (int c = threadIdx.x; c < P; c += PICK_THREADS) {
-    const long long v = __ldcg(counts + c);
+    long long v = __ldcg(counts + c);
+    if (PACKED) {
+      v = (long long)((unsigned long long)v & COUNT_MASK);
+      counts[c] = v;
+    }
     if (v > bc) { bc = v; bi = c; }      // ascending c per thread: first maximum is kept
   }
   s_cnt[threadIdx.x] = bc;
@@ -155,7 +306,13 @@ __device__ __forceinline__ void pick_body(const long long* counts, const int32_t
   }
   const int best = s_idx[0];
   if (threadIdx.x == 0) *best_idx = best;
-  for (int i = threadIdx.x; i < I; i += PICK_THREADS) best_perm[i] = cands[(long long)best * I + i];
+  const int32_t* src = cands + (long long)best * I;
+  if ((I & 3) == 0) {
+    for (int i = threadIdx.x; i < (I >> 2); i += PICK_THREADS)
+      reinterpret_cast<int4*>(best_perm)[i] = __ldg(reinterpret_cast<const int4*>(src) + i);
+  } else {
+    for (int i = threadIdx.x; i < I; i += PICK_THREADS) best_perm[i] = src[i];
+  }
 }
 
 __global__ void __launch_bounds__(PICK_THREADS)
@@ -163,7 +320,7 @@ pick_kernel(const long long* __restrict__ counts, const int32_t* __restrict__ ca
             int32_t* __restrict__ best_idx, int32_t* __restrict__ best_perm) {
   pdl_launch_dependents();
   pdl_wait();
-  pick_body(counts, cands, P, I, best_idx, best_perm);
+  pick_body<false>(const_cast<long long*>(counts), cands, P, I, best_idx, best_perm);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -173,7 +330,7 @@ pick_kernel(const long long* __restrict__ counts, const int32_t* __restrict__ ca
 // four bits hold at most N ones.  One 64-bit atomic per CTA.
 // ---------------------------------------------------------------------------------------
 constexpr int SCORE_THREADS = 256;
-constexpr int SCORE_KB_PER_CTA = 64;
+constexpr int SCORE_KB_MAX = 256;                      // row blocks of one candidate per CTA: 32 .. 256, chosen by the launcher
 
 // Columns (bits) where more than N of the four rows are set.  a + b + c = 2 * maj + par (a full adder per bit,
 // two three-input logic operations); adding d: at least two  <=>  maj | (par & d), at least three  <=>
@@ -190,27 +347,27 @@ __device__ __forceinline__ uint32_t ineligible(uint32_t a, uint32_t b, uint32_t 
 
 template <int N>
 __global__ void __launch_bounds__(SCORE_THREADS, 4)
-score_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cands, int I, int jwords,
+score_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cands, int I, int jwords, int kb_per_cta,
              unsigned long long* __restrict__ counts, int P, int32_t* best_idx, int32_t* __restrict__ best_perm) {
   pdl_launch_dependents();
   pdl_wait();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int c = blockIdx.y;
   const int nkb = I >> 2;
-  const int kb0 = blockIdx.x * SCORE_KB_PER_CTA;
-  const int kb1 = min(nkb, kb0 + SCORE_KB_PER_CTA);
+  const int kb0 = blockIdx.x * kb_per_cta;
+  const int kb1 = min(nkb, kb0 + kb_per_cta);
   const int4* cand4 = reinterpret_cast<const int4*>(cands + (long long)c * I);
   uint32_t cnt = 0;
   if ((jwords & 3) == 0) {
     const int jq = jwords >> 2;
     // the CTA's row indices first (one coalesced load, clamped), so that the row loads below do
     // not wait on a dependent global load
-    __shared__ int4 idx_s[SCORE_KB_PER_CTA];
+    __shared__ int4 idx_s[SCORE_KB_MAX];
     const unsigned last_row = (unsigned)(I - 1);
-    if (threadIdx.x < kb1 - kb0) {
-      const int4 r = __ldg(cand4 + kb0 + threadIdx.x);
-      idx_s[threadIdx.x] = make_int4((int)min((unsigned)r.x, last_row), (int)min((unsigned)r.y, last_row),
-                                     (int)min((unsigned)r.z, last_row), (int)min((unsigned)r.w, last_row));
+    for (int t = threadIdx.x; t < kb1 - kb0; t += SCORE_THREADS) {
+      const int4 r = __ldg(cand4 + kb0 + t);
+      idx_s[t] = make_int4((int)min((unsigned)r.x, last_row), (int)min((unsigned)r.y, last_row),
+                           (int)min((unsigned)r.z, last_row), (int)min((unsigned)r.w, last_row));
     }
     __syncthreads();
     // two row blocks per trip: eight independent 128-bit loads in flight per lane
@@ -261,20 +418,24 @@ score_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cand
     unsigned long long s = 0;
 #pragma unroll
     for (int w = 0; w < SCORE_THREADS / 32; ++w) s += part[w];
-    atomicAdd(counts + c, s);
     last_cta = false;
     if (best_idx) {
-      // fused pick: *best_idx counts the CTAs that have added their share (zeroed before the launch); the CTA that
-      // completes the grid sees every sum (fence on both sides of the counter) and picks the winner
-      __threadfence();
-      const unsigned done = atomicAdd(reinterpret_cast<unsigned*>(best_idx), 1u);
-      last_cta = done == gridDim.x * gridDim.y - 1u;
+      // fused pick: the sum travels with a one in bits [48,64), so the count word also tells how many CTAs of this
+      // candidate have reported; the CTA that completes a candidate bumps *best_idx (zeroed before the launch), and
+      // the one that completes the last candidate sees every sum (fence on both sides of the counters) and picks
+      const unsigned long long old = atomicAdd(counts + c, s + (1ull << 48));
+      if ((unsigned)(old >> 48) + 1u == gridDim.x) {
+        __threadfence();
+        last_cta = atomicAdd(reinterpret_cast<unsigned*>(best_idx), 1u) == gridDim.y - 1u;
+      }
+    } else {
+      atomicAdd(counts + c, s);
     }
   }
   __syncthreads();
   if (last_cta) {
     __threadfence();
-    pick_body(reinterpret_cast<const long long*>(counts), cands, P, I, best_idx, best_perm);
+    pick_body<true>(reinterpret_cast<long long*>(counts), cands, P, I, best_idx, best_perm);
   }
 }
 
@@ -306,6 +467,26 @@ int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStrea
                           int32_t* zero_ticket) {
   int lg = 1;
   while ((1 << lg) < I) ++lg;                             // one bucket per key on average
+  unsigned long long* zc = reinterpret_cast<unsigned long long*>(zero_counts);
+  if (I <= 16384) {
+    // a CTA per candidate with the keys in registers: 4, 8 or 16 per thread
+    const int kpt = I <= 4096 ? 4 : I <= 8192 ? 8 : 16;
+    int threads = ((I + kpt - 1) / kpt + 31) / 32 * 32;
+    const size_t smem = ((size_t)I + ((size_t)1 << lg) + ((size_t)1 << lg >> 5) + 4) * sizeof(uint32_t);
+    if (kpt == 4) {
+      if (int rc = set_smem_attr(gen_candidates_reg_kernel<4>, 200 * 1024)) return rc;
+      BIMASK_CUDA_OK(launch_pdl(gen_candidates_reg_kernel<4>, P, threads, smem, s, (unsigned long long)seed, I, lg, cands, zc, zero_ticket));
+    } else if (kpt == 8) {
+      if (int rc = set_smem_attr(gen_candidates_reg_kernel<8>, 200 * 1024)) return rc;
+      BIMASK_CUDA_OK(launch_pdl(gen_candidates_reg_kernel<8>, P, threads, smem, s, (unsigned long long)seed, I, lg, cands, zc, zero_ticket));
+    } else {
+      if (int rc = set_smem_attr(gen_candidates_reg_kernel<16>, 200 * 1024)) return rc;
+      BIMASK_CUDA_OK(launch_pdl(gen_candidates_reg_kernel<16>, P, threads, smem, s, (unsigned long long)seed, I, lg, cands, zc, zero_ticket));
+    }
+    count_launch();
+    BIMASK_CUDA_OK(cudaGetLastError());
+    return BIMASK_OK;
+  }
   int ql = 0;
   while ((I >> ql) > 8192 && ql < lg - 1) ++ql;           // at most 8192 keys per part (measured best)
   const int mean = (I + (1 << ql) - 1) >> ql;
@@ -314,7 +495,7 @@ int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStrea
   if (int rc = set_smem_attr(gen_candidates_kernel, 200 * 1024)) return rc;
   dim3 grid(P, 1 << ql);
   BIMASK_CUDA_OK(launch_pdl(gen_candidates_kernel, grid, GEN_THREADS, smem, s, (unsigned long long)seed, I, lg, ql, cap, cands,
-                                                        reinterpret_cast<unsigned long long*>(zero_counts), zero_ticket));
+                                                        zc, zero_ticket));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -325,12 +506,14 @@ int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStrea
 // candidate generator.
 int launch_score(const uint32_t* maskbits_f, const int32_t* cands, int I, int J, int N, int P,
                  int64_t* counts, cudaStream_t s, bool zeroed, int32_t* best_idx, int32_t* best_perm) {
-  dim3 grid((I / 4 + SCORE_KB_PER_CTA - 1) / SCORE_KB_PER_CTA, P);
-  // The fused pick costs every CTA a fence and an atomic on one counter: a win for small grids (it saves a launch
-  // of a few microseconds), a loss for thousands of CTAs (measured: +8 us on 2048 CTAs, +24 us on 8192), which keep the
-  // separate pick kernel.
+  // row blocks per CTA: as many as still give every SM a dozen CTAs (fewer, longer CTAs start and drain less often)
+  const int nkb = I / 4;
+  int kb = SCORE_KB_MAX;
+  while (kb > 32 && (long long)P * ((nkb + kb - 1) / kb) < 12 * 148) kb >>= 1;
+  dim3 grid((nkb + kb - 1) / kb, P);
+  // the fused pick counts a candidate's CTAs in 16 bits of its count word and needs sums below 2^48
   int32_t* pick_idx = best_idx, *pick_perm = best_perm;
-  const bool fuse = best_idx != nullptr && (long long)grid.x * grid.y <= 1024;
+  const bool fuse = best_idx != nullptr && grid.x <= 65535u && (long long)nkb * J < (1ll << 48);
   if (!fuse) best_idx = nullptr;
   if (!zeroed) {
     BIMASK_CUDA_OK(cudaMemsetAsync(counts, 0, (size_t)P * sizeof(int64_t), s));
@@ -338,10 +521,10 @@ int launch_score(const uint32_t* maskbits_f, const int32_t* cands, int I, int J,
   }
   unsigned long long* cnt = reinterpret_cast<unsigned long long*>(counts);
   switch (N) {
-    case 1: BIMASK_CUDA_OK(launch_pdl(score_kernel<1>, grid, SCORE_THREADS, 0, s, maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm)); break;
-    case 2: BIMASK_CUDA_OK(launch_pdl(score_kernel<2>, grid, SCORE_THREADS, 0, s, maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm)); break;
-    case 3: BIMASK_CUDA_OK(launch_pdl(score_kernel<3>, grid, SCORE_THREADS, 0, s, maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm)); break;
-    default: BIMASK_CUDA_OK(launch_pdl(score_kernel<4>, grid, SCORE_THREADS, 0, s, maskbits_f, cands, I, J / 32, cnt, P, best_idx, best_perm)); break;
+    case 1: BIMASK_CUDA_OK(launch_pdl(score_kernel<1>, grid, SCORE_THREADS, 0, s, maskbits_f, cands, I, J / 32, kb, cnt, P, best_idx, best_perm)); break;
+    case 2: BIMASK_CUDA_OK(launch_pdl(score_kernel<2>, grid, SCORE_THREADS, 0, s, maskbits_f, cands, I, J / 32, kb, cnt, P, best_idx, best_perm)); break;
+    case 3: BIMASK_CUDA_OK(launch_pdl(score_kernel<3>, grid, SCORE_THREADS, 0, s, maskbits_f, cands, I, J / 32, kb, cnt, P, best_idx, best_perm)); break;
+    default: BIMASK_CUDA_OK(launch_pdl(score_kernel<4>, grid, SCORE_THREADS, 0, s, maskbits_f, cands, I, J / 32, kb, cnt, P, best_idx, best_perm)); break;
   }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
