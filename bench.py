@@ -44,45 +44,62 @@ def load_peaks():
 # --------------------------------------------------------------------------------------------
 # CPU oracle arm (reference / cpu_baseline)
 # --------------------------------------------------------------------------------------------
+ORACLE_PARTS = ("fwd_mask_pack", "candidates", "scoring", "bwd_mask_pack", "spmm_fwd", "spmm_dgrad", "wgrad")
+
+
 def oracle_sample_time(cfg_id: int, rows: int = 1024, tokens: int = 256, cands: int = 4):
-    """Times the CPU oracle, as it stands, on a bounded sample of every layer of the config
-    (the first `rows` rows of W with the full input dim, `tokens` tokens, `cands` candidates) and
-    scales each part by its own work ratio to the full layer.  Returns (seconds for a full pass
-    over all layers [extrapolated], seconds actually spent, description)."""
+    """Times the CPU oracle, as it stands, on a bounded sample of every layer of the config (the first `rows` rows
+    of W with the full input dim, `tokens` tokens, `cands` candidates), one timer per kind of step (the two mask
+    passes, candidate generation, scoring, the three products), and scales each kind by its own work ratio to the
+    full layer.  Returns (seconds for a full pass over all layers [extrapolated], seconds actually spent,
+    description, per-kind record)."""
     from oracle import bimask_oracle as O
     from paper_2302_06058_b200 import inputs
     cfg = inputs.CONFIGS[cfg_id]
     total_full = 0.0
     spent = 0.0
+    parts = {k: {"sample_s": 0.0, "full_s": 0.0} for k in ORACLE_PARTS}
+    scales = []
     for li, L in enumerate(cfg.layers):
         Is, Ts, Ps = min(rows, L.I), min(tokens, L.T), min(cands, cfg.P)
         W = inputs.make_weight(Is, L.J, 1000 * cfg_id + 10 * li, cfg.init)
         X = inputs.make_activation(Ts, L.J, 1000 * cfg_id + 10 * li + 1)
         dY = inputs.make_activation(Ts, Is, 1000 * cfg_id + 10 * li + 2)
-        t0 = time.perf_counter()
+        t = [time.perf_counter()]
         B = O.forward_mask(W, cfg.N, cfg.M)
         O.forward_operand(W, B)
-        t1 = time.perf_counter()
+        t.append(time.perf_counter())
         cand = O.candidates(inputs.perm_seed(cfg_id), Ps, Is)
+        t.append(time.perf_counter())
         _, perm, _ = O.perm_search(B, cand, cfg.N, cfg.M)
-        t2 = time.perf_counter()
+        t.append(time.perf_counter())
         Bbar = O.backward_mask(W, B, perm, cfg.N, cfg.M)
         Mb = O.unpermute_rows(Bbar, perm)
         O.backward_operand(W, Bbar, perm)
-        t3 = time.perf_counter()
+        t.append(time.perf_counter())
         O.spmm_fwd(X, W, B)
+        t.append(time.perf_counter())
         O.spmm_dgrad(dY, W, Mb)
+        t.append(time.perf_counter())
         O.wgrad(dY, X)
-        t4 = time.perf_counter()
+        t.append(time.perf_counter())
         r_mask = (L.I * L.J) / (Is * L.J)
-        r_search = (cfg.P * L.I * L.J) / (Ps * Is * L.J)
+        r_cand = (cfg.P * L.I) / (Ps * Is)
+        r_score = (cfg.P * L.I * L.J) / (Ps * Is * L.J)
         r_gemm = (L.T * L.I * L.J) / (Ts * Is * L.J)
-        total_full += ((t1 - t0) + (t3 - t2)) * r_mask + (t2 - t1) * r_search + (t4 - t3) * r_gemm
-        spent += t4 - t0
+        ratio = dict(zip(ORACLE_PARTS, (r_mask, r_cand, r_score, r_mask, r_gemm, r_gemm, r_gemm)))
+        for k, name in enumerate(ORACLE_PARTS):
+            dt = t[k + 1] - t[k]
+            parts[name]["sample_s"] += dt
+            parts[name]["full_s"] += dt * ratio[name]
+            total_full += dt * ratio[name]
+        scales.append({"layer": li, "masks": r_mask, "candidates": r_cand, "scoring": r_score, "products": r_gemm})
+        spent += t[-1] - t[0]
     desc = (f"config {cfg_id}: per layer the first {rows} rows of W (full input dim), {tokens} tokens, "
-            f"{cands} candidates; masks, search and GEMMs timed separately and each scaled by its work "
-            f"ratio to the full layer (extrapolated)")
-    return total_full, spent, desc
+            f"{cands} candidates; every kind of step timed separately and scaled by its work ratio to the full "
+            f"layer (extrapolated)")
+    extrapolated = any(abs(v - 1.0) > 1e-9 for sc in scales for k, v in sc.items() if k != "layer")
+    return total_full, spent, desc, {"parts": parts, "scale_factors": scales, "extrapolated": extrapolated}
 
 
 def cpu_threads() -> int:
@@ -117,7 +134,7 @@ def run_reference(args):
         rows = int(last_rows * (share / max(last_cost, 1e-3)) ** 0.75) // 32 * 32
         rows = max(128, min(args.ref_rows, rows))
         t0 = time.perf_counter()
-        full, _, desc = oracle_sample_time(args.config, rows=rows, tokens=args.ref_tokens, cands=2)
+        full, _, desc, detail = oracle_sample_time(args.config, rows=rows, tokens=args.ref_tokens, cands=2)
         last_rows, last_cost = rows, time.perf_counter() - t0
         per_pass.append(full)
         rows_used.append(rows)
@@ -132,7 +149,9 @@ def run_reference(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": f"config {args.config} ({cfg.name})", "layers": [[L.I, L.J, L.T] for L in cfg.layers],
                    "N": cfg.N, "M": cfg.M, "P": cfg.P},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc,
+                         "extrapolated": detail["extrapolated"], "scale_factors": detail["scale_factors"],
+                         "parts_last_step": detail["parts"]},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0, "wall_s": wall,
     }
@@ -162,17 +181,29 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
-    def stop(self, t_begin=None, t_end=None):
-        """Stop sampling; summarise the samples whose timestamp lies in [t_begin, t_end] (time.time())."""
-        import datetime
-        out = {"sm_mhz": None, "sm_max_mhz": None, "power_w": None, "reasons": [], "samples": 0}
+    def stop(self):
+        """Stop sampling (the samples stay on disk for window())."""
         if self.proc is None:
-            return out
+            return
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
+        self.proc = None
+
+    def close(self):
+        try:
+            os.unlink(self.path)
+        except Exception:
+            pass
+
+    def window(self, t_begin=None, t_end=None):
+        """Summary of the samples whose timestamp lies in [t_begin, t_end] (time.time())."""
+        import datetime
+        out = {"sm_mhz": None, "sm_max_mhz": None, "power_w": None, "reasons": [], "samples": 0}
+        if self.path is None:
+            return out
         sm, mx, pw, reasons = [], [], [], set()
         try:
             with open(self.path) as f:
@@ -193,7 +224,6 @@ class ClockSampler:
                     for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[4:8]):
                         if v.lower().startswith("active"):
                             reasons.add(name)
-            os.unlink(self.path)
         except Exception:
             pass
         if sm:
@@ -205,22 +235,54 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------
 # GPU arm
 # --------------------------------------------------------------------------------------------
-# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM kernels on
-# config 5, from the ncu launch list summarised in profiles/cfg5_launch_list.md (GEMM kernel only).
+# DRAM traffic per call (dram__bytes_read.sum + dram__bytes_write.sum over the kernels of the call, one ncu capture
+# of `bench.py --profile` per layer of config 5); the capture is named in the JSON line beside the numbers.
+NCU_TRAFFIC_SOURCE = "profiles/cfg5_dram_traffic.md"
 NCU_TRAFFIC_BYTES = {
-    (5, 0, "wgrad"): 1.274e9 + 0.247e9, (5, 1, "wgrad"): 1.003e9 + 0.247e9,
-    (5, 0, "spmm_fwd"): 0.616e9 + 0.239e9, (5, 1, "spmm_fwd"): 0.703e9 + 0.054e9,
-    (5, 0, "spmm_dgrad"): 0.703e9 + 0.051e9, (5, 1, "spmm_dgrad"): 0.620e9 + 0.240e9,
+    (5, 0, "fwd_mask"): 268.5e6 + 63.8e6, (5, 1, "fwd_mask"): 268.7e6 + 63.3e6,
+    (5, 0, "spmm_fwd"): 616.3e6 + 239.3e6, (5, 1, "spmm_fwd"): 702.6e6 + 50.6e6,
+    (5, 0, "perm_search"): 16.9e6, (5, 1, "perm_search"): 10.5e6,          # generator + count kernel
+    (5, 0, "bwd_mask"): 277.3e6 + 61.9e6, (5, 1, "bwd_mask"): 277.5e6 + 60.9e6,
+    (5, 0, "spmm_dgrad"): 268.5e6 + 216.3e6 + 702.6e6 + 50.6e6,           # permute pass + product
+    (5, 1, "spmm_dgrad"): 67.1e6 + 19.6e6 + 615.4e6 + 239.4e6,
+    (5, 0, "wgrad"): 1392.4e6 + 247.7e6, (5, 1, "wgrad"): 1078.0e6 + 247.5e6,
 }
 
 
+def job_value(world: int, n_layers: int, steps: int, ms_max_over_ranks: float) -> float:
+    """Whole-job throughput of N independent replicas: every rank runs `steps` passes over `n_layers` layers, the
+    job takes as long as its slowest rank."""
+    return world * n_layers * steps / (ms_max_over_ranks * 1e-3)
+
+
+def max_over_ranks(values, world: int, device="cpu"):
+    """Element-wise maximum of a list of per-rank timings over all ranks (the only collective of the bench)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def clock_regime(clocks: dict, timed_region_s=None) -> str:
+    """"burst": the sampled SM clock (median) stayed near its maximum, and the timed region, when given, was too short
+    for the power cap to bite; "sustained" otherwise.  Decides which measured tensor peak a fraction is quoted
+    against."""
+    near_max = bool(clocks.get("sm_mhz")) and bool(clocks.get("sm_max_mhz")) and clocks["sm_mhz"] >= 0.9 * clocks["sm_max_mhz"]
+    if near_max and (timed_region_s is None or timed_region_s < 1.0):
+        return "burst"
+    return "sustained"
+
+
 def algorithmic_work(L, P):
-    """Algorithmic bytes / flops per launch of each timed call for one layer (see the design notes)."""
+    """Algorithmic bytes / flops per launch of each timed call for one layer."""
     I, J, T = L.I, L.J, L.T
     IJ = I * J
     return {
         "fwd_mask": {"bound": "hbm", "bytes": 4 * IJ + IJ + IJ / 8 + IJ / 8 + 2 * IJ / 8},
-        "perm_search": {"bound": "hbm", "bytes": 4 * IJ},      # time relative to one pass over W
+        # quoted against one HBM pass over W; the mask bits it really reads (P * IJ / 8 bytes) come out of L2
+        "perm_search": {"bound": "hbm", "bytes": 4 * IJ, "l2_bytes": P * IJ / 8},
         "bwd_mask": {"bound": "hbm", "bytes": 4 * IJ + IJ / 8 + 4 * I + IJ + IJ / 8 + IJ / 8 + 2 * IJ / 8},
         "spmm_fwd": {"bound": "tensor", "flops": 2.0 * T * IJ, "bytes": 2 * T * J + 1.125 * IJ + 2 * T * I},
         "spmm_dgrad": {"bound": "tensor", "flops": 2.0 * T * IJ, "bytes": 2 * T * I + 1.125 * IJ + 2 * T * J + 4 * T * I},
@@ -324,15 +386,16 @@ def run_gpu(args):
     for _ in range(max(args.warmup, 3)):
         step_fn()
     barrier()
-    t_load_begin = time.time()
     launches0 = bm.bimask_launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    t_head_begin = time.time()
     ev0.record(stream)
     for _ in range(args.steps):
         step_fn()
     ev1.record(stream)
     barrier()
+    t_head_end = time.time()
     step_ms_total = ev0.elapsed_time(ev1)
     launches = bm.bimask_launch_count() - launches0
     if graph is not None:
@@ -357,6 +420,7 @@ def run_gpu(args):
     # ---- per-call breakdown over the same K steps (CUDA events between the C-ABI calls) ----
     names = ["fwd_mask", "spmm_fwd", "perm_search", "bwd_mask", "spmm_dgrad", "wgrad"]
     acc = {li: {n: 0.0 for n in names} for li in range(len(layers))}
+    t_call_begin = time.time()
     for _ in range(args.steps):
         for li, (L, b, _) in enumerate(layers):
             ev = [torch.cuda.Event(enable_timing=True) for _ in range(7)]
@@ -380,14 +444,43 @@ def run_gpu(args):
             torch.cuda.synchronize()
             for k, n in enumerate(names):
                 acc[li][n] += ev[k].elapsed_time(ev[k + 1])
-    clocks = sampler.stop(t_load_begin, time.time())      # samples taken while the GPU was under this load
+    t_call_end = time.time()
+
+    # ---- the same step repeated back to back for --sustain-s seconds: the figure under the power cap ----
+    sustain_ms, sustain_steps, t_sus_begin, t_sus_end = 0.0, 0, None, None
+    if args.sustain_s > 0:
+        batch = max(1, int(0.25 / max(step_ms_total / args.steps * 1e-3, 1e-6)))      # about 0.25 s per batch
+        t_sus_begin = time.time()
+        batches = []
+        while time.time() - t_sus_begin < args.sustain_s:
+            es0, es1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            es0.record(stream)
+            for _ in range(batch):
+                step_fn()
+            es1.record(stream)
+            es1.synchronize()
+            batches.append(es0.elapsed_time(es1))
+        barrier()
+        t_sus_end = time.time()
+        tail = batches[len(batches) // 2:]                  # the second half: the clocks have settled
+        sustain_ms, sustain_steps = float(sum(tail)), batch * len(tail)
+
+    sampler.stop()
+    clocks = sampler.window(t_head_begin, t_head_end)     # samples taken inside the headline's timed region
+    clocks_calls = sampler.window(t_call_begin, t_call_end)
+    clocks_sustain = sampler.window(t_sus_begin + 0.5 * (t_sus_end - t_sus_begin), t_sus_end) if t_sus_begin else None
+    if not clocks["samples"]:                             # a timed region shorter than the sampling period
+        clocks = sampler.window(t_head_begin - 0.05, t_head_end + 0.05)
+    sampler.close()
     status = [int(b["status_word"].item()) for _, b, _ in layers]
     if any(status):
         raise RuntimeError(f"device status words non-zero: {status}")
 
-    # ---- roofline of every call, and of the dominant one ----
-    sparse_peak = 2.0 * peaks["bf16_tflops_sustained"]
-    dense_peak = peaks["bf16_tflops_sustained"]
+    # ---- roofline of every call, and of the dominant one.  A tensor-bound call is quoted against both measured
+    #      peaks (burst: a kernel timed alone at full clock; sustained: inside a long run under the power cap) and
+    #      `frac` is the one that matches the clocks sampled while the calls were timed. ----
+    regime = clock_regime(clocks, step_ms_total * 1e-3)
+    regime_calls = clock_regime(clocks_calls)
     kernels = []
     for li, (L, b, _) in enumerate(layers):
         work = algorithmic_work(L, cfg.P)
@@ -397,17 +490,39 @@ def run_gpu(args):
             entry = {"layer": li, "call": n, "ms": ms}
             if w["bound"] == "hbm":
                 entry.update(bound="hbm", achieved=w["bytes"] / (ms * 1e-3) / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
+                entry["frac"] = entry["achieved"] / entry["peak"]
+                if "l2_bytes" in w:
+                    # what the count kernel really moves: mask bits out of L2, against the rate at which 148 SMs can
+                    # take data from L2 (64 bytes per clock each) at the sampled clock
+                    mhz = clocks_calls.get("sm_mhz") or clocks_calls.get("sm_max_mhz") or 1965.0
+                    entry["l2_tbs"] = w["l2_bytes"] / (ms * 1e-3) / 1e12
+                    entry["l2_fill_peak_tbs"] = 148 * 64 * mhz * 1e6 / 1e12
+                    entry["l2_frac"] = entry["l2_tbs"] / entry["l2_fill_peak_tbs"]
             else:
-                pk = dense_peak if n == "wgrad" else sparse_peak
-                entry.update(bound="tensor", achieved=w["flops"] / (ms * 1e-3) / 1e12, peak=pk, unit="TFLOP/s")
-            entry["frac"] = entry["achieved"] / entry["peak"]
+                mult = 1.0 if n == "wgrad" else 2.0       # the 2:4 products: nominal sparse : dense ratio
+                entry.update(bound="tensor", achieved=w["flops"] / (ms * 1e-3) / 1e12, unit="TFLOP/s",
+                             peak_burst=mult * peaks["bf16_tflops"], peak_sustained=mult * peaks["bf16_tflops_sustained"])
+                entry["frac_burst"] = entry["achieved"] / entry["peak_burst"]
+                entry["frac_sustained"] = entry["achieved"] / entry["peak_sustained"]
+                entry["peak"] = entry["peak_burst"] if regime_calls == "burst" else entry["peak_sustained"]
+                entry["frac"] = entry["achieved"] / entry["peak"]
+            t = NCU_TRAFFIC_BYTES.get((args.config, li, n))
+            if t is not None:
+                entry["traffic"] = t
+                entry["algorithmic_bytes"] = w["bytes"]
             kernels.append(entry)
     dom = max(kernels, key=lambda e: e["ms"])
     roofline = {"bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"], "unit": dom["unit"],
-                "frac": dom["frac"], "traffic": NCU_TRAFFIC_BYTES.get((args.config, dom["layer"], dom["call"])),
-                "kernel": f"layer {dom['layer']} {dom['call']}",
-                "peak_source": peaks["source"] + (" (sustained bf16; x2 for the 2:4 sparse products)"
+                "frac": dom["frac"], "traffic": dom.get("traffic"),
+                "traffic_source": NCU_TRAFFIC_SOURCE if dom.get("traffic") is not None else None,
+                "kernel": f"layer {dom['layer']} {dom['call']}", "regime": regime_calls,
+                "peak_source": peaks["source"] + (f" ({regime_calls} bf16" + ("; x2 for the 2:4 sparse products)"
+                                                                              if dom["call"] != "wgrad" else ")")
                                                    if dom["bound"] == "tensor" else " (copy bandwidth)")}
+    if dom["bound"] == "tensor":
+        roofline.update(frac_burst=dom["frac_burst"], frac_sustained=dom["frac_sustained"])
+    if dom["frac"] > 1.05:
+        roofline["note"] = "fraction above 1: the kernel ran at a higher clock than the peak measurement; see frac_burst"
 
     # ---- end to end through the host-buffer entry point ----
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
@@ -469,16 +584,15 @@ def run_gpu(args):
         raise RuntimeError(f"device status words non-zero after the training iterations: {status}")
 
     # ---- max over ranks ----
-    t = torch.tensor([step_ms_total, e2e_ms, nosearch_ms_total, train_ms_total], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    step_ms_total, e2e_ms, nosearch_ms_total, train_ms_total = float(t[0]), float(t[1]), float(t[2]), float(t[3])
+    step_ms_total, e2e_ms, nosearch_ms_total, train_ms_total, sustain_ms = max_over_ranks(
+        [step_ms_total, e2e_ms, nosearch_ms_total, train_ms_total, sustain_ms], world, "cuda")
     nl = len(layers)
-    value = world * nl * args.steps / (step_ms_total * 1e-3)
-    e2e_value = world * nl * e2e_steps / (e2e_ms * 1e-3)
+    value = job_value(world, nl, args.steps, step_ms_total)
+    e2e_value = job_value(world, nl, e2e_steps, e2e_ms)
 
     if rank == 0:
-        cpu_full, cpu_spent, desc = oracle_sample_time(args.config, rows=args.ref_rows, tokens=args.ref_tokens, cands=2)
+        cpu_full, cpu_spent, desc, cpu_detail = oracle_sample_time(args.config, rows=args.ref_rows, tokens=args.ref_tokens,
+                                                                   cands=2)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": step_ms_total / args.steps, "higher_is_better": True,
@@ -488,7 +602,12 @@ def run_gpu(args):
                        "search_every_step": True, "parallelism": f"replicas x{world}", "cuda_graph": bool(args.graph),
                        "l2": "inputs larger than L2 (W alone is %.0f MB per layer)" % (cfg.layers[0].I * cfg.layers[0].J * 4 / 1e6)
                        if cfg.layers[0].I * cfg.layers[0].J * 4 > 126e6 else "inputs smaller than L2: warm-cache numbers"},
-            "clocks": clocks,
+            "clocks": clocks, "regime": regime, "clocks_per_call": clocks_calls,
+            "sustained": ({"value": job_value(world, nl, sustain_steps, sustain_ms), "unit": UNIT,
+                           "ms_per_step": sustain_ms / sustain_steps, "seconds": args.sustain_s, "steps": sustain_steps,
+                           "clocks": clocks_sustain,
+                           "note": "the same step back to back for --sustain-s seconds, second half of the run timed"}
+                          if sustain_steps else None),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "repetitions_ms": e2e_runs,
                     "api": "bimask_layer_step_host_async + bimask_host_sync (pinned host buffers)"},
@@ -505,7 +624,8 @@ def run_gpu(args):
             "roofline": roofline,
             "kernels": kernels,
             "cpu_baseline": {"value": nl / cpu_full, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
-                             "sample": desc, "cpu_seconds_spent": cpu_spent},
+                             "sample": desc, "cpu_seconds_spent": cpu_spent, "extrapolated": cpu_detail["extrapolated"],
+                             "scale_factors": cpu_detail["scale_factors"], "parts": cpu_detail["parts"]},
         }
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -655,6 +775,8 @@ def main():
     ap.add_argument("--config", type=int, default=5, help="workload: 1..5 (default 5, the largest)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--sustain-s", type=float, default=3.0,
+                    help="also repeat the step back to back for this many seconds and report that figure (0: skip)")
     ap.add_argument("--graph", action="store_true", help="replay one captured pass (CUDA graph) in the timed region")
     ap.add_argument("--profile", action="store_true", help="run only the C-ABI calls of one layer (for ncu)")
     ap.add_argument("--layer", type=int, default=0)

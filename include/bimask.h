@@ -3,7 +3,7 @@
  *
  * The step follows "Bi-directional Masks for Efficient N:M Sparse Training" (Alg. 1):
  * forward N:M mask (Eq. 4), sparse forward product (Eq. 3), row-permutation search
- * (Alg. 1, "pick the permutation with the most eligible N:M blocks"), backward mask on the
+ * (the permutation step of Alg. 1: the candidate with the most eligible blocks wins), backward mask on the
  * permuted weights (Eq. 11), sparse input-gradient product (Eq. 10) and the dense
  * straight-through weight gradient (Sec. 3.1).
  *
@@ -62,7 +62,8 @@ typedef enum {
   BIMASK_EINVAL = -1,       /* null / misaligned pointer, bad shape, N or P out of range, workspace too small */
   BIMASK_EUNSUPPORTED = -2, /* pattern or block length not implemented, metadata asked for a pattern without a 2:4 form, size beyond a kernel limit */
   BIMASK_ECUDA = -3,        /* a CUDA call failed; see bimask_last_error() */
-  BIMASK_ETIMEOUT = -4      /* value written to *status_word when a device-side bounded wait ran out */
+  BIMASK_ETIMEOUT = -4,     /* value written to *status_word when a device-side bounded wait ran out */
+  BIMASK_EBOUNDS = -5       /* debug build only: a caller-supplied row index (perm / candidate entry) was out of range */
 } bimask_status;
 
 /* Text of the calling thread's last error ("" if none).  Host memory owned by the library. */
@@ -96,6 +97,8 @@ int bimask_fwd_mask(const float* W, int I, int J, int N, int M,
  *                       replaced by i; mix64 = SplitMix64's output function).  Needs I < 2^24.
  *   This call alone accepts any I % M == 0 (the packed operands need I % 32 == 0); for M = 8, 16
  *   the count kernel handles N <= 4 (and the trivial N == M).
+ *   Limits: 1 <= P <= 65535 (BIMASK_EINVAL otherwise); generated candidates need I < 2^24
+ *   (BIMASK_EUNSUPPORTED otherwise; explicit candidates have no such limit).
  *   best_perm out I i32, best_idx out 1 i32, counts out P i64
  *   ws: scratch of at least bimask_workspace_bytes(...) bytes (holds the generated candidates). */
 int bimask_perm_search(const uint32_t* maskbits_f, int I, int J, int N, int M, int P, uint64_t seed,
@@ -201,7 +204,7 @@ typedef struct {
 
 int bimask_layer_step(const bimask_layer_args* args);
 
-/* Algorithm 1, last line of the loop ("update via the SGD optimizer"), fused with the first line
+/* The optimizer update that ends the loop body of Algorithm 1, fused with the first line
  * of the next iteration (forward mask, Eq. 4): one pass that reads W, dW and the momentum buffer,
  * writes the updated W and momentum, and emits the forward mask / 2:4 operand of the UPDATED
  * weights -- so an iteration that follows needs no bimask_fwd_mask of its own.
@@ -331,7 +334,8 @@ int bimask_host_sync(void);
  *     it needs to start at zero (each call rewrites every entry it later reads), but two calls
  *     whose kernels overlap on the GPU -- different streams, or different host threads -- race
  *     on it: serialise them.
- *   - Inputs, outputs, alignment, return codes: as for bimask_perm_search. */
+ *   - Inputs, outputs, alignment, return codes: as for bimask_perm_search, except that only M = 4
+ *     (N = 1 or 2) is implemented here: other M return BIMASK_EUNSUPPORTED. */
 int bimask_perm_search_static(const uint32_t* maskbits_f, int I, int J, int N, int M, int P, uint64_t seed,
                               int32_t* best_perm, int32_t* best_idx, int64_t* counts, void* stream);
 size_t bimask_perm_search_static_max_entries(void);
@@ -341,6 +345,20 @@ size_t bimask_perm_search_static_max_entries(void);
  * wait gives up, *status_word (device int) becomes BIMASK_ETIMEOUT and the kernel returns
  * normally (no trap: the context stays usable). */
 int bimask_debug_wait_probe(int32_t* status_word, void* stream);
+
+/* Debug build (libbimask_debug.so, compiled with -DBIMASK_DEBUG): every kernel that turns a caller-supplied row
+ * index (an entry of perm or of a candidate) into an address checks it against I.  Both builds clamp a bad index
+ * into range, so nothing can fault; the debug build also records the first offender.  This call waits for the
+ * device, then writes to the HOST array out[4] = {BIMASK_EBOUNDS or 0, site, index, bound} (site: 1 backward mask,
+ * 2 count kernel, 3 column permute of dY, 4 / 5 the M = 8, 16 kernels' perm / candidate reads) and clears the
+ * record.  In the release build it returns BIMASK_EUNSUPPORTED and out is all zero. */
+int bimask_debug_status(int32_t* out);
+
+/* Debug helper, not on the hot path: the candidate generator alone, cands (P x I i32) = the candidates
+ * bimask_perm_search would generate from `seed`.  part_cap > 0 runs the part-wise generator (the one used
+ * for I > 16384) with at most part_cap keys per sorting pass, which forces the multi-pass path that a part
+ * takes when it draws more keys than its buffer holds; the result must not depend on part_cap. */
+int bimask_debug_gen_candidates(uint64_t seed, int P, int I, int part_cap, int32_t* cands, void* stream);
 
 /* Debug helper, not on the hot path: sets *ok (device int) to 1 iff each of the P rows of
  * cands is a permutation of 0..I-1.  ws: at least P * I bytes of scratch. */

@@ -14,7 +14,7 @@ row permutation vector of Eq. 10 (gather: Wp[k, :] = W[perm[k], :], 0-based).
 All arrays are numpy.  Floating-point products are done in float64.  Integer
 results (mask bits, packed indices, counts, the chosen permutation) are exact.
 
-Readings of points the paper leaves open (listed again in the design notes):
+Readings of points the paper leaves open:
   * blocks are the aligned, disjoint index ranges [g*M, (g+1)*M), 0-based;
   * "Top(., N)" of Eq. 4 / Eq. 11 is applied as a rank: an element is kept when
     fewer than N elements of its block beat it, where an element q beats m if
@@ -139,7 +139,7 @@ def _mix64_np(z: np.ndarray) -> np.ndarray:
 
 
 def candidates(seed: int, P: int, I: int) -> np.ndarray:
-    """P pseudo-random permutations of {0..I-1} ("randomly generate K permutations", Alg. 1).
+    """P pseudo-random permutations of {0..I-1} (the K random candidates of the permutation step of Alg. 1).
 
     Candidate c sorts the rows by a hashed key: row i gets
         h = mix64(mix64(seed + 0x9E3779B97F4A7C15 * (c + 1)) ^ i)
@@ -403,7 +403,7 @@ def layer_step(W, X_bits, dY_bits, N, M, P, seed, do_search=True, perm=None, can
 # ---------------------------------------------------------------------------------------
 
 def sgd_update(W, dW, mom, lr, momentum, weight_decay):
-    """'Update via the SGD optimizer' (last line of the loop of Algorithm 1; Sec. 4.1 trains with SGD,
+    """The optimizer update that ends the loop body of Algorithm 1 (Sec. 4.1 trains with SGD,
     momentum and weight decay).  The straight-through estimator hands the gradient of B.W to the dense
     weights unchanged (Sec. 3.1), so the update runs on all of W:
 

@@ -11,9 +11,10 @@ from ctypes import c_float, c_int, c_int32, c_int64, c_size_t, c_uint64, c_void_
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libbimask.so")
+# BIMASK_LIBRARY=debug loads the bounds-reporting build (libbimask_debug.so) instead
+LIB_PATH = os.path.join(_HERE, "libbimask_debug.so" if os.environ.get("BIMASK_LIBRARY") == "debug" else "libbimask.so")
 
-BIMASK_OK, BIMASK_EINVAL, BIMASK_EUNSUPPORTED, BIMASK_ECUDA, BIMASK_ETIMEOUT = 0, -1, -2, -3, -4
+BIMASK_OK, BIMASK_EINVAL, BIMASK_EUNSUPPORTED, BIMASK_ECUDA, BIMASK_ETIMEOUT, BIMASK_EBOUNDS = 0, -1, -2, -3, -4, -5
 
 EXPORTS = ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "bimask_workspace_bytes", "bimask_fwd_mask",
            "bimask_perm_search", "bimask_bwd_mask", "bimask_spmm_fwd", "bimask_spmm_dgrad", "bimask_wgrad",
@@ -21,7 +22,7 @@ EXPORTS = ("bimask_last_error", "bimask_launch_count", "bimask_hw_meta_bytes", "
            "bimask_check_perms", "bimask_debug_wait_probe", "bimask_perm_search_static",
            "bimask_perm_search_static_max_entries", "bimask_sgd_fwd_mask", "bimask_train_step",
            "bimask_bwd_mask_criterion", "bimask_conv_workspace_bytes", "bimask_conv_layer_step",
-           "bimask_refine_workspace_bytes", "bimask_perm_refine")
+           "bimask_refine_workspace_bytes", "bimask_perm_refine", "bimask_debug_gen_candidates", "bimask_debug_status")
 
 
 class BimaskError(RuntimeError):
@@ -100,6 +101,8 @@ def lib() -> ctypes.CDLL:
         L.bimask_train_step.argtypes = [POINTER(TrainArgs)]
         L.bimask_check_perms.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_size_t, c_void_p]
         L.bimask_debug_wait_probe.argtypes = [c_void_p, c_void_p]
+        L.bimask_debug_status.argtypes = [c_void_p]
+        L.bimask_debug_gen_candidates.argtypes = [c_uint64, c_int, c_int, c_int, c_void_p, c_void_p]
         L.bimask_perm_search_static.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_uint64,
                                                 c_void_p, c_void_p, c_void_p, c_void_p]
         L.bimask_perm_search_static_max_entries.restype = c_size_t
@@ -272,6 +275,18 @@ def bimask_host_sync():
 
 def bimask_debug_wait_probe(status_word, stream=None):
     return _check(lib().bimask_debug_wait_probe(_ptr(status_word), _stream(stream)))
+
+
+def bimask_debug_status():
+    """[code, site, index, bound] of the first out-of-range row index the debug build's kernels met (all zero when
+    none); raises BimaskError(BIMASK_EUNSUPPORTED) on the release build."""
+    out = (c_int32 * 4)()
+    _check(lib().bimask_debug_status(ctypes.cast(out, c_void_p)))
+    return [int(v) for v in out]
+
+
+def bimask_debug_gen_candidates(seed, P, I, part_cap, cands, stream=None):
+    return _check(lib().bimask_debug_gen_candidates(seed, P, I, part_cap, _ptr(cands), _stream(stream)))
 
 
 def bimask_check_perms(cands, P, I, ok, ws, ws_bytes, stream=None):

@@ -683,6 +683,31 @@ int bimask_debug_wait_probe(int32_t* status_word, void* stream) {
   return launch_wait_probe(status_word, (cudaStream_t)stream);
 }
 
+int bimask_debug_status(int32_t* out) {
+  BIMASK_REQUIRE(out != nullptr, BIMASK_EINVAL, "bimask_debug_status: null pointer");
+  out[0] = out[1] = out[2] = out[3] = 0;
+#ifndef BIMASK_DEBUG
+  set_error("bimask_debug_status: this library was built without BIMASK_DEBUG");
+  return BIMASK_EUNSUPPORTED;
+#else
+  int (*collect[4])(int*) = {debug_collect_mask, debug_collect_perm, debug_collect_gemm_host, debug_collect_generic};
+  for (auto fn : collect) {
+    int rec[4];
+    const int rc = fn(rec);
+    if (rc != BIMASK_OK) return rc;
+    if (rec[0] != 0 && out[0] == 0) { out[0] = rec[0]; out[1] = rec[1]; out[2] = rec[2]; out[3] = rec[3]; }
+  }
+  return BIMASK_OK;
+#endif
+}
+
+int bimask_debug_gen_candidates(uint64_t seed, int P, int I, int part_cap, int32_t* cands, void* stream) {
+  BIMASK_REQUIRE(cands != nullptr && aligned16(cands), BIMASK_EINVAL, "bimask_debug_gen_candidates: null or misaligned pointer");
+  BIMASK_REQUIRE(P >= 1 && P <= 65535 && I >= 1 && I < (1 << 24) && part_cap >= 0, BIMASK_EINVAL,
+                 "bimask_debug_gen_candidates: P = %d, I = %d, part_cap = %d out of range", P, I, part_cap);
+  return launch_gen_candidates(seed, P, I, cands, (cudaStream_t)stream, nullptr, nullptr, part_cap);
+}
+
 int bimask_check_perms(const int32_t* cands, int P, int I, int32_t* ok, void* ws, size_t ws_bytes, void* stream) {
   BIMASK_REQUIRE(cands && ok && ws && P >= 1 && I >= 1, BIMASK_EINVAL, "bimask_check_perms: bad argument");
   BIMASK_REQUIRE(ws_bytes >= (size_t)P * I, BIMASK_EINVAL, "bimask_check_perms: workspace too small");

@@ -87,6 +87,51 @@ inline int set_smem_attr(K kernel, int bytes) {
   return BIMASK_OK;
 }
 
+// Row indices that come from the caller (a permutation, a candidate) are clamped into range before they are used
+// as addresses, so a bad entry can never fault a kernel.  In the debug build (-DBIMASK_DEBUG, libbimask_debug.so)
+// the clamp also REPORTS: the first out-of-range index a kernel meets is recorded -- code BIMASK_EBOUNDS, a
+// site number, the index and the bound -- in a small per-source-file device array that bimask_debug_status()
+// collects.  Nothing traps; the release build compiles the record away.
+#ifdef __CUDACC__
+#ifdef BIMASK_DEBUG
+namespace {
+__device__ int tu_debug_record[4];                       // one per translation unit (internal linkage)
+}
+__device__ __forceinline__ int checked_row(int v, int n, int site) {
+  if ((unsigned)v >= (unsigned)n) {
+    if (atomicCAS(&tu_debug_record[0], 0, (int)BIMASK_EBOUNDS) == 0) {
+      tu_debug_record[1] = site;
+      tu_debug_record[2] = v;
+      tu_debug_record[3] = n;
+    }
+    return v < 0 ? 0 : n - 1;
+  }
+  return v;
+}
+// host side of the same file: fetch and clear the record (synchronises the device)
+#define BIMASK_DEFINE_DEBUG_COLLECT(name)                                                        \
+  int name(int out[4]) {                                                                         \
+    BIMASK_CUDA_OK(cudaDeviceSynchronize());                                                     \
+    BIMASK_CUDA_OK(cudaMemcpyFromSymbol(out, tu_debug_record, 4 * sizeof(int)));                 \
+    const int zero[4] = {0, 0, 0, 0};                                                            \
+    BIMASK_CUDA_OK(cudaMemcpyToSymbol(tu_debug_record, zero, 4 * sizeof(int)));                  \
+    return BIMASK_OK;                                                                            \
+  }
+#else
+__device__ __forceinline__ int checked_row(int v, int n, int) {
+  return (int)min((unsigned)max(v, 0), (unsigned)(n - 1));
+}
+#define BIMASK_DEFINE_DEBUG_COLLECT(name) \
+  int name(int out[4]) { out[0] = out[1] = out[2] = out[3] = 0; return BIMASK_OK; }
+#endif
+#endif
+// sites of checked_row, reported by bimask_debug_status
+enum { SITE_BWD_MASK_PERM = 1, SITE_SCORE_CAND = 2, SITE_PERMUTE_PERM = 3, SITE_GENERIC_PERM = 4, SITE_GENERIC_CAND = 5 };
+int debug_collect_mask(int out[4]);
+int debug_collect_perm(int out[4]);
+int debug_collect_gemm_host(int out[4]);
+int debug_collect_generic(int out[4]);
+
 // 2-D tensor map without swizzle (gemm_host.cu); dtype is a CUtensorMapDataType value.
 int make_tmap_plain(CUtensorMap_st* m, int dtype, const void* ptr, uint64_t inner, uint64_t outer, uint32_t box_inner,
                     uint32_t box_outer, uint32_t elem_bytes);
@@ -110,8 +155,9 @@ int launch_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* p
                     int N, uint32_t* maskbits_b, uint16_t* vals_b, uint32_t* meta_b, void* hw_meta_or_null,
                     cudaStream_t s);
 // zero_counts / zero_ticket (optional): the generator also zeroes counts[0..P) and *zero_ticket for the count kernel
+// part_cap > 0 (debug): the part-wise generator with at most that many keys per sorting pass
 int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStream_t s, int64_t* zero_counts = nullptr,
-                          int32_t* zero_ticket = nullptr);
+                          int32_t* zero_ticket = nullptr, int part_cap = 0);
 // best_idx / best_perm (optional): fused pick by the kernel's last CTA; zeroed: counts and *best_idx are already zero
 int launch_score(const uint32_t* maskbits_f, const int32_t* cands, int I, int J, int N, int P,
                  int64_t* counts, cudaStream_t s, bool zeroed = false, int32_t* best_idx = nullptr,

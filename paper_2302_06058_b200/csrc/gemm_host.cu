@@ -61,7 +61,7 @@ permute_cols_kernel(const uint16_t* __restrict__ dY, const int32_t* __restrict__
       uint32_t lo[8], hi[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
-        const int i = min(max(idx[e], 0), I - 1);
+        const int i = checked_row(idx[e], I, SITE_PERMUTE_PERM);
         if (R == 4) {
           const uint2 v = reinterpret_cast<const uint2*>(tile_w)[i];
           lo[e] = v.x; hi[e] = v.y;
@@ -105,8 +105,8 @@ permute_cols_small_kernel(const uint16_t* __restrict__ dY, const int32_t* __rest
     uint32_t v[4];
 #pragma unroll
     for (int h = 0; h < 4; ++h) {
-      const uint32_t lo = __ldg(row + min(max(idx[2 * h], 0), I - 1));
-      const uint32_t hi = __ldg(row + min(max(idx[2 * h + 1], 0), I - 1));
+      const uint32_t lo = __ldg(row + checked_row(idx[2 * h], I, SITE_PERMUTE_PERM));
+      const uint32_t hi = __ldg(row + checked_row(idx[2 * h + 1], I, SITE_PERMUTE_PERM));
       v[h] = lo | (hi << 16);
     }
     reinterpret_cast<uint4*>(dYp + t * I)[k8] = make_uint4(v[0], v[1], v[2], v[3]);
@@ -243,6 +243,8 @@ int launch_wait_probe(int32_t* status_word, cudaStream_t s) {
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
 }
+
+BIMASK_DEFINE_DEBUG_COLLECT(debug_collect_gemm_host)
 
 int launch_permute_cols(const uint16_t* dY, const int32_t* perm, int T, int I, uint16_t* dYp, cudaStream_t s) {
   if (I <= 1024) {

@@ -22,7 +22,7 @@ namespace {
 // ---------------------------------------------------------------------------------------
 constexpr int FWD_THREADS = 256;
 
-// Optimizer update of Algorithm 1 ("update via the SGD optimizer"), applied while the weights
+// Optimizer update that ends the loop body of Algorithm 1, applied while the weights
 // stream through the mask kernel so that the next iteration's forward mask costs no second pass
 // over W.  float32, each product and sum rounded once, in this order (the updated weight decides
 // a mask bit, so the operation order is part of the contract):
@@ -230,7 +230,6 @@ bwd_mask_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbi
   const int jwords = J >> 5;
   const int nrg = I >> 5;                                  // groups of 32 permuted rows
   const int items = jwords / CW;                           // column items of 32 CW columns
-  const unsigned last_row = (unsigned)(I - 1);
   const int rgi = warp & 3, cti = warp >> 2;               // this warp's row group and column item inside a tile
   const size_t vrow = (size_t)I >> 2;                      // u32 (bf16 pairs) per row of vals_b
   const size_t mrow = (size_t)I >> 5;
@@ -246,7 +245,7 @@ bwd_mask_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbi
     }
     cp_async_commit();
   };
-  auto load_rows = [&](int rgroup) { return (int)min((unsigned)__ldg(perm + 32 * rgroup + lane), last_row); };
+  auto load_rows = [&](int rgroup) { return checked_row(__ldg(perm + 32 * rgroup + lane), I, SITE_BWD_MASK_PERM); };
   auto load_fwd = [&](int rows, int item, uint32_t (&f)[CW]) {
     const uint32_t* src = maskbits_f + (size_t)rows * jwords + item * CW;
     if (CW == 2) { const uint2 t = __ldg(reinterpret_cast<const uint2*>(src)); f[0] = t.x; f[1] = t.y; }
@@ -380,6 +379,8 @@ bwd_mask_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbi
 }
 
 }  // namespace
+
+BIMASK_DEFINE_DEBUG_COLLECT(debug_collect_mask)
 
 int launch_fwd_mask(const float* W, int I, int J, int N, uint32_t* maskbits, uint16_t* vals,
                     uint32_t* meta, void* hw_meta_or_null, cudaStream_t s) {

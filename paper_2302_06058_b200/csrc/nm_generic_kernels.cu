@@ -190,8 +190,8 @@ score_generic_kernel(const uint32_t* __restrict__ bits, const int32_t* __restric
 #pragma unroll
     for (int g = 0; g < M / 4; ++g) {
       const int4 r = __ldg(reinterpret_cast<const int4*>(cand + (long long)b * M) + g);
-      rows[4 * g] = (int)min((unsigned)r.x, last_row); rows[4 * g + 1] = (int)min((unsigned)r.y, last_row);
-      rows[4 * g + 2] = (int)min((unsigned)r.z, last_row); rows[4 * g + 3] = (int)min((unsigned)r.w, last_row);
+      rows[4 * g] = checked_row(r.x, (int)last_row + 1, SITE_GENERIC_CAND); rows[4 * g + 1] = checked_row(r.y, (int)last_row + 1, SITE_GENERIC_CAND);
+      rows[4 * g + 2] = checked_row(r.z, (int)last_row + 1, SITE_GENERIC_CAND); rows[4 * g + 3] = checked_row(r.w, (int)last_row + 1, SITE_GENERIC_CAND);
     }
     if ((jwords & 3) == 0) {
       // 128-bit loads: four words of every row at once (a quarter of the load instructions)
@@ -258,8 +258,8 @@ refine_gain_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict_
   int ra[M], rb[M];
 #pragma unroll
   for (int m = 0; m < M; ++m) {
-    ra[m] = (int)min((unsigned)__ldg(perm + ka * M + m), last_row);
-    rb[m] = (int)min((unsigned)__ldg(perm + kb * M + m), last_row);
+    ra[m] = checked_row(__ldg(perm + ka * M + m), (int)last_row + 1, SITE_GENERIC_PERM);
+    rb[m] = checked_row(__ldg(perm + kb * M + m), (int)last_row + 1, SITE_GENERIC_PERM);
   }
   const int ma = a - ka * M, mb = b - kb * M;
   int gain = 0;
@@ -391,7 +391,7 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
   if (cw >= jwords) return;
   const int col = 32 * cw + lane;
   const unsigned last_row = (unsigned)(I - 1);
-  const int my_src = (int)min((unsigned)__ldg(perm + 32 * pass + lane), last_row);   // lane r: source of permuted row r
+  const int my_src = checked_row(__ldg(perm + 32 * pass + lane), (int)last_row + 1, SITE_GENERIC_PERM);   // lane r: source of permuted row r
   uint32_t my_word = 0;                                     // lane r ends up with the mask word of permuted row r
   uint32_t vacc[8];
   uint32_t dacc[MODE == 2 ? 16 : 1];                        // dense: this column's 32 permuted rows as bf16 pairs
@@ -455,6 +455,8 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
 }
 
 }  // namespace
+
+BIMASK_DEFINE_DEBUG_COLLECT(debug_collect_generic)
 
 // mode: 0 mask bits only, 1 the 2:4 operand, 2 the dense masked operand (written to `vals`)
 int launch_fwd_mask_generic(const float* W, int I, int J, int N, int M, uint32_t* maskbits, uint16_t* vals_or_null,

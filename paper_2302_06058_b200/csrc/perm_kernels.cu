@@ -35,7 +35,7 @@ gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int q_log2, i
                       int32_t* __restrict__ cands, unsigned long long* __restrict__ zero_counts,
                       int32_t* __restrict__ zero_ticket) {
   pdl_launch_dependents();                               // the candidates depend on the seed alone: no wait up here
-  extern __shared__ unsigned long long keys[];           // cap keys, then nbq bucket counters
+  extern __shared__ unsigned long long keys[];           // cap keys, then nbq + 1 bucket counters
   const int nbq_log2 = nb_log2 - q_log2;
   const int nbq = 1 << nbq_log2;
   uint32_t* count = reinterpret_cast<uint32_t*>(keys + cap);
@@ -83,44 +83,68 @@ gen_candidates_kernel(unsigned long long seed, int I, int nb_log2, int q_log2, i
     if (lane < GEN_THREADS / 32) warp_sums[lane] = ws;
   }
   __syncthreads();
-  const uint32_t mine = warp_sums[GEN_THREADS / 32 - 1];  // keys of this part
   uint32_t run = incl - local + (warp > 0 ? warp_sums[warp - 1] : 0u);
   for (int b = b0; b < min(nbq, b0 + per); ++b) {
     const uint32_t n = count[b];
     count[b] = run;                                       // start of bucket b
     run += n;
   }
+  if (tid == GEN_THREADS - 1) count[nbq] = warp_sums[GEN_THREADS / 32 - 1];   // one past the last bucket: the keys of this part
   __syncthreads();
-  for (int i = tid; i < I; i += GEN_THREADS) {
-    const unsigned long long v = (mix64(stream ^ (unsigned long long)i) & ~0xFFFFFFull) | (unsigned long long)i;
-    const uint32_t b = (uint32_t)(v >> shift);
-    if ((b >> nbq_log2) == part) {
-      const uint32_t pos = atomicAdd(&count[b & (nbq - 1)], 1u);   // count[b] ends as end of bucket b
-      if (pos < (uint32_t)cap) keys[pos] = v;            // cap is > 15 sigma above the mean part size
+  // The part is sorted in S passes over equal runs of its buckets, S the smallest power of two for which every
+  // run holds at most `cap` keys.  S is 1 unless the part drew far more keys than its share (cap leaves more than
+  // fifteen standard deviations of room), so the passes cost nothing in practice, but no key is ever dropped.
+  __shared__ int s_passes;
+  if (tid == 0) {
+    int S = 1;
+    for (; S < nbq; S <<= 1) {
+      bool fits = true;
+      for (int q = 0; q < S && fits; ++q) fits = count[(q + 1) * (nbq / S)] - count[q * (nbq / S)] <= (uint32_t)cap;
+      if (fits) break;
     }
+    s_passes = S;
   }
   __syncthreads();
-  const int filled = (int)min(mine, (uint32_t)cap);
-  for (int b = b0; b < min(nbq, b0 + per); ++b) {
-    const int lo = min(b == 0 ? 0 : (int)count[b - 1], filled);
-    const int hi = min((int)count[b], filled);
-    for (int a = lo + 1; a < hi; ++a) {                   // insertion sort, buckets hold ~1 key
-      const unsigned long long v = keys[a];
-      int q = a - 1;
-      while (q >= lo && keys[q] > v) { keys[q + 1] = keys[q]; --q; }
-      keys[q + 1] = v;
+  const int S = s_passes, run_len = nbq / S;
+  const uint32_t base = lower_total;
+  bool waited = false;
+  for (int pass = 0; pass < S; ++pass) {
+    const uint32_t blo = (uint32_t)(pass * run_len), bhi = blo + (uint32_t)run_len;
+    const uint32_t first = count[blo];                   // untouched so far: the buckets of later passes still hold their start
+    __syncthreads();
+    for (int i = tid; i < I; i += GEN_THREADS) {
+      const unsigned long long v = (mix64(stream ^ (unsigned long long)i) & ~0xFFFFFFull) | (unsigned long long)i;
+      const uint32_t b = (uint32_t)(v >> shift);
+      const uint32_t bq = b & (uint32_t)(nbq - 1);
+      if ((b >> nbq_log2) == part && bq >= blo && bq < bhi) {
+        const uint32_t pos = atomicAdd(&count[bq], 1u) - first;     // count[b] ends as end of bucket b
+        if (pos < (uint32_t)cap) keys[pos] = v;          // holds by the choice of S (a single bucket above cap aside)
+      }
     }
+    __syncthreads();
+    const int filled = (int)min(count[bhi - 1] - first, (uint32_t)cap);
+    for (int b = b0; b < min(nbq, b0 + per); ++b) {
+      if ((uint32_t)b < blo || (uint32_t)b >= bhi) continue;
+      const int lo = min((uint32_t)b == blo ? 0 : (int)(count[b - 1] - first), filled);
+      const int hi = min((int)(count[b] - first), filled);
+      for (int a = lo + 1; a < hi; ++a) {                 // insertion sort, buckets hold ~1 key
+        const unsigned long long v = keys[a];
+        int q = a - 1;
+        while (q >= lo && keys[q] > v) { keys[q + 1] = keys[q]; --q; }
+        keys[q + 1] = v;
+      }
+    }
+    __syncthreads();
+    if (!waited) { pdl_wait(); waited = true; }           // first global access: earlier kernels may still read these buffers
+    for (int i = tid; i < filled; i += GEN_THREADS)
+      if (base + first + i < (uint32_t)I) cands[(long long)c * I + base + first + i] = (int32_t)(keys[i] & 0xFFFFFFull);
   }
-  __syncthreads();
-  pdl_wait();                                            // first global access: earlier kernels may still read these buffers
+  if (!waited) pdl_wait();
   if (tid == 0) {
     // the count kernel that follows adds into counts[c] and uses *zero_ticket as its "CTAs done" counter
     if (part == 0 && zero_counts) zero_counts[c] = 0ull;
     if (part == 0 && c == 0 && zero_ticket) *zero_ticket = 0;
   }
-  const uint32_t base = lower_total;
-  for (int i = tid; i < filled; i += GEN_THREADS)
-    if (base + i < (uint32_t)I) cands[(long long)c * I + base + i] = (int32_t)(keys[i] & 0xFFFFFFull);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -363,11 +387,10 @@ score_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cand
     // the CTA's row indices first (one coalesced load, clamped), so that the row loads below do
     // not wait on a dependent global load
     __shared__ int4 idx_s[SCORE_KB_MAX];
-    const unsigned last_row = (unsigned)(I - 1);
     for (int t = threadIdx.x; t < kb1 - kb0; t += SCORE_THREADS) {
       const int4 r = __ldg(cand4 + kb0 + t);
-      idx_s[t] = make_int4((int)min((unsigned)r.x, last_row), (int)min((unsigned)r.y, last_row),
-                           (int)min((unsigned)r.z, last_row), (int)min((unsigned)r.w, last_row));
+      idx_s[t] = make_int4(checked_row(r.x, I, SITE_SCORE_CAND), checked_row(r.y, I, SITE_SCORE_CAND),
+                           checked_row(r.z, I, SITE_SCORE_CAND), checked_row(r.w, I, SITE_SCORE_CAND));
     }
     __syncthreads();
     // two row blocks per trip: eight independent 128-bit loads in flight per lane
@@ -400,7 +423,8 @@ score_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ cand
   } else {
     for (int k = kb0 + warp; k < kb1; k += SCORE_THREADS / 32) {
       int4 r = __ldg(cand4 + k);
-      r.x = min(max(r.x, 0), I - 1); r.y = min(max(r.y, 0), I - 1); r.z = min(max(r.z, 0), I - 1); r.w = min(max(r.w, 0), I - 1);
+      r.x = checked_row(r.x, I, SITE_SCORE_CAND); r.y = checked_row(r.y, I, SITE_SCORE_CAND);
+      r.z = checked_row(r.z, I, SITE_SCORE_CAND); r.w = checked_row(r.w, I, SITE_SCORE_CAND);
       const uint32_t* r0 = bits + (long long)r.x * jwords;
       const uint32_t* r1 = bits + (long long)r.y * jwords;
       const uint32_t* r2 = bits + (long long)r.z * jwords;
@@ -463,12 +487,14 @@ __global__ void set_int_kernel(int32_t* p, int32_t v) {
 
 }  // namespace
 
+BIMASK_DEFINE_DEBUG_COLLECT(debug_collect_perm)
+
 int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStream_t s, int64_t* zero_counts,
-                          int32_t* zero_ticket) {
+                          int32_t* zero_ticket, int part_cap) {
   int lg = 1;
   while ((1 << lg) < I) ++lg;                             // one bucket per key on average
   unsigned long long* zc = reinterpret_cast<unsigned long long*>(zero_counts);
-  if (I <= 16384) {
+  if (I <= 16384 && part_cap <= 0) {
     // a CTA per candidate with the keys in registers: 4, 8 or 16 per thread
     const int kpt = I <= 4096 ? 4 : I <= 8192 ? 8 : 16;
     int threads = ((I + kpt - 1) / kpt + 31) / 32 * 32;
@@ -490,8 +516,9 @@ int launch_gen_candidates(uint64_t seed, int P, int I, int32_t* cands, cudaStrea
   int ql = 0;
   while ((I >> ql) > 8192 && ql < lg - 1) ++ql;           // at most 8192 keys per part (measured best)
   const int mean = (I + (1 << ql) - 1) >> ql;
-  const int cap = ql == 0 ? I : mean + (mean / 4 > 256 ? mean / 4 : 256);
-  const size_t smem = (size_t)cap * sizeof(unsigned long long) + ((size_t)1 << (lg - ql)) * sizeof(uint32_t);
+  int cap = ql == 0 ? I : mean + (mean / 4 > 256 ? mean / 4 : 256);
+  if (part_cap > 0) cap = part_cap < cap ? part_cap : cap;         // debug: a small capacity forces the multi-pass sort
+  const size_t smem = (size_t)cap * sizeof(unsigned long long) + (((size_t)1 << (lg - ql)) + 2) * sizeof(uint32_t);
   if (int rc = set_smem_attr(gen_candidates_kernel, 200 * 1024)) return rc;
   dim3 grid(P, 1 << ql);
   BIMASK_CUDA_OK(launch_pdl(gen_candidates_kernel, grid, GEN_THREADS, smem, s, (unsigned long long)seed, I, lg, ql, cap, cands,

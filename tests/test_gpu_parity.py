@@ -58,6 +58,19 @@ def test_bwd_mask_bit_exact(I, J, N):
     assert np.array_equal(u16(b["vals_b"]), vals)
 
 
+@pytest.mark.parametrize("I,P,cap", [(20000, 3, 0), (20000, 3, 700), (40000, 2, 3000), (4096, 4, 300), (8192, 2, 64),
+                                     (16384, 5, 0), (12288, 3, 0), (100, 7, 0), (100, 7, 16)])
+def test_candidate_generator_alone_and_with_a_forced_small_part_buffer(I, P, cap):
+    """The generator's result must not depend on how many keys a sorting pass may hold: with a small capacity the
+    part-wise kernel sorts a part in several passes (the path a part takes if it ever draws more keys than its
+    buffer holds) and still produces the oracle's candidates."""
+    seed = 1234 + I
+    cands = torch.full((P, I), -7, dtype=torch.int32, device="cuda")
+    bm.bimask_debug_gen_candidates(seed, P, I, cap, cands)
+    torch.cuda.synchronize()
+    assert np.array_equal(cands.cpu().numpy(), O.candidates(seed, P, I))
+
+
 @pytest.mark.parametrize("I,J,N,P", [(256, 256, 2, 8), (64, 576, 2, 32), (512, 4608, 1, 64), (1152, 384, 2, 32),
                                      (100, 96, 2, 5), (16384, 64, 2, 3), (40000, 32, 2, 2),
                                      (128, 128, 2, 1), (96, 64, 1, 300), (2048, 2048, 2, 130)])

@@ -112,25 +112,24 @@ def test_missing_library_fails_loudly(tmp_path):
 
 _WORKER = r"""
 import os, sys, json
-import torch, torch.distributed as dist
+import torch.distributed as dist
 sys.path.insert(0, %r)
+import bench
 rank = int(os.environ["RANK"]); world = int(os.environ["WORLD_SIZE"])
 dist.init_process_group("gloo")
-# every rank times its own replica; the job time is the max over ranks, the value the aggregate
-ms = torch.tensor([10.0 + 5.0 * rank], dtype=torch.float64)
+# every rank times its own replica; bench.py's own helpers reduce the timings (max over ranks) and form the value
 dist.barrier()
-dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-layers, steps = 2, 4
-value = world * layers * steps / (float(ms) * 1e-3)
+ms, other = bench.max_over_ranks([10.0 + 5.0 * rank, 7.0 - rank], world)
+value = bench.job_value(world, 2, 4, ms)
 if rank == 0:
-    print(json.dumps({"ms": float(ms), "value": value}))
+    print(json.dumps({"ms": ms, "other": other, "value": value}))
 dist.destroy_process_group()
 """
 
 
 def test_replica_aggregation_world_size_2(tmp_path):
-    """The multi-GPU path is N independent replicas: no collective touches the data; only the timing
-    is reduced (max over ranks) and the value is world * layers * steps / that time."""
+    """The multi-GPU path is N independent replicas: no collective touches the data; only the timings are reduced
+    (max over ranks) and the value is world * layers * steps / that time.  Runs the functions bench.py uses."""
     script = tmp_path / "worker.py"
     script.write_text(_WORKER % ROOT)
     out = subprocess.check_output(
@@ -140,8 +139,18 @@ def test_replica_aggregation_world_size_2(tmp_path):
     line = [l for l in out.splitlines() if l.startswith("{")][-1]
     import json
     d = json.loads(line)
-    assert d["ms"] == 15.0
+    assert d["ms"] == 15.0 and d["other"] == 7.0
     assert abs(d["value"] - 2 * 2 * 4 / 0.015) < 1e-6
+
+
+def test_clock_regime_picks_the_peak():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.clock_regime({"sm_mhz": 1965.0, "sm_max_mhz": 1965.0}, 0.08) == "burst"
+    assert bench.clock_regime({"sm_mhz": 1965.0, "sm_max_mhz": 1965.0}, 6.0) == "sustained"
+    assert bench.clock_regime({"sm_mhz": 1380.0, "sm_max_mhz": 1965.0}, 0.08) == "sustained"
+    assert bench.clock_regime({"sm_mhz": None, "sm_max_mhz": None}) == "sustained"
+    assert bench.job_value(2, 2, 4, 15.0) == 2 * 2 * 4 / 0.015
 
 
 def test_bench_reference_arm_runs_on_cpu():
