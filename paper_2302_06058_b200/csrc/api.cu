@@ -341,6 +341,47 @@ struct ConvPlan {
   float* wpart;       // split-K partial sums of the implicit weight gradient
 };
 
+// A layer step is a chain of short kernels.  On small layers the kernels are too short to fill the GPU and the
+// step takes as long as its longest dependent chain, so the step is spread over three streams there:
+//   caller's stream:  forward mask -> count candidates -> backward mask -> permute dY -> sparse input gradient
+//   side stream A:    candidate generation (needs the seed alone) -> dense weight gradient (needs dY and X alone)
+//   side stream B:    sparse forward product (needs the forward mask alone)
+// forked after the inputs are ready and joined before the step returns to the caller's stream.  Two side streams and
+// five events per device and host thread, created on first use and kept until exit.  (On the large configuration
+// co-resident kernels contend for issue slots and the step gets slower, so there everything stays in line.)
+namespace bimask {
+struct SideStream {
+  cudaStream_t a = nullptr, b = nullptr;
+  cudaEvent_t fork = nullptr, gen_done = nullptr, mask_done = nullptr, join_a = nullptr, join_b = nullptr;
+};
+static int get_side_stream(SideStream** out) {
+  static thread_local SideStream side[64];
+  int dev = 0;
+  BIMASK_CUDA_OK(cudaGetDevice(&dev));
+  BIMASK_REQUIRE(dev >= 0 && dev < 64, BIMASK_EUNSUPPORTED, "device ordinal %d out of range", dev);
+  SideStream& sd = side[dev];
+  if (!sd.a) {
+    BIMASK_CUDA_OK(cudaStreamCreateWithFlags(&sd.a, cudaStreamNonBlocking));
+    BIMASK_CUDA_OK(cudaStreamCreateWithFlags(&sd.b, cudaStreamNonBlocking));
+    for (cudaEvent_t* e : {&sd.fork, &sd.gen_done, &sd.mask_done, &sd.join_a, &sd.join_b})
+      BIMASK_CUDA_OK(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
+  }
+  *out = &sd;
+  return BIMASK_OK;
+}
+// Joins the side streams back into the caller's stream when the layer step leaves, on every path.
+struct SideJoin {
+  SideStream* side = nullptr;
+  cudaStream_t main = nullptr;
+  bool a_forked = false, b_forked = false;
+  ~SideJoin() {
+    if (!side) return;
+    if (a_forked && cudaEventRecord(side->join_a, side->a) == cudaSuccess) cudaStreamWaitEvent(main, side->join_a, 0);
+    if (b_forked && cudaEventRecord(side->join_b, side->b) == cudaSuccess) cudaStreamWaitEvent(main, side->join_b, 0);
+  }
+};
+}  // namespace bimask
+
 // skip_fwd_mask: the forward mask / operand of the current W is already in place.
 // conv: null for a linear layer; otherwise a->X is x (T x C) and a->dX is dx (T x C).
 static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const ConvPlan* conv = nullptr) {
@@ -380,9 +421,7 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
   uint16_t* dYp = reinterpret_cast<uint16_t*>(ws + w.dyp_off);
   float* partials = w.part_bytes ? reinterpret_cast<float*>(ws + w.part_off) : nullptr;
 
-  // Alg. 1 in order, on the caller's stream.  (Running the dense weight gradient concurrently
-  // with the bandwidth-bound chain on a second stream was measured and rejected: the co-resident
-  // kernels contend for issue slots and the step became slower and erratic.)
+  // Alg. 1 in order on the caller's stream; small layers spread it over three streams (see SideStream).
   cudaStream_t s = (cudaStream_t)a->stream;
   const uint16_t* Xmat = a->X;                       // the T x J activation matrix of the explicit products
   uint16_t* dXmat = a->dX;
@@ -391,6 +430,35 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
     dXmat = conv->dxcol;
     if (!conv->imp_fwd || !conv->imp_wgrad)
       if ((rc = launch_im2col3x3(a->X, conv->NB, conv->H, conv->W, conv->C, conv->stride, conv->xcol, s))) return rc;
+  }
+  // small layers (between a gigaflop and a hundred): three streams, see SideStream
+  const double flops = 2.0 * a->T * a->I * a->J;
+  const bool spread = flops >= 1e9 && flops < 1e11;
+  SideJoin join;
+  SideStream* side = nullptr;
+  cudaStream_t sa = s, sb = s;                          // where generation + weight gradient / the forward product go
+  const bool gen_here = a->do_search && !a->cands;
+  if (spread) {
+    if ((rc = get_side_stream(&side))) return rc;
+    join.side = side;
+    join.main = s;
+    sa = side->a;
+    sb = side->b;
+    BIMASK_CUDA_OK(cudaEventRecord(side->fork, s));
+    BIMASK_CUDA_OK(cudaStreamWaitEvent(sa, side->fork, 0));
+    join.a_forked = true;
+    if (gen_here) {
+      if ((rc = launch_gen_candidates(a->seed, a->P, a->I, gen, sa, a->M == 4 ? a->counts : nullptr,
+                                      a->M == 4 ? a->best_idx : nullptr)))
+        return rc;
+      BIMASK_CUDA_OK(cudaEventRecord(side->gen_done, sa));
+    }
+    if (conv && conv->imp_wgrad)
+      rc = launch_wgrad_conv(a->dY, a->X, conv->NB, conv->H, conv->W, conv->C, a->I, conv->stride, a->dW, conv->wpart,
+                             a->status_word, sa);
+    else
+      rc = launch_wgrad_impl(a->dY, Xmat, a->T, a->I, a->J, a->dW, partials, a->status_word, sa);
+    if (rc) return rc;
   }
   // unpadded shapes: the mask kernels write the metadata images themselves
   const bool fused = pack && (a->I % 128 == 0) && (a->J % 128 == 0);
@@ -403,18 +471,26 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
     if (rc) return rc;
     if (pack && !fused && (rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, s))) return rc;
   }
+  if (spread) {
+    BIMASK_CUDA_OK(cudaEventRecord(side->mask_done, s));
+    BIMASK_CUDA_OK(cudaStreamWaitEvent(sb, side->mask_done, 0));
+    join.b_forked = true;
+  }
   if (conv && conv->imp_fwd)
     rc = launch_spmm_conv(1, a->vals_f, a->hw_meta_f, a->X, conv->NB, conv->H, conv->W, conv->C, a->I, conv->stride, a->Y,
-                          a->status_word, s);
-  else if (pack) rc = launch_spmm(a->vals_f, a->hw_meta_f, Xmat, a->I, a->T, a->J, a->Y, a->status_word, s);
-  else rc = launch_dense_nt(a->vals_f, Xmat, a->I, a->T, a->J, a->Y, a->status_word, s);
+                          a->status_word, sb);
+  else if (pack) rc = launch_spmm(a->vals_f, a->hw_meta_f, Xmat, a->I, a->T, a->J, a->Y, a->status_word, sb);
+  else rc = launch_dense_nt(a->vals_f, Xmat, a->I, a->T, a->J, a->Y, a->status_word, sb);
   if (rc) return rc;
   if (a->do_search) {
     const int32_t* cands = a->cands;
     if (!cands) {
-      if ((rc = launch_gen_candidates(a->seed, a->P, a->I, gen, s, a->M == 4 ? a->counts : nullptr,
-                                      a->M == 4 ? a->best_idx : nullptr)))
+      if (spread) {
+        BIMASK_CUDA_OK(cudaStreamWaitEvent(s, side->gen_done, 0));
+      } else if ((rc = launch_gen_candidates(a->seed, a->P, a->I, gen, s, a->M == 4 ? a->counts : nullptr,
+                                             a->M == 4 ? a->best_idx : nullptr))) {
         return rc;
+      }
       cands = gen;
     }
     if (a->M == 4) {
@@ -442,6 +518,7 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
   if (rc) return rc;
   if (conv && !conv->imp_dgrad)
     if ((rc = launch_col2im3x3(dXmat, conv->NB, conv->H, conv->W, conv->C, conv->stride, a->dX, s))) return rc;
+  if (spread) return BIMASK_OK;                           // already running beside the chain; joined on return
   if (conv && conv->imp_wgrad)
     return launch_wgrad_conv(a->dY, a->X, conv->NB, conv->H, conv->W, conv->C, a->I, conv->stride, a->dW, conv->wpart,
                              a->status_word, s);
