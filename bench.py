@@ -237,15 +237,15 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------
 # DRAM traffic per call (dram__bytes_read.sum + dram__bytes_write.sum over the kernels of the call, one ncu capture
 # of `bench.py --profile` per layer of config 5); the capture is named in the JSON line beside the numbers.
-NCU_TRAFFIC_SOURCE = "profiles/cfg5_dram_traffic.md"
+NCU_TRAFFIC_SOURCE = "profiles/cfg5_launch_list.md"
 NCU_TRAFFIC_BYTES = {
-    (5, 0, "fwd_mask"): 268.5e6 + 63.8e6, (5, 1, "fwd_mask"): 268.7e6 + 63.3e6,
-    (5, 0, "spmm_fwd"): 616.3e6 + 239.3e6, (5, 1, "spmm_fwd"): 702.6e6 + 50.6e6,
-    (5, 0, "perm_search"): 16.9e6, (5, 1, "perm_search"): 10.5e6,          # generator + count kernel
-    (5, 0, "bwd_mask"): 277.3e6 + 61.9e6, (5, 1, "bwd_mask"): 277.5e6 + 60.9e6,
-    (5, 0, "spmm_dgrad"): 268.5e6 + 216.3e6 + 702.6e6 + 50.6e6,           # permute pass + product
-    (5, 1, "spmm_dgrad"): 67.1e6 + 19.6e6 + 615.4e6 + 239.4e6,
-    (5, 0, "wgrad"): 1392.4e6 + 247.7e6, (5, 1, "wgrad"): 1078.0e6 + 247.5e6,
+    (5, 0, "fwd_mask"): 268e6 + 64e6, (5, 1, "fwd_mask"): 269e6 + 68e6,
+    (5, 0, "spmm_fwd"): 362e6 + 235e6, (5, 1, "spmm_fwd"): 592e6 + 51e6,
+    (5, 0, "perm_search"): 17e6, (5, 1, "perm_search"): 11e6,              # generator + count kernel
+    (5, 0, "bwd_mask"): 277e6 + 62e6, (5, 1, "bwd_mask"): 277e6 + 61e6,
+    (5, 0, "spmm_dgrad"): 269e6 + 216e6 + 592e6 + 51e6,                    # permute pass + product
+    (5, 1, "spmm_dgrad"): 67e6 + 18e6 + 368e6 + 236e6,
+    (5, 0, "wgrad"): 1243e6 + 246e6, (5, 1, "wgrad"): 1011e6 + 246e6,
 }
 
 
