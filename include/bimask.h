@@ -268,9 +268,11 @@ int bimask_train_step(const bimask_train_args* args);
  * patches with 4-D tensor loads (out-of-image pixels read as zero); BIMASK_CONV_AUTO takes the
  * implicit form for every product whose shape allows it (C % 64 == 0; the input gradient needs
  * C == 64 or C % 128 == 0; patterns with a 2:4 form) when the column matrix would
- * exceed 16 MiB and an output image has more than 64 pixels, and the explicit form otherwise.  With stride 2 the forward product and the
- * weight gradient have an implicit form (the tensor loads take every second pixel), the input
- * gradient always takes the explicit one.  IMPLICIT with a shape that does not allow it returns
+ * exceed 16 MiB and an output image has more than 64 pixels, and the explicit form otherwise.  Stride 2: the forward
+ * product and the weight gradient take every second pixel in their tensor loads; the input gradient runs as four
+ * stride-1 products, one per parity class (h % 2, w % 2) of the input pixels, each over the filter taps that reach
+ * that class (one, two, two and four of the nine).  IMPLICIT needs C % 64 == 0 and a pattern with a 2:4 form; an
+ * input gradient whose C is neither 64 nor a multiple of 128 keeps the explicit form then.  Otherwise IMPLICIT returns
  * BIMASK_EUNSUPPORTED.  C % 32 == 0 and I % 32 == 0 always.  The two forms round the
  * input gradient differently (explicit: nine bf16 partial results summed in fp32; implicit: one
  * fp32 accumulation), both within the products' tolerance. */

@@ -512,7 +512,7 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
   if (pack && !fused && (rc = launch_hw_meta(a->meta_b, a->J, a->I, a->hw_meta_b, s))) return rc;
   if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, s))) return rc;
   if (conv && conv->imp_dgrad)
-    rc = launch_spmm_conv(2, a->vals_b, a->hw_meta_b, dYp, conv->NB, conv->H, conv->W, conv->C, a->I, 1, a->dX, a->status_word, s);
+    rc = launch_spmm_conv(2, a->vals_b, a->hw_meta_b, dYp, conv->NB, conv->H, conv->W, conv->C, a->I, conv->stride, a->dX, a->status_word, s);
   else if (pack) rc = launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, dXmat, a->status_word, s);
   else rc = launch_dense_nt(a->vals_b, dYp, a->J, a->T, a->I, dXmat, a->status_word, s);
   if (rc) return rc;
@@ -564,15 +564,17 @@ int bimask_conv_layer_step(const bimask_conv_args* c) {
                  a->ws_bytes, need);
   ConvPlan plan;
   plan.NB = c->NB; plan.H = c->H; plan.W = c->W; plan.C = c->C; plan.stride = c->stride;
-  // the forward product and the weight gradient have an implicit form for both strides (strided tensor-map
-  // traversal), the input gradient for stride 1 only: with stride 2 it always takes the explicit form
-  const bool packs = a->N <= 2, unit = c->stride == 1;
+  // all three products have an implicit form for both strides: the forward product and the weight gradient through a
+  // strided tensor-map traversal, the input gradient of a stride-2 layer as four stride-1 problems, one per parity
+  // class of the input pixels.  The input gradient needs whole 128-row operand tiles per filter tap (C % 128 == 0, or
+  // C = 64); where it cannot go implicit (other C % 64 == 0) it keeps the explicit form beside the implicit others.
+  const bool packs = a->N <= 2;
   const bool can_fwd = packs && c->C % 64 == 0;
-  const bool can_dgrad = unit && packs && (c->C % 128 == 0 || c->C == 64);
+  const bool can_dgrad = packs && (c->C % 128 == 0 || c->C == 64);
   const bool can_wgrad = c->C % 64 == 0;
-  BIMASK_REQUIRE(c->mode != BIMASK_CONV_IMPLICIT || (can_fwd && can_wgrad && (can_dgrad || !unit)), BIMASK_EUNSUPPORTED,
-                 "bimask_conv_layer_step: the implicit form needs C = 64 or a multiple of 128 (a multiple of 64 with stride 2) "
-                 "and a pattern with a 2:4 form (stride %d, C = %d, I = %d, N:M = %d:%d)", c->stride, c->C, a->I, a->N, a->M);
+  BIMASK_REQUIRE(c->mode != BIMASK_CONV_IMPLICIT || (can_fwd && can_wgrad), BIMASK_EUNSUPPORTED,
+                 "bimask_conv_layer_step: the implicit form needs C %% 64 == 0 and a pattern with a 2:4 form "
+                 "(stride %d, C = %d, I = %d, N:M = %d:%d)", c->stride, c->C, a->I, a->N, a->M);
   // AUTO: a column matrix that fits comfortably in L2 costs little, and the explicit form then has
   // fewer, denser k tiles (measured: 7x7 images of 512 channels are faster explicit, 14x14 of 256
   // channels faster implicit); above 16 MiB the implicit form wins by the HBM traffic it avoids.

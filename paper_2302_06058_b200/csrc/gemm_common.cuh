@@ -50,7 +50,19 @@ struct ConvGeom {
   int tiles_w, tiles_h;     // boxes per image
   int kt_per_tap;           // mode 2: 128-wide k tiles per filter tap (I / 128)
   int rows_per_tap;         // mode 2: rows of the 2:4 operand per tap (C)
+  // mode 2: the filter taps this launch sums over, in k order: tap id (kh * 3 + kw, selects the operand rows) and the
+  // shift of the dy box.  Stride 1: all nine, shift (1 - kw, 1 - kh).  Stride 2: the input pixels of one parity class
+  // (h % 2, w % 2) receive gradient through the taps with kh = h + 1 and kw = w + 1 (mod 2) only -- one, two, two and
+  // four taps for the four classes -- from dy pixel ((h + 1 - kh) / 2, (w + 1 - kw) / 2); the token grid is then the
+  // class's sub-grid and the results go to every second pixel of dx.
+  signed char tap_id[9], tap_dw[9], tap_dh[9];
+  int out_step, out_h0, out_w0, out_H, out_W;   // token (h, w) is stored at pixel (out_step * h + out_h0, out_step * w + out_w0) of out_H x out_W
 };
+
+// Where the results of token pixel (n, h, w) go: element offset of its first channel in the NHWC output.
+__device__ __forceinline__ size_t conv_out_pixel(const ConvGeom& g, int n, int h, int w) {
+  return ((size_t)n * g.out_H + (g.out_step * h + g.out_h0)) * g.out_W + (g.out_step * w + g.out_w0);
+}
 
 __device__ __forceinline__ void conv_box_origin(const ConvGeom& g, int box, int& w0, int& h0, int& n0) {
   w0 = (box % g.tiles_w) * g.wb;
@@ -73,8 +85,8 @@ __device__ __forceinline__ void conv_k_coords(const ConvGeom& g, int kt, int q, 
     const int tap = kt / g.kt_per_tap;
     c0 = (kt - tap * g.kt_per_tap) * 128 + 64 * q;
     valid = true;
-    dh = 1 - tap / 3;
-    dw = 1 - tap % 3;
+    dh = g.tap_dh[tap];
+    dw = g.tap_dw[tap];
   }
 }
 

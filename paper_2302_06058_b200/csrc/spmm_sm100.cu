@@ -93,7 +93,7 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
             const int tap = kt / p.conv.kt_per_tap;
             meta_kt = kt - tap * p.conv.kt_per_tap;
             a_col = meta_kt * 64;
-            a_row = tap * p.conv.rows_per_tap + m0;
+            a_row = p.conv.tap_id[tap] * p.conv.rows_per_tap + m0;
             meta_row = a_row >> 7;
           }
           ptx::tma_load_2d(a_s, &tmapA, a_col, a_row, full_bar(s));
@@ -184,7 +184,7 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
           const int h = ch0 + ((rr >> p.conv.lg_wb) & (p.conv.hb - 1));
           const int n = cn0 + (rr >> (p.conv.lg_wb + p.conv.lg_hb));
           if (w >= p.conv.W || h >= p.conv.H || n >= p.conv.NB) return nullptr;
-          return outp + ((size_t)(n * p.conv.H + h) * p.conv.W + w) * p.Mdim + m0;
+          return outp + conv_out_pixel(p.conv, n, h, w) * p.Mdim + m0;
         }
         const int n = n0 + 32 * c + t;
         return n < p.Ndim ? outp + (size_t)n * p.Mdim + m0 : nullptr;
@@ -311,7 +311,7 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
               const int tap = kt / p.conv.kt_per_tap;
               meta_kt = kt - tap * p.conv.kt_per_tap;
               a_col = meta_kt * 64;
-              a_row = tap * p.conv.rows_per_tap + m0;
+              a_row = p.conv.tap_id[tap] * p.conv.rows_per_tap + m0;
               meta_row = a_row >> 7;
             }
             ptx::tma_load_2d_pair(a_s, &tmapA, a_col, a_row, bar);
@@ -408,7 +408,7 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
           const int h = ch0 + ((rr >> p.conv.lg_wb) & (p.conv.hb - 1));
           const int n = cn0 + (rr >> (p.conv.lg_wb + p.conv.lg_hb));
           if (w >= p.conv.W || h >= p.conv.H || n >= p.conv.NB) return nullptr;
-          return outp + ((size_t)(n * p.conv.H + h) * p.conv.W + w) * p.Mdim + m0;
+          return outp + conv_out_pixel(p.conv, n, h, w) * p.Mdim + m0;
         });
       } else if ((SP_N & 31) == 0) {
         drain_chunks<32>(acc, eg, EPI_WARPS / 4, nchunks, false, release_bar, stg, 1 + eg, q, lane, p.Mdim - m0,
@@ -842,24 +842,54 @@ int run_conv_pair(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_m
 int launch_spmm_conv(int mode, const uint16_t* vals, const void* hw_meta, const uint16_t* tok, int NB, int H, int W, int C,
                      int I, int stride, uint16_t* out, int32_t* status_word, cudaStream_t s) {
   ConvGeom g{};
-  // the tokens are the output pixels; with stride 2 (forward only) the input tensor is H x W, the output Ho x Wo
-  g.mode = mode; g.NB = NB; g.stride = stride;
-  g.H = (H - 1) / stride + 1; g.W = (W - 1) / stride + 1;
-  const long long T = (long long)NB * g.H * g.W;
-  int Mdim, Kdim, a_rows, a_kdim, tiles_k_meta;
+  g.mode = mode; g.NB = NB;
+  const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;       // the convolution's output image
+  auto run = [&](const ConvGeom& gg, int tok_h, int tok_w, int Mdim, int Kdim, int a_rows, int a_kdim, int tiles_k_meta) {
+    const long long T = (long long)NB * gg.H * gg.W;
+    if (Mdim > 128 && T > 128)
+      return run_conv_pair(vals, a_rows, a_kdim, hw_meta, tok, tok_h, tok_w, gg, Mdim, Kdim, tiles_k_meta, out, status_word, s);
+    if (T > 128)
+      return run_conv_single<256, 2>(vals, a_rows, a_kdim, hw_meta, tok, tok_h, tok_w, gg, Mdim, Kdim, tiles_k_meta, out, status_word, s);
+    return run_conv_single<128, 3>(vals, a_rows, a_kdim, hw_meta, tok, tok_h, tok_w, gg, Mdim, Kdim, tiles_k_meta, out, status_word, s);
+  };
   if (mode == 1) {
+    // the tokens are the output pixels; with stride 2 the input tensor map is traversed with stride 2
+    g.stride = stride; g.H = Ho; g.W = Wo;
     g.CB = C; g.kt_per_tap = 0; g.rows_per_tap = 0;
-    Mdim = I; Kdim = 9 * C; a_rows = I; a_kdim = 9 * C; tiles_k_meta = (9 * C + 127) / 128;
-  } else {
-    BIMASK_REQUIRE(stride == 1, BIMASK_EUNSUPPORTED, "implicit input gradient: stride %d", stride);
-    g.CB = I; g.kt_per_tap = (I + 127) / 128; g.rows_per_tap = C;
-    Mdim = C; Kdim = 9 * g.kt_per_tap * 128; a_rows = 9 * C; a_kdim = I; tiles_k_meta = g.kt_per_tap;
+    g.out_step = 1; g.out_h0 = 0; g.out_w0 = 0; g.out_H = Ho; g.out_W = Wo;
+    return run(g, H, W, I, 9 * C, I, 9 * C, (9 * C + 127) / 128);
   }
-  if (Mdim > 128 && T > 128)
-    return run_conv_pair(vals, a_rows, a_kdim, hw_meta, tok, H, W, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
-  if (T > 128)
-    return run_conv_single<256, 2>(vals, a_rows, a_kdim, hw_meta, tok, H, W, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
-  return run_conv_single<128, 3>(vals, a_rows, a_kdim, hw_meta, tok, H, W, g, Mdim, Kdim, tiles_k_meta, out, status_word, s);
+  // input gradient: the tokens are pixels of dx (H x W), the token operand is the permuted dy (Ho x Wo), read with unit stride
+  g.stride = 1;
+  g.CB = I; g.kt_per_tap = (I + 127) / 128; g.rows_per_tap = C;
+  g.out_H = H; g.out_W = W;
+  if (stride == 1) {
+    g.H = H; g.W = W;
+    g.out_step = 1; g.out_h0 = 0; g.out_w0 = 0;
+    for (int t = 0; t < 9; ++t) { g.tap_id[t] = (signed char)t; g.tap_dh[t] = (signed char)(1 - t / 3); g.tap_dw[t] = (signed char)(1 - t % 3); }
+    return run(g, Ho, Wo, C, 9 * g.kt_per_tap * 128, 9 * C, I, g.kt_per_tap);
+  }
+  BIMASK_REQUIRE(stride == 2, BIMASK_EUNSUPPORTED, "implicit input gradient: stride %d", stride);
+  // stride 2: one stride-1 problem per parity class of the input pixels (see ConvGeom)
+  for (int ph = 0; ph < 2; ++ph)
+    for (int pw = 0; pw < 2; ++pw) {
+      ConvGeom gc = g;
+      gc.H = (H - ph + 1) / 2; gc.W = (W - pw + 1) / 2;
+      if (gc.H <= 0 || gc.W <= 0) continue;
+      gc.out_step = 2; gc.out_h0 = ph; gc.out_w0 = pw;
+      int nt = 0;
+      for (int kh = 0; kh < 3; ++kh)
+        for (int kw = 0; kw < 3; ++kw) {
+          if (((ph + 1 - kh) & 1) || ((pw + 1 - kw) & 1)) continue;
+          gc.tap_id[nt] = (signed char)(kh * 3 + kw);
+          gc.tap_dh[nt] = (signed char)((ph + 1 - kh) / 2);
+          gc.tap_dw[nt] = (signed char)((pw + 1 - kw) / 2);
+          ++nt;
+        }
+      const int rc = run(gc, Ho, Wo, C, nt * g.kt_per_tap * 128, 9 * C, I, g.kt_per_tap);
+      if (rc != BIMASK_OK) return rc;
+    }
+  return BIMASK_OK;
 }
 
 namespace {
