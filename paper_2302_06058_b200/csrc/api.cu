@@ -343,16 +343,18 @@ struct ConvPlan {
 
 // A layer step is a chain of short kernels.  On small layers the kernels are too short to fill the GPU and the
 // step takes as long as its longest dependent chain, so the step is spread over three streams there:
-//   caller's stream:  forward mask -> count candidates -> backward mask -> permute dY -> sparse input gradient
+//   caller's stream:  forward mask -> count candidates -> backward mask -> sparse input gradient
 //   side stream A:    candidate generation (needs the seed alone) -> dense weight gradient (needs dY and X alone)
-//   side stream B:    sparse forward product (needs the forward mask alone)
-// forked after the inputs are ready and joined before the step returns to the caller's stream.  Two side streams and
-// five events per device and host thread, created on first use and kept until exit.  (On the large configuration
+//   side stream B:    [metadata image of a padded forward operand ->] sparse forward product (needs the forward mask alone)
+//   side stream C:    column permutation of dY (needs the permutation alone; the input gradient waits for it)
+// forked after the inputs are ready and joined before the step returns to the caller's stream.  Three side streams
+// and eight events per device and host thread, created on first use and kept until exit.  (On the large configuration
 // co-resident kernels contend for issue slots and the step gets slower, so there everything stays in line.)
 namespace bimask {
 struct SideStream {
-  cudaStream_t a = nullptr, b = nullptr;
-  cudaEvent_t fork = nullptr, gen_done = nullptr, mask_done = nullptr, join_a = nullptr, join_b = nullptr;
+  cudaStream_t a = nullptr, b = nullptr, c = nullptr;
+  cudaEvent_t fork = nullptr, gen_done = nullptr, mask_done = nullptr, perm_done = nullptr, permuted = nullptr,
+              join_a = nullptr, join_b = nullptr, join_c = nullptr;
 };
 static int get_side_stream(SideStream** out) {
   static thread_local SideStream side[64];
@@ -363,7 +365,8 @@ static int get_side_stream(SideStream** out) {
   if (!sd.a) {
     BIMASK_CUDA_OK(cudaStreamCreateWithFlags(&sd.a, cudaStreamNonBlocking));
     BIMASK_CUDA_OK(cudaStreamCreateWithFlags(&sd.b, cudaStreamNonBlocking));
-    for (cudaEvent_t* e : {&sd.fork, &sd.gen_done, &sd.mask_done, &sd.join_a, &sd.join_b})
+    BIMASK_CUDA_OK(cudaStreamCreateWithFlags(&sd.c, cudaStreamNonBlocking));
+    for (cudaEvent_t* e : {&sd.fork, &sd.gen_done, &sd.mask_done, &sd.perm_done, &sd.permuted, &sd.join_a, &sd.join_b, &sd.join_c})
       BIMASK_CUDA_OK(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
   }
   *out = &sd;
@@ -373,11 +376,12 @@ static int get_side_stream(SideStream** out) {
 struct SideJoin {
   SideStream* side = nullptr;
   cudaStream_t main = nullptr;
-  bool a_forked = false, b_forked = false;
+  bool a_forked = false, b_forked = false, c_forked = false;
   ~SideJoin() {
     if (!side) return;
     if (a_forked && cudaEventRecord(side->join_a, side->a) == cudaSuccess) cudaStreamWaitEvent(main, side->join_a, 0);
     if (b_forked && cudaEventRecord(side->join_b, side->b) == cudaSuccess) cudaStreamWaitEvent(main, side->join_b, 0);
+    if (c_forked && cudaEventRecord(side->join_c, side->c) == cudaSuccess) cudaStreamWaitEvent(main, side->join_c, 0);
   }
 };
 }  // namespace bimask
@@ -469,13 +473,14 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
       rc = launch_fwd_mask_generic(a->W, a->I, a->J, a->N, a->M, a->maskbits_f, a->vals_f, a->meta_f, pack ? 1 : 2,
                                    fused ? a->hw_meta_f : nullptr, s);
     if (rc) return rc;
-    if (pack && !fused && (rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, s))) return rc;
   }
   if (spread) {
     BIMASK_CUDA_OK(cudaEventRecord(side->mask_done, s));
     BIMASK_CUDA_OK(cudaStreamWaitEvent(sb, side->mask_done, 0));
     join.b_forked = true;
   }
+  // padded shapes: the metadata image of the forward operand is a pass of its own, needed by the forward product only
+  if (!skip_fwd_mask && pack && !fused && (rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, sb))) return rc;
   if (conv && conv->imp_fwd)
     rc = launch_spmm_conv(1, a->vals_f, a->hw_meta_f, a->X, conv->NB, conv->H, conv->W, conv->C, a->I, conv->stride, a->Y,
                           a->status_word, sb);
@@ -502,6 +507,15 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
       if ((rc = launch_pick(a->counts, cands, a->P, a->I, a->best_idx, a->perm, s))) return rc;
     }
   }
+  cudaStream_t sc = s;
+  if (spread) {                                          // the permutation is final: dY[:, perm] goes to side stream C
+    sc = side->c;
+    BIMASK_CUDA_OK(cudaEventRecord(side->perm_done, s));
+    BIMASK_CUDA_OK(cudaStreamWaitEvent(sc, side->perm_done, 0));
+    join.c_forked = true;
+    if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, sc))) return rc;
+    BIMASK_CUDA_OK(cudaEventRecord(side->permuted, sc));
+  }
   if (a->M == 4)
     rc = launch_bwd_mask(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->maskbits_b, a->vals_b, a->meta_b,
                          fused ? a->hw_meta_b : nullptr, s);
@@ -510,7 +524,11 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
                                  pack ? 1 : 2, fused ? a->hw_meta_b : nullptr, s);
   if (rc) return rc;
   if (pack && !fused && (rc = launch_hw_meta(a->meta_b, a->J, a->I, a->hw_meta_b, s))) return rc;
-  if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, s))) return rc;
+  if (spread) {
+    BIMASK_CUDA_OK(cudaStreamWaitEvent(s, side->permuted, 0));
+  } else if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, s))) {
+    return rc;
+  }
   if (conv && conv->imp_dgrad)
     rc = launch_spmm_conv(2, a->vals_b, a->hw_meta_b, dYp, conv->NB, conv->H, conv->W, conv->C, a->I, conv->stride, a->dX, a->status_word, s);
   else if (pack) rc = launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, dXmat, a->status_word, s);
