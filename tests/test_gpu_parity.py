@@ -491,12 +491,13 @@ def test_async_host_calls_with_alternating_buffer_sets():
         assert torch.equal(host["dW"], ref["dW"].cpu()), c
 
 
-@pytest.mark.parametrize("I,J,T", [(256, 384, 512), (64, 576, 3000)])
+@pytest.mark.parametrize("I,J,T", [(256, 384, 512), (64, 576, 3000), (256, 384, 6000), (64, 576, 16000), (1152, 384, 1500)])
 def test_back_to_back_steps_on_reused_buffers(I, J, T):
     """Every kernel is launched as a programmatic dependent of the one before it and may begin before that one
-    has finished.  Steps on alternating inputs, enqueued back to back into the same buffers with no synchronisation
-    in between, must give each step's own results: a kernel that read or wrote ahead of its dependency would pick
-    up the other input's data."""
+    has finished; layers of more than a gigaflop (the last three shapes) also run parts of the step on side streams
+    that fork from and join the caller's stream.  Steps on alternating inputs, enqueued back to back into the same
+    buffers with no synchronisation in between, must give each step's own results: a kernel that read or wrote ahead
+    of its dependency would pick up the other input's data."""
     N, M, P = 2, 4, 6
     sets = []
     for k in range(2):
@@ -566,10 +567,12 @@ def test_layer_step_parity_on_drawn_shapes(I, J, T, N, M):
         assert rel_err(b[n].float().cpu().numpy(), ref[n]) <= TOL, n
 
 
-def test_layer_step_captured_in_a_cuda_graph():
-    """The entry points enqueue kernels only (programmatic dependent launches included), so a step can be captured
-    once and replayed: the replay on new contents of the same buffers must give that input's results."""
-    I, J, T, N, M, P = 256, 384, 700, 2, 4, 6
+@pytest.mark.parametrize("T", [700, 6000])
+def test_layer_step_captured_in_a_cuda_graph(T):
+    """The entry points enqueue kernels only (programmatic dependent launches included; at T = 6000 also the forks to
+    and joins from the side streams of a layer above a gigaflop), so a step can be captured once and replayed: the
+    replay on new contents of the same buffers must give that input's results."""
+    I, J, N, M, P = 256, 384, 2, 4, 6
     sets = [(inputs.make_weight(I, J, 600 + k), inputs.make_activation(T, J, 610 + k), inputs.make_activation(T, I, 620 + k))
             for k in range(2)]
     b = bm.alloc_layer_buffers(T, I, J, P)

@@ -88,7 +88,8 @@ def test_sgd_fwd_mask_at_config5_size_on_samples():
 
 @pytest.mark.parametrize("I,J,T,N,M,P,dT", [(256, 256, 64, 2, 4, 8, 2), (128, 384, 96, 1, 4, 6, 3),
                                             (96, 160, 40, 2, 4, 5, 2), (128, 128, 64, 2, 8, 6, 2),
-                                            (128, 256, 64, 4, 8, 6, 2)])
+                                            (128, 256, 64, 4, 8, 6, 2),
+                                            (256, 384, 6000, 2, 4, 6, 2)])     # above a gigaflop: side streams
 def test_train_step_trajectory_bit_exact(I, J, T, N, M, P, dT):
     iters, seed = 5, 77
     lr, mu, wd = 2.0 ** -9, 0.5, 2.0 ** -7
