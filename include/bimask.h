@@ -179,8 +179,14 @@ int bimask_wgrad(const uint16_t* dY, const uint16_t* X, int T, int I, int J, flo
 
 /* One iteration of Alg. 1 for one layer (without the optimizer update): fwd mask + pack, sparse
  * forward, [search if do_search], bwd mask + pack, sparse input gradient, dense weight
- * gradient, all enqueued on `stream` in that order.  When the search is skipped, perm is used
- * as given. */
+ * gradient.  The caller sees one ordered step on `stream`: everything the call enqueues starts after the work
+ * already on `stream` and is complete, as far as `stream` is concerned, when the work enqueued after the call starts.
+ * Inside, layers between 1 and 100 GFLOP (2 T I J) run the parts that do not depend on each other (candidate
+ * generation + weight gradient, forward product, permutation of dY) on three library-owned side streams that fork
+ * from and join `stream` by events; the first such call of a host thread on a device creates those streams and
+ * events (make it before any stream capture; later calls can be captured, forks and joins included).
+ * When the search is skipped, perm is used as given.  Limits: I <= 51200 (column permute of dY); with do_search
+ * 1 <= P <= 65535, and I < 2^24 when the candidates are generated. */
 typedef struct {
   int T, I, J, N, M, P;
   uint64_t seed;
