@@ -5,7 +5,9 @@ runtime owns the whole GPU heap, or they are only lent pointers).  For them the 
 generated candidates in an array built into the library.  This test calls that entry point through
 the C ABI twice in a row -- the second time with a smaller problem, so that the shared array still
 holds entries of the first call -- and requires exactly the results of bimask_perm_search (all
-outputs are integers, so the comparison is bit for bit)."""
+outputs are integers, so the comparison is bit for bit).  The reference here is the workspace entry
+point, not the CPU oracle: that one is checked against the oracle in tests/test_gpu_parity.py
+(generated candidates, counts, chosen permutation), so agreement with it carries the parity over."""
 import numpy as np
 import pytest
 import torch
