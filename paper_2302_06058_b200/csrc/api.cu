@@ -100,9 +100,7 @@ int bimask_fwd_mask(const float* W, int I, int J, int N, int M, uint32_t* maskbi
       return rc;
     return pack && !gfused ? launch_hw_meta(meta_f, I, J, hw_meta_f, s) : BIMASK_OK;
   }
-  const bool fused = (I % 128 == 0) && (J % 128 == 0);   // no padding in the metadata image
-  if ((rc = launch_fwd_mask(W, I, J, N, maskbits_f, vals_f, meta_f, fused ? hw_meta_f : nullptr, s)) != BIMASK_OK) return rc;
-  return fused ? BIMASK_OK : launch_hw_meta(meta_f, I, J, hw_meta_f, s);
+  return launch_fwd_mask(W, I, J, N, maskbits_f, vals_f, meta_f, hw_meta_f, s);   // writes the metadata image too, padding included
 }
 
 size_t bimask_refine_workspace_bytes(int I, int M, int rounds) {
@@ -173,11 +171,7 @@ int bimask_sgd_fwd_mask(float* W, const float* dW, float* mom, int I, int J, int
       return rc;
     return pack && !gfused ? launch_hw_meta(meta_f, I, J, hw_meta_f, s) : BIMASK_OK;
   }
-  const bool fused = (I % 128 == 0) && (J % 128 == 0);   // no padding in the metadata image
-  if ((rc = launch_sgd_fwd_mask(W, dW, mom, I, J, N, lr, momentum, weight_decay, maskbits_f, vals_f, meta_f,
-                                fused ? hw_meta_f : nullptr, s)) != BIMASK_OK)
-    return rc;
-  return fused ? BIMASK_OK : launch_hw_meta(meta_f, I, J, hw_meta_f, s);
+  return launch_sgd_fwd_mask(W, dW, mom, I, J, N, lr, momentum, weight_decay, maskbits_f, vals_f, meta_f, hw_meta_f, s);
 }
 
 int bimask_perm_search(const uint32_t* maskbits_f, int I, int J, int N, int M, int P, uint64_t seed,
@@ -237,11 +231,7 @@ int bimask_bwd_mask(const float* W, const uint32_t* maskbits_f, const int32_t* p
       return rc;
     return pack && !gfused ? launch_hw_meta(meta_b, J, I, hw_meta_b, s) : BIMASK_OK;
   }
-  const bool fused = (I % 128 == 0) && (J % 128 == 0);
-  if ((rc = launch_bwd_mask(W, maskbits_f, perm, I, J, N, maskbits_b, vals_b, meta_b, fused ? hw_meta_b : nullptr, s)) !=
-      BIMASK_OK)
-    return rc;
-  return fused ? BIMASK_OK : launch_hw_meta(meta_b, J, I, hw_meta_b, s);
+  return launch_bwd_mask(W, maskbits_f, perm, I, J, N, maskbits_b, vals_b, meta_b, hw_meta_b, s);
 }
 
 int bimask_bwd_mask_criterion(const float* W, const float* S, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
@@ -464,8 +454,9 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
       rc = launch_wgrad_impl(a->dY, Xmat, a->T, a->I, a->J, a->dW, partials, a->status_word, sa);
     if (rc) return rc;
   }
-  // unpadded shapes: the mask kernels write the metadata images themselves
-  const bool fused = pack && (a->I % 128 == 0) && (a->J % 128 == 0);
+  // the 2:4 mask kernels (M = 4) write the metadata images themselves, padding included; the generic ones (M = 8, 16)
+  // do so on unpadded shapes and need the re-ordering pass otherwise
+  const bool fused = pack && (a->M == 4 || ((a->I % 128 == 0) && (a->J % 128 == 0)));
   if (!skip_fwd_mask) {
     if (a->M == 4)
       rc = launch_fwd_mask(a->W, a->I, a->J, a->N, a->maskbits_f, a->vals_f, a->meta_f, fused ? a->hw_meta_f : nullptr, s);

@@ -137,8 +137,9 @@ int make_tmap_plain(CUtensorMap_st* m, int dtype, const void* ptr, uint64_t inne
                     uint32_t box_outer, uint32_t elem_bytes);
 
 // Launchers implemented in the .cu files (all enqueue on `s`, none synchronise).
-// hw_meta_or_null: when given (operand without padding: rows and K multiples of 128) the kernel
-// also writes the tensor-core metadata image; otherwise call launch_hw_meta afterwards.
+// hw_meta_or_null: when given, the kernel also writes the tensor-core metadata image.  The 2:4 kernels (launch_fwd_mask,
+// launch_sgd_fwd_mask, launch_bwd_mask) do so for any shape, padding included; the generic ones (M = 8, 16) only for
+// operands without padding (rows and K multiples of 128): otherwise pass null and call launch_hw_meta afterwards.
 int launch_fwd_mask(const float* W, int I, int J, int N, uint32_t* maskbits, uint16_t* vals,
                     uint32_t* meta, void* hw_meta_or_null, cudaStream_t s);
 // forward mask of the weights after one SGD step, which the same kernel applies in place

@@ -128,5 +128,21 @@ __device__ __forceinline__ void scatter_hw(uint16_t* __restrict__ hw16, int tile
   hw16[idx + 64] = (uint16_t)(word >> 16);               // lane + 8: 8 lanes x 4 words x 2 halves
 }
 
+// Padding of the tensor-memory image (operands whose rows or k extent are not multiples of 128): every 32-bit entry
+// that belongs wholly to rows >= rows or code words >= kwords gets the harmless code 0x4 (slots (0, 1); the values
+// there are zero).  rows % 16 == 0, so an entry (two rows eight apart) is never half real.  Called by all threads of
+// a grid (tid of nthreads); the real entries are written by the mask kernels themselves.
+__device__ __forceinline__ void pad_hw_image(uint32_t* __restrict__ hw32, int rows, int kwords, long long tid, long long nthreads) {
+  const int tiles_k = (kwords + 3) >> 2;
+  const long long n = (long long)((rows + 127) >> 7) * tiles_k * 512;
+  for (long long e = tid; e < n; e += nthreads) {
+    const long long tile = e >> 9;
+    const int L = (int)(e & 511) >> 2, kc = (int)(e & 3);
+    const int mt = (int)(tile / tiles_k), kt = (int)(tile - (long long)mt * tiles_k);
+    const int r_lo = mt * 128 + (L & 7) + 16 * (L >> 4);
+    if (r_lo >= rows || kt * 4 + kc >= kwords) hw32[e] = 0x44444444u;
+  }
+}
+
 }  // namespace
 }  // namespace bimask

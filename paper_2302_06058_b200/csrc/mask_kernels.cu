@@ -44,7 +44,7 @@ template <bool N_IS_2, bool UPDATE>
 __global__ void __launch_bounds__(FWD_THREADS)
 fwd_mask_pack_kernel(const float4* __restrict__ W4, long long nblk, int N,
                      uint32_t* __restrict__ maskbits, uint4* __restrict__ vals4,
-                     uint32_t* __restrict__ meta, uint16_t* __restrict__ hw16, int jwords, SgdParams sgd) {
+                     uint32_t* __restrict__ meta, uint16_t* __restrict__ hw16, int jwords, int pad_rows, SgdParams sgd) {
   pdl_launch_dependents();
   pdl_wait();
   __shared__ uint32_t lut[64];
@@ -99,12 +99,16 @@ fwd_mask_pack_kernel(const float4* __restrict__ W4, long long nblk, int N,
       meta[word] = codes;
       if (hw16) {
         const int r = (int)(word / jwords);
-        scatter_hw(hw16, jwords >> 2, r, (int)(word - (long long)r * jwords), codes);
+        scatter_hw(hw16, (jwords + 3) >> 2, r, (int)(word - (long long)r * jwords), codes);
       }
       vals4[2 * word] = make_uint4(v[0], v[1], v[2], v[3]);
       vals4[2 * word + 1] = make_uint4(v[4], v[5], v[6], v[7]);
     }
   }
+  // padded operand (pad_rows = its row count): the image entries past the matrix
+  if (hw16 && pad_rows)
+    pad_hw_image(reinterpret_cast<uint32_t*>(hw16), pad_rows, jwords, (long long)blockIdx.x * FWD_THREADS + threadIdx.x,
+                 (long long)gridDim.x * FWD_THREADS);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -360,22 +364,26 @@ bwd_mask_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbi
       }
     }
     if (hw32) {
-      // tensor-memory image (I and J multiples of 128): the tile's codes fill a contiguous run of the 2048-byte
-      // block (operand rows col0 .., k words rg0 ..): image lane L = m0 + 8 h + 16 m2 holds half h of the code
-      // words of rows m0 + 16 m2 (low 16 bits) and m0 + 8 + 16 m2 (high 16 bits)
-      uint32_t* blk = hw32 + ((size_t)(col0 >> 7) * (I >> 7) + tr) * 512 + (col0 & 127) * 4;
+      // tensor-memory image: the tile's codes fill a run of the 2048-byte block (operand rows col0 .., k words
+      // rg0 ..): image lane L = m0 + 8 h + 16 m2 holds half h of the code words of rows m0 + 16 m2 (low 16 bits) and
+      // m0 + 8 + 16 m2 (high 16 bits).  Entries past the matrix (padded shapes) are filled after the tile loop.
+      uint32_t* blk = hw32 + ((size_t)(col0 >> 7) * ((I + 127) >> 7) + tr) * 512 + (col0 & 127) * 4;
 #pragma unroll
       for (int it = 0; it < C::COLS * 4 / BM_THREADS; ++it) {
         const int idx = it * BM_THREADS + threadIdx.x;
         const int L = idx >> 2, kc = idx & 3;
         const int r_lo = (L & 7) + 16 * (L >> 4);
-        const uint32_t lo = sc[r_lo * 4 + kc], hi = sc[(r_lo + 8) * 4 + kc];
-        blk[idx] = __byte_perm(lo, hi, (L & 8) ? 0x7632u : 0x5410u);
+        if (r_lo < cols_here && kc < rgs_here) {
+          const uint32_t lo = sc[r_lo * 4 + kc], hi = sc[(r_lo + 8) * 4 + kc];
+          blk[idx] = __byte_perm(lo, hi, (L & 8) ? 0x7632u : 0x5410u);
+        }
       }
     }
     __syncthreads();                                       // the staging tile is free again
   }
   cp_async_wait<0>();
+  if (hw32 && ((I | J) & 127))                             // padded operand (J rows, I / 32 code words per row)
+    pad_hw_image(hw32, J, I >> 5, (long long)blockIdx.x * BM_THREADS + threadIdx.x, (long long)gridDim.x * BM_THREADS);
 }
 
 }  // namespace
@@ -391,12 +399,13 @@ int launch_fwd_mask(const float* W, int I, int J, int N, uint32_t* maskbits, uin
   if (ctas > 148 * 8) ctas = 148 * 8;
   if (ctas < 1) ctas = 1;
   const SgdParams none{nullptr, nullptr, nullptr, 0.f, 0.f, 0.f};
+  const int pad_rows = (I % 128 || J % 128) ? I : 0;       // padded image: the kernel also fills the entries past the matrix
   if (N == 2)
     BIMASK_CUDA_OK(launch_pdl(fwd_mask_pack_kernel<true, false>, (unsigned)ctas, FWD_THREADS, 0, s,
-        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, none));
+        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, pad_rows, none));
   else
     BIMASK_CUDA_OK(launch_pdl(fwd_mask_pack_kernel<false, false>, (unsigned)ctas, FWD_THREADS, 0, s,
-        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, none));
+        reinterpret_cast<const float4*>(W), nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, pad_rows, none));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -412,12 +421,13 @@ int launch_sgd_fwd_mask(float* W, const float* dW, float* mom, int I, int J, int
   if (ctas < 1) ctas = 1;
   const SgdParams p{reinterpret_cast<float4*>(W), reinterpret_cast<const float4*>(dW), reinterpret_cast<float4*>(mom),
                     lr, momentum, weight_decay};
+  const int pad_rows = (I % 128 || J % 128) ? I : 0;
   if (N == 2)
     BIMASK_CUDA_OK(launch_pdl(fwd_mask_pack_kernel<true, true>, (unsigned)ctas, FWD_THREADS, 0, s,
-        nullptr, nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, p));
+        nullptr, nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, pad_rows, p));
   else
     BIMASK_CUDA_OK(launch_pdl(fwd_mask_pack_kernel<false, true>, (unsigned)ctas, FWD_THREADS, 0, s,
-        nullptr, nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, p));
+        nullptr, nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, pad_rows, p));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
