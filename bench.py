@@ -420,6 +420,7 @@ def run_gpu(args):
     # ---- per-call breakdown over the same K steps (CUDA events between the C-ABI calls) ----
     names = ["fwd_mask", "spmm_fwd", "perm_search", "bwd_mask", "spmm_dgrad", "wgrad"]
     acc = {li: {n: 0.0 for n in names} for li in range(len(layers))}
+    time.sleep(1.0)      # an idle second: the breakdown starts from the same power state as the headline's timed region
     t_call_begin = time.time()
     for _ in range(args.steps):
         for li, (L, b, _) in enumerate(layers):
