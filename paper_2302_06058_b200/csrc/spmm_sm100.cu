@@ -444,9 +444,11 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
 // owns 512 x N outputs: TWO 256-row MMA tiles that share the activation tile in shared memory, so
 // a stage carries 2 x 16 KB + <= 28 KB + 2 x 2 KB for twice the tensor-pipe work (a third fewer
 // bytes per clock).  Both accumulators (tensor-memory columns 0.. and 256.., N <= 224) belong to
-// the same token tile, so the epilogue cannot overlap the next main loop; instead two groups of four
-// epilogue warps per CTA drain the two accumulators side by side.  Metadata: columns 496..499 and 500..503.
-// Roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 accumulator 0, warps 6-9 accumulator 1.
+// the same token tile and tensor memory has no room for a second pair, so the epilogue cannot overlap a whole
+// main loop; the two groups of four epilogue warps per CTA drain accumulator 0 first, then accumulator 1, and the
+// MMA thread starts the next tile's row tile 0 on the stages already loaded while accumulator 1 is still being
+// drained (about half of the drain is hidden).  Metadata: columns 496..499 and 500..503.
+// Roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-9 epilogue.
 // ------------------------------------------------------------------------------------------
 constexpr int GEMM2M_THREADS = PAIR_THREADS;
 
@@ -478,8 +480,9 @@ spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   const uint32_t tmem_full_bar = bar_base + 8u * (2 * STAGES);
-  const uint32_t tmem_empty_bar = bar_base + 8u * (2 * STAGES + 1);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(staging_ptr + C::STAGING_BYTES + 8 * (2 * STAGES + 2));
+  const uint32_t tmem_empty_bar0 = bar_base + 8u * (2 * STAGES + 1);   // accumulator 0 drained
+  const uint32_t tmem_empty_bar1 = bar_base + 8u * (2 * STAGES + 2);   // accumulator 1 drained
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(staging_ptr + C::STAGING_BYTES + 8 * (2 * STAGES + 3));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -498,7 +501,8 @@ spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
       ptx::mbar_init(empty_bar(s), 1);
     }
     ptx::mbar_init(tmem_full_bar, 1);
-    ptx::mbar_init(tmem_empty_bar, 2 * EPI_WARPS);        // the epilogue warps of both CTAs of the pair
+    ptx::mbar_init(tmem_empty_bar0, 2 * EPI_WARPS);       // the epilogue warps of both CTAs of the pair
+    ptx::mbar_init(tmem_empty_bar1, 2 * EPI_WARPS);
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmapA);
     ptx::prefetch_tmap(&tmapB);
@@ -552,58 +556,81 @@ spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
       const uint32_t idesc = ptx::idesc_bf16(256, SP_N, false, false, true);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++tcount) {
-        // both accumulators must have been drained by all sixteen epilogue warps of the pair
-        if (!ptx::mbar_wait_bounded(tmem_empty_bar, (tcount & 1u) ^ 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
+      // the MMAs of row tile mt (0 / 1) on the stage that holds k tile number `it`
+      auto issue = [&](uint32_t it_, int kt, int mt) {
+        const uint32_t a_s = base + (it_ % STAGES) * C::STAGE_BYTES;
+        const uint32_t b_s = a_s + 2 * C::A_BYTES;
+        const uint32_t e_s = b_s + C::B_MAX;
+        ptx::tmem_cp_128x128b_pair(tmem_meta + 4u * mt, ptx::smem_desc(e_s + mt * C::E_BYTES, 0, 128, 0));
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+          const uint64_t ad = ptx::smem_desc(a_s + mt * C::A_BYTES + kb * 32, 16, 1024, 2);
+          const uint64_t bd = ptx::smem_desc(b_s + (kb >> 1) * b_box + (kb & 1) * 64, 16, 1024, 2);
+          ptx::mma_sparse_pair(tmem_base + 256u * mt, ad, bd, tmem_meta + 4u * mt + (kb & ~1), idesc | (uint32_t)(kb & 1),
+                               (kt | kb) != 0);
+        }
+      };
+      auto wait_full = [&](uint32_t it_) {
+        if (!ptx::mbar_wait_bounded(full_bar(it_ % STAGES), (it_ / STAGES) & 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; ok = false; }
         ptx::tc_fence_after();
-        for (int kt = 0; kt < num_kt; ++kt, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1u;
-          if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; ok = false; break; }
-          ptx::tc_fence_after();
-          const uint32_t a_s = base + s * C::STAGE_BYTES;
-          const uint32_t b_s = a_s + 2 * C::A_BYTES;
-          const uint32_t e_s = b_s + C::B_MAX;
-          ptx::tmem_cp_128x128b_pair(tmem_meta, ptx::smem_desc(e_s, 0, 128, 0));
-          ptx::tmem_cp_128x128b_pair(tmem_meta + 4u, ptx::smem_desc(e_s + C::E_BYTES, 0, 128, 0));
-#pragma unroll
-          for (int mt = 0; mt < 2; ++mt) {
-#pragma unroll
-            for (int kb = 0; kb < 4; ++kb) {
-              const uint64_t ad = ptx::smem_desc(a_s + mt * C::A_BYTES + kb * 32, 16, 1024, 2);
-              const uint64_t bd = ptx::smem_desc(b_s + (kb >> 1) * b_box + (kb & 1) * 64, 16, 1024, 2);
-              ptx::mma_sparse_pair(tmem_base + 256u * mt, ad, bd, tmem_meta + 4u * mt + (kb & ~1), idesc | (uint32_t)(kb & 1),
-                                   (kt | kb) != 0);
-            }
-          }
-          ptx::tc_commit_pair(empty_bar(s), 3);
+        return ok;
+      };
+      for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++tcount) {
+        // The epilogue drains accumulator 0 first (all sixteen warps of the pair), then accumulator 1.  As soon as
+        // accumulator 0 is free, row tile 0 runs ahead over the stages that are already loaded; row tile 1 follows
+        // on the same stages once its accumulator is free, and only then are those stages handed back.
+        const uint32_t eph = (tcount & 1u) ^ 1u;
+        if (!ptx::mbar_wait_bounded(tmem_empty_bar0, eph, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
+        ptx::tc_fence_after();
+        const int ahead = num_kt < STAGES ? num_kt : STAGES;
+        for (int kt = 0; kt < ahead && ok; ++kt)
+          if (wait_full(it + kt)) issue(it + kt, kt, 0);
+        if (!ok) break;
+        if (!ptx::mbar_wait_bounded(tmem_empty_bar1, eph, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; ok = false; break; }
+        ptx::tc_fence_after();
+        for (int kt = 0; kt < ahead; ++kt) {
+          issue(it + kt, kt, 1);
+          ptx::tc_commit_pair(empty_bar((it + kt) % STAGES), 3);
+        }
+        it += ahead;
+        for (int kt = ahead; kt < num_kt && ok; ++kt, ++it) {
+          if (!wait_full(it)) break;
+          issue(it, kt, 0);
+          issue(it, kt, 1);
+          ptx::tc_commit_pair(empty_bar(it % STAGES), 3);
         }
         if (ok) ptx::tc_commit_pair(tmem_full_bar, 3);
       }
     }
   } else {
-    // warps 2-5 drain accumulator 0 (row tile 0), warps 6-9 accumulator 1; a warp reads its own
-    // tensor-memory lane quadrant, a group shares one staging tile
+    // two groups of four epilogue warps (one warp per tensor-memory lane quadrant); both groups drain accumulator 0
+    // first, taking alternate 32-token chunks, then accumulator 1: accumulator 0 is free again at half time, which
+    // is what lets the next tile's first MMAs start under the second half of the drain
     const int q = warp & 3;
-    const int mt = (warp - 2) >> 2;                        // the group of four warps that drains accumulator mt
-    const uint32_t stg = staging + mt * 16384;
+    const int g = (warp - 2) >> 2;
+    const uint32_t stg = staging + g * 16384;
     uint16_t* outp = reinterpret_cast<uint16_t*>(p.out);
-    const uint32_t release_bar = ptx::mapa(tmem_empty_bar, 0);
+    const uint32_t release0 = ptx::mapa(tmem_empty_bar0, 0), release1 = ptx::mapa(tmem_empty_bar1, 0);
     uint32_t tcount = 0;
     for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++tcount) {
       int tile_m, tile_n;
       raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
-      const int m0 = mt128_of(tile_m, mt) * 128, n0 = tile_n * SP_N;
+      const int n0 = tile_n * SP_N;
       bool ok = ptx::mbar_wait_bounded(tmem_full_bar, tcount & 1u, abort_flag, WAIT_BUDGET);
-      ok = ptx::named_bar_and(1 + mt, 128, ok);            // the four warps of a group go on or give up together
+      ok = ptx::named_bar_and(1 + g, 128, ok);             // the four warps of a group go on or give up together
       if (!ok) { *abort_flag = 1; break; }
       ptx::tc_fence_after();
-      const uint32_t acc = tmem_base + 256u * mt + ((uint32_t)(32 * q) << 16);
-      drain_chunks<32>(acc, 0, 1, SP_N / 32, false, release_bar, stg, 1 + mt, q, lane, p.Mdim - m0,
-                       [&](int c, int t) -> uint16_t* {
-        const int n = n0 + 32 * c + t;
-        return n < p.Ndim ? outp + (size_t)n * p.Mdim + m0 : nullptr;
-      });
+#pragma unroll 1
+      for (int mt = 0; mt < 2; ++mt) {
+        const int m0 = mt128_of(tile_m, mt) * 128;
+        const uint32_t acc = tmem_base + 256u * mt + ((uint32_t)(32 * q) << 16);
+        if (mt) ptx::named_bar_sync(1 + g, 128);           // the group's staging tiles are free again
+        drain_chunks<32>(acc, (g ^ mt) & 1, 2, SP_N / 32, false, mt ? release1 : release0, stg, 1 + g, q, lane, p.Mdim - m0,
+                         [&](int c, int t) -> uint16_t* {
+          const int n = n0 + 32 * c + t;
+          return n < p.Ndim ? outp + (size_t)n * p.Mdim + m0 : nullptr;
+        });
+      }
     }
   }
 
