@@ -332,7 +332,7 @@ struct ConvPlan {
 };
 
 // A layer step is a chain of short kernels.  On small layers the kernels are too short to fill the GPU and the
-// step takes as long as its longest dependent chain, so the step is spread over three streams there:
+// step takes as long as its longest dependent chain, so the step is spread over the caller's stream and three side streams there:
 //   caller's stream:  forward mask -> count candidates -> backward mask -> sparse input gradient
 //   side stream A:    candidate generation (needs the seed alone) -> dense weight gradient (needs dY and X alone)
 //   side stream B:    [metadata image of a padded forward operand ->] sparse forward product (needs the forward mask alone)
@@ -415,7 +415,7 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
   uint16_t* dYp = reinterpret_cast<uint16_t*>(ws + w.dyp_off);
   float* partials = w.part_bytes ? reinterpret_cast<float*>(ws + w.part_off) : nullptr;
 
-  // Alg. 1 in order on the caller's stream; small layers spread it over three streams (see SideStream).
+  // Alg. 1 in order on the caller's stream; small layers spread it over side streams as well (see SideStream).
   cudaStream_t s = (cudaStream_t)a->stream;
   const uint16_t* Xmat = a->X;                       // the T x J activation matrix of the explicit products
   uint16_t* dXmat = a->dX;
@@ -425,7 +425,7 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
     if (!conv->imp_fwd || !conv->imp_wgrad)
       if ((rc = launch_im2col3x3(a->X, conv->NB, conv->H, conv->W, conv->C, conv->stride, conv->xcol, s))) return rc;
   }
-  // small layers (between a gigaflop and a hundred): three streams, see SideStream
+  // small layers (between a gigaflop and a hundred): side streams, see SideStream
   const double flops = 2.0 * a->T * a->I * a->J;
   const bool spread = flops >= 1e9 && flops < 1e11;
   SideJoin join;
