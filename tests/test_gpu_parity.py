@@ -191,6 +191,42 @@ def test_metadata_round_trip_through_the_tensor_core():
     assert np.array_equal(Y.float().cpu().numpy().astype(np.float64), expect)
 
 
+def _tmem_image(meta, rows, kwords):
+    """The tensor-memory image of the index codes, rebuilt from the canonical code words by the layout the header
+    documents: one 2048-byte block per (128 rows, 4 code words); image lane L = m0 + 8 h + 16 m2 (m0 < 8, h < 2,
+    m2 < 8) and column c hold, for code word 4 kt + c, half h (low / high 16 bits) of row m0 + 16 m2 in the low 16
+    bits and of row m0 + 8 + 16 m2 in the high 16 bits; entries past the matrix hold the code 0x4 in every nibble."""
+    tm, tk = (rows + 127) // 128, (kwords + 3) // 4
+    full = np.full((tm * 128, tk * 4), 0x44444444, dtype=np.uint64)
+    full[:rows, :kwords] = meta.astype(np.uint64)
+    img = np.zeros((tm, tk, 128, 4), dtype=np.uint32)
+    for L in range(128):
+        m0, h, m2 = L & 7, (L >> 3) & 1, L >> 4
+        lo_rows = np.arange(tm) * 128 + m0 + 16 * m2
+        lo = (full[lo_rows] >> (16 * h)) & 0xFFFF                 # [tm, tk * 4]
+        hi = (full[lo_rows + 8] >> (16 * h)) & 0xFFFF
+        img[:, :, L, :] = (lo | (hi << 16)).astype(np.uint32).reshape(tm, tk, 4)
+    return img.reshape(-1)
+
+
+@pytest.mark.parametrize("I,J,N", [(256, 256, 2), (64, 576, 2), (96, 160, 1), (512, 1184, 2), (1152, 384, 2), (32, 32, 2)])
+def test_metadata_images_of_both_operands_padding_included(I, J, N):
+    """The mask kernels write the tensor-core order of the index codes themselves, on shapes with and without
+    padding: compare both images, word for word, with a re-ordering of the (oracle-checked) canonical code words."""
+    W = special_weights(I, J, 7 * I + J) if I < 1000 else inputs.make_weight(I, J, 6)
+    Wd, b = run_fwd_mask(W, N)
+    b["hw_meta_f"].fill_(255)                             # stale contents must not survive anywhere, padding included
+    bm.bimask_fwd_mask(Wd, I, J, N, 4, b["maskbits_f"], b["vals_f"], b["meta_f"], b["hw_meta_f"])
+    perm = np.random.default_rng(J).permutation(I).astype(np.int32)
+    b["hw_meta_b"].fill_(255)
+    bm.bimask_bwd_mask(Wd, b["maskbits_f"], dev(perm), I, J, N, 4, b["maskbits_b"], b["vals_b"], b["meta_b"], b["hw_meta_b"])
+    torch.cuda.synchronize()
+    got_f = b["hw_meta_f"].cpu().numpy().view(np.uint32)
+    got_b = b["hw_meta_b"].cpu().numpy().view(np.uint32)
+    assert np.array_equal(got_f[: ((I + 127) // 128) * ((J // 32 + 3) // 4) * 512], _tmem_image(u32(b["meta_f"]), I, J // 32))
+    assert np.array_equal(got_b[: ((J + 127) // 128) * ((I // 32 + 3) // 4) * 512], _tmem_image(u32(b["meta_b"]), J, I // 32))
+
+
 def test_do_search_zero_uses_given_perm():
     I, J, T = 128, 160, 70
     W = inputs.make_weight(I, J, 3)
