@@ -17,7 +17,16 @@ constexpr int GEMM_THREADS = 192;                    // warp 0 TMA, warp 1 MMA, 
 // tensor-memory lane quadrant, taking alternate column chunks): products with a short reduction are bound by
 // that drain, not by the tensor pipe.
 constexpr int EPI_WARPS = 8;
-constexpr int PAIR_THREADS = 64 + 32 * EPI_WARPS;
+// One more warp per group of four epilogue warps issues the tensor stores of the group's staged chunks (see
+// drain_chunks_tma / store_chunks): a tensor store costs its issuing thread a few hundred clocks, which the warps
+// that drain tensor memory should not wait for.
+constexpr int EPI_GROUPS = EPI_WARPS / 4;
+constexpr int PAIR_THREADS = 64 + 32 * EPI_WARPS + 32 * EPI_GROUPS;
+// Epilogue staging: per group NT tiles of [32 tokens][128 rows] bf16 (8 KB each), and per group NT "staged" plus NT
+// "freed" mbarriers, kept EPI_BAR_OFFSET bytes into the kernels' barrier area.
+__host__ __device__ constexpr int epi_staging_bytes(int nt) { return EPI_GROUPS * nt * 8192; }
+constexpr uint32_t EPI_BAR_OFFSET = 128;
+
 
 template <int N_TILE, int STAGES, bool SPARSE = true>
 struct Cfg {
@@ -28,9 +37,10 @@ struct Cfg {
   static constexpr int E_BYTES = SPARSE ? 2048 : 0;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
   static constexpr int META_COLS = SPARSE ? 4 : 0;
+  static constexpr int EPI_NT = SPARSE ? 3 : 2;                  // staging tiles per epilogue group (the dense stages leave room for two)
   static constexpr int TMEM_COLS = (N_TILE + META_COLS) <= 128 ? 128 : (N_TILE + META_COLS) <= 256 ? 256 : 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */ +
-                                    EPI_WARPS * 4096 /* epilogue staging: two [32 tokens][128 rows] bf16 tiles per group of four warps */;
+                                    epi_staging_bytes(EPI_NT) /* epilogue staging */;
 };
 
 // A 3x3 convolution as an implicit GEMM: the token operand is an NHWC tensor and a "tile of
@@ -145,12 +155,13 @@ __device__ __forceinline__ uint32_t pack_bf16(uint32_t lo, uint32_t hi) {
   return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-// `dst`: this lane's row address for token group 0 (see drain_chunks); token group g is 2048 bytes further.
-template <int W>
+// `dst`: this lane's row address for token group 0 (see drain_chunks); token group g is GROUP_BYTES further (eight
+// token rows of the staging tile).
+template <int W, uint32_t GROUP_BYTES = 2048u>
 __device__ __forceinline__ void epi_stage(const uint32_t (&r)[W], uint32_t dst) {
 #pragma unroll
   for (int g = 0; g < W / 8; ++g)
-    ptx::stmatrix_x4_trans(dst + 2048u * g, pack_bf16(r[4 * g], r[4 * g + 1]), pack_bf16(r[4 * g + 2], r[4 * g + 3]),
+    ptx::stmatrix_x4_trans(dst + GROUP_BYTES * g, pack_bf16(r[4 * g], r[4 * g + 1]), pack_bf16(r[4 * g + 2], r[4 * g + 3]),
                            pack_bf16(r[W / 2 + 4 * g], r[W / 2 + 4 * g + 1]),
                            pack_bf16(r[W / 2 + 4 * g + 2], r[W / 2 + 4 * g + 3]));
 }
@@ -210,14 +221,12 @@ __device__ __forceinline__ void release_accumulator(uint32_t release_bar, int la
   }
 }
 
-// Drains chunks c0, c0 + cstep, ... (< nchunks) of one accumulator; called by the four warps of a group with the
-// same arguments except `acc` (the warp's lane quadrant q = warp % 4, column of chunk c: W * c).  One chunk is
-// converted and stored while the tensor-memory load of the next is in flight.
-template <int W, typename RowOf>
-__device__ __forceinline__ void drain_chunks(uint32_t acc, int c0, int cstep, int nchunks, bool zero, uint32_t release_bar,
-                                             uint32_t stg, uint32_t bar_id, int q, int lane, int rows_valid, RowOf&& row_of) {
-  if (c0 >= nchunks) { release_accumulator(release_bar, lane); return; }
-  DrainWarp<W> d(stg, bar_id, q, lane, rows_valid);
+// The accumulator loop shared by the two write-out forms below: chunks c0, c0 + cstep, ... (< nchunks) of one
+// accumulator (column of chunk c: W * c) go through emit(registers, c); one chunk is converted and written while the
+// tensor-memory load of the next is in flight.
+template <int W, typename Emit>
+__device__ __forceinline__ void drain_loop(uint32_t acc, int c0, int cstep, int nchunks, bool zero, uint32_t release_bar,
+                                           int lane, Emit&& emit) {
   uint32_t ra[W], rb[W];
   epi_load<W>(acc + W * c0, ra, zero);
 #pragma unroll 1
@@ -225,13 +234,97 @@ __device__ __forceinline__ void drain_chunks(uint32_t acc, int c0, int cstep, in
     if (!zero) ptx::tmem_ld_wait();
     const bool more1 = c + cstep < nchunks;
     if (more1) epi_load<W>(acc + W * (c + cstep), rb, zero); else release_accumulator(release_bar, lane);
-    d.emit(ra, c, row_of);
+    emit(ra, c);
     if (!more1) break;
     if (!zero) ptx::tmem_ld_wait();
     if (c + 2 * cstep < nchunks) epi_load<W>(acc + W * (c + 2 * cstep), ra, zero); else release_accumulator(release_bar, lane);
-    d.emit(rb, c + cstep, row_of);
+    emit(rb, c + cstep);
   }
 }
+
+// Drains chunks c0, c0 + cstep, ... (< nchunks) of one accumulator; called by the four warps of a group with the
+// same arguments except `acc` (the warp's lane quadrant q = warp % 4).  Results leave through per-lane 16-byte
+// stores to addresses that row_of supplies (any token-to-address mapping: the implicit convolution's pixel boxes).
+template <int W, typename RowOf>
+__device__ __forceinline__ void drain_chunks(uint32_t acc, int c0, int cstep, int nchunks, bool zero, uint32_t release_bar,
+                                             uint32_t stg, uint32_t bar_id, int q, int lane, int rows_valid, RowOf&& row_of) {
+  if (c0 >= nchunks) { release_accumulator(release_bar, lane); return; }
+  DrainWarp<W> d(stg, bar_id, q, lane, rows_valid);
+  drain_loop<W>(acc, c0, cstep, nchunks, zero, release_bar, lane, [&](const uint32_t (&r)[W], int c) { d.emit(r, c, row_of); });
+}
+
+// The same drain for results that are a plain [token][row] matrix: a chunk leaves as two tensor stores (TMA) of
+// W tokens x 64 rows, straight from a staging tile, issued by the group's STORE thread (store_chunks below) so
+// that the draining warps never wait for a store to be issued.  A staging tile is two halves [W tokens][64 rows] of
+// 128-byte token rows in the 128-byte-swizzled layout of the tensor map (16-byte unit index XOR token index mod 8
+// -- the same XOR that keeps stmatrix free of bank conflicts).  The group's NT tiles are used in turn over the
+// whole kernel (chunk number u of the group -> tile u % NT); two mbarriers per tile hand it back and forth:
+//   staged[t]  (4 arrivals: one per draining warp, after stmatrix and a proxy fence)   drain -> store thread
+//   freed[t]   (1 arrival: the store thread, once the tile's stores have read it)       store thread -> drain
+// `bars`: the group's barriers (NT staged, then NT freed); `u`: the group's chunk counter, carried from call to
+// call.  Returns false when a wait ran out of budget (the caller raises the abort flag).
+template <int NT>
+__device__ __forceinline__ void epi_bars_init(uint32_t bar_area) {
+#pragma unroll
+  for (int g = 0; g < EPI_GROUPS; ++g)
+#pragma unroll
+    for (int t = 0; t < NT; ++t) {
+      ptx::mbar_init(bar_area + EPI_BAR_OFFSET + 8u * (g * 2 * NT + t), 4);
+      ptx::mbar_init(bar_area + EPI_BAR_OFFSET + 8u * (g * 2 * NT + NT + t), 1);
+    }
+}
+template <int NT>
+__device__ __forceinline__ uint32_t epi_bars_of(uint32_t bar_area, int g) { return bar_area + EPI_BAR_OFFSET + 8u * (g * 2 * NT); }
+
+template <int W, int NT>
+__device__ __forceinline__ bool drain_chunks_tma(uint32_t acc, int c0, int cstep, int nchunks, bool zero, uint32_t release_bar,
+                                                 uint32_t stg, uint32_t bars, uint32_t& u, int q, int lane,
+                                                 volatile int* abort_flag) {
+  if (c0 >= nchunks) { release_accumulator(release_bar, lane); return true; }
+  // stmatrix: lane 8 i + k addresses token k (of a group of eight) of matrix i = rows 32 q + 8 i .. + 7, i.e. 16-byte
+  // unit 4 (q & 1) + i of the token's row in half q >> 1
+  const uint32_t dst = stg + (uint32_t)(q >> 1) * (uint32_t)(W * 128) + (uint32_t)(lane & 7) * 128u +
+                       ((((uint32_t)(4 * (q & 1)) + ((uint32_t)lane >> 3)) ^ ((uint32_t)lane & 7u)) << 4);
+  bool ok = true;
+  drain_loop<W>(acc, c0, cstep, nchunks, zero, release_bar, lane, [&](const uint32_t (&r)[W], int) {
+    const uint32_t slot = u % NT, use = u / NT;
+    ++u;
+    if (use > 0 && ok) ok = ptx::mbar_wait_bounded(bars + 8u * (NT + slot), (use - 1u) & 1u, abort_flag, WAIT_BUDGET);
+    epi_stage<W, 1024u>(r, dst + slot * 8192u);
+    ptx::fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) ptx::mbar_arrive(bars + 8u * slot);
+  });
+  return ok;
+}
+
+// The store thread's side of drain_chunks_tma, called with the same chunk sequence: waits for a staged tile, issues
+// its stores (rows and tokens outside the result are clipped by the tensor map, extent Mdim x Ndim; a store that
+// would start outside is not issued), and hands back the tile of the previous chunk once its stores have read it.
+// x0: first row of the CTA's 128; y0: first token of chunk 0.  After its last call the thread runs store_finish().
+template <int W, int NT>
+__device__ __forceinline__ bool store_chunks(const CUtensorMap* tmapD, int c0, int cstep, int nchunks, uint32_t stg,
+                                             uint32_t bars, uint32_t& u, int x0, int y0, int Mdim, int Ndim,
+                                             volatile int* abort_flag) {
+  for (int c = c0; c < nchunks; c += cstep) {
+    const uint32_t slot = u % NT, use = u / NT;
+    if (!ptx::mbar_wait_bounded(bars + 8u * slot, use & 1u, abort_flag, WAIT_BUDGET)) return false;
+    const int y = y0 + W * c;
+    if (y < Ndim && x0 < Mdim) {
+      ptx::tma_store_2d(tmapD, x0, y, stg + slot * 8192u);
+      if (x0 + 64 < Mdim) ptx::tma_store_2d(tmapD, x0 + 64, y, stg + slot * 8192u + (uint32_t)(W * 128));
+    }
+    ptx::bulk_commit();
+    if (u > 0) {
+      ptx::bulk_wait_read<1>();
+      ptx::mbar_arrive(bars + 8u * (NT + (u - 1u) % NT));
+    }
+    ++u;
+  }
+  return true;
+}
+// Shared memory must outlive the stores that read it.
+__device__ __forceinline__ void store_finish() { ptx::bulk_wait_read<0>(); }
 
 // ---- host helpers (gemm_host.cu) -----------------------------------------------------------
 int sm_count();

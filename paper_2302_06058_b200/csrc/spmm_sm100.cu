@@ -27,19 +27,19 @@ namespace {
 template <int N_TILE, int STAGES, bool SPARSE, bool CONV>
 __global__ void __launch_bounds__(PAIR_THREADS, 1)
 spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-                   const GemmParams p) {
+                   const __grid_constant__ CUtensorMap tmapD, const GemmParams p) {
   pdl_launch_dependents();
   using C = Cfg<N_TILE, STAGES, SPARSE>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - raw);
-  const uint32_t staging = base + STAGES * C::STAGE_BYTES;      // epilogue staging, 8 KB per group of four warps
-  const uint32_t bar_base = staging + EPI_WARPS * 4096;
+  const uint32_t staging = base + STAGES * C::STAGE_BYTES;      // epilogue staging, C::EPI_NT tiles of 8 KB per group of four warps
+  const uint32_t bar_base = staging + epi_staging_bytes(C::EPI_NT);
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   const uint32_t tmem_full_bar = bar_base + 8u * (2 * STAGES);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * C::STAGE_BYTES + EPI_WARPS * 4096 + 8 * (2 * STAGES + 1));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * C::STAGE_BYTES + epi_staging_bytes(C::EPI_NT) + 8 * (2 * STAGES + 1));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -61,9 +61,11 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
       ptx::mbar_init(empty_bar(s), 1);
     }
     ptx::mbar_init(tmem_full_bar, 1);
+    epi_bars_init<C::EPI_NT>(bar_base);
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmapA);
     ptx::prefetch_tmap(&tmapB);
+    if (!CONV) ptx::prefetch_tmap(&tmapD);
   }
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
@@ -164,7 +166,7 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
       }
       if (ok) ptx::tc_commit(tmem_full_bar);
     }
-  } else {
+  } else if (warp < 2 + EPI_WARPS) {
     // ------------------------------ epilogue ------------------------------
     const int q = warp & 3;                               // TMEM lane quadrant this warp may read
     bool ok = true;
@@ -174,10 +176,10 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     const int eg = (warp - 2) >> 2;                      // EPI_WARPS / 4 groups of four warps take chunks in turn
     ok = ptx::named_bar_and(1 + eg, 128, ok);            // the four warps of a group go on or give up together
     if (ok) {
-      uint16_t* outp = reinterpret_cast<uint16_t*>(p.out);
-      drain_chunks<32>(tmem_base + ((uint32_t)(32 * q) << 16), eg, EPI_WARPS / 4, N_TILE / 32, num_kt <= 0, 0u,
-                       staging + eg * 16384, 1 + eg, q, lane, p.Mdim - m0, [&](int c, int t) -> uint16_t* {
-        if (CONV) {
+      if constexpr (CONV) {
+        uint16_t* outp = reinterpret_cast<uint16_t*>(p.out);
+        drain_chunks<32>(tmem_base + ((uint32_t)(32 * q) << 16), eg, EPI_GROUPS, N_TILE / 32, num_kt <= 0, 0u,
+                         staging + eg * (C::EPI_NT * 8192), 1 + eg, q, lane, p.Mdim - m0, [&](int c, int t) -> uint16_t* {
           // token 32c + t of the box: pixel (cw0 + ., ch0 + .) of image cn0 + .
           const int rr = 32 * c + t;
           const int w = cw0 + (rr & (p.conv.wb - 1));
@@ -185,10 +187,24 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
           const int n = cn0 + (rr >> (p.conv.lg_wb + p.conv.lg_hb));
           if (w >= p.conv.W || h >= p.conv.H || n >= p.conv.NB) return nullptr;
           return outp + conv_out_pixel(p.conv, n, h, w) * p.Mdim + m0;
-        }
-        const int n = n0 + 32 * c + t;
-        return n < p.Ndim ? outp + (size_t)n * p.Mdim + m0 : nullptr;
-      });
+        });
+      } else {
+        uint32_t u = 0;
+        if (!drain_chunks_tma<32, C::EPI_NT>(tmem_base + ((uint32_t)(32 * q) << 16), eg, EPI_GROUPS, N_TILE / 32, num_kt <= 0, 0u,
+                                             staging + eg * (C::EPI_NT * 8192), epi_bars_of<C::EPI_NT>(bar_base, eg), u, q, lane,
+                                             abort_flag))
+          *abort_flag = 1;
+      }
+    }
+  } else if (!CONV) {
+    // ------------------------------ store threads: one per epilogue group ------------------------------
+    if (ptx::elect_one()) {
+      const int g = warp - 2 - EPI_WARPS;
+      uint32_t u = 0;
+      if (!store_chunks<32, C::EPI_NT>(&tmapD, g, EPI_GROUPS, N_TILE / 32, staging + g * (C::EPI_NT * 8192),
+                                       epi_bars_of<C::EPI_NT>(bar_base, g), u, m0, n0, p.Mdim, p.Ndim, abort_flag))
+        *abort_flag = 1;
+      store_finish();
     }
   }
 
@@ -219,7 +235,8 @@ struct PairPCfg {
   static constexpr int B_MAX = 32768;                      // up to 128 rows x 128 bf16 (two 64-wide boxes)
   static constexpr int E_BYTES = SPARSE ? 2048 : 0;
   static constexpr int STAGE_BYTES = A_BYTES + B_MAX + E_BYTES;        // 50 KB / 64 KB (the B part is N / 2 rows)
-  static constexpr int STAGING_BYTES = EPI_WARPS * 4096;   // per group of four epilogue warps: two [32 tokens][128 rows] bf16 tiles
+  static constexpr int EPI_NT = SPARSE ? 3 : 2;            // staging tiles ([32 tokens][128 rows] bf16) per group of four epilogue warps
+  static constexpr int STAGING_BYTES = epi_staging_bytes(EPI_NT);
   static constexpr int TMEM_COLS = 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 + 256;
 };
@@ -230,7 +247,8 @@ struct PairPCfg {
 template <int STAGES, bool CONV, bool SPARSE = true>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PAIR_THREADS, 1)
 spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-                            const __grid_constant__ CUtensorMap tmapE, const GemmParams p) {
+                            const __grid_constant__ CUtensorMap tmapE, const __grid_constant__ CUtensorMap tmapD,
+                            const GemmParams p) {
   static_assert(SPARSE || !CONV, "the implicit convolution runs on 2:4 operands only");
   pdl_launch_dependents();
   using C = PairPCfg<STAGES, SPARSE>;
@@ -268,10 +286,12 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
       ptx::mbar_init(tmem_full_bar(b), 1);
       ptx::mbar_init(tmem_empty_bar(b), 2 * EPI_WARPS);   // the epilogue warps of both CTAs of the pair
     }
+    epi_bars_init<C::EPI_NT>(bar_base);
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmapA);
     ptx::prefetch_tmap(&tmapB);
     ptx::prefetch_tmap(&tmapE);
+    if (!CONV) ptx::prefetch_tmap(&tmapD);
   }
   if (warp == 1) {
     ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
@@ -376,14 +396,15 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
         if (ok) ptx::tc_commit_pair(tmem_full_bar(buf), 3);
       }
     }
-  } else {
+  } else if (warp < 2 + EPI_WARPS) {
     // Each epilogue warp reads 32 accumulator rows (its TMEM lane quadrant); the four warps of a group share
-    // one staging tile.
+    // the group's staging tiles.
     const int q = warp & 3;
-    const int eg = (warp - 2) >> 2;                        // EPI_WARPS / 4 groups of four warps take chunks in turn
-    const uint32_t stg = staging + eg * 16384;
+    const int eg = (warp - 2) >> 2;                        // EPI_GROUPS groups of four warps take chunks in turn
+    const uint32_t stg = staging + eg * (C::EPI_NT * 8192);
+    const uint32_t ebars = epi_bars_of<C::EPI_NT>(bar_base, eg);
     uint16_t* outp = reinterpret_cast<uint16_t*>(p.out);
-    uint32_t tcount = 0;
+    uint32_t tcount = 0, u = 0;
     for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++tcount) {
       int tile_m, tile_n;
       raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
@@ -398,7 +419,7 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
       const int nchunks = (CONV || (SP_N & 31) == 0) ? SP_N / 32 : SP_N / 16;
       if (CONV) {
         // accumulator columns [0, SP_N/2) are the pixels of box 2*tile_n, the rest those of box 2*tile_n + 1
-        drain_chunks<32>(acc, eg, EPI_WARPS / 4, nchunks, false, release_bar, stg, 1 + eg, q, lane, p.Mdim - m0,
+        drain_chunks<32>(acc, eg, EPI_GROUPS, nchunks, false, release_bar, stg, 1 + eg, q, lane, p.Mdim - m0,
                          [&](int c, int t) -> uint16_t* {
           const int half = (32 * c) / (SP_N / 2);
           const int rr = 32 * c - half * (SP_N / 2) + t;
@@ -411,18 +432,34 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
           return outp + conv_out_pixel(p.conv, n, h, w) * p.Mdim + m0;
         });
       } else if ((SP_N & 31) == 0) {
-        drain_chunks<32>(acc, eg, EPI_WARPS / 4, nchunks, false, release_bar, stg, 1 + eg, q, lane, p.Mdim - m0,
-                         [&](int c, int t) -> uint16_t* {
-          const int n = n0 + 32 * c + t;
-          return n < p.Ndim ? outp + (size_t)n * p.Mdim + m0 : nullptr;
-        });
+        if (!drain_chunks_tma<32, C::EPI_NT>(acc, eg, EPI_GROUPS, nchunks, false, release_bar, stg, ebars, u, q, lane, abort_flag)) {
+          *abort_flag = 1;
+          break;
+        }
       } else {
-        drain_chunks<16>(acc, eg, EPI_WARPS / 4, nchunks, false, release_bar, stg, 1 + eg, q, lane, p.Mdim - m0,
-                         [&](int c, int t) -> uint16_t* {
-          const int n = n0 + 16 * c + t;
-          return n < p.Ndim ? outp + (size_t)n * p.Mdim + m0 : nullptr;
-        });
+        if (!drain_chunks_tma<16, C::EPI_NT>(acc, eg, EPI_GROUPS, nchunks, false, release_bar, stg, ebars, u, q, lane, abort_flag)) {
+          *abort_flag = 1;
+          break;
+        }
       }
+    }
+  } else if (!CONV) {
+    // store threads, one per epilogue group: the same walk over tiles and chunks as the group's draining warps
+    if (ptx::elect_one()) {
+      const int g = warp - 2 - EPI_WARPS;
+      const uint32_t stg = staging + g * (C::EPI_NT * 8192);
+      const uint32_t ebars = epi_bars_of<C::EPI_NT>(bar_base, g);
+      uint32_t u = 0;
+      for (int tile = cluster_id; tile < num_tiles; tile += num_clusters) {
+        int tile_m, tile_n;
+        raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
+        const int m0 = (2 * tile_m + (int)rank) * 128, n0 = tile_n * SP_N;
+        const bool ok = (SP_N & 31) == 0
+            ? store_chunks<32, C::EPI_NT>(&tmapD, g, EPI_GROUPS, SP_N / 32, stg, ebars, u, m0, n0, p.Mdim, p.Ndim, abort_flag)
+            : store_chunks<16, C::EPI_NT>(&tmapD, g, EPI_GROUPS, SP_N / 16, stg, ebars, u, m0, n0, p.Mdim, p.Ndim, abort_flag);
+        if (!ok) { *abort_flag = 1; break; }
+      }
+      store_finish();
     }
   }
 
@@ -458,7 +495,8 @@ struct Pair2MCfg {
   static constexpr int B_MAX = 28672;                      // 112 rows x 128 bf16 (two 64-wide boxes), N <= 224
   static constexpr int E_BYTES = 2048;
   static constexpr int STAGE_BYTES = 2 * A_BYTES + B_MAX + 2 * E_BYTES;      // 64 KB
-  static constexpr int STAGING_BYTES = EPI_WARPS * 4096;   // per group of four epilogue warps: two [32 tokens][128 rows] bf16 tiles
+  static constexpr int EPI_NT = 2;                         // staging tiles per epilogue group: 8 KB each, and 3 x 64 KB of stages leave room for four
+  static constexpr int STAGING_BYTES = epi_staging_bytes(EPI_NT);
   static constexpr int TMEM_COLS = 512;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 + 256;
 };
@@ -466,7 +504,7 @@ struct Pair2MCfg {
 template <int STAGES>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2M_THREADS, 1)
 spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-                   const __grid_constant__ CUtensorMap tmapE,
+                   const __grid_constant__ CUtensorMap tmapE, const __grid_constant__ CUtensorMap tmapD,
                    const GemmParams p) {
   pdl_launch_dependents();
   using C = Pair2MCfg<STAGES>;
@@ -503,10 +541,12 @@ spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
     ptx::mbar_init(tmem_full_bar, 1);
     ptx::mbar_init(tmem_empty_bar0, 2 * EPI_WARPS);       // the epilogue warps of both CTAs of the pair
     ptx::mbar_init(tmem_empty_bar1, 2 * EPI_WARPS);
+    epi_bars_init<C::EPI_NT>(bar_base);
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmapA);
     ptx::prefetch_tmap(&tmapB);
     ptx::prefetch_tmap(&tmapE);
+    ptx::prefetch_tmap(&tmapD);
   }
   if (warp == 1) {
     ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
@@ -602,35 +642,48 @@ spmm_pair2m_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
         if (ok) ptx::tc_commit_pair(tmem_full_bar, 3);
       }
     }
-  } else {
+  } else if (warp < 2 + EPI_WARPS) {
     // two groups of four epilogue warps (one warp per tensor-memory lane quadrant); both groups drain accumulator 0
     // first, taking alternate 32-token chunks, then accumulator 1: accumulator 0 is free again at half time, which
     // is what lets the next tile's first MMAs start under the second half of the drain
     const int q = warp & 3;
     const int g = (warp - 2) >> 2;
-    const uint32_t stg = staging + g * 16384;
-    uint16_t* outp = reinterpret_cast<uint16_t*>(p.out);
+    const uint32_t stg = staging + g * (C::EPI_NT * 8192);
+    const uint32_t ebars = epi_bars_of<C::EPI_NT>(bar_base, g);
+    uint32_t u = 0;
     const uint32_t release0 = ptx::mapa(tmem_empty_bar0, 0), release1 = ptx::mapa(tmem_empty_bar1, 0);
     uint32_t tcount = 0;
     for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++tcount) {
-      int tile_m, tile_n;
-      raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
-      const int n0 = tile_n * SP_N;
       bool ok = ptx::mbar_wait_bounded(tmem_full_bar, tcount & 1u, abort_flag, WAIT_BUDGET);
       ok = ptx::named_bar_and(1 + g, 128, ok);             // the four warps of a group go on or give up together
       if (!ok) { *abort_flag = 1; break; }
       ptx::tc_fence_after();
 #pragma unroll 1
       for (int mt = 0; mt < 2; ++mt) {
-        const int m0 = mt128_of(tile_m, mt) * 128;
         const uint32_t acc = tmem_base + 256u * mt + ((uint32_t)(32 * q) << 16);
-        if (mt) ptx::named_bar_sync(1 + g, 128);           // the group's staging tiles are free again
-        drain_chunks<32>(acc, (g ^ mt) & 1, 2, SP_N / 32, false, mt ? release1 : release0, stg, 1 + g, q, lane, p.Mdim - m0,
-                         [&](int c, int t) -> uint16_t* {
-          const int n = n0 + 32 * c + t;
-          return n < p.Ndim ? outp + (size_t)n * p.Mdim + m0 : nullptr;
-        });
+        if (!drain_chunks_tma<32, C::EPI_NT>(acc, (g ^ mt) & 1, 2, SP_N / 32, false, mt ? release1 : release0, stg, ebars, u, q,
+                                             lane, abort_flag))
+          *abort_flag = 1;
       }
+      if (*abort_flag) break;
+    }
+  } else {
+    // store threads, one per epilogue group: the same walk over tiles, row tiles and chunks as the group's draining warps
+    if (ptx::elect_one()) {
+      const int g = warp - 2 - EPI_WARPS;
+      const uint32_t stg = staging + g * (C::EPI_NT * 8192);
+      const uint32_t ebars = epi_bars_of<C::EPI_NT>(bar_base, g);
+      uint32_t u = 0;
+      bool ok = true;
+      for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+        int tile_m, tile_n;
+        raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
+        for (int mt = 0; mt < 2 && ok; ++mt)
+          ok = store_chunks<32, C::EPI_NT>(&tmapD, (g ^ mt) & 1, 2, SP_N / 32, stg, ebars, u, mt128_of(tile_m, mt) * 128, tile_n * SP_N,
+                                           p.Mdim, p.Ndim, abort_flag);
+      }
+      if (!ok) *abort_flag = 1;
+      store_finish();
     }
   }
 
@@ -648,10 +701,11 @@ template <int N_TILE, int STAGES, bool SPARSE = true>
 int run_single(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, int Mdim, int Ndim, int Kdim,
                uint16_t* out, int32_t* status_word, cudaStream_t s) {
   using C = Cfg<N_TILE, STAGES, SPARSE>;
-  CUtensorMap ta, tb;
+  CUtensorMap ta, tb, td;
   int rc;
   if ((rc = make_tmap(&ta, vals, SPARSE ? (uint64_t)Kdim / 2 : (uint64_t)Kdim, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, N_TILE)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap(&td, out, (uint64_t)Mdim, (uint64_t)Ndim, 32)) != BIMASK_OK) return rc;   // result: 32 tokens x 64 rows per store
   auto kern = spmm_single_kernel<N_TILE, STAGES, SPARSE, false>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
@@ -666,7 +720,7 @@ int run_single(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, i
   p.tiles_n = (Ndim + N_TILE - 1) / N_TILE;
   p.raster_group = 16;
   dim3 grid(p.tiles_m * p.tiles_n, 1, 1);
-  BIMASK_CUDA_OK(launch_pdl(kern, grid, PAIR_THREADS, C::SMEM_BYTES, s, ta, tb, p));
+  BIMASK_CUDA_OK(launch_pdl(kern, grid, PAIR_THREADS, C::SMEM_BYTES, s, ta, tb, td, p));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -697,7 +751,7 @@ int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const 
                                int Kdim, uint16_t* out, int32_t* status_word, cudaStream_t s) {
   constexpr int STAGES = 3;
   using C = PairPCfg<STAGES>;
-  CUtensorMap ta, tb, te;
+  CUtensorMap ta, tb, te, td;
   int rc;
   const int tiles_m = (Mdim + 127) / 128, tiles_k = (Kdim + 127) / 128;
   const int sms = sm_count();
@@ -705,6 +759,7 @@ int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const 
   if ((rc = make_tmap(&ta, vals, (uint64_t)Kdim / 2, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, n_tile / 2)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_meta(&te, hw_meta, (uint64_t)tiles_m * tiles_k)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap(&td, out, (uint64_t)Mdim, (uint64_t)Ndim, n_tile % 32 == 0 ? 32 : 16)) != BIMASK_OK) return rc;   // one chunk of the drain
   auto kern = spmm_pair_persistent_kernel<STAGES, false>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
@@ -721,7 +776,7 @@ int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const 
   p.raster_group = 8;
   const int total = p.tiles_m * p.tiles_n;
   const int clusters = total < sms / 2 ? total : sms / 2;
-  BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s, ta, tb, te, p));
+  BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s, ta, tb, te, td, p));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -745,7 +800,7 @@ int run_sparse_pair2m(const uint16_t* vals, const void* hw_meta, const uint16_t*
                       uint16_t* out, int32_t* status_word, cudaStream_t s) {
   constexpr int STAGES = 3;
   using C = Pair2MCfg<STAGES>;
-  CUtensorMap ta, tb, te;
+  CUtensorMap ta, tb, te, td;
   int rc;
   const int tiles_m = (Mdim + 127) / 128, tiles_k = (Kdim + 127) / 128;
   const int sms = sm_count();
@@ -754,6 +809,7 @@ int run_sparse_pair2m(const uint16_t* vals, const void* hw_meta, const uint16_t*
   if ((rc = make_tmap(&ta, vals, (uint64_t)Kdim / 2, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, n_tile / 2)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_meta(&te, hw_meta, (uint64_t)tiles_m * tiles_k)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap(&td, out, (uint64_t)Mdim, (uint64_t)Ndim, 32)) != BIMASK_OK) return rc;
   auto kern = spmm_pair2m_kernel<STAGES>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
@@ -772,7 +828,7 @@ int run_sparse_pair2m(const uint16_t* vals, const void* hw_meta, const uint16_t*
   p.raster_group = 8;
   const int total = p.tiles_m * p.tiles_n;
   const int clusters = total < sms / 2 ? total : sms / 2;
-  BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, GEMM2M_THREADS, C::SMEM_BYTES, s, ta, tb, te, p));
+  BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, GEMM2M_THREADS, C::SMEM_BYTES, s, ta, tb, te, td, p));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -818,7 +874,7 @@ int run_conv_single(const uint16_t* vals, int a_rows, int a_kdim, const void* hw
   p.raster_group = 16;
   p.n_tile = N_TILE;
   dim3 grid(p.tiles_m * p.tiles_n, 1, 1);
-  BIMASK_CUDA_OK(launch_pdl(kern, grid, PAIR_THREADS, C::SMEM_BYTES, s, ta, tb, p));
+  BIMASK_CUDA_OK(launch_pdl(kern, grid, PAIR_THREADS, C::SMEM_BYTES, s, ta, tb, ta /* result map: not used by the convolution */, p));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -854,7 +910,7 @@ int run_conv_pair(const uint16_t* vals, int a_rows, int a_kdim, const void* hw_m
   p.raster_group = 8;
   const int total = p.tiles_m * p.tiles_n;
   const int clusters = total < sms / 2 ? total : sms / 2;
-  BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s, ta, tb, te, p));
+  BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s, ta, tb, te, ta /* result map: not used by the convolution */, p));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
@@ -927,7 +983,7 @@ int run_dense_pair_persistent(const uint16_t* A, const uint16_t* Bop, int Mdim, 
                               int32_t* status_word, cudaStream_t s) {
   constexpr int STAGES = 3;
   using C = PairPCfg<STAGES, false>;
-  CUtensorMap ta, tb;
+  CUtensorMap ta, tb, td;
   int rc;
   const int tiles_m = (Mdim + 127) / 128, tiles_k = (Kdim + 127) / 128;
   const int sms = sm_count();
@@ -941,6 +997,7 @@ int run_dense_pair_persistent(const uint16_t* A, const uint16_t* Bop, int Mdim, 
   }
   if ((rc = make_tmap(&ta, A, (uint64_t)Kdim, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, n_tile / 2)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap(&td, out, (uint64_t)Mdim, (uint64_t)Ndim, 32)) != BIMASK_OK) return rc;
   auto kern = spmm_pair_persistent_kernel<STAGES, false, false>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
@@ -957,7 +1014,7 @@ int run_dense_pair_persistent(const uint16_t* A, const uint16_t* Bop, int Mdim, 
   p.raster_group = 8;
   const int total = p.tiles_m * p.tiles_n;
   const int clusters = total < sms / 2 ? total : sms / 2;
-  BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s, ta, tb, ta, p));
+  BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, PAIR_THREADS, C::SMEM_BYTES, s, ta, tb, ta /* no metadata */, td, p));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
