@@ -333,6 +333,8 @@ int sm_count();
 int make_tmap(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, uint32_t box_rows);
 // The metadata image as a 2-D tensor of u32: 256 words per row, two rows per 2048-byte block.
 int make_tmap_meta(CUtensorMap* m, const void* ptr, uint64_t blocks);
+// fp32 [planes][rows][inner] for stores of 32 x 128 boxes (the dense product's result or its split-K partial sums).
+int make_tmap_f32_store(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t rows, uint64_t planes);
 // 4-D bf16 map of an NHWC tensor (channels, W, H, NB) for loads of 64-channel pixel boxes, 128-byte swizzle.
 // estride 2: a box takes every second pixel along W and H (wb x hb pixels all the same).
 int make_tmap_nhwc_load(CUtensorMap* m, const void* ptr, int CH, int W, int H, int NB, int wb, int hb, int nb, int estride = 1);

@@ -230,6 +230,14 @@ int make_tmap_nhwc_load(CUtensorMap* m, const void* ptr, int CH, int W, int H, i
   return encode_cached(m, k);
 }
 
+// fp32 result of the dense product, [planes][rows][inner] densely packed (planes = split-K partial sums), for stores
+// of 32-column x 128-row boxes in the 128-byte-swizzled layout; rows and columns past the extents are clipped.
+int make_tmap_f32_store(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t rows, uint64_t planes) {
+  TmapKey k{ptr, inner, rows, inner * 4, 32, 128, (int)CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (int)CU_TENSOR_MAP_SWIZZLE_128B};
+  k.d2 = planes; k.d3 = 1; k.box2 = 1; k.box3 = 1;
+  return encode_cached(m, k);
+}
+
 // Generic 2-D tensor map without swizzle: `inner` contiguous elements of `elem_bytes` per row.
 int make_tmap_plain(CUtensorMap* m, int dtype, const void* ptr, uint64_t inner, uint64_t outer, uint32_t box_inner,
                     uint32_t box_outer, uint32_t elem_bytes) {

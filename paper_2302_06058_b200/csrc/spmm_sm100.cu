@@ -726,22 +726,23 @@ int run_single(const uint16_t* vals, const void* hw_meta, const uint16_t* Bop, i
   return BIMASK_OK;
 }
 
-// Output-tile width of the CTA-pair 2:4 product.  Cost model in SM clocks, fitted to measurements: a tile's main
-// loop takes 2 N clocks per 128-deep k tile; its epilogue (eight warps, two per lane quadrant) about 1100 clocks per
-// 32-column chunk and warp, or 890 per 16-column chunk when N is not a multiple of 32; with N <= 240 the two
-// overlap (two accumulators), with N = 256 they add up; narrower tiles re-read the compressed operand more often
-// (L2 traffic), 0.3 % per column given up; the kernel's time is the number of passes over the clusters times the
-// tile time.  (Short reductions are epilogue-bound: there a multiple of 32 wins.)
+// Output-tile width of the CTA-pair 2:4 product.  Cost model in SM clocks, fitted to measurements: per 128-deep k
+// tile a CTA takes in 18 KB of compressed weights and metadata plus 128 N bytes of activations at about 64 bytes per
+// clock (short reductions and narrow tiles are bound by that, not by the 2 N clocks of the MMAs); the epilogue (two
+// groups of four draining warps, a store warp each) takes about 430 clocks per 32-column chunk and group; with
+// N <= 224 the two overlap (two accumulators), with N = 256 they add up; the kernel's time is the number of passes
+// over the clusters times the tile time.
 int choose_sparse_n(int pair_tiles_m, int Ndim, int k_tiles, int clusters) {
   int best_n = 256;
   double best = 1e30;
-  for (int n = 256; n >= 160; n -= 16) {
+  for (int n = 256; n >= 96; n -= 32) {                     // multiples of 32 only: 16-column chunks drain at 570 clocks each
     const long long tiles = (long long)pair_tiles_m * ((Ndim + n - 1) / n);
     const long long rounds = (tiles + clusters - 1) / clusters;
-    const double mainloop = (double)k_tiles * 2.0 * n;
-    const double epilogue = (n % 32 == 0) ? ((n / 32 + 1) / 2) * 1100.0 : ((n / 16 + 1) / 2) * 890.0;
+    const double feed = (18432.0 + 128.0 * n) / 64.0;
+    const double mainloop = (double)k_tiles * (2.0 * n > feed ? 2.0 * n : feed);
+    const double epilogue = ((n / 32 + 1) / 2) * 430.0;
     const double tile = n == 256 ? mainloop + epilogue : (mainloop > epilogue ? mainloop : epilogue);
-    const double cost = (double)rounds * tile * (1.0 + 0.003 * (256 - n));
+    const double cost = (double)rounds * tile * (1.0 + 0.001 * (256 - n));
     if (cost < best) { best = cost; best_n = n; }
   }
   return best_n;

@@ -16,32 +16,108 @@ namespace {
 // 128-byte runs of fp32 in global memory) overlaps the main loop of the next.
 // Work items are (tile, k-split) pairs; with more than one split the partial sums go to scratch.
 // ------------------------------------------------------------------------------------------
+// Epilogue of both kernels.  The accumulator holds D[row][column] with row = tensor-memory lane, and dW is
+// row-major, so a lane owns 128 contiguous bytes per 32-column chunk -- but stored from registers every instruction
+// of a warp would touch 32 different lines.  Instead the four draining warps write the chunk (128 rows x 128 bytes)
+// into one of two staging tiles in the 128-byte-swizzled layout (16-byte unit index XOR row mod 8: conflict-free
+// 16-byte shared stores) and a fifth warp's elected thread sends the tile off with one tensor store (TMA) of a
+// 32 x 128 box; rows and columns outside dW are clipped by the tensor map.  Two mbarriers per tile hand it back and
+// forth: staged[t] (four arrivals, one per draining warp) and freed[t] (the store thread, once the store has read
+// the tile).  `u`: the CTA's chunk counter, carried from work item to work item (tile u % 2).
+constexpr int WGRAD_THREADS = GEMM_THREADS + 32;                 // + the store warp
+constexpr int WGRAD_STAGING_BYTES = 2 * 16384;
+constexpr uint32_t WGRAD_EPI_BAR_OFFSET = 160;                   // staged[2], freed[2] inside the barrier area, past the kernels' own barriers and words
+
+__device__ __forceinline__ void wgrad_epi_bars_init(uint32_t bar_area) {
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    ptx::mbar_init(bar_area + WGRAD_EPI_BAR_OFFSET + 8u * t, 4);
+    ptx::mbar_init(bar_area + WGRAD_EPI_BAR_OFFSET + 8u * (2 + t), 1);
+  }
+}
+
+// One draining warp's share of an accumulator: lane quadrant q, columns 0..255 in eight chunks.  `acc`: the
+// accumulator's tensor-memory address with the quadrant's lane offset.  release() is called once the last chunk has
+// been read from tensor memory.  Returns false when a wait ran out of budget.
+template <typename Release>
+__device__ __forceinline__ bool wgrad_drain(uint32_t acc, uint32_t stg, uint32_t bar_area, uint32_t& u, int q, int lane,
+                                            volatile int* abort_flag, Release&& release) {
+  const uint32_t bars = bar_area + WGRAD_EPI_BAR_OFFSET;
+  const uint32_t row = (uint32_t)(32 * q + lane);
+  const uint32_t row_addr = stg + row * 128u;
+  const uint32_t sw = row & 7u;
+  bool ok = true;
+  auto stage = [&](const uint32_t (&r)[32]) {
+    const uint32_t slot = u & 1u, use = u >> 1;
+    ++u;
+    if (use > 0 && ok) ok = ptx::mbar_wait_bounded(bars + 8u * (2 + slot), (use - 1u) & 1u, abort_flag, WAIT_BUDGET);
+#pragma unroll
+    for (uint32_t j = 0; j < 8; ++j)
+      ptx::st_shared_v4(row_addr + slot * 16384u + ((j ^ sw) << 4), r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+    ptx::fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) ptx::mbar_arrive(bars + 8u * slot);
+  };
+  uint32_t ra[32], rb[32];
+  ptx::tmem_ld_32x32(acc, ra);
+#pragma unroll 1
+  for (int c = 0; c < 8; c += 2) {
+    ptx::tmem_ld_wait();
+    ptx::tmem_ld_32x32(acc + 32 * (c + 1), rb);
+    stage(ra);
+    ptx::tmem_ld_wait();
+    if (c + 2 < 8) ptx::tmem_ld_32x32(acc + 32 * (c + 2), ra); else release();
+    stage(rb);
+  }
+  return ok;
+}
+
+// The store thread's side for one work item: first row m0 of the CTA's 128, first column n0 of the tile's 256.
+__device__ __forceinline__ bool wgrad_store_item(const CUtensorMap* tmapD, uint32_t stg, uint32_t bar_area, uint32_t& u, int m0,
+                                                 int n0, int split, int Mdim, int Ndim, volatile int* abort_flag) {
+  const uint32_t bars = bar_area + WGRAD_EPI_BAR_OFFSET;
+  for (int c = 0; c < 8; ++c) {
+    const uint32_t slot = u & 1u, use = u >> 1;
+    if (!ptx::mbar_wait_bounded(bars + 8u * slot, use & 1u, abort_flag, WAIT_BUDGET)) return false;
+    const int nb = n0 + 32 * c;
+    if (nb < Ndim && m0 < Mdim) ptx::tma_store_4d(tmapD, nb, m0, split, 0, stg + slot * 16384u);
+    ptx::bulk_commit();
+    if (u > 0) {
+      ptx::bulk_wait_read<1>();
+      ptx::mbar_arrive(bars + 8u * (2 + ((u - 1u) & 1u)));
+    }
+    ++u;
+  }
+  return true;
+}
+
 template <int STAGES>
 struct WgradCfg {
   static constexpr int A_BYTES = 16384, B_BYTES = 16384;     // 128 x 64 bf16 each, as two 64-wide boxes
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = 512;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + WGRAD_STAGING_BYTES + 1024 + 256;
 };
 
 // CONV: k tile kt is pixel box kt (64 pixels) of the NHWC tensors; the dy operand is that box, the
 // x operand the same box shifted by the filter tap its 64 columns of dW belong to.
 template <int STAGES, bool CONV>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(WGRAD_THREADS, 1)
 wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-                  const GemmParams p, int splits) {
+                  const __grid_constant__ CUtensorMap tmapD, const GemmParams p, int splits) {
   pdl_launch_dependents();
   using C = WgradCfg<STAGES>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - raw);
-  const uint32_t bar_base = base + STAGES * C::STAGE_BYTES;
+  const uint32_t staging = base + STAGES * C::STAGE_BYTES;
+  const uint32_t bar_base = staging + WGRAD_STAGING_BYTES;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   auto tmem_full_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
   auto tmem_empty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * C::STAGE_BYTES + 8 * (2 * STAGES + 4));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * C::STAGE_BYTES + WGRAD_STAGING_BYTES + 8 * (2 * STAGES + 4));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -61,9 +137,11 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_consta
       ptx::mbar_init(tmem_full_bar(b), 1);
       ptx::mbar_init(tmem_empty_bar(b), 8);
     }
+    wgrad_epi_bars_init(bar_base);
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmapA);
     ptx::prefetch_tmap(&tmapB);
+    ptx::prefetch_tmap(&tmapD);
   }
   if (warp == 1) {
     ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
@@ -155,36 +233,33 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_consta
         if (ok) ptx::tc_commit_pair(tmem_full_bar(buf), 3);
       }
     }
-  } else {
+  } else if (warp < 6) {
     const int q = warp & 3;
-    uint32_t tcount = 0;
+    uint32_t tcount = 0, u = 0;
     for (int item = cluster_id; item < num_items; item += num_clusters, ++tcount) {
-      int m0, n0, kt0, nkt, split;
-      item_coords(item, m0, n0, kt0, nkt, split);
       const uint32_t buf = tcount & 1u;
       if (!ptx::mbar_wait_bounded(tmem_full_bar(buf), (tcount >> 1) & 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
       ptx::tc_fence_after();
-      const int m = m0 + 32 * q + lane;
-      float* out = reinterpret_cast<float*>(p.out) + (size_t)split * p.Mdim * p.Ndim;
-#pragma unroll 1
-      for (int c = 0; c < 8; ++c) {
-        uint32_t r[32];
-        ptx::tmem_ld_32x32(tmem_base + 256u * buf + ((uint32_t)(32 * q) << 16) + 32 * c, r);
-        ptx::tmem_ld_wait();
-        if (c == 7) {                                      // accumulator drained: release it
-          ptx::tc_fence_before();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa(tmem_empty_bar(buf), 0));
-        }
-        const int nb = n0 + 32 * c;
-        if (m < p.Mdim && nb < p.Ndim) {                  // Ndim % 32 == 0: a chunk is all in or all out
-          float4* dst = reinterpret_cast<float4*>(out + (size_t)m * p.Ndim + nb);
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                                 __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
-        }
+      const uint32_t release_bar = ptx::mapa(tmem_empty_bar(buf), 0);
+      if (!wgrad_drain(tmem_base + 256u * buf + ((uint32_t)(32 * q) << 16), staging, bar_base, u, q, lane, abort_flag, [&] {
+            ptx::tc_fence_before();                        // accumulator drained: release it
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(release_bar);
+          })) {
+        *abort_flag = 1;
+        break;
       }
+    }
+  } else {
+    // store thread: the same walk over the work items as the draining warps
+    if (ptx::elect_one()) {
+      uint32_t u = 0;
+      for (int item = cluster_id; item < num_items; item += num_clusters) {
+        int m0, n0, kt0, nkt, split;
+        item_coords(item, m0, n0, kt0, nkt, split);
+        if (!wgrad_store_item(&tmapD, staging, bar_base, u, m0, n0, split, p.Mdim, p.Ndim, abort_flag)) { *abort_flag = 1; break; }
+      }
+      ptx::bulk_wait_read<0>();                            // shared memory must outlive the stores that read it
     }
   }
 
@@ -209,25 +284,26 @@ struct WgradSingleCfg {
   static constexpr int A_BYTES = 16384, B_BYTES = 32768;     // 128 and 256 columns x 64 tokens, 64-wide boxes
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = 512;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + WGRAD_STAGING_BYTES + 1024 + 256;
 };
 
 template <int STAGES, bool CONV>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __launch_bounds__(WGRAD_THREADS, 1)
 wgrad_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
-                    const GemmParams p, int splits) {
+                    const __grid_constant__ CUtensorMap tmapD, const GemmParams p, int splits) {
   pdl_launch_dependents();
   using C = WgradSingleCfg<STAGES>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - raw);
-  const uint32_t bar_base = base + STAGES * C::STAGE_BYTES;
+  const uint32_t staging = base + STAGES * C::STAGE_BYTES;
+  const uint32_t bar_base = staging + WGRAD_STAGING_BYTES;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   auto tmem_full_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
   auto tmem_empty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * C::STAGE_BYTES + 8 * (2 * STAGES + 4));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + STAGES * C::STAGE_BYTES + WGRAD_STAGING_BYTES + 8 * (2 * STAGES + 4));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -245,9 +321,11 @@ wgrad_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_cons
       ptx::mbar_init(tmem_full_bar(b), 1);
       ptx::mbar_init(tmem_empty_bar(b), 4);               // four epilogue warps
     }
+    wgrad_epi_bars_init(bar_base);
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmapA);
     ptx::prefetch_tmap(&tmapB);
+    ptx::prefetch_tmap(&tmapD);
   }
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_u32(tmem_slot), C::TMEM_COLS);
@@ -336,36 +414,32 @@ wgrad_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_cons
         if (ok) ptx::tc_commit(tmem_full_bar(buf));
       }
     }
-  } else {
+  } else if (warp < 6) {
     const int q = warp & 3;
-    uint32_t tcount = 0;
+    uint32_t tcount = 0, u = 0;
     for (int item = blockIdx.x; item < num_items; item += gridDim.x, ++tcount) {
-      int m0, n0, kt0, nkt, split;
-      item_coords(item, m0, n0, kt0, nkt, split);
       const uint32_t buf = tcount & 1u;
       if (!ptx::mbar_wait_bounded(tmem_full_bar(buf), (tcount >> 1) & 1u, abort_flag, WAIT_BUDGET)) { *abort_flag = 1; break; }
       ptx::tc_fence_after();
-      const int m = m0 + 32 * q + lane;
-      float* out = reinterpret_cast<float*>(p.out) + (size_t)split * p.Mdim * p.Ndim;
-#pragma unroll 1
-      for (int c = 0; c < 8; ++c) {
-        uint32_t r[32];
-        ptx::tmem_ld_32x32(tmem_base + 256u * buf + ((uint32_t)(32 * q) << 16) + 32 * c, r);
-        ptx::tmem_ld_wait();
-        if (c == 7) {                                      // accumulator drained: release it
-          ptx::tc_fence_before();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive_relaxed(tmem_empty_bar(buf));
-        }
-        const int nb = n0 + 32 * c;
-        if (m < p.Mdim && nb < p.Ndim) {                  // Ndim % 32 == 0: a chunk is all in or all out
-          float4* dst = reinterpret_cast<float4*>(out + (size_t)m * p.Ndim + nb);
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                                 __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
-        }
+      if (!wgrad_drain(tmem_base + 256u * buf + ((uint32_t)(32 * q) << 16), staging, bar_base, u, q, lane, abort_flag, [&] {
+            ptx::tc_fence_before();                        // accumulator drained: release it
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_relaxed(tmem_empty_bar(buf));
+          })) {
+        *abort_flag = 1;
+        break;
       }
+    }
+  } else {
+    // store thread: the same walk over the work items as the draining warps
+    if (ptx::elect_one()) {
+      uint32_t u = 0;
+      for (int item = blockIdx.x; item < num_items; item += gridDim.x) {
+        int m0, n0, kt0, nkt, split;
+        item_coords(item, m0, n0, kt0, nkt, split);
+        if (!wgrad_store_item(&tmapD, staging, bar_base, u, m0, n0, split, p.Mdim, p.Ndim, abort_flag)) { *abort_flag = 1; break; }
+      }
+      ptx::bulk_wait_read<0>();                            // shared memory must outlive the stores that read it
     }
   }
 
@@ -491,10 +565,11 @@ int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int 
   wgrad_plan_k(boxes, I, J, &splits, &per);
   constexpr int STAGES = 6;
   using Cf = WgradCfg<STAGES>;
-  CUtensorMap ta, tb;
+  CUtensorMap ta, tb, td;
   int rc;
   if ((rc = make_tmap_nhwc_load(&ta, dy, I, g.W, g.H, NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_nhwc_load(&tb, x, C, W, H, NB, g.wb, g.hb, g.nb, stride)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_f32_store(&td, splits > 1 ? partials : dW, (uint64_t)J, (uint64_t)I, (uint64_t)splits)) != BIMASK_OK) return rc;
   GemmParams p;
   p.conv = g;
   p.hw_meta = nullptr; p.tiles_k_meta = 0;
@@ -510,14 +585,14 @@ int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int 
     if ((rc = set_smem_attr(kern1, WgradSingleCfg<4>::SMEM_BYTES)) != BIMASK_OK) return rc;
     p.tiles_m = 1;
     const int items = p.tiles_n * splits;
-    BIMASK_CUDA_OK(launch_pdl(kern1, items < sms ? items : sms, GEMM_THREADS, WgradSingleCfg<4>::SMEM_BYTES, s, ta, tb, p, splits));
+    BIMASK_CUDA_OK(launch_pdl(kern1, items < sms ? items : sms, WGRAD_THREADS, WgradSingleCfg<4>::SMEM_BYTES, s, ta, tb, td, p, splits));
   } else {
     auto kern = wgrad_pair_kernel<STAGES, true>;
     if ((rc = set_smem_attr(kern, Cf::SMEM_BYTES)) != BIMASK_OK) return rc;
     p.tiles_m = ((I + 127) / 128 + 1) / 2;
     const int items = p.tiles_m * p.tiles_n * splits;
     const int clusters = items < sms / 2 ? items : sms / 2;
-    BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, GEMM_THREADS, Cf::SMEM_BYTES, s, ta, tb, p, splits));
+    BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, WGRAD_THREADS, Cf::SMEM_BYTES, s, ta, tb, td, p, splits));
   }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
@@ -540,10 +615,11 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
   wgrad_plan(T, I, J, &nt, &splits, &per);
   constexpr int STAGES = 6;
   using C = WgradCfg<STAGES>;
-  CUtensorMap ta, tb;
+  CUtensorMap ta, tb, td;
   int rc;
   if ((rc = make_tmap(&ta, dY, (uint64_t)I, (uint64_t)T, 64)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, X, (uint64_t)J, (uint64_t)T, 64)) != BIMASK_OK) return rc;
+  if ((rc = make_tmap_f32_store(&td, splits > 1 ? partials : dW, (uint64_t)J, (uint64_t)I, (uint64_t)splits)) != BIMASK_OK) return rc;
   GemmParams p;
   p.conv.mode = 0;
   p.hw_meta = nullptr; p.tiles_k_meta = 0;
@@ -559,14 +635,14 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
     if ((rc = set_smem_attr(kern1, WgradSingleCfg<4>::SMEM_BYTES)) != BIMASK_OK) return rc;
     p.tiles_m = 1;
     const int items = p.tiles_n * splits;
-    BIMASK_CUDA_OK(launch_pdl(kern1, items < sms ? items : sms, GEMM_THREADS, WgradSingleCfg<4>::SMEM_BYTES, s, ta, tb, p, splits));
+    BIMASK_CUDA_OK(launch_pdl(kern1, items < sms ? items : sms, WGRAD_THREADS, WgradSingleCfg<4>::SMEM_BYTES, s, ta, tb, td, p, splits));
   } else {
     auto kern = wgrad_pair_kernel<STAGES, false>;
     if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
     p.tiles_m = ((I + 127) / 128 + 1) / 2;
     const int items = p.tiles_m * p.tiles_n * splits;
     const int clusters = items < sms / 2 ? items : sms / 2;
-    BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, GEMM_THREADS, C::SMEM_BYTES, s, ta, tb, p, splits));
+    BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, WGRAD_THREADS, C::SMEM_BYTES, s, ta, tb, td, p, splits));
   }
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
