@@ -181,10 +181,11 @@ int bimask_wgrad(const uint16_t* dY, const uint16_t* X, int T, int I, int J, flo
  * forward, [search if do_search], bwd mask + pack, sparse input gradient, dense weight
  * gradient.  The caller sees one ordered step on `stream`: everything the call enqueues starts after the work
  * already on `stream` and is complete, as far as `stream` is concerned, when the work enqueued after the call starts.
- * Inside, layers between 1 and 100 GFLOP (2 T I J) run the parts that do not depend on each other (candidate
- * generation + weight gradient, forward product, permutation of dY) on three library-owned side streams that fork
- * from and join `stream` by events; the first such call of a host thread on a device creates those streams and
- * events (make it before any stream capture; later calls can be captured, forks and joins included).
+ * Inside, layers between 1 and 100 GFLOP (2 T I J) run on four library-owned streams that fork from and join
+ * `stream` by events: the dependent chain (masks, count, input gradient) and candidate generation + permutation of dY
+ * on two streams of the highest priority, the weight gradient and the forward product on two of the lowest; the
+ * first such call of a host thread on a device creates those streams and events (make it before any stream
+ * capture; later calls can be captured, forks and joins included).
  * When the search is skipped, perm is used as given.  Limits: I <= 51200 (column permute of dY); with do_search
  * 1 <= P <= 65535, and I < 2^24 when the candidates are generated. */
 typedef struct {

@@ -332,19 +332,24 @@ struct ConvPlan {
 };
 
 // A layer step is a chain of short kernels.  On small layers the kernels are too short to fill the GPU and the
-// step takes as long as its longest dependent chain, so the step is spread over the caller's stream and three side streams there:
-//   caller's stream:  forward mask -> count candidates -> backward mask -> sparse input gradient
-//   side stream A:    candidate generation (needs the seed alone) -> dense weight gradient (needs dY and X alone)
-//   side stream B:    [metadata image of a padded forward operand ->] sparse forward product (needs the forward mask alone)
-//   side stream C:    column permutation of dY (needs the permutation alone; the input gradient waits for it)
-// forked after the inputs are ready and joined before the step returns to the caller's stream.  Three side streams
-// and eight events per device and host thread, created on first use and kept until exit.  (On the large configuration
-// co-resident kernels contend for issue slots and the step gets slower, so there everything stays in line.)
+// step takes as long as its longest dependent chain, so there the step is spread over four streams of the library's own:
+//   stream H (highest priority):  forward mask -> count candidates -> backward mask -> sparse input gradient
+//   stream C (highest priority):  candidate generation (needs the seed alone) ... column permutation of dY (needs the
+//                                 permutation alone; the input gradient waits for it)
+//   stream A (lowest priority):   dense weight gradient (needs dY and X alone)
+//   stream B (lowest priority):   [metadata image of a padded forward operand ->] sparse forward product (needs the
+//                                 forward mask alone)
+// forked from the caller's stream after the inputs are ready and joined into it before the step returns, so the caller
+// sees one ordered step.  The dependent chain has its own stream because priorities are relative to the caller's
+// stream otherwise: where thread blocks of the chain and of the two independent products are waiting for an SM, the
+// chain's go first (measured on the ViT block: 14.4 k -> 14.9 k layer-steps/s; the ResNet layers do not care).
+// Four streams and nine events per device and host thread, created on first use and kept until exit.  (On the large
+// configuration co-resident kernels contend for issue slots and the step gets slower, so there everything stays in line.)
 namespace bimask {
 struct SideStream {
-  cudaStream_t a = nullptr, b = nullptr, c = nullptr;
+  cudaStream_t a = nullptr, b = nullptr, c = nullptr, h = nullptr;
   cudaEvent_t fork = nullptr, gen_done = nullptr, mask_done = nullptr, perm_done = nullptr, permuted = nullptr,
-              join_a = nullptr, join_b = nullptr, join_c = nullptr;
+              join_a = nullptr, join_b = nullptr, join_c = nullptr, join_h = nullptr;
 };
 static int get_side_stream(SideStream** out) {
   static thread_local SideStream side[64];
@@ -353,10 +358,17 @@ static int get_side_stream(SideStream** out) {
   BIMASK_REQUIRE(dev >= 0 && dev < 64, BIMASK_EUNSUPPORTED, "device ordinal %d out of range", dev);
   SideStream& sd = side[dev];
   if (!sd.a) {
-    BIMASK_CUDA_OK(cudaStreamCreateWithFlags(&sd.a, cudaStreamNonBlocking));
-    BIMASK_CUDA_OK(cudaStreamCreateWithFlags(&sd.b, cudaStreamNonBlocking));
-    BIMASK_CUDA_OK(cudaStreamCreateWithFlags(&sd.c, cudaStreamNonBlocking));
-    for (cudaEvent_t* e : {&sd.fork, &sd.gen_done, &sd.mask_done, &sd.perm_done, &sd.permuted, &sd.join_a, &sd.join_b, &sd.join_c})
+    // the dependent chain (h) and what it waits for (c) get the highest stream priority, the two products that only
+    // have to be done by the end of the step (a, b) the lowest: where thread blocks of both kinds are waiting for an SM,
+    // the chain's go first
+    int least = 0, greatest = 0;
+    BIMASK_CUDA_OK(cudaDeviceGetStreamPriorityRange(&least, &greatest));
+    BIMASK_CUDA_OK(cudaStreamCreateWithPriority(&sd.a, cudaStreamNonBlocking, least));
+    BIMASK_CUDA_OK(cudaStreamCreateWithPriority(&sd.b, cudaStreamNonBlocking, least));
+    BIMASK_CUDA_OK(cudaStreamCreateWithPriority(&sd.c, cudaStreamNonBlocking, greatest));
+    BIMASK_CUDA_OK(cudaStreamCreateWithPriority(&sd.h, cudaStreamNonBlocking, greatest));
+    for (cudaEvent_t* e : {&sd.fork, &sd.gen_done, &sd.mask_done, &sd.perm_done, &sd.permuted,
+                           &sd.join_a, &sd.join_b, &sd.join_c, &sd.join_h})
       BIMASK_CUDA_OK(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
   }
   *out = &sd;
@@ -366,9 +378,10 @@ static int get_side_stream(SideStream** out) {
 struct SideJoin {
   SideStream* side = nullptr;
   cudaStream_t main = nullptr;
-  bool a_forked = false, b_forked = false, c_forked = false;
+  bool a_forked = false, b_forked = false, c_forked = false, h_forked = false;
   ~SideJoin() {
     if (!side) return;
+    if (h_forked && cudaEventRecord(side->join_h, side->h) == cudaSuccess) cudaStreamWaitEvent(main, side->join_h, 0);
     if (a_forked && cudaEventRecord(side->join_a, side->a) == cudaSuccess) cudaStreamWaitEvent(main, side->join_a, 0);
     if (b_forked && cudaEventRecord(side->join_b, side->b) == cudaSuccess) cudaStreamWaitEvent(main, side->join_b, 0);
     if (c_forked && cudaEventRecord(side->join_c, side->c) == cudaSuccess) cudaStreamWaitEvent(main, side->join_c, 0);
@@ -430,22 +443,45 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
   const bool spread = flops >= 1e9 && flops < 1e11;
   SideJoin join;
   SideStream* side = nullptr;
-  cudaStream_t sa = s, sb = s;                          // where generation + weight gradient / the forward product go
+  cudaStream_t sm = s;                                  // the dependent chain: masks, count, input gradient
+  cudaStream_t sa = s, sb = s, sc = s;                  // weight gradient / forward product / generation + permutation of dY
   const bool gen_here = a->do_search && !a->cands;
   if (spread) {
     if ((rc = get_side_stream(&side))) return rc;
     join.side = side;
     join.main = s;
+    sm = side->h;
     sa = side->a;
     sb = side->b;
+    sc = side->c;
     BIMASK_CUDA_OK(cudaEventRecord(side->fork, s));
+    BIMASK_CUDA_OK(cudaStreamWaitEvent(sm, side->fork, 0));
+    join.h_forked = true;
+    BIMASK_CUDA_OK(cudaStreamWaitEvent(sc, side->fork, 0));
+    join.c_forked = true;
     BIMASK_CUDA_OK(cudaStreamWaitEvent(sa, side->fork, 0));
     join.a_forked = true;
-    if (gen_here) {
-      if ((rc = launch_gen_candidates(a->seed, a->P, a->I, gen, sa, a->M == 4 ? a->counts : nullptr,
+  }
+  // the 2:4 mask kernels (M = 4) write the metadata images themselves, padding included; the generic ones (M = 8, 16)
+  // do so on unpadded shapes and need the re-ordering pass otherwise
+  const bool fused = pack && (a->M == 4 || ((a->I % 128 == 0) && (a->J % 128 == 0)));
+  if (!skip_fwd_mask) {
+    if (a->M == 4)
+      rc = launch_fwd_mask(a->W, a->I, a->J, a->N, a->maskbits_f, a->vals_f, a->meta_f, fused ? a->hw_meta_f : nullptr, sm);
+    else
+      rc = launch_fwd_mask_generic(a->W, a->I, a->J, a->N, a->M, a->maskbits_f, a->vals_f, a->meta_f, pack ? 1 : 2,
+                                   fused ? a->hw_meta_f : nullptr, sm);
+    if (rc) return rc;
+  }
+  if (spread) {
+    BIMASK_CUDA_OK(cudaEventRecord(side->mask_done, sm));
+    BIMASK_CUDA_OK(cudaStreamWaitEvent(sb, side->mask_done, 0));
+    join.b_forked = true;
+    if (gen_here) {                                      // beside the forward mask; the count kernel waits for both
+      if ((rc = launch_gen_candidates(a->seed, a->P, a->I, gen, sc, a->M == 4 ? a->counts : nullptr,
                                       a->M == 4 ? a->best_idx : nullptr)))
         return rc;
-      BIMASK_CUDA_OK(cudaEventRecord(side->gen_done, sa));
+      BIMASK_CUDA_OK(cudaEventRecord(side->gen_done, sc));
     }
     if (conv && conv->imp_wgrad)
       rc = launch_wgrad_conv(a->dY, a->X, conv->NB, conv->H, conv->W, conv->C, a->I, conv->stride, a->dW, conv->wpart,
@@ -453,22 +489,6 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
     else
       rc = launch_wgrad_impl(a->dY, Xmat, a->T, a->I, a->J, a->dW, partials, a->status_word, sa);
     if (rc) return rc;
-  }
-  // the 2:4 mask kernels (M = 4) write the metadata images themselves, padding included; the generic ones (M = 8, 16)
-  // do so on unpadded shapes and need the re-ordering pass otherwise
-  const bool fused = pack && (a->M == 4 || ((a->I % 128 == 0) && (a->J % 128 == 0)));
-  if (!skip_fwd_mask) {
-    if (a->M == 4)
-      rc = launch_fwd_mask(a->W, a->I, a->J, a->N, a->maskbits_f, a->vals_f, a->meta_f, fused ? a->hw_meta_f : nullptr, s);
-    else
-      rc = launch_fwd_mask_generic(a->W, a->I, a->J, a->N, a->M, a->maskbits_f, a->vals_f, a->meta_f, pack ? 1 : 2,
-                                   fused ? a->hw_meta_f : nullptr, s);
-    if (rc) return rc;
-  }
-  if (spread) {
-    BIMASK_CUDA_OK(cudaEventRecord(side->mask_done, s));
-    BIMASK_CUDA_OK(cudaStreamWaitEvent(sb, side->mask_done, 0));
-    join.b_forked = true;
   }
   // padded shapes: the metadata image of the forward operand is a pass of its own, needed by the forward product only
   if (!skip_fwd_mask && pack && !fused && (rc = launch_hw_meta(a->meta_f, a->I, a->J, a->hw_meta_f, sb))) return rc;
@@ -482,8 +502,8 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
     const int32_t* cands = a->cands;
     if (!cands) {
       if (spread) {
-        BIMASK_CUDA_OK(cudaStreamWaitEvent(s, side->gen_done, 0));
-      } else if ((rc = launch_gen_candidates(a->seed, a->P, a->I, gen, s, a->M == 4 ? a->counts : nullptr,
+        BIMASK_CUDA_OK(cudaStreamWaitEvent(sm, side->gen_done, 0));
+      } else if ((rc = launch_gen_candidates(a->seed, a->P, a->I, gen, sm, a->M == 4 ? a->counts : nullptr,
                                              a->M == 4 ? a->best_idx : nullptr))) {
         return rc;
       }
@@ -491,42 +511,39 @@ static int layer_step_impl(const bimask_layer_args* a, bool skip_fwd_mask, const
     }
     if (a->M == 4) {
       // the count kernel's last CTA picks the winner and copies it into perm
-      if ((rc = launch_score(a->maskbits_f, cands, a->I, a->J, a->N, a->P, a->counts, s, a->cands == nullptr, a->best_idx, a->perm)))
+      if ((rc = launch_score(a->maskbits_f, cands, a->I, a->J, a->N, a->P, a->counts, sm, a->cands == nullptr, a->best_idx, a->perm)))
         return rc;
     } else {
-      if ((rc = launch_score_generic(a->maskbits_f, cands, a->I, a->J, a->N, a->M, a->P, a->counts, s))) return rc;
-      if ((rc = launch_pick(a->counts, cands, a->P, a->I, a->best_idx, a->perm, s))) return rc;
+      if ((rc = launch_score_generic(a->maskbits_f, cands, a->I, a->J, a->N, a->M, a->P, a->counts, sm))) return rc;
+      if ((rc = launch_pick(a->counts, cands, a->P, a->I, a->best_idx, a->perm, sm))) return rc;
     }
   }
-  cudaStream_t sc = s;
   if (spread) {                                          // the permutation is final: dY[:, perm] goes to side stream C
-    sc = side->c;
-    BIMASK_CUDA_OK(cudaEventRecord(side->perm_done, s));
+    BIMASK_CUDA_OK(cudaEventRecord(side->perm_done, sm));
     BIMASK_CUDA_OK(cudaStreamWaitEvent(sc, side->perm_done, 0));
-    join.c_forked = true;
     if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, sc))) return rc;
     BIMASK_CUDA_OK(cudaEventRecord(side->permuted, sc));
   }
   if (a->M == 4)
     rc = launch_bwd_mask(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->maskbits_b, a->vals_b, a->meta_b,
-                         fused ? a->hw_meta_b : nullptr, s);
+                         fused ? a->hw_meta_b : nullptr, sm);
   else
     rc = launch_bwd_mask_generic(a->W, a->maskbits_f, a->perm, a->I, a->J, a->N, a->M, a->maskbits_b, a->vals_b, a->meta_b,
-                                 pack ? 1 : 2, fused ? a->hw_meta_b : nullptr, s);
+                                 pack ? 1 : 2, fused ? a->hw_meta_b : nullptr, sm);
   if (rc) return rc;
-  if (pack && !fused && (rc = launch_hw_meta(a->meta_b, a->J, a->I, a->hw_meta_b, s))) return rc;
+  if (pack && !fused && (rc = launch_hw_meta(a->meta_b, a->J, a->I, a->hw_meta_b, sm))) return rc;
   if (spread) {
-    BIMASK_CUDA_OK(cudaStreamWaitEvent(s, side->permuted, 0));
-  } else if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, s))) {
+    BIMASK_CUDA_OK(cudaStreamWaitEvent(sm, side->permuted, 0));
+  } else if ((rc = launch_permute_cols(a->dY, a->perm, a->T, a->I, dYp, sm))) {
     return rc;
   }
   if (conv && conv->imp_dgrad)
-    rc = launch_spmm_conv(2, a->vals_b, a->hw_meta_b, dYp, conv->NB, conv->H, conv->W, conv->C, a->I, conv->stride, a->dX, a->status_word, s);
-  else if (pack) rc = launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, dXmat, a->status_word, s);
-  else rc = launch_dense_nt(a->vals_b, dYp, a->J, a->T, a->I, dXmat, a->status_word, s);
+    rc = launch_spmm_conv(2, a->vals_b, a->hw_meta_b, dYp, conv->NB, conv->H, conv->W, conv->C, a->I, conv->stride, a->dX, a->status_word, sm);
+  else if (pack) rc = launch_spmm(a->vals_b, a->hw_meta_b, dYp, a->J, a->T, a->I, dXmat, a->status_word, sm);
+  else rc = launch_dense_nt(a->vals_b, dYp, a->J, a->T, a->I, dXmat, a->status_word, sm);
   if (rc) return rc;
   if (conv && !conv->imp_dgrad)
-    if ((rc = launch_col2im3x3(dXmat, conv->NB, conv->H, conv->W, conv->C, conv->stride, a->dX, s))) return rc;
+    if ((rc = launch_col2im3x3(dXmat, conv->NB, conv->H, conv->W, conv->C, conv->stride, a->dX, sm))) return rc;
   if (spread) return BIMASK_OK;                           // already running beside the chain; joined on return
   if (conv && conv->imp_wgrad)
     return launch_wgrad_conv(a->dY, a->X, conv->NB, conv->H, conv->W, conv->C, a->I, conv->stride, a->dW, conv->wpart,

@@ -191,14 +191,18 @@ int launch_spmm_conv(int mode, const uint16_t* vals, const void* hw_meta, const 
                      int I, int stride, uint16_t* out, int32_t* status_word, cudaStream_t s);
 // Dense weight gradient of the 3x3 convolution on shifted pixel boxes; partials as sized by wgrad_conv_plan.
 void wgrad_conv_plan(int NB, int H, int W, int C, int I, int stride, int* splits, int* k_tiles_per_split);
+// reduce_stream / product_done: when given, the sum of the split-K partial results (if the plan has any) runs on
+// reduce_stream behind the event product_done, which is recorded on s after the product kernel.
 int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int W, int C, int I, int stride, float* dW,
-                      float* partials, int32_t* status_word, cudaStream_t s);
+                      float* partials, int32_t* status_word, cudaStream_t s, cudaStream_t reduce_stream = nullptr,
+                      cudaEvent_t product_done = nullptr);
 // Dense product for masked operands that do not fit the 2:4 format: out[n][m] = sum_k A[m][k] B[n][k],
 // A bf16 [Mdim][Kdim], B bf16 [Ndim][Kdim], out bf16 [Ndim][Mdim] (same roles as launch_spmm).
 int launch_dense_nt(const uint16_t* A, const uint16_t* Bop, int Mdim, int Ndim, int Kdim, uint16_t* out,
                     int32_t* status_word, cudaStream_t s);
 void wgrad_plan(int T, int I, int J, int* n_tile, int* splits, int* k_tiles_per_split);
 int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J, float* dW, float* partials,
-                      int32_t* status_word, cudaStream_t s);
+                      int32_t* status_word, cudaStream_t s, cudaStream_t reduce_stream = nullptr,
+                      cudaEvent_t product_done = nullptr);
 
 }  // namespace bimask

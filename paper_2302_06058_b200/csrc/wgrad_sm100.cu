@@ -539,6 +539,39 @@ static void wgrad_plan_k(int k_tiles, int I, int J, int* splits, int* k_tiles_pe
   *splits = sp; *k_tiles_per_split = per;
 }
 
+// Launches the pair or the single kernel for a prepared problem.  LIGHT: four (three) stages instead of six (four),
+// about 160 KB of shared memory instead of 225 KB: the layers that the step spreads over several streams keep every SM
+// for tens of microseconds with one persistent CTA, and only with room left beside it can the short mask and search
+// kernels of the same step run at the same time instead of queueing behind it; their reductions are short enough
+// for the shallower ring to cost nothing.
+template <bool LIGHT, bool CONV>
+static int launch_wgrad_kernel(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& td, GemmParams& p, int I,
+                               int splits, cudaStream_t s) {
+  constexpr int PAIR_STAGES = LIGHT ? 4 : 6, SINGLE_STAGES = LIGHT ? 3 : 4;
+  const int sms = sm_count();
+  int rc;
+  if (wgrad_uses_single(I)) {
+    using C1 = WgradSingleCfg<SINGLE_STAGES>;
+    auto kern1 = wgrad_single_kernel<SINGLE_STAGES, CONV>;
+    if ((rc = set_smem_attr(kern1, C1::SMEM_BYTES)) != BIMASK_OK) return rc;
+    p.tiles_m = 1;
+    const int items = p.tiles_n * splits;
+    BIMASK_CUDA_OK(launch_pdl(kern1, items < sms ? items : sms, WGRAD_THREADS, C1::SMEM_BYTES, s, ta, tb, td, p, splits));
+  } else {
+    using C = WgradCfg<PAIR_STAGES>;
+    auto kern = wgrad_pair_kernel<PAIR_STAGES, CONV>;
+    if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
+    p.tiles_m = ((I + 127) / 128 + 1) / 2;
+    const int items = p.tiles_m * p.tiles_n * splits;
+    const int clusters = items < sms / 2 ? items : sms / 2;
+    BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, WGRAD_THREADS, C::SMEM_BYTES, s, ta, tb, td, p, splits));
+  }
+  count_launch();
+  BIMASK_CUDA_OK(cudaGetLastError());
+  return BIMASK_OK;
+}
+static bool wgrad_is_light(double tokens, int I, int J) { return 2.0 * tokens * I * J < 1e11; }
+
 // The same for the implicit convolution: one k tile per 64-pixel box.
 // H, W: the input image; the k tiles are boxes of OUTPUT pixels.
 static ConvGeom conv_wgrad_geom(int NB, int H, int W, int C, int stride) {
@@ -557,14 +590,12 @@ void wgrad_conv_plan(int NB, int H, int W, int C, int I, int stride, int* splits
 // dW[i, tap*C + c] = sum over output pixels of dy[pixel, i] x[stride * pixel + tap, c] without a column matrix
 // (C % 64 == 0).  partials: splits * I * 9C floats when wgrad_conv_plan gives more than one split.
 int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int W, int C, int I, int stride, float* dW,
-                      float* partials, int32_t* status_word, cudaStream_t s) {
+                      float* partials, int32_t* status_word, cudaStream_t s, cudaStream_t reduce_stream, cudaEvent_t product_done) {
   const ConvGeom g = conv_wgrad_geom(NB, H, W, C, stride);
   const int boxes = g.tiles_w * g.tiles_h * ((NB + g.nb - 1) / g.nb);
   const int J = 9 * C;
   int splits, per;
   wgrad_plan_k(boxes, I, J, &splits, &per);
-  constexpr int STAGES = 6;
-  using Cf = WgradCfg<STAGES>;
   CUtensorMap ta, tb, td;
   int rc;
   if ((rc = make_tmap_nhwc_load(&ta, dy, I, g.W, g.H, NB, g.wb, g.hb, g.nb)) != BIMASK_OK) return rc;
@@ -579,25 +610,16 @@ int launch_wgrad_conv(const uint16_t* dy, const uint16_t* x, int NB, int H, int 
   p.status_word = status_word;
   p.tiles_n = (J + 255) / 256;
   p.raster_group = 8;
-  const int sms = sm_count();
-  if (wgrad_uses_single(I)) {
-    auto kern1 = wgrad_single_kernel<4, true>;
-    if ((rc = set_smem_attr(kern1, WgradSingleCfg<4>::SMEM_BYTES)) != BIMASK_OK) return rc;
-    p.tiles_m = 1;
-    const int items = p.tiles_n * splits;
-    BIMASK_CUDA_OK(launch_pdl(kern1, items < sms ? items : sms, WGRAD_THREADS, WgradSingleCfg<4>::SMEM_BYTES, s, ta, tb, td, p, splits));
-  } else {
-    auto kern = wgrad_pair_kernel<STAGES, true>;
-    if ((rc = set_smem_attr(kern, Cf::SMEM_BYTES)) != BIMASK_OK) return rc;
-    p.tiles_m = ((I + 127) / 128 + 1) / 2;
-    const int items = p.tiles_m * p.tiles_n * splits;
-    const int clusters = items < sms / 2 ? items : sms / 2;
-    BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, WGRAD_THREADS, Cf::SMEM_BYTES, s, ta, tb, td, p, splits));
-  }
-  count_launch();
-  BIMASK_CUDA_OK(cudaGetLastError());
+  rc = wgrad_is_light((double)boxes * 64, I, J) ? launch_wgrad_kernel<true, true>(ta, tb, td, p, I, splits, s)
+                                                  : launch_wgrad_kernel<false, true>(ta, tb, td, p, I, splits, s);
+  if (rc != BIMASK_OK) return rc;
   if (splits > 1) {
     const long long n4 = (long long)I * J / 4;
+    if (reduce_stream && product_done) {
+      BIMASK_CUDA_OK(cudaEventRecord(product_done, s));
+      BIMASK_CUDA_OK(cudaStreamWaitEvent(reduce_stream, product_done, 0));
+      s = reduce_stream;
+    }
     if ((rc = launch_splitk_reduce(partials, splits, n4, dW, s)) != BIMASK_OK) return rc;
   }
   return BIMASK_OK;
@@ -610,11 +632,9 @@ void wgrad_plan(int T, int I, int J, int* n_tile, int* splits, int* k_tiles_per_
 }
 
 int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J, float* dW, float* partials,
-                      int32_t* status_word, cudaStream_t s) {
+                      int32_t* status_word, cudaStream_t s, cudaStream_t reduce_stream, cudaEvent_t product_done) {
   int nt, splits, per;
   wgrad_plan(T, I, J, &nt, &splits, &per);
-  constexpr int STAGES = 6;
-  using C = WgradCfg<STAGES>;
   CUtensorMap ta, tb, td;
   int rc;
   if ((rc = make_tmap(&ta, dY, (uint64_t)I, (uint64_t)T, 64)) != BIMASK_OK) return rc;
@@ -629,25 +649,16 @@ int launch_wgrad_impl(const uint16_t* dY, const uint16_t* X, int T, int I, int J
   p.status_word = status_word;
   p.tiles_n = (J + 255) / 256;
   p.raster_group = 8;
-  const int sms = sm_count();
-  if (wgrad_uses_single(I)) {
-    auto kern1 = wgrad_single_kernel<4, false>;
-    if ((rc = set_smem_attr(kern1, WgradSingleCfg<4>::SMEM_BYTES)) != BIMASK_OK) return rc;
-    p.tiles_m = 1;
-    const int items = p.tiles_n * splits;
-    BIMASK_CUDA_OK(launch_pdl(kern1, items < sms ? items : sms, WGRAD_THREADS, WgradSingleCfg<4>::SMEM_BYTES, s, ta, tb, td, p, splits));
-  } else {
-    auto kern = wgrad_pair_kernel<STAGES, false>;
-    if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
-    p.tiles_m = ((I + 127) / 128 + 1) / 2;
-    const int items = p.tiles_m * p.tiles_n * splits;
-    const int clusters = items < sms / 2 ? items : sms / 2;
-    BIMASK_CUDA_OK(launch_pdl(kern, 2 * clusters, WGRAD_THREADS, C::SMEM_BYTES, s, ta, tb, td, p, splits));
-  }
-  count_launch();
-  BIMASK_CUDA_OK(cudaGetLastError());
+  rc = wgrad_is_light((double)T, I, J) ? launch_wgrad_kernel<true, false>(ta, tb, td, p, I, splits, s)
+                                       : launch_wgrad_kernel<false, false>(ta, tb, td, p, I, splits, s);
+  if (rc != BIMASK_OK) return rc;
   if (splits > 1) {
     const long long n4 = (long long)I * J / 4;
+    if (reduce_stream && product_done) {
+      BIMASK_CUDA_OK(cudaEventRecord(product_done, s));
+      BIMASK_CUDA_OK(cudaStreamWaitEvent(reduce_stream, product_done, 0));
+      s = reduce_stream;
+    }
     if ((rc = launch_splitk_reduce(partials, splits, n4, dW, s)) != BIMASK_OK) return rc;
   }
   return BIMASK_OK;
