@@ -349,6 +349,34 @@ def test_small_layer_with_split_k_weight_gradient():
     assert rel_err(b["dX"].float().cpu().numpy(), ref["dX"]) <= TOL
 
 
+@pytest.mark.parametrize("I,J,T", [(96, 160, 129), (32, 32, 70), (64, 96, 9000), (160, 288, 1000), (1152, 384, 1500),
+                                   (2080, 4128, 530)])
+def test_products_write_nothing_outside_their_results(I, J, T):
+    """Y, dX and dW leave the kernels as tensor stores of whole boxes that the tensor maps clip at the edge of the
+    result: the three results are placed inside larger buffers filled with a sentinel, on ragged shapes in every
+    dimension (partial row tiles, partial token chunks, split-K partial sums), and the sentinel must survive around
+    them while the results themselves still match."""
+    W = inputs.make_weight(I, J, 3 * I + J)
+    X = inputs.make_activation(T, J, I + T)
+    dY = inputs.make_activation(T, I, J + T)
+    P, seed, pad = 3, 99, 4096
+    b = bm.alloc_layer_buffers(T, I, J, P)
+    b["W"], b["X"], b["dY"] = dev(W), bits_dev(X), bits_dev(dY)
+    guards = {}
+    for name, dt, sentinel in (("Y", torch.bfloat16, 7.0), ("dX", torch.bfloat16, 7.0), ("dW", torch.float32, 7.0)):
+        n = b[name].numel()
+        big = torch.full((n + 2 * pad,), sentinel, dtype=dt, device="cuda")
+        guards[name] = big
+        b[name] = big[pad:pad + n].view(b[name].shape)
+    bm.bimask_layer_step(bm.make_layer_args(T, I, J, 2, 4, P, seed, True, b))
+    torch.cuda.synchronize()
+    ref = O.layer_step(W, X, dY, 2, 4, P, seed, do_search=True)
+    assert int(b["status_word"].item()) == 0
+    for name, big in guards.items():
+        assert bool((big[:pad] == 7.0).all()) and bool((big[-pad:] == 7.0).all()), name
+        assert rel_err(b[name].float().cpu().numpy(), ref[name]) <= TOL, name
+
+
 # ---------------------------------------------------------------------------------------------
 # The other N:M patterns the paper trains (4:8, 2:8, 1:8, 1:16): masks, search, backward mask bit
 # for bit; those that fit the 2:4 container (N <= 2) also run the whole layer step.
