@@ -240,12 +240,12 @@ class ClockSampler:
 NCU_TRAFFIC_SOURCE = "profiles/cfg5_launch_list.md"
 NCU_TRAFFIC_BYTES = {
     (5, 0, "fwd_mask"): 268e6 + 64e6, (5, 1, "fwd_mask"): 269e6 + 69e6,
-    (5, 0, "spmm_fwd"): 356e6 + 235e6, (5, 1, "spmm_fwd"): 592e6 + 51e6,
+    (5, 0, "spmm_fwd"): 360e6 + 235e6, (5, 1, "spmm_fwd"): 592e6 + 51e6,
     (5, 0, "perm_search"): 17e6, (5, 1, "perm_search"): 11e6,              # generator + count kernel
     (5, 0, "bwd_mask"): 277e6 + 62e6, (5, 1, "bwd_mask"): 277e6 + 61e6,
     (5, 0, "spmm_dgrad"): 269e6 + 216e6 + 592e6 + 51e6,                    # permute pass + product
-    (5, 1, "spmm_dgrad"): 67e6 + 18e6 + 360e6 + 236e6,
-    (5, 0, "wgrad"): 1237e6 + 246e6, (5, 1, "wgrad"): 1002e6 + 246e6,
+    (5, 1, "spmm_dgrad"): 67e6 + 19e6 + 365e6 + 236e6,
+    (5, 0, "wgrad"): 1402e6 + 249e6, (5, 1, "wgrad"): 1117e6 + 249e6,
 }
 
 
