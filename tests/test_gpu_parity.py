@@ -240,6 +240,57 @@ def test_do_search_zero_uses_given_perm():
     assert rel_err(b["dX"].float().cpu().numpy(), ref["dX"]) <= TOL
 
 
+def test_search_with_the_largest_candidate_count():
+    """P = 65535, the documented maximum (one grid row per candidate): counts, winner and permutation against the
+    oracle on a matrix small enough for the oracle to score every candidate; one more candidate is refused."""
+    I, J, P, seed = 32, 64, 65535, 5
+    W = inputs.make_weight(I, J, 17)
+    B = O.forward_mask(W, 2, 4)
+    bits = dev(O.pack_bits(B).view(np.int32))
+    ws_bytes = bm.bimask_workspace_bytes(1, I, J, P)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    best_perm = torch.empty(I, dtype=torch.int32, device="cuda")
+    best_idx = torch.empty(1, dtype=torch.int32, device="cuda")
+    counts = torch.empty(P + 1, dtype=torch.int64, device="cuda")
+    bm.bimask_perm_search(bits, I, J, 2, 4, P, seed, None, best_perm, best_idx, counts, ws, ws_bytes)
+    torch.cuda.synchronize()
+    cands = O.candidates(seed, P, I)
+    best, perm, cnt = O.perm_search(B, cands, 2, 4)
+    assert np.array_equal(counts[:P].cpu().numpy(), cnt)
+    assert int(best_idx.item()) == best
+    assert np.array_equal(best_perm.cpu().numpy(), perm)
+    with pytest.raises(bm.BimaskError) as e:
+        bm.bimask_perm_search(bits, I, J, 2, 4, P + 1, seed, None, best_perm, best_idx, counts, ws, ws_bytes)
+    assert e.value.code == bm.binding.BIMASK_EINVAL
+
+
+def test_layer_step_at_the_largest_row_count():
+    """I = 51200, the documented limit of the layer step (the permutation pass keeps a row of dY in shared memory):
+    masks, counts and the permutation bit for bit, the three products within tolerance; four rows more are refused."""
+    I, J, T, P, seed = 51200, 64, 96, 2, 11
+    W = inputs.make_weight(I, J, 23)
+    X = inputs.make_activation(T, J, 24)
+    dY = inputs.make_activation(T, I, 25)
+    b = run_layer_step(W, X, dY, 2, 4, P, seed, do_search=True)
+    ref = O.layer_step(W, X, dY, 2, 4, P, seed, do_search=True)
+    assert int(b["status_word"].item()) == 0
+    assert np.array_equal(u32(b["maskbits_f"]), ref["maskbits_f"])
+    assert np.array_equal(b["counts"].cpu().numpy(), ref["counts"])
+    assert np.array_equal(b["perm"].cpu().numpy(), ref["perm"])
+    assert np.array_equal(u32(b["maskbits_b"]), ref["maskbits_b"])
+    assert np.array_equal(u16(b["vals_b"]), ref["vals_b"])
+    for n in ("Y", "dX", "dW"):
+        assert rel_err(b[n].float().cpu().numpy(), ref[n]) <= TOL, n
+    I2 = I + 4
+    b2 = bm.alloc_layer_buffers(T, I2, J, P)
+    b2["W"] = torch.zeros(I2, J, device="cuda")
+    b2["X"] = torch.zeros(T, J, dtype=torch.bfloat16, device="cuda")
+    b2["dY"] = torch.zeros(T, I2, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(bm.BimaskError) as e:
+        bm.bimask_layer_step(bm.make_layer_args(T, I2, J, 2, 4, P, seed, True, b2))
+    assert e.value.code in (bm.binding.BIMASK_EUNSUPPORTED, bm.binding.BIMASK_EINVAL)
+
+
 def test_error_paths_launch_nothing():
     W = torch.zeros(64, 64, device="cuda")
     b = bm.alloc_layer_buffers(8, 64, 64, 2)
