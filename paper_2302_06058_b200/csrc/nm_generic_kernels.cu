@@ -16,7 +16,7 @@ namespace {
 // (q beats m when key_q > key_m, or key_q == key_m with q < m).
 //   N <= 2: N rounds of "largest remaining candidate, lowest index on ties" -- about 5 M operations
 //           per round instead of all M (M - 1) / 2 pairwise comparisons;
-//   N  > 2: pairwise ranks.
+//   N  > 2: threshold = the N-th largest key, found by a sorting network (below).
 template <int M>
 __device__ __forceinline__ uint32_t keep_block(const uint32_t (&key)[M], uint32_t valid, int N) {
   uint32_t kb = 0;
@@ -43,19 +43,54 @@ __device__ __forceinline__ uint32_t keep_block(const uint32_t (&key)[M], uint32_
     }
     return kb;
   }
-  int rank[M];
+  // N > 2: the N-th largest candidate key t from a sorting network on the keys alone (bitonic, min / max pairs with
+  // compile-time indices: 24 pairs for M = 8, 80 for M = 16, against M (M - 1) / 2 pairwise comparisons with two
+  // conditional increments each); kept are the candidates above t and, of those equal to t, the lowest indices up
+  // to N in all -- which is the rank rule: q beats m when key_q > key_m, or key_q == key_m with q < m.
+  uint32_t k[M], srt[M];                                  // 0 = not a candidate (keys are < 2^31, so +1 fits)
 #pragma unroll
-  for (int m = 0; m < M; ++m) rank[m] = 0;
+  for (int m = 0; m < M; ++m) k[m] = srt[m] = ((valid >> m) & 1u) ? key[m] + 1u : 0u;
 #pragma unroll
-  for (int m = 1; m < M; ++m)
+  for (int span = 2; span <= M; span <<= 1)
 #pragma unroll
-    for (int q = 0; q < m; ++q) {
-      const bool q_beats_m = key[q] >= key[m];             // equal keys: the lower index wins
-      rank[m] += (q_beats_m && ((valid >> q) & 1u)) ? 1 : 0;
-      rank[q] += (!q_beats_m && ((valid >> m) & 1u)) ? 1 : 0;
+    for (int j = span >> 1; j > 0; j >>= 1)
+#pragma unroll
+      for (int i = 0; i < M; ++i) {
+        const int l = i ^ j;
+        if (l > i) {
+          const uint32_t lo = min(srt[i], srt[l]), hi = max(srt[i], srt[l]);
+          const bool descending = (i & span) == 0;        // the whole array ends up in descending order
+          srt[i] = descending ? hi : lo;
+          srt[l] = descending ? lo : hi;
+        }
+      }
+  uint32_t t = srt[0];
+#pragma unroll
+  for (int m = 1; m < M; ++m) t = (m == N - 1) ? srt[m] : t;
+  uint32_t ge = 0;
+#pragma unroll
+  for (int m = 0; m < M; ++m) ge |= (k[m] >= t ? 1u : 0u) << m;
+  // the usual cases: no tie at the threshold (exactly N at or above it), or fewer than N candidates (t == 0: all of
+  // them are kept).  Taken only when every lane of the warp is in one of them (every caller runs whole warps).
+  if (__all_sync(0xFFFFFFFFu, t == 0u || __popc(ge) == N)) return t == 0u ? valid : ge;
+  uint32_t gt = 0, eq = 0;
+#pragma unroll
+  for (int m = 0; m < M; ++m) {
+    gt |= (k[m] > t ? 1u : 0u) << m;
+    eq |= (k[m] == t ? 1u : 0u) << m;
+  }
+  eq &= valid;                                            // t == 0: fewer than N candidates, all of them are above it
+  kb = gt;
+  int need = N - __popc(gt);
+#pragma unroll
+  for (int i = 0; i < M; ++i) {
+    if (i < N && need > 0) {
+      const uint32_t b = eq & (0u - eq);
+      kb |= b;
+      eq ^= b;
+      --need;
     }
-#pragma unroll
-  for (int m = 0; m < M; ++m) kb |= (((valid >> m) & 1u) && rank[m] < N) ? (1u << m) : 0u;
+  }
   return kb;
 }
 
@@ -123,15 +158,24 @@ fwd_mask_generic_kernel(const float4* __restrict__ W4, long long nblocks, int N,
     }
     if (MODE == 2 && live) {
       uint4* dst = reinterpret_cast<uint4*>(vals32) + b * (M / 8);
+      uint32_t mx = key[0];
+#pragma unroll
+      for (int m = 1; m < M; ++m) mx = max(mx, key[m]);
+      const bool has_nan = mx > 0x7F800000u;              // the packed conversion would canonicalise a NaN's payload
 #pragma unroll
       for (int h = 0; h < M / 8; ++h) {
         uint32_t d[4];
+        if (has_nan) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) d[j] = to_bf16(w[8 * h + 2 * j]) | (to_bf16(w[8 * h + 2 * j + 1]) << 16);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) d[j] = cvt_bf16x2(w[8 * h + 2 * j + 1], w[8 * h + 2 * j]);
+        }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const int m = 8 * h + 2 * j;
-          const uint32_t lo = ((kb >> m) & 1u) ? to_bf16(w[m]) : 0u;
-          const uint32_t hi = ((kb >> (m + 1)) & 1u) ? to_bf16(w[m + 1]) : 0u;
-          d[j] = lo | (hi << 16);
+          const uint32_t f = (kb >> (8 * h + 2 * j)) & 3u;  // kept bits of the pair -> 16-bit masks
+          d[j] &= (f & 1u) * 0xFFFFu + (f >> 1) * 0xFFFF0000u;
         }
         dst[h] = make_uint4(d[0], d[1], d[2], d[3]);
       }
