@@ -606,6 +606,56 @@ def test_async_host_calls_with_alternating_buffer_sets():
         assert torch.equal(host["dW"], ref["dW"].cpu()), c
 
 
+def test_two_host_threads_on_their_own_streams():
+    """Two host threads call the layer step at the same time, each on its own stream and buffers (the library's side
+    streams, events and tensor-map cache are per host thread, its shared-memory attribute table per device and
+    atomic): twelve steps each on alternating inputs, sizes on both sides of the side-stream threshold; every result
+    equals that of the same step run alone."""
+    import threading
+    jobs = [(256, 384, 6000, 2), (1152, 384, 1500, 2), (64, 576, 300, 1), (512, 1184, 1568, 2)]
+    refs, work = [], []
+    for t, (I, J, T, N) in enumerate(jobs):
+        ins = [(inputs.make_weight(I, J, 31 * t + v), inputs.make_activation(T, J, 37 * t + v),
+                inputs.make_activation(T, I, 41 * t + v)) for v in range(2)]
+        refs.append([run_layer_step(W, X, dY, N, 4, 4, 9 + t, do_search=True) for (W, X, dY) in ins])
+        work.append(ins)
+    torch.cuda.synchronize()
+    results, errors = {}, []
+
+    def worker(tid):
+        try:
+            st = torch.cuda.Stream()
+            for t in (tid, tid + 2):                       # two jobs per thread, one after the other
+                I, J, T, N = jobs[t]
+                b = bm.alloc_layer_buffers(T, I, J, 4)
+                dev_in = [(dev(W), bits_dev(X), bits_dev(dY)) for (W, X, dY) in work[t]]
+                torch.cuda.synchronize()
+                got = []
+                for step in range(12):
+                    b["W"], b["X"], b["dY"] = dev_in[step & 1]
+                    bm.bimask_layer_step(bm.make_layer_args(T, I, J, N, 4, 4, 9 + t, True, b, stream=st))
+                    if step >= 10:                         # keep the last two (one per input set)
+                        st.synchronize()
+                        got.append({k: b[k].clone() for k in ("perm", "counts", "Y", "dX", "dW", "maskbits_b", "status_word")})
+                st.synchronize()
+                results[t] = got
+        except Exception as e:                             # surfaced by the main thread
+            errors.append(e)
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    assert not errors, errors
+    for t in range(4):
+        for v, got in enumerate(results[t]):
+            ref = refs[t][v]
+            assert int(got["status_word"].item()) == 0
+            for k in ("perm", "counts", "maskbits_b", "Y", "dX", "dW"):
+                assert torch.equal(got[k], ref[k]), (t, v, k)
+
+
 @pytest.mark.parametrize("I,J,T", [(256, 384, 512), (64, 576, 3000), (256, 384, 6000), (64, 576, 16000), (1152, 384, 1500)])
 def test_back_to_back_steps_on_reused_buffers(I, J, T):
     """Every kernel is launched as a programmatic dependent of the one before it and may begin before that one
