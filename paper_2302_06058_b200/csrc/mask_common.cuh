@@ -114,6 +114,29 @@ __device__ __forceinline__ uint32_t slots_signs(uint32_t e, float w0, float w1, 
   return __byte_perm(cvt_bf16x2(w1, w0), cvt_bf16x2(w3, w2), e) & keep;
 }
 
+// Transpose of a 32 x 32 bit matrix held one row per lane (bit b of lane r = element (r, b)): five exchange
+// stages, each swapping the off-diagonal quadrants of every 2s x 2s block; afterwards lane c holds column c.
+__device__ __forceinline__ uint32_t transpose32(uint32_t x, int lane) {
+  {
+    const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, 16);
+    x = __byte_perm(x, y, (lane & 16) ? 0x3276u : 0x5410u);
+  }
+  {
+    const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, 8);
+    x = __byte_perm(x, y, (lane & 8) ? 0x3715u : 0x6240u);
+  }
+#pragma unroll
+  for (int s = 4; s >= 1; s >>= 1) {
+    const uint32_t m = s == 4 ? 0x0F0F0F0Fu : s == 2 ? 0x33333333u : 0x55555555u;
+    const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, s);
+    const bool low = (lane & s) == 0;                      // this lane keeps its low half of every 2s group
+    const uint32_t keep = low ? m : ~m;
+    const uint32_t moved = low ? (y << s) : (y >> s);
+    x = (x & keep) | (moved & ~keep);
+  }
+  return x;
+}
+
 // One canonical code word (row r of the packed operand, 32-column word w) scattered into the
 // tensor-memory image of the metadata (one 2048-byte block per 128 rows x 128 k: 128 lanes x 4
 // columns of u32, lane = m0 + 8*h + 16*m2 holding rows m0 + 16*m2 / + 8 of k-half h): its low 16 bits (k-half 0) and high 16 bits

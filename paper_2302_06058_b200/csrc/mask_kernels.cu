@@ -188,29 +188,6 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// Transpose of a 32 x 32 bit matrix held one row per lane (bit b of lane r = element (r, b)): five exchange
-// stages, each swapping the off-diagonal quadrants of every 2s x 2s block; afterwards lane c holds column c.
-__device__ __forceinline__ uint32_t transpose32(uint32_t x, int lane) {
-  {
-    const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, 16);
-    x = __byte_perm(x, y, (lane & 16) ? 0x3276u : 0x5410u);
-  }
-  {
-    const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, 8);
-    x = __byte_perm(x, y, (lane & 8) ? 0x3715u : 0x6240u);
-  }
-#pragma unroll
-  for (int s = 4; s >= 1; s >>= 1) {
-    const uint32_t m = s == 4 ? 0x0F0F0F0Fu : s == 2 ? 0x33333333u : 0x55555555u;
-    const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, s);
-    const bool low = (lane & s) == 0;                      // this lane keeps its low half of every 2s group
-    const uint32_t keep = low ? m : ~m;
-    const uint32_t moved = low ? (y << s) : (y >> s);
-    x = (x & keep) | (moved & ~keep);
-  }
-  return x;
-}
-
 template <int CW>
 __global__ void __launch_bounds__(BM_THREADS, BM_CTAS_PER_SM)
 bwd_mask_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,

@@ -436,7 +436,10 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
   const int col = 32 * cw + lane;
   const unsigned last_row = (unsigned)(I - 1);
   const int my_src = checked_row(__ldg(perm + 32 * pass + lane), (int)last_row + 1, SITE_GENERIC_PERM);   // lane r: source of permuted row r
-  uint32_t my_word = 0;                                     // lane r ends up with the mask word of permuted row r
+  // lane r loads the forward-mask word of permuted row r; one 32 x 32 bit transpose gives every lane (= column) the
+  // candidate bits of its column in the 32 rows, and the kept bits go back to row words the same way
+  const uint32_t cand = transpose32(__ldg(maskbits_f + (size_t)my_src * jwords + cw), lane);
+  uint32_t colkeep = 0;
   uint32_t vacc[8];
   uint32_t dacc[MODE == 2 ? 16 : 1];                        // dense: this column's 32 permuted rows as bf16 pairs
   uint32_t cacc = 0;
@@ -445,13 +448,11 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
     float w[M];
     uint32_t key[M];                                        // magnitude of the weight (values, NaN handling)
     uint32_t skey[(CRIT == 1 || CRIT == 3) ? M : 1];        // what the criterion ranks by
-    uint32_t valid = 0;
+    const uint32_t valid = (cand >> (nb * M)) & ((1u << M) - 1u);
 #pragma unroll
     for (int m = 0; m < M; ++m) {
       const int src = __shfl_sync(0xFFFFFFFFu, my_src, nb * M + m);
       w[m] = __ldg(W + (size_t)src * J + col);
-      const uint32_t f = __ldg(maskbits_f + (size_t)src * jwords + cw);
-      valid |= ((f >> lane) & 1u) << m;
       key[m] = mag_key(w[m]);
       if constexpr (CRIT == 1) skey[m] = mag_key(__ldg(S + (size_t)src * J + col));
       if constexpr (CRIT == 3) skey[m] = (uint32_t)(mix64_dev(seed + (uint64_t)src * (uint64_t)J + (uint64_t)col) >> 33);
@@ -460,11 +461,7 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
     if constexpr (CRIT == 0) kb = keep_block<M>(key, valid, N);
     else if constexpr (CRIT == 2) kb = multinomial_block<M>(w, valid, N, seed, (uint64_t)(pass * NB + nb) * (uint64_t)J + (uint64_t)col);
     else kb = keep_block<M>(skey, valid, N);
-#pragma unroll
-    for (int m = 0; m < M; ++m) {
-      const uint32_t word = __ballot_sync(0xFFFFFFFFu, (kb >> m) & 1u);
-      if (lane == nb * M + m) my_word = word;
-    }
+    colkeep |= kb << (nb * M);
     if (MODE == 2) {
 #pragma unroll
       for (int m = 0; m < M; m += 2) {
@@ -483,7 +480,7 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
       }
     }
   }
-  maskbits_b[(size_t)(32 * pass + lane) * jwords + cw] = my_word;
+  maskbits_b[(size_t)(32 * pass + lane) * jwords + cw] = transpose32(colkeep, lane);
   if (MODE == 1) {
     uint4* dst = reinterpret_cast<uint4*>(vals_b + (size_t)col * (I >> 2) + 8 * pass);
     dst[0] = make_uint4(vacc[0], vacc[1], vacc[2], vacc[3]);
