@@ -414,6 +414,11 @@ __device__ __forceinline__ uint32_t multinomial_block(const float (&w)[M], uint3
   return keep;
 }
 
+// Passes (groups of 32 permuted rows) a warp handles per trip: as many as make a column's share of the operand a
+// whole 128-byte line (32 B per pass in the 2:4 container, 64 B per pass in the dense operand).
+template <int MODE>
+struct BwdGenericTrip { static constexpr int PASSES = MODE == 2 ? 2 : 4; };
+
 template <int M, int MODE, int CRIT>
 __global__ void __launch_bounds__(256)
 bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,
@@ -425,73 +430,107 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
   pdl_wait();
   constexpr int NB = 32 / M;                                // blocks per 32-row pass
   constexpr int G = M / 4;
+  constexpr int PP = BwdGenericTrip<MODE>::PASSES;
   __shared__ uint32_t pad16[16];
+  // operand rows are columns of W: a lane's results of one pass are 32 or 64 bytes of ITS row, so stored from
+  // registers every instruction of a warp would touch 32 lines.  They are staged per warp as [32 columns][eight
+  // 16-byte units] (unit index XOR column mod 8: conflict-free 16-byte stores and loads) over PP passes and written
+  // out as whole 128-byte lines, four columns per instruction.
+  __shared__ uint4 stage_all[MODE == 0 ? 1 : 8 * 256];
+  __shared__ uint32_t code_all[MODE == 1 ? 8 * 32 * 4 : 1];
   if (threadIdx.x < 16) pad16[threadIdx.x] = lut_entry(0u, threadIdx.x, 4);
   __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int jwords = J >> 5;
   const int cw = blockIdx.y * 8 + warp;                     // column word of this warp
-  const int pass = blockIdx.x;                              // 32 permuted rows
   if (cw >= jwords) return;
   const int col = 32 * cw + lane;
-  const unsigned last_row = (unsigned)(I - 1);
-  const int my_src = checked_row(__ldg(perm + 32 * pass + lane), (int)last_row + 1, SITE_GENERIC_PERM);   // lane r: source of permuted row r
-  // lane r loads the forward-mask word of permuted row r; one 32 x 32 bit transpose gives every lane (= column) the
-  // candidate bits of its column in the 32 rows, and the kept bits go back to row words the same way
-  const uint32_t cand = transpose32(__ldg(maskbits_f + (size_t)my_src * jwords + cw), lane);
-  uint32_t colkeep = 0;
-  uint32_t vacc[8];
-  uint32_t dacc[MODE == 2 ? 16 : 1];                        // dense: this column's 32 permuted rows as bf16 pairs
-  uint32_t cacc = 0;
+  const int npass = I >> 5, pass0 = blockIdx.x * PP;
+  const int done = npass - pass0 < PP ? npass - pass0 : PP; // passes of this trip
+  uint4* stage = stage_all + (MODE == 0 ? 0 : warp * 256);
+  uint32_t* codes = code_all + (MODE == 1 ? warp * 128 : 0);
+#pragma unroll 1
+  for (int pp = 0; pp < done; ++pp) {
+    const int pass = pass0 + pp;                            // 32 permuted rows
+    const int my_src = checked_row(__ldg(perm + 32 * pass + lane), I, SITE_GENERIC_PERM);   // lane r: source of permuted row r
+    // lane r loads the forward-mask word of permuted row r; one 32 x 32 bit transpose gives every lane (= column) the
+    // candidate bits of its column in the 32 rows, and the kept bits go back to row words the same way
+    const uint32_t cand = transpose32(__ldg(maskbits_f + (size_t)my_src * jwords + cw), lane);
+    uint32_t colkeep = 0;
+    uint32_t vacc[8];
+    uint32_t dacc[MODE == 2 ? 16 : 1];                      // dense: this column's 32 permuted rows as bf16 pairs
+    uint32_t cacc = 0;
 #pragma unroll
-  for (int nb = 0; nb < NB; ++nb) {
-    float w[M];
-    uint32_t key[M];                                        // magnitude of the weight (values, NaN handling)
-    uint32_t skey[(CRIT == 1 || CRIT == 3) ? M : 1];        // what the criterion ranks by
-    const uint32_t valid = (cand >> (nb * M)) & ((1u << M) - 1u);
+    for (int nb = 0; nb < NB; ++nb) {
+      float w[M];
+      uint32_t key[M];                                      // magnitude of the weight (values, NaN handling)
+      uint32_t skey[(CRIT == 1 || CRIT == 3) ? M : 1];      // what the criterion ranks by
+      const uint32_t valid = (cand >> (nb * M)) & ((1u << M) - 1u);
 #pragma unroll
-    for (int m = 0; m < M; ++m) {
-      const int src = __shfl_sync(0xFFFFFFFFu, my_src, nb * M + m);
-      w[m] = __ldg(W + (size_t)src * J + col);
-      key[m] = mag_key(w[m]);
-      if constexpr (CRIT == 1) skey[m] = mag_key(__ldg(S + (size_t)src * J + col));
-      if constexpr (CRIT == 3) skey[m] = (uint32_t)(mix64_dev(seed + (uint64_t)src * (uint64_t)J + (uint64_t)col) >> 33);
+      for (int m = 0; m < M; ++m) {
+        const int src = __shfl_sync(0xFFFFFFFFu, my_src, nb * M + m);
+        w[m] = __ldg(W + (size_t)src * J + col);
+        key[m] = mag_key(w[m]);
+        if constexpr (CRIT == 1) skey[m] = mag_key(__ldg(S + (size_t)src * J + col));
+        if constexpr (CRIT == 3) skey[m] = (uint32_t)(mix64_dev(seed + (uint64_t)src * (uint64_t)J + (uint64_t)col) >> 33);
+      }
+      uint32_t kb;
+      if constexpr (CRIT == 0) kb = keep_block<M>(key, valid, N);
+      else if constexpr (CRIT == 2) kb = multinomial_block<M>(w, valid, N, seed, (uint64_t)(pass * NB + nb) * (uint64_t)J + (uint64_t)col);
+      else kb = keep_block<M>(skey, valid, N);
+      colkeep |= kb << (nb * M);
+      if (MODE == 2) {
+#pragma unroll
+        for (int m = 0; m < M; m += 2) {
+          const uint32_t lo = ((kb >> m) & 1u) ? to_bf16(w[m]) : 0u;
+          const uint32_t hi = ((kb >> (m + 1)) & 1u) ? to_bf16(w[m + 1]) : 0u;
+          dacc[(nb * M + m) / 2] = lo | (hi << 16);
+        }
+      }
+      if (MODE == 1) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          const uint32_t e = pad16[(kb >> (4 * g)) & 15u];
+          vacc[nb * G + g] = slots<false>(e, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3], key[4 * g],
+                                          key[4 * g + 1], key[4 * g + 2], key[4 * g + 3]);
+          cacc |= ((e >> 4) & 15u) << (4 * (nb * G + g));
+        }
+      }
     }
-    uint32_t kb;
-    if constexpr (CRIT == 0) kb = keep_block<M>(key, valid, N);
-    else if constexpr (CRIT == 2) kb = multinomial_block<M>(w, valid, N, seed, (uint64_t)(pass * NB + nb) * (uint64_t)J + (uint64_t)col);
-    else kb = keep_block<M>(skey, valid, N);
-    colkeep |= kb << (nb * M);
+    maskbits_b[(size_t)(32 * pass + lane) * jwords + cw] = transpose32(colkeep, lane);
+    if (MODE == 1) {
+      stage[lane * 8 + ((2 * pp) ^ (lane & 7))] = make_uint4(vacc[0], vacc[1], vacc[2], vacc[3]);
+      stage[lane * 8 + ((2 * pp + 1) ^ (lane & 7))] = make_uint4(vacc[4], vacc[5], vacc[6], vacc[7]);
+      codes[lane * 4 + pp] = cacc;
+      if (hw16) scatter_hw(hw16, I >> 7, col, pass, cacc);
+    }
     if (MODE == 2) {
 #pragma unroll
-      for (int m = 0; m < M; m += 2) {
-        const uint32_t lo = ((kb >> m) & 1u) ? to_bf16(w[m]) : 0u;
-        const uint32_t hi = ((kb >> (m + 1)) & 1u) ? to_bf16(w[m + 1]) : 0u;
-        dacc[(nb * M + m) / 2] = lo | (hi << 16);
-      }
-    }
-    if (MODE == 1) {
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        const uint32_t e = pad16[(kb >> (4 * g)) & 15u];
-        vacc[nb * G + g] = slots<false>(e, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3], key[4 * g],
-                                        key[4 * g + 1], key[4 * g + 2], key[4 * g + 3]);
-        cacc |= ((e >> 4) & 15u) << (4 * (nb * G + g));
-      }
+      for (int q = 0; q < 4; ++q)
+        stage[lane * 8 + ((4 * pp + q) ^ (lane & 7))] = make_uint4(dacc[4 * q], dacc[4 * q + 1], dacc[4 * q + 2], dacc[4 * q + 3]);
     }
   }
-  maskbits_b[(size_t)(32 * pass + lane) * jwords + cw] = transpose32(colkeep, lane);
-  if (MODE == 1) {
-    uint4* dst = reinterpret_cast<uint4*>(vals_b + (size_t)col * (I >> 2) + 8 * pass);
-    dst[0] = make_uint4(vacc[0], vacc[1], vacc[2], vacc[3]);
-    dst[1] = make_uint4(vacc[4], vacc[5], vacc[6], vacc[7]);
-    meta_b[(size_t)col * (I >> 5) + pass] = cacc;
-    if (hw16) scatter_hw(hw16, I >> 7, col, pass, cacc);
-  }
-  if (MODE == 2) {
-    uint4* dst = reinterpret_cast<uint4*>(vals_b + (size_t)col * (I >> 1) + 16 * pass);   // row `col` of the J x I operand
+  if (MODE != 0) {
+    __syncwarp();
+    // row `c` of the J x I operand, the trip's 16-byte units u = 0 .. 8 done / PP - 1: four columns per instruction
+    const int units = done * (8 / PP);
+    const size_t row_words = MODE == 1 ? (size_t)(I >> 2) : (size_t)(I >> 1);
+    const int u = lane & 7;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) dst[q] = make_uint4(dacc[4 * q], dacc[4 * q + 1], dacc[4 * q + 2], dacc[4 * q + 3]);
+    for (int it = 0; it < 8; ++it) {
+      const int c = 4 * it + (lane >> 3);
+      if (u < units)
+        reinterpret_cast<uint4*>(vals_b + (size_t)(32 * cw + c) * row_words + (size_t)pass0 * (MODE == 1 ? 8 : 16))[u] =
+            stage[c * 8 + (u ^ (c & 7))];
+    }
+    if (MODE == 1) {                                        // the trip's index-code words of this lane's column
+      uint32_t* dst = meta_b + (size_t)col * (I >> 5) + pass0;
+      if (done == 4 && (I & 127) == 0) {
+        *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(codes + lane * 4);
+      } else {
+        for (int pp = 0; pp < done; ++pp) dst[pp] = codes[lane * 4 + pp];
+      }
+    }
   }
 }
 
@@ -581,7 +620,8 @@ static int launch_bwd_m(int crit, dim3 grid, int mode, const float* W, const uin
 int launch_bwd_mask_criterion(const float* W, const float* S, const uint32_t* maskbits_f, const int32_t* perm, int I, int J,
                               int N, int M, int crit, uint64_t seed, uint32_t* maskbits_b, uint16_t* vals_b_or_null,
                               uint32_t* meta_b_or_null, int mode, void* hw_meta_or_null, cudaStream_t s) {
-  dim3 grid(I / 32, (J / 32 + 7) / 8);
+  const int trip = mode == 2 ? BwdGenericTrip<2>::PASSES : BwdGenericTrip<1>::PASSES;   // 32-row passes per warp trip
+  dim3 grid((I / 32 + trip - 1) / trip, (J / 32 + 7) / 8);
   uint32_t* v32 = reinterpret_cast<uint32_t*>(vals_b_or_null);
   uint16_t* hw16 = reinterpret_cast<uint16_t*>(hw_meta_or_null);
   if (crit == 3) {
