@@ -100,8 +100,12 @@ __device__ __forceinline__ uint32_t keep_block(const uint32_t (&key)[M], uint32_
 // ---------------------------------------------------------------------------------------
 // MODE 0: mask bits only; 1: 2:4 operand (values + index codes); 2: dense masked bf16 operand
 // (kept weights rounded to bf16, +0 elsewhere) for patterns the 2:4 format cannot hold.
+// (blocks of sixteen weights per lane would take 104-115 registers: two CTAs per SM, a quarter of the warps an SM can
+// hold, for kernels that live on hiding load latency.  Measured at 1:16 on 16384 x 4096: forward mask 168 us
+// unbounded, 131 us at three CTAs per SM, 123 us at four (64 registers, a few dozen bytes of spills); the backward
+// mask is best at three)
 template <int M, int MODE>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)
 fwd_mask_generic_kernel(const float4* __restrict__ W4, long long nblocks, int N,
                         uint32_t* __restrict__ maskbits, uint32_t* __restrict__ vals32,
                         uint32_t* __restrict__ meta, uint16_t* __restrict__ hw16, int jwords) {
@@ -420,7 +424,7 @@ template <int MODE>
 struct BwdGenericTrip { static constexpr int PASSES = MODE == 2 ? 2 : 4; };
 
 template <int M, int MODE, int CRIT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, M == 16 ? 3 : 4)
 bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict__ maskbits_f,
                         const int32_t* __restrict__ perm, int I, int J, int N,
                         uint32_t* __restrict__ maskbits_b, uint32_t* __restrict__ vals_b,
