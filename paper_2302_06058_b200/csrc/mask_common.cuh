@@ -82,10 +82,11 @@ __device__ __forceinline__ uint32_t cvt_bf16x2(float hi, float lo) {
 // The two bf16 slots of a block from its table entry.  Fast path: two packed conversions and
 // one byte permute; a block that holds a NaN takes the exact integer conversion instead so that
 // the NaN payload rule (quiet bit set, sign and top payload bits kept) holds bit for bit.
-template <bool BOTH_KEPT>
+// CHECK_NAN = false: the caller has already established that none of the four is a NaN.
+template <bool BOTH_KEPT, bool CHECK_NAN = true>
 __device__ __forceinline__ uint32_t slots(uint32_t e, float w0, float w1, float w2, float w3,
                                           uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3) {
-  if (max(max(k0, k1), max(k2, k3)) > 0x7F800000u) {
+  if (CHECK_NAN && max(max(k0, k1), max(k2, k3)) > 0x7F800000u) {
     const uint32_t idx0 = (e >> 4) & 3u, idx1 = (e >> 6) & 3u;
     const float s0 = idx0 == 0 ? w0 : idx0 == 1 ? w1 : w2;      // idx0 is never 3
     const float s1 = idx1 == 1 ? w1 : idx1 == 2 ? w2 : w3;      // idx1 is never 0

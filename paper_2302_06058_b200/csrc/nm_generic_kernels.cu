@@ -148,12 +148,25 @@ fwd_mask_generic_kernel(const float4* __restrict__ W4, long long nblocks, int N,
     uint32_t codes = 0;
     if (MODE == 1) {
       uint32_t pv[G];                                     // the block's G packed pairs: one 8- or 16-byte store
+      uint32_t mxk = key[0];
 #pragma unroll
-      for (int g = 0; g < G; ++g) {
-        const uint32_t e = pad16[(kb >> (4 * g)) & 15u];
-        pv[g] = slots<false>(e, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3], key[4 * g], key[4 * g + 1],
-                             key[4 * g + 2], key[4 * g + 3]);
-        codes |= ((e >> 4) & 15u) << (4 * g);
+      for (int m = 1; m < M; ++m) mxk = max(mxk, key[m]);
+      // one NaN test per warp trip instead of a branch per group of four (a NaN takes the exact integer conversion)
+      if (__any_sync(0xFFFFFFFFu, mxk > 0x7F800000u)) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          const uint32_t e = pad16[(kb >> (4 * g)) & 15u];
+          pv[g] = slots<false, true>(e, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3], key[4 * g], key[4 * g + 1],
+                                     key[4 * g + 2], key[4 * g + 3]);
+          codes |= ((e >> 4) & 15u) << (4 * g);
+        }
+      } else {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          const uint32_t e = pad16[(kb >> (4 * g)) & 15u];
+          pv[g] = slots<false, false>(e, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3], 0u, 0u, 0u, 0u);
+          codes |= ((e >> 4) & 15u) << (4 * g);
+        }
       }
       if (live) {
         if (G == 2) reinterpret_cast<uint2*>(vals32)[b] = make_uint2(pv[0], pv[1]);
@@ -492,11 +505,16 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
         }
       }
       if (MODE == 1) {
+        uint32_t mxk = key[0];
+#pragma unroll
+        for (int m = 1; m < M; ++m) mxk = max(mxk, key[m]);
+        const bool nan_here = __any_sync(0xFFFFFFFFu, mxk > 0x7F800000u);   // one test per warp and block row
 #pragma unroll
         for (int g = 0; g < G; ++g) {
           const uint32_t e = pad16[(kb >> (4 * g)) & 15u];
-          vacc[nb * G + g] = slots<false>(e, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3], key[4 * g],
-                                          key[4 * g + 1], key[4 * g + 2], key[4 * g + 3]);
+          vacc[nb * G + g] = nan_here ? slots<false, true>(e, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3], key[4 * g],
+                                                           key[4 * g + 1], key[4 * g + 2], key[4 * g + 3])
+                                      : slots<false, false>(e, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3], 0u, 0u, 0u, 0u);
           cacc |= ((e >> 4) & 15u) << (4 * (nb * G + g));
         }
       }
