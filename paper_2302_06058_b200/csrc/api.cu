@@ -164,10 +164,9 @@ int bimask_sgd_fwd_mask(float* W, const float* dW, float* mom, int I, int J, int
                  "bimask_sgd_fwd_mask: NaN hyper-parameter");
   cudaStream_t s = (cudaStream_t)stream;
   if (M != 4) {
-    if ((rc = launch_sgd_update(W, dW, mom, (long long)I * J, lr, momentum, weight_decay, s)) != BIMASK_OK) return rc;
     const bool gfused = pack && (I % 128 == 0) && (J % 128 == 0);   // unpadded: the mask kernel writes the metadata image
     if ((rc = launch_fwd_mask_generic(W, I, J, N, M, maskbits_f, vals_f, meta_f, pack ? 1 : vals_f ? 2 : 0,
-                                      gfused ? hw_meta_f : nullptr, s)) != BIMASK_OK)
+                                      gfused ? hw_meta_f : nullptr, s, dW, mom, lr, momentum, weight_decay)) != BIMASK_OK)
       return rc;
     return pack && !gfused ? launch_hw_meta(meta_f, I, J, hw_meta_f, s) : BIMASK_OK;
   }

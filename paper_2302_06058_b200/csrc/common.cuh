@@ -146,8 +146,6 @@ int launch_fwd_mask(const float* W, int I, int J, int N, uint32_t* maskbits, uin
 int launch_sgd_fwd_mask(float* W, const float* dW, float* mom_or_null, int I, int J, int N, float lr, float momentum,
                         float weight_decay, uint32_t* maskbits, uint16_t* vals, uint32_t* meta,
                         void* hw_meta_or_null, cudaStream_t s);
-int launch_sgd_update(float* W, const float* dW, float* mom_or_null, long long n, float lr, float momentum,
-                      float weight_decay, cudaStream_t s);
 int launch_hw_meta(const uint32_t* meta, int rows, int K, void* hw_meta, cudaStream_t s);
 // 3x3 convolution, explicit form: x (NHWC) -> column matrix [T][9C]; column-space gradient -> dx (NHWC)
 int launch_im2col3x3(const uint16_t* x, int NB, int H, int W, int C, int stride, uint16_t* cols, cudaStream_t s);
@@ -167,8 +165,11 @@ int launch_pick(const int64_t* counts, const int32_t* cands, int P, int I, int32
                 int32_t* best_perm, cudaStream_t s);
 // N:M patterns with M = 8 or 16 (nm_generic_kernels.cu); vals / meta may be null (mask bits only).
 // mode (generic mask launchers): 0 mask bits only, 1 the 2:4 operand, 2 the dense masked bf16 operand in `vals`
+// dW != nullptr: the optimizer update of Alg. 1 is applied to W (and mom_or_null) as the weights stream through.
 int launch_fwd_mask_generic(const float* W, int I, int J, int N, int M, uint32_t* maskbits, uint16_t* vals_or_null,
-                            uint32_t* meta_or_null, int mode, void* hw_meta_or_null, cudaStream_t s);
+                            uint32_t* meta_or_null, int mode, void* hw_meta_or_null, cudaStream_t s,
+                            const float* dW = nullptr, float* mom_or_null = nullptr, float lr = 0.f, float momentum = 0.f,
+                            float weight_decay = 0.f);
 int launch_score_generic(const uint32_t* bits, const int32_t* cands, int I, int J, int N, int M, int P,
                          int64_t* counts, cudaStream_t s);
 int launch_bwd_mask_generic(const float* W, const uint32_t* maskbits_f, const int32_t* perm, int I, int J, int N, int M,

@@ -115,6 +115,21 @@ __device__ __forceinline__ uint32_t slots_signs(uint32_t e, float w0, float w1, 
   return __byte_perm(cvt_bf16x2(w1, w0), cvt_bf16x2(w3, w2), e) & keep;
 }
 
+// The optimizer update fused into a forward-mask pass (fp32, every operation rounded once, in this order:
+//   g = dW + weight_decay * W ;  mom = momentum * mom + g ;  W = W - lr * mom).
+struct SgdParams {
+  float4* W4;            // read and written
+  const float4* dW4;
+  float4* mom4;          // nullptr: momentum buffer treated as zero and not stored
+  float lr, momentum, weight_decay;
+};
+
+__device__ __forceinline__ float sgd_one(float w, float dw, float& m, const SgdParams& p) {
+  const float g = __fadd_rn(dw, __fmul_rn(p.weight_decay, w));
+  m = __fadd_rn(__fmul_rn(p.momentum, m), g);
+  return __fsub_rn(w, __fmul_rn(p.lr, m));
+}
+
 // Transpose of a 32 x 32 bit matrix held one row per lane (bit b of lane r = element (r, b)): five exchange
 // stages, each swapping the off-diagonal quadrants of every 2s x 2s block; afterwards lane c holds column c.
 __device__ __forceinline__ uint32_t transpose32(uint32_t x, int lane) {

@@ -27,19 +27,6 @@ constexpr int FWD_THREADS = 256;
 // over W.  float32, each product and sum rounded once, in this order (the updated weight decides
 // a mask bit, so the operation order is part of the contract):
 //   g = dW + weight_decay * W ;  mom = momentum * mom + g ;  W = W - lr * mom
-struct SgdParams {
-  float4* W4;            // read and written
-  const float4* dW4;
-  float4* mom4;          // nullptr: momentum buffer treated as zero and not stored
-  float lr, momentum, weight_decay;
-};
-
-__device__ __forceinline__ float sgd_one(float w, float dw, float& m, const SgdParams& p) {
-  const float g = __fadd_rn(dw, __fmul_rn(p.weight_decay, w));
-  m = __fadd_rn(__fmul_rn(p.momentum, m), g);
-  return __fsub_rn(w, __fmul_rn(p.lr, m));
-}
-
 template <bool N_IS_2, bool UPDATE>
 __global__ void __launch_bounds__(FWD_THREADS)
 fwd_mask_pack_kernel(const float4* __restrict__ W4, long long nblk, int N,
@@ -405,37 +392,6 @@ int launch_sgd_fwd_mask(float* W, const float* dW, float* mom, int I, int J, int
   else
     BIMASK_CUDA_OK(launch_pdl(fwd_mask_pack_kernel<false, true>, (unsigned)ctas, FWD_THREADS, 0, s,
         nullptr, nblk, N, maskbits, reinterpret_cast<uint4*>(vals), meta, hw16, J / 32, pad_rows, p));
-  count_launch();
-  BIMASK_CUDA_OK(cudaGetLastError());
-  return BIMASK_OK;
-}
-
-// Plain update pass (same arithmetic), for the patterns whose mask kernel is the generic one.
-__global__ void sgd_update_kernel(long long n4, SgdParams p) {
-  pdl_launch_dependents();
-  pdl_wait();
-  for (long long at = (long long)blockIdx.x * blockDim.x + threadIdx.x; at < n4; at += (long long)gridDim.x * blockDim.x) {
-    float4 w = p.W4[at];
-    const float4 dw = __ldg(p.dW4 + at);
-    float4 m = p.mom4 ? p.mom4[at] : make_float4(0.f, 0.f, 0.f, 0.f);
-    w.x = sgd_one(w.x, dw.x, m.x, p);
-    w.y = sgd_one(w.y, dw.y, m.y, p);
-    w.z = sgd_one(w.z, dw.z, m.z, p);
-    w.w = sgd_one(w.w, dw.w, m.w, p);
-    p.W4[at] = w;
-    if (p.mom4) p.mom4[at] = m;
-  }
-}
-
-int launch_sgd_update(float* W, const float* dW, float* mom, long long n, float lr, float momentum, float weight_decay,
-                      cudaStream_t s) {
-  const long long n4 = n / 4;
-  long long ctas = (n4 + 255) / 256;
-  if (ctas > 148 * 8) ctas = 148 * 8;
-  if (ctas < 1) ctas = 1;
-  const SgdParams p{reinterpret_cast<float4*>(W), reinterpret_cast<const float4*>(dW), reinterpret_cast<float4*>(mom),
-                    lr, momentum, weight_decay};
-  BIMASK_CUDA_OK(launch_pdl(sgd_update_kernel, (unsigned)ctas, 256, 0, s, n4, p));
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;

@@ -104,11 +104,13 @@ __device__ __forceinline__ uint32_t keep_block(const uint32_t (&key)[M], uint32_
 // hold, for kernels that live on hiding load latency.  Measured at 1:16 on 16384 x 4096: forward mask 168 us
 // unbounded, 131 us at three CTAs per SM, 123 us at four (64 registers, a few dozen bytes of spills); the backward
 // mask is best at three)
-template <int M, int MODE>
+// UPDATE: the optimizer update of Alg. 1 applied to the block as it is loaded (W, dW and the momentum buffer are read,
+// W and the momentum buffer written back), so that the next iteration's mask costs no second pass over W.
+template <int M, int MODE, bool UPDATE = false>
 __global__ void __launch_bounds__(256, 4)
 fwd_mask_generic_kernel(const float4* __restrict__ W4, long long nblocks, int N,
                         uint32_t* __restrict__ maskbits, uint32_t* __restrict__ vals32,
-                        uint32_t* __restrict__ meta, uint16_t* __restrict__ hw16, int jwords) {
+                        uint32_t* __restrict__ meta, uint16_t* __restrict__ hw16, int jwords, SgdParams sgd) {
   pdl_launch_dependents();
   pdl_wait();
   constexpr int LPW = 32 / M;                               // lanes per 32-column word
@@ -122,8 +124,8 @@ fwd_mask_generic_kernel(const float4* __restrict__ W4, long long nblocks, int N,
   const long long stride = (long long)gridDim.x * blockDim.x;
   const long long nround = (nblocks + 31) & ~31ll;          // whole warps stay in the loop together
   // the next trip's block is loaded before this trip's is worked on (one block of loads always in flight)
-  float4 nxt[G];
-  {
+  float4 nxt[UPDATE ? 1 : G];
+  if (!UPDATE) {
     const long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x;
 #pragma unroll
     for (int g = 0; g < G; ++g) nxt[g] = b < nblocks ? __ldg(W4 + b * G + g) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -131,12 +133,33 @@ fwd_mask_generic_kernel(const float4* __restrict__ W4, long long nblocks, int N,
   for (long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x; b < nround; b += stride) {
     const bool live = b < nblocks;
     float w[M];
+    if (UPDATE) {
+      // three streams in, two out; no look-ahead (it would triple the registers held across the trip)
+      float4 wv[G], dv[G], mv[G];
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-      const float4 v = nxt[g];
-      w[4 * g] = v.x; w[4 * g + 1] = v.y; w[4 * g + 2] = v.z; w[4 * g + 3] = v.w;
-    }
-    {
+      for (int g = 0; g < G; ++g) {
+        wv[g] = live ? sgd.W4[b * G + g] : make_float4(0.f, 0.f, 0.f, 0.f);
+        dv[g] = live ? __ldg(sgd.dW4 + b * G + g) : make_float4(0.f, 0.f, 0.f, 0.f);
+        mv[g] = (live && sgd.mom4) ? sgd.mom4[b * G + g] : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        wv[g].x = sgd_one(wv[g].x, dv[g].x, mv[g].x, sgd);
+        wv[g].y = sgd_one(wv[g].y, dv[g].y, mv[g].y, sgd);
+        wv[g].z = sgd_one(wv[g].z, dv[g].z, mv[g].z, sgd);
+        wv[g].w = sgd_one(wv[g].w, dv[g].w, mv[g].w, sgd);
+        if (live) {
+          sgd.W4[b * G + g] = wv[g];
+          if (sgd.mom4) sgd.mom4[b * G + g] = mv[g];
+        }
+        w[4 * g] = wv[g].x; w[4 * g + 1] = wv[g].y; w[4 * g + 2] = wv[g].z; w[4 * g + 3] = wv[g].w;
+      }
+    } else {
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const float4 v = nxt[g];
+        w[4 * g] = v.x; w[4 * g + 1] = v.y; w[4 * g + 2] = v.z; w[4 * g + 3] = v.w;
+      }
       const long long bn = b + stride;
 #pragma unroll
       for (int g = 0; g < G; ++g) nxt[g] = bn < nblocks ? __ldg(W4 + bn * G + g) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -561,8 +584,19 @@ bwd_mask_generic_kernel(const float* __restrict__ W, const uint32_t* __restrict_
 BIMASK_DEFINE_DEBUG_COLLECT(debug_collect_generic)
 
 // mode: 0 mask bits only, 1 the 2:4 operand, 2 the dense masked operand (written to `vals`)
+template <int M, bool UPDATE>
+static int launch_fwd_generic_m(int mode, unsigned ctas, cudaStream_t s, const float4* W4, long long nblocks, int N, uint32_t* maskbits,
+                                uint32_t* v32, uint32_t* meta, uint16_t* hw16, int jw, const SgdParams& sgd) {
+  if (mode == 1) BIMASK_CUDA_OK(launch_pdl(fwd_mask_generic_kernel<M, 1, UPDATE>, ctas, 256, 0, s, W4, nblocks, N, maskbits, v32, meta, hw16, jw, sgd));
+  else if (mode == 2) BIMASK_CUDA_OK(launch_pdl(fwd_mask_generic_kernel<M, 2, UPDATE>, ctas, 256, 0, s, W4, nblocks, N, maskbits, v32, meta, hw16, jw, sgd));
+  else BIMASK_CUDA_OK(launch_pdl(fwd_mask_generic_kernel<M, 0, UPDATE>, ctas, 256, 0, s, W4, nblocks, N, maskbits, v32, meta, hw16, jw, sgd));
+  return BIMASK_OK;
+}
+
+// dW != nullptr: the optimizer update (lr, momentum, weight_decay; mom_or_null) is applied to W on the way.
 int launch_fwd_mask_generic(const float* W, int I, int J, int N, int M, uint32_t* maskbits, uint16_t* vals_or_null,
-                            uint32_t* meta_or_null, int mode, void* hw_meta_or_null, cudaStream_t s) {
+                            uint32_t* meta_or_null, int mode, void* hw_meta_or_null, cudaStream_t s, const float* dW,
+                            float* mom_or_null, float lr, float momentum, float weight_decay) {
   uint16_t* hw16 = reinterpret_cast<uint16_t*>(hw_meta_or_null);
   const int jw = J / 32;
   const long long nblocks = (long long)I * J / M;
@@ -570,15 +604,14 @@ int launch_fwd_mask_generic(const float* W, int I, int J, int N, int M, uint32_t
   if (ctas > 148 * 16) ctas = 148 * 16;
   const float4* W4 = reinterpret_cast<const float4*>(W);
   uint32_t* v32 = reinterpret_cast<uint32_t*>(vals_or_null);
-  if (M == 8) {
-    if (mode == 1) BIMASK_CUDA_OK(launch_pdl(fwd_mask_generic_kernel<8, 1>, (unsigned)ctas, 256, 0, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw));
-    else if (mode == 2) BIMASK_CUDA_OK(launch_pdl(fwd_mask_generic_kernel<8, 2>, (unsigned)ctas, 256, 0, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw));
-    else BIMASK_CUDA_OK(launch_pdl(fwd_mask_generic_kernel<8, 0>, (unsigned)ctas, 256, 0, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw));
-  } else {
-    if (mode == 1) BIMASK_CUDA_OK(launch_pdl(fwd_mask_generic_kernel<16, 1>, (unsigned)ctas, 256, 0, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw));
-    else if (mode == 2) BIMASK_CUDA_OK(launch_pdl(fwd_mask_generic_kernel<16, 2>, (unsigned)ctas, 256, 0, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw));
-    else BIMASK_CUDA_OK(launch_pdl(fwd_mask_generic_kernel<16, 0>, (unsigned)ctas, 256, 0, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw));
-  }
+  const SgdParams sgd{reinterpret_cast<float4*>(const_cast<float*>(W)), reinterpret_cast<const float4*>(dW),
+                      reinterpret_cast<float4*>(mom_or_null), lr, momentum, weight_decay};
+  int rc;
+  if (dW) rc = M == 8 ? launch_fwd_generic_m<8, true>(mode, (unsigned)ctas, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw, sgd)
+                      : launch_fwd_generic_m<16, true>(mode, (unsigned)ctas, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw, sgd);
+  else rc = M == 8 ? launch_fwd_generic_m<8, false>(mode, (unsigned)ctas, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw, sgd)
+                   : launch_fwd_generic_m<16, false>(mode, (unsigned)ctas, s, W4, nblocks, N, maskbits, v32, meta_or_null, hw16, jw, sgd);
+  if (rc != BIMASK_OK) return rc;
   count_launch();
   BIMASK_CUDA_OK(cudaGetLastError());
   return BIMASK_OK;
