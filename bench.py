@@ -484,7 +484,8 @@ def run_gpu(args):
     #      peaks (burst: a kernel timed alone at full clock; sustained: inside a long run under the power cap) and
     #      `frac` is the one that matches the clocks sampled while the calls were timed. ----
     regime = clock_regime(clocks, step_ms_total * 1e-3)
-    regime_calls = clock_regime(clocks_calls)
+    # (a per-call loop too short for the sampler to catch takes the regime of the timed run just before it)
+    regime_calls = clock_regime(clocks_calls) if clocks_calls.get("samples") else regime
     kernels = []
     for li, (L, b, _) in enumerate(layers):
         work = algorithmic_work(L, cfg.P)
