@@ -422,6 +422,7 @@ def run_gpu(args):
     acc = {li: {n: 0.0 for n in names} for li in range(len(layers))}
     time.sleep(1.0)      # an idle second: the breakdown starts from the same power state as the headline's timed region
     t_call_begin = time.time()
+    all_evs = []
     for _ in range(args.steps):
         evs = []
         for li, (L, b, _) in enumerate(layers):
@@ -444,11 +445,15 @@ def run_gpu(args):
             bm.bimask_wgrad(b["dY"], b["X"], L.T, L.I, L.J, b["dW"], b["ws"], wsb, b["status_word"])
             ev[6].record(stream)
             evs.append(ev)
-        torch.cuda.synchronize()                          # once per pass: the calls of a pass run back to back
-        for li, ev in enumerate(evs):
-            for k, n in enumerate(names):
-                acc[li][n] += ev[k].elapsed_time(ev[k + 1])
+        all_evs.append(evs)
+    torch.cuda.synchronize()      # once, after the last pass: every call follows the one before it as in the timed step
     t_call_end = time.time()
+    # per call the MEDIAN over the passes, times the number of passes (the first call after the idle second starts on an
+    # idle GPU and would carry its launch latency into a mean)
+    for li in range(len(layers)):
+        for k, n in enumerate(names):
+            per_pass = sorted(evs[li][k].elapsed_time(evs[li][k + 1]) for evs in all_evs)
+            acc[li][n] = per_pass[len(per_pass) // 2] * args.steps
 
     # ---- the same step repeated back to back for --sustain-s seconds: the figure under the power cap ----
     sustain_ms, sustain_steps, t_sus_begin, t_sus_end = 0.0, 0, None, None
