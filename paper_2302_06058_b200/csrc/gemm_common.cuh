@@ -108,7 +108,7 @@ struct GemmParams {
   int k_tiles_per_split;    // dense split-K: k tiles handled by one blockIdx.z
   int tiles_m, tiles_n;     // output tiles (CTA pairs along M for the pair kernel)
   int raster_group;         // tiles walked along M before advancing along N
-  int n_tile;               // pair kernel: output columns per tile (multiple of 16, <= 256)
+  int n_tile;               // pair kernel: output columns per tile (multiple of 32, <= 256)
   void* out;                // sparse: bf16 [Ndim][Mdim];  dense: fp32 [split][Mdim][Ndim]
   int32_t* status_word;
 };

@@ -416,7 +416,7 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
       ptx::tc_fence_after();
       const uint32_t acc = tmem_base + 256u * buf + ((uint32_t)(32 * q) << 16);
       const uint32_t release_bar = ptx::mapa(tmem_empty_bar(buf), 0);
-      const int nchunks = (CONV || (SP_N & 31) == 0) ? SP_N / 32 : SP_N / 16;
+      const int nchunks = SP_N / 32;                        // the hosts pick multiples of 32
       if (CONV) {
         // accumulator columns [0, SP_N/2) are the pixels of box 2*tile_n, the rest those of box 2*tile_n + 1
         drain_chunks<32>(acc, eg, EPI_GROUPS, nchunks, false, release_bar, stg, 1 + eg, q, lane, p.Mdim - m0,
@@ -431,16 +431,10 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
           if (w >= p.conv.W || h >= p.conv.H || n >= p.conv.NB) return nullptr;
           return outp + conv_out_pixel(p.conv, n, h, w) * p.Mdim + m0;
         });
-      } else if ((SP_N & 31) == 0) {
-        if (!drain_chunks_tma<32, C::EPI_NT>(acc, eg, EPI_GROUPS, nchunks, false, release_bar, stg, ebars, u, q, lane, abort_flag)) {
-          *abort_flag = 1;
-          break;
-        }
-      } else {
-        if (!drain_chunks_tma<16, C::EPI_NT>(acc, eg, EPI_GROUPS, nchunks, false, release_bar, stg, ebars, u, q, lane, abort_flag)) {
-          *abort_flag = 1;
-          break;
-        }
+      } else if (!drain_chunks_tma<32, C::EPI_NT>(acc, eg, EPI_GROUPS, nchunks, false, release_bar, stg, ebars, u, q, lane,
+                                                  abort_flag)) {
+        *abort_flag = 1;
+        break;
       }
     }
   } else if (!CONV) {
@@ -454,10 +448,10 @@ spmm_pair_persistent_kernel(const __grid_constant__ CUtensorMap tmapA, const __g
         int tile_m, tile_n;
         raster(tile, p.tiles_m, p.tiles_n, p.raster_group, tile_m, tile_n);
         const int m0 = (2 * tile_m + (int)rank) * 128, n0 = tile_n * SP_N;
-        const bool ok = (SP_N & 31) == 0
-            ? store_chunks<32, C::EPI_NT>(&tmapD, g, EPI_GROUPS, SP_N / 32, stg, ebars, u, m0, n0, p.Mdim, p.Ndim, abort_flag)
-            : store_chunks<16, C::EPI_NT>(&tmapD, g, EPI_GROUPS, SP_N / 16, stg, ebars, u, m0, n0, p.Mdim, p.Ndim, abort_flag);
-        if (!ok) { *abort_flag = 1; break; }
+        if (!store_chunks<32, C::EPI_NT>(&tmapD, g, EPI_GROUPS, SP_N / 32, stg, ebars, u, m0, n0, p.Mdim, p.Ndim, abort_flag)) {
+          *abort_flag = 1;
+          break;
+        }
       }
       store_finish();
     }
@@ -760,7 +754,7 @@ int run_sparse_pair_persistent(const uint16_t* vals, const void* hw_meta, const 
   if ((rc = make_tmap(&ta, vals, (uint64_t)Kdim / 2, (uint64_t)Mdim, 128)) != BIMASK_OK) return rc;
   if ((rc = make_tmap(&tb, Bop, (uint64_t)Kdim, (uint64_t)Ndim, n_tile / 2)) != BIMASK_OK) return rc;
   if ((rc = make_tmap_meta(&te, hw_meta, (uint64_t)tiles_m * tiles_k)) != BIMASK_OK) return rc;
-  if ((rc = make_tmap(&td, out, (uint64_t)Mdim, (uint64_t)Ndim, n_tile % 32 == 0 ? 32 : 16)) != BIMASK_OK) return rc;   // one chunk of the drain
+  if ((rc = make_tmap(&td, out, (uint64_t)Mdim, (uint64_t)Ndim, 32)) != BIMASK_OK) return rc;   // one chunk of the drain: 32 tokens x 64 rows per store
   auto kern = spmm_pair_persistent_kernel<STAGES, false>;
   if ((rc = set_smem_attr(kern, C::SMEM_BYTES)) != BIMASK_OK) return rc;
   GemmParams p;
