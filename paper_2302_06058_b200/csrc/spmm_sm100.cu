@@ -220,12 +220,13 @@ spmm_single_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_const
 
 // ------------------------------------------------------------------------------------------
 // Persistent CTA-pair 2:4 product.  One pair per two SMs walks 256 x N output tiles in raster
-// order.  With N <= 240 tensor memory holds TWO accumulators (columns 0.. and 256..) plus the
-// four metadata columns (496..499), so the epilogue of one tile overlaps the main loop of the
+// order.  With N <= 224 (a multiple of 32) tensor memory holds TWO accumulators (columns 0.. and 256..)
+// plus the four metadata columns (496..499), so the epilogue of one tile overlaps the main loop of the
 // next; N = 256 leaves room for one accumulator only (metadata at 256..259) and is used when the
 // tile count would otherwise round up to an extra pass over the SMs (the host picks N).  The TMA
 // producer runs ahead across tile boundaries; two groups of four epilogue warps drain an accumulator
-// in chunks of 32 (16) columns, taking chunks in turn (see drain_chunks).
+// in chunks of 32 columns, taking chunks in turn, and a store warp per group sends the staged chunks
+// off as tensor stores (see drain_chunks_tma / store_chunks).
 // ------------------------------------------------------------------------------------------
 
 
