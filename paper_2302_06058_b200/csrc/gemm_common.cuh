@@ -127,7 +127,9 @@ __device__ __forceinline__ void raster(int id, int tiles_m, int tiles_n, int gro
   tn = in / gsize;
 }
 
-// Epilogue of the 2:4 products.  The accumulator holds D[row][token] (row = tensor-memory lane), the result is
+// Epilogue of the 2:4 products, form with per-lane global stores (used where a token's address is not affine in
+// its index: the pixel boxes of the implicit convolution; drain_chunks_tma below is the form for plain matrices).
+// The accumulator holds D[row][token] (row = tensor-memory lane), the result is
 // stored token-major, so a chunk of W tokens x the CTA's 128 rows is transposed on its way out by a GROUP of four
 // warps, one per tensor-memory lane quadrant:
 //   tensor memory -> registers in the accumulator-fragment layout (two 16-lane loads per warp) -> bf16 pairs ->

@@ -6,8 +6,10 @@
 // All kernels are warp-specialised: a TMA producer thread fills a ring of shared-memory stages
 // (operands in the 128-byte-swizzled layouts the tensor core reads directly), one thread issues
 // tcgen05.mma.sp (the index metadata of the 2:4 operand is copied shared -> tensor memory with
-// tcgen05.cp right before the MMAs that use it), accumulators live in tensor memory, and eight
-// epilogue warps drain them (drain_chunks in gemm_common.cuh).  The large-shape kernels
+// tcgen05.cp right before the MMAs that use it), accumulators live in tensor memory, eight
+// epilogue warps drain them into swizzled staging tiles and two store warps send those off as
+// tensor stores (drain_chunks_tma / store_chunks in gemm_common.cuh; the implicit convolution,
+// whose tokens are pixels, writes from the draining warps: drain_chunks).  The large-shape kernels
 // (spmm_pair2m_kernel, spmm_pair_persistent_kernel) run CTA pairs persistently; spmm_single_kernel
 // is the one-CTA-per-tile form for operands of at most 128 rows or at most 128 tokens, and also
 // takes a dense A operand (masked weights of a pattern the 2:4 format cannot hold).
